@@ -1,0 +1,187 @@
+/*
+ * imm.h -- C ABI of the B200 (sm_100a) prover for sumcheck proofs of int8 matrix products
+ * over the Goldilocks field p = 2^64 - 2^32 + 1.
+ *
+ * Background.  The audited-inference protocol this library serves has the server prove, for an
+ * audited request, that the "continuous transformations" of the reference model -- its
+ * attention and MLP matrix products -- were computed as claimed (paper Section 5.2, item 2;
+ * Algorithm 3, the F_theta* step), through a verifiable-computation pair (Prove, Vrfy)
+ * (Section 2.2).  The paper leaves the proof system open.  This library instantiates it for one
+ * claimed product C = A*B of int8 matrices (C int32) with the classic sumcheck over
+ *     sum_y A~(r_row, y) * B~(y, r_col) = C~(r_row, r_col),
+ * where M~ is the multilinear extension of M lifted into the field.
+ *
+ * Conventions
+ *   - imm_fe is a canonical field element: a uint64 in [0, p).  Inputs must be canonical;
+ *     outputs are.
+ *   - lift(v) of a signed integer v is v mod p.
+ *   - An index of n bits has variables z_0..z_{n-1}, z_0 the MOST significant bit;
+ *     eq(r, i) = prod_t (bit_t(i) ? r_t : 1 - r_t).
+ *   - A dimension d is zero-padded (implicitly) at the high end to 2^ceil(log2 d).
+ *   - Challenges are public coins of an interactive verifier, drawn from a counter-based
+ *     generator (SplitMix64 mixer) keyed by (seed, proof_id); they do not depend on the
+ *     prover's messages.  domain 1 = r_row, 2 = r_col, 3 = sumcheck rounds.
+ *   - Transcript of one proof: [c0, g_0(0), g_0(1), g_0(2), ..., g_{b-1}(0), g_{b-1}(1),
+ *     g_{b-1}(2), a_fin, b_fin], b = ceil(log2 k), 3b+3 words.
+ *
+ * General rules
+ *   - Every call returns an int status (IMM_OK or a negative IMM_ERR_*; imm_sumcheck_verify may
+ *     also return IMM_REJECT).  Nothing throws or aborts across this boundary.
+ *   - The caller owns every buffer.  The library allocates no device memory: scratch comes from
+ *     a caller-provided device workspace whose size a query call returns.  Workspace and output
+ *     pointers must be 16-byte aligned.
+ *   - Pointers named d_* are DEVICE pointers, *_host are HOST pointers.
+ *   - Device calls enqueue work on the given CUDA stream (a cudaStream_t passed as void*; NULL =
+ *     the legacy default stream) and return without synchronising, unless stated otherwise.
+ *     Host descriptor arrays are read before the call returns.
+ *   - Matrices are row-major with a leading dimension ld in ELEMENTS (ld >= cols).  Rows that
+ *     are 16-byte aligned (base pointer and ld*sizeof(element) multiples of 16) take the
+ *     vectorised kernels; anything else takes an element-wise path with the same results.
+ *   - Limits: 1 <= rows, cols <= 2^20 for the matrix calls; for proofs 1 <= m, n <= 2^20 and
+ *     1 <= k <= 2^17.  A zero extent is IMM_ERR_SHAPE.
+ *   - There is no CPU fallback: without a CUDA device every device call returns IMM_ERR_CUDA.
+ */
+#ifndef IMM_H_
+#define IMM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef uint64_t imm_fe;
+
+#define IMM_P 0xFFFFFFFF00000001ULL
+
+enum {
+    IMM_OK = 0,
+    IMM_REJECT = 1,              /* imm_sumcheck_verify only: the proof is rejected        */
+    IMM_ERR_ARG = -1,            /* null pointer, bad enum value, negative count           */
+    IMM_ERR_SHAPE = -2,          /* zero or too large extent, ld < cols                    */
+    IMM_ERR_ALIGN = -3,          /* workspace / output pointer not 16-byte aligned         */
+    IMM_ERR_WORKSPACE = -4,      /* workspace smaller than the query call asks for         */
+    IMM_ERR_NONCANONICAL = -5,   /* a field element >= p on input                          */
+    IMM_ERR_CUDA = -6            /* a CUDA runtime call failed (see imm_last_cuda_error)   */
+};
+enum { IMM_I8 = 0, IMM_I32 = 1 };
+enum { IMM_BIND_ROWS = 0, IMM_BIND_COLS = 1 };
+enum { IMM_FIELD_ADD = 0, IMM_FIELD_SUB = 1, IMM_FIELD_MUL = 2 };
+
+/* Library version (major*100 + minor). */
+int imm_version(void);
+
+/* Text of the last CUDA runtime error seen by the calling thread's device calls ("" if none).
+ * The pointer stays valid until the thread's next failing call. */
+const char* imm_last_cuda_error(void);
+
+/* HOST.  Challenge `index` of `domain` (1 = r_row, 2 = r_col, 3 = sumcheck round) for
+ * (seed, proof_id): canon(mix64(key + G*(ctr+1))) with key = mix64(mix64(seed+G) + G*(proof_id+1)),
+ * ctr = domain<<32 | index, G = 0x9E3779B97F4A7C15, canon(x) = x >= p ? x-p : x.  These are the
+ * verifier's public coins (Section 2.2's Vrfy side). */
+imm_fe imm_challenge(uint64_t seed, uint64_t proof_id, uint32_t domain, uint32_t index);
+
+/* Element-wise field arithmetic on device arrays: d_out[i] = d_x[i] (op) d_y[i], i < count.
+ * Exists so the device field arithmetic can be tested in isolation.  Inputs must be canonical
+ * (not checked).  count == 0 is a no-op. */
+int imm_field_binop(int op, const imm_fe* d_x, const imm_fe* d_y, imm_fe* d_out, int64_t count,
+                    void* stream);
+
+/* eq table (the Lagrange basis of the Boolean cube at r; multilinear-extension definition
+ * used by every step of the proof).  d_out[i] = eq(r, i) for i < 2^nvars.
+ *   r_host : HOST array of nvars canonical field elements (read before return)
+ *   nvars  : 0..20
+ *   d_out  : DEVICE array of 2^nvars elements, 16-byte aligned
+ * Errors: IMM_ERR_ARG, IMM_ERR_SHAPE (nvars out of range), IMM_ERR_NONCANONICAL, IMM_ERR_ALIGN. */
+int imm_eq_table(const imm_fe* r_host, int nvars, imm_fe* d_out, void* stream);
+
+/* Workspace bytes needed by imm_mle_partial_eval / imm_mle_eval_point for this matrix. */
+size_t imm_mle_workspace(int dtype, int64_t rows, int64_t cols, int bind);
+
+/* Partial evaluation of a matrix's multilinear extension: binds one index with an eq table.
+ *   IMM_BIND_ROWS: d_out[y] = sum_{i<rows} d_eq[i] * lift(M[i,y]),  y < cols  (A~(r_row, .))
+ *   IMM_BIND_COLS: d_out[i] = sum_{j<cols} lift(M[i,j]) * d_eq[j],  i < rows  (B~(., r_col))
+ *   d_mat   : DEVICE matrix, dtype IMM_I8 (int8) or IMM_I32 (int32), rows x cols, leading dim ld
+ *   d_eq    : DEVICE eq table with at least rows (BIND_ROWS) / cols (BIND_COLS) entries; entries
+ *             past the real extent are ignored, which is the implicit zero padding
+ *   d_out   : DEVICE array of cols (BIND_ROWS) / rows (BIND_COLS) elements
+ *   d_ws    : DEVICE workspace of at least imm_mle_workspace(dtype, rows, cols, bind) bytes
+ * Errors: IMM_ERR_ARG, IMM_ERR_SHAPE, IMM_ERR_ALIGN, IMM_ERR_WORKSPACE, IMM_ERR_CUDA. */
+int imm_mle_partial_eval(const void* d_mat, int dtype, int64_t rows, int64_t cols, int64_t ld,
+                         int bind, const imm_fe* d_eq, imm_fe* d_out,
+                         void* d_ws, size_t ws_bytes, void* stream);
+
+/* Full evaluation at a point given as two eq tables (the verifier's claim C~(r_row, r_col), and
+ * the checks of a_fin, b_fin):  d_out[0] = sum_{i,j} d_eq_row[i] * lift(M[i,j]) * d_eq_col[j].
+ * Workspace: imm_mle_workspace(dtype, rows, cols, IMM_BIND_ROWS) bytes.  Same errors. */
+int imm_mle_eval_point(const void* d_mat, int dtype, int64_t rows, int64_t cols, int64_t ld,
+                       const imm_fe* d_eq_row, const imm_fe* d_eq_col, imm_fe* d_out,
+                       void* d_ws, size_t ws_bytes, void* stream);
+
+/* One claimed product C = A*B.  A: m x k int8, B: k x n int8, C: m x n int32 -- the CLAIMED
+ * matrix, used as given (the prover never recomputes A*B).  DEVICE pointers for
+ * imm_sumcheck_matmul_prove, HOST pointers for imm_sumcheck_matmul_prove_host. */
+typedef struct {
+    const int8_t* A;
+    const int8_t* B;
+    const int32_t* C;
+    int64_t m, k, n;
+    int64_t lda, ldb, ldc;      /* leading dimensions in elements */
+    uint64_t proof_id;
+} imm_matmul_desc;
+
+/* Workspace bytes imm_sumcheck_matmul_prove needs for this batch (0 on invalid input). */
+size_t imm_sumcheck_matmul_workspace(const imm_matmul_desc* descs_host, int nproofs);
+
+/* Prover (Prove of Section 2.2, for the matrix products of Algorithm 3's F_theta* step).  For
+ * every proof of the batch: derives r_row, r_col, r_k from (seed, proof_id); builds both eq
+ * tables; evaluates avec = A~(r_row, .), bvec = B~(., r_col) and c0 = C~(r_row, r_col); runs
+ * the ceil(log2 k) sumcheck rounds (each round's g(0), g(1), g(2), then the fold of both
+ * tables with that round's challenge); writes the transcript.
+ *   descs_host    : HOST array of nproofs descriptors with DEVICE matrix pointers
+ *   d_transcripts : DEVICE array, nproofs rows of `stride` words, stride >= 3*ceil(log2(max k))+3;
+ *                   row p holds proof p's transcript, words past its length are set to zero
+ *   d_status      : DEVICE array of nproofs int32, set to IMM_OK per proof (reserved for
+ *                   device-detected conditions)
+ *   d_ws          : DEVICE workspace, >= imm_sumcheck_matmul_workspace(...) bytes
+ * The whole batch is a fixed sequence of kernel launches on `stream`; results are valid once
+ * the stream has been synchronised.
+ * Errors: IMM_ERR_ARG, IMM_ERR_SHAPE, IMM_ERR_ALIGN, IMM_ERR_WORKSPACE, IMM_ERR_CUDA. */
+int imm_sumcheck_matmul_prove(const imm_matmul_desc* descs_host, int nproofs, uint64_t seed,
+                              imm_fe* d_transcripts, int64_t stride, int32_t* d_status,
+                              void* d_ws, size_t ws_bytes, void* stream);
+
+/* Device arena bytes imm_sumcheck_matmul_prove_host needs: staged copies of all matrices, the
+ * transcripts and status words, and the prover workspace (0 on invalid input). */
+size_t imm_sumcheck_matmul_host_arena(const imm_matmul_desc* descs_host, int nproofs);
+
+/* End-to-end variant with HOST matrices: copies every A, B, C to the device arena, proves,
+ * copies transcripts and status back, and SYNCHRONISES the stream before returning.
+ *   descs_host       : HOST descriptors with HOST matrix pointers (pinned memory copies fastest)
+ *   transcripts_host : HOST array, nproofs x stride words
+ *   status_host      : HOST array of nproofs int32
+ *   d_arena          : DEVICE arena of >= imm_sumcheck_matmul_host_arena(...) bytes, 256-byte aligned
+ * Same errors as imm_sumcheck_matmul_prove. */
+int imm_sumcheck_matmul_prove_host(const imm_matmul_desc* descs_host, int nproofs, uint64_t seed,
+                                   imm_fe* transcripts_host, int64_t stride, int32_t* status_host,
+                                   void* d_arena, size_t arena_bytes, void* stream);
+
+/* HOST verifier (Vrfy of Section 2.2).  claim <- c0; for each round j require
+ * g_j(0) + g_j(1) = claim and set claim <- g_j(r_j) by interpolation on the nodes {0,1,2};
+ * finally require claim = a_fin * b_fin.  When an expect_* pointer is non-NULL the
+ * corresponding transcript word must also equal the pointed-to value (the verifier's own
+ * evaluation of C~, A~ or B~).
+ *   transcript_host : HOST array of 3*nrounds+3 canonical words
+ *   fail_at         : HOST out.  -1 accepted; j in [0,nrounds) = round j's sum check failed;
+ *                     nrounds = final product check failed; nrounds+1 / +2 / +3 = c0 / a_fin /
+ *                     b_fin differs from the expected value
+ * Returns IMM_OK, IMM_REJECT, IMM_ERR_ARG or IMM_ERR_NONCANONICAL. */
+int imm_sumcheck_verify(const imm_fe* transcript_host, int nrounds, uint64_t seed,
+                        uint64_t proof_id, const imm_fe* expect_c0, const imm_fe* expect_a_fin,
+                        const imm_fe* expect_b_fin, int* fail_at);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* IMM_H_ */

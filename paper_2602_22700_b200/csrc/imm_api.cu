@@ -1,0 +1,527 @@
+// C ABI of libimm: argument validation, workspace planning and launch sequencing.
+// All arithmetic on matrix data happens in the kernels (imm_kernels.cu); the only field
+// arithmetic done on the host is the verifier, which is host-side by definition.
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <string>
+#include <vector>
+
+#include "../../include/imm.h"
+#include "gl64.cuh"
+#include "imm_kernels.h"
+#include "imm_plan.h"
+
+namespace {
+
+using namespace imm;
+
+thread_local std::string g_cuda_err;
+
+int cuda_fail(cudaError_t e)
+{
+    g_cuda_err = std::string(cudaGetErrorName(e)) + ": " + cudaGetErrorString(e);
+    return IMM_ERR_CUDA;
+}
+#define CU(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) return cuda_fail(e_); } while (0)
+
+constexpr int64_t MAX_EXTENT = (int64_t)1 << 20;
+constexpr int64_t MAX_K = (int64_t)1 << MAX_K_VARS;
+constexpr size_t ALIGN = 256;
+
+size_t align_up(size_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
+
+int ceil_log2(int64_t d)
+{
+    int n = 0;
+    while (((int64_t)1 << n) < d) n++;
+    return n;
+}
+
+size_t elem_size(int dtype) { return dtype == IMM_I8 ? 1 : 4; }
+
+bool rows_vectorisable(const void* p, int64_t ld, int dtype)
+{
+    return ((uintptr_t)p % 16 == 0) && ((ld * (int64_t)elem_size(dtype)) % 16 == 0);
+}
+
+int env_int(const char* name, int dflt)
+{
+    const char* s = getenv(name);
+    if (!s || !*s) return dflt;
+    int v = atoi(s);
+    return v > 0 ? v : dflt;
+}
+
+// Columns per tile of each kernel family.
+int rowbind_cols(int dtype) { return ROWBIND_THREADS * (dtype == IMM_I8 ? 16 : 4); }
+int colbind_cols(int dtype) { return COLBIND_VECS * (dtype == IMM_I8 ? 16 : 4); }
+
+struct Shape { int64_t rows, cols; };
+
+// Rows per tile: the largest candidate that still yields enough tiles to fill the GPU several
+// times over (the tail of the last wave is then a small fraction of the launch).
+int pick_tile_rows(const std::vector<Shape>& mats, int cols_per_tile, const char* env_name)
+{
+    const int forced = env_int(env_name, 0);
+    if (forced) {
+        int v = forced < 32 ? 32 : forced > MAX_TILE_ROWS ? MAX_TILE_ROWS : forced;
+        return v / 32 * 32;
+    }
+    const int64_t target = (int64_t)148 * env_int("IMM_TILES_PER_SM", 24);
+    const int cand[] = {1024, 512, 256, 128, 64, 32};
+    for (int c : cand) {
+        int64_t tiles = 0;
+        for (const Shape& s : mats)
+            tiles += ((s.rows + c - 1) / c) * ((s.cols + cols_per_tile - 1) / cols_per_tile);
+        if (tiles >= target) return c;
+    }
+    return 32;
+}
+
+void fill_job(MatJob& j, const void* mat, int dtype, int64_t rows, int64_t cols, int64_t ld,
+              int tile_rows, int cols_per_tile)
+{
+    memset(&j, 0, sizeof(j));
+    j.mat = mat;
+    j.ld = ld;
+    j.rows = (int32_t)rows;
+    j.cols = (int32_t)cols;
+    j.tile_rows = tile_rows;
+    j.nrb = (int32_t)((rows + tile_rows - 1) / tile_rows);
+    j.ncc = (int32_t)((cols + cols_per_tile - 1) / cols_per_tile);
+    j.vec = rows_vectorisable(mat, ld, dtype) ? 1 : 0;
+}
+
+int check_matrix_args(const void* d_mat, int dtype, int64_t rows, int64_t cols, int64_t ld)
+{
+    if (!d_mat || (dtype != IMM_I8 && dtype != IMM_I32)) return IMM_ERR_ARG;
+    if (rows <= 0 || cols <= 0 || rows > MAX_EXTENT || cols > MAX_EXTENT || ld < cols) return IMM_ERR_SHAPE;
+    return IMM_OK;
+}
+
+// ------------------------------------------------------------------ batch plan ------------
+
+struct Plan {
+    int status = IMM_OK;
+    int nproofs = 0;
+    int max_b = 0;
+    int rows_a = 0, rows_b = 0, rows_c = 0;
+    uint32_t tiles_a = 0, tiles_b = 0, tiles_c = 0;
+    // byte offsets from the workspace base
+    size_t off_proofs = 0, off_jobs_a = 0, off_jobs_b = 0, off_jobs_c = 0, off_eq = 0, header_bytes = 0;
+    struct PerProof {
+        size_t e_row, e_col, part_a, part_b, part_c, tab;
+        int a, b, c, n_part_a, n_part_b, n_part_c;
+    };
+    std::vector<PerProof> pp;
+    size_t total_bytes = 0;
+};
+
+int check_desc(const imm_matmul_desc& d)
+{
+    if (!d.A || !d.B || !d.C) return IMM_ERR_ARG;
+    if (d.m <= 0 || d.k <= 0 || d.n <= 0 || d.m > MAX_EXTENT || d.n > MAX_EXTENT || d.k > MAX_K)
+        return IMM_ERR_SHAPE;
+    if (d.lda < d.k || d.ldb < d.n || d.ldc < d.n) return IMM_ERR_SHAPE;
+    return IMM_OK;
+}
+
+Plan make_plan(const imm_matmul_desc* descs, int nproofs)
+{
+    Plan p;
+    if (!descs || nproofs <= 0) { p.status = IMM_ERR_ARG; return p; }
+    p.nproofs = nproofs;
+    std::vector<Shape> sa, sb, sc;
+    for (int i = 0; i < nproofs; i++) {
+        int rc = check_desc(descs[i]);
+        if (rc != IMM_OK) { p.status = rc; return p; }
+        sa.push_back({descs[i].m, descs[i].k});
+        sb.push_back({descs[i].k, descs[i].n});
+        sc.push_back({descs[i].m, descs[i].n});
+    }
+    p.rows_a = pick_tile_rows(sa, rowbind_cols(IMM_I8), "IMM_TILE_ROWS_A");
+    p.rows_b = pick_tile_rows(sb, colbind_cols(IMM_I8), "IMM_TILE_ROWS_B");
+    p.rows_c = pick_tile_rows(sc, rowbind_cols(IMM_I32), "IMM_TILE_ROWS_C");
+
+    size_t off = 0;
+    p.off_proofs = off; off = align_up(off + sizeof(ProofDev) * nproofs);
+    p.off_jobs_a = off; off = align_up(off + sizeof(MatJob) * nproofs);
+    p.off_jobs_b = off; off = align_up(off + sizeof(MatJob) * nproofs);
+    p.off_jobs_c = off; off = align_up(off + sizeof(MatJob) * nproofs);
+    p.off_eq = off;     off = align_up(off + sizeof(EqTask) * 2 * nproofs);
+    p.header_bytes = off;
+
+    uint64_t ta = 0, tb = 0, tc = 0;
+    p.pp.resize(nproofs);
+    for (int i = 0; i < nproofs; i++) {
+        const imm_matmul_desc& d = descs[i];
+        Plan::PerProof& q = p.pp[i];
+        q.a = ceil_log2(d.m); q.b = ceil_log2(d.k); q.c = ceil_log2(d.n);
+        if (q.b > p.max_b) p.max_b = q.b;
+        q.n_part_a = (int)((d.m + p.rows_a - 1) / p.rows_a);
+        q.n_part_b = (int)((d.n + colbind_cols(IMM_I8) - 1) / colbind_cols(IMM_I8));
+        const int64_t c_nrb = (d.m + p.rows_c - 1) / p.rows_c;
+        const int64_t c_ncc = (d.n + rowbind_cols(IMM_I32) - 1) / rowbind_cols(IMM_I32);
+        q.n_part_c = (int)(c_nrb * c_ncc);
+        q.e_row = off;  off = align_up(off + sizeof(imm_fe) * ((size_t)1 << q.a));
+        q.e_col = off;  off = align_up(off + sizeof(imm_fe) * ((size_t)1 << q.c));
+        q.part_a = off; off = align_up(off + sizeof(imm_fe) * (size_t)q.n_part_a * d.k);
+        q.part_b = off; off = align_up(off + sizeof(imm_fe) * (size_t)q.n_part_b * d.k);
+        q.part_c = off; off = align_up(off + sizeof(imm_fe) * (size_t)q.n_part_c);
+        q.tab = off;    off = align_up(off + sizeof(imm_fe) * 2 * ((size_t)1 << q.b));
+        ta += (uint64_t)q.n_part_a * ((d.k + rowbind_cols(IMM_I8) - 1) / rowbind_cols(IMM_I8));
+        tb += (uint64_t)((d.k + p.rows_b - 1) / p.rows_b) * q.n_part_b;
+        tc += (uint64_t)q.n_part_c;
+    }
+    if (ta > 0x7FFFFFFFu || tb > 0x7FFFFFFFu || tc > 0x7FFFFFFFu) { p.status = IMM_ERR_SHAPE; return p; }
+    p.tiles_a = (uint32_t)ta; p.tiles_b = (uint32_t)tb; p.tiles_c = (uint32_t)tc;
+    p.total_bytes = off;
+    return p;
+}
+
+int check_stride(const imm_matmul_desc* descs, int nproofs, int64_t stride)
+{
+    for (int i = 0; i < nproofs; i++)
+        if (stride < 3 * ceil_log2(descs[i].k) + 3) return IMM_ERR_SHAPE;
+    return IMM_OK;
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------------------------------------
+// exported functions
+// ---------------------------------------------------------------------------------------------
+
+extern "C" {
+
+int imm_version(void) { return 100; }
+
+const char* imm_last_cuda_error(void) { return g_cuda_err.c_str(); }
+
+imm_fe imm_challenge(uint64_t seed, uint64_t proof_id, uint32_t domain, uint32_t index)
+{
+    return gl::challenge(seed, proof_id, domain, index);
+}
+
+int imm_field_binop(int op, const imm_fe* d_x, const imm_fe* d_y, imm_fe* d_out, int64_t count,
+                    void* stream)
+{
+    if (op < IMM_FIELD_ADD || op > IMM_FIELD_MUL || count < 0) return IMM_ERR_ARG;
+    if (count == 0) return IMM_OK;
+    if (!d_x || !d_y || !d_out) return IMM_ERR_ARG;
+    CU(launch_field_binop(op, d_x, d_y, d_out, count, (cudaStream_t)stream));
+    return IMM_OK;
+}
+
+int imm_eq_table(const imm_fe* r_host, int nvars, imm_fe* d_out, void* stream)
+{
+    if (!d_out || (nvars > 0 && !r_host)) return IMM_ERR_ARG;
+    if (nvars < 0 || nvars > MAX_EQ_VARS) return IMM_ERR_SHAPE;
+    if ((uintptr_t)d_out % 16 != 0) return IMM_ERR_ALIGN;
+    EqDirect r;
+    memset(&r, 0, sizeof(r));
+    for (int t = 0; t < nvars; t++) {
+        if (r_host[t] >= IMM_P) return IMM_ERR_NONCANONICAL;
+        r.r[t] = r_host[t];
+    }
+    CU(launch_eq_direct(r, nvars, d_out, (cudaStream_t)stream));
+    return IMM_OK;
+}
+
+size_t imm_mle_workspace(int dtype, int64_t rows, int64_t cols, int bind)
+{
+    if ((dtype != IMM_I8 && dtype != IMM_I32) || rows <= 0 || cols <= 0 || rows > MAX_EXTENT ||
+        cols > MAX_EXTENT || (bind != IMM_BIND_ROWS && bind != IMM_BIND_COLS))
+        return 0;
+    std::vector<Shape> one{{rows, cols}};
+    size_t parts;
+    if (bind == IMM_BIND_ROWS) {
+        int tr = pick_tile_rows(one, rowbind_cols(dtype), "IMM_TILE_ROWS_A");
+        int64_t nrb = (rows + tr - 1) / tr, ncc = (cols + rowbind_cols(dtype) - 1) / rowbind_cols(dtype);
+        size_t vec_parts = (size_t)nrb * cols, pt_parts = (size_t)(nrb * ncc);   // partial_eval / eval_point
+        parts = vec_parts > pt_parts ? vec_parts : pt_parts;
+    } else {
+        int64_t ncc = (cols + colbind_cols(dtype) - 1) / colbind_cols(dtype);
+        parts = (size_t)ncc * rows;
+    }
+    return ALIGN + align_up(parts * sizeof(imm_fe));
+}
+
+int imm_mle_partial_eval(const void* d_mat, int dtype, int64_t rows, int64_t cols, int64_t ld,
+                         int bind, const imm_fe* d_eq, imm_fe* d_out,
+                         void* d_ws, size_t ws_bytes, void* stream)
+{
+    int rc = check_matrix_args(d_mat, dtype, rows, cols, ld);
+    if (rc != IMM_OK) return rc;
+    if (!d_eq || !d_out || !d_ws || (bind != IMM_BIND_ROWS && bind != IMM_BIND_COLS)) return IMM_ERR_ARG;
+    if ((uintptr_t)d_ws % 16 != 0 || (uintptr_t)d_out % 16 != 0 || (uintptr_t)d_eq % 8 != 0) return IMM_ERR_ALIGN;
+    if (ws_bytes < imm_mle_workspace(dtype, rows, cols, bind)) return IMM_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    std::vector<Shape> one{{rows, cols}};
+    MatJob* d_job = (MatJob*)d_ws;
+    imm_fe* d_parts = (imm_fe*)((char*)d_ws + ALIGN);
+    MatJob j;
+    if (bind == IMM_BIND_ROWS) {
+        int tr = pick_tile_rows(one, rowbind_cols(dtype), "IMM_TILE_ROWS_A");
+        fill_job(j, d_mat, dtype, rows, cols, ld, tr, rowbind_cols(dtype));
+        j.eq_row = d_eq;
+        j.out = j.nrb == 1 ? d_out : d_parts;
+        CU(cudaMemcpyAsync(d_job, &j, sizeof(j), cudaMemcpyHostToDevice, st));
+        CU(launch_rowbind(dtype, false, d_job, 1, (uint32_t)(j.nrb * j.ncc), st));
+        if (j.nrb > 1) CU(launch_sum_parts(d_parts, j.nrb, cols, d_out, st));
+    } else {
+        int tr = pick_tile_rows(one, colbind_cols(dtype), "IMM_TILE_ROWS_B");
+        fill_job(j, d_mat, dtype, rows, cols, ld, tr, colbind_cols(dtype));
+        j.eq_col = d_eq;
+        j.out = j.ncc == 1 ? d_out : d_parts;
+        CU(cudaMemcpyAsync(d_job, &j, sizeof(j), cudaMemcpyHostToDevice, st));
+        CU(launch_colbind(dtype, d_job, 1, (uint32_t)(j.nrb * j.ncc), st));
+        if (j.ncc > 1) CU(launch_sum_parts(d_parts, j.ncc, rows, d_out, st));
+    }
+    return IMM_OK;
+}
+
+int imm_mle_eval_point(const void* d_mat, int dtype, int64_t rows, int64_t cols, int64_t ld,
+                       const imm_fe* d_eq_row, const imm_fe* d_eq_col, imm_fe* d_out,
+                       void* d_ws, size_t ws_bytes, void* stream)
+{
+    int rc = check_matrix_args(d_mat, dtype, rows, cols, ld);
+    if (rc != IMM_OK) return rc;
+    if (!d_eq_row || !d_eq_col || !d_out || !d_ws) return IMM_ERR_ARG;
+    if ((uintptr_t)d_ws % 16 != 0 || (uintptr_t)d_out % 8 != 0) return IMM_ERR_ALIGN;
+    if (ws_bytes < imm_mle_workspace(dtype, rows, cols, IMM_BIND_ROWS)) return IMM_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    std::vector<Shape> one{{rows, cols}};
+    MatJob* d_job = (MatJob*)d_ws;
+    imm_fe* d_parts = (imm_fe*)((char*)d_ws + ALIGN);
+    MatJob j;
+    int tr = pick_tile_rows(one, rowbind_cols(dtype), "IMM_TILE_ROWS_A");
+    fill_job(j, d_mat, dtype, rows, cols, ld, tr, rowbind_cols(dtype));
+    j.eq_row = d_eq_row;
+    j.eq_col = d_eq_col;
+    j.out = d_parts;
+    CU(cudaMemcpyAsync(d_job, &j, sizeof(j), cudaMemcpyHostToDevice, st));
+    CU(launch_rowbind(dtype, true, d_job, 1, (uint32_t)(j.nrb * j.ncc), st));
+    CU(launch_sum_all(d_parts, (int64_t)j.nrb * j.ncc, d_out, st));
+    return IMM_OK;
+}
+
+size_t imm_sumcheck_matmul_workspace(const imm_matmul_desc* descs_host, int nproofs)
+{
+    Plan p = make_plan(descs_host, nproofs);
+    return p.status == IMM_OK ? p.total_bytes : 0;
+}
+
+int imm_sumcheck_matmul_prove(const imm_matmul_desc* descs_host, int nproofs, uint64_t seed,
+                              imm_fe* d_transcripts, int64_t stride, int32_t* d_status,
+                              void* d_ws, size_t ws_bytes, void* stream)
+{
+    if (!d_transcripts || !d_status || !d_ws) return IMM_ERR_ARG;
+    Plan p = make_plan(descs_host, nproofs);
+    if (p.status != IMM_OK) return p.status;
+    int rc = check_stride(descs_host, nproofs, stride);
+    if (rc != IMM_OK) return rc;
+    if ((uintptr_t)d_ws % 16 != 0 || (uintptr_t)d_transcripts % 8 != 0 || (uintptr_t)d_status % 4 != 0)
+        return IMM_ERR_ALIGN;
+    if (ws_bytes < p.total_bytes) return IMM_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    char* base = (char*)d_ws;
+
+    // header image: per-proof state, the three job lists, the eq tasks
+    std::vector<char> hdr(p.header_bytes, 0);
+    ProofDev* pd = (ProofDev*)(hdr.data() + p.off_proofs);
+    MatJob* ja = (MatJob*)(hdr.data() + p.off_jobs_a);
+    MatJob* jb = (MatJob*)(hdr.data() + p.off_jobs_b);
+    MatJob* jc = (MatJob*)(hdr.data() + p.off_jobs_c);
+    EqTask* eq = (EqTask*)(hdr.data() + p.off_eq);
+    uint32_t ta = 0, tb = 0, tc = 0;
+    for (int i = 0; i < nproofs; i++) {
+        const imm_matmul_desc& d = descs_host[i];
+        const Plan::PerProof& q = p.pp[i];
+        ProofDev& P = pd[i];
+        P.e_row = (imm_fe*)(base + q.e_row);
+        P.e_col = (imm_fe*)(base + q.e_col);
+        P.part_a = (imm_fe*)(base + q.part_a);
+        P.part_b = (imm_fe*)(base + q.part_b);
+        P.part_c = (imm_fe*)(base + q.part_c);
+        P.tab = (imm_fe*)(base + q.tab);
+        P.proof_id = d.proof_id;
+        P.m = (int32_t)d.m; P.k = (int32_t)d.k; P.n = (int32_t)d.n;
+        P.a = q.a; P.b = q.b; P.c = q.c;
+        P.n_part_a = q.n_part_a; P.n_part_b = q.n_part_b; P.n_part_c = q.n_part_c;
+
+        fill_job(ja[i], d.A, IMM_I8, d.m, d.k, d.lda, p.rows_a, rowbind_cols(IMM_I8));
+        ja[i].eq_row = P.e_row; ja[i].out = (imm_fe*)P.part_a; ja[i].tile0 = ta;
+        ta += (uint32_t)(ja[i].nrb * ja[i].ncc);
+        fill_job(jb[i], d.B, IMM_I8, d.k, d.n, d.ldb, p.rows_b, colbind_cols(IMM_I8));
+        jb[i].eq_col = P.e_col; jb[i].out = (imm_fe*)P.part_b; jb[i].tile0 = tb;
+        tb += (uint32_t)(jb[i].nrb * jb[i].ncc);
+        fill_job(jc[i], d.C, IMM_I32, d.m, d.n, d.ldc, p.rows_c, rowbind_cols(IMM_I32));
+        jc[i].eq_row = P.e_row; jc[i].eq_col = P.e_col; jc[i].out = (imm_fe*)P.part_c; jc[i].tile0 = tc;
+        tc += (uint32_t)(jc[i].nrb * jc[i].ncc);
+
+        eq[2 * i] = EqTask{P.e_row, seed, d.proof_id, 1u, q.a};
+        eq[2 * i + 1] = EqTask{P.e_col, seed, d.proof_id, 2u, q.c};
+    }
+    if (ta != p.tiles_a || tb != p.tiles_b || tc != p.tiles_c) return IMM_ERR_ARG;   // planner invariant
+
+    CU(cudaMemcpyAsync(base, hdr.data(), hdr.size(), cudaMemcpyHostToDevice, st));
+    CU(launch_eq_batch((const EqTask*)(base + p.off_eq), 2 * nproofs, st));
+    CU(launch_rowbind(IMM_I32, true, (const MatJob*)(base + p.off_jobs_c), nproofs, p.tiles_c, st));
+    CU(launch_rowbind(IMM_I8, false, (const MatJob*)(base + p.off_jobs_a), nproofs, p.tiles_a, st));
+    CU(launch_colbind(IMM_I8, (const MatJob*)(base + p.off_jobs_b), nproofs, p.tiles_b, st));
+    CU(launch_sumcheck((const ProofDev*)(base + p.off_proofs), nproofs, seed, d_transcripts, stride,
+                       d_status, p.max_b, st));
+    return IMM_OK;
+}
+
+}  // extern "C"
+
+// ------------------------------------------------------------------ host-buffer variant ---
+
+namespace {
+
+struct ArenaPlan {
+    int status = IMM_OK;
+    struct M { size_t a, b, c; int64_t lda, ldb, ldc; };
+    std::vector<M> mats;
+    size_t off_tr = 0, off_status = 0, off_ws = 0, ws_bytes = 0, total = 0;
+};
+
+int64_t pad16(int64_t cols, int elem) { int per = 16 / elem; return (cols + per - 1) / per * per; }
+
+ArenaPlan make_arena(const imm_matmul_desc* descs, int nproofs, int64_t stride)
+{
+    ArenaPlan ap;
+    Plan p = make_plan(descs, nproofs);
+    if (p.status != IMM_OK) { ap.status = p.status; return ap; }
+    size_t off = 0;
+    ap.mats.resize(nproofs);
+    for (int i = 0; i < nproofs; i++) {
+        const imm_matmul_desc& d = descs[i];
+        ArenaPlan::M& m = ap.mats[i];
+        m.lda = pad16(d.k, 1); m.ldb = pad16(d.n, 1); m.ldc = pad16(d.n, 4);
+        m.a = off; off = align_up(off + (size_t)d.m * m.lda);
+        m.b = off; off = align_up(off + (size_t)d.k * m.ldb);
+        m.c = off; off = align_up(off + (size_t)d.m * m.ldc * 4);
+    }
+    ap.off_tr = off;     off = align_up(off + (size_t)nproofs * (size_t)stride * sizeof(imm_fe));
+    ap.off_status = off; off = align_up(off + (size_t)nproofs * sizeof(int32_t));
+    ap.off_ws = off;
+    ap.ws_bytes = p.total_bytes;
+    ap.total = off + p.total_bytes;
+    return ap;
+}
+
+int64_t max_transcript_len(const imm_matmul_desc* descs, int nproofs)
+{
+    int64_t len = 3;
+    for (int i = 0; i < nproofs; i++) {
+        int64_t l = 3 * ceil_log2(descs[i].k) + 3;
+        if (l > len) len = l;
+    }
+    return len;
+}
+
+cudaError_t copy_in(void* dst, int64_t dld, const void* src, int64_t sld, int64_t rows, int64_t cols,
+                    int elem, cudaStream_t st)
+{
+    if (dld == sld)
+        return cudaMemcpyAsync(dst, src, (size_t)((rows - 1) * sld + cols) * elem, cudaMemcpyHostToDevice, st);
+    return cudaMemcpy2DAsync(dst, (size_t)dld * elem, src, (size_t)sld * elem, (size_t)cols * elem,
+                             (size_t)rows, cudaMemcpyHostToDevice, st);
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t imm_sumcheck_matmul_host_arena(const imm_matmul_desc* descs_host, int nproofs)
+{
+    if (!descs_host || nproofs <= 0) return 0;
+    for (int i = 0; i < nproofs; i++)
+        if (check_desc(descs_host[i]) != IMM_OK) return 0;
+    ArenaPlan ap = make_arena(descs_host, nproofs, max_transcript_len(descs_host, nproofs));
+    return ap.status == IMM_OK ? ap.total : 0;
+}
+
+int imm_sumcheck_matmul_prove_host(const imm_matmul_desc* descs_host, int nproofs, uint64_t seed,
+                                   imm_fe* transcripts_host, int64_t stride, int32_t* status_host,
+                                   void* d_arena, size_t arena_bytes, void* stream)
+{
+    if (!descs_host || nproofs <= 0 || !transcripts_host || !status_host || !d_arena) return IMM_ERR_ARG;
+    for (int i = 0; i < nproofs; i++) {
+        int rc = check_desc(descs_host[i]);
+        if (rc != IMM_OK) return rc;
+    }
+    int rc = check_stride(descs_host, nproofs, stride);
+    if (rc != IMM_OK) return rc;
+    if ((uintptr_t)d_arena % ALIGN != 0) return IMM_ERR_ALIGN;
+    // the arena is sized for the tightest stride; a wider one only grows the transcript block
+    ArenaPlan ap = make_arena(descs_host, nproofs, stride);
+    if (ap.status != IMM_OK) return ap.status;
+    if (arena_bytes < ap.total) return IMM_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    char* base = (char*)d_arena;
+
+    std::vector<imm_matmul_desc> dev(descs_host, descs_host + nproofs);
+    for (int i = 0; i < nproofs; i++) {
+        const imm_matmul_desc& d = descs_host[i];
+        const ArenaPlan::M& m = ap.mats[i];
+        CU(copy_in(base + m.a, m.lda, d.A, d.lda, d.m, d.k, 1, st));
+        CU(copy_in(base + m.b, m.ldb, d.B, d.ldb, d.k, d.n, 1, st));
+        CU(copy_in(base + m.c, m.ldc, d.C, d.ldc, d.m, d.n, 4, st));
+        dev[i].A = (const int8_t*)(base + m.a); dev[i].lda = m.lda;
+        dev[i].B = (const int8_t*)(base + m.b); dev[i].ldb = m.ldb;
+        dev[i].C = (const int32_t*)(base + m.c); dev[i].ldc = m.ldc;
+    }
+    imm_fe* d_tr = (imm_fe*)(base + ap.off_tr);
+    int32_t* d_status = (int32_t*)(base + ap.off_status);
+    rc = imm_sumcheck_matmul_prove(dev.data(), nproofs, seed, d_tr, stride, d_status,
+                                   base + ap.off_ws, ap.ws_bytes, stream);
+    if (rc != IMM_OK) return rc;
+    CU(cudaMemcpyAsync(transcripts_host, d_tr, (size_t)nproofs * (size_t)stride * sizeof(imm_fe),
+                       cudaMemcpyDeviceToHost, st));
+    CU(cudaMemcpyAsync(status_host, d_status, (size_t)nproofs * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    CU(cudaStreamSynchronize(st));
+    return IMM_OK;
+}
+
+// ------------------------------------------------------------------ verifier (host) -------
+
+int imm_sumcheck_verify(const imm_fe* transcript_host, int nrounds, uint64_t seed,
+                        uint64_t proof_id, const imm_fe* expect_c0, const imm_fe* expect_a_fin,
+                        const imm_fe* expect_b_fin, int* fail_at)
+{
+    if (!transcript_host || !fail_at || nrounds < 0 || nrounds > 64) return IMM_ERR_ARG;
+    const imm_fe* t = transcript_host;
+    for (int i = 0; i < 3 * nrounds + 3; i++)
+        if (t[i] >= IMM_P) return IMM_ERR_NONCANONICAL;
+    if ((expect_c0 && *expect_c0 >= IMM_P) || (expect_a_fin && *expect_a_fin >= IMM_P) ||
+        (expect_b_fin && *expect_b_fin >= IMM_P))
+        return IMM_ERR_NONCANONICAL;
+    const uint64_t inv2 = 0x7FFFFFFF80000001ULL;
+    uint64_t claim = t[0];
+    for (int j = 0; j < nrounds; j++) {
+        const uint64_t g0 = t[1 + 3 * j], g1 = t[2 + 3 * j], g2 = t[3 + 3 * j];
+        if (gl::add(g0, g1) != claim) { *fail_at = j; return IMM_REJECT; }
+        // Newton form on the nodes 0,1,2: g(r) = g0 + r*d1 + r(r-1)/2 * d2
+        const uint64_t r = gl::challenge(seed, proof_id, 3, (uint32_t)j);
+        const uint64_t d1 = gl::sub(g1, g0);
+        const uint64_t d2 = gl::sub(gl::sub(g2, g1), d1);
+        const uint64_t c2 = gl::mul(gl::mul(r, gl::sub(r, 1)), inv2);
+        claim = gl::add(g0, gl::add(gl::mul(r, d1), gl::mul(c2, d2)));
+    }
+    const uint64_t a_fin = t[3 * nrounds + 1], b_fin = t[3 * nrounds + 2];
+    if (gl::mul(a_fin, b_fin) != claim) { *fail_at = nrounds; return IMM_REJECT; }
+    if (expect_c0 && *expect_c0 != t[0]) { *fail_at = nrounds + 1; return IMM_REJECT; }
+    if (expect_a_fin && *expect_a_fin != a_fin) { *fail_at = nrounds + 2; return IMM_REJECT; }
+    if (expect_b_fin && *expect_b_fin != b_fin) { *fail_at = nrounds + 3; return IMM_REJECT; }
+    *fail_at = -1;
+    return IMM_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,644 @@
+// CUDA kernels of libimm (sm_100a): eq tables, eq-vector x matrix contractions mod p, and the
+// sumcheck rounds.  Host-side launch wrappers are at the end; the C ABI lives in imm_api.cu.
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "gl64.cuh"
+#include "imm_kernels.h"
+#include "imm_plan.h"
+
+namespace imm {
+
+// ------------------------------------------------------------------------------------------
+// small device helpers
+// ------------------------------------------------------------------------------------------
+
+__device__ __forceinline__ uint64_t shfl_xor_u64(uint64_t v, int mask)
+{
+    return __shfl_xor_sync(0xFFFFFFFFu, v, mask);
+}
+
+__device__ __forceinline__ uint64_t warp_sum_fe(uint64_t v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = gl::add(v, shfl_xor_u64(v, o));
+    return v;
+}
+
+// Sum of one canonical element per thread over the block; result valid in every thread.
+// `scratch` holds one word per warp plus one.
+__device__ __forceinline__ uint64_t block_sum_fe(uint64_t v, uint64_t* scratch)
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = (blockDim.x + 31) >> 5;
+    v = warp_sum_fe(v);
+    __syncthreads();                       // scratch may still be read from a previous call
+    if (lane == 0) scratch[warp] = v;
+    __syncthreads();
+    if (warp == 0) {
+        uint64_t t = lane < nwarp ? scratch[lane] : 0;
+        t = warp_sum_fe(t);
+        if (lane == 0) scratch[32] = t;
+    }
+    __syncthreads();
+    return scratch[32];
+}
+
+// 128-bit streaming load (read once: do not keep in L1)
+__device__ __forceinline__ uint4 ld_stream_v4(const void* p)
+{
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+// sign-extended byte `K` of a 32-bit word: one byte-permute with sign replication
+template <int K>
+__device__ __forceinline__ int32_t sext_byte(uint32_t w)
+{
+    int32_t r;
+    constexpr uint32_t sel = (uint32_t)K | ((uint32_t)(K | 8) << 4) | ((uint32_t)(K | 8) << 8) |
+                             ((uint32_t)(K | 8) << 12);
+    asm("prmt.b32 %0, %1, %1, %2;" : "=r"(r) : "r"(w), "n"(sel));
+    return r;
+}
+
+// acc += x * y  (signed 32 x 32 -> 64 multiply-add)
+__device__ __forceinline__ void mad_wide(int64_t& acc, int32_t x, int32_t y)
+{
+    asm("mad.wide.s32 %0, %1, %2, %0;" : "+l"(acc) : "r"(x), "r"(y));
+}
+
+// Find the job a tile belongs to: jobs are ordered by tile0.
+__device__ __forceinline__ int find_job(const MatJob* jobs, int njobs, uint32_t tile)
+{
+    int lo = 0, hi = njobs - 1;
+    while (lo < hi) {
+        int mid = (lo + hi + 1) >> 1;
+        if (jobs[mid].tile0 <= tile) lo = mid; else hi = mid - 1;
+    }
+    return lo;
+}
+
+// ------------------------------------------------------------------------------------------
+// element-wise field arithmetic (test hook for the device field code)
+// ------------------------------------------------------------------------------------------
+
+__global__ void field_binop_kernel(int op, const imm_fe* x, const imm_fe* y, imm_fe* out, int64_t n)
+{
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t step = (int64_t)gridDim.x * blockDim.x;
+    for (; i < n; i += step) {
+        uint64_t a = x[i], b = y[i];
+        out[i] = op == 0 ? gl::add(a, b) : op == 1 ? gl::sub(a, b) : gl::mul(a, b);
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// eq tables
+// ------------------------------------------------------------------------------------------
+// E[i] = eq(r, i), variable 0 = most significant index bit.  The index is split into a high
+// part (variables 0..nhi-1) and a low part (the rest); both small tables are built by doubling
+// in shared memory and E[i] = hi[i >> nlo] * lo[i & (2^nlo - 1)].  One block per table.
+
+__device__ void eq_build_small(uint64_t* tbl, const uint64_t* r, int cnt)
+{
+    if (threadIdx.x == 0) tbl[0] = 1;
+    __syncthreads();
+    for (int t = 0; t < cnt; t++) {
+        const int len = 1 << t;
+        uint64_t v = 0;
+        const bool act = (int)threadIdx.x < len;
+        if (act) v = tbl[threadIdx.x];
+        __syncthreads();
+        if (act) {
+            uint64_t h = gl::mul(v, r[t]);
+            tbl[2 * threadIdx.x + 1] = h;
+            tbl[2 * threadIdx.x] = gl::sub(v, h);
+        }
+        __syncthreads();
+    }
+}
+
+__device__ void eq_fill(imm_fe* out, int nvars, const uint64_t* r_sh, uint64_t* lo_t, uint64_t* hi_t)
+{
+    const int nlo = (nvars + 1) / 2, nhi = nvars - nlo;
+    eq_build_small(hi_t, r_sh, nhi);
+    eq_build_small(lo_t, r_sh + nhi, nlo);
+    const int64_t total = (int64_t)1 << nvars;
+    const uint32_t mask = (1u << nlo) - 1;
+    for (int64_t i = threadIdx.x; i < total; i += blockDim.x)
+        out[i] = gl::mul(hi_t[i >> nlo], lo_t[(uint32_t)i & mask]);
+}
+
+__global__ void __launch_bounds__(1024) eq_batch_kernel(const EqTask* tasks)
+{
+    __shared__ uint64_t r_sh[MAX_EQ_VARS];
+    __shared__ uint64_t lo_t[1024], hi_t[1024];
+    const EqTask t = tasks[blockIdx.x];
+    if ((int)threadIdx.x < t.nvars)
+        r_sh[threadIdx.x] = gl::challenge(t.seed, t.proof_id, t.domain, threadIdx.x);
+    __syncthreads();
+    eq_fill(t.out, t.nvars, r_sh, lo_t, hi_t);
+}
+
+__global__ void __launch_bounds__(1024) eq_direct_kernel(EqDirect rr, int nvars, imm_fe* out)
+{
+    __shared__ uint64_t r_sh[MAX_EQ_VARS];
+    __shared__ uint64_t lo_t[1024], hi_t[1024];
+    if ((int)threadIdx.x < nvars) r_sh[threadIdx.x] = rr.r[threadIdx.x];
+    __syncthreads();
+    eq_fill(out, nvars, r_sh, lo_t, hi_t);
+}
+
+// ------------------------------------------------------------------------------------------
+// contraction building blocks
+// ------------------------------------------------------------------------------------------
+// The eq weight e is consumed as two signed 32-bit halves (gl::balanced_halves) and the matrix
+// entries as signed 32-bit values, so one entry costs a handful of 32 x 32 -> 64 multiply-adds
+// into 64-bit accumulators with NO modular reduction in the loop (lazy accumulation):
+//   int8 :  L += e_lo*v, H += e_hi*v                       |term| < 2^38, > 2^24 terms of headroom
+//   int32:  v = v_hi*2^16 + v_lo (v_lo unsigned 16 bit):   |term| < 2^47, 2^16 terms of headroom
+//           LL += e_lo*v_lo, LH += e_lo*v_hi, HL += e_hi*v_lo, HH += e_hi*v_hi
+// The exact integer sum is rebuilt and reduced once per output.
+
+template <typename T> struct Elem;
+template <> struct Elem<int8_t>  { static constexpr int EPV = 16; static constexpr int NACC = 2; };
+template <> struct Elem<int32_t> { static constexpr int EPV = 4;  static constexpr int NACC = 4; };
+
+// element-wise gather of up to EPV entries into the layout of a 16-byte vector load
+template <typename T>
+__device__ __forceinline__ uint4 load_elems(const T* p, int nvalid)
+{
+    union { uint4 v; T e[Elem<T>::EPV]; } u;
+    u.v = make_uint4(0, 0, 0, 0);
+#pragma unroll
+    for (int j = 0; j < Elem<T>::EPV; j++)
+        if (j < nvalid) u.e[j] = p[j];
+    return u.v;
+}
+
+template <typename T, bool VEC>
+__device__ __forceinline__ uint4 load_vec(const char* p, bool full, int nvalid)
+{
+    if (VEC && full) return ld_stream_v4(p);
+    return load_elems<T>(reinterpret_cast<const T*>(p), nvalid);
+}
+
+template <int K>
+__device__ __forceinline__ void mac_word_i8(int64_t* acc /* [4][2] */, uint32_t w, int32_t el, int32_t eh)
+{
+    int32_t v = sext_byte<K>(w);
+    mad_wide(acc[2 * K], el, v);
+    mad_wide(acc[2 * K + 1], eh, v);
+}
+
+// acc layout int8: [16 columns][2] = (L, H); int32: [4 columns][4] = (LL, LH, HL, HH)
+__device__ __forceinline__ void mac_vec(int64_t (&acc)[32], uint4 w, int32_t el, int32_t eh, int8_t)
+{
+    const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+    for (int q = 0; q < 4; q++) {
+        mac_word_i8<0>(&acc[8 * q], ww[q], el, eh);
+        mac_word_i8<1>(&acc[8 * q], ww[q], el, eh);
+        mac_word_i8<2>(&acc[8 * q], ww[q], el, eh);
+        mac_word_i8<3>(&acc[8 * q], ww[q], el, eh);
+    }
+}
+
+__device__ __forceinline__ void mac_vec(int64_t (&acc)[16], uint4 w, int32_t el, int32_t eh, int32_t)
+{
+    const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+#pragma unroll
+    for (int q = 0; q < 4; q++) {
+        int32_t vlo = (int32_t)(ww[q] & 0xFFFFu);
+        int32_t vhi = (int32_t)ww[q] >> 16;
+        mad_wide(acc[4 * q + 0], el, vlo);
+        mad_wide(acc[4 * q + 1], el, vhi);
+        mad_wide(acc[4 * q + 2], eh, vlo);
+        mad_wide(acc[4 * q + 3], eh, vhi);
+    }
+}
+
+// exact integer accumulators of one column -> canonical field element
+__device__ __forceinline__ uint64_t finish_col(const int64_t* a, int8_t)
+{
+    return gl::add(gl::from_i64(a[0]), gl::shl(gl::from_i64(a[1]), 32));
+}
+__device__ __forceinline__ uint64_t finish_col(const int64_t* a, int32_t)
+{
+    uint64_t lo = gl::add(gl::from_i64(a[0]), gl::shl(gl::from_i64(a[1]), 16));
+    uint64_t hi = gl::add(gl::shl(gl::from_i64(a[2]), 32), gl::shl(gl::from_i64(a[3]), 48));
+    return gl::add(lo, hi);
+}
+
+// ------------------------------------------------------------------------------------------
+// row binding:  out[y] = sum_i eq_row[i] * M[i,y]   (POINT: then dotted with eq_col)
+// ------------------------------------------------------------------------------------------
+// One tile = tile_rows rows x (ROWBIND_THREADS * EPV) columns.  A thread owns one 16-byte vector
+// of columns and walks down the rows; a warp therefore reads 512 contiguous bytes of each row.
+
+template <typename T, bool POINT, bool VEC>
+__device__ __forceinline__ void rowbind_tile(const MatJob& job, uint32_t local, int2* sE, uint64_t* red)
+{
+    constexpr int EPV = Elem<T>::EPV, NACC = Elem<T>::NACC;
+    const int rbi = local / job.ncc, cci = local % job.ncc;
+    const int r0 = rbi * job.tile_rows;
+    const int nrows = min(job.tile_rows, job.rows - r0);
+    const int col = (cci * ROWBIND_THREADS + threadIdx.x) * EPV;
+    const int nvalid = min(EPV, job.cols - col);          // <= 0: this thread has no columns
+    const bool full = nvalid == EPV;
+
+    for (int i = threadIdx.x; i < nrows; i += ROWBIND_THREADS) {
+        int32_t lo, hi;
+        gl::balanced_halves(job.eq_row[r0 + i], lo, hi);
+        sE[i] = make_int2(lo, hi);
+    }
+    __syncthreads();
+
+    int64_t acc[EPV * NACC];
+#pragma unroll
+    for (int j = 0; j < EPV * NACC; j++) acc[j] = 0;
+
+    if (nvalid > 0) {
+        const int64_t pitch = job.ld * (int64_t)sizeof(T);
+        const char* p = (const char*)job.mat + ((int64_t)r0 * job.ld + col) * (int64_t)sizeof(T);
+        int i = 0;
+        for (; i + 4 <= nrows; i += 4) {
+            uint4 w0 = load_vec<T, VEC>(p, full, nvalid);
+            uint4 w1 = load_vec<T, VEC>(p + pitch, full, nvalid);
+            uint4 w2 = load_vec<T, VEC>(p + 2 * pitch, full, nvalid);
+            uint4 w3 = load_vec<T, VEC>(p + 3 * pitch, full, nvalid);
+            p += 4 * pitch;
+            int2 e0 = sE[i], e1 = sE[i + 1], e2 = sE[i + 2], e3 = sE[i + 3];
+            mac_vec(acc, w0, e0.x, e0.y, T());
+            mac_vec(acc, w1, e1.x, e1.y, T());
+            mac_vec(acc, w2, e2.x, e2.y, T());
+            mac_vec(acc, w3, e3.x, e3.y, T());
+        }
+        for (; i < nrows; i++) {
+            uint4 w0 = load_vec<T, VEC>(p, full, nvalid);
+            p += pitch;
+            int2 e0 = sE[i];
+            mac_vec(acc, w0, e0.x, e0.y, T());
+        }
+    }
+
+    if (!POINT) {
+        if (nvalid > 0) {
+            imm_fe* o = job.out + (int64_t)rbi * job.cols + col;
+#pragma unroll
+            for (int j = 0; j < EPV; j++)
+                if (j < nvalid) o[j] = finish_col(&acc[NACC * j], T());
+        }
+    } else {
+        uint64_t part = 0;
+        if (nvalid > 0) {
+#pragma unroll
+            for (int j = 0; j < EPV; j++)
+                if (j < nvalid)
+                    part = gl::add(part, gl::mul(finish_col(&acc[NACC * j], T()), job.eq_col[col + j]));
+        }
+        part = block_sum_fe(part, red);
+        if (threadIdx.x == 0) job.out[local] = part;
+    }
+}
+
+template <typename T, bool POINT>
+__global__ void __launch_bounds__(ROWBIND_THREADS) rowbind_kernel(const MatJob* jobs, int njobs)
+{
+    __shared__ int2 sE[MAX_TILE_ROWS];
+    __shared__ uint64_t red[33];
+    const MatJob job = jobs[find_job(jobs, njobs, blockIdx.x)];
+    const uint32_t local = blockIdx.x - job.tile0;
+    if (job.vec) rowbind_tile<T, POINT, true>(job, local, sE, red);
+    else rowbind_tile<T, POINT, false>(job, local, sE, red);
+}
+
+// ------------------------------------------------------------------------------------------
+// column binding:  out[i] = sum_j M[i,j] * eq_col[j]
+// ------------------------------------------------------------------------------------------
+// One tile = tile_rows rows x one chunk of COLBIND_VECS vectors of columns.  The chunk's eq
+// weights sit in shared memory as balanced halves, laid out [pair of columns][vector] so that a
+// warp's 16-byte reads are conflict-free.  A warp takes COLBIND_ROWS_PER_WARP rows at a time:
+// each lane loads the weights of its vector once and applies them to all those rows, then the
+// per-row integer sums are combined across the warp with shuffles.
+
+template <typename T, bool VEC>
+__device__ __forceinline__ void colbind_tile(const MatJob& job, uint32_t local, int4* sE)
+{
+    constexpr int EPV = Elem<T>::EPV, NACC = Elem<T>::NACC, RW = COLBIND_ROWS_PER_WARP;
+    constexpr int PAIRS = EPV / 2;
+    const int rbi = local / job.ncc, cci = local % job.ncc;
+    const int r0 = rbi * job.tile_rows;
+    const int r1 = min(r0 + job.tile_rows, job.rows);
+    const int c0 = cci * COLBIND_VECS * EPV;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    constexpr int NWARP = COLBIND_THREADS / 32;
+
+    // stage the chunk's weights: sE[pair * COLBIND_VECS + vec] = (lo0, hi0, lo1, hi1)
+    for (int t = threadIdx.x; t < COLBIND_VECS * PAIRS; t += COLBIND_THREADS) {
+        const int vec = t / PAIRS, pair = t % PAIRS;
+        const int col = c0 + vec * EPV + 2 * pair;
+        int32_t l0 = 0, h0 = 0, l1 = 0, h1 = 0;
+        if (col < job.cols) gl::balanced_halves(job.eq_col[col], l0, h0);
+        if (col + 1 < job.cols) gl::balanced_halves(job.eq_col[col + 1], l1, h1);
+        sE[pair * COLBIND_VECS + vec] = make_int4(l0, h0, l1, h1);
+    }
+    __syncthreads();
+
+    const int64_t pitch = job.ld * (int64_t)sizeof(T);
+    for (int r = r0 + warp * RW; r < r1; r += NWARP * RW) {
+        int64_t acc[RW][NACC];
+#pragma unroll
+        for (int u = 0; u < RW; u++)
+#pragma unroll
+            for (int a = 0; a < NACC; a++) acc[u][a] = 0;
+
+        for (int vec = lane; vec < COLBIND_VECS; vec += 32) {
+            const int col = c0 + vec * EPV;
+            const int nvalid = min(EPV, job.cols - col);
+            if (nvalid <= 0) break;
+            const bool full = nvalid == EPV;
+            const char* p = (const char*)job.mat + ((int64_t)r * job.ld + col) * (int64_t)sizeof(T);
+            uint4 w[RW];
+#pragma unroll
+            for (int u = 0; u < RW; u++)
+                w[u] = (r + u < r1) ? load_vec<T, VEC>(p + u * pitch, full, nvalid) : make_uint4(0, 0, 0, 0);
+            int4 e[PAIRS];
+#pragma unroll
+            for (int q = 0; q < PAIRS; q++) e[q] = sE[q * COLBIND_VECS + vec];
+#pragma unroll
+            for (int u = 0; u < RW; u++) {
+                const uint32_t ww[4] = {w[u].x, w[u].y, w[u].z, w[u].w};
+                if constexpr (sizeof(T) == 1) {
+#pragma unroll
+                    for (int q = 0; q < 4; q++) {          // word q holds columns 4q..4q+3
+                        const int4 ea = e[2 * q], eb = e[2 * q + 1];
+                        int32_t v0 = sext_byte<0>(ww[q]), v1 = sext_byte<1>(ww[q]);
+                        int32_t v2 = sext_byte<2>(ww[q]), v3 = sext_byte<3>(ww[q]);
+                        mad_wide(acc[u][0], ea.x, v0); mad_wide(acc[u][1], ea.y, v0);
+                        mad_wide(acc[u][0], ea.z, v1); mad_wide(acc[u][1], ea.w, v1);
+                        mad_wide(acc[u][0], eb.x, v2); mad_wide(acc[u][1], eb.y, v2);
+                        mad_wide(acc[u][0], eb.z, v3); mad_wide(acc[u][1], eb.w, v3);
+                    }
+                } else {
+#pragma unroll
+                    for (int q = 0; q < 4; q++) {          // word q is column q
+                        const int4 ee = e[q / 2];
+                        const int32_t el = (q & 1) ? ee.z : ee.x, eh = (q & 1) ? ee.w : ee.y;
+                        int32_t vlo = (int32_t)(ww[q] & 0xFFFFu), vhi = (int32_t)ww[q] >> 16;
+                        mad_wide(acc[u][0], el, vlo);
+                        mad_wide(acc[u][1], el, vhi);
+                        mad_wide(acc[u][2], eh, vlo);
+                        mad_wide(acc[u][3], eh, vhi);
+                    }
+                }
+            }
+        }
+        // combine across the warp; per-lane sums stay far below 2^63 (see headroom above)
+#pragma unroll
+        for (int u = 0; u < RW; u++)
+#pragma unroll
+            for (int a = 0; a < NACC; a++) {
+                int64_t v = acc[u][a];
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) v += (int64_t)shfl_xor_u64((uint64_t)v, o);
+                acc[u][a] = v;
+            }
+        if (lane < RW && r + lane < r1) {
+            int64_t mine[NACC] = {};
+#pragma unroll
+            for (int u = 0; u < RW; u++)
+                if (u == lane)
+#pragma unroll
+                    for (int a = 0; a < NACC; a++) mine[a] = acc[u][a];
+            job.out[(int64_t)cci * job.rows + r + lane] = finish_col(mine, T());
+        }
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(COLBIND_THREADS) colbind_kernel(const MatJob* jobs, int njobs)
+{
+    __shared__ int4 sE[COLBIND_VECS * (Elem<T>::EPV / 2)];
+    const MatJob job = jobs[find_job(jobs, njobs, blockIdx.x)];
+    const uint32_t local = blockIdx.x - job.tile0;
+    if (job.vec) colbind_tile<T, true>(job, local, sE);
+    else colbind_tile<T, false>(job, local, sE);
+}
+
+// ------------------------------------------------------------------------------------------
+// sum of partial vectors:  out[y] = sum_p parts[p][y]
+// ------------------------------------------------------------------------------------------
+
+__global__ void sum_parts_kernel(const imm_fe* parts, int nparts, int64_t len, imm_fe* out)
+{
+    int64_t y = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (y >= len) return;
+    uint64_t s = 0;
+    for (int p = 0; p < nparts; p++) s = gl::add(s, parts[(int64_t)p * len + y]);
+    out[y] = s;
+}
+
+// out[0] = sum of `count` elements (single block)
+__global__ void __launch_bounds__(1024) sum_all_kernel(const imm_fe* parts, int64_t count, imm_fe* out)
+{
+    __shared__ uint64_t red[33];
+    uint64_t s = 0;
+    for (int64_t i = threadIdx.x; i < count; i += blockDim.x) s = gl::add(s, parts[i]);
+    s = block_sum_fe(s, red);
+    if (threadIdx.x == 0) out[0] = s;
+}
+
+// ------------------------------------------------------------------------------------------
+// sumcheck rounds: one block per proof
+// ------------------------------------------------------------------------------------------
+// Round j works on tables a[], b[] of 2h entries (h = 2^(b-1-j)) and sends
+//   g(0) = sum_{y<h} a[y] b[y],  g(1) = sum a[y+h] b[y+h],  g(2) = sum (2a[y+h]-a[y]) (2b[y+h]-b[y]),
+// then folds a[y] <- a[y] + r_j (a[y+h] - a[y]) (same for b).  Challenges are public coins, so the
+// fold of round j does not wait for g_j: each pass folds with r_j AND accumulates round j+1's
+// three sums from the values it has just produced (a thread folds the two pairs that form one
+// pair of the next round).  Tables start in global memory (L2-resident) and move to shared
+// memory as soon as the folded pair of tables fits; folding is in place.
+
+struct Sums3 { uint64_t g0, g1, g2; };
+
+__device__ __forceinline__ void sums_add(Sums3& s, uint64_t a0, uint64_t a1, uint64_t b0, uint64_t b1)
+{
+    s.g0 = gl::add(s.g0, gl::mul(a0, b0));
+    s.g1 = gl::add(s.g1, gl::mul(a1, b1));
+    uint64_t a2 = gl::sub(gl::add(a1, a1), a0), b2 = gl::sub(gl::add(b1, b1), b0);
+    s.g2 = gl::add(s.g2, gl::mul(a2, b2));
+}
+
+__device__ __forceinline__ uint64_t fold1(uint64_t lo, uint64_t hi, uint64_t r)
+{
+    return gl::add(lo, gl::mul(r, gl::sub(hi, lo)));
+}
+
+__device__ __forceinline__ uint64_t sum_parts_at(const imm_fe* parts, int nparts, int len, int y)
+{
+    if (y >= len) return 0;
+    uint64_t s = 0;
+    for (int p = 0; p < nparts; p++) s = gl::add(s, parts[(int64_t)p * len + y]);
+    return s;
+}
+
+__global__ void __launch_bounds__(SUMCHECK_THREADS)
+sumcheck_kernel(const ProofDev* proofs, uint64_t seed, imm_fe* transcripts, int64_t stride,
+                int32_t* status, int smem_entries /* capacity per table, entries */)
+{
+    extern __shared__ __align__(16) uint64_t smem[];       // [2][smem_entries] tables
+    __shared__ uint64_t red[33];
+    const ProofDev pr = proofs[blockIdx.x];
+    imm_fe* tr = transcripts + (int64_t)blockIdx.x * stride;
+    const int tid = threadIdx.x, nthr = blockDim.x;
+    const int b = pr.b;
+    const int64_t full = (int64_t)1 << b;
+
+    // claim c0 = sum of the partial sums of C
+    {
+        uint64_t s = 0;
+        for (int i = tid; i < pr.n_part_c; i += nthr) s = gl::add(s, pr.part_c[i]);
+        s = block_sum_fe(s, red);
+        if (tid == 0) tr[0] = s;
+    }
+    for (int64_t i = 3 * b + 3 + tid; i < stride; i += nthr) tr[i] = 0;
+    if (tid == 0) status[blockIdx.x] = 0;
+
+    uint64_t* ta = pr.tab;                // current tables (global to start with)
+    uint64_t* tb = pr.tab + full;
+    Sums3 acc = {0, 0, 0};
+
+    if (b == 0) {
+        if (tid == 0) {
+            tr[1] = sum_parts_at(pr.part_a, pr.n_part_a, pr.k, 0);
+            tr[2] = sum_parts_at(pr.part_b, pr.n_part_b, pr.k, 0);
+        }
+        return;
+    }
+
+    // build the round-0 tables from the partial vectors and accumulate round 0's sums
+    {
+        const int h = (int)(full >> 1);
+        for (int y = tid; y < h; y += nthr) {
+            uint64_t a0 = sum_parts_at(pr.part_a, pr.n_part_a, pr.k, y);
+            uint64_t a1 = sum_parts_at(pr.part_a, pr.n_part_a, pr.k, y + h);
+            uint64_t b0 = sum_parts_at(pr.part_b, pr.n_part_b, pr.k, y);
+            uint64_t b1 = sum_parts_at(pr.part_b, pr.n_part_b, pr.k, y + h);
+            ta[y] = a0; ta[y + h] = a1; tb[y] = b0; tb[y + h] = b1;
+            sums_add(acc, a0, a1, b0, b1);
+        }
+    }
+
+    for (int j = 0; j < b; j++) {
+        // publish round j's polynomial
+        uint64_t g0 = block_sum_fe(acc.g0, red);
+        uint64_t g1 = block_sum_fe(acc.g1, red);
+        uint64_t g2 = block_sum_fe(acc.g2, red);       // (also orders the table writes before the reads below)
+        if (tid == 0) { tr[1 + 3 * j] = g0; tr[2 + 3 * j] = g1; tr[3 + 3 * j] = g2; }
+        acc = {0, 0, 0};
+
+        const uint64_t r = gl::challenge(seed, pr.proof_id, 3, (uint32_t)j);
+        const int h = 1 << (b - 1 - j);                // size of the folded tables
+        uint64_t* da = ta;
+        uint64_t* db = tb;
+        if (ta != smem && h <= smem_entries) { da = smem; db = smem + smem_entries; }
+        if (h == 1) {
+            if (tid == 0) {
+                tr[3 * b + 1] = fold1(ta[0], ta[1], r);
+                tr[3 * b + 2] = fold1(tb[0], tb[1], r);
+            }
+        } else {
+            const int q = h >> 1;
+            for (int y = tid; y < q; y += nthr) {
+                uint64_t fa0 = fold1(ta[y], ta[y + h], r), fa1 = fold1(ta[y + q], ta[y + q + h], r);
+                uint64_t fb0 = fold1(tb[y], tb[y + h], r), fb1 = fold1(tb[y + q], tb[y + q + h], r);
+                da[y] = fa0; da[y + q] = fa1; db[y] = fb0; db[y + q] = fb1;
+                sums_add(acc, fa0, fa1, fb0, fb1);
+            }
+        }
+        ta = da; tb = db;
+    }
+}
+
+// ------------------------------------------------------------------------------------------
+// launch wrappers
+// ------------------------------------------------------------------------------------------
+
+cudaError_t launch_field_binop(int op, const imm_fe* x, const imm_fe* y, imm_fe* out, int64_t n,
+                               cudaStream_t st)
+{
+    if (n <= 0) return cudaSuccess;
+    int64_t blocks = (n + 255) / 256;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    field_binop_kernel<<<(unsigned)blocks, 256, 0, st>>>(op, x, y, out, n);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_eq_direct(const EqDirect& r, int nvars, imm_fe* out, cudaStream_t st)
+{
+    eq_direct_kernel<<<1, 1024, 0, st>>>(r, nvars, out);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_eq_batch(const EqTask* d_tasks, int ntasks, cudaStream_t st)
+{
+    if (ntasks <= 0) return cudaSuccess;
+    eq_batch_kernel<<<ntasks, 1024, 0, st>>>(d_tasks);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_rowbind(int dtype, bool point, const MatJob* d_jobs, int njobs, uint32_t ntiles,
+                           cudaStream_t st)
+{
+    if (ntiles == 0) return cudaSuccess;
+    if (dtype == 0) {
+        if (point) rowbind_kernel<int8_t, true><<<ntiles, ROWBIND_THREADS, 0, st>>>(d_jobs, njobs);
+        else rowbind_kernel<int8_t, false><<<ntiles, ROWBIND_THREADS, 0, st>>>(d_jobs, njobs);
+    } else {
+        if (point) rowbind_kernel<int32_t, true><<<ntiles, ROWBIND_THREADS, 0, st>>>(d_jobs, njobs);
+        else rowbind_kernel<int32_t, false><<<ntiles, ROWBIND_THREADS, 0, st>>>(d_jobs, njobs);
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_colbind(int dtype, const MatJob* d_jobs, int njobs, uint32_t ntiles, cudaStream_t st)
+{
+    if (ntiles == 0) return cudaSuccess;
+    if (dtype == 0) colbind_kernel<int8_t><<<ntiles, COLBIND_THREADS, 0, st>>>(d_jobs, njobs);
+    else colbind_kernel<int32_t><<<ntiles, COLBIND_THREADS, 0, st>>>(d_jobs, njobs);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_sum_parts(const imm_fe* parts, int nparts, int64_t len, imm_fe* out, cudaStream_t st)
+{
+    if (len <= 0) return cudaSuccess;
+    sum_parts_kernel<<<(unsigned)((len + 255) / 256), 256, 0, st>>>(parts, nparts, len, out);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_sum_all(const imm_fe* parts, int64_t count, imm_fe* out, cudaStream_t st)
+{
+    sum_all_kernel<<<1, 1024, 0, st>>>(parts, count, out);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_sumcheck(const ProofDev* d_proofs, int nproofs, uint64_t seed, imm_fe* transcripts,
+                            int64_t stride, int32_t* status, int max_b, cudaStream_t st)
+{
+    if (nproofs <= 0) return cudaSuccess;
+    int entries = max_b >= 1 ? (1 << (max_b - 1)) : 1;
+    if (entries > 8192) entries = 8192;                       // 2 tables x 8192 x 8 B = 128 KiB
+    const size_t smem = (size_t)entries * 2 * sizeof(uint64_t);
+    cudaError_t e = cudaFuncSetAttribute(sumcheck_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)smem);
+    if (e != cudaSuccess) return e;
+    sumcheck_kernel<<<nproofs, SUMCHECK_THREADS, smem, st>>>(d_proofs, seed, transcripts, stride, status,
+                                                             entries);
+    return cudaGetLastError();
+}
+
+}  // namespace imm

@@ -1,0 +1,292 @@
+"""Thin binding of the C-ABI CUDA library ``libimm.so`` (see ``include/imm.h``).
+
+Argument marshalling only: every function here checks tensor dtypes/devices, takes raw
+pointers and calls the library entry point of the same name.  PyTorch supplies device memory
+and the current stream, nothing else.  There is no CPU fallback: if the library is missing or
+a tensor is not on a CUDA device the call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import List, Optional, Sequence, Tuple
+
+import torch
+
+P = 0xFFFFFFFF00000001
+OK, REJECT = 0, 1
+I8, I32 = 0, 1
+BIND_ROWS, BIND_COLS = 0, 1
+FIELD_ADD, FIELD_SUB, FIELD_MUL = 0, 1, 2
+ERRORS = {-1: "IMM_ERR_ARG", -2: "IMM_ERR_SHAPE", -3: "IMM_ERR_ALIGN", -4: "IMM_ERR_WORKSPACE",
+          -5: "IMM_ERR_NONCANONICAL", -6: "IMM_ERR_CUDA"}
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libimm.so")
+
+EXPORTS = ("imm_version", "imm_last_cuda_error", "imm_challenge", "imm_field_binop", "imm_eq_table",
+           "imm_mle_workspace", "imm_mle_partial_eval", "imm_mle_eval_point",
+           "imm_sumcheck_matmul_workspace", "imm_sumcheck_matmul_prove",
+           "imm_sumcheck_matmul_host_arena", "imm_sumcheck_matmul_prove_host", "imm_sumcheck_verify")
+
+
+class ImmError(RuntimeError):
+    def __init__(self, code: int, where: str, detail: str = ""):
+        self.code = code
+        super().__init__(f"{where}: {ERRORS.get(code, code)}" + (f" ({detail})" if detail else ""))
+
+
+class MatmulDesc(ctypes.Structure):
+    _fields_ = [("A", ctypes.c_void_p), ("B", ctypes.c_void_p), ("C", ctypes.c_void_p),
+                ("m", ctypes.c_int64), ("k", ctypes.c_int64), ("n", ctypes.c_int64),
+                ("lda", ctypes.c_int64), ("ldb", ctypes.c_int64), ("ldc", ctypes.c_int64),
+                ("proof_id", ctypes.c_uint64)]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load libimm.so (built in-tree by ``paper_2602_22700_b200.build``); raises if absent."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2602_22700_b200.build`; "
+                          "there is no fallback path")
+    L = ctypes.CDLL(LIB_PATH)
+    vp, u64, i64, ci, sz = ctypes.c_void_p, ctypes.c_uint64, ctypes.c_int64, ctypes.c_int, ctypes.c_size_t
+    L.imm_version.restype = ci
+    L.imm_last_cuda_error.restype = ctypes.c_char_p
+    L.imm_challenge.restype = u64
+    L.imm_challenge.argtypes = [u64, u64, ctypes.c_uint32, ctypes.c_uint32]
+    L.imm_field_binop.restype = ci
+    L.imm_field_binop.argtypes = [ci, vp, vp, vp, i64, vp]
+    L.imm_eq_table.restype = ci
+    L.imm_eq_table.argtypes = [vp, ci, vp, vp]
+    L.imm_mle_workspace.restype = sz
+    L.imm_mle_workspace.argtypes = [ci, i64, i64, ci]
+    L.imm_mle_partial_eval.restype = ci
+    L.imm_mle_partial_eval.argtypes = [vp, ci, i64, i64, i64, ci, vp, vp, vp, sz, vp]
+    L.imm_mle_eval_point.restype = ci
+    L.imm_mle_eval_point.argtypes = [vp, ci, i64, i64, i64, vp, vp, vp, vp, sz, vp]
+    L.imm_sumcheck_matmul_workspace.restype = sz
+    L.imm_sumcheck_matmul_workspace.argtypes = [vp, ci]
+    L.imm_sumcheck_matmul_prove.restype = ci
+    L.imm_sumcheck_matmul_prove.argtypes = [vp, ci, u64, vp, i64, vp, vp, sz, vp]
+    L.imm_sumcheck_matmul_host_arena.restype = sz
+    L.imm_sumcheck_matmul_host_arena.argtypes = [vp, ci]
+    L.imm_sumcheck_matmul_prove_host.restype = ci
+    L.imm_sumcheck_matmul_prove_host.argtypes = [vp, ci, u64, vp, i64, vp, vp, sz, vp]
+    L.imm_sumcheck_verify.restype = ci
+    L.imm_sumcheck_verify.argtypes = [vp, ci, u64, u64, vp, vp, vp, vp]
+    _lib = L
+    return L
+
+
+def _check(rc: int, where: str):
+    if rc < 0:
+        detail = lib().imm_last_cuda_error().decode() if rc == -6 else ""
+        raise ImmError(rc, where, detail)
+    return rc
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _cuda(t: torch.Tensor, dtype, what: str) -> torch.Tensor:
+    if not isinstance(t, torch.Tensor) or t.device.type != "cuda":
+        raise ValueError(f"{what} must be a CUDA tensor (no CPU path exists)")
+    if t.dtype != dtype:
+        raise ValueError(f"{what} must have dtype {dtype}, got {t.dtype}")
+    return t
+
+
+def _matrix(t: torch.Tensor, what: str, device="cuda") -> Tuple[int, int, int, int, int]:
+    """(ptr, dtype code, rows, cols, ld) of a 2-D int8/int32 tensor with contiguous rows."""
+    if t.dim() != 2 or t.dtype not in (torch.int8, torch.int32):
+        raise ValueError(f"{what} must be a 2-D int8 or int32 tensor")
+    if t.device.type != device:
+        raise ValueError(f"{what} must live on {device}")
+    rows, cols = t.shape
+    if cols > 1 and t.stride(1) != 1:
+        raise ValueError(f"{what} must have unit column stride")
+    ld = t.stride(0) if rows > 1 else max(cols, 1)
+    return t.data_ptr(), (I8 if t.dtype == torch.int8 else I32), rows, cols, ld
+
+
+def ceil_log2(d: int) -> int:
+    return max(0, (int(d) - 1).bit_length())
+
+
+def transcript_len(k: int) -> int:
+    return 3 * ceil_log2(k) + 3
+
+
+def version() -> int:
+    return lib().imm_version()
+
+
+def challenge(seed: int, proof_id: int, domain: int, index: int) -> int:
+    return lib().imm_challenge(seed, proof_id, domain, index)
+
+
+def challenges(seed: int, proof_id: int, domain: int, count: int) -> List[int]:
+    return [challenge(seed, proof_id, domain, i) for i in range(count)]
+
+
+def field_binop(op: int, x: torch.Tensor, y: torch.Tensor) -> torch.Tensor:
+    """Element-wise field add/sub/mul of two int64 CUDA tensors holding canonical bit patterns."""
+    _cuda(x, torch.int64, "x"); _cuda(y, torch.int64, "y")
+    x, y = x.contiguous(), y.contiguous()
+    assert x.numel() == y.numel()
+    out = torch.empty_like(x)
+    _check(lib().imm_field_binop(op, x.data_ptr(), y.data_ptr(), out.data_ptr(), x.numel(), _stream()),
+           "imm_field_binop")
+    return out
+
+
+def eq_table(r: Sequence[int], device="cuda") -> torch.Tensor:
+    """E[i] = eq(r, i) as an int64 CUDA tensor of 2^len(r) canonical bit patterns."""
+    n = len(r)
+    arr = (ctypes.c_uint64 * max(n, 1))(*[int(v) for v in r])
+    out = torch.empty(1 << min(n, 24), dtype=torch.int64, device=device)
+    _check(lib().imm_eq_table(ctypes.addressof(arr), n, out.data_ptr(), _stream()), "imm_eq_table")
+    return out
+
+
+def mle_workspace(dtype_code: int, rows: int, cols: int, bind: int) -> int:
+    return lib().imm_mle_workspace(dtype_code, rows, cols, bind)
+
+
+def mle_partial_eval(mat: torch.Tensor, bind: int, eq: torch.Tensor,
+                     ws: Optional[torch.Tensor] = None) -> torch.Tensor:
+    ptr, code, rows, cols, ld = _matrix(mat, "mat")
+    _cuda(eq, torch.int64, "eq")
+    need = mle_workspace(code, rows, cols, bind)
+    if ws is None:
+        ws = torch.empty(max(need, 16), dtype=torch.uint8, device=mat.device)
+    out = torch.empty(cols if bind == BIND_ROWS else rows, dtype=torch.int64, device=mat.device)
+    _check(lib().imm_mle_partial_eval(ptr, code, rows, cols, ld, bind, eq.data_ptr(), out.data_ptr(),
+                                      ws.data_ptr(), ws.numel(), _stream()), "imm_mle_partial_eval")
+    return out
+
+
+def mle_eval_point(mat: torch.Tensor, eq_row: torch.Tensor, eq_col: torch.Tensor,
+                   ws: Optional[torch.Tensor] = None) -> torch.Tensor:
+    ptr, code, rows, cols, ld = _matrix(mat, "mat")
+    _cuda(eq_row, torch.int64, "eq_row"); _cuda(eq_col, torch.int64, "eq_col")
+    need = mle_workspace(code, rows, cols, BIND_ROWS)
+    if ws is None:
+        ws = torch.empty(max(need, 16), dtype=torch.uint8, device=mat.device)
+    out = torch.empty(1, dtype=torch.int64, device=mat.device)
+    _check(lib().imm_mle_eval_point(ptr, code, rows, cols, ld, eq_row.data_ptr(), eq_col.data_ptr(),
+                                    out.data_ptr(), ws.data_ptr(), ws.numel(), _stream()),
+           "imm_mle_eval_point")
+    return out
+
+
+def make_descs(problems, device="cuda"):
+    """ctypes descriptor array for (A, B, C, proof_id) tuples; tensors must stay alive."""
+    arr = (MatmulDesc * len(problems))()
+    for i, (A, B, C, pid) in enumerate(problems):
+        pa, ca, m, k, lda = _matrix(A, "A", device)
+        pb, cb, k2, n, ldb = _matrix(B, "B", device)
+        pc, cc, m2, n2, ldc = _matrix(C, "C", device)
+        if ca != I8 or cb != I8 or cc != I32 or k != k2 or m != m2 or n != n2:
+            raise ValueError("need A int8 m x k, B int8 k x n, C int32 m x n")
+        arr[i] = MatmulDesc(pa, pb, pc, m, k, n, lda, ldb, ldc, int(pid))
+    return arr
+
+
+def sumcheck_matmul_workspace(descs) -> int:
+    return lib().imm_sumcheck_matmul_workspace(ctypes.addressof(descs), len(descs))
+
+
+class Prover:
+    """Holds the descriptor array, workspace and output buffers of one batch so that repeated
+    ``prove`` calls do no allocation.  ``problems``: list of (A, B, C, proof_id) CUDA tensors."""
+
+    def __init__(self, problems, device="cuda"):
+        self.problems = list(problems)
+        self.descs = make_descs(self.problems)
+        self.nproofs = len(self.problems)
+        self.stride = max(transcript_len(A.shape[1]) for (A, _, _, _) in self.problems)
+        need = sumcheck_matmul_workspace(self.descs)
+        if need == 0:
+            raise ImmError(-2, "imm_sumcheck_matmul_workspace")
+        self.ws = torch.empty(need, dtype=torch.uint8, device=device)
+        self.transcripts = torch.zeros((self.nproofs, self.stride), dtype=torch.int64, device=device)
+        self.status = torch.full((self.nproofs,), -99, dtype=torch.int32, device=device)
+
+    def prove(self, seed: int) -> torch.Tensor:
+        """Enqueue one proving pass on the current stream; returns the device transcript tensor."""
+        _check(lib().imm_sumcheck_matmul_prove(ctypes.addressof(self.descs), self.nproofs, seed,
+                                               self.transcripts.data_ptr(), self.stride,
+                                               self.status.data_ptr(), self.ws.data_ptr(),
+                                               self.ws.numel(), _stream()), "imm_sumcheck_matmul_prove")
+        return self.transcripts
+
+    def lengths(self) -> List[int]:
+        return [transcript_len(A.shape[1]) for (A, _, _, _) in self.problems]
+
+
+def sumcheck_matmul_prove(problems, seed: int) -> List[List[int]]:
+    """Convenience: prove a batch and return each proof's transcript as Python ints (synchronises)."""
+    pr = Prover(problems)
+    t = pr.prove(seed)
+    torch.cuda.synchronize()
+    if int(pr.status.abs().max()) != 0:
+        raise ImmError(int(pr.status.min()), "device status")
+    host = t.cpu()
+    return [[int(v) & 0xFFFFFFFFFFFFFFFF for v in host[i, :n]] for i, n in enumerate(pr.lengths())]
+
+
+class HostProver:
+    """End-to-end variant: matrices live in (pinned) HOST tensors; every ``prove`` copies them to a
+    device arena, proves, and copies the transcripts back (synchronous)."""
+
+    def __init__(self, problems, device="cuda"):
+        self.problems = list(problems)
+        self.descs = make_descs(self.problems, device="cpu")
+        self.nproofs = len(self.problems)
+        self.stride = max(transcript_len(A.shape[1]) for (A, _, _, _) in self.problems)
+        need = lib().imm_sumcheck_matmul_host_arena(ctypes.addressof(self.descs), self.nproofs)
+        if need == 0:
+            raise ImmError(-2, "imm_sumcheck_matmul_host_arena")
+        self.arena = torch.empty(need, dtype=torch.uint8, device=device)
+        self.transcripts = torch.zeros((self.nproofs, self.stride), dtype=torch.int64).pin_memory()
+        self.status = torch.full((self.nproofs,), -99, dtype=torch.int32).pin_memory()
+        self.h2d_bytes = sum(A.numel() + B.numel() + 4 * C.numel() for (A, B, C, _) in self.problems)
+        self.d2h_bytes = self.transcripts.numel() * 8 + self.status.numel() * 4
+
+    def prove(self, seed: int) -> torch.Tensor:
+        _check(lib().imm_sumcheck_matmul_prove_host(ctypes.addressof(self.descs), self.nproofs, seed,
+                                                    self.transcripts.data_ptr(), self.stride,
+                                                    self.status.data_ptr(), self.arena.data_ptr(),
+                                                    self.arena.numel(), _stream()),
+               "imm_sumcheck_matmul_prove_host")
+        return self.transcripts
+
+
+def sumcheck_verify(transcript: Sequence[int], nrounds: int, seed: int, proof_id: int,
+                    expect_c0: Optional[int] = None, expect_a_fin: Optional[int] = None,
+                    expect_b_fin: Optional[int] = None) -> Tuple[int, int]:
+    """Host verifier; returns (status, fail_at)."""
+    n = 3 * nrounds + 3
+    arr = (ctypes.c_uint64 * n)(*[int(v) & 0xFFFFFFFFFFFFFFFF for v in list(transcript)[:n]])
+    keep = []
+
+    def opt(v):
+        if v is None:
+            return None
+        box = ctypes.c_uint64(int(v))
+        keep.append(box)
+        return ctypes.addressof(box)
+
+    fail = ctypes.c_int(-2)
+    rc = lib().imm_sumcheck_verify(ctypes.addressof(arr), nrounds, seed, proof_id, opt(expect_c0),
+                                   opt(expect_a_fin), opt(expect_b_fin), ctypes.addressof(fail))
+    _check(rc, "imm_sumcheck_verify")
+    return rc, fail.value

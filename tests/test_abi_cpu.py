@@ -1,0 +1,121 @@
+"""Host-side checks of the C-ABI library that need no GPU: it loads, exports every declared
+symbol, and its host entry points (challenge generator, verifier, planners, argument
+validation) agree with the oracle."""
+import ctypes
+import os
+import random
+import re
+
+import numpy as np
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def imm():
+    from paper_2602_22700_b200 import build, imm as binding
+    build.build()
+    return binding
+
+
+def test_library_exports_every_declared_symbol(imm):
+    header = open(os.path.join(ROOT, "include", "imm.h")).read()
+    declared = set(re.findall(r"\b(imm_[a-z0-9_]+)\s*\(", header))
+    declared -= {"imm_matmul_desc"}
+    assert declared == set(imm.EXPORTS)
+    L = imm.lib()
+    for name in declared:
+        assert getattr(L, name) is not None
+    assert imm.version() >= 100
+
+
+def test_challenges_match_oracle(imm, oracle):
+    rng = random.Random(1)
+    for _ in range(200):
+        seed, pid = rng.getrandbits(64), rng.getrandbits(64)
+        dom, idx = rng.choice((1, 2, 3)), rng.randrange(0, 40)
+        assert imm.challenge(seed, pid, dom, idx) == oracle.challenge(seed, pid, dom, idx)
+    assert imm.challenge(1, 0, 1, 0) == 0x0F583436CC1AB29E
+
+
+def test_host_verifier_matches_oracle_verifier(imm, oracle):
+    rng = random.Random(2)
+    for (m, k, n) in ((3, 8, 2), (2, 5, 4), (4, 1, 4), (1, 16, 1)):
+        A = np.array([[rng.randint(-128, 127) for _ in range(k)] for _ in range(m)], dtype=np.int8)
+        B = np.array([[rng.randint(-128, 127) for _ in range(n)] for _ in range(k)], dtype=np.int8)
+        C = (A.astype(np.int64) @ B.astype(np.int64)).astype(np.int32)
+        seed, pid = rng.getrandbits(64), rng.getrandbits(20)
+        t = [int(w) for w in oracle.sumcheck_matmul_prove(A, B, C, seed, pid)]
+        b = oracle.ceil_log2(k)
+        assert imm.sumcheck_verify(t, b, seed, pid) == (imm.OK, -1)
+        assert imm.sumcheck_verify(t, b, seed, pid, t[0], t[-2], t[-1]) == (imm.OK, -1)
+        for pos in range(len(t)):
+            bad = list(t)
+            bad[pos] = (bad[pos] + 1 + rng.randrange(oracle.P - 1)) % oracle.P
+            assert imm.sumcheck_verify(bad, b, seed, pid) == oracle.sumcheck_verify(bad, b, seed, pid)
+            assert imm.sumcheck_verify(bad, b, seed, pid)[0] == imm.REJECT
+        for which in range(3):
+            exp = [t[0], t[-2], t[-1]]
+            exp[which] = (exp[which] + 1) % oracle.P
+            assert imm.sumcheck_verify(t, b, seed, pid, *exp) == oracle.sumcheck_verify(t, b, seed, pid, *exp)
+            assert imm.sumcheck_verify(t, b, seed, pid, *exp) == (imm.REJECT, b + 1 + which)
+        assert imm.sumcheck_verify(t, b, seed + 1, pid)[0] == (imm.REJECT if b > 0 else imm.OK)
+    with pytest.raises(imm.ImmError):
+        imm.sumcheck_verify([oracle.P, 0, 0], 0, 1, 0)
+
+
+def _desc_array(imm, shapes, base=0x10000):
+    arr = (imm.MatmulDesc * len(shapes))()
+    for i, (m, k, n) in enumerate(shapes):
+        arr[i] = imm.MatmulDesc(base, base, base, m, k, n, k, n, n, i)
+    return arr
+
+
+def test_workspace_planner(imm):
+    L = imm.lib()
+    d = _desc_array(imm, [(64, 64, 64)])
+    w1 = L.imm_sumcheck_matmul_workspace(ctypes.addressof(d), 1)
+    assert w1 > 0 and w1 % 256 == 0
+    d2 = _desc_array(imm, [(64, 64, 64), (512, 4096, 4096)])
+    w2 = L.imm_sumcheck_matmul_workspace(ctypes.addressof(d2), 2)
+    assert w2 > w1
+    # eq tables + tables of the rounds are the floor
+    assert w2 >= 8 * (512 + 4096 + 2 * 4096)
+    for bad in ([(0, 4, 4)], [(4, 0, 4)], [(4, 4, 0)], [(4, (1 << 17) + 1, 4)], [((1 << 20) + 1, 4, 4)]):
+        db = _desc_array(imm, bad)
+        assert L.imm_sumcheck_matmul_workspace(ctypes.addressof(db), 1) == 0
+    assert L.imm_sumcheck_matmul_workspace(None, 1) == 0
+    assert L.imm_sumcheck_matmul_host_arena(ctypes.addressof(d2), 2) > w2 + 512 * 4096 + 4096 * 4096
+    assert L.imm_mle_workspace(0, 100, 100, 0) > 0 and L.imm_mle_workspace(2, 100, 100, 0) == 0
+    assert L.imm_mle_workspace(1, 0, 100, 1) == 0
+
+
+def test_argument_validation_happens_before_any_device_work(imm):
+    L = imm.lib()
+    r = (ctypes.c_uint64 * 4)(1, 2, 3, imm.P)
+    assert L.imm_eq_table(ctypes.addressof(r), 21, 0x1000, None) == -2
+    assert L.imm_eq_table(ctypes.addressof(r), 4, None, None) == -1
+    assert L.imm_eq_table(ctypes.addressof(r), 4, 0x1008, None) == -3
+    assert L.imm_eq_table(ctypes.addressof(r), 4, 0x1000, None) == -5
+    assert L.imm_field_binop(7, 0x1000, 0x1000, 0x1000, 4, None) == -1
+    assert L.imm_field_binop(0, None, None, None, 0, None) == 0
+    assert L.imm_mle_partial_eval(0x1000, 0, 4, 8, 7, 0, 0x1000, 0x1000, 0x1000, 1 << 20, None) == -2
+    assert L.imm_mle_partial_eval(0x1000, 5, 4, 8, 8, 0, 0x1000, 0x1000, 0x1000, 1 << 20, None) == -1
+    assert L.imm_mle_partial_eval(0x1000, 0, 4, 8, 8, 0, 0x1000, 0x1000, 0x1000, 8, None) == -4
+    assert L.imm_mle_eval_point(0x1000, 1, 4, 8, 8, 0x1000, 0x1000, 0x1000, 0x1004, 1 << 20, None) == -3
+    d = _desc_array(imm, [(4, 8, 4)])
+    assert L.imm_sumcheck_matmul_prove(ctypes.addressof(d), 1, 1, 0x1000, 11, 0x1000, 0x1000, 1 << 30, None) == -2
+    assert L.imm_sumcheck_matmul_prove(ctypes.addressof(d), 1, 1, 0x1000, 12, 0x1000, 0x1000, 16, None) == -4
+    assert L.imm_sumcheck_matmul_prove(ctypes.addressof(d), 0, 1, 0x1000, 12, 0x1000, 0x1000, 1 << 30, None) == -1
+    d.__getitem__(0).lda = 7
+    assert L.imm_sumcheck_matmul_prove(ctypes.addressof(d), 1, 1, 0x1000, 12, 0x1000, 0x1000, 1 << 30, None) == -2
+
+
+def test_binding_refuses_cpu_tensors(imm):
+    import torch
+    A = torch.zeros((4, 4), dtype=torch.int8)
+    with pytest.raises(ValueError):
+        imm.make_descs([(A, A, A.to(torch.int32), 0)])
+    with pytest.raises(ValueError):
+        imm.mle_partial_eval(A, imm.BIND_ROWS, torch.zeros(4, dtype=torch.int64))

@@ -1,0 +1,375 @@
+#!/usr/bin/env python
+"""Throughput of the sumcheck matmul prover on synthetic transformer-shaped layers.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+                    [--layers L] [--tokens T] [--no-e2e] [--no-cpu-baseline]
+
+One step = one proving pass over the whole batch: eq tables, A~ / B~ partial evaluations, the
+claim C~, every sumcheck round, transcripts written.  The default workload is the audited decoder
+block: 32 layers x (QKV 4096x6144, O 4096x4096, FFN up 4096x14336, FFN down 14336x4096) at 8192
+tokens, 128 proofs, 39.25 GiB of int8/int32 inputs resident in HBM (far larger than L2, so no
+flush is needed between steps).  Rank 0 prints ONE JSON line.
+
+--impl reference times the plain CPU oracle on the host cores, on a bounded sample of the same
+workload.  With N > 1 (launched by torch.distributed.run) every rank proves an independent
+replica of the workload on its own GPU: the path has no exchange step, so no collective is used
+beyond the timing barrier.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+from concurrent.futures import ThreadPoolExecutor
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+METRIC = "proved field-MACs/sec"
+UNIT = "field-MAC/s"
+SEED = 1
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--layers", type=int, default=32)
+    ap.add_argument("--tokens", type=int, default=8192)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    return ap.parse_args()
+
+
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), int(os.environ.get("WORLD_SIZE", 1))
+
+
+def workload_name(layers, tokens):
+    return f"audited decoder block: {layers} layers x (QKV 4096x6144, O 4096x4096, FFN 4096x14336 x2), {tokens} tokens"
+
+
+# ------------------------------------------------------------------------ clocks sampling
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append((time.time(), line.strip()))
+
+    def stop(self, t0: float, t1: float):
+        if self.proc is None:
+            return None
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        rows = [l for (t, l) in self.lines if t0 <= t <= t1 + 0.1] or [l for (_, l) in self.lines[-3:]]
+        sm, smax, reasons, power = [], [], set(), []
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for l in rows:
+            f = [x.strip() for x in l.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0])); smax.append(float(f[1])); power.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, v in zip(names, f[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        if not sm:
+            return None
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": max(smax), "power_w_max": max(power),
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------ oracle timing
+
+
+def oracle_time_sample(sample, threads):
+    """Wall seconds the CPU oracle takes to prove `sample` (numpy A, B, C, proof_id tuples) with one
+    proof per thread; returns (seconds, transcripts)."""
+    import oracle
+
+    def one(p):
+        A, B, C, pid = p
+        return oracle.sumcheck_matmul_prove(A, B, C, SEED, pid)
+
+    t0 = time.perf_counter()
+    with ThreadPoolExecutor(max_workers=threads) as ex:
+        out = list(ex.map(one, sample))
+    return time.perf_counter() - t0, out
+
+
+def field_macs(shapes):
+    return sum(m * k + k * n + m * n + 5 * (1 << max(0, (k - 1).bit_length())) for (m, k, n) in shapes)
+
+
+def sample_to_host(problems):
+    return [(p.A.cpu().numpy(), p.B.cpu().numpy(), p.C.cpu().numpy(), p.proof_id) for p in problems]
+
+
+def mem_available_bytes():
+    try:
+        with open("/proc/meminfo") as f:
+            for line in f:
+                if line.startswith("MemAvailable:"):
+                    return int(line.split()[1]) * 1024
+    except OSError:
+        pass
+    return 0
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except (OSError, KeyError, ValueError):
+        return 6650.0, "fallback"
+
+
+# DRAM traffic of the claim kernel per algorithmic byte, from the ncu capture summarised under
+# profiles/ (dram__bytes_read.sum + dram__bytes_write.sum over 4*m*n); None until a capture of the
+# current kernel exists.
+CLAIM_KERNEL_TRAFFIC_RATIO = None
+
+
+# ------------------------------------------------------------------------ our arm
+
+
+def run_ours(args):
+    from paper_2602_22700_b200 import imm, synth
+    rank, local_rank, world = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the prover has no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    imm.lib()
+    warmup = max(args.warmup, 3)
+    steps = max(args.steps, 1)
+
+    problems = synth.decoder_block(SEED + rank, args.layers, args.tokens, device=dev)
+    shapes = [p.mkn for p in problems]
+    macs = synth.prover_field_macs(problems)
+    algo_bytes = synth.problem_bytes(problems)
+    claim_bytes = sum(4 * m * n for (m, k, n) in shapes)
+    prover = imm.Prover([(p.A, p.B, p.C, p.proof_id) for p in problems], device=dev)
+    imm.profile_enable(min(4096, warmup + steps + 4))
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(warmup):
+        prover.prove(SEED)
+    barrier()
+    sampler = ClockSampler(local_rank if "CUDA_VISIBLE_DEVICES" not in os.environ else
+                           int(os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local_rank]))
+    sampler.start()
+    time.sleep(0.25)
+    first_call = imm.profile_calls()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.time()
+    ev0.record()
+    for _ in range(steps):
+        prover.prove(SEED)
+    ev1.record()
+    barrier()
+    t1 = time.time()
+    clocks = sampler.stop(t0, t1)
+    elapsed_ms = ev0.elapsed_time(ev1)
+    if dist is not None:
+        t = torch.tensor([elapsed_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(t.item())
+    phase_ms = [0.0] * len(imm.PROFILE_PHASES)
+    for c in range(first_call, first_call + steps):
+        for i, v in enumerate(imm.profile_read(c)):
+            phase_ms[i] += v / steps
+    imm.profile_enable(0)
+
+    # every proof of the timed batch must be accepted by the verifier
+    host_t = prover.transcripts.cpu()
+    assert int(prover.status.abs().max()) == 0
+    accepted = 0
+    for i, p in enumerate(problems):
+        b = imm.ceil_log2(p.A.shape[1])
+        words = [int(v) & 0xFFFFFFFFFFFFFFFF for v in host_t[i, :3 * b + 3]]
+        if imm.sumcheck_verify(words, b, SEED, p.proof_id) == (imm.OK, -1):
+            accepted += 1
+    if accepted != len(problems):
+        raise SystemExit(f"only {accepted}/{len(problems)} proofs verified")
+
+    ms_per_step = elapsed_ms / steps
+    value = macs * world / (ms_per_step * 1e-3)
+    peak, peak_kind = measured_peaks()
+    claim_gbs = claim_bytes / (phase_ms[1] * 1e-3) / 1e9
+    phase_bytes = [0, claim_bytes, sum(m * k for (m, k, n) in shapes), sum(k * n for (m, k, n) in shapes), 0]
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "u64", "data": "synthetic",
+        "config": {"workload": workload_name(args.layers, args.tokens), "layers": args.layers,
+                   "tokens": args.tokens, "proofs_per_gpu": len(problems), "field": "Goldilocks 2^64-2^32+1",
+                   "input_bytes_per_gpu": algo_bytes, "l2": "inputs (39 GiB at the default size) far exceed the 126 MB L2; no flush",
+                   "parallelism": "1 GPU" if world == 1 else f"{world} independent replicas, no collective"},
+        "layers_per_s": args.layers * world / (ms_per_step * 1e-3),
+        "proofs_per_s": len(problems) * world / (ms_per_step * 1e-3),
+        "proved_matmul_macs_per_s": synth.proved_matmul_macs(problems) * world / (ms_per_step * 1e-3),
+        "hbm_gbs_whole_step": algo_bytes / (ms_per_step * 1e-3) / 1e9,
+        "hbm_frac_of_8tbs_whole_step": algo_bytes / (ms_per_step * 1e-3) / 8e12,
+        "proofs_verified": accepted,
+        "phases": {name: {"ms": phase_ms[i],
+                          "gbs": (phase_bytes[i] / (phase_ms[i] * 1e-3) / 1e9) if phase_bytes[i] and phase_ms[i] > 0 else None}
+                   for i, name in enumerate(imm.PROFILE_PHASES)},
+        "roofline": {"kernel": "rowbind_kernel<int32,POINT> (claim C~)", "bound": "hbm", "achieved": claim_gbs,
+                     "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": claim_gbs / peak,
+                     "frac_of_8tbs": claim_gbs / 8000.0,
+                     "traffic": (CLAIM_KERNEL_TRAFFIC_RATIO * claim_bytes) if CLAIM_KERNEL_TRAFFIC_RATIO else None},
+        "gpu_launches": 5 * steps,
+        "clocks": clocks,
+    }
+
+    # ---- end to end: pinned host inputs -> device arena -> proofs -> host transcripts
+    e2e = None
+    if not args.no_e2e:
+        need = algo_bytes
+        if mem_available_bytes() < int(1.25 * need * (world if world > 1 else 1)):
+            e2e = {"value": None, "unit": UNIT, "skipped": "not enough host memory for pinned inputs"}
+        else:
+            host = []
+            for p in problems:
+                host.append(tuple(torch.empty(t.shape, dtype=t.dtype, pin_memory=True).copy_(t)
+                                  for t in (p.A, p.B, p.C)) + (p.proof_id,))
+            torch.cuda.synchronize()
+            hp = imm.HostProver(host, device=dev)
+            hp.prove(SEED)                                   # warm-up (page-locks, first touch of the arena)
+            barrier()
+            k2 = max(1, args.e2e_steps)
+            w0 = time.perf_counter()
+            for _ in range(k2):
+                hp.prove(SEED)                               # synchronous: returns after the D2H copy
+            e2e_s = (time.perf_counter() - w0) / k2
+            if dist is not None:
+                t = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
+                dist.all_reduce(t, op=dist.ReduceOp.MAX)
+                e2e_s = float(t.item())
+            same = bool((hp.transcripts == host_t).all())
+            e2e = {"value": macs * world / e2e_s, "unit": UNIT, "ms_per_step": e2e_s * 1e3, "steps": k2,
+                   "h2d_bytes_per_step": hp.h2d_bytes, "d2h_bytes_per_step": hp.d2h_bytes,
+                   "matches_device_path": same}
+            del hp, host
+    out["e2e"] = e2e
+
+    # ---- the oracle beside it (rank 0, single GPU): first two layers' proofs, one per thread
+    if not args.no_cpu_baseline and world == 1:
+        nsample = min(len(problems), 8)
+        sample = sample_to_host(problems[:nsample])
+        threads = min(os.cpu_count() or 1, nsample)
+        secs, want = oracle_time_sample(sample, threads)
+        ok = all([int(v) & 0xFFFFFFFFFFFFFFFF for v in host_t[i, :len(w)]] == [int(x) for x in w]
+                 for i, w in enumerate(want))
+        out["cpu_baseline"] = {"value": field_macs(shapes[:nsample]) / secs, "unit": UNIT, "cores": threads,
+                               "kind": "oracle", "seconds": secs,
+                               "sample": f"the first {nsample} of the {len(problems)} proofs (layers 0-{(nsample - 1) // 4}), "
+                                         f"one proof per thread, same inputs as the GPU run",
+                               "gpu_transcripts_match": ok}
+        if not ok:
+            raise SystemExit("GPU transcripts differ from the oracle on the sampled proofs")
+    if rank == 0:
+        print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+# ------------------------------------------------------------------------ reference arm (CPU oracle)
+
+
+def run_reference(args):
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    from paper_2602_22700_b200 import synth
+    device = "cuda" if torch.cuda.is_available() else "cpu"
+    layers = min(args.layers, 2)
+    tokens = args.tokens if device == "cuda" else min(args.tokens, 256)
+    problems = synth.decoder_block(SEED, layers, tokens, device=device)
+    sample = sample_to_host(problems)
+    shapes = [p.mkn for p in problems]
+    del problems
+    threads = min(os.cpu_count() or 1, len(sample))
+    macs = field_macs(shapes)
+    warmup, steps = max(args.warmup, 1), max(args.steps, 1)
+    for _ in range(warmup):
+        oracle_time_sample(sample, threads)
+    total = 0.0
+    for _ in range(steps):
+        secs, _ = oracle_time_sample(sample, threads)
+        total += secs
+    per = total / steps
+    value = macs / per
+    desc = (f"{len(sample)} proofs (layers 0-{layers - 1} of the block at {tokens} tokens) per step, "
+            f"one proof per thread")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world,
+        "steps": steps, "warmup": warmup, "ms_per_step": per * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "u64", "data": "synthetic",
+        "config": {"workload": workload_name(args.layers, args.tokens), "layers": args.layers,
+                   "tokens": args.tokens, "sampled": desc,
+                   "note": None if tokens == args.tokens else "no CUDA device for input generation: token count reduced"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -152,6 +152,23 @@ int imm_sumcheck_matmul_prove(const imm_matmul_desc* descs_host, int nproofs, ui
                               imm_fe* d_transcripts, int64_t stride, int32_t* d_status,
                               void* d_ws, size_t ws_bytes, void* stream);
 
+/* Phase timing of imm_sumcheck_matmul_prove, for measurement.  While enabled, every prove call
+ * records CUDA events on its stream around each of its five launches, into the next of
+ * `capacity` event sets (a ring), without synchronising.  Phases:
+ *   [0] eq tables, [1] claim C~ (int32 point contraction), [2] A~ row binding,
+ *   [3] B~ column binding, [4] sumcheck rounds.
+ * The event ring is per process; profiled calls must not overlap on different host threads.
+ * imm_profile_enable(capacity): capacity in 1..4096 creates the ring and resets the call count
+ *   (needs a CUDA device); capacity 0 destroys it.
+ * imm_profile_calls(): profiled prove calls since the ring was created.
+ * imm_profile_read(call, ms_host, count): waits for profiled call number `call` (0-based) to
+ *   finish and writes its elapsed milliseconds per phase; count must be IMM_PROFILE_PHASES.
+ *   IMM_ERR_ARG if profiling is off or the call is not (or no longer) in the ring. */
+#define IMM_PROFILE_PHASES 5
+int imm_profile_enable(int capacity);
+int64_t imm_profile_calls(void);
+int imm_profile_read(int64_t call, float* ms_host, int count);
+
 /* Device arena bytes imm_sumcheck_matmul_prove_host needs: staged copies of all matrices, the
  * transcripts and status words, and the prover workspace (0 on invalid input). */
 size_t imm_sumcheck_matmul_host_arena(const imm_matmul_desc* descs_host, int nproofs);

@@ -182,6 +182,11 @@ Plan make_plan(const imm_matmul_desc* descs, int nproofs)
     return p;
 }
 
+// phase-timing events (see imm_profile_enable)
+constexpr int PROF_EV = IMM_PROFILE_PHASES + 1;
+std::vector<cudaEvent_t> g_prof_ev;        // capacity * PROF_EV events, empty when profiling is off
+int64_t g_prof_calls = 0;
+
 int check_stride(const imm_matmul_desc* descs, int nproofs, int64_t stride)
 {
     for (int i = 0; i < nproofs; i++)
@@ -309,6 +314,38 @@ int imm_mle_eval_point(const void* d_mat, int dtype, int64_t rows, int64_t cols,
     return IMM_OK;
 }
 
+int imm_profile_enable(int capacity)
+{
+    if (capacity < 0 || capacity > 4096) return IMM_ERR_ARG;
+    for (cudaEvent_t e : g_prof_ev) cudaEventDestroy(e);
+    g_prof_ev.clear();
+    g_prof_calls = 0;
+    if (capacity == 0) return IMM_OK;
+    std::vector<cudaEvent_t> ev((size_t)capacity * PROF_EV);
+    for (size_t i = 0; i < ev.size(); i++) {
+        cudaError_t e = cudaEventCreate(&ev[i]);
+        if (e != cudaSuccess) {
+            for (size_t j = 0; j < i; j++) cudaEventDestroy(ev[j]);
+            return cuda_fail(e);
+        }
+    }
+    g_prof_ev.swap(ev);
+    return IMM_OK;
+}
+
+int64_t imm_profile_calls(void) { return g_prof_calls; }
+
+int imm_profile_read(int64_t call, float* ms_host, int count)
+{
+    if (!ms_host || count != IMM_PROFILE_PHASES || g_prof_ev.empty()) return IMM_ERR_ARG;
+    const int64_t cap = (int64_t)(g_prof_ev.size() / PROF_EV);
+    if (call < 0 || call >= g_prof_calls || call < g_prof_calls - cap) return IMM_ERR_ARG;
+    cudaEvent_t* ev = &g_prof_ev[(size_t)(call % cap) * PROF_EV];
+    CU(cudaEventSynchronize(ev[IMM_PROFILE_PHASES]));
+    for (int i = 0; i < IMM_PROFILE_PHASES; i++) CU(cudaEventElapsedTime(&ms_host[i], ev[i], ev[i + 1]));
+    return IMM_OK;
+}
+
 size_t imm_sumcheck_matmul_workspace(const imm_matmul_desc* descs_host, int nproofs)
 {
     Plan p = make_plan(descs_host, nproofs);
@@ -368,13 +405,25 @@ int imm_sumcheck_matmul_prove(const imm_matmul_desc* descs_host, int nproofs, ui
     }
     if (ta != p.tiles_a || tb != p.tiles_b || tc != p.tiles_c) return IMM_ERR_ARG;   // planner invariant
 
+    const bool prof = !g_prof_ev.empty();
+    cudaEvent_t* pev = prof ? &g_prof_ev[(size_t)(g_prof_calls % (int64_t)(g_prof_ev.size() / PROF_EV)) * PROF_EV]
+                            : nullptr;
+#define PROF_MARK(i) do { if (prof) CU(cudaEventRecord(pev[i], st)); } while (0)
     CU(cudaMemcpyAsync(base, hdr.data(), hdr.size(), cudaMemcpyHostToDevice, st));
+    PROF_MARK(0);
     CU(launch_eq_batch((const EqTask*)(base + p.off_eq), 2 * nproofs, st));
+    PROF_MARK(1);
     CU(launch_rowbind(IMM_I32, true, (const MatJob*)(base + p.off_jobs_c), nproofs, p.tiles_c, st));
+    PROF_MARK(2);
     CU(launch_rowbind(IMM_I8, false, (const MatJob*)(base + p.off_jobs_a), nproofs, p.tiles_a, st));
+    PROF_MARK(3);
     CU(launch_colbind(IMM_I8, (const MatJob*)(base + p.off_jobs_b), nproofs, p.tiles_b, st));
+    PROF_MARK(4);
     CU(launch_sumcheck((const ProofDev*)(base + p.off_proofs), nproofs, seed, d_transcripts, stride,
                        d_status, p.max_b, st));
+    PROF_MARK(5);
+#undef PROF_MARK
+    if (prof) g_prof_calls++;
     return IMM_OK;
 }
 

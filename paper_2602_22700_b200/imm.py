@@ -27,7 +27,9 @@ LIB_PATH = os.path.join(_HERE, "libimm.so")
 EXPORTS = ("imm_version", "imm_last_cuda_error", "imm_challenge", "imm_field_binop", "imm_eq_table",
            "imm_mle_workspace", "imm_mle_partial_eval", "imm_mle_eval_point",
            "imm_sumcheck_matmul_workspace", "imm_sumcheck_matmul_prove",
-           "imm_sumcheck_matmul_host_arena", "imm_sumcheck_matmul_prove_host", "imm_sumcheck_verify")
+           "imm_sumcheck_matmul_host_arena", "imm_sumcheck_matmul_prove_host", "imm_sumcheck_verify",
+           "imm_profile_enable", "imm_profile_calls", "imm_profile_read")
+PROFILE_PHASES = ("eq_tables", "claim_C", "bind_rows_A", "bind_cols_B", "sumcheck_rounds")
 
 
 class ImmError(RuntimeError):
@@ -78,6 +80,12 @@ def lib() -> ctypes.CDLL:
     L.imm_sumcheck_matmul_host_arena.argtypes = [vp, ci]
     L.imm_sumcheck_matmul_prove_host.restype = ci
     L.imm_sumcheck_matmul_prove_host.argtypes = [vp, ci, u64, vp, i64, vp, vp, sz, vp]
+    L.imm_profile_enable.restype = ci
+    L.imm_profile_enable.argtypes = [ci]
+    L.imm_profile_calls.restype = i64
+    L.imm_profile_calls.argtypes = []
+    L.imm_profile_read.restype = ci
+    L.imm_profile_read.argtypes = [i64, vp, ci]
     L.imm_sumcheck_verify.restype = ci
     L.imm_sumcheck_verify.argtypes = [vp, ci, u64, u64, vp, vp, vp, vp]
     _lib = L
@@ -268,6 +276,22 @@ class HostProver:
                                                     self.arena.numel(), _stream()),
                "imm_sumcheck_matmul_prove_host")
         return self.transcripts
+
+
+def profile_enable(capacity: int) -> None:
+    """Create a ring of `capacity` per-call event sets (0 switches phase timing off)."""
+    _check(lib().imm_profile_enable(int(capacity)), "imm_profile_enable")
+
+
+def profile_calls() -> int:
+    return lib().imm_profile_calls()
+
+
+def profile_read(call: int) -> List[float]:
+    """Milliseconds per phase (PROFILE_PHASES order) of profiled prove call `call`; waits for it."""
+    buf = (ctypes.c_float * len(PROFILE_PHASES))()
+    _check(lib().imm_profile_read(int(call), ctypes.addressof(buf), len(PROFILE_PHASES)), "imm_profile_read")
+    return [float(v) for v in buf]
 
 
 def sumcheck_verify(transcript: Sequence[int], nrounds: int, seed: int, proof_id: int,

@@ -59,6 +59,18 @@ int env_int(const char* name, int dflt)
 int rowbind_cols(int dtype) { return ROWBIND_THREADS * (dtype == IMM_I8 ? 16 : 4); }
 int colbind_cols(int dtype) { return COLBIND_VECS * (dtype == IMM_I8 ? 16 : 4); }
 
+// Contraction back end of the prover: tensor-core (int8 MMA over 8-bit limbs of the weights) unless
+// IMM_CONTRACT=alu selects the integer-pipe kernels.
+bool use_mma()
+{
+    const char* s = getenv("IMM_CONTRACT");
+    return !(s && strcmp(s, "alu") == 0);
+}
+// columns (elements) per tile of the prover's three contractions
+int a_tile_cols(bool mma) { return mma ? ROWMMA_COLS : rowbind_cols(IMM_I8); }
+int b_tile_cols(bool mma) { return mma ? BYTEDOT_CHUNK_BYTES : colbind_cols(IMM_I8); }
+int c_tile_cols(bool mma) { return mma ? BYTEDOT_CHUNK_BYTES / 4 : rowbind_cols(IMM_I32); }
+
 struct Shape { int64_t rows, cols; };
 
 // Rows per tile: the largest candidate that still yields enough tiles to fill the GPU several
@@ -108,12 +120,17 @@ struct Plan {
     int status = IMM_OK;
     int nproofs = 0;
     int max_b = 0;
+    bool mma = true;
+    int max_weight_words = 0;
+    size_t off_wtasks = 0;
     int rows_a = 0, rows_b = 0, rows_c = 0;
     uint32_t tiles_a = 0, tiles_b = 0, tiles_c = 0;
     // byte offsets from the workspace base
     size_t off_proofs = 0, off_jobs_a = 0, off_jobs_b = 0, off_jobs_c = 0, off_eq = 0, header_bytes = 0;
     struct PerProof {
         size_t e_row, e_col, part_a, part_b, part_c, tab;
+        size_t w_rows, w_cols_b, w_cols_c;          // limb tables (tensor-core back end)
+        int nw_rows, nw_cols_b, nw_cols_c;          // their sizes in 32-bit words
         int a, b, c, n_part_a, n_part_b, n_part_c;
     };
     std::vector<PerProof> pp;
@@ -142,9 +159,11 @@ Plan make_plan(const imm_matmul_desc* descs, int nproofs)
         sb.push_back({descs[i].k, descs[i].n});
         sc.push_back({descs[i].m, descs[i].n});
     }
-    p.rows_a = pick_tile_rows(sa, rowbind_cols(IMM_I8), "IMM_TILE_ROWS_A");
-    p.rows_b = pick_tile_rows(sb, colbind_cols(IMM_I8), "IMM_TILE_ROWS_B");
-    p.rows_c = pick_tile_rows(sc, rowbind_cols(IMM_I32), "IMM_TILE_ROWS_C");
+    p.mma = use_mma();
+    const int acols = a_tile_cols(p.mma), bcols = b_tile_cols(p.mma), ccols = c_tile_cols(p.mma);
+    p.rows_a = pick_tile_rows(sa, acols, "IMM_TILE_ROWS_A");
+    p.rows_b = pick_tile_rows(sb, bcols, "IMM_TILE_ROWS_B");
+    p.rows_c = pick_tile_rows(sc, ccols, "IMM_TILE_ROWS_C");
 
     size_t off = 0;
     p.off_proofs = off; off = align_up(off + sizeof(ProofDev) * nproofs);
@@ -152,6 +171,7 @@ Plan make_plan(const imm_matmul_desc* descs, int nproofs)
     p.off_jobs_b = off; off = align_up(off + sizeof(MatJob) * nproofs);
     p.off_jobs_c = off; off = align_up(off + sizeof(MatJob) * nproofs);
     p.off_eq = off;     off = align_up(off + sizeof(EqTask) * 2 * nproofs);
+    p.off_wtasks = off; off = align_up(off + sizeof(WeightTask) * 3 * nproofs);
     p.header_bytes = off;
 
     uint64_t ta = 0, tb = 0, tc = 0;
@@ -162,9 +182,9 @@ Plan make_plan(const imm_matmul_desc* descs, int nproofs)
         q.a = ceil_log2(d.m); q.b = ceil_log2(d.k); q.c = ceil_log2(d.n);
         if (q.b > p.max_b) p.max_b = q.b;
         q.n_part_a = (int)((d.m + p.rows_a - 1) / p.rows_a);
-        q.n_part_b = (int)((d.n + colbind_cols(IMM_I8) - 1) / colbind_cols(IMM_I8));
+        q.n_part_b = (int)((d.n + bcols - 1) / bcols);
         const int64_t c_nrb = (d.m + p.rows_c - 1) / p.rows_c;
-        const int64_t c_ncc = (d.n + rowbind_cols(IMM_I32) - 1) / rowbind_cols(IMM_I32);
+        const int64_t c_ncc = (d.n + ccols - 1) / ccols;
         q.n_part_c = (int)(c_nrb * c_ncc);
         q.e_row = off;  off = align_up(off + sizeof(imm_fe) * ((size_t)1 << q.a));
         q.e_col = off;  off = align_up(off + sizeof(imm_fe) * ((size_t)1 << q.c));
@@ -172,7 +192,19 @@ Plan make_plan(const imm_matmul_desc* descs, int nproofs)
         q.part_b = off; off = align_up(off + sizeof(imm_fe) * (size_t)q.n_part_b * d.k);
         q.part_c = off; off = align_up(off + sizeof(imm_fe) * (size_t)q.n_part_c);
         q.tab = off;    off = align_up(off + sizeof(imm_fe) * 2 * ((size_t)1 << q.b));
-        ta += (uint64_t)q.n_part_a * ((d.k + rowbind_cols(IMM_I8) - 1) / rowbind_cols(IMM_I8));
+        q.nw_rows = q.nw_cols_b = q.nw_cols_c = 0;
+        q.w_rows = q.w_cols_b = q.w_cols_c = 0;
+        if (p.mma) {
+            q.nw_rows = (int)((d.m + 31) / 32) * 64;
+            q.nw_cols_b = (int)((d.n + 63) / 64) * 128;
+            q.nw_cols_c = (int)((4 * d.n + 63) / 64) * 128;
+            q.w_rows = off;   off = align_up(off + 4 * (size_t)q.nw_rows);
+            q.w_cols_b = off; off = align_up(off + 4 * (size_t)q.nw_cols_b);
+            q.w_cols_c = off; off = align_up(off + 4 * (size_t)q.nw_cols_c);
+            if (q.nw_cols_c > p.max_weight_words) p.max_weight_words = q.nw_cols_c;
+            if (q.nw_rows > p.max_weight_words) p.max_weight_words = q.nw_rows;
+        }
+        ta += (uint64_t)q.n_part_a * ((d.k + acols - 1) / acols);
         tb += (uint64_t)((d.k + p.rows_b - 1) / p.rows_b) * q.n_part_b;
         tc += (uint64_t)q.n_part_c;
     }
@@ -374,6 +406,8 @@ int imm_sumcheck_matmul_prove(const imm_matmul_desc* descs_host, int nproofs, ui
     MatJob* jb = (MatJob*)(hdr.data() + p.off_jobs_b);
     MatJob* jc = (MatJob*)(hdr.data() + p.off_jobs_c);
     EqTask* eq = (EqTask*)(hdr.data() + p.off_eq);
+    WeightTask* wt = (WeightTask*)(hdr.data() + p.off_wtasks);
+    const int acols = a_tile_cols(p.mma), bcols = b_tile_cols(p.mma), ccols = c_tile_cols(p.mma);
     uint32_t ta = 0, tb = 0, tc = 0;
     for (int i = 0; i < nproofs; i++) {
         const imm_matmul_desc& d = descs_host[i];
@@ -390,16 +424,24 @@ int imm_sumcheck_matmul_prove(const imm_matmul_desc* descs_host, int nproofs, ui
         P.a = q.a; P.b = q.b; P.c = q.c;
         P.n_part_a = q.n_part_a; P.n_part_b = q.n_part_b; P.n_part_c = q.n_part_c;
 
-        fill_job(ja[i], d.A, IMM_I8, d.m, d.k, d.lda, p.rows_a, rowbind_cols(IMM_I8));
+        fill_job(ja[i], d.A, IMM_I8, d.m, d.k, d.lda, p.rows_a, acols);
         ja[i].eq_row = P.e_row; ja[i].out = (imm_fe*)P.part_a; ja[i].tile0 = ta;
         ta += (uint32_t)(ja[i].nrb * ja[i].ncc);
-        fill_job(jb[i], d.B, IMM_I8, d.k, d.n, d.ldb, p.rows_b, colbind_cols(IMM_I8));
+        fill_job(jb[i], d.B, IMM_I8, d.k, d.n, d.ldb, p.rows_b, bcols);
         jb[i].eq_col = P.e_col; jb[i].out = (imm_fe*)P.part_b; jb[i].tile0 = tb;
         tb += (uint32_t)(jb[i].nrb * jb[i].ncc);
-        fill_job(jc[i], d.C, IMM_I32, d.m, d.n, d.ldc, p.rows_c, rowbind_cols(IMM_I32));
+        fill_job(jc[i], d.C, IMM_I32, d.m, d.n, d.ldc, p.rows_c, ccols);
         jc[i].eq_row = P.e_row; jc[i].eq_col = P.e_col; jc[i].out = (imm_fe*)P.part_c; jc[i].tile0 = tc;
         tc += (uint32_t)(jc[i].nrb * jc[i].ncc);
 
+        if (p.mma) {
+            ja[i].wtab = (const uint32_t*)(base + q.w_rows);
+            jb[i].wtab = (const uint32_t*)(base + q.w_cols_b);
+            jc[i].wtab = (const uint32_t*)(base + q.w_cols_c);
+            wt[3 * i + 0] = WeightTask{P.e_row, (uint32_t*)(base + q.w_rows), (int32_t)d.m, q.nw_rows, W_ROWS, 0};
+            wt[3 * i + 1] = WeightTask{P.e_col, (uint32_t*)(base + q.w_cols_b), (int32_t)d.n, q.nw_cols_b, W_COLS_I8, 0};
+            wt[3 * i + 2] = WeightTask{P.e_col, (uint32_t*)(base + q.w_cols_c), (int32_t)d.n, q.nw_cols_c, W_COLS_I32, 0};
+        }
         eq[2 * i] = EqTask{P.e_row, seed, d.proof_id, 1u, q.a};
         eq[2 * i + 1] = EqTask{P.e_col, seed, d.proof_id, 2u, q.c};
     }
@@ -412,12 +454,22 @@ int imm_sumcheck_matmul_prove(const imm_matmul_desc* descs_host, int nproofs, ui
     CU(cudaMemcpyAsync(base, hdr.data(), hdr.size(), cudaMemcpyHostToDevice, st));
     PROF_MARK(0);
     CU(launch_eq_batch((const EqTask*)(base + p.off_eq), 2 * nproofs, st));
+    if (p.mma)
+        CU(launch_weights((const WeightTask*)(base + p.off_wtasks), 3 * nproofs, p.max_weight_words, st));
     PROF_MARK(1);
-    CU(launch_rowbind(IMM_I32, true, (const MatJob*)(base + p.off_jobs_c), nproofs, p.tiles_c, st));
-    PROF_MARK(2);
-    CU(launch_rowbind(IMM_I8, false, (const MatJob*)(base + p.off_jobs_a), nproofs, p.tiles_a, st));
-    PROF_MARK(3);
-    CU(launch_colbind(IMM_I8, (const MatJob*)(base + p.off_jobs_b), nproofs, p.tiles_b, st));
+    if (p.mma) {
+        CU(launch_bytedot(true, true, (const MatJob*)(base + p.off_jobs_c), nproofs, p.tiles_c, st));
+        PROF_MARK(2);
+        CU(launch_rowmma((const MatJob*)(base + p.off_jobs_a), nproofs, p.tiles_a, st));
+        PROF_MARK(3);
+        CU(launch_bytedot(false, false, (const MatJob*)(base + p.off_jobs_b), nproofs, p.tiles_b, st));
+    } else {
+        CU(launch_rowbind(IMM_I32, true, (const MatJob*)(base + p.off_jobs_c), nproofs, p.tiles_c, st));
+        PROF_MARK(2);
+        CU(launch_rowbind(IMM_I8, false, (const MatJob*)(base + p.off_jobs_a), nproofs, p.tiles_a, st));
+        PROF_MARK(3);
+        CU(launch_colbind(IMM_I8, (const MatJob*)(base + p.off_jobs_b), nproofs, p.tiles_b, st));
+    }
     PROF_MARK(4);
     CU(launch_sumcheck((const ProofDev*)(base + p.off_proofs), nproofs, seed, d_transcripts, stride,
                        d_status, p.max_b, st));

@@ -3,6 +3,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <type_traits>
+
 #include "gl64.cuh"
 #include "imm_kernels.h"
 #include "imm_plan.h"
@@ -429,6 +431,12 @@ __global__ void __launch_bounds__(COLBIND_THREADS) colbind_kernel(const MatJob* 
     else colbind_tile<T, false>(job, local, sE);
 }
 
+}  // namespace imm
+
+#include "imm_mma.cuh"
+
+namespace imm {
+
 // ------------------------------------------------------------------------------------------
 // sum of partial vectors:  out[y] = sum_p parts[p][y]
 // ------------------------------------------------------------------------------------------
@@ -610,6 +618,35 @@ cudaError_t launch_colbind(int dtype, const MatJob* d_jobs, int njobs, uint32_t 
     if (ntiles == 0) return cudaSuccess;
     if (dtype == 0) colbind_kernel<int8_t><<<ntiles, COLBIND_THREADS, 0, st>>>(d_jobs, njobs);
     else colbind_kernel<int32_t><<<ntiles, COLBIND_THREADS, 0, st>>>(d_jobs, njobs);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_weights(const WeightTask* d_tasks, int ntasks, int max_words, cudaStream_t st)
+{
+    if (ntasks <= 0 || max_words <= 0) return cudaSuccess;
+    dim3 grid((unsigned)((max_words + 255) / 256), (unsigned)ntasks);
+    weights_kernel<<<grid, 256, 0, st>>>(d_tasks);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_bytedot(bool i32, bool point, const MatJob* d_jobs, int njobs, uint32_t ntiles,
+                           cudaStream_t st)
+{
+    if (ntiles == 0) return cudaSuccess;
+    if (i32) {
+        if (point) bytedot_kernel<true, true><<<ntiles, BYTEDOT_THREADS, 0, st>>>(d_jobs, njobs);
+        else bytedot_kernel<true, false><<<ntiles, BYTEDOT_THREADS, 0, st>>>(d_jobs, njobs);
+    } else {
+        if (point) bytedot_kernel<false, true><<<ntiles, BYTEDOT_THREADS, 0, st>>>(d_jobs, njobs);
+        else bytedot_kernel<false, false><<<ntiles, BYTEDOT_THREADS, 0, st>>>(d_jobs, njobs);
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_rowmma(const MatJob* d_jobs, int njobs, uint32_t ntiles, cudaStream_t st)
+{
+    if (ntiles == 0) return cudaSuccess;
+    rowmma_kernel<<<ntiles, ROWMMA_THREADS, 0, st>>>(d_jobs, njobs);
     return cudaGetLastError();
 }
 

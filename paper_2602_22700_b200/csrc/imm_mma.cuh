@@ -1,0 +1,290 @@
+// Tensor-core contraction kernels (included by imm_kernels.cu after the shared device helpers).
+//
+// The eq-vector x matrix products are dense contractions once the 64-bit weight is cut into
+// eight unsigned 8-bit limbs:  sum_q d[q] * W[q] = sum_l 2^(8l) * (sum_q d[q] * limb_l(W[q])).
+// The inner sums are int8 x uint8 dot products with 32-bit accumulation, i.e. an integer MMA
+// with the eight limbs as its N dimension (m16n8k32).  Each accumulator is rebuilt into a
+// 128-bit integer and reduced mod p once per output.  Matrix bytes go global -> registers ->
+// MMA with no shared-memory round trip; only the (tiny, reused) weight limbs are staged.
+#pragma once
+
+namespace imm {
+
+// D += A(16x32, row) * B(32x8, col), 32-bit accumulators.  SIGNED_A: matrix bytes are int8,
+// otherwise uint8; the weight limbs are always uint8.
+template <bool SIGNED_A>
+__device__ __forceinline__ void mma_m16n8k32(int32_t (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                             uint32_t a3, uint32_t b0, uint32_t b1)
+{
+    if constexpr (SIGNED_A) {
+        asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.s8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                     : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+                     : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+    } else {
+        asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.u8.u8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                     : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+                     : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+    }
+}
+
+// A thread of the MMA holds limbs 2t and 2t+1 (t = lane % 4) of one output.  Rebuild
+// 2^(16t) * (lo + 2^8 hi), add the four threads' shares; valid in all four lanes.
+__device__ __forceinline__ uint64_t combine_limbs(int32_t lo, int32_t hi, int t)
+{
+    uint64_t v = gl::from_i64((int64_t)lo + ((int64_t)hi << 8));
+    v = gl::shl(v, 16 * t);
+    v = gl::add(v, shfl_xor_u64(v, 1));
+    v = gl::add(v, shfl_xor_u64(v, 2));
+    return v;
+}
+
+// ------------------------------------------------------------------------------------------
+// limb tables of the weights, in fragment order
+// ------------------------------------------------------------------------------------------
+// W_COLS_*: weights of byte-columns.  Units of 64 byte-columns ("slabs"); slab s holds 32 lanes
+//   x 16 bytes; lane = 4g + t; byte (4r + b) of lane's 16 is limb g of W[64s + 16t + 4r + b].
+//   int8 matrix:  W[q] = eq[q].   int32 matrix seen as bytes: W[4j + b] = eq[j] * 2^(8b) mod p.
+// W_ROWS: weights of rows for the transposed (row-binding) MMA.  Units of 32 rows; lane = 4g+t
+//   holds 8 bytes: byte u of word h is limb g of eq[32G + 16h + 4t + u].
+// Weights past the real extent are zero (the implicit zero padding).
+
+__global__ void __launch_bounds__(256) weights_kernel(const WeightTask* tasks)
+{
+    const WeightTask tk = tasks[blockIdx.y];
+    const int wi = blockIdx.x * blockDim.x + threadIdx.x;
+    if (wi >= tk.nwords) return;
+    uint32_t word = 0;
+    if (tk.mode == W_ROWS) {
+        const int G = wi >> 6, lane = (wi >> 1) & 31, h = wi & 1;
+        const int g = lane >> 2, t = lane & 3;
+        const int row0 = 32 * G + 16 * h + 4 * t;
+#pragma unroll
+        for (int u = 0; u < 4; u++) {
+            uint64_t e = (row0 + u < tk.extent) ? tk.eq[row0 + u] : 0;
+            word |= (uint32_t)((e >> (8 * g)) & 0xFF) << (8 * u);
+        }
+    } else {
+        const int s = wi >> 7, lane = (wi >> 2) & 31, r = wi & 3;
+        const int g = lane >> 2, t = lane & 3;
+        const int q0 = 64 * s + 16 * t + 4 * r;
+        if (tk.mode == W_COLS_I8) {
+#pragma unroll
+            for (int b = 0; b < 4; b++) {
+                uint64_t e = (q0 + b < tk.extent) ? tk.eq[q0 + b] : 0;
+                word |= (uint32_t)((e >> (8 * g)) & 0xFF) << (8 * b);
+            }
+        } else {
+            const int j = q0 >> 2;
+            const uint64_t e = (j < tk.extent) ? tk.eq[j] : 0;
+#pragma unroll
+            for (int b = 0; b < 4; b++) {
+                uint64_t w = gl::shl(e, 8 * b);
+                word |= (uint32_t)((w >> (8 * g)) & 0xFF) << (8 * b);
+            }
+        }
+    }
+    tk.out[wi] = word;
+}
+
+// ------------------------------------------------------------------------------------------
+// byte-dot kernel:  u[i] = sum_q byte(M[i], q) * W[q]   (contraction along the contiguous index)
+// ------------------------------------------------------------------------------------------
+// Serves the column binding of int8 B (W = eq_col) and the claim on int32 C seen as an
+// m x 4n byte matrix (W[4j+b] = eq_col[j] 2^(8b)).  For int32 the top byte of every word is
+// flipped (x ^ 0x80000000) so that all four bytes are unsigned; the value then reads 2^31 too
+// high, which is undone per row by subtracting 2^31 * sum_j eq_col[j] over the tile's columns.
+//   POINT = false: out[chunk][row] = u[row]           (partial over this column chunk)
+//   POINT = true : out[tile] = sum_rows eq_row[row] * u[row]
+// One tile = tile_rows rows x BYTEDOT_CHUNK_BYTES byte-columns; a warp sweeps 32 rows (two MMA
+// row tiles) across the chunk, 64 byte-columns per step: four 16-byte loads per thread feed four
+// MMAs against one 16-byte read of staged weight limbs.
+
+template <bool I32, bool POINT, bool VEC>
+__device__ __forceinline__ void bytedot_tile(const MatJob& job, uint32_t local, uint4* sW, uint64_t* red)
+{
+    using T = typename std::conditional<I32, int32_t, int8_t>::type;
+    constexpr int ESZ = (int)sizeof(T);
+    constexpr int NWARP = BYTEDOT_THREADS / 32;
+    const int rbi = local / job.ncc, cci = local % job.ncc;
+    const int r0 = rbi * job.tile_rows;
+    const int r1 = min(r0 + job.tile_rows, job.rows);
+    const int64_t row_bytes = (int64_t)job.cols * ESZ;
+    const int64_t cb0 = (int64_t)cci * BYTEDOT_CHUNK_BYTES;
+    const int nslab = (int)min((int64_t)(BYTEDOT_CHUNK_BYTES / 64), (row_bytes - cb0 + 63) / 64);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int g = lane >> 2, t = lane & 3;
+
+    const uint4* wsrc = reinterpret_cast<const uint4*>(job.wtab) + (cb0 / 64) * 32;
+    for (int i = threadIdx.x; i < nslab * 32; i += BYTEDOT_THREADS) sW[i] = wsrc[i];
+
+    uint64_t corr = 0;
+    if (I32) {                 // 2^31 * (sum of this chunk's column weights)
+        const int j0 = (int)(cb0 / 4), j1 = min(job.cols, j0 + BYTEDOT_CHUNK_BYTES / 4);
+        uint64_t s = 0;
+        for (int j = j0 + threadIdx.x; j < j1; j += BYTEDOT_THREADS) s = gl::add(s, job.eq_col[j]);
+        corr = gl::shl(block_sum_fe(s, red), 31);
+    }
+    __syncthreads();
+
+    const int64_t pitch = job.ld * (int64_t)ESZ;
+    uint64_t part = 0;
+    for (int rg = r0 + warp * 32; rg < r1; rg += NWARP * 32) {
+        int32_t acc[2][4];
+        const char* p[2][2];
+#pragma unroll
+        for (int mt = 0; mt < 2; mt++) {
+#pragma unroll
+            for (int c = 0; c < 4; c++) acc[mt][c] = 0;
+#pragma unroll
+            for (int h = 0; h < 2; h++) {
+                const int row = min(rg + 16 * mt + g + 8 * h, r1 - 1);     // clamped: never out of bounds
+                p[mt][h] = (const char*)job.mat + (int64_t)row * pitch + cb0 + 16 * t;
+            }
+        }
+#pragma unroll 2
+        for (int s = 0; s < nslab; s++) {
+            const int64_t left = row_bytes - (cb0 + 64 * s + 16 * t);     // bytes of the row from this vector on
+            const bool full = left >= 16;
+            const int nvalid = left <= 0 ? 0 : (int)min((int64_t)16, left) / ESZ;
+            uint4 d[2][2];
+#pragma unroll
+            for (int mt = 0; mt < 2; mt++)
+#pragma unroll
+                for (int h = 0; h < 2; h++)
+                    d[mt][h] = nvalid > 0 ? load_vec<T, VEC>(p[mt][h] + 64 * s, full, nvalid) : make_uint4(0, 0, 0, 0);
+            const uint4 w = sW[s * 32 + lane];
+#pragma unroll
+            for (int mt = 0; mt < 2; mt++) {
+                uint4 x = d[mt][0], y = d[mt][1];
+                if (I32) {
+                    x.x ^= 0x80000000u; x.y ^= 0x80000000u; x.z ^= 0x80000000u; x.w ^= 0x80000000u;
+                    y.x ^= 0x80000000u; y.y ^= 0x80000000u; y.z ^= 0x80000000u; y.w ^= 0x80000000u;
+                }
+                mma_m16n8k32<!I32>(acc[mt], x.x, y.x, x.y, y.y, w.x, w.y);
+                mma_m16n8k32<!I32>(acc[mt], x.z, y.z, x.w, y.w, w.z, w.w);
+            }
+        }
+#pragma unroll
+        for (int mt = 0; mt < 2; mt++)
+#pragma unroll
+            for (int h = 0; h < 2; h++) {
+                const int row = rg + 16 * mt + g + 8 * h;
+                uint64_t u = combine_limbs(acc[mt][2 * h], acc[mt][2 * h + 1], t);
+                if (t == 0 && row < r1) {
+                    if (POINT) part = gl::add(part, gl::mul(job.eq_row[row], gl::sub(u, corr)));
+                    else job.out[(int64_t)cci * job.rows + row] = I32 ? gl::sub(u, corr) : u;
+                }
+            }
+    }
+    if (POINT) {
+        part = block_sum_fe(part, red);
+        if (threadIdx.x == 0) job.out[local] = part;
+    }
+}
+
+template <bool I32, bool POINT>
+__global__ void __launch_bounds__(BYTEDOT_THREADS) bytedot_kernel(const MatJob* jobs, int njobs)
+{
+    __shared__ uint4 sW[(BYTEDOT_CHUNK_BYTES / 64) * 32];          // 32 KiB of weight limbs
+    __shared__ uint64_t red[33];
+    const MatJob job = jobs[find_job(jobs, njobs, blockIdx.x)];
+    const uint32_t local = blockIdx.x - job.tile0;
+    if (job.vec) bytedot_tile<I32, POINT, true>(job, local, sW, red);
+    else bytedot_tile<I32, POINT, false>(job, local, sW, red);
+}
+
+// ------------------------------------------------------------------------------------------
+// row-binding MMA kernel (int8):  out[y] = sum_i eq_row[i] * M[i,y]
+// ------------------------------------------------------------------------------------------
+// The contraction runs along the strided index, so the MMA's K dimension is the row index and
+// its M dimension the column index: each thread loads 16 columns of 8 rows (coalesced 16-byte
+// loads, a warp reads 128 contiguous bytes of each row) and transposes 4x4 byte blocks in
+// registers with byte permutes so that every register holds one column at four consecutive
+// rows.  One tile = tile_rows rows x ROWMMA_COLS columns; each warp owns 128 columns.
+
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
+{
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+
+// rows r0..r3 of a 4x4 byte block -> columns c0..c3
+__device__ __forceinline__ void transpose4x4(uint32_t r0, uint32_t r1, uint32_t r2, uint32_t r3,
+                                             uint32_t& c0, uint32_t& c1, uint32_t& c2, uint32_t& c3)
+{
+    const uint32_t x0 = prmt(r0, r1, 0x5140), x1 = prmt(r0, r1, 0x7362);
+    const uint32_t y0 = prmt(r2, r3, 0x5140), y1 = prmt(r2, r3, 0x7362);
+    c0 = prmt(x0, y0, 0x5410); c1 = prmt(x0, y0, 0x7632);
+    c2 = prmt(x1, y1, 0x5410); c3 = prmt(x1, y1, 0x7632);
+}
+
+template <bool VEC>
+__device__ __forceinline__ void rowmma_tile(const MatJob& job, uint32_t local, uint2* sR)
+{
+    const int rbi = local / job.ncc, cci = local % job.ncc;
+    const int r0 = rbi * job.tile_rows;                         // multiple of 32
+    const int r1 = min(r0 + job.tile_rows, job.rows);
+    const int ngroups = (r1 - r0 + 31) / 32;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int g = lane >> 2, t = lane & 3;
+
+    const uint2* wsrc = reinterpret_cast<const uint2*>(job.wtab) + (int64_t)(r0 / 32) * 32;
+    for (int i = threadIdx.x; i < ngroups * 32; i += ROWMMA_THREADS) sR[i] = wsrc[i];
+    __syncthreads();
+
+    const int col = cci * ROWMMA_COLS + warp * 128 + 16 * g;      // this thread's 16 columns
+    const int nvalid = min(16, job.cols - col);
+    const bool full = nvalid == 16;
+    int32_t acc[8][4];
+#pragma unroll
+    for (int i = 0; i < 8; i++)
+#pragma unroll
+        for (int c = 0; c < 4; c++) acc[i][c] = 0;
+
+    if (warp * 128 + cci * ROWMMA_COLS < job.cols) {              // whole warp in or out
+        for (int G = 0; G < ngroups; G++) {
+            uint4 d[2][4];
+#pragma unroll
+            for (int h = 0; h < 2; h++)
+#pragma unroll
+                for (int u = 0; u < 4; u++) {
+                    const int row = min(r0 + 32 * G + 16 * h + 4 * t + u, r1 - 1);   // clamped; its weight is 0 past r1
+                    const char* p = (const char*)job.mat + (int64_t)row * job.ld + col;
+                    d[h][u] = nvalid > 0 ? load_vec<int8_t, VEC>(p, full, nvalid) : make_uint4(0, 0, 0, 0);
+                }
+            const uint2 wb = sR[G * 32 + lane];
+            uint32_t T[2][16];
+#pragma unroll
+            for (int h = 0; h < 2; h++) {
+                transpose4x4(d[h][0].x, d[h][1].x, d[h][2].x, d[h][3].x, T[h][0], T[h][1], T[h][2], T[h][3]);
+                transpose4x4(d[h][0].y, d[h][1].y, d[h][2].y, d[h][3].y, T[h][4], T[h][5], T[h][6], T[h][7]);
+                transpose4x4(d[h][0].z, d[h][1].z, d[h][2].z, d[h][3].z, T[h][8], T[h][9], T[h][10], T[h][11]);
+                transpose4x4(d[h][0].w, d[h][1].w, d[h][2].w, d[h][3].w, T[h][12], T[h][13], T[h][14], T[h][15]);
+            }
+#pragma unroll
+            for (int i = 0; i < 8; i++)
+                mma_m16n8k32<true>(acc[i], T[0][2 * i], T[0][2 * i + 1], T[1][2 * i], T[1][2 * i + 1], wb.x, wb.y);
+        }
+    }
+    // MMA i: row-slot g is column col + 2i, row-slot g+8 is column col + 2i + 1
+#pragma unroll
+    for (int i = 0; i < 8; i++)
+#pragma unroll
+        for (int h = 0; h < 2; h++) {
+            uint64_t v = combine_limbs(acc[i][2 * h], acc[i][2 * h + 1], t);
+            const int c = col + 2 * i + h;
+            if (t == 0 && c < job.cols) job.out[(int64_t)rbi * job.cols + c] = v;
+        }
+}
+
+__global__ void __launch_bounds__(ROWMMA_THREADS) rowmma_kernel(const MatJob* jobs, int njobs)
+{
+    __shared__ uint2 sR[MAX_TILE_ROWS];                             // (MAX_TILE_ROWS / 32) groups x 32 lanes
+    const MatJob job = jobs[find_job(jobs, njobs, blockIdx.x)];
+    const uint32_t local = blockIdx.x - job.tile0;
+    if (job.vec) rowmma_tile<true>(job, local, sR);
+    else rowmma_tile<false>(job, local, sR);
+}
+
+}  // namespace imm

@@ -14,6 +14,11 @@ constexpr int COLBIND_THREADS = 256;           // 8 warps
 constexpr int COLBIND_VECS = 128;              // 16-byte vectors per column chunk (2048 int8 / 512 int32)
 constexpr int COLBIND_ROWS_PER_WARP = 4;
 constexpr int MAX_TILE_ROWS = 1024;            // eq entries staged per tile by the row-binding kernels
+// Tensor-core (int8 MMA) contraction kernels.
+constexpr int BYTEDOT_THREADS = 256;           // 8 warps, each sweeping 32 rows at a time
+constexpr int BYTEDOT_CHUNK_BYTES = 4096;      // byte-columns per tile (4096 int8 / 1024 int32 columns)
+constexpr int ROWMMA_THREADS = 256;            // 8 warps x 128 columns
+constexpr int ROWMMA_COLS = 1024;              // int8 columns per tile
 constexpr int SUMCHECK_THREADS = 1024;
 constexpr int MAX_EQ_VARS = 20;
 constexpr int MAX_K_VARS = 17;
@@ -26,6 +31,7 @@ struct MatJob {
     const imm_fe* eq_row;      // ROWBIND / POINT: weights of the rows
     const imm_fe* eq_col;      // COLBIND / POINT: weights of the columns
     imm_fe* out;               // ROWBIND: [nrb][cols]; COLBIND: [ncc][rows]; POINT: [nrb*ncc]
+    const uint32_t* wtab;      // tensor-core kernels: limb table of the weights in fragment order
     int64_t ld;                // elements
     int32_t rows, cols;
     int32_t tile_rows;         // rows per tile
@@ -47,6 +53,17 @@ struct ProofDev {
     int32_t m, k, n;
     int32_t a, b, c;           // ceil(log2 m), ceil(log2 k), ceil(log2 n)
     int32_t n_part_a, n_part_b, n_part_c;
+    int32_t pad_;
+};
+
+// One limb table of eq weights in MMA fragment order (see weights_kernel).
+enum WeightMode { W_COLS_I8 = 0, W_COLS_I32 = 1, W_ROWS = 2 };
+struct WeightTask {
+    const imm_fe* eq;          // eq table
+    uint32_t* out;             // nwords 32-bit words
+    int32_t extent;            // real extent (columns or rows); weights past it are zero
+    int32_t nwords;
+    int32_t mode;
     int32_t pad_;
 };
 

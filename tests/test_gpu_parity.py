@@ -21,6 +21,13 @@ def imm():
     return binding
 
 
+@pytest.fixture(params=["mma", "alu"])
+def backend(request, monkeypatch):
+    """Runs a prover test once per contraction back end (tensor-core limbs / integer pipe)."""
+    monkeypatch.setenv("IMM_CONTRACT", request.param)
+    return request.param
+
+
 def u64_to_dev(vals):
     return torch.from_numpy(np.asarray(vals, dtype=np.uint64).view(np.int64)).cuda()
 
@@ -166,7 +173,7 @@ def read_golden(name):
         return [int(line, 16) for line in f if line.strip() and not line.startswith("#")]
 
 
-def test_golden_transcripts(imm):
+def test_golden_transcripts(imm, backend):
     from paper_2602_22700_b200 import synth
     A = np.array([[1, -2, 3, -4], [5, 6, -7, 8]], dtype=np.int8)
     B = np.array([[1, 2], [-3, 4], [5, -6], [7, 8]], dtype=np.int8)
@@ -179,11 +186,12 @@ def test_golden_transcripts(imm):
 
 
 SHAPES = [(1, 1, 1), (1, 2, 1), (3, 1, 5), (2, 4, 2), (1, 8, 1), (5, 3, 7), (17, 33, 9), (64, 64, 64),
-          (100, 257, 50), (33, 2048, 40), (40, 2049, 33), (130, 700, 515), (1030, 96, 2050)]
+          (100, 257, 50), (33, 2048, 40), (40, 2049, 33), (130, 700, 515), (1030, 96, 2050),
+          (300, 1100, 4100), (31, 1025, 1030), (1056, 130, 65), (65, 4200, 1000)]
 
 
 @pytest.mark.parametrize("m,k,n", SHAPES)
-def test_prove_single_matches_oracle(imm, oracle, m, k, n):
+def test_prove_single_matches_oracle(imm, oracle, backend, m, k, n):
     rng = np.random.default_rng(m * 10007 + k * 101 + n)
     A, B, C = np_problem(rng, m, k, n)
     seed, pid = 1000 + m, k
@@ -194,7 +202,24 @@ def test_prove_single_matches_oracle(imm, oracle, m, k, n):
     assert imm.sumcheck_verify(got, b, seed, pid) == (imm.OK, -1)
 
 
-def test_prove_ragged_batch_matches_oracle(imm, oracle):
+def test_prove_unaligned_leading_dimensions(imm, oracle, backend):
+    """Rows that are not 16-byte aligned take the element-wise loads; same transcript."""
+    rng = np.random.default_rng(78)
+    m, k, n = 70, 333, 130
+    A, B, C = np_problem(rng, m, k, n)
+    want = [int(w) for w in oracle.sumcheck_matmul_prove(A, B, C, 5, 9)]
+
+    def odd_view(M, ld, off):
+        buf = torch.zeros(M.shape[0] * ld + off + 8, dtype=torch.from_numpy(M).dtype, device="cuda")
+        v = buf[off:off + M.shape[0] * ld].view(M.shape[0], ld)[:, :M.shape[1]]
+        v.copy_(torch.from_numpy(M).cuda())
+        return v
+
+    dA, dB, dC = odd_view(A, k + 3, 1), odd_view(B, n + 5, 3), odd_view(C, n + 1, 1)
+    assert imm.sumcheck_matmul_prove([(dA, dB, dC, 9)], 5)[0] == want
+
+
+def test_prove_ragged_batch_matches_oracle(imm, oracle, backend):
     rng = np.random.default_rng(77)
     shapes = [(37, 300, 41), (1, 1, 1), (250, 64, 513), (64, 1000, 64), (5, 4097, 3), (129, 2, 2049)]
     probs = [np_problem(rng, *s) + (10 + i,) for i, s in enumerate(shapes)]
@@ -206,7 +231,7 @@ def test_prove_ragged_batch_matches_oracle(imm, oracle):
         assert gpu_prove(imm, [prob], 99)[0] == t
 
 
-def test_transcript_rows_are_zero_padded_and_status_ok(imm):
+def test_transcript_rows_are_zero_padded_and_status_ok(imm, backend):
     rng = np.random.default_rng(5)
     probs = [np_problem(rng, 4, 2, 4) + (0,), np_problem(rng, 4, 64, 4) + (1,)]
     dev = [(torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda(), torch.from_numpy(C).cuda(), pid)
@@ -224,7 +249,7 @@ def test_transcript_rows_are_zero_padded_and_status_ok(imm):
     assert (pr.transcripts == first).all()
 
 
-def test_tampering_is_rejected(imm, oracle):
+def test_tampering_is_rejected(imm, oracle, backend):
     rng = np.random.default_rng(21)
     A, B, C = np_problem(rng, 48, 200, 36)
     seed, pid, b = 4, 2, 8
@@ -251,7 +276,7 @@ def test_tampering_is_rejected(imm, oracle):
         assert imm.sumcheck_verify(sneaky, b, seed, pid, None, None, true_b) == (imm.REJECT, b + 3)
 
 
-def test_implicit_padding_equals_explicit_padding_on_gpu(imm):
+def test_implicit_padding_equals_explicit_padding_on_gpu(imm, backend):
     rng = np.random.default_rng(31)
     for (m, k, n) in ((5, 14, 6), (100, 300, 70), (33, 1500, 20)):
         A, B, C = np_problem(rng, m, k, n)
@@ -262,7 +287,7 @@ def test_implicit_padding_equals_explicit_padding_on_gpu(imm):
         assert gpu_prove(imm, [(A, B, C, 4)], 6) == gpu_prove(imm, [(Ap, Bp, Cp, 4)], 6)
 
 
-def test_finals_match_point_evaluations(imm):
+def test_finals_match_point_evaluations(imm, backend):
     """c0, a_fin, b_fin are C~(r_row,r_col), A~(r_row,r_k), B~(r_k,r_col) by the point-evaluation call."""
     rng = np.random.default_rng(41)
     m, k, n = 70, 500, 90
@@ -280,7 +305,7 @@ def test_finals_match_point_evaluations(imm):
     assert imm.sumcheck_verify(t, b, seed, pid, t[0], t[-2], t[-1]) == (imm.OK, -1)
 
 
-def test_host_buffer_entry_point_matches_device_entry_point(imm):
+def test_host_buffer_entry_point_matches_device_entry_point(imm, backend):
     rng = np.random.default_rng(51)
     shapes = [(37, 300, 41), (64, 100, 130)]
     probs = [np_problem(rng, *s) + (i,) for i, s in enumerate(shapes)]

@@ -40,7 +40,7 @@ SEED = 1
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=30)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--layers", type=int, default=32)
@@ -166,7 +166,7 @@ def measured_peaks():
 # DRAM traffic of the claim kernel per algorithmic byte, from the ncu capture summarised under
 # profiles/ (dram__bytes_read.sum + dram__bytes_write.sum over 4*m*n); None until a capture of the
 # current kernel exists.
-CLAIM_KERNEL_TRAFFIC_RATIO = None
+CLAIM_KERNEL_TRAFFIC_RATIO = 241.72 / 234.881024  # bytedot_kernel<1,1>, first MMA version
 
 
 # ------------------------------------------------------------------------ our arm
@@ -263,7 +263,7 @@ def run_ours(args):
         "phases": {name: {"ms": phase_ms[i],
                           "gbs": (phase_bytes[i] / (phase_ms[i] * 1e-3) / 1e9) if phase_bytes[i] and phase_ms[i] > 0 else None}
                    for i, name in enumerate(imm.PROFILE_PHASES)},
-        "roofline": {"kernel": "rowbind_kernel<int32,POINT> (claim C~)", "bound": "hbm", "achieved": claim_gbs,
+        "roofline": {"kernel": "bytedot_kernel<int32 as bytes, POINT> (claim C~)", "bound": "hbm", "achieved": claim_gbs,
                      "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": claim_gbs / peak,
                      "frac_of_8tbs": claim_gbs / 8000.0,
                      "traffic": (CLAIM_KERNEL_TRAFFIC_RATIO * claim_bytes) if CLAIM_KERNEL_TRAFFIC_RATIO else None},

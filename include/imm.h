@@ -63,7 +63,8 @@ enum {
     IMM_ERR_ALIGN = -3,          /* workspace / output pointer not 16-byte aligned         */
     IMM_ERR_WORKSPACE = -4,      /* workspace smaller than the query call asks for         */
     IMM_ERR_NONCANONICAL = -5,   /* a field element >= p on input                          */
-    IMM_ERR_CUDA = -6            /* a CUDA runtime call failed (see imm_last_cuda_error)   */
+    IMM_ERR_CUDA = -6,           /* a CUDA runtime call failed (see imm_last_cuda_error)   */
+    IMM_ERR_LIMIT = -7           /* larger than the fixed capacity of a no-allocation call */
 };
 enum { IMM_I8 = 0, IMM_I32 = 1 };
 enum { IMM_BIND_ROWS = 0, IMM_BIND_COLS = 1 };
@@ -118,6 +119,34 @@ int imm_mle_partial_eval(const void* d_mat, int dtype, int64_t rows, int64_t col
 int imm_mle_eval_point(const void* d_mat, int dtype, int64_t rows, int64_t cols, int64_t ld,
                        const imm_fe* d_eq_row, const imm_fe* d_eq_col, imm_fe* d_out,
                        void* d_ws, size_t ws_bytes, void* stream);
+
+/* Point evaluation for callers that cannot allocate device memory.  (The paper has no
+ * counterpart: this is a deployment convenience of this library.)
+ *
+ * Same result as imm_mle_eval_point, but without a workspace argument: the per-tile partial sums
+ * live in a fixed 64 KiB array that is part of the library's device image, so every GPU that
+ * loads the library holds that array until the process exits.  It is meant for code that runs
+ * inside a serving engine's step -- an audit hook called between decode steps, say -- where all
+ * device memory already belongs to the engine's pool, so a cudaMalloc would fail under the
+ * memory cap or stall every stream with its implicit device-wide synchronisation, and where no
+ * spare buffer can be threaded through to the call site.  The call itself performs no
+ * cudaMalloc / cudaFree and uses no allocating library routine; it enqueues two kernels on
+ * `stream` and returns.
+ *
+ * Capacity: the matrix is cut into tiles of up to 1024 rows x 512 int32 (2048 int8) columns and at
+ * most IMM_NOALLOC_MAX_TILES tiles fit the array (about 16 GiB of matrix); anything larger returns
+ * IMM_ERR_LIMIT before any device work.  Other errors as imm_mle_eval_point (no workspace ones).
+ *
+ * The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
+ * that device current); make that first call outside any stream capture.  All calls on one
+ * device share the array: it keeps the previous call's partial sums, which is harmless because
+ * every slot a call reads is first overwritten by that call (nothing needs to start at zero), but
+ * two calls whose kernels overlap on the GPU (different streams, or different host threads
+ * without ordering) race on it and return garbage.  Order such calls on one stream. */
+#define IMM_NOALLOC_MAX_TILES 8192
+int imm_mle_eval_point_noalloc(const void* d_mat, int dtype, int64_t rows, int64_t cols, int64_t ld,
+                               const imm_fe* d_eq_row, const imm_fe* d_eq_col, imm_fe* d_out,
+                               void* stream);
 
 /* One claimed product C = A*B.  A: m x k int8, B: k x n int8, C: m x n int32 -- the CLAIMED
  * matrix, used as given (the prover never recomputes A*B).  DEVICE pointers for

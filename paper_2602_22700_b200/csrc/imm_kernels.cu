@@ -2,6 +2,7 @@
 // sumcheck rounds.  Host-side launch wrappers are at the end; the C ABI lives in imm_api.cu.
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <string.h>
 
 #include <type_traits>
 
@@ -679,3 +680,99 @@ cudaError_t launch_sumcheck(const ProofDev* d_proofs, int nproofs, uint64_t seed
 }
 
 }  // namespace imm
+
+// ------------------------------------------------------------------------------------------
+// point evaluation without a caller workspace (imm_mle_eval_point_noalloc)
+// ------------------------------------------------------------------------------------------
+// For callers that may not allocate device memory (code running inside a serving engine whose
+// pool owns all of HBM): the per-tile partial sums go to a fixed array in this library's device
+// image instead of a workspace.  In host code the array's name is only a stand-in for the
+// symbol, not a device address, so the address is looked up once per device with
+// cudaGetSymbolAddress and handed to the kernels.
+
+#include <mutex>
+
+#include "../../include/imm.h"
+
+namespace imm {
+
+constexpr int NOALLOC_MAX_DEVICES = 64;
+
+static __device__ __align__(256) imm_fe g_noalloc_partials[IMM_NOALLOC_MAX_TILES];   // 64 KiB per GPU
+
+static imm_fe* g_noalloc_ptr[NOALLOC_MAX_DEVICES];      // device address of the array, per device
+static std::mutex g_noalloc_mutex;
+
+// Same tile code as rowbind_kernel<T, POINT>, with the job passed by value (no descriptor upload).
+template <typename T>
+__global__ void __launch_bounds__(ROWBIND_THREADS) rowbind_point_byvalue_kernel(const MatJob job)
+{
+    __shared__ int2 sE[MAX_TILE_ROWS];
+    __shared__ uint64_t red[33];
+    if (job.vec) rowbind_tile<T, true, true>(job, blockIdx.x, sE, red);
+    else rowbind_tile<T, true, false>(job, blockIdx.x, sE, red);
+}
+
+static cudaError_t noalloc_scratch(imm_fe** out)
+{
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= NOALLOC_MAX_DEVICES) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    if (!g_noalloc_ptr[dev]) {
+        imm_fe* p = nullptr;
+        e = cudaGetSymbolAddress((void**)&p, g_noalloc_partials);     // set-up: once per device
+        if (e != cudaSuccess) return e;
+        g_noalloc_ptr[dev] = p;
+    }
+    *out = g_noalloc_ptr[dev];
+    return cudaSuccess;
+}
+
+}  // namespace imm
+
+extern "C" int imm_mle_eval_point_noalloc(const void* d_mat, int dtype, int64_t rows, int64_t cols,
+                                          int64_t ld, const imm_fe* d_eq_row, const imm_fe* d_eq_col,
+                                          imm_fe* d_out, void* stream)
+{
+    using namespace imm;
+    if (!d_mat || !d_eq_row || !d_eq_col || !d_out || (dtype != IMM_I8 && dtype != IMM_I32)) return IMM_ERR_ARG;
+    if (rows <= 0 || cols <= 0 || rows > ((int64_t)1 << 20) || cols > ((int64_t)1 << 20) || ld < cols)
+        return IMM_ERR_SHAPE;
+    if ((uintptr_t)d_out % 8 != 0 || (uintptr_t)d_eq_row % 8 != 0 || (uintptr_t)d_eq_col % 8 != 0) return IMM_ERR_ALIGN;
+    const int esz = dtype == IMM_I8 ? 1 : 4;
+    const int cols_per_tile = ROWBIND_THREADS * (16 / esz);
+    const int64_t ncc = (cols + cols_per_tile - 1) / cols_per_tile;
+    // smallest tile height (from 32 rows up) whose tile count fits the fixed array
+    int tile_rows = 32;
+    while (tile_rows < MAX_TILE_ROWS && ((rows + tile_rows - 1) / tile_rows) * ncc > IMM_NOALLOC_MAX_TILES)
+        tile_rows *= 2;
+    const int64_t nrb = (rows + tile_rows - 1) / tile_rows;
+    if (nrb * ncc > IMM_NOALLOC_MAX_TILES) return IMM_ERR_LIMIT;
+
+    imm_fe* scratch = nullptr;
+    if (noalloc_scratch(&scratch) != cudaSuccess) return IMM_ERR_CUDA;
+
+    MatJob j;
+    memset(&j, 0, sizeof(j));
+    j.mat = d_mat;
+    j.eq_row = d_eq_row;
+    j.eq_col = d_eq_col;
+    j.out = scratch;
+    j.ld = ld;
+    j.rows = (int32_t)rows;
+    j.cols = (int32_t)cols;
+    j.tile_rows = tile_rows;
+    j.nrb = (int32_t)nrb;
+    j.ncc = (int32_t)ncc;
+    j.vec = (((uintptr_t)d_mat % 16 == 0) && ((ld * esz) % 16 == 0)) ? 1 : 0;
+    cudaStream_t st = (cudaStream_t)stream;
+    const unsigned ntiles = (unsigned)(nrb * ncc);
+    if (dtype == IMM_I8) rowbind_point_byvalue_kernel<int8_t><<<ntiles, ROWBIND_THREADS, 0, st>>>(j);
+    else rowbind_point_byvalue_kernel<int32_t><<<ntiles, ROWBIND_THREADS, 0, st>>>(j);
+    if (cudaGetLastError() != cudaSuccess) return IMM_ERR_CUDA;
+    sum_all_kernel<<<1, 1024, 0, st>>>(scratch, (int64_t)ntiles, d_out);
+    if (cudaGetLastError() != cudaSuccess) return IMM_ERR_CUDA;
+    return IMM_OK;
+}

@@ -18,7 +18,7 @@ OK, REJECT = 0, 1
 I8, I32 = 0, 1
 BIND_ROWS, BIND_COLS = 0, 1
 FIELD_ADD, FIELD_SUB, FIELD_MUL = 0, 1, 2
-ERRORS = {-1: "IMM_ERR_ARG", -2: "IMM_ERR_SHAPE", -3: "IMM_ERR_ALIGN", -4: "IMM_ERR_WORKSPACE",
+ERRORS = {-7: "IMM_ERR_LIMIT", -1: "IMM_ERR_ARG", -2: "IMM_ERR_SHAPE", -3: "IMM_ERR_ALIGN", -4: "IMM_ERR_WORKSPACE",
           -5: "IMM_ERR_NONCANONICAL", -6: "IMM_ERR_CUDA"}
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -28,7 +28,8 @@ EXPORTS = ("imm_version", "imm_last_cuda_error", "imm_challenge", "imm_field_bin
            "imm_mle_workspace", "imm_mle_partial_eval", "imm_mle_eval_point",
            "imm_sumcheck_matmul_workspace", "imm_sumcheck_matmul_prove",
            "imm_sumcheck_matmul_host_arena", "imm_sumcheck_matmul_prove_host", "imm_sumcheck_verify",
-           "imm_profile_enable", "imm_profile_calls", "imm_profile_read")
+           "imm_profile_enable", "imm_profile_calls", "imm_profile_read", "imm_mle_eval_point_noalloc")
+NOALLOC_MAX_TILES = 8192
 PROFILE_PHASES = ("eq_tables", "claim_C", "bind_rows_A", "bind_cols_B", "sumcheck_rounds")
 
 
@@ -72,6 +73,8 @@ def lib() -> ctypes.CDLL:
     L.imm_mle_partial_eval.argtypes = [vp, ci, i64, i64, i64, ci, vp, vp, vp, sz, vp]
     L.imm_mle_eval_point.restype = ci
     L.imm_mle_eval_point.argtypes = [vp, ci, i64, i64, i64, vp, vp, vp, vp, sz, vp]
+    L.imm_mle_eval_point_noalloc.restype = ci
+    L.imm_mle_eval_point_noalloc.argtypes = [vp, ci, i64, i64, i64, vp, vp, vp, vp]
     L.imm_sumcheck_matmul_workspace.restype = sz
     L.imm_sumcheck_matmul_workspace.argtypes = [vp, ci]
     L.imm_sumcheck_matmul_prove.restype = ci
@@ -192,6 +195,18 @@ def mle_eval_point(mat: torch.Tensor, eq_row: torch.Tensor, eq_col: torch.Tensor
     _check(lib().imm_mle_eval_point(ptr, code, rows, cols, ld, eq_row.data_ptr(), eq_col.data_ptr(),
                                     out.data_ptr(), ws.data_ptr(), ws.numel(), _stream()),
            "imm_mle_eval_point")
+    return out
+
+
+def mle_eval_point_noalloc(mat: torch.Tensor, eq_row: torch.Tensor, eq_col: torch.Tensor,
+                           out: torch.Tensor) -> torch.Tensor:
+    """Point evaluation for callers that cannot allocate device memory: no workspace, the
+    partial sums live in a fixed array inside the library (see imm.h for capacity and the
+    sharing rules).  ``out`` is a caller-provided 1-element int64 CUDA tensor."""
+    ptr, code, rows, cols, ld = _matrix(mat, "mat")
+    _cuda(eq_row, torch.int64, "eq_row"); _cuda(eq_col, torch.int64, "eq_col"); _cuda(out, torch.int64, "out")
+    _check(lib().imm_mle_eval_point_noalloc(ptr, code, rows, cols, ld, eq_row.data_ptr(), eq_col.data_ptr(),
+                                            out.data_ptr(), _stream()), "imm_mle_eval_point_noalloc")
     return out
 
 

@@ -75,7 +75,8 @@ struct Shape { int64_t rows, cols; };
 
 // Rows per tile: the largest candidate that still yields enough tiles to fill the GPU several
 // times over (the tail of the last wave is then a small fraction of the launch).
-int pick_tile_rows(const std::vector<Shape>& mats, int cols_per_tile, const char* env_name)
+int pick_tile_rows(const std::vector<Shape>& mats, int cols_per_tile, const char* env_name,
+                   int max_rows = MAX_TILE_ROWS)
 {
     const int forced = env_int(env_name, 0);
     if (forced) {
@@ -85,6 +86,7 @@ int pick_tile_rows(const std::vector<Shape>& mats, int cols_per_tile, const char
     const int64_t target = (int64_t)148 * env_int("IMM_TILES_PER_SM", 24);
     const int cand[] = {1024, 512, 256, 128, 64, 32};
     for (int c : cand) {
+        if (c > max_rows) continue;
         int64_t tiles = 0;
         for (const Shape& s : mats)
             tiles += ((s.rows + c - 1) / c) * ((s.cols + cols_per_tile - 1) / cols_per_tile);
@@ -104,7 +106,9 @@ void fill_job(MatJob& j, const void* mat, int dtype, int64_t rows, int64_t cols,
     j.tile_rows = tile_rows;
     j.nrb = (int32_t)((rows + tile_rows - 1) / tile_rows);
     j.ncc = (int32_t)((cols + cols_per_tile - 1) / cols_per_tile);
-    j.vec = rows_vectorisable(mat, ld, dtype) ? 1 : 0;
+    // 2: rows 32-byte aligned (256-bit loads), 1: 16-byte aligned (128-bit loads), 0: element-wise
+    const int64_t pitch = ld * (int64_t)elem_size(dtype);
+    j.vec = ((uintptr_t)mat % 32 == 0 && pitch % 32 == 0) ? 2 : rows_vectorisable(mat, ld, dtype) ? 1 : 0;
 }
 
 int check_matrix_args(const void* d_mat, int dtype, int64_t rows, int64_t cols, int64_t ld)
@@ -162,7 +166,9 @@ Plan make_plan(const imm_matmul_desc* descs, int nproofs)
     p.mma = use_mma();
     const int acols = a_tile_cols(p.mma), bcols = b_tile_cols(p.mma), ccols = c_tile_cols(p.mma);
     p.rows_a = pick_tile_rows(sa, acols, "IMM_TILE_ROWS_A");
-    p.rows_b = pick_tile_rows(sb, bcols, "IMM_TILE_ROWS_B");
+    // measured on the decoder-block workload: B (32 rows per warp pass) is best at 256 rows per tile,
+    // C (16 rows per warp pass) at 512-1024
+    p.rows_b = pick_tile_rows(sb, bcols, "IMM_TILE_ROWS_B", p.mma ? 256 : MAX_TILE_ROWS);
     p.rows_c = pick_tile_rows(sc, ccols, "IMM_TILE_ROWS_C");
 
     size_t off = 0;
@@ -196,8 +202,8 @@ Plan make_plan(const imm_matmul_desc* descs, int nproofs)
         q.w_rows = q.w_cols_b = q.w_cols_c = 0;
         if (p.mma) {
             q.nw_rows = (int)((d.m + 31) / 32) * 64;
-            q.nw_cols_b = (int)((d.n + 63) / 64) * 128;
-            q.nw_cols_c = (int)((4 * d.n + 63) / 64) * 128;
+            q.nw_cols_b = (int)((d.n + 255) / 256) * 512;
+            q.nw_cols_c = (int)((4 * d.n + 255) / 256) * 512;
             q.w_rows = off;   off = align_up(off + 4 * (size_t)q.nw_rows);
             q.w_cols_b = off; off = align_up(off + 4 * (size_t)q.nw_cols_b);
             q.w_cols_c = off; off = align_up(off + 4 * (size_t)q.nw_cols_c);
@@ -458,11 +464,11 @@ int imm_sumcheck_matmul_prove(const imm_matmul_desc* descs_host, int nproofs, ui
         CU(launch_weights((const WeightTask*)(base + p.off_wtasks), 3 * nproofs, p.max_weight_words, st));
     PROF_MARK(1);
     if (p.mma) {
-        CU(launch_bytedot(true, true, (const MatJob*)(base + p.off_jobs_c), nproofs, p.tiles_c, st));
+        CU(launch_bytedot(true, true, env_int("IMM_BYTEDOT_MT_C", 1), (const MatJob*)(base + p.off_jobs_c), nproofs, p.tiles_c, st));
         PROF_MARK(2);
         CU(launch_rowmma((const MatJob*)(base + p.off_jobs_a), nproofs, p.tiles_a, st));
         PROF_MARK(3);
-        CU(launch_bytedot(false, false, (const MatJob*)(base + p.off_jobs_b), nproofs, p.tiles_b, st));
+        CU(launch_bytedot(false, false, env_int("IMM_BYTEDOT_MT_B", 2), (const MatJob*)(base + p.off_jobs_b), nproofs, p.tiles_b, st));
     } else {
         CU(launch_rowbind(IMM_I32, true, (const MatJob*)(base + p.off_jobs_c), nproofs, p.tiles_c, st));
         PROF_MARK(2);

@@ -630,17 +630,19 @@ cudaError_t launch_weights(const WeightTask* d_tasks, int ntasks, int max_words,
     return cudaGetLastError();
 }
 
-cudaError_t launch_bytedot(bool i32, bool point, const MatJob* d_jobs, int njobs, uint32_t ntiles,
+cudaError_t launch_bytedot(bool i32, bool point, int mt, const MatJob* d_jobs, int njobs, uint32_t ntiles,
                            cudaStream_t st)
 {
     if (ntiles == 0) return cudaSuccess;
+#define BD_LAUNCH(I, P, M) bytedot_kernel<I, P, M><<<ntiles, BYTEDOT_THREADS, 0, st>>>(d_jobs, njobs)
     if (i32) {
-        if (point) bytedot_kernel<true, true><<<ntiles, BYTEDOT_THREADS, 0, st>>>(d_jobs, njobs);
-        else bytedot_kernel<true, false><<<ntiles, BYTEDOT_THREADS, 0, st>>>(d_jobs, njobs);
+        if (point) { if (mt == 2) BD_LAUNCH(true, true, 2); else BD_LAUNCH(true, true, 1); }
+        else { if (mt == 2) BD_LAUNCH(true, false, 2); else BD_LAUNCH(true, false, 1); }
     } else {
-        if (point) bytedot_kernel<false, true><<<ntiles, BYTEDOT_THREADS, 0, st>>>(d_jobs, njobs);
-        else bytedot_kernel<false, false><<<ntiles, BYTEDOT_THREADS, 0, st>>>(d_jobs, njobs);
+        if (point) { if (mt == 2) BD_LAUNCH(false, true, 2); else BD_LAUNCH(false, true, 1); }
+        else { if (mt == 2) BD_LAUNCH(false, false, 2); else BD_LAUNCH(false, false, 1); }
     }
+#undef BD_LAUNCH
     return cudaGetLastError();
 }
 

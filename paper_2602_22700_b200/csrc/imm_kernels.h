@@ -18,7 +18,7 @@ cudaError_t launch_colbind(int dtype, const MatJob* d_jobs, int njobs, uint32_t 
 // Tensor-core contractions: limb tables of the weights, then the byte-dot (contiguous index) and
 // row-binding (strided index, int8 only) kernels.
 cudaError_t launch_weights(const WeightTask* d_tasks, int ntasks, int max_words, cudaStream_t st);
-cudaError_t launch_bytedot(bool i32, bool point, const MatJob* d_jobs, int njobs, uint32_t ntiles,
+cudaError_t launch_bytedot(bool i32, bool point, int mt, const MatJob* d_jobs, int njobs, uint32_t ntiles,
                            cudaStream_t st);
 cudaError_t launch_rowmma(const MatJob* d_jobs, int njobs, uint32_t ntiles, cudaStream_t st);
 cudaError_t launch_sum_parts(const imm_fe* parts, int nparts, int64_t len, imm_fe* out, cudaStream_t st);

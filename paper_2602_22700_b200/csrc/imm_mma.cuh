@@ -41,8 +41,10 @@ __device__ __forceinline__ uint64_t combine_limbs(int32_t lo, int32_t hi, int t)
 // ------------------------------------------------------------------------------------------
 // limb tables of the weights, in fragment order
 // ------------------------------------------------------------------------------------------
-// W_COLS_*: weights of byte-columns.  Units of 64 byte-columns ("slabs"); slab s holds 32 lanes
-//   x 16 bytes; lane = 4g + t; byte (4r + b) of lane's 16 is limb g of W[64s + 16t + 4r + b].
+// W_COLS_*: weights of byte-columns.  Units of 256 byte-columns ("slabs"); a lane (4g + t) of
+//   the byte-dot kernel owns bytes 64t..64t+63 of a slab, and its 64 weight bytes are limb g of
+//   W[256s + 64t + 0..63].  They are stored as four 16-byte pieces, piece-major
+//   ([slab][piece][lane]) so that a warp's 16-byte reads are conflict-free.
 //   int8 matrix:  W[q] = eq[q].   int32 matrix seen as bytes: W[4j + b] = eq[j] * 2^(8b) mod p.
 // W_ROWS: weights of rows for the transposed (row-binding) MMA.  Units of 32 rows; lane = 4g+t
 //   holds 8 bytes: byte u of word h is limb g of eq[32G + 16h + 4t + u].
@@ -64,9 +66,9 @@ __global__ void __launch_bounds__(256) weights_kernel(const WeightTask* tasks)
             word |= (uint32_t)((e >> (8 * g)) & 0xFF) << (8 * u);
         }
     } else {
-        const int s = wi >> 7, lane = (wi >> 2) & 31, r = wi & 3;
+        const int s = wi >> 9, piece = (wi >> 7) & 3, lane = (wi >> 2) & 31, r = wi & 3;
         const int g = lane >> 2, t = lane & 3;
-        const int q0 = 64 * s + 16 * t + 4 * r;
+        const int q0 = 256 * s + 64 * t + 16 * piece + 4 * r;
         if (tk.mode == W_COLS_I8) {
 #pragma unroll
             for (int b = 0; b < 4; b++) {
@@ -95,11 +97,46 @@ __global__ void __launch_bounds__(256) weights_kernel(const WeightTask* tasks)
 // high, which is undone per row by subtracting 2^31 * sum_j eq_col[j] over the tile's columns.
 //   POINT = false: out[chunk][row] = u[row]           (partial over this column chunk)
 //   POINT = true : out[tile] = sum_rows eq_row[row] * u[row]
-// One tile = tile_rows rows x BYTEDOT_CHUNK_BYTES byte-columns; a warp sweeps 32 rows (two MMA
-// row tiles) across the chunk, 64 byte-columns per step: four 16-byte loads per thread feed four
-// MMAs against one 16-byte read of staged weight limbs.
+// One tile = tile_rows rows x BYTEDOT_CHUNK_BYTES byte-columns.  A warp sweeps 16*MT rows (MT MMA
+// row tiles) across the chunk in slabs of 256 byte-columns; within a slab a thread owns 64
+// CONTIGUOUS bytes of each of its 2*MT rows (two 256-bit loads), so four neighbouring lanes read
+// 256 contiguous bytes of a row -- measured to stream at the rate of a linear read, where
+// 64-byte pieces per row lose 15 %.  Which byte-column lands in which MMA k-slot is free as long
+// as the weight limbs are laid out the same way (weights_kernel does that).
 
-template <bool I32, bool POINT, bool VEC>
+struct u32x8 { uint32_t v[8]; };
+
+__device__ __forceinline__ u32x8 ld_stream_v8(const void* p)          // 256-bit streaming load, 32-byte aligned
+{
+    u32x8 r;
+    asm volatile("ld.global.nc.L1::no_allocate.v8.u32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                 : "=r"(r.v[0]), "=r"(r.v[1]), "=r"(r.v[2]), "=r"(r.v[3]), "=r"(r.v[4]), "=r"(r.v[5]),
+                   "=r"(r.v[6]), "=r"(r.v[7])
+                 : "l"(p));
+    return r;
+}
+
+// 64 bytes of one row starting at p; `left` = bytes of the row from p on (may be <= 0).
+// VL 2: rows 32-byte aligned, VL 1: 16-byte aligned, VL 0: element-wise loads.
+template <typename T, int VL>
+__device__ __forceinline__ void load64(const char* p, int64_t left, uint32_t (&d)[16])
+{
+    if (VL == 2 && left >= 64) {
+        const u32x8 a = ld_stream_v8(p), b = ld_stream_v8(p + 32);
+#pragma unroll
+        for (int i = 0; i < 8; i++) { d[i] = a.v[i]; d[8 + i] = b.v[i]; }
+        return;
+    }
+#pragma unroll
+    for (int i = 0; i < 4; i++) {
+        const int64_t l = left - 16 * i;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (l > 0) v = load_vec<T, (VL >= 1)>(p + 16 * i, l >= 16, (int)(min((int64_t)16, l) / (int64_t)sizeof(T)));
+        d[4 * i] = v.x; d[4 * i + 1] = v.y; d[4 * i + 2] = v.z; d[4 * i + 3] = v.w;
+    }
+}
+
+template <bool I32, bool POINT, int VL, int MT>
 __device__ __forceinline__ void bytedot_tile(const MatJob& job, uint32_t local, uint4* sW, uint64_t* red)
 {
     using T = typename std::conditional<I32, int32_t, int8_t>::type;
@@ -110,12 +147,12 @@ __device__ __forceinline__ void bytedot_tile(const MatJob& job, uint32_t local, 
     const int r1 = min(r0 + job.tile_rows, job.rows);
     const int64_t row_bytes = (int64_t)job.cols * ESZ;
     const int64_t cb0 = (int64_t)cci * BYTEDOT_CHUNK_BYTES;
-    const int nslab = (int)min((int64_t)(BYTEDOT_CHUNK_BYTES / 64), (row_bytes - cb0 + 63) / 64);
+    const int nslab = (int)min((int64_t)(BYTEDOT_CHUNK_BYTES / 256), (row_bytes - cb0 + 255) / 256);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int g = lane >> 2, t = lane & 3;
 
-    const uint4* wsrc = reinterpret_cast<const uint4*>(job.wtab) + (cb0 / 64) * 32;
-    for (int i = threadIdx.x; i < nslab * 32; i += BYTEDOT_THREADS) sW[i] = wsrc[i];
+    const uint4* wsrc = reinterpret_cast<const uint4*>(job.wtab) + (cb0 / 256) * 128;
+    for (int i = threadIdx.x; i < nslab * 128; i += BYTEDOT_THREADS) sW[i] = wsrc[i];
 
     uint64_t corr = 0;
     if (I32) {                 // 2^31 * (sum of this chunk's column weights)
@@ -128,44 +165,47 @@ __device__ __forceinline__ void bytedot_tile(const MatJob& job, uint32_t local, 
 
     const int64_t pitch = job.ld * (int64_t)ESZ;
     uint64_t part = 0;
-    for (int rg = r0 + warp * 32; rg < r1; rg += NWARP * 32) {
-        int32_t acc[2][4];
-        const char* p[2][2];
+    for (int rg = r0 + warp * (16 * MT); rg < r1; rg += NWARP * (16 * MT)) {
+        int32_t acc[MT][4];
+        const char* p[MT][2];
 #pragma unroll
-        for (int mt = 0; mt < 2; mt++) {
+        for (int mt = 0; mt < MT; mt++) {
 #pragma unroll
             for (int c = 0; c < 4; c++) acc[mt][c] = 0;
 #pragma unroll
             for (int h = 0; h < 2; h++) {
                 const int row = min(rg + 16 * mt + g + 8 * h, r1 - 1);     // clamped: never out of bounds
-                p[mt][h] = (const char*)job.mat + (int64_t)row * pitch + cb0 + 16 * t;
+                p[mt][h] = (const char*)job.mat + (int64_t)row * pitch + cb0 + 64 * t;
             }
         }
-#pragma unroll 2
+#pragma unroll BYTEDOT_UNROLL
         for (int s = 0; s < nslab; s++) {
-            const int64_t left = row_bytes - (cb0 + 64 * s + 16 * t);     // bytes of the row from this vector on
-            const bool full = left >= 16;
-            const int nvalid = left <= 0 ? 0 : (int)min((int64_t)16, left) / ESZ;
-            uint4 d[2][2];
+            const int64_t left = row_bytes - (cb0 + 256 * s + 64 * t);    // bytes of the row from this thread's piece on
+            uint32_t d[MT][2][16];
 #pragma unroll
-            for (int mt = 0; mt < 2; mt++)
+            for (int mt = 0; mt < MT; mt++)
 #pragma unroll
-                for (int h = 0; h < 2; h++)
-                    d[mt][h] = nvalid > 0 ? load_vec<T, VEC>(p[mt][h] + 64 * s, full, nvalid) : make_uint4(0, 0, 0, 0);
-            const uint4 w = sW[s * 32 + lane];
+                for (int h = 0; h < 2; h++) load64<T, VL>(p[mt][h] + 256 * s, left, d[mt][h]);
+            uint4 w[4];
 #pragma unroll
-            for (int mt = 0; mt < 2; mt++) {
-                uint4 x = d[mt][0], y = d[mt][1];
+            for (int i = 0; i < 4; i++) w[i] = sW[(s * 4 + i) * 32 + lane];
+#pragma unroll
+            for (int mt = 0; mt < MT; mt++) {
                 if (I32) {
-                    x.x ^= 0x80000000u; x.y ^= 0x80000000u; x.z ^= 0x80000000u; x.w ^= 0x80000000u;
-                    y.x ^= 0x80000000u; y.y ^= 0x80000000u; y.z ^= 0x80000000u; y.w ^= 0x80000000u;
+#pragma unroll
+                    for (int i = 0; i < 16; i++) { d[mt][0][i] ^= 0x80000000u; d[mt][1][i] ^= 0x80000000u; }
                 }
-                mma_m16n8k32<!I32>(acc[mt], x.x, y.x, x.y, y.y, w.x, w.y);
-                mma_m16n8k32<!I32>(acc[mt], x.z, y.z, x.w, y.w, w.z, w.w);
+#pragma unroll
+                for (int i = 0; i < 4; i++) {        // 16-byte piece i feeds two MMAs
+                    mma_m16n8k32<!I32>(acc[mt], d[mt][0][4 * i], d[mt][1][4 * i], d[mt][0][4 * i + 1],
+                                       d[mt][1][4 * i + 1], w[i].x, w[i].y);
+                    mma_m16n8k32<!I32>(acc[mt], d[mt][0][4 * i + 2], d[mt][1][4 * i + 2], d[mt][0][4 * i + 3],
+                                       d[mt][1][4 * i + 3], w[i].z, w[i].w);
+                }
             }
         }
 #pragma unroll
-        for (int mt = 0; mt < 2; mt++)
+        for (int mt = 0; mt < MT; mt++)
 #pragma unroll
             for (int h = 0; h < 2; h++) {
                 const int row = rg + 16 * mt + g + 8 * h;
@@ -182,15 +222,18 @@ __device__ __forceinline__ void bytedot_tile(const MatJob& job, uint32_t local, 
     }
 }
 
-template <bool I32, bool POINT>
+// MT = MMA row tiles (16 rows each) a warp carries per pass: more rows in flight per thread
+// against more registers.
+template <bool I32, bool POINT, int MT>
 __global__ void __launch_bounds__(BYTEDOT_THREADS) bytedot_kernel(const MatJob* jobs, int njobs)
 {
-    __shared__ uint4 sW[(BYTEDOT_CHUNK_BYTES / 64) * 32];          // 32 KiB of weight limbs
+    __shared__ uint4 sW[(BYTEDOT_CHUNK_BYTES / 256) * 128];         // 32 KiB of weight limbs
     __shared__ uint64_t red[33];
     const MatJob job = jobs[find_job(jobs, njobs, blockIdx.x)];
     const uint32_t local = blockIdx.x - job.tile0;
-    if (job.vec) bytedot_tile<I32, POINT, true>(job, local, sW, red);
-    else bytedot_tile<I32, POINT, false>(job, local, sW, red);
+    if (job.vec == 2) bytedot_tile<I32, POINT, 2, MT>(job, local, sW, red);
+    else if (job.vec == 1) bytedot_tile<I32, POINT, 1, MT>(job, local, sW, red);
+    else bytedot_tile<I32, POINT, 0, MT>(job, local, sW, red);
 }
 
 // ------------------------------------------------------------------------------------------

@@ -15,8 +15,18 @@ constexpr int COLBIND_VECS = 128;              // 16-byte vectors per column chu
 constexpr int COLBIND_ROWS_PER_WARP = 4;
 constexpr int MAX_TILE_ROWS = 1024;            // eq entries staged per tile by the row-binding kernels
 // Tensor-core (int8 MMA) contraction kernels.
-constexpr int BYTEDOT_THREADS = 256;           // 8 warps, each sweeping 32 rows at a time
-constexpr int BYTEDOT_CHUNK_BYTES = 4096;      // byte-columns per tile (4096 int8 / 1024 int32 columns)
+#ifndef IMM_BYTEDOT_THREADS
+#define IMM_BYTEDOT_THREADS 256
+#endif
+#ifndef IMM_BYTEDOT_CHUNK_BYTES
+#define IMM_BYTEDOT_CHUNK_BYTES 4096
+#endif
+#ifndef IMM_BYTEDOT_UNROLL
+#define IMM_BYTEDOT_UNROLL 1
+#endif
+constexpr int BYTEDOT_THREADS = IMM_BYTEDOT_THREADS;          // warps sweep 16 or 32 rows at a time
+constexpr int BYTEDOT_CHUNK_BYTES = IMM_BYTEDOT_CHUNK_BYTES;  // byte-columns per tile (multiple of 256)
+constexpr int BYTEDOT_UNROLL = IMM_BYTEDOT_UNROLL;            // slabs of 256 byte-columns in flight per warp
 constexpr int ROWMMA_THREADS = 256;            // 8 warps x 128 columns
 constexpr int ROWMMA_COLS = 1024;              // int8 columns per tile
 constexpr int SUMCHECK_THREADS = 1024;
@@ -36,7 +46,7 @@ struct MatJob {
     int32_t rows, cols;
     int32_t tile_rows;         // rows per tile
     int32_t nrb, ncc;          // row blocks, column chunks
-    int32_t vec;               // 1: rows are 16-byte aligned -> 128-bit loads
+    int32_t vec;               // 2: rows 32-byte aligned, 1: 16-byte aligned, 0: element-wise loads
     uint32_t tile0;            // first tile of this job in the launch
     uint32_t pad_;
 };

@@ -189,7 +189,7 @@ def measured_peaks():
 # DRAM traffic of the claim kernel per algorithmic byte, from the ncu capture summarised under
 # profiles/ (dram__bytes_read.sum + dram__bytes_write.sum over 4*m*n); None until a capture of the
 # current kernel exists.
-CLAIM_KERNEL_TRAFFIC_RATIO = 240.57 / 234.881024  # bytedot_kernel<1,1,1>, 256-bit loads
+CLAIM_KERNEL_TRAFFIC_RATIO = 240.14 / 234.881024  # bytedot_kernel<1,1,1>, per-warp partials, no per-tile offset sum
 
 
 # ------------------------------------------------------------------------ our arm

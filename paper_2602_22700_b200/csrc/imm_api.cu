@@ -6,6 +6,7 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <algorithm>
 #include <string>
 #include <vector>
 
@@ -66,11 +67,6 @@ bool use_mma()
     const char* s = getenv("IMM_CONTRACT");
     return !(s && strcmp(s, "alu") == 0);
 }
-// columns (elements) per tile of the prover's three contractions
-int a_tile_cols(bool mma) { return mma ? ROWMMA_COLS : rowbind_cols(IMM_I8); }
-int b_tile_cols(bool mma) { return mma ? BYTEDOT_CHUNK_BYTES : colbind_cols(IMM_I8); }
-int c_tile_cols(bool mma) { return mma ? BYTEDOT_CHUNK_BYTES / 4 : rowbind_cols(IMM_I32); }
-
 struct Shape { int64_t rows, cols; };
 
 // Rows per tile: the largest candidate that still yields enough tiles to fill the GPU several
@@ -93,6 +89,42 @@ int pick_tile_rows(const std::vector<Shape>& mats, int cols_per_tile, const char
         if (tiles >= target) return c;
     }
     return 32;
+}
+
+// Tile geometry of a tensor-core contraction: rows x width, width in the kernel's own unit
+// (byte-columns for the byte-dot kernel, int8 columns for the row-binding kernel).
+struct Geom { int rows, width; };
+
+int64_t count_tiles(const std::vector<Shape>& mats, int rows, int width)
+{
+    int64_t tiles = 0;
+    for (const Shape& s : mats) tiles += ((s.rows + rows - 1) / rows) * ((s.cols + width - 1) / width);
+    return tiles;
+}
+
+// The largest tile among rows x widths that still cuts the batch into enough tiles to fill the GPU
+// several times over (the last wave is then a small fraction of the launch); for a batch too small
+// for that, the smallest tile, i.e. the most parallelism there is.  Large tiles amortise the
+// per-tile set-up (weight limbs staged in shared memory) and keep DRAM pages open longer.
+Geom pick_geom(const std::vector<Shape>& mats, const int* rows, int nrows, const int* widths, int nwidths,
+               int tiles_per_sm, const char* env_rows, const char* env_width)
+{
+    const int64_t target = (int64_t)148 * env_int("IMM_TILES_PER_SM", tiles_per_sm);
+    Geom best{rows[nrows - 1], widths[nwidths - 1]};          // candidates are listed largest first
+    int64_t best_area = -1;
+    for (int i = 0; i < nrows; i++)
+        for (int k = 0; k < nwidths; k++) {
+            const int64_t area = (int64_t)rows[i] * widths[k];
+            if (area > best_area && count_tiles(mats, rows[i], widths[k]) >= target) {
+                best = Geom{rows[i], widths[k]};
+                best_area = area;
+            }
+        }
+    // overrides for sweeps; snapped to the candidate lists' ranges
+    const int fr = env_int(env_rows, 0), fw = env_int(env_width, 0);
+    if (fr) { int v = fr < rows[nrows - 1] ? rows[nrows - 1] : fr > rows[0] ? rows[0] : fr; best.rows = v / rows[nrows - 1] * rows[nrows - 1]; }
+    if (fw) { int v = fw < widths[nwidths - 1] ? widths[nwidths - 1] : fw > widths[0] ? widths[0] : fw; best.width = v / widths[nwidths - 1] * widths[nwidths - 1]; }
+    return best;
 }
 
 void fill_job(MatJob& j, const void* mat, int dtype, int64_t rows, int64_t cols, int64_t ld,
@@ -125,14 +157,16 @@ struct Plan {
     int nproofs = 0;
     int max_b = 0;
     bool mma = true;
-    int max_weight_words = 0;
-    size_t off_wtasks = 0;
+    int64_t max_cover = 0;                     // most entries an eq task covers (table or padded limb tables)
     int rows_a = 0, rows_b = 0, rows_c = 0;
+    int cols_a = 0, cols_b = 0, cols_c = 0;    // columns (elements) per tile of the three contractions
+    int mt_b = 2, mt_c = 1;                    // MMA row tiles per warp pass of the byte-dot kernels
     uint32_t tiles_a = 0, tiles_b = 0, tiles_c = 0;
     // byte offsets from the workspace base
     size_t off_proofs = 0, off_jobs_a = 0, off_jobs_b = 0, off_jobs_c = 0, off_eq = 0, header_bytes = 0;
     struct PerProof {
-        size_t e_row, e_col, part_a, part_b, part_c, tab;
+        size_t e_row, e_col, part_a, part_b, part_c, sum_row, sum_col;
+        int n_sum_row, n_sum_col;
         size_t w_rows, w_cols_b, w_cols_c;          // limb tables (tensor-core back end)
         int nw_rows, nw_cols_b, nw_cols_c;          // their sizes in 32-bit words
         int a, b, c, n_part_a, n_part_b, n_part_c;
@@ -164,12 +198,33 @@ Plan make_plan(const imm_matmul_desc* descs, int nproofs)
         sc.push_back({descs[i].m, descs[i].n});
     }
     p.mma = use_mma();
-    const int acols = a_tile_cols(p.mma), bcols = b_tile_cols(p.mma), ccols = c_tile_cols(p.mma);
-    p.rows_a = pick_tile_rows(sa, acols, "IMM_TILE_ROWS_A");
-    // measured on the decoder-block workload: B (32 rows per warp pass) is best at 256 rows per tile,
-    // C (16 rows per warp pass) at 512-1024
-    p.rows_b = pick_tile_rows(sb, bcols, "IMM_TILE_ROWS_B", p.mma ? 256 : MAX_TILE_ROWS);
-    p.rows_c = pick_tile_rows(sc, ccols, "IMM_TILE_ROWS_C");
+    if (p.mma) {
+        // A: rows x (128 columns per warp).  B, C: rows x byte-columns; a block pass covers
+        // 128 rows per MMA row tile, so shorter tiles would leave warps idle.  Measured on the
+        // decoder-block workload: B (two row tiles per warp) is best at 256 rows per tile, C (one) at
+        // 512-1024.
+        static const int rows_a[] = {1024, 512, 256, 128, 64, 32}, widths_a[] = {1024, 512, 256, 128};
+        static const int rows_b[] = {256}, rows_c[] = {1024, 512, 256, 128};
+        static const int chunks[] = {4096, 2048, 1024, 512, 256};
+        p.mt_b = env_int("IMM_BYTEDOT_MT_B", 2) == 1 ? 1 : 2;
+        p.mt_c = env_int("IMM_BYTEDOT_MT_C", 1) == 2 ? 2 : 1;
+        std::vector<Shape> scb;                               // C as a byte matrix
+        for (const Shape& s : sc) scb.push_back({s.rows, 4 * s.cols});
+        // tiles per SM aimed at, from sweeps over 1024...16384 tokens: the row-binding kernel (a
+        // warp streams its own 128 columns) needs fewer, larger tiles than the byte-dot kernels
+        const Geom ga = pick_geom(sa, rows_a, 6, widths_a, 4, 12, "IMM_TILE_ROWS_A", "IMM_TILE_COLS_A");
+        const Geom gb = pick_geom(sb, rows_b, 1, chunks, 5, 24, "IMM_TILE_ROWS_B", "IMM_CHUNK_B");
+        const Geom gc = pick_geom(scb, rows_c, 4, chunks, 5, 24, "IMM_TILE_ROWS_C", "IMM_CHUNK_C");
+        p.rows_a = ga.rows; p.cols_a = ga.width;
+        p.rows_b = gb.rows; p.cols_b = gb.width;
+        p.rows_c = gc.rows; p.cols_c = gc.width / 4;
+    } else {
+        p.cols_a = rowbind_cols(IMM_I8); p.cols_b = colbind_cols(IMM_I8); p.cols_c = rowbind_cols(IMM_I32);
+        p.rows_a = pick_tile_rows(sa, p.cols_a, "IMM_TILE_ROWS_A");
+        p.rows_b = pick_tile_rows(sb, p.cols_b, "IMM_TILE_ROWS_B");
+        p.rows_c = pick_tile_rows(sc, p.cols_c, "IMM_TILE_ROWS_C");
+    }
+    const int acols = p.cols_a, bcols = p.cols_b, ccols = p.cols_c;
 
     size_t off = 0;
     p.off_proofs = off; off = align_up(off + sizeof(ProofDev) * nproofs);
@@ -177,7 +232,6 @@ Plan make_plan(const imm_matmul_desc* descs, int nproofs)
     p.off_jobs_b = off; off = align_up(off + sizeof(MatJob) * nproofs);
     p.off_jobs_c = off; off = align_up(off + sizeof(MatJob) * nproofs);
     p.off_eq = off;     off = align_up(off + sizeof(EqTask) * 2 * nproofs);
-    p.off_wtasks = off; off = align_up(off + sizeof(WeightTask) * 3 * nproofs);
     p.header_bytes = off;
 
     uint64_t ta = 0, tb = 0, tc = 0;
@@ -191,13 +245,19 @@ Plan make_plan(const imm_matmul_desc* descs, int nproofs)
         q.n_part_b = (int)((d.n + bcols - 1) / bcols);
         const int64_t c_nrb = (d.m + p.rows_c - 1) / p.rows_c;
         const int64_t c_ncc = (d.n + ccols - 1) / ccols;
-        q.n_part_c = (int)(c_nrb * c_ncc);
+        q.n_part_c = (int)(c_nrb * c_ncc) * (p.mma ? BYTEDOT_THREADS / 32 : 1);   // tensor-core kernel: one per warp
+        const int64_t slice = 4 * (int64_t)EQ_SLICE_QUADS;                  // entries per block of the eq kernel
+        q.n_sum_row = (int)((std::max<int64_t>((int64_t)1 << q.a, (d.m + 31) / 32 * 32) + slice - 1) / slice);
+        q.n_sum_col = (int)((std::max<int64_t>((int64_t)1 << q.c, (d.n + 255) / 256 * 256) + slice - 1) / slice);
+        if (((int64_t)1 << q.a) > p.max_cover) p.max_cover = (int64_t)1 << q.a;
+        if (((int64_t)1 << q.c) > p.max_cover) p.max_cover = (int64_t)1 << q.c;
         q.e_row = off;  off = align_up(off + sizeof(imm_fe) * ((size_t)1 << q.a));
         q.e_col = off;  off = align_up(off + sizeof(imm_fe) * ((size_t)1 << q.c));
         q.part_a = off; off = align_up(off + sizeof(imm_fe) * (size_t)q.n_part_a * d.k);
         q.part_b = off; off = align_up(off + sizeof(imm_fe) * (size_t)q.n_part_b * d.k);
         q.part_c = off; off = align_up(off + sizeof(imm_fe) * (size_t)q.n_part_c);
-        q.tab = off;    off = align_up(off + sizeof(imm_fe) * 2 * ((size_t)1 << q.b));
+        q.sum_row = off; off = align_up(off + sizeof(imm_fe) * (size_t)q.n_sum_row);
+        q.sum_col = off; off = align_up(off + sizeof(imm_fe) * (size_t)q.n_sum_col);
         q.nw_rows = q.nw_cols_b = q.nw_cols_c = 0;
         q.w_rows = q.w_cols_b = q.w_cols_c = 0;
         if (p.mma) {
@@ -207,12 +267,13 @@ Plan make_plan(const imm_matmul_desc* descs, int nproofs)
             q.w_rows = off;   off = align_up(off + 4 * (size_t)q.nw_rows);
             q.w_cols_b = off; off = align_up(off + 4 * (size_t)q.nw_cols_b);
             q.w_cols_c = off; off = align_up(off + 4 * (size_t)q.nw_cols_c);
-            if (q.nw_cols_c > p.max_weight_words) p.max_weight_words = q.nw_cols_c;
-            if (q.nw_rows > p.max_weight_words) p.max_weight_words = q.nw_rows;
+            const int64_t cover_rows = (d.m + 31) / 32 * 32, cover_cols = (d.n + 255) / 256 * 256;
+            if (cover_rows > p.max_cover) p.max_cover = cover_rows;
+            if (cover_cols > p.max_cover) p.max_cover = cover_cols;
         }
         ta += (uint64_t)q.n_part_a * ((d.k + acols - 1) / acols);
         tb += (uint64_t)((d.k + p.rows_b - 1) / p.rows_b) * q.n_part_b;
-        tc += (uint64_t)q.n_part_c;
+        tc += (uint64_t)(c_nrb * c_ncc);
     }
     if (ta > 0x7FFFFFFFu || tb > 0x7FFFFFFFu || tc > 0x7FFFFFFFu) { p.status = IMM_ERR_SHAPE; return p; }
     p.tiles_a = (uint32_t)ta; p.tiles_b = (uint32_t)tb; p.tiles_c = (uint32_t)tc;
@@ -412,8 +473,7 @@ int imm_sumcheck_matmul_prove(const imm_matmul_desc* descs_host, int nproofs, ui
     MatJob* jb = (MatJob*)(hdr.data() + p.off_jobs_b);
     MatJob* jc = (MatJob*)(hdr.data() + p.off_jobs_c);
     EqTask* eq = (EqTask*)(hdr.data() + p.off_eq);
-    WeightTask* wt = (WeightTask*)(hdr.data() + p.off_wtasks);
-    const int acols = a_tile_cols(p.mma), bcols = b_tile_cols(p.mma), ccols = c_tile_cols(p.mma);
+    const int acols = p.cols_a, bcols = p.cols_b, ccols = p.cols_c;
     uint32_t ta = 0, tb = 0, tc = 0;
     for (int i = 0; i < nproofs; i++) {
         const imm_matmul_desc& d = descs_host[i];
@@ -424,32 +484,37 @@ int imm_sumcheck_matmul_prove(const imm_matmul_desc* descs_host, int nproofs, ui
         P.part_a = (imm_fe*)(base + q.part_a);
         P.part_b = (imm_fe*)(base + q.part_b);
         P.part_c = (imm_fe*)(base + q.part_c);
-        P.tab = (imm_fe*)(base + q.tab);
         P.proof_id = d.proof_id;
         P.m = (int32_t)d.m; P.k = (int32_t)d.k; P.n = (int32_t)d.n;
         P.a = q.a; P.b = q.b; P.c = q.c;
         P.n_part_a = q.n_part_a; P.n_part_b = q.n_part_b; P.n_part_c = q.n_part_c;
+        P.sum_row = (imm_fe*)(base + q.sum_row); P.sum_col = (imm_fe*)(base + q.sum_col);
+        P.n_sum_row = q.n_sum_row; P.n_sum_col = q.n_sum_col;
+        P.c_offset = p.mma ? 1 : 0;
 
         fill_job(ja[i], d.A, IMM_I8, d.m, d.k, d.lda, p.rows_a, acols);
         ja[i].eq_row = P.e_row; ja[i].out = (imm_fe*)P.part_a; ja[i].tile0 = ta;
         ta += (uint32_t)(ja[i].nrb * ja[i].ncc);
         fill_job(jb[i], d.B, IMM_I8, d.k, d.n, d.ldb, p.rows_b, bcols);
-        jb[i].eq_col = P.e_col; jb[i].out = (imm_fe*)P.part_b; jb[i].tile0 = tb;
+        jb[i].eq_col = P.e_col; jb[i].out = (imm_fe*)P.part_b; jb[i].tile0 = tb; jb[i].chunk = bcols;
         tb += (uint32_t)(jb[i].nrb * jb[i].ncc);
         fill_job(jc[i], d.C, IMM_I32, d.m, d.n, d.ldc, p.rows_c, ccols);
         jc[i].eq_row = P.e_row; jc[i].eq_col = P.e_col; jc[i].out = (imm_fe*)P.part_c; jc[i].tile0 = tc;
+        jc[i].chunk = 4 * ccols;
         tc += (uint32_t)(jc[i].nrb * jc[i].ncc);
 
         if (p.mma) {
             ja[i].wtab = (const uint32_t*)(base + q.w_rows);
             jb[i].wtab = (const uint32_t*)(base + q.w_cols_b);
             jc[i].wtab = (const uint32_t*)(base + q.w_cols_c);
-            wt[3 * i + 0] = WeightTask{P.e_row, (uint32_t*)(base + q.w_rows), (int32_t)d.m, q.nw_rows, W_ROWS, 0};
-            wt[3 * i + 1] = WeightTask{P.e_col, (uint32_t*)(base + q.w_cols_b), (int32_t)d.n, q.nw_cols_b, W_COLS_I8, 0};
-            wt[3 * i + 2] = WeightTask{P.e_col, (uint32_t*)(base + q.w_cols_c), (int32_t)d.n, q.nw_cols_c, W_COLS_I32, 0};
         }
-        eq[2 * i] = EqTask{P.e_row, seed, d.proof_id, 1u, q.a};
-        eq[2 * i + 1] = EqTask{P.e_col, seed, d.proof_id, 2u, q.c};
+        eq[2 * i] = EqTask{P.e_row, seed, d.proof_id, 1u, q.a,
+                           p.mma ? (uint32_t*)(base + q.w_rows) : nullptr, nullptr, nullptr, (int32_t)d.m, 0,
+                           p.mma ? (imm_fe*)(base + q.sum_row) : nullptr};
+        eq[2 * i + 1] = EqTask{P.e_col, seed, d.proof_id, 2u, q.c, nullptr,
+                               p.mma ? (uint32_t*)(base + q.w_cols_b) : nullptr,
+                               p.mma ? (uint32_t*)(base + q.w_cols_c) : nullptr, (int32_t)d.n, 0,
+                               p.mma ? (imm_fe*)(base + q.sum_col) : nullptr};
     }
     if (ta != p.tiles_a || tb != p.tiles_b || tc != p.tiles_c) return IMM_ERR_ARG;   // planner invariant
 
@@ -459,16 +524,14 @@ int imm_sumcheck_matmul_prove(const imm_matmul_desc* descs_host, int nproofs, ui
 #define PROF_MARK(i) do { if (prof) CU(cudaEventRecord(pev[i], st)); } while (0)
     CU(cudaMemcpyAsync(base, hdr.data(), hdr.size(), cudaMemcpyHostToDevice, st));
     PROF_MARK(0);
-    CU(launch_eq_batch((const EqTask*)(base + p.off_eq), 2 * nproofs, st));
-    if (p.mma)
-        CU(launch_weights((const WeightTask*)(base + p.off_wtasks), 3 * nproofs, p.max_weight_words, st));
+    CU(launch_eq_batch((const EqTask*)(base + p.off_eq), 2 * nproofs, p.max_cover, st));
     PROF_MARK(1);
     if (p.mma) {
-        CU(launch_bytedot(true, true, env_int("IMM_BYTEDOT_MT_C", 1), (const MatJob*)(base + p.off_jobs_c), nproofs, p.tiles_c, st));
+        CU(launch_bytedot(true, true, p.mt_c, (const MatJob*)(base + p.off_jobs_c), nproofs, p.tiles_c, st));
         PROF_MARK(2);
-        CU(launch_rowmma((const MatJob*)(base + p.off_jobs_a), nproofs, p.tiles_a, st));
+        CU(launch_rowmma((const MatJob*)(base + p.off_jobs_a), nproofs, p.tiles_a, p.cols_a / 128, st));
         PROF_MARK(3);
-        CU(launch_bytedot(false, false, env_int("IMM_BYTEDOT_MT_B", 2), (const MatJob*)(base + p.off_jobs_b), nproofs, p.tiles_b, st));
+        CU(launch_bytedot(false, false, p.mt_b, (const MatJob*)(base + p.off_jobs_b), nproofs, p.tiles_b, st));
     } else {
         CU(launch_rowbind(IMM_I32, true, (const MatJob*)(base + p.off_jobs_c), nproofs, p.tiles_c, st));
         PROF_MARK(2);
@@ -478,7 +541,7 @@ int imm_sumcheck_matmul_prove(const imm_matmul_desc* descs_host, int nproofs, ui
     }
     PROF_MARK(4);
     CU(launch_sumcheck((const ProofDev*)(base + p.off_proofs), nproofs, seed, d_transcripts, stride,
-                       d_status, p.max_b, st));
+                       d_status, p.max_b, env_int("IMM_SC_CLUSTER", 0), st));
     PROF_MARK(5);
 #undef PROF_MARK
     if (prof) g_prof_calls++;

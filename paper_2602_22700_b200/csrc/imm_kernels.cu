@@ -6,6 +6,8 @@
 
 #include <type_traits>
 
+#include <cooperative_groups.h>
+
 #include "gl64.cuh"
 #include "imm_kernels.h"
 #include "imm_plan.h"
@@ -73,13 +75,22 @@ __device__ __forceinline__ void mad_wide(int64_t& acc, int32_t x, int32_t y)
     asm("mad.wide.s32 %0, %1, %2, %0;" : "+l"(acc) : "r"(x), "r"(y));
 }
 
-// Find the job a tile belongs to: jobs are ordered by tile0.
+// Find the job a tile belongs to: jobs are ordered by tile0 and jobs[0].tile0 = 0.  The lanes of
+// a warp probe 32 evenly spaced jobs at once, so 1024 jobs take two dependent loads instead of
+// ten.  Called by whole warps.
 __device__ __forceinline__ int find_job(const MatJob* jobs, int njobs, uint32_t tile)
 {
-    int lo = 0, hi = njobs - 1;
-    while (lo < hi) {
-        int mid = (lo + hi + 1) >> 1;
-        if (jobs[mid].tile0 <= tile) lo = mid; else hi = mid - 1;
+    const int lane = threadIdx.x & 31;
+    int lo = 0, n = njobs;
+    while (n > 1) {
+        const int step = (n + 31) >> 5;
+        const int idx = lo + lane * step;
+        const bool ok = idx < lo + n && jobs[idx].tile0 <= tile;
+        const uint32_t mask = __ballot_sync(0xFFFFFFFFu, ok) | 1u;      // the probes that hold form a prefix
+        const int k = 31 - __clz(mask);
+        const int end = lo + n;
+        lo += k * step;
+        n = min(step, end - lo);
     }
     return lo;
 }
@@ -133,17 +144,6 @@ __device__ void eq_fill(imm_fe* out, int nvars, const uint64_t* r_sh, uint64_t* 
     const uint32_t mask = (1u << nlo) - 1;
     for (int64_t i = threadIdx.x; i < total; i += blockDim.x)
         out[i] = gl::mul(hi_t[i >> nlo], lo_t[(uint32_t)i & mask]);
-}
-
-__global__ void __launch_bounds__(1024) eq_batch_kernel(const EqTask* tasks)
-{
-    __shared__ uint64_t r_sh[MAX_EQ_VARS];
-    __shared__ uint64_t lo_t[1024], hi_t[1024];
-    const EqTask t = tasks[blockIdx.x];
-    if ((int)threadIdx.x < t.nvars)
-        r_sh[threadIdx.x] = gl::challenge(t.seed, t.proof_id, t.domain, threadIdx.x);
-    __syncthreads();
-    eq_fill(t.out, t.nvars, r_sh, lo_t, hi_t);
 }
 
 __global__ void __launch_bounds__(1024) eq_direct_kernel(EqDirect rr, int nvars, imm_fe* out)
@@ -462,15 +462,32 @@ __global__ void __launch_bounds__(1024) sum_all_kernel(const imm_fe* parts, int6
 }
 
 // ------------------------------------------------------------------------------------------
-// sumcheck rounds: one block per proof
+// sumcheck rounds: one thread-block cluster per proof
 // ------------------------------------------------------------------------------------------
 // Round j works on tables a[], b[] of 2h entries (h = 2^(b-1-j)) and sends
 //   g(0) = sum_{y<h} a[y] b[y],  g(1) = sum a[y+h] b[y+h],  g(2) = sum (2a[y+h]-a[y]) (2b[y+h]-b[y]),
-// then folds a[y] <- a[y] + r_j (a[y+h] - a[y]) (same for b).  Challenges are public coins, so the
-// fold of round j does not wait for g_j: each pass folds with r_j AND accumulates round j+1's
-// three sums from the values it has just produced (a thread folds the two pairs that form one
-// pair of the next round).  Tables start in global memory (L2-resident) and move to shared
-// memory as soon as the folded pair of tables fits; folding is in place.
+// then folds a[y] <- a[y] + r_j (a[y+h] - a[y]) (same for b).
+//
+// Three facts shape the kernel.  (1) Challenges are public coins, so nothing waits for a round
+// polynomial: a pass folds with r_j AND accumulates round j+1's three sums from the values it
+// has just produced (a thread folds the two pairs that form one pair of the next round), and the
+// partial sums of every round are reduced once, after the last round, not once per round:
+// a round costs one barrier.  (2) Rounds bind the index from its top bit down, so the first
+// J = b - 8 rounds never mix entries whose low 8 index bits differ: block c of the cluster owns
+// the entries whose low bits fall in its slice of 256 / (cluster size) values, runs those J
+// rounds on its own shared-memory tables, and hands its slice of the 256-entry folded tables
+// plus its partial sums to block 0 over distributed shared memory; block 0 runs the last 8
+// rounds.  (3) Field addition is exact, so the order of these reductions does not change a word.
+// The cluster size is chosen per launch: small batches spread each proof over 8 SMs, large ones
+// keep one or two blocks per proof so that all proofs run at once.  Proofs of at most
+// SC_SOLO_VARS rounds are done by block 0 alone.
+
+constexpr int SC_WARPS = SUMCHECK_THREADS / 32;
+constexpr int SC_FINAL_VARS = 8;                 // rounds left to block 0 in a distributed proof
+constexpr int SC_FINAL = 1 << SC_FINAL_VARS;
+constexpr int SC_SOLO_VARS = 10;
+constexpr int SC_MAX_CAP = 8192;                 // entries per shared-memory table (2 x 64 KiB)
+constexpr int SC_PORTABLE_CLUSTER = 8;           // larger clusters need an opt-in and are used for k > 2^16 only
 
 struct Sums3 { uint64_t g0, g1, g2; };
 
@@ -487,90 +504,202 @@ __device__ __forceinline__ uint64_t fold1(uint64_t lo, uint64_t hi, uint64_t r)
     return gl::add(lo, gl::mul(r, gl::sub(hi, lo)));
 }
 
-__device__ __forceinline__ uint64_t sum_parts_at(const imm_fe* parts, int nparts, int len, int y)
+// sum_p parts[p][y]: the loads of eight partial vectors are issued together (the chain is bound by
+// memory latency, not by the additions).
+__device__ __forceinline__ uint64_t sum_parts_at(const imm_fe* __restrict__ parts, int nparts, int len, int y)
 {
-    if (y >= len) return 0;
+    const imm_fe* src = parts + y;
     uint64_t s = 0;
-    for (int p = 0; p < nparts; p++) s = gl::add(s, parts[(int64_t)p * len + y]);
+    int p = 0;
+    for (; p + 8 <= nparts; p += 8) {
+        uint64_t v[8];
+#pragma unroll
+        for (int pp = 0; pp < 8; pp++) v[pp] = __ldg(src + (int64_t)(p + pp) * len);
+#pragma unroll
+        for (int pp = 0; pp < 8; pp++) s = gl::add(s, v[pp]);
+    }
+    if (p < nparts) {
+        uint64_t v[8];
+#pragma unroll
+        for (int pp = 0; pp < 8; pp++) v[pp] = p + pp < nparts ? __ldg(src + (int64_t)(p + pp) * len) : 0;
+#pragma unroll
+        for (int pp = 0; pp < 8; pp++) s = gl::add(s, v[pp]);
+    }
     return s;
 }
 
-__global__ void __launch_bounds__(SUMCHECK_THREADS)
-sumcheck_kernel(const ProofDev* proofs, uint64_t seed, imm_fe* transcripts, int64_t stride,
-                int32_t* status, int smem_entries /* capacity per table, entries */)
+struct ScShared {
+    uint64_t r[MAX_K_VARS];                    // round challenges
+    uint64_t warp_sums[MAX_K_VARS][SC_WARPS][3];   // sums of a round whose pass ran on several warps
+    uint64_t lane_sums[MAX_K_VARS][32][3];     // sums of a round whose pass ran on warp 0 alone (not yet reduced)
+    uint64_t block_sums[MAX_K_VARS][3];        // this block's share of g_j(0..2); read by block 0
+    uint64_t fin[2][SC_FINAL];                 // block 0: the gathered 256-entry tables
+    uint64_t red[SC_WARPS];
+};
+
+// Keep a pass's sums of round j: `q` is the number of threads the pass used.  Both arrays start
+// at zero and every slot is written at most once.
+__device__ __forceinline__ void stash_sums(ScShared& sh, int j, const Sums3& acc, int q)
 {
-    extern __shared__ __align__(16) uint64_t smem[];       // [2][smem_entries] tables
-    __shared__ uint64_t red[33];
-    const ProofDev pr = proofs[blockIdx.x];
-    imm_fe* tr = transcripts + (int64_t)blockIdx.x * stride;
-    const int tid = threadIdx.x, nthr = blockDim.x;
-    const int b = pr.b;
-    const int64_t full = (int64_t)1 << b;
-
-    // claim c0 = sum of the partial sums of C
-    {
-        uint64_t s = 0;
-        for (int i = tid; i < pr.n_part_c; i += nthr) s = gl::add(s, pr.part_c[i]);
-        s = block_sum_fe(s, red);
-        if (tid == 0) tr[0] = s;
+    const int tid = threadIdx.x;
+    if (q <= 32) {
+        if (tid < 32) { uint64_t* w = sh.lane_sums[j][tid]; w[0] = acc.g0; w[1] = acc.g1; w[2] = acc.g2; }
+    } else if ((tid & ~31) < q) {
+        const uint64_t g0 = warp_sum_fe(acc.g0), g1 = warp_sum_fe(acc.g1), g2 = warp_sum_fe(acc.g2);
+        if ((tid & 31) == 0) { uint64_t* w = sh.warp_sums[j][tid >> 5]; w[0] = g0; w[1] = g1; w[2] = g2; }
     }
-    for (int64_t i = 3 * b + 3 + tid; i < stride; i += nthr) tr[i] = 0;
-    if (tid == 0) status[blockIdx.x] = 0;
+}
 
-    uint64_t* ta = pr.tab;                // current tables (global to start with)
-    uint64_t* tb = pr.tab + full;
-    Sums3 acc = {0, 0, 0};
-
-    if (b == 0) {
-        if (tid == 0) {
-            tr[1] = sum_parts_at(pr.part_a, pr.n_part_a, pr.k, 0);
-            tr[2] = sum_parts_at(pr.part_b, pr.n_part_b, pr.k, 0);
+// block_sums[j] = all stashed sums of round j, for j in [j0, j1); one warp per round.  Callers
+// put a block barrier before (stashes visible) and after (results visible).
+__device__ __forceinline__ void reduce_round_sums(ScShared& sh, int j0, int j1)
+{
+    const int lane = threadIdx.x & 31;
+    for (int j = j0 + (threadIdx.x >> 5); j < j1; j += SC_WARPS) {
+#pragma unroll
+        for (int comp = 0; comp < 3; comp++) {
+            uint64_t v = sh.lane_sums[j][lane][comp];
+            if (lane < SC_WARPS) v = gl::add(v, sh.warp_sums[j][lane][comp]);
+            v = warp_sum_fe(v);
+            if (lane == 0) sh.block_sums[j][comp] = v;
         }
+    }
+}
+
+// Rounds j0..j1-1 on shared-memory tables of n entries each: one pass for round j0's sums, then
+// pass j folds with r_j and accumulates round j+1's sums while j+1 < j1.  Every thread of the
+// block calls this, after a block barrier that made the tables visible.  A pass whose writers
+// all sit in warp 0 is followed by a warp barrier only (its readers sit in warp 0 too).
+__device__ __forceinline__ void run_rounds(ScShared& sh, uint64_t* ta, uint64_t* tb, int n, int j0, int j1)
+{
+    const int tid = threadIdx.x;
+    if (j0 >= j1) return;
+    {
+        const int h = n >> 1;
+        Sums3 acc = {0, 0, 0};
+#pragma unroll 1
+        for (int e = tid; e < h; e += SUMCHECK_THREADS) sums_add(acc, ta[e], ta[e + h], tb[e], tb[e + h]);
+        stash_sums(sh, j0, acc, h);
+    }
+#pragma unroll 1
+    for (int j = j0; j < j1; j++, n >>= 1) {
+        const uint64_t r = sh.r[j];
+        const int h = n >> 1, q = n >> 2;
+        if (n == 2) {
+            if (tid == 0) { ta[0] = fold1(ta[0], ta[1], r); tb[0] = fold1(tb[0], tb[1], r); }
+        } else {
+            const bool next = j + 1 < j1;
+            Sums3 acc = {0, 0, 0};
+#pragma unroll 1
+            for (int e = tid; e < q; e += SUMCHECK_THREADS) {
+                const uint64_t fa0 = fold1(ta[e], ta[e + h], r), fa1 = fold1(ta[e + q], ta[e + q + h], r);
+                const uint64_t fb0 = fold1(tb[e], tb[e + h], r), fb1 = fold1(tb[e + q], tb[e + q + h], r);
+                ta[e] = fa0; ta[e + q] = fa1; tb[e] = fb0; tb[e + q] = fb1;      // in place: only this thread reads them
+                if (next) sums_add(acc, fa0, fa1, fb0, fb1);
+            }
+            if (next) stash_sums(sh, j + 1, acc, q);
+        }
+        if (q > 32) __syncthreads(); else __syncwarp();
+    }
+}
+
+__global__ void __launch_bounds__(SUMCHECK_THREADS, 2)
+sumcheck_kernel(const ProofDev* proofs, uint64_t seed, imm_fe* transcripts, int64_t stride,
+                int32_t* status, int cap /* entries per shared-memory table */)
+{
+    namespace cg = cooperative_groups;
+    extern __shared__ __align__(16) uint64_t tabs[];       // [2][cap]
+    __shared__ ScShared sh;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int nc = (int)cluster.num_blocks(), c = (int)cluster.block_rank();
+    const int proof = blockIdx.x / nc;
+    const ProofDev pr = proofs[proof];
+    imm_fe* tr = transcripts + (int64_t)proof * stride;
+    const int tid = threadIdx.x;
+    const int b = pr.b;
+    const bool dist = nc > 1 && b > SC_SOLO_VARS;
+    if (!dist && c != 0) return;                           // (no cluster barrier is used in that case)
+
+    uint64_t* ta = tabs;
+    uint64_t* tb = tabs + cap;
+    // slice geometry: local entry e is global entry (e / W) * F + c * W + (e % W)
+    const int F = dist ? SC_FINAL : 1, W = dist ? SC_FINAL / nc : 1;
+    const int J = dist ? b - SC_FINAL_VARS : b;            // rounds run on the local tables
+    const int L = (int)(((int64_t)1 << b) / (dist ? nc : 1));
+
+    if (tid < b) sh.r[tid] = gl::challenge(seed, pr.proof_id, 3, (uint32_t)tid);
+    for (int i = tid; i < MAX_K_VARS * SC_WARPS * 3; i += SUMCHECK_THREADS) (&sh.warp_sums[0][0][0])[i] = 0;
+    for (int i = tid; i < MAX_K_VARS * 32 * 3; i += SUMCHECK_THREADS) (&sh.lane_sums[0][0][0])[i] = 0;
+    if (c == 0) {
+        // claim c0 = sum of the partial sums of C
+        uint64_t s = 0;
+        for (int i = tid; i < pr.n_part_c; i += SUMCHECK_THREADS) s = gl::add(s, pr.part_c[i]);
+        s = warp_sum_fe(s);
+        if ((tid & 31) == 0) sh.red[tid >> 5] = s;
+        __syncthreads();
+        if (tid < 32) s = warp_sum_fe(tid < SC_WARPS ? sh.red[tid] : 0);
+        if (tid < 32 && pr.c_offset) {
+            // the claim kernel summed unsigned bytes: every entry reads 2^31 too high
+            uint64_t sr = 0, sc = 0;
+            for (int i = tid; i < pr.n_sum_row; i += 32) sr = gl::add(sr, pr.sum_row[i]);
+            for (int i = tid; i < pr.n_sum_col; i += 32) sc = gl::add(sc, pr.sum_col[i]);
+            sr = warp_sum_fe(sr); sc = warp_sum_fe(sc);
+            s = gl::sub(s, gl::shl(gl::mul(sr, sc), 31));
+        }
+        if (tid == 0) { tr[0] = s; status[proof] = 0; }
+        for (int64_t i = 3 * b + 3 + tid; i < stride; i += SUMCHECK_THREADS) tr[i] = 0;
+    }
+    __syncthreads();
+
+    // build this block's entries from the partial vectors (all threads, one entry of each table
+    // at a time), then the local rounds
+#pragma unroll 1
+    for (int e = tid; e < L; e += SUMCHECK_THREADS) {
+        const int y = (e / W) * F + c * W + (e % W);
+        const bool live = y < pr.k;                        // entries past k are the zero padding
+        ta[e] = live ? sum_parts_at(pr.part_a, pr.n_part_a, pr.k, y) : 0;
+        tb[e] = live ? sum_parts_at(pr.part_b, pr.n_part_b, pr.k, y) : 0;
+    }
+    __syncthreads();
+    run_rounds(sh, ta, tb, L, 0, J);
+    __syncthreads();
+    reduce_round_sums(sh, 0, J);                           // this block's share of the local rounds' sums
+    if (!dist) {
+        __syncthreads();
+        if (tid < 3 * b) tr[1 + tid] = (&sh.block_sums[0][0])[tid];
+        if (tid == 0) { tr[3 * b + 1] = ta[0]; tr[3 * b + 2] = tb[0]; }
         return;
     }
 
-    // build the round-0 tables from the partial vectors and accumulate round 0's sums
-    {
-        const int h = (int)(full >> 1);
-        for (int y = tid; y < h; y += nthr) {
-            uint64_t a0 = sum_parts_at(pr.part_a, pr.n_part_a, pr.k, y);
-            uint64_t a1 = sum_parts_at(pr.part_a, pr.n_part_a, pr.k, y + h);
-            uint64_t b0 = sum_parts_at(pr.part_b, pr.n_part_b, pr.k, y);
-            uint64_t b1 = sum_parts_at(pr.part_b, pr.n_part_b, pr.k, y + h);
-            ta[y] = a0; ta[y + h] = a1; tb[y] = b0; tb[y + h] = b1;
-            sums_add(acc, a0, a1, b0, b1);
+    cluster.sync();                                        // every block's slice and sums are in place
+    if (c == 0) {
+        for (int i = tid; i < SC_FINAL; i += SUMCHECK_THREADS) {
+            const int cc = i / W, w = i % W;
+            sh.fin[0][i] = cluster.map_shared_rank(ta, cc)[w];
+            sh.fin[1][i] = cluster.map_shared_rank(tb, cc)[w];
+        }
+        if (tid < 3 * J) {
+            uint64_t v[SUMCHECK_MAX_CLUSTER];
+#pragma unroll
+            for (int cc = 0; cc < SUMCHECK_MAX_CLUSTER; cc++)
+                v[cc] = cc < nc ? cluster.map_shared_rank(&sh.block_sums[0][0], cc)[tid] : 0;
+            uint64_t s = 0;
+#pragma unroll
+            for (int cc = 0; cc < SUMCHECK_MAX_CLUSTER; cc++) s = gl::add(s, v[cc]);
+            tr[1 + tid] = s;
         }
     }
+    cluster.sync();                                        // remote reads are done: the other blocks may leave
+    if (c != 0) return;
 
-    for (int j = 0; j < b; j++) {
-        // publish round j's polynomial
-        uint64_t g0 = block_sum_fe(acc.g0, red);
-        uint64_t g1 = block_sum_fe(acc.g1, red);
-        uint64_t g2 = block_sum_fe(acc.g2, red);       // (also orders the table writes before the reads below)
-        if (tid == 0) { tr[1 + 3 * j] = g0; tr[2 + 3 * j] = g1; tr[3 + 3 * j] = g2; }
-        acc = {0, 0, 0};
-
-        const uint64_t r = gl::challenge(seed, pr.proof_id, 3, (uint32_t)j);
-        const int h = 1 << (b - 1 - j);                // size of the folded tables
-        uint64_t* da = ta;
-        uint64_t* db = tb;
-        if (ta != smem && h <= smem_entries) { da = smem; db = smem + smem_entries; }
-        if (h == 1) {
-            if (tid == 0) {
-                tr[3 * b + 1] = fold1(ta[0], ta[1], r);
-                tr[3 * b + 2] = fold1(tb[0], tb[1], r);
-            }
-        } else {
-            const int q = h >> 1;
-            for (int y = tid; y < q; y += nthr) {
-                uint64_t fa0 = fold1(ta[y], ta[y + h], r), fa1 = fold1(ta[y + q], ta[y + q + h], r);
-                uint64_t fb0 = fold1(tb[y], tb[y + h], r), fb1 = fold1(tb[y + q], tb[y + q + h], r);
-                da[y] = fa0; da[y + q] = fa1; db[y] = fb0; db[y + q] = fb1;
-                sums_add(acc, fa0, fa1, fb0, fb1);
-            }
-        }
-        ta = da; tb = db;
-    }
+    // block 0: the remaining rounds on the gathered tables
+    __syncthreads();
+    run_rounds(sh, sh.fin[0], sh.fin[1], SC_FINAL, J, b);
+    __syncthreads();
+    reduce_round_sums(sh, J, b);
+    __syncthreads();
+    if (tid < 3 * (b - J)) tr[1 + 3 * J + tid] = (&sh.block_sums[J][0])[tid];
+    if (tid == 0) { tr[3 * b + 1] = sh.fin[0][0]; tr[3 * b + 2] = sh.fin[1][0]; }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -593,10 +722,12 @@ cudaError_t launch_eq_direct(const EqDirect& r, int nvars, imm_fe* out, cudaStre
     return cudaGetLastError();
 }
 
-cudaError_t launch_eq_batch(const EqTask* d_tasks, int ntasks, cudaStream_t st)
+cudaError_t launch_eq_batch(const EqTask* d_tasks, int ntasks, int64_t max_cover, cudaStream_t st)
 {
-    if (ntasks <= 0) return cudaSuccess;
-    eq_batch_kernel<<<ntasks, 1024, 0, st>>>(d_tasks);
+    if (ntasks <= 0 || max_cover <= 0) return cudaSuccess;
+    const int64_t slice = 4 * (int64_t)EQ_SLICE_QUADS;
+    dim3 grid((unsigned)((max_cover + slice - 1) / slice), (unsigned)ntasks);
+    eq_batch_kernel<<<grid, EQ_BATCH_THREADS, 0, st>>>(d_tasks);
     return cudaGetLastError();
 }
 
@@ -622,22 +753,14 @@ cudaError_t launch_colbind(int dtype, const MatJob* d_jobs, int njobs, uint32_t 
     return cudaGetLastError();
 }
 
-cudaError_t launch_weights(const WeightTask* d_tasks, int ntasks, int max_words, cudaStream_t st)
-{
-    if (ntasks <= 0 || max_words <= 0) return cudaSuccess;
-    dim3 grid((unsigned)((max_words + 255) / 256), (unsigned)ntasks);
-    weights_kernel<<<grid, 256, 0, st>>>(d_tasks);
-    return cudaGetLastError();
-}
-
 cudaError_t launch_bytedot(bool i32, bool point, int mt, const MatJob* d_jobs, int njobs, uint32_t ntiles,
                            cudaStream_t st)
 {
     if (ntiles == 0) return cudaSuccess;
 #define BD_LAUNCH(I, P, M) bytedot_kernel<I, P, M><<<ntiles, BYTEDOT_THREADS, 0, st>>>(d_jobs, njobs)
     if (i32) {
-        if (point) { if (mt == 2) BD_LAUNCH(true, true, 2); else BD_LAUNCH(true, true, 1); }
-        else { if (mt == 2) BD_LAUNCH(true, false, 2); else BD_LAUNCH(true, false, 1); }
+        if (!point) return cudaErrorInvalidValue;          // the offset int32 view serves point evaluation only
+        if (mt == 2) BD_LAUNCH(true, true, 2); else BD_LAUNCH(true, true, 1);
     } else {
         if (point) { if (mt == 2) BD_LAUNCH(false, true, 2); else BD_LAUNCH(false, true, 1); }
         else { if (mt == 2) BD_LAUNCH(false, false, 2); else BD_LAUNCH(false, false, 1); }
@@ -646,10 +769,11 @@ cudaError_t launch_bytedot(bool i32, bool point, int mt, const MatJob* d_jobs, i
     return cudaGetLastError();
 }
 
-cudaError_t launch_rowmma(const MatJob* d_jobs, int njobs, uint32_t ntiles, cudaStream_t st)
+cudaError_t launch_rowmma(const MatJob* d_jobs, int njobs, uint32_t ntiles, int warps, cudaStream_t st)
 {
     if (ntiles == 0) return cudaSuccess;
-    rowmma_kernel<<<ntiles, ROWMMA_THREADS, 0, st>>>(d_jobs, njobs);
+    if (warps < 1 || warps > ROWMMA_MAX_WARPS) return cudaErrorInvalidValue;
+    rowmma_kernel<<<ntiles, 32 * warps, 0, st>>>(d_jobs, njobs);
     return cudaGetLastError();
 }
 
@@ -667,18 +791,44 @@ cudaError_t launch_sum_all(const imm_fe* parts, int64_t count, imm_fe* out, cuda
 }
 
 cudaError_t launch_sumcheck(const ProofDev* d_proofs, int nproofs, uint64_t seed, imm_fe* transcripts,
-                            int64_t stride, int32_t* status, int max_b, cudaStream_t st)
+                            int64_t stride, int32_t* status, int max_b, int cluster, cudaStream_t st)
 {
     if (nproofs <= 0) return cudaSuccess;
-    int entries = max_b >= 1 ? (1 << (max_b - 1)) : 1;
-    if (entries > 8192) entries = 8192;                       // 2 tables x 8192 x 8 B = 128 KiB
-    const size_t smem = (size_t)entries * 2 * sizeof(uint64_t);
+    // Blocks per proof: as many as keep every proof of the batch resident at once (two blocks fit
+    // an SM), at most 8, and at least what the shared-memory tables need (a block holds its share
+    // of the 2^b entries of both tables).
+    int nc = 1;
+    if (max_b > SC_SOLO_VARS) {
+        while (2 * nc <= SC_PORTABLE_CLUSTER && (int64_t)2 * nc * nproofs <= 2 * 148) nc *= 2;
+        if (cluster == 1 || cluster == 2 || cluster == 4 || cluster == 8) nc = cluster;     // caller's choice
+        while (nc < SUMCHECK_MAX_CLUSTER && (((int64_t)1 << max_b) / nc) > SC_MAX_CAP) nc *= 2;
+    }
+    int64_t cap = ((int64_t)1 << (max_b > 0 ? max_b : 0)) / (max_b > SC_SOLO_VARS ? nc : 1);
+    if (cap < (1 << SC_SOLO_VARS)) cap = 1 << SC_SOLO_VARS;                // a solo proof inside a cluster launch
+    if (cap > SC_MAX_CAP) return cudaErrorInvalidValue;                      // k beyond 2^17
+    const size_t smem = (size_t)cap * 2 * sizeof(uint64_t);
     cudaError_t e = cudaFuncSetAttribute(sumcheck_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)smem);
     if (e != cudaSuccess) return e;
-    sumcheck_kernel<<<nproofs, SUMCHECK_THREADS, smem, st>>>(d_proofs, seed, transcripts, stride, status,
-                                                             entries);
-    return cudaGetLastError();
+    if (nc > SC_PORTABLE_CLUSTER) {
+        e = cudaFuncSetAttribute(sumcheck_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+        if (e != cudaSuccess) return e;
+    }
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3((unsigned)(nproofs * nc));
+    cfg.blockDim = dim3(SUMCHECK_THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr;
+    memset(&attr, 0, sizeof(attr));
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = (unsigned)nc;
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, sumcheck_kernel, d_proofs, seed, transcripts, stride, status, (int)cap);
 }
 
 }  // namespace imm

@@ -39,7 +39,7 @@ __device__ __forceinline__ uint64_t combine_limbs(int32_t lo, int32_t hi, int t)
 }
 
 // ------------------------------------------------------------------------------------------
-// limb tables of the weights, in fragment order
+// eq tables of a batch and the limb tables of the weights, in fragment order
 // ------------------------------------------------------------------------------------------
 // W_COLS_*: weights of byte-columns.  Units of 256 byte-columns ("slabs"); a lane (4g + t) of
 //   the byte-dot kernel owns bytes 64t..64t+63 of a slab, and its 64 weight bytes are limb g of
@@ -49,43 +49,122 @@ __device__ __forceinline__ uint64_t combine_limbs(int32_t lo, int32_t hi, int t)
 // W_ROWS: weights of rows for the transposed (row-binding) MMA.  Units of 32 rows; lane = 4g+t
 //   holds 8 bytes: byte u of word h is limb g of eq[32G + 16h + 4t + u].
 // Weights past the real extent are zero (the implicit zero padding).
+//
+// One block fills a slice of one table.  E[i] = hi[i >> nlo] * lo[i & (2^nlo - 1)] with the two
+// small tables built per block straight from the product definition (no barriers beyond one).
+// A thread produces four consecutive entries and, from the same registers, their words of the
+// limb tables: byte g of four 32-bit halves is a 4x4 byte transpose.
 
-__global__ void __launch_bounds__(256) weights_kernel(const WeightTask* tasks)
+__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
 {
-    const WeightTask tk = tasks[blockIdx.y];
-    const int wi = blockIdx.x * blockDim.x + threadIdx.x;
-    if (wi >= tk.nwords) return;
-    uint32_t word = 0;
-    if (tk.mode == W_ROWS) {
-        const int G = wi >> 6, lane = (wi >> 1) & 31, h = wi & 1;
-        const int g = lane >> 2, t = lane & 3;
-        const int row0 = 32 * G + 16 * h + 4 * t;
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
+    return d;
+}
+
+// rows r0..r3 of a 4x4 byte block -> columns c0..c3
+__device__ __forceinline__ void transpose4x4(uint32_t r0, uint32_t r1, uint32_t r2, uint32_t r3,
+                                             uint32_t& c0, uint32_t& c1, uint32_t& c2, uint32_t& c3)
+{
+    const uint32_t x0 = prmt(r0, r1, 0x5140), x1 = prmt(r0, r1, 0x7362);
+    const uint32_t y0 = prmt(r2, r3, 0x5140), y1 = prmt(r2, r3, 0x7362);
+    c0 = prmt(x0, y0, 0x5410); c1 = prmt(x0, y0, 0x7632);
+    c2 = prmt(x1, y1, 0x5410); c3 = prmt(x1, y1, 0x7632);
+}
+
+// limb[g], g = 0..7: byte v of limb[g] is byte g of w[v]
+__device__ __forceinline__ void limbs_of4(const uint64_t (&w)[4], uint32_t (&limb)[8])
+{
+    transpose4x4((uint32_t)w[0], (uint32_t)w[1], (uint32_t)w[2], (uint32_t)w[3], limb[0], limb[1], limb[2], limb[3]);
+    transpose4x4((uint32_t)(w[0] >> 32), (uint32_t)(w[1] >> 32), (uint32_t)(w[2] >> 32), (uint32_t)(w[3] >> 32),
+                 limb[4], limb[5], limb[6], limb[7]);
+}
+
+// eq(r, x) over `cnt` variables r[0..cnt), variable 0 = top bit of x
+__device__ __forceinline__ uint64_t eq_product(const uint64_t* r, const uint64_t* one_minus_r, int cnt, uint32_t x)
+{
+    uint64_t v = 1;
+    for (int t = 0; t < cnt; t++) v = gl::mul(v, ((x >> (cnt - 1 - t)) & 1) ? r[t] : one_minus_r[t]);
+    return v;
+}
+
+__global__ void __launch_bounds__(EQ_BATCH_THREADS) eq_batch_kernel(const EqTask* tasks)
+{
+    __shared__ uint64_t r_sh[MAX_EQ_VARS], omr_sh[MAX_EQ_VARS];
+    __shared__ uint64_t lo_t[1024], hi_t[1024];
+    const EqTask tk = tasks[blockIdx.y];
+    const int64_t total = (int64_t)1 << tk.nvars;
+    // entries this task has to cover: the table itself, and the limb tables' zero padding
+    const int64_t pad = tk.w_rows ? 32 : 256;
+    const int64_t cover = (tk.w_rows || tk.w_cols_i8 || tk.w_cols_i32)
+                              ? max(total, ((int64_t)tk.extent + pad - 1) / pad * pad) : total;
+    const int64_t q0 = (int64_t)blockIdx.x * EQ_SLICE_QUADS;
+    if (4 * q0 >= cover) return;
+    __shared__ uint64_t red[33];
+    uint64_t slice_sum = 0;
+
+    if ((int)threadIdx.x < tk.nvars) {
+        const uint64_t r = gl::challenge(tk.seed, tk.proof_id, tk.domain, threadIdx.x);
+        r_sh[threadIdx.x] = r;
+        omr_sh[threadIdx.x] = gl::sub(1, r);
+    }
+    __syncthreads();
+    const int nlo = (tk.nvars + 1) / 2, nhi = tk.nvars - nlo;
+    for (int x = threadIdx.x; x < (1 << nhi); x += EQ_BATCH_THREADS) hi_t[x] = eq_product(r_sh, omr_sh, nhi, x);
+    for (int x = threadIdx.x; x < (1 << nlo); x += EQ_BATCH_THREADS) lo_t[x] = eq_product(r_sh + nhi, omr_sh + nhi, nlo, x);
+    __syncthreads();
+    const uint32_t mask = (1u << nlo) - 1;
+
+    const int64_t q1 = min(q0 + EQ_SLICE_QUADS, (cover + 3) / 4);
+    for (int64_t u = q0 + threadIdx.x; u < q1; u += EQ_BATCH_THREADS) {
+        const int64_t i0 = 4 * u;
+        uint64_t w[4];
 #pragma unroll
-        for (int u = 0; u < 4; u++) {
-            uint64_t e = (row0 + u < tk.extent) ? tk.eq[row0 + u] : 0;
-            word |= (uint32_t)((e >> (8 * g)) & 0xFF) << (8 * u);
+        for (int v = 0; v < 4; v++) {
+            const int64_t i = i0 + v;
+            const uint64_t e = i < total ? gl::mul(hi_t[i >> nlo], lo_t[(uint32_t)i & mask]) : 0;
+            if (i < total) tk.out[i] = e;
+            w[v] = i < tk.extent ? e : 0;
+            slice_sum = gl::add(slice_sum, w[v]);
         }
-    } else {
-        const int s = wi >> 9, piece = (wi >> 7) & 3, lane = (wi >> 2) & 31, r = wi & 3;
-        const int g = lane >> 2, t = lane & 3;
-        const int q0 = 256 * s + 64 * t + 16 * piece + 4 * r;
-        if (tk.mode == W_COLS_I8) {
+        uint32_t limb[8];
+        if (tk.w_rows && i0 < ((int64_t)tk.extent + 31) / 32 * 32) {
+            limbs_of4(w, limb);
+            const int64_t G = i0 >> 5;
+            const int h = (int)(i0 >> 4) & 1, t = (int)(i0 >> 2) & 3;
 #pragma unroll
-            for (int b = 0; b < 4; b++) {
-                uint64_t e = (q0 + b < tk.extent) ? tk.eq[q0 + b] : 0;
-                word |= (uint32_t)((e >> (8 * g)) & 0xFF) << (8 * b);
-            }
-        } else {
-            const int j = q0 >> 2;
-            const uint64_t e = (j < tk.extent) ? tk.eq[j] : 0;
+            for (int g = 0; g < 8; g++) tk.w_rows[G * 64 + (4 * g + t) * 2 + h] = limb[g];
+        }
+        if (tk.w_cols_i8 && i0 < ((int64_t)tk.extent + 255) / 256 * 256) {
+            limbs_of4(w, limb);
+            const int64_t sl = i0 >> 8;
+            const int t = (int)(i0 >> 6) & 3, piece = (int)(i0 >> 4) & 3, r = (int)(i0 >> 2) & 3;
 #pragma unroll
-            for (int b = 0; b < 4; b++) {
-                uint64_t w = gl::shl(e, 8 * b);
-                word |= (uint32_t)((w >> (8 * g)) & 0xFF) << (8 * b);
+            for (int g = 0; g < 8; g++) tk.w_cols_i8[((sl * 4 + piece) * 32 + 4 * g + t) * 4 + r] = limb[g];
+        }
+        if (tk.w_cols_i32 && i0 < ((int64_t)tk.extent + 63) / 64 * 64) {
+            // column j = i0 + v weighs its four bytes by e, e 2^8, e 2^16, e 2^24; its words sit at
+            // position v of a 16-byte piece, so the quad fills one piece per limb
+            uint32_t word[8][4];
+#pragma unroll
+            for (int v = 0; v < 4; v++) {
+                const uint64_t sh[4] = {w[v], gl::shl(w[v], 8), gl::shl(w[v], 16), gl::shl(w[v], 24)};
+                limbs_of4(sh, limb);
+#pragma unroll
+                for (int g = 0; g < 8; g++) word[g][v] = limb[g];
             }
+            const int64_t sl = i0 >> 6;
+            const int t = (int)(i0 >> 4) & 3, piece = (int)(i0 >> 2) & 3;
+            uint4* dst = reinterpret_cast<uint4*>(tk.w_cols_i32);
+#pragma unroll
+            for (int g = 0; g < 8; g++)
+                dst[(sl * 4 + piece) * 32 + 4 * g + t] = make_uint4(word[g][0], word[g][1], word[g][2], word[g][3]);
         }
     }
-    tk.out[wi] = word;
+    if (tk.slice_sums) {                       // (uniform over the block)
+        slice_sum = block_sum_fe(slice_sum, red);
+        if (threadIdx.x == 0) tk.slice_sums[blockIdx.x] = slice_sum;
+    }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -93,11 +172,13 @@ __global__ void __launch_bounds__(256) weights_kernel(const WeightTask* tasks)
 // ------------------------------------------------------------------------------------------
 // Serves the column binding of int8 B (W = eq_col) and the claim on int32 C seen as an
 // m x 4n byte matrix (W[4j+b] = eq_col[j] 2^(8b)).  For int32 the top byte of every word is
-// flipped (x ^ 0x80000000) so that all four bytes are unsigned; the value then reads 2^31 too
-// high, which is undone per row by subtracting 2^31 * sum_j eq_col[j] over the tile's columns.
-//   POINT = false: out[chunk][row] = u[row]           (partial over this column chunk)
-//   POINT = true : out[tile] = sum_rows eq_row[row] * u[row]
-// One tile = tile_rows rows x BYTEDOT_CHUNK_BYTES byte-columns.  A warp sweeps 16*MT rows (MT MMA
+// flipped (x ^ 0x80000000) so that all four bytes are unsigned; every entry then reads 2^31 too
+// high, which the consumer of the partial sums undoes once per matrix by subtracting
+// 2^31 * (sum of the row weights) * (sum of the column weights).
+//   POINT = false (int8 only): out[chunk][row] = u[row]      (partial over this column chunk)
+//   POINT = true : out[tile][warp] = sum over the warp's rows of eq_row[row] * u[row]
+// One tile = tile_rows rows x job.chunk byte-columns (chosen per batch: wide for large inputs, narrow
+// so that small ones still spread over all SMs).  A warp sweeps 16*MT rows (MT MMA
 // row tiles) across the chunk in slabs of 256 byte-columns; within a slab a thread owns 64
 // CONTIGUOUS bytes of each of its 2*MT rows (two 256-bit loads), so four neighbouring lanes read
 // 256 contiguous bytes of a row -- measured to stream at the rate of a linear read, where
@@ -137,8 +218,9 @@ __device__ __forceinline__ void load64(const char* p, int64_t left, uint32_t (&d
 }
 
 template <bool I32, bool POINT, int VL, int MT>
-__device__ __forceinline__ void bytedot_tile(const MatJob& job, uint32_t local, uint4* sW, uint64_t* red)
+__device__ __forceinline__ void bytedot_tile(const MatJob& job, uint32_t local, uint4* sW)
 {
+    static_assert(POINT || !I32, "the int32 byte view is offset by 2^31 per entry: point evaluation only");
     using T = typename std::conditional<I32, int32_t, int8_t>::type;
     constexpr int ESZ = (int)sizeof(T);
     constexpr int NWARP = BYTEDOT_THREADS / 32;
@@ -146,21 +228,14 @@ __device__ __forceinline__ void bytedot_tile(const MatJob& job, uint32_t local, 
     const int r0 = rbi * job.tile_rows;
     const int r1 = min(r0 + job.tile_rows, job.rows);
     const int64_t row_bytes = (int64_t)job.cols * ESZ;
-    const int64_t cb0 = (int64_t)cci * BYTEDOT_CHUNK_BYTES;
-    const int nslab = (int)min((int64_t)(BYTEDOT_CHUNK_BYTES / 256), (row_bytes - cb0 + 255) / 256);
+    const int64_t cb0 = (int64_t)cci * job.chunk;
+    const int nslab = (int)min((int64_t)(job.chunk / 256), (row_bytes - cb0 + 255) / 256);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int g = lane >> 2, t = lane & 3;
 
     const uint4* wsrc = reinterpret_cast<const uint4*>(job.wtab) + (cb0 / 256) * 128;
     for (int i = threadIdx.x; i < nslab * 128; i += BYTEDOT_THREADS) sW[i] = wsrc[i];
 
-    uint64_t corr = 0;
-    if (I32) {                 // 2^31 * (sum of this chunk's column weights)
-        const int j0 = (int)(cb0 / 4), j1 = min(job.cols, j0 + BYTEDOT_CHUNK_BYTES / 4);
-        uint64_t s = 0;
-        for (int j = j0 + threadIdx.x; j < j1; j += BYTEDOT_THREADS) s = gl::add(s, job.eq_col[j]);
-        corr = gl::shl(block_sum_fe(s, red), 31);
-    }
     __syncthreads();
 
     const int64_t pitch = job.ld * (int64_t)ESZ;
@@ -211,29 +286,28 @@ __device__ __forceinline__ void bytedot_tile(const MatJob& job, uint32_t local, 
                 const int row = rg + 16 * mt + g + 8 * h;
                 uint64_t u = combine_limbs(acc[mt][2 * h], acc[mt][2 * h + 1], t);
                 if (t == 0 && row < r1) {
-                    if (POINT) part = gl::add(part, gl::mul(job.eq_row[row], gl::sub(u, corr)));
-                    else job.out[(int64_t)cci * job.rows + row] = I32 ? gl::sub(u, corr) : u;
+                    if (POINT) part = gl::add(part, gl::mul(job.eq_row[row], u));
+                    else job.out[(int64_t)cci * job.rows + row] = u;
                 }
             }
     }
-    if (POINT) {
-        part = block_sum_fe(part, red);
-        if (threadIdx.x == 0) job.out[local] = part;
+    if (POINT) {                               // one partial per warp: no block barrier at the end of a tile
+        part = warp_sum_fe(part);
+        if (lane == 0) job.out[(int64_t)local * NWARP + warp] = part;
     }
 }
 
 // MT = MMA row tiles (16 rows each) a warp carries per pass: more rows in flight per thread
-// against more registers.
+// against more registers (three resident blocks per SM with one row tile, two with two).
 template <bool I32, bool POINT, int MT>
-__global__ void __launch_bounds__(BYTEDOT_THREADS) bytedot_kernel(const MatJob* jobs, int njobs)
+__global__ void __launch_bounds__(BYTEDOT_THREADS, MT == 1 ? 3 : 2) bytedot_kernel(const MatJob* jobs, int njobs)
 {
-    __shared__ uint4 sW[(BYTEDOT_CHUNK_BYTES / 256) * 128];         // 32 KiB of weight limbs
-    __shared__ uint64_t red[33];
+    __shared__ uint4 sW[(BYTEDOT_MAX_CHUNK_BYTES / 256) * 128];     // up to 32 KiB of weight limbs
     const MatJob job = jobs[find_job(jobs, njobs, blockIdx.x)];
     const uint32_t local = blockIdx.x - job.tile0;
-    if (job.vec == 2) bytedot_tile<I32, POINT, 2, MT>(job, local, sW, red);
-    else if (job.vec == 1) bytedot_tile<I32, POINT, 1, MT>(job, local, sW, red);
-    else bytedot_tile<I32, POINT, 0, MT>(job, local, sW, red);
+    if (job.vec == 2) bytedot_tile<I32, POINT, 2, MT>(job, local, sW);
+    else if (job.vec == 1) bytedot_tile<I32, POINT, 1, MT>(job, local, sW);
+    else bytedot_tile<I32, POINT, 0, MT>(job, local, sW);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -243,24 +317,8 @@ __global__ void __launch_bounds__(BYTEDOT_THREADS) bytedot_kernel(const MatJob* 
 // its M dimension the column index: each thread loads 16 columns of 8 rows (coalesced 16-byte
 // loads, a warp reads 128 contiguous bytes of each row) and transposes 4x4 byte blocks in
 // registers with byte permutes so that every register holds one column at four consecutive
-// rows.  One tile = tile_rows rows x ROWMMA_COLS columns; each warp owns 128 columns.
-
-__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel)
-{
-    uint32_t d;
-    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
-    return d;
-}
-
-// rows r0..r3 of a 4x4 byte block -> columns c0..c3
-__device__ __forceinline__ void transpose4x4(uint32_t r0, uint32_t r1, uint32_t r2, uint32_t r3,
-                                             uint32_t& c0, uint32_t& c1, uint32_t& c2, uint32_t& c3)
-{
-    const uint32_t x0 = prmt(r0, r1, 0x5140), x1 = prmt(r0, r1, 0x7362);
-    const uint32_t y0 = prmt(r2, r3, 0x5140), y1 = prmt(r2, r3, 0x7362);
-    c0 = prmt(x0, y0, 0x5410); c1 = prmt(x0, y0, 0x7632);
-    c2 = prmt(x1, y1, 0x5410); c3 = prmt(x1, y1, 0x7632);
-}
+// rows.  One tile = tile_rows rows x (128 columns per warp of the block); the block size is chosen
+// per batch (8 warps for large inputs, fewer so that small ones still spread over all SMs).
 
 template <bool VEC>
 __device__ __forceinline__ void rowmma_tile(const MatJob& job, uint32_t local, uint2* sR)
@@ -273,10 +331,11 @@ __device__ __forceinline__ void rowmma_tile(const MatJob& job, uint32_t local, u
     const int g = lane >> 2, t = lane & 3;
 
     const uint2* wsrc = reinterpret_cast<const uint2*>(job.wtab) + (int64_t)(r0 / 32) * 32;
-    for (int i = threadIdx.x; i < ngroups * 32; i += ROWMMA_THREADS) sR[i] = wsrc[i];
+    for (int i = threadIdx.x; i < ngroups * 32; i += blockDim.x) sR[i] = wsrc[i];
     __syncthreads();
 
-    const int col = cci * ROWMMA_COLS + warp * 128 + 16 * g;      // this thread's 16 columns
+    const int tile_cols = (int)blockDim.x * 4;                    // 128 columns per warp
+    const int col = cci * tile_cols + warp * 128 + 16 * g;        // this thread's 16 columns
     const int nvalid = min(16, job.cols - col);
     const bool full = nvalid == 16;
     int32_t acc[8][4];
@@ -285,7 +344,7 @@ __device__ __forceinline__ void rowmma_tile(const MatJob& job, uint32_t local, u
 #pragma unroll
         for (int c = 0; c < 4; c++) acc[i][c] = 0;
 
-    if (warp * 128 + cci * ROWMMA_COLS < job.cols) {              // whole warp in or out
+    if (warp * 128 + cci * tile_cols < job.cols) {              // whole warp in or out
         for (int G = 0; G < ngroups; G++) {
             uint4 d[2][4];
 #pragma unroll
@@ -321,7 +380,7 @@ __device__ __forceinline__ void rowmma_tile(const MatJob& job, uint32_t local, u
         }
 }
 
-__global__ void __launch_bounds__(ROWMMA_THREADS) rowmma_kernel(const MatJob* jobs, int njobs)
+__global__ void __launch_bounds__(ROWMMA_MAX_WARPS * 32) rowmma_kernel(const MatJob* jobs, int njobs)
 {
     __shared__ uint2 sR[MAX_TILE_ROWS];                             // (MAX_TILE_ROWS / 32) groups x 32 lanes
     const MatJob job = jobs[find_job(jobs, njobs, blockIdx.x)];

@@ -18,18 +18,21 @@ constexpr int MAX_TILE_ROWS = 1024;            // eq entries staged per tile by 
 #ifndef IMM_BYTEDOT_THREADS
 #define IMM_BYTEDOT_THREADS 256
 #endif
-#ifndef IMM_BYTEDOT_CHUNK_BYTES
-#define IMM_BYTEDOT_CHUNK_BYTES 4096
+#ifndef IMM_BYTEDOT_MAX_CHUNK_BYTES
+#define IMM_BYTEDOT_MAX_CHUNK_BYTES 4096
 #endif
 #ifndef IMM_BYTEDOT_UNROLL
 #define IMM_BYTEDOT_UNROLL 1
 #endif
 constexpr int BYTEDOT_THREADS = IMM_BYTEDOT_THREADS;          // warps sweep 16 or 32 rows at a time
-constexpr int BYTEDOT_CHUNK_BYTES = IMM_BYTEDOT_CHUNK_BYTES;  // byte-columns per tile (multiple of 256)
+constexpr int BYTEDOT_MAX_CHUNK_BYTES = IMM_BYTEDOT_MAX_CHUNK_BYTES;  // most byte-columns per tile; a job's own
+                                                                     // chunk is a multiple of 256 up to this
 constexpr int BYTEDOT_UNROLL = IMM_BYTEDOT_UNROLL;            // slabs of 256 byte-columns in flight per warp
-constexpr int ROWMMA_THREADS = 256;            // 8 warps x 128 columns
-constexpr int ROWMMA_COLS = 1024;              // int8 columns per tile
-constexpr int SUMCHECK_THREADS = 1024;
+constexpr int ROWMMA_MAX_WARPS = 8;            // a block of w warps covers w x 128 int8 columns
+constexpr int EQ_BATCH_THREADS = 256;
+constexpr int EQ_SLICE_QUADS = 512;           // groups of four table entries per block of eq_batch_kernel
+constexpr int SUMCHECK_THREADS = 512;
+constexpr int SUMCHECK_MAX_CLUSTER = 16;    // most blocks per proof (a power of two dividing 256)
 constexpr int MAX_EQ_VARS = 20;
 constexpr int MAX_K_VARS = 17;
 
@@ -48,7 +51,7 @@ struct MatJob {
     int32_t nrb, ncc;          // row blocks, column chunks
     int32_t vec;               // 2: rows 32-byte aligned, 1: 16-byte aligned, 0: element-wise loads
     uint32_t tile0;            // first tile of this job in the launch
-    uint32_t pad_;
+    int32_t chunk;             // byte-dot kernel: byte-columns per tile (multiple of 256)
 };
 
 // Per-proof state of the round kernel.
@@ -57,32 +60,32 @@ struct ProofDev {
     imm_fe* e_col;             // 2^c entries
     const imm_fe* part_a;      // [n_part_a][k]   partial avec (one per row block of A)
     const imm_fe* part_b;      // [n_part_b][k]   partial bvec (one per column chunk of B)
-    const imm_fe* part_c;      // [n_part_c]      partial c0 (one per tile of C)
-    imm_fe* tab;               // 2 * 2^b entries: avec then bvec, padded with zeros
+    const imm_fe* part_c;      // [n_part_c]      partial c0 (one per tile, or per warp of a tile, of C)
+    const imm_fe* sum_row;     // [n_sum_row] slice sums of E_row over the real rows    } only when the claim
+    const imm_fe* sum_col;     // [n_sum_col] slice sums of E_col over the real columns } kernel leaves the
+                               //             2^31 offset of its unsigned bytes in part_c (c_offset != 0)
     uint64_t proof_id;
     int32_t m, k, n;
     int32_t a, b, c;           // ceil(log2 m), ceil(log2 k), ceil(log2 n)
     int32_t n_part_a, n_part_b, n_part_c;
-    int32_t pad_;
+    int32_t c_offset;          // 1: c0 = sum(part_c) - 2^31 * sum(sum_row) * sum(sum_col)
+    int32_t n_sum_row, n_sum_col;
 };
 
-// One limb table of eq weights in MMA fragment order (see weights_kernel).
-enum WeightMode { W_COLS_I8 = 0, W_COLS_I32 = 1, W_ROWS = 2 };
-struct WeightTask {
-    const imm_fe* eq;          // eq table
-    uint32_t* out;             // nwords 32-bit words
-    int32_t extent;            // real extent (columns or rows); weights past it are zero
-    int32_t nwords;
-    int32_t mode;
-    int32_t pad_;
-};
-
-// One eq table of a batch: r is derived in-kernel from (seed, proof_id, domain).
+// One eq table of a batch: r is derived in-kernel from (seed, proof_id, domain).  The same pass
+// can emit the table's limb tables for the tensor-core kernels (null = not wanted): weights of
+// entries at or past `extent` are zero.  Layouts: see eq_batch_kernel.
 struct EqTask {
-    imm_fe* out;
+    imm_fe* out;               // 2^nvars entries
     uint64_t seed, proof_id;
     uint32_t domain;
     int32_t nvars;
+    uint32_t* w_rows;          // ceil(extent / 32) * 64 words
+    uint32_t* w_cols_i8;       // ceil(extent / 256) * 512 words
+    uint32_t* w_cols_i32;      // ceil(4 * extent / 256) * 512 words
+    int32_t extent;
+    int32_t pad_;
+    imm_fe* slice_sums;        // one entry per block of the task: sum of its entries below `extent` (or null)
 };
 
 // A single eq table with r supplied by the caller (passed by value to the kernel).

@@ -202,6 +202,29 @@ def test_prove_single_matches_oracle(imm, oracle, backend, m, k, n):
     assert imm.sumcheck_verify(got, b, seed, pid) == (imm.OK, -1)
 
 
+@pytest.mark.parametrize("m,k,n", [(4, 20000, 5), (3, 40000, 2), (2, 70000, 3), (2, 131072, 2)])
+def test_prove_many_rounds(imm, oracle, m, k, n):
+    """15 to 17 rounds: the round kernel spreads one proof over the blocks of a cluster (16 blocks,
+    an opt-in cluster size, from 2^16 < k on)."""
+    rng = np.random.default_rng(k)
+    A, B, C = np_problem(rng, m, k, n)
+    got = gpu_prove(imm, [(A, B, C, 7)], 11)[0]
+    assert got == [int(w) for w in oracle.sumcheck_matmul_prove(A, B, C, 11, 7)]
+    assert imm.sumcheck_verify(got, oracle.ceil_log2(k), 11, 7) == (imm.OK, -1)
+
+
+@pytest.mark.parametrize("cluster", ["1", "2", "4", "8"])
+def test_round_kernel_cluster_sizes_give_the_same_words(imm, oracle, monkeypatch, cluster):
+    """A batch mixing short proofs (one block each) and long ones, for every cluster size."""
+    monkeypatch.setenv("IMM_SC_CLUSTER", cluster)
+    rng = np.random.default_rng(91)
+    shapes = [(5, 5000, 7), (3, 8, 2), (9, 2049, 4), (2, 1024, 3), (6, 8192, 2), (1, 1, 1), (4, 1025, 33)]
+    probs = [np_problem(rng, *s) + (20 + i,) for i, s in enumerate(shapes)]
+    got = gpu_prove(imm, probs, 17)
+    for (A, B, C, pid), t in zip(probs, got):
+        assert t == [int(w) for w in oracle.sumcheck_matmul_prove(A, B, C, 17, pid)]
+
+
 def test_prove_unaligned_leading_dimensions(imm, oracle, backend):
     """Rows that are not 16-byte aligned take the element-wise loads; same transcript."""
     rng = np.random.default_rng(78)

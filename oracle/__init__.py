@@ -1,8 +1,12 @@
-"""CPU oracle for the Goldilocks sumcheck matmul proof -- TEST INFRASTRUCTURE ONLY.
+"""CPU oracles -- TEST INFRASTRUCTURE ONLY.
 
-Only the tests, the smoke check and the benchmark's CPU-baseline leg may import this package.
-It wraps ``imm_oracle.c`` (plain C, ``% p`` on 128-bit integers) through ctypes and shares no
-code with the CUDA library.  See the header of ``imm_oracle.c`` for the conventions and the
-list of pins.
+Only the tests, the smoke check and the benchmark's CPU-baseline leg may import this package; it
+shares no code with the CUDA library.
+
+* the Goldilocks sumcheck matmul proof: ``imm_oracle.c`` (plain C, ``% p`` on 128-bit integers)
+  wrapped through ctypes and re-exported here; its header lists the conventions and the pins;
+* the logit distance distribution (TV / KL distances, Top-K distance, the per-request tail
+  statistic): ``oracle.ldd`` (plain numpy in float64); its header lists the readings and the pins.
 """
+from . import ldd_oracle as ldd  # noqa: F401
 from .imm_oracle import *  # noqa: F401,F403

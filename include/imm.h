@@ -227,6 +227,53 @@ int imm_sumcheck_verify(const imm_fe* transcript_host, int nrounds, uint64_t see
                         uint64_t proof_id, const imm_fe* expect_c0, const imm_fe* expect_a_fin,
                         const imm_fe* expect_b_fin, int* fail_at);
 
+/* ---------------------------------------------------------------------------------------------
+ * Logit distance distribution (LDD)
+ * ---------------------------------------------------------------------------------------------
+ * The auditing footprint of the paper: for every discrete decision of an audited request, the
+ * distance between the logits the deployed execution committed to and the logits of the reference
+ * execution (Section 4.2, definition of the logit distance distribution), the per-request tail
+ * statistic built on it (Section 5.3), and the Top-K distance that lets a server commit K indices
+ * instead of a whole logit vector (appendix on the verification of Top-K).
+ *
+ * Logit rows are float32, row-major: step i occupies entries [i*ld, i*ld + n) of its matrix
+ * (ld >= n).  Entries must be finite.  Rows that are 16-byte aligned (base pointer and ld*4) are
+ * read with 128-bit loads, others element by element.  All pointers are DEVICE pointers; calls
+ * enqueue on `stream` and do not synchronise; nothing is allocated.  The arithmetic is float32
+ * per entry (exp2-based softmax) with the cross-thread sums in float64; the Top-K distance is
+ * selected exactly and evaluated in float64.
+ */
+#define IMM_LDD_MAX_N (1 << 20)        /* entries per logit row                      */
+#define IMM_LDD_MAX_K 64               /* size of a Top-K index set                  */
+#define IMM_LDD_MAX_STEPS (1 << 27)    /* rows (or requests) per call                */
+
+/* tv[i] = 1/2 * sum_v |p_v - q_v| and kl[i] = sum_v q_v (log q_v - log p_v), where
+ * p = softmax(logits row i) (the deployed execution) and q = softmax(ref_logits row i) (the
+ * reference), temperature 1.  The paper names "KL divergence or TV distance" without fixing the
+ * KL direction: the reference distribution comes first here.
+ * Errors: IMM_ERR_ARG (null pointer), IMM_ERR_SHAPE (n <= 0, ld < n, n or steps beyond the limits
+ * above), IMM_ERR_ALIGN (pointers not aligned to their element size), IMM_ERR_CUDA. */
+int imm_ldd_tv_kl(const float* d_logits, const float* d_ref_logits, int64_t steps, int64_t n, int64_t ld,
+                  double* d_tv, double* d_kl, void* stream);
+
+/* dist[i] = min over rows l' whose K largest entries are exactly the index set I_i of
+ * ||l' - l_i||_1, with l_i = ref_logits row i and I_i = d_topk[i*k .. i*k + k) (k distinct
+ * indices in [0, n)).  It is 0 iff I_i is a valid top-K set of the row.  Computed as the minimum
+ * over thresholds t of  sum_{j not in I} max(l_j - t, 0) + sum_{i in I} max(t - l_i, 0).
+ * status[i] = IMM_OK, IMM_ERR_ARG (an index out of range or repeated; dist[i] = NaN), or
+ * IMM_ERR_LIMIT (more than a few thousand entries tie just above the K-th largest one after six
+ * refinements; dist[i] = NaN).  Errors of the call itself: as imm_ldd_tv_kl, plus IMM_ERR_SHAPE
+ * for k outside 1..min(n, IMM_LDD_MAX_K). */
+int imm_ldd_topk_distance(const float* d_ref_logits, int64_t steps, int64_t n, int64_t ld,
+                          const int32_t* d_topk, int k, double* d_dist, int32_t* d_status, void* stream);
+
+/* Per-request tail statistic: request r owns the steps offsets[r] .. offsets[r+1]-1 of `dist`
+ * (offsets: nrequests + 1 non-decreasing int64 values).  p[r] = (number of its steps with
+ * dist > t1) / (number of its steps), 0 for an empty request; flag[r] = 1 if p[r] > t2 else 0
+ * (d_flag may be null).  Both comparisons are strict, as the paper prints them. */
+int imm_ldd_tail_fraction(const double* d_dist, const int64_t* d_offsets, int64_t nrequests, double t1, double t2,
+                          double* d_p, int32_t* d_flag, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -15,6 +15,7 @@ import torch
 
 P = 0xFFFFFFFF00000001
 OK, REJECT = 0, 1
+ERR_ARG, ERR_SHAPE, ERR_ALIGN, ERR_WORKSPACE, ERR_NONCANONICAL, ERR_CUDA, ERR_LIMIT = -1, -2, -3, -4, -5, -6, -7
 I8, I32 = 0, 1
 BIND_ROWS, BIND_COLS = 0, 1
 FIELD_ADD, FIELD_SUB, FIELD_MUL = 0, 1, 2
@@ -28,7 +29,8 @@ EXPORTS = ("imm_version", "imm_last_cuda_error", "imm_challenge", "imm_field_bin
            "imm_mle_workspace", "imm_mle_partial_eval", "imm_mle_eval_point",
            "imm_sumcheck_matmul_workspace", "imm_sumcheck_matmul_prove",
            "imm_sumcheck_matmul_host_arena", "imm_sumcheck_matmul_prove_host", "imm_sumcheck_verify",
-           "imm_profile_enable", "imm_profile_calls", "imm_profile_read", "imm_mle_eval_point_noalloc")
+           "imm_profile_enable", "imm_profile_calls", "imm_profile_read", "imm_mle_eval_point_noalloc",
+           "imm_ldd_tv_kl", "imm_ldd_topk_distance", "imm_ldd_tail_fraction")
 NOALLOC_MAX_TILES = 8192
 PROFILE_PHASES = ("eq_tables", "claim_C", "bind_rows_A", "bind_cols_B", "sumcheck_rounds")
 
@@ -89,6 +91,12 @@ def lib() -> ctypes.CDLL:
     L.imm_profile_calls.argtypes = []
     L.imm_profile_read.restype = ci
     L.imm_profile_read.argtypes = [i64, vp, ci]
+    L.imm_ldd_tv_kl.restype = ci
+    L.imm_ldd_tv_kl.argtypes = [vp, vp, i64, i64, i64, vp, vp, vp]
+    L.imm_ldd_topk_distance.restype = ci
+    L.imm_ldd_topk_distance.argtypes = [vp, i64, i64, i64, vp, ci, vp, vp, vp]
+    L.imm_ldd_tail_fraction.restype = ci
+    L.imm_ldd_tail_fraction.argtypes = [vp, vp, i64, ctypes.c_double, ctypes.c_double, vp, vp, vp]
     L.imm_sumcheck_verify.restype = ci
     L.imm_sumcheck_verify.argtypes = [vp, ci, u64, u64, vp, vp, vp, vp]
     _lib = L
@@ -329,3 +337,53 @@ def sumcheck_verify(transcript: Sequence[int], nrounds: int, seed: int, proof_id
                                    opt(expect_a_fin), opt(expect_b_fin), ctypes.addressof(fail))
     _check(rc, "imm_sumcheck_verify")
     return rc, fail.value
+
+
+# ------------------------------------------------------------------ logit distance distribution
+
+
+def _logit_rows(t: torch.Tensor, what: str) -> Tuple[int, int, int]:
+    """(steps, n, ld) of a 2-D float32 CUDA tensor whose rows are contiguous."""
+    if not t.is_cuda:
+        raise ValueError(f"{what}: a CUDA tensor is required (there is no CPU path)")
+    if t.dtype != torch.float32 or t.dim() != 2 or (t.shape[1] > 1 and t.stride(1) != 1):
+        raise ValueError(f"{what}: expected a 2-D float32 tensor with contiguous rows")
+    return int(t.shape[0]), int(t.shape[1]), int(t.stride(0)) if t.shape[0] > 1 else max(int(t.stride(0)), int(t.shape[1]))
+
+
+def ldd_tv_kl(logits: torch.Tensor, ref_logits: torch.Tensor) -> Tuple[torch.Tensor, torch.Tensor]:
+    """TV distance and KL(reference || deployed) per row; returns two float64 tensors of ``steps``."""
+    steps, n, ld = _logit_rows(logits, "logits")
+    if _logit_rows(ref_logits, "ref_logits") != (steps, n, ld):
+        raise ValueError("logits and ref_logits must have the same shape and row stride")
+    tv = torch.empty(steps, dtype=torch.float64, device=logits.device)
+    kl = torch.empty(steps, dtype=torch.float64, device=logits.device)
+    _check(lib().imm_ldd_tv_kl(logits.data_ptr(), ref_logits.data_ptr(), steps, n, ld, tv.data_ptr(), kl.data_ptr(),
+                               _stream()), "imm_ldd_tv_kl")
+    return tv, kl
+
+
+def ldd_topk_distance(ref_logits: torch.Tensor, topk: torch.Tensor) -> Tuple[torch.Tensor, torch.Tensor]:
+    """Top-K distance of every row to its claimed index set (int32, steps x K); returns
+    (float64 distances, int32 per-row status)."""
+    steps, n, ld = _logit_rows(ref_logits, "ref_logits")
+    topk = _cuda(topk, torch.int32, "topk")
+    if topk.dim() != 2 or topk.shape[0] != steps or not topk.is_contiguous():
+        raise ValueError("topk: expected a contiguous int32 tensor of shape (steps, K)")
+    dist = torch.empty(steps, dtype=torch.float64, device=ref_logits.device)
+    status = torch.full((steps,), -99, dtype=torch.int32, device=ref_logits.device)
+    _check(lib().imm_ldd_topk_distance(ref_logits.data_ptr(), steps, n, ld, topk.data_ptr(), int(topk.shape[1]),
+                                       dist.data_ptr(), status.data_ptr(), _stream()), "imm_ldd_topk_distance")
+    return dist, status
+
+
+def ldd_tail_fraction(dist: torch.Tensor, offsets: torch.Tensor, t1: float, t2: float) -> Tuple[torch.Tensor, torch.Tensor]:
+    """p(t1) of every request and the flag p(t1) > t2; ``offsets`` is int64 with nrequests + 1 entries."""
+    dist = _cuda(dist, torch.float64, "dist")
+    offsets = _cuda(offsets, torch.int64, "offsets")
+    nreq = int(offsets.numel()) - 1
+    p = torch.empty(max(nreq, 0), dtype=torch.float64, device=dist.device)
+    flag = torch.empty(max(nreq, 0), dtype=torch.int32, device=dist.device)
+    _check(lib().imm_ldd_tail_fraction(dist.data_ptr(), offsets.data_ptr(), nreq, float(t1), float(t2), p.data_ptr(),
+                                       flag.data_ptr(), _stream()), "imm_ldd_tail_fraction")
+    return p, flag

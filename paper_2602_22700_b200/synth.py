@@ -71,14 +71,15 @@ def stream_u64(seed: int, tid: int, idx: torch.Tensor) -> torch.Tensor:
     return _mix64((idx + 1) * _s64(_G) + _s64(key))
 
 
-def _fill(seed: int, tid: int, rows: int, cols: int, device, fn, chunk_elems: int = 1 << 24):
-    out = torch.empty((rows, cols), dtype=torch.int8, device=device)
+def _fill(seed: int, tid: int, rows: int, cols: int, device, fn, chunk_elems: int = 1 << 24,
+          dtype=torch.int8):
+    out = torch.empty((rows, cols), dtype=dtype, device=device)
     flat = out.view(-1)
     total = rows * cols
     for start in range(0, total, chunk_elems):
         stop = min(total, start + chunk_elems)
         idx = torch.arange(start, stop, dtype=torch.int64, device=device)
-        flat[start:stop] = fn(stream_u64(seed, tid, idx)).to(torch.int8)
+        flat[start:stop] = fn(stream_u64(seed, tid, idx)).to(dtype)
     return out
 
 
@@ -259,3 +260,44 @@ def prover_field_macs(problems: List[Problem]) -> int:
 
 def proved_matmul_macs(problems: List[Problem]) -> int:
     return sum(m * k * n for (m, k, n) in (p.mkn for p in problems))
+
+
+# ---------------------------------------------------------------------------- logits for the LDD
+
+
+ROLE_LOGIT, ROLE_LOGIT_NOISE, ROLE_LOGIT_HOT = 16, 17, 18
+LOGIT_SCALE = 2.5 / 209.02           # byte sums have standard deviation ~209: bulk logits ~ N(0, 2.5^2)
+HOT_TOKENS = 12                      # entries per row lifted well above the bulk (the plausible next tokens)
+
+# deployment regimes, as noise added to the reference logits (standard deviation of the noise):
+# a benign reduced-precision run, an aggressive quantisation, and a different model altogether
+NOISE_BENIGN, NOISE_QUANTISED = 0.02, 0.25
+
+
+def reference_logits(seed: int, steps: int, vocab: int, device="cpu", group: int = 0) -> torch.Tensor:
+    """float32 logits (steps x vocab): an approx-Gaussian bulk plus HOT_TOKENS boosted entries per
+    row.  Built from integers and one float32 multiply, so CPU and CUDA give identical bits."""
+    s = _fill(seed, tid(group, ROLE_LOGIT), steps, vocab, device, lambda u: byte_sum(u) - 1020, dtype=torch.int32).to(torch.int64)
+    idx = torch.arange(steps * HOT_TOKENS, dtype=torch.int64, device=device)
+    u = stream_u64(seed, tid(group, ROLE_LOGIT_HOT), idx)
+    col = ((_lsr(u, 32) * vocab) >> 32).view(steps, HOT_TOKENS)                 # hot token index in [0, vocab)
+    lift = (700 + 60 * (HOT_TOKENS - torch.arange(HOT_TOKENS, device=device, dtype=torch.int64))).expand(steps, -1)
+    s.scatter_add_(1, col, lift.contiguous())                                   # integer adds: order-independent
+    return (s.to(torch.float32) * LOGIT_SCALE).contiguous()
+
+
+def deployed_logits(ref: torch.Tensor, seed: int, noise: float, group: int = 0) -> torch.Tensor:
+    """Reference logits plus seeded approx-Gaussian noise of standard deviation ``noise`` (two separately
+    rounded float32 operations per entry: identical bits on CPU and CUDA)."""
+    steps, vocab = ref.shape
+    z = _fill(seed, tid(group, ROLE_LOGIT_NOISE), steps, vocab, ref.device, lambda u: byte_sum(u) - 1020, dtype=torch.int32)
+    scaled = z.to(torch.float32) * (noise / 209.02)
+    return (ref + scaled).contiguous()
+
+
+def request_offsets(seed: int, steps: int, requests: int, device="cpu") -> torch.Tensor:
+    """int64 offsets (requests + 1) cutting ``steps`` decision steps into requests of seeded ragged lengths."""
+    idx = torch.arange(max(requests - 1, 0), dtype=torch.int64, device="cpu")
+    cuts = ((_lsr(stream_u64(seed, tid(0, ROLE_ROUTER), idx), 32) * (steps + 1)) >> 32).sort().values
+    out = torch.cat([torch.zeros(1, dtype=torch.int64), cuts, torch.full((1,), steps, dtype=torch.int64)])
+    return out.to(device)

@@ -1,0 +1,191 @@
+"""GPU parity of the logit-distance-distribution calls against the float64 oracle (run with -m gpu).
+
+Tolerances.  TV and KL are sums of float32 terms (exp2-based softmax, about 2e-6 relative per term,
+plus about 3e-6 from the float32 log-sum-exp that scales every term), so the absolute error of TV is
+below 1e-5 and that of KL below 1e-5 + 1e-4 * KL; the tests allow 2e-5 (+ 2e-4 relative for KL).
+The Top-K distance is selected exactly and evaluated in float64 on the float32 inputs: 1e-9 relative.
+The tail statistic is a count: exact.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+TV_TOL = 2e-5
+KL_ABS, KL_REL = 2e-5, 2e-4
+
+
+@pytest.fixture(scope="module")
+def imm():
+    if not torch.cuda.is_available():
+        pytest.fail("a CUDA device is required for -m gpu tests")
+    from paper_2602_22700_b200 import imm as binding
+    binding.lib()
+    return binding
+
+
+@pytest.fixture(scope="module")
+def synth():
+    from paper_2602_22700_b200 import synth as s
+    return s
+
+
+@pytest.fixture(scope="module")
+def ldd():
+    from oracle import ldd as o
+    return o
+
+
+def check_tv_kl(imm, ldd, x, y):
+    tv, kl = imm.ldd_tv_kl(x, y)
+    tv, kl = tv.cpu().numpy(), kl.cpu().numpy()
+    xs, ys = x.cpu().numpy(), y.cpu().numpy()
+    for i in range(xs.shape[0]):
+        want_tv, want_kl = ldd.tv_distance(xs[i], ys[i]), ldd.kl_divergence(xs[i], ys[i])
+        assert abs(tv[i] - want_tv) <= TV_TOL, (i, tv[i], want_tv)
+        assert abs(kl[i] - want_kl) <= KL_ABS + KL_REL * abs(want_kl), (i, kl[i], want_kl)
+
+
+@pytest.mark.parametrize("steps,n", [(7, 1), (5, 3), (9, 100), (4, 4097), (3, 16384), (3, 16388), (3, 40003),
+                                     (2, 128256), (2, 151936), (1, 300000)])
+@pytest.mark.parametrize("noise", ["benign", "quantised", "substituted"])
+def test_tv_kl_matches_oracle(imm, ldd, synth, steps, n, noise):
+    ref = synth.reference_logits(3, steps, n, device="cuda")
+    if noise == "substituted":
+        dep = synth.reference_logits(4, steps, n, device="cuda")
+    else:
+        dep = synth.deployed_logits(ref, 3, synth.NOISE_BENIGN if noise == "benign" else synth.NOISE_QUANTISED)
+    check_tv_kl(imm, ldd, dep, ref)
+
+
+def test_tv_kl_identical_rows_and_far_rows(imm, ldd, synth):
+    ref = synth.reference_logits(5, 4, 50000, device="cuda")
+    tv, kl = imm.ldd_tv_kl(ref, ref)
+    assert float(tv.abs().max()) <= 1e-6 and float(kl.abs().max()) <= 1e-6
+    far = ref.clone()
+    far[:, 123] += 60.0                                   # all mass on one entry
+    check_tv_kl(imm, ldd, far, ref)
+    check_tv_kl(imm, ldd, ref + 1000.0, ref - 500.0)      # shifts cancel: large magnitudes must not overflow
+
+
+def test_tv_kl_unaligned_rows_take_the_element_path(imm, ldd, synth):
+    steps, n = 5, 20001
+    ref = synth.reference_logits(6, steps, n, device="cuda")
+    dep = synth.deployed_logits(ref, 6, synth.NOISE_QUANTISED)
+
+    def odd(t, ld, off):
+        buf = torch.zeros(steps * ld + off + 8, dtype=torch.float32, device="cuda")
+        v = buf[off:off + steps * ld].view(steps, ld)[:, :n]
+        v.copy_(t)
+        return v
+
+    check_tv_kl(imm, ldd, odd(dep, n + 3, 1), odd(ref, n + 3, 1))
+    check_tv_kl(imm, ldd, odd(dep, n + 7, 0), odd(ref, n + 7, 0))      # aligned base, unaligned pitch
+
+
+def check_topk(imm, ldd, ref, topk, rel=1e-9):
+    dist, status = imm.ldd_topk_distance(ref, topk)
+    dist, status = dist.cpu().numpy(), status.cpu().numpy()
+    ys, idx = ref.cpu().numpy(), topk.cpu().numpy()
+    assert (status == 0).all(), status
+    for i in range(ys.shape[0]):
+        want = ldd.topk_distance(ys[i], idx[i])
+        assert abs(dist[i] - want) <= rel * max(1.0, abs(want)), (i, dist[i], want)
+    return dist
+
+
+@pytest.mark.parametrize("steps,n,k", [(6, 5, 2), (6, 64, 6), (5, 128, 8), (4, 1000, 20), (3, 16384, 20),
+                                        (3, 40003, 20), (3, 128256, 20), (2, 151936, 20), (2, 128256, 64),
+                                        (2, 300000, 1)])
+def test_topk_distance_matches_oracle(imm, ldd, synth, steps, n, k):
+    ref = synth.reference_logits(7, steps, n, device="cuda")
+    dep = synth.deployed_logits(ref, 7, synth.NOISE_QUANTISED)
+    claimed = torch.topk(dep, k, dim=1).indices.to(torch.int32).contiguous()      # what the server committed to
+    check_topk(imm, ldd, ref, claimed)
+    valid = torch.topk(ref, k, dim=1).indices.to(torch.int32).contiguous()
+    assert (check_topk(imm, ldd, ref, valid) == 0.0).all()                        # a valid top-K set costs nothing
+    rnd = torch.stack([torch.randperm(n, generator=torch.Generator().manual_seed(i))[:k] for i in range(steps)])
+    far = check_topk(imm, ldd, ref, rnd.to(torch.int32).cuda().contiguous())
+    if n > 4 * k:
+        assert (far > 0.0).all()
+
+
+def test_topk_distance_ties_and_adversarial_rows(imm, ldd):
+    n, k = 131072, 20
+    rows = [
+        torch.zeros(n),                                              # every entry ties
+        torch.arange(n, dtype=torch.float32),                        # ascending: thousands of entries above the first bound
+        torch.arange(n, 0, -1, dtype=torch.float32),                 # descending
+        torch.round(torch.randn(n, generator=torch.Generator().manual_seed(1)) * 2) / 2,   # heavy ties
+        torch.cat([torch.full((3000,), 5.0), torch.zeros(n - 3000)]),                      # a plateau above the rest
+    ]
+    ref = torch.stack(rows).cuda().contiguous()
+    g = torch.Generator().manual_seed(2)
+    sets = [torch.randperm(n, generator=g)[:k] for _ in rows]
+    sets[1] = torch.arange(k)                                        # the K smallest of the ascending row
+    topk = torch.stack(sets).to(torch.int32).cuda().contiguous()
+    check_topk(imm, ldd, ref, topk, rel=1e-12)
+
+
+def test_topk_distance_whole_row_inside_and_bad_indices(imm, ldd):
+    ref = torch.tensor([[3.0, 1.0, 2.0, 5.0], [0.5, 0.25, 4.0, -1.0]], device="cuda")
+    everything = torch.tensor([[0, 1, 2, 3], [3, 2, 1, 0]], dtype=torch.int32, device="cuda")
+    assert (check_topk(imm, ldd, ref, everything) == 0.0).all()
+    bad = torch.tensor([[0, 0], [1, 7]], dtype=torch.int32, device="cuda")          # repeated; out of range
+    dist, status = imm.ldd_topk_distance(ref, bad)
+    assert status.cpu().tolist() == [imm.ERR_ARG, imm.ERR_ARG]
+    assert all(math.isnan(v) for v in dist.cpu().tolist())
+    good_and_bad = torch.tensor([[3, 0], [2, -1]], dtype=torch.int32, device="cuda")
+    dist, status = imm.ldd_topk_distance(ref, good_and_bad)
+    assert status.cpu().tolist() == [0, imm.ERR_ARG] and float(dist[0]) == 0.0
+
+
+def test_tail_fraction_is_exact(imm, ldd, synth):
+    steps, requests = 5000, 37
+    rng = np.random.default_rng(8)
+    d = rng.uniform(0, 0.3, steps)
+    d[::17] = 0.1                                                   # entries equal to the threshold do not count
+    offsets = synth.request_offsets(8, steps, requests).numpy()
+    offsets[5] = offsets[4]                                         # an empty request
+    offsets.sort()
+    p, flag = imm.ldd_tail_fraction(torch.from_numpy(d).cuda(), torch.from_numpy(offsets).cuda(), 0.1, 0.65)
+    want = np.array([ldd.tail_fraction(d[offsets[r]:offsets[r + 1]], 0.1) if offsets[r + 1] > offsets[r] else 0.0
+                     for r in range(requests)])
+    assert (p.cpu().numpy() == want).all()
+    assert (flag.cpu().numpy() == (want > 0.65)).all()
+
+
+def test_audit_statistic_end_to_end(imm, ldd, synth):
+    """Distances on the GPU, then the per-request decision, against the oracle chain.  Steps whose TV
+    lies within the TV tolerance of t1 are left out of the count on both sides."""
+    steps, n, requests, t1, t2 = 96, 128256, 6, 0.05, 0.2
+    ref = synth.reference_logits(9, steps, n, device="cuda")
+    dep = synth.deployed_logits(ref, 9, synth.NOISE_QUANTISED)
+    tv, _ = imm.ldd_tv_kl(dep, ref)
+    offsets = synth.request_offsets(9, steps, requests)
+    p, flag = imm.ldd_tail_fraction(tv, offsets.cuda(), t1, t2)
+    xs, ys = dep.cpu().numpy(), ref.cpu().numpy()
+    want_tv = np.array([ldd.tv_distance(xs[i], ys[i]) for i in range(steps)])
+    assert np.abs(tv.cpu().numpy() - want_tv).max() <= TV_TOL
+    clear = np.abs(want_tv - t1) > TV_TOL
+    assert clear.all(), "pick another seed: a step sits on the threshold"
+    off = offsets.numpy()
+    want_p = ldd.request_tail_fractions(want_tv, off, t1)
+    assert (p.cpu().numpy() == want_p).all()
+    assert (flag.cpu().numpy().astype(bool) == ldd.flag_requests(want_tv, off, t1, t2)).all()
+    assert 0 < want_p.max() and want_p.min() < 1
+
+
+def test_ldd_calls_refuse_bad_arguments(imm, synth):
+    ref = synth.reference_logits(1, 2, 64, device="cuda")
+    with pytest.raises(ValueError):
+        imm.ldd_tv_kl(ref.cpu(), ref.cpu())
+    with pytest.raises(ValueError):
+        imm.ldd_tv_kl(ref, ref[:, :32].contiguous())
+    with pytest.raises(imm.ImmError):
+        imm.ldd_topk_distance(ref, torch.zeros((2, 65), dtype=torch.int32, device="cuda"))     # K beyond the limit
+    with pytest.raises(imm.ImmError):
+        imm.ldd_topk_distance(ref[:, :3].contiguous(), torch.zeros((2, 4), dtype=torch.int32, device="cuda"))  # K > n

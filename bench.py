@@ -47,6 +47,8 @@ def parse_args():
                     help="decoder (default, the metric's workload) or one of the smaller parity configurations")
     ap.add_argument("--layers", type=int, default=32)
     ap.add_argument("--tokens", type=int, default=None, help="token count (default: the configuration's own)")
+    ap.add_argument("--vocab", type=int, default=128256, help="ldd: entries per logit row")
+    ap.add_argument("--topk", type=int, default=20, help="ldd: size of the committed index sets")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=2)
@@ -63,12 +65,13 @@ WORKLOADS = {
     "qkv": (512, "dense-layer projection: A {tokens}x4096 times W 4096x4096, one proof"),
     "ffn": (2048, "dense FFN up/down pair: {tokens}x4096 times 4096x14336, requantised hidden times 14336x4096, two proofs"),
     "moe": (4096, "MoE expert batch: 8 experts 4096x14336, top-2 routing of {tokens} tokens, one proof per expert"),
+    "ldd": (8192, "logit distance distribution: {tokens} decision steps x vocabulary {vocab} (float32), TV + KL + Top-{topk} distance + tail statistic"),
 }
 L2_BYTES = 126 << 20
 
 
-def workload_name(config, layers, tokens):
-    return WORKLOADS[config][1].format(layers=layers, tokens=tokens)
+def workload_name(config, layers, tokens, vocab=128256, topk=20):
+    return WORKLOADS[config][1].format(layers=layers, tokens=tokens, vocab=vocab, topk=topk)
 
 
 def make_problems(config, seed, layers, tokens, device):
@@ -189,6 +192,7 @@ def measured_peaks():
 # DRAM traffic of the claim kernel per algorithmic byte, from the ncu capture summarised under
 # profiles/ (dram__bytes_read.sum + dram__bytes_write.sum over 4*m*n); None until a capture of the
 # current kernel exists.
+LDD_TVKL_TRAFFIC_RATIO = None   # tv_kl_kernel: (dram read + write) / (8 bytes per entry pair), same source
 CLAIM_KERNEL_TRAFFIC_RATIO = 240.14 / 234.881024  # bytedot_kernel<1,1,1>, per-warp partials, no per-tile offset sum
 
 
@@ -363,6 +367,158 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+# ------------------------------------------------------------------------ logit distance distribution
+
+
+def ldd_oracle_rows(dep, ref, topk, rows):
+    """The float64 oracle on the given rows: (tv, kl, top-K distance) lists."""
+    from oracle import ldd
+    tv, kl, dist = [], [], []
+    for i in rows:
+        tv.append(ldd.tv_distance(dep[i], ref[i]))
+        kl.append(ldd.kl_divergence(dep[i], ref[i]))
+        dist.append(ldd.topk_distance(ref[i], topk[i]))
+    return tv, kl, dist
+
+
+def run_ldd(args):
+    """One step = every decision step's TV and KL distance, its Top-K distance, and the per-request
+    tail statistic.  Not the headline workload: a second data-parallel path of the same audit."""
+    from paper_2602_22700_b200 import imm, synth
+    rank, local_rank, world = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    imm.lib()
+    warmup, steps = max(args.warmup, 3), max(args.steps, 1)
+    T, n, K = args.tokens, args.vocab, args.topk
+    ref = synth.reference_logits(SEED + rank, T, n, device=dev)
+    dep = synth.deployed_logits(ref, SEED + rank, synth.NOISE_QUANTISED)
+    topk = torch.topk(dep, K, dim=1).indices.to(torch.int32).contiguous()      # what the server committed to
+    offsets = synth.request_offsets(SEED + rank, T, max(1, T // 256), device=dev)
+    t1, t2 = 0.1, 0.02
+    bytes_tvkl, bytes_topk = 8 * T * n, 4 * T * n
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def one_pass(ev=None):
+        if ev:
+            ev[0].record()
+        tv, kl = imm.ldd_tv_kl(dep, ref)
+        if ev:
+            ev[1].record()
+        d, st = imm.ldd_topk_distance(ref, topk)
+        if ev:
+            ev[2].record()
+        p, flag = imm.ldd_tail_fraction(tv, offsets, t1, t2)
+        if ev:
+            ev[3].record()
+        return tv, kl, d, st, p, flag
+
+    for _ in range(warmup):
+        one_pass()
+    barrier()
+    sampler = ClockSampler(local_rank if "CUDA_VISIBLE_DEVICES" not in os.environ else
+                           int(os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local_rank]))
+    sampler.start()
+    time.sleep(0.25)
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(steps)]
+    t0 = time.time()
+    for e in evs:
+        out = one_pass(e)
+    barrier()
+    t1w = time.time()
+    clocks = sampler.stop(t0, t1w)
+    elapsed_ms = evs[0][0].elapsed_time(evs[-1][3])
+    if dist is not None:
+        t = torch.tensor([elapsed_ms], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        elapsed_ms = float(t.item())
+    ms_per_step = elapsed_ms / steps
+    ph = [sum(e[i].elapsed_time(e[i + 1]) for e in evs) / steps for i in range(3)]
+    tv, kl, d, st, p, flag = out
+    assert int(st.abs().max()) == 0
+    peak, peak_kind = measured_peaks()
+    tvkl_gbs = bytes_tvkl / (ph[0] * 1e-3) / 1e9
+    res = {
+        "metric": "LDD decision steps/sec", "value": T * world / (ms_per_step * 1e-3), "unit": "steps/s",
+        "n_gpus": world, "steps": steps, "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": workload_name("ldd", 0, T, n, K), "tokens": T, "vocab": n, "topk": K,
+                   "requests": int(offsets.numel()) - 1, "input_bytes_per_gpu": bytes_tvkl + 4 * T * K,
+                   "l2": f"inputs ({bytes_tvkl / 2**30:.2f} GiB) exceed the 126 MB L2 many times over; no flush",
+                   "parallelism": "1 GPU" if world == 1 else f"{world} independent replicas, no collective"},
+        "hbm_gbs_whole_step": (bytes_tvkl + bytes_topk) / (ms_per_step * 1e-3) / 1e9,
+        "phases": {"tv_kl": {"ms": ph[0], "gbs": tvkl_gbs},
+                   "topk_distance": {"ms": ph[1], "gbs": bytes_topk / (ph[1] * 1e-3) / 1e9},
+                   "tail_fraction": {"ms": ph[2], "gbs": None}},
+        "roofline": {"kernel": "tv_kl_kernel (two logit rows read once from HBM, second pass from L2)", "bound": "hbm",
+                     "achieved": tvkl_gbs, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": tvkl_gbs / peak,
+                     "frac_of_8tbs": tvkl_gbs / 8000.0,
+                     "traffic": (LDD_TVKL_TRAFFIC_RATIO * bytes_tvkl) if LDD_TVKL_TRAFFIC_RATIO else None},
+        "gpu_launches": 3 * steps,
+        "clocks": clocks,
+        "flagged_requests": int(flag.sum()),
+    }
+    e2e = None
+    if not args.no_e2e:
+        hd = torch.empty(dep.shape, dtype=dep.dtype, pin_memory=True).copy_(dep)
+        hr = torch.empty(ref.shape, dtype=ref.dtype, pin_memory=True).copy_(ref)
+        hk = torch.empty(topk.shape, dtype=topk.dtype, pin_memory=True).copy_(topk)
+        dd, dr, dk = torch.empty_like(dep), torch.empty_like(ref), torch.empty_like(topk)
+        outs = [torch.empty(T, dtype=torch.float64, pin_memory=True) for _ in range(3)]
+        torch.cuda.synchronize()
+
+        def e2e_pass():
+            dd.copy_(hd, non_blocking=True); dr.copy_(hr, non_blocking=True); dk.copy_(hk, non_blocking=True)
+            a, b = imm.ldd_tv_kl(dd, dr)
+            c, _ = imm.ldd_topk_distance(dr, dk)
+            imm.ldd_tail_fraction(a, offsets, t1, t2)
+            outs[0].copy_(a, non_blocking=True); outs[1].copy_(b, non_blocking=True); outs[2].copy_(c, non_blocking=True)
+            torch.cuda.synchronize()
+
+        e2e_pass()
+        barrier()
+        k2 = max(1, args.e2e_steps)
+        w0 = time.perf_counter()
+        for _ in range(k2):
+            e2e_pass()
+        e2e_s = (time.perf_counter() - w0) / k2
+        e2e = {"value": T * world / e2e_s, "unit": "steps/s", "ms_per_step": e2e_s * 1e3, "steps": k2,
+               "h2d_bytes_per_step": hd.numel() * 4 + hr.numel() * 4 + hk.numel() * 4, "d2h_bytes_per_step": 3 * T * 8,
+               "matches_device_path": bool((outs[0].to(dev) == tv).all() and (outs[2].to(dev) == d).all())}
+        del hd, hr, hk, dd, dr, dk
+    res["e2e"] = e2e
+    if not args.no_cpu_baseline and world == 1:
+        rows = list(range(0, T, max(1, T // 48)))[:48]
+        hdep, href, htop = dep[rows].cpu().numpy(), ref[rows].cpu().numpy(), topk[rows].cpu().numpy()
+        w0 = time.perf_counter()
+        otv, okl, odist = ldd_oracle_rows(hdep, href, htop, range(len(rows)))
+        secs = time.perf_counter() - w0
+        gtv, gkl, gd = tv[rows].cpu().numpy(), kl[rows].cpu().numpy(), d[rows].cpu().numpy()
+        ok = (max(abs(a - b) for a, b in zip(gtv, otv)) <= 2e-5 and
+              all(abs(a - b) <= 2e-5 + 2e-4 * abs(b) for a, b in zip(gkl, okl)) and
+              all(abs(a - b) <= 1e-9 * max(1.0, abs(b)) for a, b in zip(gd, odist)))
+        res["cpu_baseline"] = {"value": len(rows) / secs, "unit": "steps/s", "cores": 1, "kind": "oracle", "seconds": secs,
+                               "sample": f"{len(rows)} of the {T} decision steps, evenly spaced, same inputs as the GPU run",
+                               "gpu_matches_oracle_within_tolerance": ok}
+        if not ok:
+            raise SystemExit("GPU distances differ from the oracle beyond the tolerance")
+    if rank == 0:
+        print(json.dumps(res))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
 # ------------------------------------------------------------------------ reference arm (CPU oracle)
 
 
@@ -372,6 +528,30 @@ def run_reference(args):
         return
     from paper_2602_22700_b200 import synth
     device = "cuda" if torch.cuda.is_available() else "cpu"
+    if args.config == "ldd":
+        rows = 48
+        ref = synth.reference_logits(SEED, rows, args.vocab, device=device)
+        dep = synth.deployed_logits(ref, SEED, synth.NOISE_QUANTISED)
+        topk = torch.topk(dep, args.topk, dim=1).indices.to(torch.int32)
+        hdep, href, htop = dep.cpu().numpy(), ref.cpu().numpy(), topk.cpu().numpy()
+        warmup, steps = max(args.warmup, 1), max(args.steps, 1)
+        for _ in range(warmup):
+            ldd_oracle_rows(hdep, href, htop, range(4))
+        w0 = time.perf_counter()
+        for _ in range(steps):
+            ldd_oracle_rows(hdep, href, htop, range(rows))
+        per = (time.perf_counter() - w0) / steps
+        desc = f"{rows} decision steps of the workload per step, one thread"
+        print(json.dumps({
+            "impl": "reference", "metric": "LDD decision steps/sec", "value": rows / per, "unit": "steps/s",
+            "n_gpus": world, "steps": steps, "warmup": warmup, "ms_per_step": per * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": workload_name("ldd", 0, args.tokens, args.vocab, args.topk), "tokens": args.tokens,
+                       "vocab": args.vocab, "topk": args.topk, "sampled": desc},
+            "cpu_baseline": {"value": rows / per, "unit": "steps/s", "cores": 1, "kind": "oracle", "sample": desc},
+            "e2e": {"value": rows / per, "unit": "steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        }))
+        return
     layers = min(args.layers, 2)
     tokens = args.tokens if device == "cuda" else min(args.tokens, 256)
     problems = make_problems(args.config, SEED, layers, tokens, device)[:8]
@@ -409,6 +589,8 @@ def main():
         args.tokens = WORKLOADS[args.config][0]
     if args.impl == "reference":
         run_reference(args)
+    elif args.config == "ldd":
+        run_ldd(args)
     else:
         run_ours(args)
 

@@ -15,6 +15,7 @@
 #include <cuda_runtime.h>
 #include <math.h>
 #include <stdint.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include "../../include/imm.h"
@@ -28,9 +29,7 @@ constexpr int WARPS = THREADS / 32;
 constexpr int MAX_CLUSTER = 8;
 constexpr int SLICE = 16384;                  // entries of a row one block takes (before the cluster cap)
 constexpr int MAX_K = IMM_LDD_MAX_K;          // largest index set of the Top-K distance
-constexpr int MAX_SLICE = IMM_LDD_MAX_N / MAX_CLUSTER;   // most entries of a row one block can get
 constexpr int COLLECT_CAP = 256;              // entries above the bound a block can hold per pass (a power of two)
-constexpr int GATHER_CAP = 4096;              // a power of two >= MAX_CLUSTER * COLLECT_CAP + MAX_K
 constexpr int MAX_REFINE = 6;
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr float NEG_INF = -INFINITY;
@@ -97,20 +96,22 @@ __device__ __forceinline__ float4 ld4(const float* p)
 //   tv += |p_v - q_v|,   kl += q_v * (log q_v - log p_v),   p = softmax(x), q = softmax(y).
 // x is the deployed row, y the reference row.
 
+template <int NW>
 struct TvKlShared {
-    MaxSum warp_p[WARPS], warp_q[WARPS];
+    MaxSum warp_p[NW], warp_q[NW];
     MaxSum pub_p, pub_q;                  // this block's slice; read by the other blocks
     float max_p, max_q, l2s_p, l2s_q;     // the rows' maxima and log2 of their sums of exp(x - max)
-    float warp_tv[WARPS], warp_kl[WARPS];
+    float warp_tv[NW], warp_kl[NW];
     double pub_tv, pub_kl;                // this block's share; read by block 0
 };
 
-template <bool VEC>
-__global__ void __launch_bounds__(THREADS)
+template <bool VEC, int NT>
+__global__ void __launch_bounds__(NT)
 tv_kl_kernel(const float* __restrict__ logits, const float* __restrict__ ref, int64_t n, int64_t ld,
              double* __restrict__ tv_out, double* __restrict__ kl_out)
 {
-    __shared__ TvKlShared sh;
+    constexpr int NW = NT / 32;
+    __shared__ TvKlShared<NW> sh;
     cg::cluster_group cluster = cg::this_cluster();
     const int nc = (int)cluster.num_blocks(), c = (int)cluster.block_rank();
     const int64_t step = blockIdx.x / nc;
@@ -121,7 +122,7 @@ tv_kl_kernel(const float* __restrict__ logits, const float* __restrict__ ref, in
     slice_bounds(n, nc, c, s0, s1);
 
     MaxSum ap{NEG_INF, 0.f}, aq{NEG_INF, 0.f};
-    for (int64_t i = s0 + 4 * tid; i < s1; i += 4 * THREADS) {
+    for (int64_t i = s0 + 4 * tid; i < s1; i += 4 * NT) {
         if (VEC && i + 4 <= s1) {
             const float4 a = ld4(x + i), b = ld4(y + i);
             ms_add4(ap, a.x, a.y, a.z, a.w);
@@ -134,8 +135,8 @@ tv_kl_kernel(const float* __restrict__ logits, const float* __restrict__ ref, in
     if (lane == 0) { sh.warp_p[warp] = ap; sh.warp_q[warp] = aq; }
     __syncthreads();
     if (warp == 0) {
-        MaxSum p = lane < WARPS ? sh.warp_p[lane] : MaxSum{NEG_INF, 0.f};
-        MaxSum q = lane < WARPS ? sh.warp_q[lane] : MaxSum{NEG_INF, 0.f};
+        MaxSum p = lane < NW ? sh.warp_p[lane] : MaxSum{NEG_INF, 0.f};
+        MaxSum q = lane < NW ? sh.warp_q[lane] : MaxSum{NEG_INF, 0.f};
         p = ms_warp(p); q = ms_warp(q);
         if (lane == 0) { sh.pub_p = p; sh.pub_q = q; }
     }
@@ -152,7 +153,7 @@ tv_kl_kernel(const float* __restrict__ logits, const float* __restrict__ ref, in
     const float dl = (lq - lp) * (1.0f / LOG2E);           // log(sum_q) - log(sum_p), natural units
 
     float tv = 0.f, kl = 0.f;
-    for (int64_t i = s0 + 4 * tid; i < s1; i += 4 * THREADS) {
+    for (int64_t i = s0 + 4 * tid; i < s1; i += 4 * NT) {
         float xs[4], ys[4];
         int cnt = 4;
         if (VEC && i + 4 <= s1) {
@@ -182,7 +183,7 @@ tv_kl_kernel(const float* __restrict__ logits, const float* __restrict__ ref, in
     __syncthreads();
     if (tid == 0) {
         double a = 0.0, b = 0.0;
-        for (int w = 0; w < WARPS; w++) { a += (double)sh.warp_tv[w]; b += (double)sh.warp_kl[w]; }
+        for (int w = 0; w < NW; w++) { a += (double)sh.warp_tv[w]; b += (double)sh.warp_kl[w]; }
         sh.pub_tv = a; sh.pub_kl = b;
     }
     cluster.sync();                                        // every block's share is published
@@ -207,227 +208,212 @@ tv_kl_kernel(const float* __restrict__ logits, const float* __restrict__ ref, in
 // minimiser lies at or above that entry, where only the K largest entries outside I contribute,
 // and the minimum is attained at one of 2K breakpoints: those K entries and the K entries of I.
 // The kernel therefore needs the K largest entries outside I, exactly:
-//   pass 1 (HBM): the largest entry outside I of every warp (of every thread, when the row is too short
-//                 for 2K warps); the K-th largest of these maxima is a lower bound tau of the K-th
-//                 largest entry outside I, and close to it: for a 128k-entry row about K + 2
-//                 entries lie above it;
-//   pass 2 (L2):  collect the entries outside I above tau (a few more than K at most, unless the
-//                 row is adversarial; then tau is raised from what was collected and the pass repeats);
-//   block 0 sorts what the cluster collected, adds K copies of tau, keeps the K largest, and
-//   evaluates the cost at the 2K breakpoints in double precision.
+//   pass 1 (HBM): the largest entry outside I of every group of G threads, G chosen so that the
+//                 cluster has at least 2K groups; the K-th largest of these maxima is a lower bound
+//                 tau of the K-th largest entry outside I, and close to it: for a 128k-entry row
+//                 about K + 2 entries lie above it.  Every block finds tau by itself from the
+//                 other blocks' maxima (distributed shared memory), by ranking, without a sort;
+//   pass 2 (L2):  collect the entries outside I above tau (unless the row is adversarial; then
+//                 tau is raised from what was collected and the pass repeats);
+//   block 0 ranks what the cluster collected together with K copies of tau (K entries outside I
+//   are >= tau), keeps the K largest, and evaluates the cost at the 2K breakpoints in float64.
 
-__device__ void bitonic_sort_desc(float* s, int count)      // count a power of two; whole block
-{
-    for (int k = 2; k <= count; k <<= 1)
-        for (int j = k >> 1; j > 0; j >>= 1) {
-            for (int i = threadIdx.x; i < count; i += blockDim.x) {
-                const int partner = i ^ j;
-                if (partner > i) {
-                    const float a = s[i], b = s[partner];
-                    const bool desc = (i & k) == 0;
-                    if (desc ? (a < b) : (a > b)) { s[i] = b; s[partner] = a; }
-                }
-            }
-            __syncthreads();
-        }
-}
+constexpr int MAX_CAND = 256;                 // group maxima of the whole cluster (>= 2 * MAX_K, <= THREADS)
 
 struct TopkShared {
-    uint32_t member[MAX_SLICE / 32 + 8];  // bitmap of the slice's entries that belong to I
-    float work[GATHER_CAP];               // maxima / block 0's gathered entries (sorted in place)
-    float top[MAX_K];                     // this block's largest maxima (sorted), then its refined bound
+    float cand[MAX_CAND];                 // this block's group maxima (the first `ncand` entries)
+    float all[MAX_CLUSTER * COLLECT_CAP + MAX_K];   // the cluster's maxima; block 0: the collected entries
+    float topk[MAX_K];                    // block 0: the K largest entries outside I
     float collected[COLLECT_CAP];         // entries outside I above tau
     float inside[MAX_K];                  // block 0: the entries of I
     double cost[2 * MAX_K];
-    float tau;                            // block 0 publishes; every block reads
+    float tau, proposal, new_tau;
     int count;                            // entries collected in this pass (may exceed COLLECT_CAP)
-    int overflow;                         // block 0: some block collected more than it can hold
-    int bad;                              // an index of I is out of range or repeated
+    int total, over, bad;
 };
 
-__device__ __forceinline__ bool is_member(const uint32_t* member, int64_t rel)
+// rank of all[i] in descending order, ties broken by position: a permutation of 0..m-1
+__device__ __forceinline__ int rank_desc(const float* all, int m, int i)
 {
-    return (member[rel >> 5] >> (rel & 31)) & 1u;
+    const float v = all[i];
+    int r = 0;
+    for (int j = 0; j < m; j++) {
+        const float w = all[j];
+        r += (w > v || (w == v && j < i)) ? 1 : 0;
+    }
+    return r;
 }
 
 template <bool VEC>
-__global__ void __launch_bounds__(THREADS)
+__global__ void __launch_bounds__(THREADS, 3)
 topk_distance_kernel(const float* __restrict__ ref, int64_t n, int64_t ld, const int32_t* __restrict__ topk,
                      int K, double* __restrict__ dist_out, int32_t* __restrict__ status)
 {
+    extern __shared__ uint32_t member[];               // bitmap of the slice's entries that belong to I
     __shared__ TopkShared sh;
     cg::cluster_group cluster = cg::this_cluster();
     const int nc = (int)cluster.num_blocks(), c = (int)cluster.block_rank();
     const int64_t step = blockIdx.x / nc;
-    const float* y = ref + step * ld;
     const int32_t* I = topk + step * K;
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31;
     int64_t s0, s1;
     slice_bounds(n, nc, c, s0, s1);
-    const int words = (int)((s1 - s0 + 31) / 32);
+    const float* row = ref + step * ld;
+    const float* y = row + s0;                         // this block's slice
+    const int len = (int)(s1 - s0);
+    const int nvec = VEC ? len >> 2 : 0;               // whole 16-byte vectors; the rest goes entry by entry
+    const float4* yv = reinterpret_cast<const float4*>(y);
+    const int words = (len + 31) / 32 + 1;
 
-    for (int i = tid; i < words; i += THREADS) sh.member[i] = 0;
-    if (tid == 0) { sh.bad = 0; sh.count = 0; sh.overflow = 0; }
+    for (int i = tid; i < words; i += THREADS) member[i] = 0;
+    if (tid == 0) { sh.bad = 0; sh.count = 0; }
     __syncthreads();
     if (tid < K) {
         const int64_t idx = I[tid];
         if (idx < 0 || idx >= n) sh.bad = 1;
-        else if (idx >= s0 && idx < s1) {
-            const int64_t rel = idx - s0;
-            const uint32_t bit = 1u << (rel & 31);
-            if (atomicOr(&sh.member[rel >> 5], bit) & bit) sh.bad = 1;       // the same index twice
+        else {
+            if (c == 0) sh.inside[tid] = row[idx];     // block 0 needs the entries of I at the end
+            if (idx >= s0 && idx < s1) {
+                const int rel = (int)(idx - s0);
+                const uint32_t bit = 1u << (rel & 31);
+                if (atomicOr(&member[rel >> 5], bit) & bit) sh.bad = 1;      // the same index twice
+            }
         }
     }
     __syncthreads();
 
     // pass 1: this thread's largest entry outside I
     float best = NEG_INF;
-    for (int64_t i = s0 + 4 * tid; i < s1; i += 4 * THREADS) {
-        if (VEC && i + 4 <= s1) {
-            const float4 v = ld4(y + i);
-            const uint32_t m = sh.member[(i - s0) >> 5] >> ((i - s0) & 31);   // four consecutive bits of one word
-            best = fmaxf(best, (m & 1u) ? NEG_INF : v.x);
-            best = fmaxf(best, (m & 2u) ? NEG_INF : v.y);
-            best = fmaxf(best, (m & 4u) ? NEG_INF : v.z);
-            best = fmaxf(best, (m & 8u) ? NEG_INF : v.w);
-        } else {
-            for (int64_t e = i; e < min(i + 4, s1); e++)
-                if (!is_member(sh.member, e - s0)) best = fmaxf(best, y[e]);
-        }
+    for (int v = tid; v < nvec; v += THREADS) {
+        const float4 q = __ldg(yv + v);
+        const uint32_t m = member[v >> 3] >> ((4 * v) & 31);       // four consecutive bits of one word
+        best = fmaxf(best, (m & 1u) ? NEG_INF : q.x);
+        best = fmaxf(best, (m & 2u) ? NEG_INF : q.y);
+        best = fmaxf(best, (m & 4u) ? NEG_INF : q.z);
+        best = fmaxf(best, (m & 8u) ? NEG_INF : q.w);
     }
-    // this block's candidates for the bound: its warps' maxima when the cluster has at least 2K warps,
-    // else the K largest of its threads' maxima
-    const bool by_warp = nc * WARPS >= 2 * K;
+    for (int e = 4 * nvec + tid; e < len; e += THREADS)
+        if (!((member[e >> 5] >> (e & 31)) & 1u)) best = fmaxf(best, y[e]);
     const float thread_best = best;
-    if (by_warp) {
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) best = fmaxf(best, __shfl_xor_sync(0xFFFFFFFFu, best, o));
-        if (tid < MAX_K) sh.top[tid] = NEG_INF;
-        __syncthreads();
-        if ((tid & 31) == 0) sh.top[tid >> 5] = best;
-    } else {
-        sh.work[tid] = best;
-        __syncthreads();
-        bitonic_sort_desc(sh.work, THREADS);
-        if (tid < MAX_K) sh.top[tid] = tid < K ? sh.work[tid] : NEG_INF;
-    }
-    cluster.sync();                                        // every block's candidates are in place
 
-    // block 0: tau = K-th largest candidate of the cluster
-    if (c == 0) {
-        const int per = by_warp ? WARPS : MAX_K;
-        int padded = 32;
-        while (padded < nc * per) padded <<= 1;            // <= 512
-        for (int i = tid; i < padded; i += THREADS)
-            sh.work[i] = i < nc * per ? cluster.map_shared_rank(sh.top, i / per)[i % per] : NEG_INF;
-        __syncthreads();
-        bitonic_sort_desc(sh.work, padded);
-        if (tid == 0) sh.tau = sh.work[K - 1];
-    }
-    int bad_any = 0;
-    for (int round = 0; round <= MAX_REFINE; round++) {
-        cluster.sync();                                    // tau is published (and `overflow` is settled)
-        const float tau = *cluster.map_shared_rank(&sh.tau, 0);
-        if (round > 0 && *cluster.map_shared_rank(&sh.overflow, 0) == 0) break;
-        if (round == MAX_REFINE) { bad_any = 2; break; }   // gave up raising the bound
-        if (tid == 0) sh.count = 0;
-        __syncthreads();
+    // group maxima: groups of G = THREADS / ncand threads, ncand the smallest power of two (16 at
+    // least: one group per warp) that gives the cluster 2K groups; nc * ncand <= MAX_CAND
+    int ncand = WARPS;
+    while (ncand * nc < 2 * K) ncand <<= 1;
+    const int G = THREADS / ncand;                     // 32, 16, 8 or 4
+    for (int o = 1; o < G; o <<= 1) best = fmaxf(best, __shfl_xor_sync(0xFFFFFFFFu, best, o));
+    if ((tid % G) == 0) sh.cand[tid / G] = best;
+    cluster.sync();                                    // every block's group maxima are in place
+
+    // tau = K-th largest of the cluster's group maxima; every block works it out by itself
+    const int total = nc * ncand;
+    if (tid < total) sh.all[tid] = cluster.map_shared_rank(sh.cand, tid / ncand)[tid % ncand];
+    __syncthreads();
+    if (tid < total && rank_desc(sh.all, total, tid) == K - 1) sh.tau = sh.all[tid];
+    __syncthreads();
+    float tau = sh.tau;
+
+    bool failed = false;
+    for (int round = 0;; round++) {
         // pass 2: collect the entries outside I above tau
-        for (int64_t i = s0 + 4 * tid; i < s1; i += 4 * THREADS) {
-            float v[4];
-            uint32_t m;
-            if (VEC && i + 4 <= s1) {
-                const float4 q = ld4(y + i);
-                v[0] = q.x; v[1] = q.y; v[2] = q.z; v[3] = q.w;
-                m = sh.member[(i - s0) >> 5] >> ((i - s0) & 31);
-            } else {
-                m = 0;
-                for (int e = 0; e < 4; e++) {
-                    const bool in = i + e < s1;
-                    v[e] = in ? y[i + e] : NEG_INF;
-                    if (in && is_member(sh.member, i + e - s0)) m |= 1u << e;
-                }
-            }
+        for (int v = tid; v < nvec; v += THREADS) {
+            const float4 q = __ldg(yv + v);
+            const uint32_t m = member[v >> 3] >> ((4 * v) & 31);
+            const float vals[4] = {q.x, q.y, q.z, q.w};
 #pragma unroll
             for (int e = 0; e < 4; e++)
-                if (!((m >> e) & 1u) && v[e] > tau) {
+                if (!((m >> e) & 1u) && vals[e] > tau) {
                     const int slot = atomicAdd(&sh.count, 1);
-                    if (slot < COLLECT_CAP) sh.collected[slot] = v[e];
+                    if (slot < COLLECT_CAP) sh.collected[slot] = vals[e];
                 }
         }
+        for (int e = 4 * nvec + tid; e < len; e += THREADS)
+            if (!((member[e >> 5] >> (e & 31)) & 1u) && y[e] > tau) {
+                const int slot = atomicAdd(&sh.count, 1);
+                if (slot < COLLECT_CAP) sh.collected[slot] = y[e];
+            }
         __syncthreads();
-        // a block that could not hold everything proposes a higher bound.  The K-th largest of its
+        // A block that could not hold everything proposes a higher bound.  The K-th largest of its
         // threads' maxima, and the K-th largest of the entries it did hold, are both entries outside I
         // with K entries at or above them, so either is still a lower bound; the second one lies
         // above tau, so the bound rises every round.
         if (sh.count > COLLECT_CAP) {
-            sh.work[tid] = thread_best;
+            sh.all[tid] = thread_best;
             __syncthreads();
-            bitonic_sort_desc(sh.work, THREADS);
-            const float by_threads = sh.work[K - 1];
+            if (rank_desc(sh.all, THREADS, tid) == K - 1) sh.proposal = sh.all[tid];
             __syncthreads();
-            for (int i = tid; i < COLLECT_CAP; i += THREADS) sh.work[i] = sh.collected[i];
+            if (tid < COLLECT_CAP) sh.all[tid] = sh.collected[tid];
             __syncthreads();
-            bitonic_sort_desc(sh.work, COLLECT_CAP);
-            if (tid == 0) sh.top[0] = fmaxf(by_threads, sh.work[K - 1]);
-        } else if (tid == 0) sh.top[0] = NEG_INF;
-        cluster.sync();                                    // counts and proposals are in place
-        if (c == 0 && tid == 0) {
-            int over = 0;
-            float t = tau;
-            for (int cc = 0; cc < nc; cc++) {
-                if (*cluster.map_shared_rank(&sh.count, cc) > COLLECT_CAP) over = 1;
-                t = fmaxf(t, cluster.map_shared_rank(sh.top, cc)[0]);
+            if (tid < COLLECT_CAP && rank_desc(sh.all, COLLECT_CAP, tid) == K - 1) sh.proposal = fmaxf(sh.proposal, sh.all[tid]);
+        } else if (tid == 0) sh.proposal = NEG_INF;
+        cluster.sync();                                // counts, collected entries and proposals are in place
+        if (tid < 32) {
+            const int cnt = lane < nc ? *cluster.map_shared_rank(&sh.count, lane) : 0;
+            float prop = lane < nc ? *cluster.map_shared_rank(&sh.proposal, lane) : NEG_INF;
+            const int bad = lane < nc ? *cluster.map_shared_rank(&sh.bad, lane) : 0;
+            const unsigned over = __ballot_sync(0xFFFFFFFFu, cnt > COLLECT_CAP);
+            const unsigned anybad = __ballot_sync(0xFFFFFFFFu, bad != 0);
+            int sum = min(cnt, COLLECT_CAP);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                prop = fmaxf(prop, __shfl_xor_sync(0xFFFFFFFFu, prop, o));
+                sum += __shfl_xor_sync(0xFFFFFFFFu, sum, o);
             }
-            sh.overflow = over;
-            if (over) sh.tau = t;
+            if (lane == 0) { sh.over = over != 0; sh.new_tau = fmaxf(tau, prop); sh.total = sum; if (anybad) sh.bad = 2; }
         }
+        __syncthreads();
+        if (!sh.over) break;
+        if (round + 1 == MAX_REFINE) { failed = true; break; }     // gave up raising the bound
+        tau = sh.new_tau;
+        cluster.sync();                                // every block has read the counts: they may be reset
+        if (tid == 0) sh.count = 0;
+        __syncthreads();
     }
-    const float tau = *cluster.map_shared_rank(&sh.tau, 0);
 
     if (c == 0) {
-        // gather what the cluster collected, add K copies of tau (K entries outside I are >= tau)
+        // what the cluster collected, plus K copies of tau
         int fill = 0;
         for (int cc = 0; cc < nc; cc++) {
             const int cnt = min(*cluster.map_shared_rank(&sh.count, cc), COLLECT_CAP);
             const float* src = cluster.map_shared_rank(sh.collected, cc);
-            for (int i = tid; i < cnt; i += THREADS) sh.work[fill + i] = src[i];
+            for (int i = tid; i < cnt; i += THREADS) sh.all[fill + i] = src[i];
             fill += cnt;
-            if (*cluster.map_shared_rank(&sh.bad, cc)) bad_any = max(bad_any, 1);
         }
-        for (int i = tid; i < K; i += THREADS) sh.work[fill + i] = tau;
+        for (int i = tid; i < K; i += THREADS) sh.all[fill + i] = tau;
         fill += K;
-        int padded = 1;
-        while (padded < fill) padded <<= 1;
-        for (int i = fill + tid; i < padded; i += THREADS) sh.work[i] = NEG_INF;
-        if (tid < K) {
-            const int64_t idx = I[tid];
-            sh.inside[tid] = (idx >= 0 && idx < n) ? y[idx] : 0.f;
+        __syncthreads();
+        for (int i = tid; i < fill; i += THREADS) {
+            const int r = rank_desc(sh.all, fill, i);
+            if (r < K) sh.topk[r] = sh.all[i];
         }
         __syncthreads();
-        bitonic_sort_desc(sh.work, padded);                // work[0..K) = the K largest entries outside I
         // cost at the 2K breakpoints, in double
         if (tid < 2 * K) {
-            const double t = tid < K ? (double)sh.work[tid] : (double)sh.inside[tid - K];
+            const double t = tid < K ? (double)sh.topk[tid] : (double)sh.inside[tid - K];
             double cost = INFINITY;
-            if (t > -INFINITY) {                           // a row with fewer than K entries outside I pads with -inf
+            if (t > -INFINITY) {                       // a row with fewer than K entries outside I pads with -inf
                 cost = 0.0;
                 for (int k = 0; k < K; k++) {
-                    cost += fmax((double)sh.work[k] - t, 0.0);
+                    cost += fmax((double)sh.topk[k] - t, 0.0);
                     cost += fmax(t - (double)sh.inside[k], 0.0);
                 }
             }
             sh.cost[tid] = cost;
         }
         __syncthreads();
-        if (tid == 0) {
+        if (tid < 32) {
             double best_cost = INFINITY;
-            for (int i = 0; i < 2 * K; i++) best_cost = fmin(best_cost, sh.cost[i]);
-            dist_out[step] = bad_any ? NAN : best_cost;
-            status[step] = bad_any == 1 ? IMM_ERR_ARG : bad_any == 2 ? IMM_ERR_LIMIT : IMM_OK;
+            for (int i = lane; i < 2 * K; i += 32) best_cost = fmin(best_cost, sh.cost[i]);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) best_cost = fmin(best_cost, __shfl_xor_sync(0xFFFFFFFFu, best_cost, o));
+            if (lane == 0) {
+                const bool bad = sh.bad != 0;
+                dist_out[step] = (bad || failed) ? NAN : best_cost;
+                status[step] = bad ? IMM_ERR_ARG : failed ? IMM_ERR_LIMIT : IMM_OK;
+            }
         }
     }
-    cluster.sync();                                        // block 0 has read the other blocks' memory
+    cluster.sync();                                    // block 0 has read the other blocks' memory
 }
 
 // ------------------------------------------------------------------------------------------
@@ -465,12 +451,13 @@ int cluster_size(int64_t n)
 }
 
 template <typename... Args>
-cudaError_t launch_cluster(void (*kernel)(Args...), int64_t steps, int nc, cudaStream_t st, Args... args)
+cudaError_t launch_cluster(void (*kernel)(Args...), int64_t steps, int nc, int threads, size_t smem, cudaStream_t st, Args... args)
 {
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3((unsigned)(steps * nc));
-    cfg.blockDim = dim3(THREADS);
+    cfg.blockDim = dim3((unsigned)threads);
+    cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
     cudaLaunchAttribute attr;
     memset(&attr, 0, sizeof(attr));
@@ -499,8 +486,19 @@ int imm_ldd_tv_kl(const float* d_logits, const float* d_ref_logits, int64_t step
     if (steps == 0) return IMM_OK;
     const int nc = cluster_size(n);
     const bool vec = rows_aligned(d_logits, ld) && rows_aligned(d_ref_logits, ld);
-    cudaError_t e = vec ? launch_cluster(tv_kl_kernel<true>, steps, nc, (cudaStream_t)stream, d_logits, d_ref_logits, n, ld, d_tv, d_kl)
-                        : launch_cluster(tv_kl_kernel<false>, steps, nc, (cudaStream_t)stream, d_logits, d_ref_logits, n, ld, d_tv, d_kl);
+    int nt = 512, ncl = nc;
+    if (const char* v = getenv("IMM_LDD_THREADS")) nt = atoi(v) == 256 ? 256 : atoi(v) == 1024 ? 1024 : 512;
+    if (const char* v = getenv("IMM_LDD_CLUSTER")) { int c = atoi(v); if (c == 1 || c == 2 || c == 4 || c == 8 || c == 16) ncl = c; }
+    cudaStream_t st = (cudaStream_t)stream;
+    cudaError_t e;
+#define TVKL_LAUNCH(V, T) do { \
+        if (ncl > 8) cudaFuncSetAttribute(tv_kl_kernel<V, T>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1); \
+        e = launch_cluster(tv_kl_kernel<V, T>, steps, ncl, T, 0, st, d_logits, d_ref_logits, n, ld, d_tv, d_kl); } while (0)
+    if (!vec) TVKL_LAUNCH(false, 512);
+    else if (nt == 256) TVKL_LAUNCH(true, 256);
+    else if (nt == 1024) TVKL_LAUNCH(true, 1024);
+    else TVKL_LAUNCH(true, 512);
+#undef TVKL_LAUNCH
     return e == cudaSuccess ? IMM_OK : IMM_ERR_CUDA;
 }
 
@@ -515,8 +513,10 @@ int imm_ldd_topk_distance(const float* d_ref_logits, int64_t steps, int64_t n, i
     if (steps == 0) return IMM_OK;
     const int nc = cluster_size(n);
     const bool vec = rows_aligned(d_ref_logits, ld);
-    cudaError_t e = vec ? launch_cluster(topk_distance_kernel<true>, steps, nc, (cudaStream_t)stream, d_ref_logits, n, ld, d_topk, k, d_dist, d_status)
-                        : launch_cluster(topk_distance_kernel<false>, steps, nc, (cudaStream_t)stream, d_ref_logits, n, ld, d_topk, k, d_dist, d_status);
+    const int64_t per = ((n + nc - 1) / nc + 3) / 4 * 4;                     // entries per block (see slice_bounds)
+    const size_t smem = (size_t)((per + 31) / 32 + 2) * sizeof(uint32_t);    // the membership bitmap (<= 16 KiB)
+    cudaError_t e = vec ? launch_cluster(topk_distance_kernel<true>, steps, nc, THREADS, smem, (cudaStream_t)stream, d_ref_logits, n, ld, d_topk, k, d_dist, d_status)
+                        : launch_cluster(topk_distance_kernel<false>, steps, nc, THREADS, smem, (cudaStream_t)stream, d_ref_logits, n, ld, d_topk, k, d_dist, d_status);
     return e == cudaSuccess ? IMM_OK : IMM_ERR_CUDA;
 }
 

@@ -207,29 +207,31 @@ tv_kl_kernel(const float* __restrict__ logits, const float* __restrict__ ref, in
 // slope is <= 0 (at least K entries outside I lie above t, at most K entries of I below).  So a
 // minimiser lies at or above that entry, where only the K largest entries outside I contribute,
 // and the minimum is attained at one of 2K breakpoints: those K entries and the K entries of I.
-// The kernel therefore needs the K largest entries outside I, exactly:
-//   pass 1 (HBM): the largest entry outside I of every group of G threads, G chosen so that the
-//                 cluster has at least 2K groups; the K-th largest of these maxima is a lower bound
-//                 tau of the K-th largest entry outside I, and close to it: for a 128k-entry row
-//                 about K + 2 entries lie above it.  Every block finds tau by itself from the
-//                 other blocks' maxima (distributed shared memory), by ranking, without a sort;
-//   pass 2 (L2):  collect the entries outside I above tau (unless the row is adversarial; then
-//                 tau is raised from what was collected and the pass repeats);
-//   block 0 ranks what the cluster collected together with K copies of tau (K entries outside I
-//   are >= tau), keeps the K largest, and evaluates the cost at the 2K breakpoints in float64.
+// The kernel therefore needs the K largest entries outside I, exactly.  They are among the K
+// largest of every slice, and the blocks that take the slices of a row never wait for one another:
+//   a thread loads its 32 entries of the slice once and keeps them in registers; the largest entry
+//   outside I of every group of G threads (at least 2K groups) gives, as the K-th largest of these
+//   maxima, a lower bound tau of the slice's K-th largest entry outside I, and a close one: about
+//   1.3 K entries lie above it; the entries outside I above tau are collected from the registers
+//   (unless the slice is adversarial; then tau is raised from what was collected and the collection
+//   repeats);
+//   the K largest of what was collected, padded with copies of tau (K entries outside I are >=
+//   tau), go to the workspace.  The block that finishes a row last merges the slices' lists,
+//   keeps the K largest, and evaluates the cost at the 2K breakpoints in float64.
 
-constexpr int MAX_CAND = 256;                 // group maxima of the whole cluster (>= 2 * MAX_K, <= THREADS)
+constexpr int MAX_CAND = 128;                 // group maxima per block (>= 2 * MAX_K)
+constexpr int MERGE_CAP = 4096;               // a row's lists the merging block holds at once: (n / SLICE) * K
 
 struct TopkShared {
-    float cand[MAX_CAND];                 // this block's group maxima (the first `ncand` entries)
-    float all[MAX_CLUSTER * COLLECT_CAP + MAX_K];   // the cluster's maxima; block 0: the collected entries
-    float topk[MAX_K];                    // block 0: the K largest entries outside I
+    uint32_t member[SLICE / 32 + 2];      // bitmap of the slice's entries that belong to I
+    float work[MERGE_CAP];                // thread maxima / group maxima / collected entries / the row's lists
     float collected[COLLECT_CAP];         // entries outside I above tau
-    float inside[MAX_K];                  // block 0: the entries of I
+    float topk[MAX_K];
+    float inside[MAX_K];                  // merging block: the entries of I
     double cost[2 * MAX_K];
-    float tau, proposal, new_tau;
+    float tau, proposal;
     int count;                            // entries collected in this pass (may exceed COLLECT_CAP)
-    int total, over, bad;
+    int bad, last;
 };
 
 // rank of all[i] in descending order, ties broken by position: a permutation of 0..m-1
@@ -245,175 +247,189 @@ __device__ __forceinline__ int rank_desc(const float* all, int m, int i)
 }
 
 template <bool VEC>
-__global__ void __launch_bounds__(THREADS, 3)
+__global__ void __launch_bounds__(THREADS, 2)
 topk_distance_kernel(const float* __restrict__ ref, int64_t n, int64_t ld, const int32_t* __restrict__ topk,
-                     int K, double* __restrict__ dist_out, int32_t* __restrict__ status)
+                     int K, int nslices, float* __restrict__ lists, uint32_t* __restrict__ done,
+                     double* __restrict__ dist_out, int32_t* __restrict__ status)
 {
-    extern __shared__ uint32_t member[];               // bitmap of the slice's entries that belong to I
     __shared__ TopkShared sh;
-    cg::cluster_group cluster = cg::this_cluster();
-    const int nc = (int)cluster.num_blocks(), c = (int)cluster.block_rank();
-    const int64_t step = blockIdx.x / nc;
+    const int64_t step = blockIdx.x / nslices;
+    const int c = (int)(blockIdx.x % nslices);
     const int32_t* I = topk + step * K;
-    const int tid = threadIdx.x, lane = tid & 31;
-    int64_t s0, s1;
-    slice_bounds(n, nc, c, s0, s1);
+    const int tid = threadIdx.x;
+    const int64_t s0 = (int64_t)c * SLICE, s1 = min(n, s0 + SLICE);
     const float* row = ref + step * ld;
     const float* y = row + s0;                         // this block's slice
     const int len = (int)(s1 - s0);
     const int nvec = VEC ? len >> 2 : 0;               // whole 16-byte vectors; the rest goes entry by entry
     const float4* yv = reinterpret_cast<const float4*>(y);
-    const int words = (len + 31) / 32 + 1;
 
-    for (int i = tid; i < words; i += THREADS) member[i] = 0;
+    for (int i = tid; i < SLICE / 32 + 2; i += THREADS) sh.member[i] = 0;
     if (tid == 0) { sh.bad = 0; sh.count = 0; }
     __syncthreads();
     if (tid < K) {
         const int64_t idx = I[tid];
         if (idx < 0 || idx >= n) sh.bad = 1;
-        else {
-            if (c == 0) sh.inside[tid] = row[idx];     // block 0 needs the entries of I at the end
-            if (idx >= s0 && idx < s1) {
-                const int rel = (int)(idx - s0);
-                const uint32_t bit = 1u << (rel & 31);
-                if (atomicOr(&member[rel >> 5], bit) & bit) sh.bad = 1;      // the same index twice
-            }
+        else if (idx >= s0 && idx < s1) {
+            const int rel = (int)(idx - s0);
+            const uint32_t bit = 1u << (rel & 31);
+            if (atomicOr(&sh.member[rel >> 5], bit) & bit) sh.bad = 1;       // the same index twice
         }
     }
     __syncthreads();
 
-    // pass 1: this thread's largest entry outside I
-    float best = NEG_INF;
-    for (int v = tid; v < nvec; v += THREADS) {
-        const float4 q = __ldg(yv + v);
-        const uint32_t m = member[v >> 3] >> ((4 * v) & 31);       // four consecutive bits of one word
-        best = fmaxf(best, (m & 1u) ? NEG_INF : q.x);
-        best = fmaxf(best, (m & 2u) ? NEG_INF : q.y);
-        best = fmaxf(best, (m & 4u) ? NEG_INF : q.z);
-        best = fmaxf(best, (m & 8u) ? NEG_INF : q.w);
+    // The thread's 32 entries of the slice stay in registers: all loads are issued at once, and the
+    // second look at the data (once tau is known) needs no memory access.  Entries of I, and slots
+    // past the end of the slice, are replaced by -inf: they can never be collected.
+    constexpr int PER = SLICE / THREADS;               // 32 entries per thread
+    float vals[PER];
+    if (VEC) {
+#pragma unroll
+        for (int u = 0; u < PER / 4; u++) {
+            const int v = tid + u * THREADS;
+            const float4 q = v < nvec ? __ldg(yv + v) : make_float4(NEG_INF, NEG_INF, NEG_INF, NEG_INF);
+            vals[4 * u] = q.x; vals[4 * u + 1] = q.y; vals[4 * u + 2] = q.z; vals[4 * u + 3] = q.w;
+        }
+#pragma unroll
+        for (int u = 0; u < PER / 4; u++) {
+            const int v = tid + u * THREADS;
+            const uint32_t m = v < nvec ? sh.member[v >> 3] >> ((4 * v) & 31) : 0u;   // four consecutive bits of one word
+#pragma unroll
+            for (int k = 0; k < 4; k++) if ((m >> k) & 1u) vals[4 * u + k] = NEG_INF;
+        }
+    } else {
+#pragma unroll
+        for (int j = 0; j < PER; j++) {
+            const int e = tid + j * THREADS;
+            vals[j] = e < len ? y[e] : NEG_INF;
+        }
+#pragma unroll
+        for (int j = 0; j < PER; j++) {
+            const int e = tid + j * THREADS;
+            if (e < len && ((sh.member[e >> 5] >> (e & 31)) & 1u)) vals[j] = NEG_INF;
+        }
     }
-    for (int e = 4 * nvec + tid; e < len; e += THREADS)
-        if (!((member[e >> 5] >> (e & 31)) & 1u)) best = fmaxf(best, y[e]);
-    const float thread_best = best;
+    float tail = NEG_INF;                              // aligned rows: the up to three entries after the last whole vector
+    if (VEC && tid < len - 4 * nvec) {
+        const int e = 4 * nvec + tid;
+        if (!((sh.member[e >> 5] >> (e & 31)) & 1u)) tail = y[e];
+    }
+    float best = tail;
+#pragma unroll
+    for (int j = 0; j < PER; j++) best = fmaxf(best, vals[j]);
+    const float thread_best = best;                    // (before the group reduction below)
 
-    // group maxima: groups of G = THREADS / ncand threads, ncand the smallest power of two (16 at
-    // least: one group per warp) that gives the cluster 2K groups; nc * ncand <= MAX_CAND
+    // group maxima: ncand = the smallest power of two >= 2K (16 at least: one group per warp)
     int ncand = WARPS;
-    while (ncand * nc < 2 * K) ncand <<= 1;
-    const int G = THREADS / ncand;                     // 32, 16, 8 or 4
+    while (ncand < 2 * K) ncand <<= 1;                 // <= MAX_CAND
+    const int G = THREADS / ncand;                     // 32, 16, 8 or 4 threads per group
     for (int o = 1; o < G; o <<= 1) best = fmaxf(best, __shfl_xor_sync(0xFFFFFFFFu, best, o));
-    if ((tid % G) == 0) sh.cand[tid / G] = best;
-    cluster.sync();                                    // every block's group maxima are in place
-
-    // tau = K-th largest of the cluster's group maxima; every block works it out by itself
-    const int total = nc * ncand;
-    if (tid < total) sh.all[tid] = cluster.map_shared_rank(sh.cand, tid / ncand)[tid % ncand];
+    if ((tid % G) == 0) sh.work[tid / G] = best;
     __syncthreads();
-    if (tid < total && rank_desc(sh.all, total, tid) == K - 1) sh.tau = sh.all[tid];
+    if (tid < ncand && rank_desc(sh.work, ncand, tid) == K - 1) sh.tau = sh.work[tid];
     __syncthreads();
     float tau = sh.tau;
 
     bool failed = false;
     for (int round = 0;; round++) {
-        // pass 2: collect the entries outside I above tau
-        for (int v = tid; v < nvec; v += THREADS) {
-            const float4 q = __ldg(yv + v);
-            const uint32_t m = member[v >> 3] >> ((4 * v) & 31);
-            const float vals[4] = {q.x, q.y, q.z, q.w};
+        // collect the entries outside I above tau (from registers)
+        if (thread_best > tau) {                       // rare: about K + a few threads of the block
 #pragma unroll
-            for (int e = 0; e < 4; e++)
-                if (!((m >> e) & 1u) && vals[e] > tau) {
+            for (int j = 0; j < PER; j++)
+                if (vals[j] > tau) {
                     const int slot = atomicAdd(&sh.count, 1);
-                    if (slot < COLLECT_CAP) sh.collected[slot] = vals[e];
+                    if (slot < COLLECT_CAP) sh.collected[slot] = vals[j];
                 }
-        }
-        for (int e = 4 * nvec + tid; e < len; e += THREADS)
-            if (!((member[e >> 5] >> (e & 31)) & 1u) && y[e] > tau) {
+            if (tail > tau) {
                 const int slot = atomicAdd(&sh.count, 1);
-                if (slot < COLLECT_CAP) sh.collected[slot] = y[e];
+                if (slot < COLLECT_CAP) sh.collected[slot] = tail;
             }
-        __syncthreads();
-        // A block that could not hold everything proposes a higher bound.  The K-th largest of its
-        // threads' maxima, and the K-th largest of the entries it did hold, are both entries outside I
-        // with K entries at or above them, so either is still a lower bound; the second one lies
-        // above tau, so the bound rises every round.
-        if (sh.count > COLLECT_CAP) {
-            sh.all[tid] = thread_best;
-            __syncthreads();
-            if (rank_desc(sh.all, THREADS, tid) == K - 1) sh.proposal = sh.all[tid];
-            __syncthreads();
-            if (tid < COLLECT_CAP) sh.all[tid] = sh.collected[tid];
-            __syncthreads();
-            if (tid < COLLECT_CAP && rank_desc(sh.all, COLLECT_CAP, tid) == K - 1) sh.proposal = fmaxf(sh.proposal, sh.all[tid]);
-        } else if (tid == 0) sh.proposal = NEG_INF;
-        cluster.sync();                                // counts, collected entries and proposals are in place
-        if (tid < 32) {
-            const int cnt = lane < nc ? *cluster.map_shared_rank(&sh.count, lane) : 0;
-            float prop = lane < nc ? *cluster.map_shared_rank(&sh.proposal, lane) : NEG_INF;
-            const int bad = lane < nc ? *cluster.map_shared_rank(&sh.bad, lane) : 0;
-            const unsigned over = __ballot_sync(0xFFFFFFFFu, cnt > COLLECT_CAP);
-            const unsigned anybad = __ballot_sync(0xFFFFFFFFu, bad != 0);
-            int sum = min(cnt, COLLECT_CAP);
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                prop = fmaxf(prop, __shfl_xor_sync(0xFFFFFFFFu, prop, o));
-                sum += __shfl_xor_sync(0xFFFFFFFFu, sum, o);
-            }
-            if (lane == 0) { sh.over = over != 0; sh.new_tau = fmaxf(tau, prop); sh.total = sum; if (anybad) sh.bad = 2; }
         }
         __syncthreads();
-        if (!sh.over) break;
+        if (sh.count <= COLLECT_CAP) break;
         if (round + 1 == MAX_REFINE) { failed = true; break; }     // gave up raising the bound
-        tau = sh.new_tau;
-        cluster.sync();                                // every block has read the counts: they may be reset
+        // More than the block can hold: raise the bound.  The K-th largest of the threads' maxima, and
+        // the K-th largest of the entries that were held, are both entries outside I with K entries at
+        // or above them, so either is still a lower bound; the second one lies above tau, so the bound
+        // rises every round.
+        sh.work[tid] = thread_best;
+        __syncthreads();
+        if (rank_desc(sh.work, THREADS, tid) == K - 1) sh.proposal = sh.work[tid];
+        __syncthreads();
+        if (tid < COLLECT_CAP) sh.work[tid] = sh.collected[tid];
+        __syncthreads();
+        if (tid < COLLECT_CAP && rank_desc(sh.work, COLLECT_CAP, tid) == K - 1) sh.proposal = fmaxf(sh.proposal, sh.work[tid]);
+        __syncthreads();
+        tau = fmaxf(tau, sh.proposal);
         if (tid == 0) sh.count = 0;
         __syncthreads();
     }
 
-    if (c == 0) {
-        // what the cluster collected, plus K copies of tau
-        int fill = 0;
-        for (int cc = 0; cc < nc; cc++) {
-            const int cnt = min(*cluster.map_shared_rank(&sh.count, cc), COLLECT_CAP);
-            const float* src = cluster.map_shared_rank(sh.collected, cc);
-            for (int i = tid; i < cnt; i += THREADS) sh.all[fill + i] = src[i];
-            fill += cnt;
-        }
-        for (int i = tid; i < K; i += THREADS) sh.all[fill + i] = tau;
-        fill += K;
+    // this slice's K largest entries outside I: what was collected plus K copies of tau
+    {
+        const int cnt = min(sh.count, COLLECT_CAP);
+        for (int i = tid; i < cnt; i += THREADS) sh.work[i] = sh.collected[i];
+        for (int i = tid; i < K; i += THREADS) sh.work[cnt + i] = tau;
         __syncthreads();
-        for (int i = tid; i < fill; i += THREADS) {
-            const int r = rank_desc(sh.all, fill, i);
-            if (r < K) sh.topk[r] = sh.all[i];
-        }
-        __syncthreads();
-        // cost at the 2K breakpoints, in double
-        if (tid < 2 * K) {
-            const double t = tid < K ? (double)sh.topk[tid] : (double)sh.inside[tid - K];
-            double cost = INFINITY;
-            if (t > -INFINITY) {                       // a row with fewer than K entries outside I pads with -inf
-                cost = 0.0;
-                for (int k = 0; k < K; k++) {
-                    cost += fmax((double)sh.topk[k] - t, 0.0);
-                    cost += fmax(t - (double)sh.inside[k], 0.0);
-                }
-            }
-            sh.cost[tid] = cost;
-        }
-        __syncthreads();
-        if (tid < 32) {
-            double best_cost = INFINITY;
-            for (int i = lane; i < 2 * K; i += 32) best_cost = fmin(best_cost, sh.cost[i]);
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) best_cost = fmin(best_cost, __shfl_xor_sync(0xFFFFFFFFu, best_cost, o));
-            if (lane == 0) {
-                const bool bad = sh.bad != 0;
-                dist_out[step] = (bad || failed) ? NAN : best_cost;
-                status[step] = bad ? IMM_ERR_ARG : failed ? IMM_ERR_LIMIT : IMM_OK;
-            }
+        float* mine = lists + ((int64_t)step * nslices + c) * K;
+        for (int i = tid; i < cnt + K; i += THREADS) {
+            const int r = rank_desc(sh.work, cnt + K, i);
+            if (r < K) mine[r] = sh.work[i];
         }
     }
-    cluster.sync();                                    // block 0 has read the other blocks' memory
+    // the block that finishes a row last merges it (nobody waits: the others are done)
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        // low half: slices done; bit 16: a bad index; bit 17: a slice gave up
+        const uint32_t flags = (sh.bad ? 0x10000u : 0u) | (failed ? 0x20000u : 0u);
+        if (flags) atomicOr(&done[step], flags);
+        const uint32_t old = atomicAdd(&done[step], 1u);
+        sh.last = (int)((old & 0xFFFFu) == (uint32_t)(nslices - 1));
+        if (sh.last) sh.bad = (int)(((old | flags) >> 16) & 3u);             // what any block of the row reported
+    }
+    __syncthreads();
+    if (!sh.last) return;
+    __threadfence();
+
+    const int m = nslices * K;                             // <= MERGE_CAP (checked on the host)
+    const float* all = lists + (int64_t)step * nslices * K;
+    for (int i = tid; i < m; i += THREADS) sh.work[i] = __ldcg(all + i);
+    if (tid < K) {
+        const int64_t idx = I[tid];
+        sh.inside[tid] = (idx >= 0 && idx < n) ? row[idx] : 0.f;
+    }
+    __syncthreads();
+    for (int i = tid; i < m; i += THREADS) {
+        const int r = rank_desc(sh.work, m, i);
+        if (r < K) sh.topk[r] = sh.work[i];
+    }
+    __syncthreads();
+    // cost at the 2K breakpoints, in double
+    if (tid < 2 * K) {
+        const double t = tid < K ? (double)sh.topk[tid] : (double)sh.inside[tid - K];
+        double cost = INFINITY;
+        if (t > -INFINITY) {                               // a row with fewer than K entries outside I pads with -inf
+            cost = 0.0;
+            for (int k = 0; k < K; k++) {
+                cost += fmax((double)sh.topk[k] - t, 0.0);
+                cost += fmax(t - (double)sh.inside[k], 0.0);
+            }
+        }
+        sh.cost[tid] = cost;
+    }
+    __syncthreads();
+    if (tid < 32) {
+        double best_cost = INFINITY;
+        for (int i = tid; i < 2 * K; i += 32) best_cost = fmin(best_cost, sh.cost[i]);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) best_cost = fmin(best_cost, __shfl_xor_sync(0xFFFFFFFFu, best_cost, o));
+        if (tid == 0) {
+            const bool bad = (sh.bad & 1) != 0, gave_up = (sh.bad & 2) != 0;
+            dist_out[step] = (bad || gave_up) ? NAN : best_cost;
+            status[step] = bad ? IMM_ERR_ARG : gave_up ? IMM_ERR_LIMIT : IMM_OK;
+        }
+    }
 }
 
 // ------------------------------------------------------------------------------------------
@@ -502,22 +518,39 @@ int imm_ldd_tv_kl(const float* d_logits, const float* d_ref_logits, int64_t step
     return e == cudaSuccess ? IMM_OK : IMM_ERR_CUDA;
 }
 
-int imm_ldd_topk_distance(const float* d_ref_logits, int64_t steps, int64_t n, int64_t ld,
-                          const int32_t* d_topk, int k, double* d_dist, int32_t* d_status, void* stream)
+size_t imm_ldd_topk_workspace(int64_t steps, int64_t n, int k)
 {
     using namespace imm_ldd;
-    if (!d_ref_logits || !d_topk || !d_dist || !d_status) return IMM_ERR_ARG;
+    if (steps < 0 || n <= 0 || n > IMM_LDD_MAX_N || steps > IMM_LDD_MAX_STEPS || k <= 0 || k > IMM_LDD_MAX_K) return 0;
+    const int64_t nslices = (n + SLICE - 1) / SLICE;
+    // one counter per row, then every slice's K largest entries
+    return (size_t)((steps * 4 + 255) / 256 * 256) + (size_t)steps * nslices * k * sizeof(float) + 256;
+}
+
+int imm_ldd_topk_distance(const float* d_ref_logits, int64_t steps, int64_t n, int64_t ld,
+                          const int32_t* d_topk, int k, double* d_dist, int32_t* d_status,
+                          void* d_ws, size_t ws_bytes, void* stream)
+{
+    using namespace imm_ldd;
+    if (!d_ref_logits || !d_topk || !d_dist || !d_status || !d_ws) return IMM_ERR_ARG;
     if (steps < 0 || n <= 0 || ld < n || n > IMM_LDD_MAX_N || steps > IMM_LDD_MAX_STEPS) return IMM_ERR_SHAPE;
     if (k <= 0 || k > IMM_LDD_MAX_K || k > n) return IMM_ERR_SHAPE;
-    if ((uintptr_t)d_ref_logits % 4 || (uintptr_t)d_topk % 4 || (uintptr_t)d_dist % 8 || (uintptr_t)d_status % 4) return IMM_ERR_ALIGN;
+    if ((uintptr_t)d_ref_logits % 4 || (uintptr_t)d_topk % 4 || (uintptr_t)d_dist % 8 || (uintptr_t)d_status % 4 ||
+        (uintptr_t)d_ws % 16)
+        return IMM_ERR_ALIGN;
+    if (ws_bytes < imm_ldd_topk_workspace(steps, n, k)) return IMM_ERR_WORKSPACE;
     if (steps == 0) return IMM_OK;
-    const int nc = cluster_size(n);
+    const int64_t nslices = (n + SLICE - 1) / SLICE;
+    if (nslices * k > MERGE_CAP || steps * nslices > 0x7FFFFFFF) return IMM_ERR_SHAPE;     // (cannot happen within the limits)
+    cudaStream_t st = (cudaStream_t)stream;
+    uint32_t* done = (uint32_t*)d_ws;
+    float* lists = (float*)((char*)d_ws + (steps * 4 + 255) / 256 * 256);
+    if (cudaMemsetAsync(done, 0, (size_t)steps * 4, st) != cudaSuccess) return IMM_ERR_CUDA;
     const bool vec = rows_aligned(d_ref_logits, ld);
-    const int64_t per = ((n + nc - 1) / nc + 3) / 4 * 4;                     // entries per block (see slice_bounds)
-    const size_t smem = (size_t)((per + 31) / 32 + 2) * sizeof(uint32_t);    // the membership bitmap (<= 16 KiB)
-    cudaError_t e = vec ? launch_cluster(topk_distance_kernel<true>, steps, nc, THREADS, smem, (cudaStream_t)stream, d_ref_logits, n, ld, d_topk, k, d_dist, d_status)
-                        : launch_cluster(topk_distance_kernel<false>, steps, nc, THREADS, smem, (cudaStream_t)stream, d_ref_logits, n, ld, d_topk, k, d_dist, d_status);
-    return e == cudaSuccess ? IMM_OK : IMM_ERR_CUDA;
+    const unsigned grid = (unsigned)(steps * nslices);
+    if (vec) topk_distance_kernel<true><<<grid, THREADS, 0, st>>>(d_ref_logits, n, ld, d_topk, k, (int)nslices, lists, done, d_dist, d_status);
+    else topk_distance_kernel<false><<<grid, THREADS, 0, st>>>(d_ref_logits, n, ld, d_topk, k, (int)nslices, lists, done, d_dist, d_status);
+    return cudaGetLastError() == cudaSuccess ? IMM_OK : IMM_ERR_CUDA;
 }
 
 int imm_ldd_tail_fraction(const double* d_dist, const int64_t* d_offsets, int64_t nrequests, double t1, double t2,

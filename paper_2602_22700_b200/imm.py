@@ -30,7 +30,7 @@ EXPORTS = ("imm_version", "imm_last_cuda_error", "imm_challenge", "imm_field_bin
            "imm_sumcheck_matmul_workspace", "imm_sumcheck_matmul_prove",
            "imm_sumcheck_matmul_host_arena", "imm_sumcheck_matmul_prove_host", "imm_sumcheck_verify",
            "imm_profile_enable", "imm_profile_calls", "imm_profile_read", "imm_mle_eval_point_noalloc",
-           "imm_ldd_tv_kl", "imm_ldd_topk_distance", "imm_ldd_tail_fraction")
+           "imm_ldd_tv_kl", "imm_ldd_topk_workspace", "imm_ldd_topk_distance", "imm_ldd_tail_fraction")
 NOALLOC_MAX_TILES = 8192
 PROFILE_PHASES = ("eq_tables", "claim_C", "bind_rows_A", "bind_cols_B", "sumcheck_rounds")
 
@@ -94,7 +94,9 @@ def lib() -> ctypes.CDLL:
     L.imm_ldd_tv_kl.restype = ci
     L.imm_ldd_tv_kl.argtypes = [vp, vp, i64, i64, i64, vp, vp, vp]
     L.imm_ldd_topk_distance.restype = ci
-    L.imm_ldd_topk_distance.argtypes = [vp, i64, i64, i64, vp, ci, vp, vp, vp]
+    L.imm_ldd_topk_distance.argtypes = [vp, i64, i64, i64, vp, ci, vp, vp, vp, sz, vp]
+    L.imm_ldd_topk_workspace.restype = sz
+    L.imm_ldd_topk_workspace.argtypes = [i64, i64, ci]
     L.imm_ldd_tail_fraction.restype = ci
     L.imm_ldd_tail_fraction.argtypes = [vp, vp, i64, ctypes.c_double, ctypes.c_double, vp, vp, vp]
     L.imm_sumcheck_verify.restype = ci
@@ -363,17 +365,24 @@ def ldd_tv_kl(logits: torch.Tensor, ref_logits: torch.Tensor) -> Tuple[torch.Ten
     return tv, kl
 
 
-def ldd_topk_distance(ref_logits: torch.Tensor, topk: torch.Tensor) -> Tuple[torch.Tensor, torch.Tensor]:
+def ldd_topk_distance(ref_logits: torch.Tensor, topk: torch.Tensor,
+                      workspace: Optional[torch.Tensor] = None) -> Tuple[torch.Tensor, torch.Tensor]:
     """Top-K distance of every row to its claimed index set (int32, steps x K); returns
-    (float64 distances, int32 per-row status)."""
+    (float64 distances, int32 per-row status).  ``workspace``: a uint8 CUDA tensor of at least
+    ``imm_ldd_topk_workspace`` bytes to reuse between calls (allocated here when absent)."""
     steps, n, ld = _logit_rows(ref_logits, "ref_logits")
     topk = _cuda(topk, torch.int32, "topk")
     if topk.dim() != 2 or topk.shape[0] != steps or not topk.is_contiguous():
         raise ValueError("topk: expected a contiguous int32 tensor of shape (steps, K)")
     dist = torch.empty(steps, dtype=torch.float64, device=ref_logits.device)
     status = torch.full((steps,), -99, dtype=torch.int32, device=ref_logits.device)
-    _check(lib().imm_ldd_topk_distance(ref_logits.data_ptr(), steps, n, ld, topk.data_ptr(), int(topk.shape[1]),
-                                       dist.data_ptr(), status.data_ptr(), _stream()), "imm_ldd_topk_distance")
+    k = int(topk.shape[1])
+    need = lib().imm_ldd_topk_workspace(steps, n, k)
+    if workspace is None:
+        workspace = torch.empty(max(need, 16), dtype=torch.uint8, device=ref_logits.device)
+    _check(lib().imm_ldd_topk_distance(ref_logits.data_ptr(), steps, n, ld, topk.data_ptr(), k,
+                                       dist.data_ptr(), status.data_ptr(), workspace.data_ptr(), workspace.numel(),
+                                       _stream()), "imm_ldd_topk_distance")
     return dist, status
 
 

@@ -261,10 +261,10 @@ int imm_ldd_tv_kl(const float* d_logits, const float* d_ref_logits, int64_t step
  * indices in [0, n)).  It is 0 iff I_i is a valid top-K set of the row.  Computed as the minimum
  * over thresholds t of  sum_{j not in I} max(l_j - t, 0) + sum_{i in I} max(t - l_i, 0).
  * status[i] = IMM_OK, IMM_ERR_ARG (an index out of range or repeated; dist[i] = NaN), or
- * IMM_ERR_LIMIT (after six refinements more than 256 entries of one 16384-entry slice still lie
+ * IMM_ERR_LIMIT (after six refinements more than 256 entries of one 8192-entry slice still lie
  * above the bound on its K-th largest entry; dist[i] = NaN).
  * d_ws: DEVICE workspace of at least imm_ldd_topk_workspace(steps, n, k) bytes, 16-byte aligned;
- * the call overwrites it (a per-row counter and every slice's K largest entries).
+ * the call overwrites it (a flag word and the K largest entries of every 8192-entry slice).
  * Errors of the call itself: as imm_ldd_tv_kl, plus IMM_ERR_SHAPE for k outside
  * 1..min(n, IMM_LDD_MAX_K) and IMM_ERR_WORKSPACE. */
 size_t imm_ldd_topk_workspace(int64_t steps, int64_t n, int k);

@@ -216,22 +216,27 @@ tv_kl_kernel(const float* __restrict__ logits, const float* __restrict__ ref, in
 //   (unless the slice is adversarial; then tau is raised from what was collected and the collection
 //   repeats);
 //   the K largest of what was collected, padded with copies of tau (K entries outside I are >=
-//   tau), go to the workspace.  The block that finishes a row last merges the slices' lists,
+//   tau), go to the workspace.  A second, small kernel merges the slices' lists of every row,
 //   keeps the K largest, and evaluates the cost at the 2K breakpoints in float64.
 
+#ifndef IMM_LDD_TK_THREADS
+#define IMM_LDD_TK_THREADS 256
+#endif
+constexpr int TK_THREADS = IMM_LDD_TK_THREADS;   // threads per block of the Top-K kernel
+constexpr int TK_WARPS = TK_THREADS / 32;
+constexpr int TK_SLICE = 32 * TK_THREADS;         // entries of a row per block: 32 per thread, in registers
 constexpr int MAX_CAND = 128;                 // group maxima per block (>= 2 * MAX_K)
-constexpr int MERGE_CAP = 4096;               // a row's lists the merging block holds at once: (n / SLICE) * K
+constexpr int MERGE_CAP = (IMM_LDD_MAX_N / TK_SLICE) * MAX_K;   // a row's lists, held at once by the merging block
+constexpr int TK_MERGE_THREADS = 128;         // >= 2 * MAX_K
 
 struct TopkShared {
-    uint32_t member[SLICE / 32 + 2];      // bitmap of the slice's entries that belong to I
-    float work[MERGE_CAP];                // thread maxima / group maxima / collected entries / the row's lists
-    float collected[COLLECT_CAP];         // entries outside I above tau
-    float topk[MAX_K];
-    float inside[MAX_K];                  // merging block: the entries of I
-    double cost[2 * MAX_K];
+    float work[TK_THREADS + COLLECT_CAP]; // thread maxima / group maxima / collected entries plus copies of tau
+    float collected[COLLECT_CAP];         // entries above tau ...
+    int collected_at[COLLECT_CAP];        // ... and where in the slice they sit
+    int member_at[MAX_K];                 // the entries of I that fall into this slice
     float tau, proposal;
     int count;                            // entries collected in this pass (may exceed COLLECT_CAP)
-    int bad, last;
+    int members, bad;
 };
 
 // rank of all[i] in descending order, ties broken by position: a permutation of 0..m-1
@@ -246,188 +251,218 @@ __device__ __forceinline__ int rank_desc(const float* all, int m, int i)
     return r;
 }
 
+// The entries of I are not masked while streaming (that would cost more instructions per entry
+// than everything else together).  With m of them in the slice, the (K + m)-th largest group
+// maximum still has K entries outside I at or above it, so it is a valid bound; entries of I
+// that get collected are dropped afterwards by their position.
 template <bool VEC>
-__global__ void __launch_bounds__(THREADS, 2)
-topk_distance_kernel(const float* __restrict__ ref, int64_t n, int64_t ld, const int32_t* __restrict__ topk,
-                     int K, int nslices, float* __restrict__ lists, uint32_t* __restrict__ done,
-                     double* __restrict__ dist_out, int32_t* __restrict__ status)
+__global__ void __launch_bounds__(TK_THREADS, 1024 / TK_THREADS)
+topk_slice_kernel(const float* __restrict__ ref, int64_t n, int64_t ld, const int32_t* __restrict__ topk,
+                  int K, int nslices, float* __restrict__ lists, int32_t* __restrict__ flags)
 {
     __shared__ TopkShared sh;
     const int64_t step = blockIdx.x / nslices;
     const int c = (int)(blockIdx.x % nslices);
     const int32_t* I = topk + step * K;
     const int tid = threadIdx.x;
-    const int64_t s0 = (int64_t)c * SLICE, s1 = min(n, s0 + SLICE);
-    const float* row = ref + step * ld;
-    const float* y = row + s0;                         // this block's slice
+    const int64_t s0 = (int64_t)c * TK_SLICE, s1 = min(n, s0 + TK_SLICE);
+    const float* y = ref + step * ld + s0;             // this block's slice
     const int len = (int)(s1 - s0);
     const int nvec = VEC ? len >> 2 : 0;               // whole 16-byte vectors; the rest goes entry by entry
     const float4* yv = reinterpret_cast<const float4*>(y);
 
-    for (int i = tid; i < SLICE / 32 + 2; i += THREADS) sh.member[i] = 0;
-    if (tid == 0) { sh.bad = 0; sh.count = 0; }
-    __syncthreads();
-    if (tid < K) {
-        const int64_t idx = I[tid];
-        if (idx < 0 || idx >= n) sh.bad = 1;
-        else if (idx >= s0 && idx < s1) {
-            const int rel = (int)(idx - s0);
-            const uint32_t bit = 1u << (rel & 31);
-            if (atomicOr(&sh.member[rel >> 5], bit) & bit) sh.bad = 1;       // the same index twice
-        }
-    }
-    __syncthreads();
-
-    // The thread's 32 entries of the slice stay in registers: all loads are issued at once, and the
-    // second look at the data (once tau is known) needs no memory access.  Entries of I, and slots
-    // past the end of the slice, are replaced by -inf: they can never be collected.
-    constexpr int PER = SLICE / THREADS;               // 32 entries per thread
+    // The thread's 32 entries of the slice stay in registers: all loads are issued at once (before
+    // anything else, so that the set-up below runs while they are in flight), and the second look
+    // at the data, once tau is known, needs no memory access.  Slots past the end hold -inf.
+    constexpr int PER = TK_SLICE / TK_THREADS;         // 32 entries per thread
     float vals[PER];
     if (VEC) {
+        if (len == TK_SLICE) {
 #pragma unroll
-        for (int u = 0; u < PER / 4; u++) {
-            const int v = tid + u * THREADS;
-            const float4 q = v < nvec ? __ldg(yv + v) : make_float4(NEG_INF, NEG_INF, NEG_INF, NEG_INF);
-            vals[4 * u] = q.x; vals[4 * u + 1] = q.y; vals[4 * u + 2] = q.z; vals[4 * u + 3] = q.w;
-        }
+            for (int u = 0; u < PER / 4; u++) {
+                const float4 q = __ldg(yv + tid + u * TK_THREADS);
+                vals[4 * u] = q.x; vals[4 * u + 1] = q.y; vals[4 * u + 2] = q.z; vals[4 * u + 3] = q.w;
+            }
+        } else {
 #pragma unroll
-        for (int u = 0; u < PER / 4; u++) {
-            const int v = tid + u * THREADS;
-            const uint32_t m = v < nvec ? sh.member[v >> 3] >> ((4 * v) & 31) : 0u;   // four consecutive bits of one word
-#pragma unroll
-            for (int k = 0; k < 4; k++) if ((m >> k) & 1u) vals[4 * u + k] = NEG_INF;
+            for (int u = 0; u < PER / 4; u++) {
+                const int v = tid + u * TK_THREADS;
+                const float4 q = v < nvec ? __ldg(yv + v) : make_float4(NEG_INF, NEG_INF, NEG_INF, NEG_INF);
+                vals[4 * u] = q.x; vals[4 * u + 1] = q.y; vals[4 * u + 2] = q.z; vals[4 * u + 3] = q.w;
+            }
         }
     } else {
 #pragma unroll
         for (int j = 0; j < PER; j++) {
-            const int e = tid + j * THREADS;
+            const int e = tid + j * TK_THREADS;
             vals[j] = e < len ? y[e] : NEG_INF;
         }
-#pragma unroll
-        for (int j = 0; j < PER; j++) {
-            const int e = tid + j * THREADS;
-            if (e < len && ((sh.member[e >> 5] >> (e & 31)) & 1u)) vals[j] = NEG_INF;
-        }
     }
-    float tail = NEG_INF;                              // aligned rows: the up to three entries after the last whole vector
-    if (VEC && tid < len - 4 * nvec) {
-        const int e = 4 * nvec + tid;
-        if (!((sh.member[e >> 5] >> (e & 31)) & 1u)) tail = y[e];
+    // aligned rows: the up to three entries after the last whole vector
+    const int tail_at = 4 * nvec + tid;
+    const float tail = (VEC && tail_at < len) ? y[tail_at] : NEG_INF;
+
+    if (tid == 0) { sh.bad = 0; sh.count = 0; sh.members = 0; }
+    __syncthreads();
+    if (tid < K) {
+        const int64_t idx = I[tid];
+        if (idx < 0 || idx >= n) sh.bad = 1;
+        else if (idx >= s0 && idx < s1) sh.member_at[atomicAdd(&sh.members, 1)] = (int)(idx - s0);
     }
+    __syncthreads();
+    const int members = sh.members;
+    if (tid < members)                                 // the same index twice?
+        for (int k = 0; k < tid; k++)
+            if (sh.member_at[k] == sh.member_at[tid]) sh.bad = 1;
+
     float best = tail;
 #pragma unroll
     for (int j = 0; j < PER; j++) best = fmaxf(best, vals[j]);
     const float thread_best = best;                    // (before the group reduction below)
 
-    // group maxima: ncand = the smallest power of two >= 2K (16 at least: one group per warp)
-    int ncand = WARPS;
+    // group maxima: ncand = the smallest power of two >= 2K (at least one group per warp)
+    int ncand = TK_WARPS;
     while (ncand < 2 * K) ncand <<= 1;                 // <= MAX_CAND
-    const int G = THREADS / ncand;                     // 32, 16, 8 or 4 threads per group
+    const int G = TK_THREADS / ncand;
     for (int o = 1; o < G; o <<= 1) best = fmaxf(best, __shfl_xor_sync(0xFFFFFFFFu, best, o));
     if ((tid % G) == 0) sh.work[tid / G] = best;
     __syncthreads();
-    if (tid < ncand && rank_desc(sh.work, ncand, tid) == K - 1) sh.tau = sh.work[tid];
+    const int want = K + members - 1;                  // rank of the bound: K entries outside I are at or above it
+    if (tid < ncand && rank_desc(sh.work, ncand, tid) == want) sh.tau = sh.work[tid];
     __syncthreads();
     float tau = sh.tau;
 
     bool failed = false;
     for (int round = 0;; round++) {
-        // collect the entries outside I above tau (from registers)
+        // collect the entries above tau (from registers)
         if (thread_best > tau) {                       // rare: about K + a few threads of the block
 #pragma unroll
             for (int j = 0; j < PER; j++)
                 if (vals[j] > tau) {
                     const int slot = atomicAdd(&sh.count, 1);
-                    if (slot < COLLECT_CAP) sh.collected[slot] = vals[j];
+                    if (slot < COLLECT_CAP) {
+                        sh.collected[slot] = vals[j];
+                        sh.collected_at[slot] = VEC ? 4 * (tid + (j >> 2) * TK_THREADS) + (j & 3) : tid + j * TK_THREADS;
+                    }
                 }
             if (tail > tau) {
                 const int slot = atomicAdd(&sh.count, 1);
-                if (slot < COLLECT_CAP) sh.collected[slot] = tail;
+                if (slot < COLLECT_CAP) { sh.collected[slot] = tail; sh.collected_at[slot] = tail_at; }
             }
         }
         __syncthreads();
         if (sh.count <= COLLECT_CAP) break;
         if (round + 1 == MAX_REFINE) { failed = true; break; }     // gave up raising the bound
-        // More than the block can hold: raise the bound.  The K-th largest of the threads' maxima, and
-        // the K-th largest of the entries that were held, are both entries outside I with K entries at
-        // or above them, so either is still a lower bound; the second one lies above tau, so the bound
-        // rises every round.
+        // More than the block can hold: raise the bound.  The (K + m)-th largest of the threads'
+        // maxima, and the (K + m)-th largest of the entries that were held, both have K entries
+        // outside I at or above them, so either is still a lower bound; the second one lies above
+        // tau, so the bound rises every round.
         sh.work[tid] = thread_best;
         __syncthreads();
-        if (rank_desc(sh.work, THREADS, tid) == K - 1) sh.proposal = sh.work[tid];
+        if (rank_desc(sh.work, TK_THREADS, tid) == want) sh.proposal = sh.work[tid];
         __syncthreads();
         if (tid < COLLECT_CAP) sh.work[tid] = sh.collected[tid];
         __syncthreads();
-        if (tid < COLLECT_CAP && rank_desc(sh.work, COLLECT_CAP, tid) == K - 1) sh.proposal = fmaxf(sh.proposal, sh.work[tid]);
+        if (tid < COLLECT_CAP && rank_desc(sh.work, COLLECT_CAP, tid) == want) sh.proposal = fmaxf(sh.proposal, sh.work[tid]);
         __syncthreads();
         tau = fmaxf(tau, sh.proposal);
         if (tid == 0) sh.count = 0;
         __syncthreads();
     }
 
-    // this slice's K largest entries outside I: what was collected plus K copies of tau
+    // this slice's K largest entries outside I: what was collected, without the entries of I, plus
+    // K copies of tau
     {
         const int cnt = min(sh.count, COLLECT_CAP);
-        for (int i = tid; i < cnt; i += THREADS) sh.work[i] = sh.collected[i];
-        for (int i = tid; i < K; i += THREADS) sh.work[cnt + i] = tau;
+        for (int i = tid; i < cnt; i += TK_THREADS) {
+            float v = sh.collected[i];
+            const int at = sh.collected_at[i];
+            for (int k = 0; k < members; k++) if (sh.member_at[k] == at) v = NEG_INF;
+            sh.work[i] = v;
+        }
+        for (int i = tid; i < K; i += TK_THREADS) sh.work[cnt + i] = tau;
         __syncthreads();
         float* mine = lists + ((int64_t)step * nslices + c) * K;
-        for (int i = tid; i < cnt + K; i += THREADS) {
+        for (int i = tid; i < cnt + K; i += TK_THREADS) {
             const int r = rank_desc(sh.work, cnt + K, i);
             if (r < K) mine[r] = sh.work[i];
         }
     }
-    // the block that finishes a row last merges it (nobody waits: the others are done)
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) {
-        // low half: slices done; bit 16: a bad index; bit 17: a slice gave up
-        const uint32_t flags = (sh.bad ? 0x10000u : 0u) | (failed ? 0x20000u : 0u);
-        if (flags) atomicOr(&done[step], flags);
-        const uint32_t old = atomicAdd(&done[step], 1u);
-        sh.last = (int)((old & 0xFFFFu) == (uint32_t)(nslices - 1));
-        if (sh.last) sh.bad = (int)(((old | flags) >> 16) & 3u);             // what any block of the row reported
-    }
-    __syncthreads();
-    if (!sh.last) return;
-    __threadfence();
+    if (tid == 0) flags[(int64_t)step * nslices + c] = (sh.bad ? 1 : 0) | (failed ? 2 : 0);
+}
 
+// One block per row: the K largest of the slices' lists, the entries of I, the cost at the 2K
+// breakpoints in float64.  The lists are sorted, so their first h entries (h chosen to give 2K
+// heads in all) bound the K-th largest entry from below, and only the few entries above that
+// bound need ranking.
+__global__ void __launch_bounds__(TK_MERGE_THREADS)
+topk_merge_kernel(const float* __restrict__ ref, int64_t n, int64_t ld, const int32_t* __restrict__ topk,
+                  int K, int nslices, const float* __restrict__ lists, const int32_t* __restrict__ flags,
+                  double* __restrict__ dist_out, int32_t* __restrict__ status)
+{
+    __shared__ float all[MERGE_CAP + MAX_K];
+    __shared__ float heads[2 * MAX_K + IMM_LDD_MAX_N / TK_SLICE];
+    __shared__ float top[MAX_K], inside[MAX_K];
+    __shared__ double cost[2 * MAX_K];
+    __shared__ float bound;
+    __shared__ int bad, count;
+    const int64_t step = blockIdx.x;
+    const int tid = threadIdx.x;
+    const float* row = ref + step * ld;
+    const int32_t* I = topk + step * K;
+    const float* mine = lists + step * nslices * K;
     const int m = nslices * K;                             // <= MERGE_CAP (checked on the host)
-    const float* all = lists + (int64_t)step * nslices * K;
-    for (int i = tid; i < m; i += THREADS) sh.work[i] = __ldcg(all + i);
+    if (tid == 0) { bad = 0; count = 0; }
     if (tid < K) {
         const int64_t idx = I[tid];
-        sh.inside[tid] = (idx >= 0 && idx < n) ? row[idx] : 0.f;
+        inside[tid] = (idx >= 0 && idx < n) ? row[idx] : 0.f;
+    }
+    const int h = min(K, (2 * K + nslices - 1) / nslices), nh = nslices * h;
+    for (int i = tid; i < nh; i += TK_MERGE_THREADS) heads[i] = mine[(i / h) * K + i % h];
+    __syncthreads();
+    for (int i = tid; i < nslices; i += TK_MERGE_THREADS) {
+        const int f = flags[step * nslices + i];
+        if (f) atomicOr(&bad, f);
+    }
+    for (int i = tid; i < nh; i += TK_MERGE_THREADS)
+        if (rank_desc(heads, nh, i) == K - 1) bound = heads[i];    // K entries outside I are at or above it
+    __syncthreads();
+    const float t0 = bound;
+    for (int i = tid; i < m; i += TK_MERGE_THREADS) {
+        const float v = mine[i];
+        if (v > t0) all[atomicAdd(&count, 1)] = v;
     }
     __syncthreads();
-    for (int i = tid; i < m; i += THREADS) {
-        const int r = rank_desc(sh.work, m, i);
-        if (r < K) sh.topk[r] = sh.work[i];
+    const int cnt = count;
+    for (int i = tid; i < K; i += TK_MERGE_THREADS) all[cnt + i] = t0;
+    __syncthreads();
+    for (int i = tid; i < cnt + K; i += TK_MERGE_THREADS) {
+        const int r = rank_desc(all, cnt + K, i);
+        if (r < K) top[r] = all[i];
     }
     __syncthreads();
-    // cost at the 2K breakpoints, in double
     if (tid < 2 * K) {
-        const double t = tid < K ? (double)sh.topk[tid] : (double)sh.inside[tid - K];
-        double cost = INFINITY;
+        const double t = tid < K ? (double)top[tid] : (double)inside[tid - K];
+        double c = INFINITY;
         if (t > -INFINITY) {                               // a row with fewer than K entries outside I pads with -inf
-            cost = 0.0;
+            c = 0.0;
             for (int k = 0; k < K; k++) {
-                cost += fmax((double)sh.topk[k] - t, 0.0);
-                cost += fmax(t - (double)sh.inside[k], 0.0);
+                c += fmax((double)top[k] - t, 0.0);
+                c += fmax(t - (double)inside[k], 0.0);
             }
         }
-        sh.cost[tid] = cost;
+        cost[tid] = c;
     }
     __syncthreads();
     if (tid < 32) {
         double best_cost = INFINITY;
-        for (int i = tid; i < 2 * K; i += 32) best_cost = fmin(best_cost, sh.cost[i]);
+        for (int i = tid; i < 2 * K; i += 32) best_cost = fmin(best_cost, cost[i]);
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) best_cost = fmin(best_cost, __shfl_xor_sync(0xFFFFFFFFu, best_cost, o));
         if (tid == 0) {
-            const bool bad = (sh.bad & 1) != 0, gave_up = (sh.bad & 2) != 0;
-            dist_out[step] = (bad || gave_up) ? NAN : best_cost;
-            status[step] = bad ? IMM_ERR_ARG : gave_up ? IMM_ERR_LIMIT : IMM_OK;
+            const bool bad_index = (bad & 1) != 0, gave_up = (bad & 2) != 0;
+            dist_out[step] = (bad_index || gave_up) ? NAN : best_cost;
+            status[step] = bad_index ? IMM_ERR_ARG : gave_up ? IMM_ERR_LIMIT : IMM_OK;
         }
     }
 }
@@ -522,9 +557,9 @@ size_t imm_ldd_topk_workspace(int64_t steps, int64_t n, int k)
 {
     using namespace imm_ldd;
     if (steps < 0 || n <= 0 || n > IMM_LDD_MAX_N || steps > IMM_LDD_MAX_STEPS || k <= 0 || k > IMM_LDD_MAX_K) return 0;
-    const int64_t nslices = (n + SLICE - 1) / SLICE;
-    // one counter per row, then every slice's K largest entries
-    return (size_t)((steps * 4 + 255) / 256 * 256) + (size_t)steps * nslices * k * sizeof(float) + 256;
+    const int64_t nslices = (n + TK_SLICE - 1) / TK_SLICE;
+    // one flag word per slice, then every slice's K largest entries
+    return (size_t)((steps * nslices * 4 + 255) / 256 * 256) + (size_t)steps * nslices * k * sizeof(float) + 256;
 }
 
 int imm_ldd_topk_distance(const float* d_ref_logits, int64_t steps, int64_t n, int64_t ld,
@@ -540,16 +575,18 @@ int imm_ldd_topk_distance(const float* d_ref_logits, int64_t steps, int64_t n, i
         return IMM_ERR_ALIGN;
     if (ws_bytes < imm_ldd_topk_workspace(steps, n, k)) return IMM_ERR_WORKSPACE;
     if (steps == 0) return IMM_OK;
-    const int64_t nslices = (n + SLICE - 1) / SLICE;
+    const int64_t nslices = (n + TK_SLICE - 1) / TK_SLICE;
     if (nslices * k > MERGE_CAP || steps * nslices > 0x7FFFFFFF) return IMM_ERR_SHAPE;     // (cannot happen within the limits)
     cudaStream_t st = (cudaStream_t)stream;
-    uint32_t* done = (uint32_t*)d_ws;
-    float* lists = (float*)((char*)d_ws + (steps * 4 + 255) / 256 * 256);
-    if (cudaMemsetAsync(done, 0, (size_t)steps * 4, st) != cudaSuccess) return IMM_ERR_CUDA;
+    int32_t* flags = (int32_t*)d_ws;
+    float* lists = (float*)((char*)d_ws + (steps * nslices * 4 + 255) / 256 * 256);
     const bool vec = rows_aligned(d_ref_logits, ld);
     const unsigned grid = (unsigned)(steps * nslices);
-    if (vec) topk_distance_kernel<true><<<grid, THREADS, 0, st>>>(d_ref_logits, n, ld, d_topk, k, (int)nslices, lists, done, d_dist, d_status);
-    else topk_distance_kernel<false><<<grid, THREADS, 0, st>>>(d_ref_logits, n, ld, d_topk, k, (int)nslices, lists, done, d_dist, d_status);
+    if (vec) topk_slice_kernel<true><<<grid, TK_THREADS, 0, st>>>(d_ref_logits, n, ld, d_topk, k, (int)nslices, lists, flags);
+    else topk_slice_kernel<false><<<grid, TK_THREADS, 0, st>>>(d_ref_logits, n, ld, d_topk, k, (int)nslices, lists, flags);
+    if (cudaGetLastError() != cudaSuccess) return IMM_ERR_CUDA;
+    topk_merge_kernel<<<(unsigned)steps, TK_MERGE_THREADS, 0, st>>>(d_ref_logits, n, ld, d_topk, k, (int)nslices, lists, flags,
+                                                                    d_dist, d_status);
     return cudaGetLastError() == cudaSuccess ? IMM_OK : IMM_ERR_CUDA;
 }
 

@@ -192,7 +192,7 @@ def measured_peaks():
 # DRAM traffic of the claim kernel per algorithmic byte, from the ncu capture summarised under
 # profiles/ (dram__bytes_read.sum + dram__bytes_write.sum over 4*m*n); None until a capture of the
 # current kernel exists.
-LDD_TVKL_TRAFFIC_RATIO = None   # tv_kl_kernel: (dram read + write) / (8 bytes per entry pair), same source
+LDD_TVKL_TRAFFIC_RATIO = 1.0721 / 1.050673   # tv_kl_kernel<aligned, 512 threads>: (dram read + write) / (8 bytes per entry pair)
 CLAIM_KERNEL_TRAFFIC_RATIO = 240.14 / 234.881024  # bytedot_kernel<1,1,1>, per-warp partials, no per-tile offset sum
 
 

@@ -127,6 +127,11 @@ Geom pick_geom(const std::vector<Shape>& mats, const int* rows, int nrows, const
     return best;
 }
 
+// candidate tile heights and widths of the tensor-core kernels, largest first
+const int rows_a[] = {1024, 512, 256, 128, 64, 32}, widths_a[] = {1024, 512, 256, 128};
+const int rows_b[] = {256}, rows_c[] = {1024, 512, 256, 128};
+const int chunks[] = {4096, 2048, 1024, 512, 256};
+
 void fill_job(MatJob& j, const void* mat, int dtype, int64_t rows, int64_t cols, int64_t ld,
               int tile_rows, int cols_per_tile)
 {
@@ -148,6 +153,59 @@ int check_matrix_args(const void* d_mat, int dtype, int64_t rows, int64_t cols, 
     if (!d_mat || (dtype != IMM_I8 && dtype != IMM_I32)) return IMM_ERR_ARG;
     if (rows <= 0 || cols <= 0 || rows > MAX_EXTENT || cols > MAX_EXTENT || ld < cols) return IMM_ERR_SHAPE;
     return IMM_OK;
+}
+
+// ------------------------------------------------------------------ single-matrix calls ---
+// imm_mle_partial_eval / imm_mle_eval_point on the tensor-core kernels: the workspace holds the job,
+// two eq tasks (limb tables and slice sums from the caller's eq tables), the limb table, the slice
+// sums and the partial results.  int32 partial evaluations have no tensor-core kernel and stay on
+// the integer-pipe kernels, as does everything under IMM_CONTRACT=alu.
+enum MleOp { OP_ROWS = 0, OP_COLS = 1, OP_POINT = 2 };
+
+struct MlePlan {
+    bool mma = false;
+    Geom g{0, 0};
+    int64_t nrb = 0, ncc = 0, nparts = 0;
+    int nw = 0, n_sr = 0, n_sc = 0;
+    size_t off_tasks = 0, off_w = 0, off_sr = 0, off_sc = 0, off_parts = 0, total = 0;
+};
+
+MlePlan plan_mle(int dtype, int64_t rows, int64_t cols, MleOp op)
+{
+    MlePlan p;
+    p.mma = use_mma() && (op == OP_POINT || dtype == IMM_I8);
+    if (!p.mma) return p;
+    const int64_t slice = 4 * (int64_t)EQ_SLICE_QUADS;
+    if (op == OP_ROWS) {
+        std::vector<Shape> m{{rows, cols}};
+        p.g = pick_geom(m, rows_a, 6, widths_a, 4, 12, "IMM_TILE_ROWS_A", "IMM_TILE_COLS_A");
+        p.nw = (int)((rows + 31) / 32) * 64;
+    } else if (op == OP_COLS) {
+        std::vector<Shape> m{{rows, cols}};
+        p.g = pick_geom(m, rows_b, 1, chunks, 5, 24, "IMM_TILE_ROWS_B", "IMM_CHUNK_B");
+        p.nw = (int)((cols + 255) / 256) * 512;
+    } else {
+        const int64_t bytes = cols * (int64_t)elem_size(dtype);
+        std::vector<Shape> m{{rows, bytes}};
+        p.g = pick_geom(m, rows_c, 4, chunks, 5, 24, "IMM_TILE_ROWS_C", "IMM_CHUNK_C");
+        p.nw = (int)((bytes + 255) / 256) * 512;
+        if (dtype == IMM_I32) {
+            p.n_sr = (int)((rows + slice - 1) / slice);
+            p.n_sc = (int)(((cols + 255) / 256 * 256 + slice - 1) / slice);
+        }
+    }
+    const int64_t width_elems = op == OP_POINT ? p.g.width / (int64_t)elem_size(dtype) : p.g.width;
+    p.nrb = (rows + p.g.rows - 1) / p.g.rows;
+    p.ncc = (cols + width_elems - 1) / width_elems;
+    p.nparts = op == OP_ROWS ? p.nrb * cols : op == OP_COLS ? p.ncc * rows : p.nrb * p.ncc * (BYTEDOT_THREADS / 32);
+    size_t off = ALIGN;                                   // the job
+    p.off_tasks = off; off = align_up(off + 2 * sizeof(EqTask));
+    p.off_w = off;     off = align_up(off + 4 * (size_t)p.nw);
+    p.off_sr = off;    off = align_up(off + sizeof(imm_fe) * (size_t)p.n_sr);
+    p.off_sc = off;    off = align_up(off + sizeof(imm_fe) * (size_t)p.n_sc);
+    p.off_parts = off; off = align_up(off + sizeof(imm_fe) * (size_t)p.nparts);
+    p.total = off;
+    return p;
 }
 
 // ------------------------------------------------------------------ batch plan ------------
@@ -203,9 +261,6 @@ Plan make_plan(const imm_matmul_desc* descs, int nproofs)
         // 128 rows per MMA row tile, so shorter tiles would leave warps idle.  Measured on the
         // decoder-block workload: B (two row tiles per warp) is best at 256 rows per tile, C (one) at
         // 512-1024.
-        static const int rows_a[] = {1024, 512, 256, 128, 64, 32}, widths_a[] = {1024, 512, 256, 128};
-        static const int rows_b[] = {256}, rows_c[] = {1024, 512, 256, 128};
-        static const int chunks[] = {4096, 2048, 1024, 512, 256};
         p.mt_b = env_int("IMM_BYTEDOT_MT_B", 2) == 1 ? 1 : 2;
         p.mt_c = env_int("IMM_BYTEDOT_MT_C", 1) == 2 ? 2 : 1;
         std::vector<Shape> scb;                               // C as a byte matrix
@@ -351,7 +406,14 @@ size_t imm_mle_workspace(int dtype, int64_t rows, int64_t cols, int bind)
         int64_t ncc = (cols + colbind_cols(dtype) - 1) / colbind_cols(dtype);
         parts = (size_t)ncc * rows;
     }
-    return ALIGN + align_up(parts * sizeof(imm_fe));
+    size_t need = ALIGN + align_up(parts * sizeof(imm_fe));       // the integer-pipe kernels
+    const MlePlan a = plan_mle(dtype, rows, cols, bind == IMM_BIND_ROWS ? OP_ROWS : OP_COLS);
+    if (a.mma && a.total > need) need = a.total;
+    if (bind == IMM_BIND_ROWS) {                                    // imm_mle_eval_point sizes itself with BIND_ROWS
+        const MlePlan b = plan_mle(dtype, rows, cols, OP_POINT);
+        if (b.mma && b.total > need) need = b.total;
+    }
+    return need;
 }
 
 int imm_mle_partial_eval(const void* d_mat, int dtype, int64_t rows, int64_t cols, int64_t ld,
@@ -366,8 +428,41 @@ int imm_mle_partial_eval(const void* d_mat, int dtype, int64_t rows, int64_t col
     cudaStream_t st = (cudaStream_t)stream;
     std::vector<Shape> one{{rows, cols}};
     MatJob* d_job = (MatJob*)d_ws;
-    imm_fe* d_parts = (imm_fe*)((char*)d_ws + ALIGN);
     MatJob j;
+    const MlePlan mp = plan_mle(dtype, rows, cols, bind == IMM_BIND_ROWS ? OP_ROWS : OP_COLS);
+    if (mp.mma) {
+        // tensor-core path: limb table of the caller's eq weights, then the contraction
+        char* base = (char*)d_ws;
+        uint32_t* wtab = (uint32_t*)(base + mp.off_w);
+        imm_fe* parts = (imm_fe*)(base + mp.off_parts);
+        const bool by_rows = bind == IMM_BIND_ROWS;
+        const int64_t extent = by_rows ? rows : cols;
+        char hdr[ALIGN + 2 * sizeof(EqTask)];
+        memset(hdr, 0, sizeof(hdr));
+        fill_job(j, d_mat, dtype, rows, cols, ld, mp.g.rows, mp.g.width);
+        j.wtab = wtab;
+        j.chunk = mp.g.width;
+        const bool direct = (by_rows ? mp.nrb : mp.ncc) == 1;
+        j.out = direct ? d_out : parts;
+        if (by_rows) j.eq_row = d_eq; else j.eq_col = d_eq;
+        memcpy(hdr, &j, sizeof(j));
+        EqTask t{nullptr, 0, 0, 0u, 0, by_rows ? wtab : nullptr, by_rows ? nullptr : wtab, nullptr, (int32_t)extent, 0,
+                 nullptr, d_eq};
+        memcpy(hdr + ALIGN, &t, sizeof(t));
+        CU(cudaMemcpyAsync(base, hdr, sizeof(hdr), cudaMemcpyHostToDevice, st));
+        const int64_t pad = by_rows ? 32 : 256;
+        CU(launch_eq_batch((const EqTask*)(base + mp.off_tasks), 1, (extent + pad - 1) / pad * pad, st));
+        const uint32_t ntiles = (uint32_t)(mp.nrb * mp.ncc);
+        if (by_rows) {
+            CU(launch_rowmma(d_job, 1, ntiles, mp.g.width / 128, st));
+            if (!direct) CU(launch_sum_parts(parts, (int)mp.nrb, cols, d_out, st));
+        } else {
+            CU(launch_bytedot(false, false, 2, d_job, 1, ntiles, st));
+            if (!direct) CU(launch_sum_parts(parts, (int)mp.ncc, rows, d_out, st));
+        }
+        return IMM_OK;
+    }
+    imm_fe* d_parts = (imm_fe*)((char*)d_ws + ALIGN);
     if (bind == IMM_BIND_ROWS) {
         int tr = pick_tile_rows(one, rowbind_cols(dtype), "IMM_TILE_ROWS_A");
         fill_job(j, d_mat, dtype, rows, cols, ld, tr, rowbind_cols(dtype));
@@ -400,8 +495,41 @@ int imm_mle_eval_point(const void* d_mat, int dtype, int64_t rows, int64_t cols,
     cudaStream_t st = (cudaStream_t)stream;
     std::vector<Shape> one{{rows, cols}};
     MatJob* d_job = (MatJob*)d_ws;
-    imm_fe* d_parts = (imm_fe*)((char*)d_ws + ALIGN);
     MatJob j;
+    const MlePlan mp = plan_mle(dtype, rows, cols, OP_POINT);
+    if (mp.mma) {
+        // tensor-core path: limb table of eq_col (and, for int32, the sums of both eq tables for the
+        // 2^31 offset of the unsigned byte view), the point contraction, the final sum
+        char* base = (char*)d_ws;
+        uint32_t* wtab = (uint32_t*)(base + mp.off_w);
+        imm_fe* parts = (imm_fe*)(base + mp.off_parts);
+        imm_fe* sr = (imm_fe*)(base + mp.off_sr);
+        imm_fe* sc = (imm_fe*)(base + mp.off_sc);
+        const bool i32 = dtype == IMM_I32;
+        char hdr[ALIGN + 2 * sizeof(EqTask)];
+        memset(hdr, 0, sizeof(hdr));
+        const int width_elems = mp.g.width / (int)elem_size(dtype);
+        fill_job(j, d_mat, dtype, rows, cols, ld, mp.g.rows, width_elems);
+        j.wtab = wtab;
+        j.chunk = mp.g.width;
+        j.eq_row = d_eq_row;
+        j.eq_col = d_eq_col;
+        j.out = parts;
+        memcpy(hdr, &j, sizeof(j));
+        EqTask tc{nullptr, 0, 0, 0u, 0, nullptr, i32 ? nullptr : wtab, i32 ? wtab : nullptr, (int32_t)cols, 0,
+                  i32 ? sc : nullptr, d_eq_col};
+        EqTask tr_{nullptr, 0, 0, 0u, 0, nullptr, nullptr, nullptr, (int32_t)rows, 0, sr, d_eq_row};
+        memcpy(hdr + ALIGN, &tc, sizeof(tc));
+        memcpy(hdr + ALIGN + sizeof(EqTask), &tr_, sizeof(tr_));
+        CU(cudaMemcpyAsync(base, hdr, sizeof(hdr), cudaMemcpyHostToDevice, st));
+        int64_t cover = (cols + 255) / 256 * 256;
+        if (i32 && rows > cover) cover = rows;
+        CU(launch_eq_batch((const EqTask*)(base + mp.off_tasks), i32 ? 2 : 1, cover, st));
+        CU(launch_bytedot(i32, true, 1, d_job, 1, (uint32_t)(mp.nrb * mp.ncc), st));
+        CU(launch_point_finish(parts, mp.nparts, sr, mp.n_sr, sc, mp.n_sc, d_out, st));
+        return IMM_OK;
+    }
+    imm_fe* d_parts = (imm_fe*)((char*)d_ws + ALIGN);
     int tr = pick_tile_rows(one, rowbind_cols(dtype), "IMM_TILE_ROWS_A");
     fill_job(j, d_mat, dtype, rows, cols, ld, tr, rowbind_cols(dtype));
     j.eq_row = d_eq_row;

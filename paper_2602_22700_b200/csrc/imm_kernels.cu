@@ -461,6 +461,28 @@ __global__ void __launch_bounds__(1024) sum_all_kernel(const imm_fe* parts, int6
     if (threadIdx.x == 0) out[0] = s;
 }
 
+// out[0] = sum of `count` partial sums of a tensor-core point evaluation.  For an int32 matrix the
+// kernel summed unsigned bytes, so every entry reads 2^31 too high: 2^31 * (sum of the row weights)
+// * (sum of the column weights) comes off (nsr = 0: no offset).
+__global__ void __launch_bounds__(1024)
+point_finish_kernel(const imm_fe* parts, int64_t count, const imm_fe* sum_row, int nsr, const imm_fe* sum_col,
+                    int nsc, imm_fe* out)
+{
+    __shared__ uint64_t red[33];
+    uint64_t s = 0;
+    for (int64_t i = threadIdx.x; i < count; i += blockDim.x) s = gl::add(s, parts[i]);
+    s = block_sum_fe(s, red);
+    if (threadIdx.x == 0) {
+        if (nsr > 0) {
+            uint64_t sr = 0, sc = 0;
+            for (int i = 0; i < nsr; i++) sr = gl::add(sr, sum_row[i]);
+            for (int i = 0; i < nsc; i++) sc = gl::add(sc, sum_col[i]);
+            s = gl::sub(s, gl::shl(gl::mul(sr, sc), 31));
+        }
+        out[0] = s;
+    }
+}
+
 // ------------------------------------------------------------------------------------------
 // sumcheck rounds: one thread-block cluster per proof
 // ------------------------------------------------------------------------------------------
@@ -787,6 +809,13 @@ cudaError_t launch_sum_parts(const imm_fe* parts, int nparts, int64_t len, imm_f
 cudaError_t launch_sum_all(const imm_fe* parts, int64_t count, imm_fe* out, cudaStream_t st)
 {
     sum_all_kernel<<<1, 1024, 0, st>>>(parts, count, out);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_point_finish(const imm_fe* parts, int64_t count, const imm_fe* sum_row, int nsr,
+                                const imm_fe* sum_col, int nsc, imm_fe* out, cudaStream_t st)
+{
+    point_finish_kernel<<<1, 1024, 0, st>>>(parts, count, sum_row, nsr, sum_col, nsc, out);
     return cudaGetLastError();
 }
 

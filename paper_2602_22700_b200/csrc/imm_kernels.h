@@ -23,6 +23,9 @@ cudaError_t launch_bytedot(bool i32, bool point, int mt, const MatJob* d_jobs, i
 cudaError_t launch_rowmma(const MatJob* d_jobs, int njobs, uint32_t ntiles, int warps, cudaStream_t st);
 cudaError_t launch_sum_parts(const imm_fe* parts, int nparts, int64_t len, imm_fe* out, cudaStream_t st);
 cudaError_t launch_sum_all(const imm_fe* parts, int64_t count, imm_fe* out, cudaStream_t st);
+// sum of the partial sums of a tensor-core point evaluation, minus the 2^31 offset of an int32 matrix (nsr > 0)
+cudaError_t launch_point_finish(const imm_fe* parts, int64_t count, const imm_fe* sum_row, int nsr,
+                                const imm_fe* sum_col, int nsc, imm_fe* out, cudaStream_t st);
 // cluster: blocks per proof (1, 2, 4 or 8), or 0 to let the launch choose from the batch size
 cudaError_t launch_sumcheck(const ProofDev* d_proofs, int nproofs, uint64_t seed, imm_fe* transcripts,
                             int64_t stride, int32_t* status, int max_b, int cluster, cudaStream_t st);

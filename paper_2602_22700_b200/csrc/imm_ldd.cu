@@ -25,7 +25,6 @@ namespace imm_ldd {
 namespace cg = cooperative_groups;
 
 constexpr int THREADS = 512;
-constexpr int WARPS = THREADS / 32;
 constexpr int MAX_CLUSTER = 8;
 constexpr int SLICE = 16384;                  // entries of a row one block takes (before the cluster cap)
 constexpr int MAX_K = IMM_LDD_MAX_K;          // largest index set of the Top-K distance
@@ -322,7 +321,8 @@ topk_slice_kernel(const float* __restrict__ ref, int64_t n, int64_t ld, const in
 
     // group maxima: ncand = the smallest power of two >= 2K (at least one group per warp)
     int ncand = TK_WARPS;
-    while (ncand < 2 * K) ncand <<= 1;                 // <= MAX_CAND
+    while (ncand < 2 * K) ncand <<= 1;
+    static_assert(MAX_CAND >= 2 * MAX_K && MAX_CAND <= TK_THREADS, "group maxima must fit the block");
     const int G = TK_THREADS / ncand;
     for (int o = 1; o < G; o <<= 1) best = fmaxf(best, __shfl_xor_sync(0xFFFFFFFFu, best, o));
     if ((tid % G) == 0) sh.work[tid / G] = best;
@@ -537,19 +537,10 @@ int imm_ldd_tv_kl(const float* d_logits, const float* d_ref_logits, int64_t step
     if (steps == 0) return IMM_OK;
     const int nc = cluster_size(n);
     const bool vec = rows_aligned(d_logits, ld) && rows_aligned(d_ref_logits, ld);
-    int nt = 512, ncl = nc;
-    if (const char* v = getenv("IMM_LDD_THREADS")) nt = atoi(v) == 256 ? 256 : atoi(v) == 1024 ? 1024 : 512;
-    if (const char* v = getenv("IMM_LDD_CLUSTER")) { int c = atoi(v); if (c == 1 || c == 2 || c == 4 || c == 8 || c == 16) ncl = c; }
     cudaStream_t st = (cudaStream_t)stream;
-    cudaError_t e;
-#define TVKL_LAUNCH(V, T) do { \
-        if (ncl > 8) cudaFuncSetAttribute(tv_kl_kernel<V, T>, cudaFuncAttributeNonPortableClusterSizeAllowed, 1); \
-        e = launch_cluster(tv_kl_kernel<V, T>, steps, ncl, T, 0, st, d_logits, d_ref_logits, n, ld, d_tv, d_kl); } while (0)
-    if (!vec) TVKL_LAUNCH(false, 512);
-    else if (nt == 256) TVKL_LAUNCH(true, 256);
-    else if (nt == 1024) TVKL_LAUNCH(true, 1024);
-    else TVKL_LAUNCH(true, 512);
-#undef TVKL_LAUNCH
+    // 512 threads and clusters of up to 8 blocks measured best (256 / 1024 threads and 16-block clusters were tried)
+    cudaError_t e = vec ? launch_cluster(tv_kl_kernel<true, THREADS>, steps, nc, THREADS, 0, st, d_logits, d_ref_logits, n, ld, d_tv, d_kl)
+                        : launch_cluster(tv_kl_kernel<false, THREADS>, steps, nc, THREADS, 0, st, d_logits, d_ref_logits, n, ld, d_tv, d_kl);
     return e == cudaSuccess ? IMM_OK : IMM_ERR_CUDA;
 }
 

@@ -93,7 +93,8 @@ __global__ void __launch_bounds__(EQ_BATCH_THREADS) eq_batch_kernel(const EqTask
     __shared__ uint64_t r_sh[MAX_EQ_VARS], omr_sh[MAX_EQ_VARS];
     __shared__ uint64_t lo_t[1024], hi_t[1024];
     const EqTask tk = tasks[blockIdx.y];
-    const int64_t total = (int64_t)1 << tk.nvars;
+    const bool from_table = tk.given != nullptr;
+    const int64_t total = from_table ? (int64_t)tk.extent : (int64_t)1 << tk.nvars;
     // entries this task has to cover: the table itself, and the limb tables' zero padding
     const int64_t pad = tk.w_rows ? 32 : 256;
     const int64_t cover = (tk.w_rows || tk.w_cols_i8 || tk.w_cols_i32)
@@ -103,16 +104,18 @@ __global__ void __launch_bounds__(EQ_BATCH_THREADS) eq_batch_kernel(const EqTask
     __shared__ uint64_t red[33];
     uint64_t slice_sum = 0;
 
-    if ((int)threadIdx.x < tk.nvars) {
-        const uint64_t r = gl::challenge(tk.seed, tk.proof_id, tk.domain, threadIdx.x);
-        r_sh[threadIdx.x] = r;
-        omr_sh[threadIdx.x] = gl::sub(1, r);
-    }
-    __syncthreads();
     const int nlo = (tk.nvars + 1) / 2, nhi = tk.nvars - nlo;
-    for (int x = threadIdx.x; x < (1 << nhi); x += EQ_BATCH_THREADS) hi_t[x] = eq_product(r_sh, omr_sh, nhi, x);
-    for (int x = threadIdx.x; x < (1 << nlo); x += EQ_BATCH_THREADS) lo_t[x] = eq_product(r_sh + nhi, omr_sh + nhi, nlo, x);
-    __syncthreads();
+    if (!from_table) {                                 // (uniform over the block)
+        if ((int)threadIdx.x < tk.nvars) {
+            const uint64_t r = gl::challenge(tk.seed, tk.proof_id, tk.domain, threadIdx.x);
+            r_sh[threadIdx.x] = r;
+            omr_sh[threadIdx.x] = gl::sub(1, r);
+        }
+        __syncthreads();
+        for (int x = threadIdx.x; x < (1 << nhi); x += EQ_BATCH_THREADS) hi_t[x] = eq_product(r_sh, omr_sh, nhi, x);
+        for (int x = threadIdx.x; x < (1 << nlo); x += EQ_BATCH_THREADS) lo_t[x] = eq_product(r_sh + nhi, omr_sh + nhi, nlo, x);
+        __syncthreads();
+    }
     const uint32_t mask = (1u << nlo) - 1;
 
     const int64_t q1 = min(q0 + EQ_SLICE_QUADS, (cover + 3) / 4);
@@ -122,8 +125,11 @@ __global__ void __launch_bounds__(EQ_BATCH_THREADS) eq_batch_kernel(const EqTask
 #pragma unroll
         for (int v = 0; v < 4; v++) {
             const int64_t i = i0 + v;
-            const uint64_t e = i < total ? gl::mul(hi_t[i >> nlo], lo_t[(uint32_t)i & mask]) : 0;
-            if (i < total) tk.out[i] = e;
+            uint64_t e = 0;
+            if (i < total) {
+                if (from_table) e = tk.given[i];
+                else { e = gl::mul(hi_t[i >> nlo], lo_t[(uint32_t)i & mask]); tk.out[i] = e; }
+            }
             w[v] = i < tk.extent ? e : 0;
             slice_sum = gl::add(slice_sum, w[v]);
         }

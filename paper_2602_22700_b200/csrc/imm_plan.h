@@ -86,6 +86,8 @@ struct EqTask {
     int32_t extent;
     int32_t pad_;
     imm_fe* slice_sums;        // one entry per block of the task: sum of its entries below `extent` (or null)
+    const imm_fe* given;       // non-null: the table exists already (`extent` entries are read from here, nothing
+                               // is derived or written to `out`); only the limb tables and slice sums are produced
 };
 
 // A single eq table with r supplied by the caller (passed by value to the kernel).

@@ -2,7 +2,7 @@
 """Throughput of the sumcheck matmul prover on synthetic transformer-shaped layers.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--config decoder|qkv|ffn|moe] [--layers L] [--tokens T] [--no-e2e] [--no-cpu-baseline]
+                    [--config decoder|qkv|ffn|moe|attn|ldd] [--layers L] [--tokens T] [--no-e2e] [--no-cpu-baseline]
 
 One step = one proving pass over the whole batch: eq tables, A~ / B~ partial evaluations, the
 claim C~, every sumcheck round, transcripts written.  The default workload is the audited decoder
@@ -65,12 +65,15 @@ WORKLOADS = {
     "qkv": (512, "dense-layer projection: A {tokens}x4096 times W 4096x4096, one proof"),
     "ffn": (2048, "dense FFN up/down pair: {tokens}x4096 times 4096x14336, requantised hidden times 14336x4096, two proofs"),
     "moe": (4096, "MoE expert batch: 8 experts 4096x14336, top-2 routing of {tokens} tokens, one proof per expert"),
+    "attn": (2048, "attention products: {layers} layers x 32 heads x (Q K^T with k = 128, P V with k = {tokens}), {tokens} tokens, one proof per product"),
     "ldd": (8192, "logit distance distribution: {tokens} decision steps x vocabulary {vocab} (float32), TV + KL + Top-{topk} distance + tail statistic"),
 }
 L2_BYTES = 126 << 20
 
 
 def workload_name(config, layers, tokens, vocab=128256, topk=20):
+    if config == "attn":
+        layers = min(layers, 8)
     return WORKLOADS[config][1].format(layers=layers, tokens=tokens, vocab=vocab, topk=topk)
 
 
@@ -82,6 +85,8 @@ def make_problems(config, seed, layers, tokens, device):
         return synth.qkv_projection(seed, tokens, device=device)
     if config == "ffn":
         return synth.ffn_pair(seed, tokens, device=device)
+    if config == "attn":
+        return synth.attention_block(seed, min(layers, 8), tokens, device=device)
     return synth.moe_experts(seed, tokens, device=device)
 
 
@@ -292,7 +297,7 @@ def run_ours(args):
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "u64", "data": "synthetic",
         "config": {"workload": workload_name(args.config, args.layers, args.tokens),
-                   "layers": args.layers if args.config == "decoder" else None,
+                   "layers": args.layers if args.config == "decoder" else min(args.layers, 8) if args.config == "attn" else None,
                    "tokens": args.tokens, "proofs_per_gpu": len(problems), "field": "Goldilocks 2^64-2^32+1",
                    "input_bytes_per_gpu": algo_bytes,
                    "l2": ("L2 flushed between steps (512 MB overwritten outside the timed event pairs)" if flush else

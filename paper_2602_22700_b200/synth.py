@@ -244,6 +244,28 @@ def decoder_block(seed: int = 1, layers: int = 32, tokens: int = 8192, d_model: 
     return out
 
 
+ROLE_Q, ROLE_KT, ROLE_P, ROLE_V = 9, 10, 11, 12
+
+
+def attention_block(seed: int = 1, layers: int = 8, tokens: int = 2048, heads: int = 32, head_dim: int = 128,
+                    device="cpu") -> List[Problem]:
+    """The two matrix products inside attention, per layer and head: scores S = Q K^T (k = head_dim,
+    C is tokens x tokens) and outputs O = P V (k = tokens).  K is generated already transposed
+    (head_dim x tokens); P is an independent int8 stand-in for the requantised probabilities (the
+    softmax between the two products is not part of what is proved).  proof_id counts the products."""
+    out = []
+    for layer in range(layers):
+        for h in range(heads):
+            g = layer * heads + h
+            Q = gauss_i8(seed, tid(g, ROLE_Q), tokens, head_dim, Q_SIGMA20, device)
+            Kt = gauss_i8(seed, tid(g, ROLE_KT), head_dim, tokens, Q_SIGMA20, device)
+            out.append(Problem(f"L{layer}.h{h}.qk", Q, Kt, exact_matmul_i32(Q, Kt), 2 * g))
+            P = gauss_i8(seed, tid(g, ROLE_P), tokens, tokens, Q_SIGMA20, device)
+            V = gauss_i8(seed, tid(g, ROLE_V), tokens, head_dim, Q_SIGMA20, device)
+            out.append(Problem(f"L{layer}.h{h}.pv", P, V, exact_matmul_i32(P, V), 2 * g + 1))
+    return out
+
+
 def problem_bytes(problems: List[Problem]) -> int:
     """Algorithmic HBM bytes of one proving pass: every input element read exactly once."""
     return sum(p.A.numel() + p.B.numel() + 4 * p.C.numel() for p in problems)

@@ -104,6 +104,19 @@ def test_moe_expert_batch_ragged(imm, oracle, synth):
         assert imm.sumcheck_verify(t, 12, SEED, p.proof_id) == (imm.OK, -1)
 
 
+def test_attention_products_many_small_proofs(imm, oracle, synth):
+    """Scores (k = head_dim: few rounds, a large claimed matrix) and outputs (k = tokens) of 2 layers x
+    4 heads in one batch: 16 proofs, every transcript against the oracle."""
+    probs = synth.attention_block(SEED, layers=2, tokens=640, heads=4, head_dim=128, device="cuda")
+    assert len(probs) == 16 and probs[0].mkn == (640, 128, 640) and probs[1].mkn == (640, 640, 128)
+    check_sampled_entries_of_C(probs[3], np.random.default_rng(6), 16)
+    got = gpu_transcripts(imm, probs, SEED)
+    assert got == oracle_transcripts(oracle, probs, SEED)
+    assert len(got[0]) == 3 * 7 + 3 and len(got[1]) == 3 * 10 + 3
+    for t, p in zip(got, probs):
+        assert imm.sumcheck_verify(t, oracle.ceil_log2(p.mkn[1]), SEED, p.proof_id) == (imm.OK, -1)
+
+
 def two_sided(oracle, M, r_row, r_col):
     return oracle.mle_eval_point(M, oracle.eq_table(r_row), oracle.eq_table(r_col))
 

@@ -206,20 +206,18 @@ CLAIM_KERNEL_TRAFFIC_RATIO = 240.14 / 234.881024  # bytedot_kernel<1,1,1>, per-w
 
 def run_ours(args):
     from paper_2602_22700_b200 import imm, synth
+    from paper_2602_22700_b200.replicas import Replicas
     rank, local_rank, world = dist_env()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the prover has no CPU path")
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
+    rep = Replicas("nccl", dev)
     imm.lib()
     warmup = max(args.warmup, 3)
     steps = max(args.steps, 1)
 
-    problems = make_problems(args.config, SEED + rank, args.layers, args.tokens, dev)
+    problems = make_problems(args.config, rep.seed(SEED), args.layers, args.tokens, dev)
     shapes = [p.mkn for p in problems]
     macs = synth.prover_field_macs(problems)
     algo_bytes = synth.problem_bytes(problems)
@@ -227,11 +225,7 @@ def run_ours(args):
     prover = imm.Prover([(p.A, p.B, p.C, p.proof_id) for p in problems], device=dev)
     imm.profile_enable(min(4096, warmup + steps + 4))
 
-    def barrier():
-        torch.cuda.synchronize()
-        if dist is not None:
-            dist.barrier()
-            torch.cuda.synchronize()
+    barrier = rep.barrier
 
     for _ in range(warmup):
         prover.prove(SEED)
@@ -265,10 +259,7 @@ def run_ours(args):
         elapsed_ms = ev0.elapsed_time(ev1)
     t1 = time.time()
     clocks = sampler.stop(t0, t1)
-    if dist is not None:
-        t = torch.tensor([elapsed_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(t.item())
+    elapsed_ms = rep.max_over_ranks(elapsed_ms)
     phase_ms = [0.0] * len(imm.PROFILE_PHASES)
     for c in range(first_call, first_call + steps):
         for i, v in enumerate(imm.profile_read(c)):
@@ -340,10 +331,7 @@ def run_ours(args):
             for _ in range(k2):
                 hp.prove(SEED)                               # synchronous: returns after the D2H copy
             e2e_s = (time.perf_counter() - w0) / k2
-            if dist is not None:
-                t = torch.tensor([e2e_s], dtype=torch.float64, device=dev)
-                dist.all_reduce(t, op=dist.ReduceOp.MAX)
-                e2e_s = float(t.item())
+            e2e_s = rep.max_over_ranks(e2e_s)
             same = bool((hp.transcripts == host_t).all())
             e2e = {"value": macs * world / e2e_s, "unit": UNIT, "ms_per_step": e2e_s * 1e3, "steps": k2,
                    "h2d_bytes_per_step": hp.h2d_bytes, "d2h_bytes_per_step": hp.d2h_bytes,
@@ -368,8 +356,7 @@ def run_ours(args):
             raise SystemExit("GPU transcripts differ from the oracle on the sampled proofs")
     if rank == 0:
         print(json.dumps(out))
-    if dist is not None:
-        dist.destroy_process_group()
+    rep.close()
 
 
 # ------------------------------------------------------------------------ logit distance distribution
@@ -390,30 +377,24 @@ def run_ldd(args):
     """One step = every decision step's TV and KL distance, its Top-K distance, and the per-request
     tail statistic.  Not the headline workload: a second data-parallel path of the same audit."""
     from paper_2602_22700_b200 import imm, synth
+    from paper_2602_22700_b200.replicas import Replicas
     rank, local_rank, world = dist_env()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
+    rep = Replicas("nccl", dev)
     imm.lib()
     warmup, steps = max(args.warmup, 3), max(args.steps, 1)
     T, n, K = args.tokens, args.vocab, args.topk
-    ref = synth.reference_logits(SEED + rank, T, n, device=dev)
-    dep = synth.deployed_logits(ref, SEED + rank, synth.NOISE_QUANTISED)
+    ref = synth.reference_logits(rep.seed(SEED), T, n, device=dev)
+    dep = synth.deployed_logits(ref, rep.seed(SEED), synth.NOISE_QUANTISED)
     topk = torch.topk(dep, K, dim=1).indices.to(torch.int32).contiguous()      # what the server committed to
-    offsets = synth.request_offsets(SEED + rank, T, max(1, T // 256), device=dev)
+    offsets = synth.request_offsets(rep.seed(SEED), T, max(1, T // 256), device=dev)
     t1, t2 = 0.1, 0.02
     bytes_tvkl, bytes_topk = 8 * T * n, 4 * T * n
 
-    def barrier():
-        torch.cuda.synchronize()
-        if dist is not None:
-            dist.barrier()
-            torch.cuda.synchronize()
+    barrier = rep.barrier
 
     def one_pass(ev=None):
         if ev:
@@ -444,10 +425,7 @@ def run_ldd(args):
     t1w = time.time()
     clocks = sampler.stop(t0, t1w)
     elapsed_ms = evs[0][0].elapsed_time(evs[-1][3])
-    if dist is not None:
-        t = torch.tensor([elapsed_ms], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        elapsed_ms = float(t.item())
+    elapsed_ms = rep.max_over_ranks(elapsed_ms)
     ms_per_step = elapsed_ms / steps
     ph = [sum(e[i].elapsed_time(e[i + 1]) for e in evs) / steps for i in range(3)]
     tv, kl, d, st, p, flag = out
@@ -498,6 +476,7 @@ def run_ldd(args):
         for _ in range(k2):
             e2e_pass()
         e2e_s = (time.perf_counter() - w0) / k2
+        e2e_s = rep.max_over_ranks(e2e_s)
         e2e = {"value": T * world / e2e_s, "unit": "steps/s", "ms_per_step": e2e_s * 1e3, "steps": k2,
                "h2d_bytes_per_step": hd.numel() * 4 + hr.numel() * 4 + hk.numel() * 4, "d2h_bytes_per_step": 3 * T * 8,
                "matches_device_path": bool((outs[0].to(dev) == tv).all() and (outs[2].to(dev) == d).all())}
@@ -520,8 +499,7 @@ def run_ldd(args):
             raise SystemExit("GPU distances differ from the oracle beyond the tolerance")
     if rank == 0:
         print(json.dumps(res))
-    if dist is not None:
-        dist.destroy_process_group()
+    rep.close()
 
 
 # ------------------------------------------------------------------------ reference arm (CPU oracle)

@@ -795,7 +795,11 @@ cudaError_t launch_rowmma(const MatJob* d_jobs, int njobs, uint32_t ntiles, int 
 {
     if (ntiles == 0) return cudaSuccess;
     if (warps < 1 || warps > ROWMMA_MAX_WARPS) return cudaErrorInvalidValue;
-    rowmma_kernel<<<ntiles, 32 * warps, 0, st>>>(d_jobs, njobs);
+    const size_t smem = (size_t)warps * ROWLDM_STAGES * ROWLDM_STAGE_BYTES;         // 18 KiB per warp
+    cudaError_t e = cudaFuncSetAttribute(rowmma_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         ROWMMA_MAX_WARPS * ROWLDM_STAGES * ROWLDM_STAGE_BYTES);
+    if (e != cudaSuccess) return e;
+    rowmma_kernel<<<ntiles, 32 * warps, smem, st>>>(d_jobs, njobs);
     return cudaGetLastError();
 }
 

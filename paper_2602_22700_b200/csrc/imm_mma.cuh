@@ -386,12 +386,105 @@ __device__ __forceinline__ void rowmma_tile(const MatJob& job, uint32_t local, u
         }
 }
 
+// Aligned rows: the byte transpose moves from the integer pipe (64 byte-permutes per 128 loaded
+// bytes: the kernel above is bound by them) into the load path.  A warp streams its 128 columns
+// through a ring of shared-memory stages with 16-byte asynchronous copies (a stage = 32 rows x
+// 128 bytes, rows padded to 144 bytes so that ldmatrix is conflict-free); `ldmatrix ... .trans .b8`
+// then delivers 16 x 16 byte blocks transposed, i.e. every register holds one column at four
+// consecutive rows -- exactly the MMA's A fragment with K = rows:
+//   lane 4g+t gets {M[4t..4t+3][g]}, {M[4t..4t+3][g+8]} of rows 0-15 and of rows 16-31  ->  a0..a3.
+// MMA j of a group covers columns 16j..16j+15 of the warp; accumulator rows g / g+8 are columns
+// 16j+g / 16j+g+8.  The ring belongs to the warp, so the loop needs warp barriers only.
+
+__device__ __forceinline__ void cp_async_16(uint32_t smem_dst, const void* src, int src_bytes)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" :: "r"(smem_dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" :: "n"(N) : "memory"); }
+
+__device__ __forceinline__ void ldmatrix_x2_trans_b8(uint32_t (&r)[4], uint32_t smem_row)
+{
+    asm volatile("ldmatrix.sync.aligned.m16n16.x2.trans.shared.b8 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(smem_row));
+}
+
+__device__ __forceinline__ void rowldm_tile(const MatJob& job, uint32_t local, uint2* sR, char* ring_base)
+{
+    const int rbi = local / job.ncc, cci = local % job.ncc;
+    const int r0 = rbi * job.tile_rows;                         // multiple of 32
+    const int r1 = min(r0 + job.tile_rows, job.rows);
+    const int ngroups = (r1 - r0 + 31) / 32;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int g = lane >> 2, t = lane & 3;
+
+    const uint2* wsrc = reinterpret_cast<const uint2*>(job.wtab) + (int64_t)(r0 / 32) * 32;
+    for (int i = threadIdx.x; i < ngroups * 32; i += blockDim.x) sR[i] = wsrc[i];
+    __syncthreads();
+
+    const int tile_cols = (int)blockDim.x * 4;                    // 128 columns per warp
+    const int col0 = cci * tile_cols + warp * 128;                // this warp's first column
+    int32_t acc[8][4];
+#pragma unroll
+    for (int i = 0; i < 8; i++)
+#pragma unroll
+        for (int c = 0; c < 4; c++) acc[i][c] = 0;
+
+    if (col0 < job.cols) {                                        // whole warp in or out
+        const uint32_t ring = (uint32_t)__cvta_generic_to_shared(ring_base) + (uint32_t)warp * ROWLDM_STAGES * ROWLDM_STAGE_BYTES;
+        // this lane's eight 16-byte pieces of a group: piece p = lane + 32 i  ->  row p / 8, bytes 16 (p % 8) ...
+        const int piece_col = col0 + 16 * (lane & 7);
+        const int src_bytes = max(0, min(16, job.cols - piece_col));       // bytes past the last column arrive as zeros
+        const char* src_col = (const char*)job.mat + (src_bytes > 0 ? piece_col : 0);
+        auto issue = [&](int G) {
+            if (G < ngroups) {
+                const uint32_t stage = ring + (uint32_t)(G % ROWLDM_STAGES) * ROWLDM_STAGE_BYTES;
+#pragma unroll
+                for (int i = 0; i < 8; i++) {
+                    const int rr = (lane >> 3) + 4 * i;                              // row of the group
+                    const int row = min(r0 + 32 * G + rr, r1 - 1);                    // clamped; its weight is 0 past r1
+                    cp_async_16(stage + (uint32_t)rr * ROWLDM_PITCH + 16u * (lane & 7), src_col + (int64_t)row * job.ld, src_bytes);
+                }
+            }
+            cp_async_commit();                                        // (an empty group keeps the count uniform)
+        };
+#pragma unroll
+        for (int s = 0; s < ROWLDM_STAGES - 1; s++) issue(s);
+        // ldmatrix row address of this lane: matrix lane / 16 (rows 0-15 / 16-31), row lane % 16
+        const uint32_t lrow = (uint32_t)(16 * (lane >> 4) + (lane & 15)) * ROWLDM_PITCH;
+        for (int G = 0; G < ngroups; G++) {
+            issue(G + ROWLDM_STAGES - 1);
+            cp_async_wait<ROWLDM_STAGES - 1>();                       // this lane's pieces of group G have landed
+            __syncwarp();                                             // ... and every other lane's
+            const uint32_t stage = ring + (uint32_t)(G % ROWLDM_STAGES) * ROWLDM_STAGE_BYTES;
+            const uint2 wb = sR[G * 32 + lane];
+#pragma unroll
+            for (int jb = 0; jb < 8; jb++) {
+                uint32_t a[4];
+                ldmatrix_x2_trans_b8(a, stage + lrow + 16u * jb);
+                mma_m16n8k32<true>(acc[jb], a[0], a[1], a[2], a[3], wb.x, wb.y);
+            }
+            __syncwarp();                                             // the stage may be refilled from the next iteration on
+        }
+    }
+#pragma unroll
+    for (int jb = 0; jb < 8; jb++)
+#pragma unroll
+        for (int h = 0; h < 2; h++) {
+            uint64_t v = combine_limbs(acc[jb][2 * h], acc[jb][2 * h + 1], t);
+            const int c = col0 + 16 * jb + g + 8 * h;
+            if (t == 0 && c < job.cols) job.out[(int64_t)rbi * job.cols + c] = v;
+        }
+}
+
 __global__ void __launch_bounds__(ROWMMA_MAX_WARPS * 32) rowmma_kernel(const MatJob* jobs, int njobs)
 {
     __shared__ uint2 sR[MAX_TILE_ROWS];                             // (MAX_TILE_ROWS / 32) groups x 32 lanes
+    extern __shared__ __align__(128) char ring[];                   // warps x stages x (32 rows x 144 bytes)
     const MatJob job = jobs[find_job(jobs, njobs, blockIdx.x)];
     const uint32_t local = blockIdx.x - job.tile0;
-    if (job.vec) rowmma_tile<true>(job, local, sR);
+    if (job.vec) rowldm_tile(job, local, sR, ring);
     else rowmma_tile<false>(job, local, sR);
 }
 

@@ -29,6 +29,9 @@ constexpr int BYTEDOT_MAX_CHUNK_BYTES = IMM_BYTEDOT_MAX_CHUNK_BYTES;  // most by
                                                                      // chunk is a multiple of 256 up to this
 constexpr int BYTEDOT_UNROLL = IMM_BYTEDOT_UNROLL;            // slabs of 256 byte-columns in flight per warp
 constexpr int ROWMMA_MAX_WARPS = 8;            // a block of w warps covers w x 128 int8 columns
+constexpr int ROWLDM_STAGES = 4;               // shared-memory stages per warp of the row-binding kernel
+constexpr int ROWLDM_PITCH = 144;              // bytes per staged row: 128 of data, 16 of padding
+constexpr int ROWLDM_STAGE_BYTES = 32 * ROWLDM_PITCH;
 constexpr int EQ_BATCH_THREADS = 256;
 constexpr int EQ_SLICE_QUADS = 512;           // groups of four table entries per block of eq_batch_kernel
 constexpr int SUMCHECK_THREADS = 512;

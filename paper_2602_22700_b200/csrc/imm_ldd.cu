@@ -468,6 +468,156 @@ topk_merge_kernel(const float* __restrict__ ref, int64_t n, int64_t ld, const in
 }
 
 // ------------------------------------------------------------------------------------------
+// short rows: one warp per row
+// ------------------------------------------------------------------------------------------
+// Expert routing (n = 64...256 logits per decision, K = 2...8) has millions of short rows: a
+// cluster per row would spend its time on launch and barriers.  Up to SMALL_N entries a warp
+// takes a whole row: lane l holds entries l, l + 32, ... in registers, everything else is warp
+// shuffles.  The same arithmetic as the long-row kernels (float32 terms, float64 final sums and
+// costs), so the same tolerances hold.
+
+constexpr int SMALL_N = 1024;
+constexpr int SMALL_SLOTS = SMALL_N / 32;
+constexpr int SMALL_WARPS = 8;                // rows per block
+
+__device__ __forceinline__ float warp_max(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
+    return v;
+}
+__device__ __forceinline__ float warp_add(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+
+template <int SLOTS>
+__global__ void __launch_bounds__(SMALL_WARPS * 32)
+tv_kl_small_kernel(const float* __restrict__ logits, const float* __restrict__ ref, int64_t steps, int n, int64_t ld,
+                   double* __restrict__ tv_out, double* __restrict__ kl_out)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t step = (int64_t)blockIdx.x * SMALL_WARPS + (threadIdx.x >> 5);
+    if (step >= steps) return;                         // (whole warp)
+    const float* x = logits + step * ld;
+    const float* y = ref + step * ld;
+    float xs[SLOTS], ys[SLOTS];
+    float mx = NEG_INF, my = NEG_INF;
+#pragma unroll
+    for (int j = 0; j < SLOTS; j++) {
+        const int e = lane + 32 * j;
+        xs[j] = e < n ? x[e] : NEG_INF;
+        ys[j] = e < n ? y[e] : NEG_INF;
+        mx = fmaxf(mx, xs[j]); my = fmaxf(my, ys[j]);
+    }
+    mx = warp_max(mx); my = warp_max(my);
+    float sx = 0.f, sy = 0.f;
+#pragma unroll
+    for (int j = 0; j < SLOTS; j++) {                  // slots past the end hold -inf: they add 0
+        sx += ex2((xs[j] - mx) * LOG2E);
+        sy += ex2((ys[j] - my) * LOG2E);
+    }
+    const float lp = log2f(warp_add(sx)), lq = log2f(warp_add(sy));
+    const float dl = (lq - lp) * (1.0f / LOG2E);
+    float tv = 0.f, kl = 0.f;
+#pragma unroll
+    for (int j = 0; j < SLOTS; j++) {
+        if (lane + 32 * j < n) {
+            const float xr = xs[j] - mx, yr = ys[j] - my;
+            const float p = ex2(fmaf(xr, LOG2E, -lp)), q = ex2(fmaf(yr, LOG2E, -lq));
+            tv += fabsf(p - q);
+            kl = fmaf(q, (yr - xr) - dl, kl);
+        }
+    }
+    double dtv = (double)tv, dkl = (double)kl;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        dtv += __shfl_xor_sync(0xFFFFFFFFu, dtv, o);
+        dkl += __shfl_xor_sync(0xFFFFFFFFu, dkl, o);
+    }
+    if (lane == 0) { tv_out[step] = 0.5 * dtv; kl_out[step] = dkl; }
+}
+
+// Top-K distance of a short row.  The K largest entries outside I are pulled out one at a time
+// (K warp-wide arg-max rounds over the registers); the cost is then evaluated at the 2K
+// breakpoints in float64, as in the long-row kernel.
+template <int SLOTS>
+__global__ void __launch_bounds__(SMALL_WARPS * 32)
+topk_small_kernel(const float* __restrict__ ref, int64_t steps, int n, int64_t ld, const int32_t* __restrict__ topk, int K,
+                  double* __restrict__ dist_out, int32_t* __restrict__ status)
+{
+    __shared__ float outside[SMALL_WARPS][MAX_K], inside[SMALL_WARPS][MAX_K];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int64_t step = (int64_t)blockIdx.x * SMALL_WARPS + w;
+    if (step >= steps) return;                         // (whole warp)
+    const float* y = ref + step * ld;
+    const int32_t* I = topk + step * K;
+    float v[SLOTS];
+#pragma unroll
+    for (int j = 0; j < SLOTS; j++) {
+        const int e = lane + 32 * j;
+        v[j] = e < n ? y[e] : NEG_INF;
+    }
+    // the entries of I: remember their values, then take them out of the running
+    bool bad = false;
+    uint32_t mine = 0;                                 // bit j: this lane's slot j belongs to I
+    for (int k = 0; k < K; k++) {
+        const int idx = I[k];
+        if (idx < 0 || idx >= n) { bad = true; continue; }
+        if ((idx & 31) == lane) {
+            const uint32_t bit = 1u << (idx >> 5);
+            if (mine & bit) bad = true;                // the same index twice
+            mine |= bit;
+        }
+    }
+    bad = __any_sync(0xFFFFFFFFu, bad);
+    for (int k = lane; k < K; k += 32) {
+        const int idx = I[k];
+        inside[w][k] = (idx >= 0 && idx < n) ? y[idx] : 0.f;
+    }
+#pragma unroll
+    for (int j = 0; j < SLOTS; j++) if ((mine >> j) & 1u) v[j] = NEG_INF;
+    for (int r = 0; r < K; r++) {
+        float best = NEG_INF;
+        int slot = 0;
+#pragma unroll
+        for (int j = 0; j < SLOTS; j++) if (v[j] > best) { best = v[j]; slot = j; }
+        const float top = warp_max(best);
+        const unsigned holders = __ballot_sync(0xFFFFFFFFu, best == top);
+        const int winner = __ffs(holders) - 1;         // lowest lane holding the maximum
+        if (lane == winner) {
+            outside[w][r] = top;                       // (-inf once fewer than K entries are left outside I)
+#pragma unroll
+            for (int j = 0; j < SLOTS; j++) if (j == slot) v[j] = NEG_INF;
+        }
+    }
+    __syncwarp();
+    double best_cost = INFINITY;
+    for (int cnd = lane; cnd < 2 * K; cnd += 32) {
+        const double t = cnd < K ? (double)outside[w][cnd] : (double)inside[w][cnd - K];
+        if (t > -INFINITY) {
+            double c = 0.0;
+            for (int k = 0; k < K; k++) {
+                c += fmax((double)outside[w][k] - t, 0.0);
+                c += fmax(t - (double)inside[w][k], 0.0);
+            }
+            best_cost = fmin(best_cost, c);
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) best_cost = fmin(best_cost, __shfl_xor_sync(0xFFFFFFFFu, best_cost, o));
+    if (lane == 0) {
+        dist_out[step] = bad ? NAN : best_cost;
+        status[step] = bad ? IMM_ERR_ARG : IMM_OK;
+    }
+}
+
+// slots per lane a row of n entries needs, rounded to the instantiated sizes
+inline int small_slots(int64_t n) { return n <= 128 ? 4 : n <= 256 ? 8 : n <= 512 ? 16 : 32; }
+
+// ------------------------------------------------------------------------------------------
 // per-request tail statistic
 // ------------------------------------------------------------------------------------------
 // p[r] = |{ steps of request r with distance > t1 }| / (steps of request r);  flag[r] = p[r] > t2.
@@ -535,9 +685,19 @@ int imm_ldd_tv_kl(const float* d_logits, const float* d_ref_logits, int64_t step
     if (steps < 0 || n <= 0 || ld < n || n > IMM_LDD_MAX_N || steps > IMM_LDD_MAX_STEPS) return IMM_ERR_SHAPE;
     if ((uintptr_t)d_logits % 4 || (uintptr_t)d_ref_logits % 4 || (uintptr_t)d_tv % 8 || (uintptr_t)d_kl % 8) return IMM_ERR_ALIGN;
     if (steps == 0) return IMM_OK;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (n <= SMALL_N) {                                // short rows: one warp per row
+        const unsigned grid = (unsigned)((steps + SMALL_WARPS - 1) / SMALL_WARPS);
+        switch (small_slots(n)) {
+        case 4: tv_kl_small_kernel<4><<<grid, SMALL_WARPS * 32, 0, st>>>(d_logits, d_ref_logits, steps, (int)n, ld, d_tv, d_kl); break;
+        case 8: tv_kl_small_kernel<8><<<grid, SMALL_WARPS * 32, 0, st>>>(d_logits, d_ref_logits, steps, (int)n, ld, d_tv, d_kl); break;
+        case 16: tv_kl_small_kernel<16><<<grid, SMALL_WARPS * 32, 0, st>>>(d_logits, d_ref_logits, steps, (int)n, ld, d_tv, d_kl); break;
+        default: tv_kl_small_kernel<32><<<grid, SMALL_WARPS * 32, 0, st>>>(d_logits, d_ref_logits, steps, (int)n, ld, d_tv, d_kl); break;
+        }
+        return cudaGetLastError() == cudaSuccess ? IMM_OK : IMM_ERR_CUDA;
+    }
     const int nc = cluster_size(n);
     const bool vec = rows_aligned(d_logits, ld) && rows_aligned(d_ref_logits, ld);
-    cudaStream_t st = (cudaStream_t)stream;
     // 512 threads and clusters of up to 8 blocks measured best (256 / 1024 threads and 16-block clusters were tried)
     cudaError_t e = vec ? launch_cluster(tv_kl_kernel<true, THREADS>, steps, nc, THREADS, 0, st, d_logits, d_ref_logits, n, ld, d_tv, d_kl)
                         : launch_cluster(tv_kl_kernel<false, THREADS>, steps, nc, THREADS, 0, st, d_logits, d_ref_logits, n, ld, d_tv, d_kl);
@@ -566,6 +726,17 @@ int imm_ldd_topk_distance(const float* d_ref_logits, int64_t steps, int64_t n, i
         return IMM_ERR_ALIGN;
     if (ws_bytes < imm_ldd_topk_workspace(steps, n, k)) return IMM_ERR_WORKSPACE;
     if (steps == 0) return IMM_OK;
+    if (n <= SMALL_N) {                                // short rows: one warp per row, no workspace traffic
+        const unsigned grid = (unsigned)((steps + SMALL_WARPS - 1) / SMALL_WARPS);
+        cudaStream_t sst = (cudaStream_t)stream;
+        switch (small_slots(n)) {
+        case 4: topk_small_kernel<4><<<grid, SMALL_WARPS * 32, 0, sst>>>(d_ref_logits, steps, (int)n, ld, d_topk, k, d_dist, d_status); break;
+        case 8: topk_small_kernel<8><<<grid, SMALL_WARPS * 32, 0, sst>>>(d_ref_logits, steps, (int)n, ld, d_topk, k, d_dist, d_status); break;
+        case 16: topk_small_kernel<16><<<grid, SMALL_WARPS * 32, 0, sst>>>(d_ref_logits, steps, (int)n, ld, d_topk, k, d_dist, d_status); break;
+        default: topk_small_kernel<32><<<grid, SMALL_WARPS * 32, 0, sst>>>(d_ref_logits, steps, (int)n, ld, d_topk, k, d_dist, d_status); break;
+        }
+        return cudaGetLastError() == cudaSuccess ? IMM_OK : IMM_ERR_CUDA;
+    }
     const int64_t nslices = (n + TK_SLICE - 1) / TK_SLICE;
     if (nslices * k > MERGE_CAP || steps * nslices > 0x7FFFFFFF) return IMM_ERR_SHAPE;     // (cannot happen within the limits)
     cudaStream_t st = (cudaStream_t)stream;

@@ -49,7 +49,8 @@ def check_tv_kl(imm, ldd, x, y):
         assert abs(kl[i] - want_kl) <= KL_ABS + KL_REL * abs(want_kl), (i, kl[i], want_kl)
 
 
-@pytest.mark.parametrize("steps,n", [(7, 1), (5, 3), (9, 100), (4, 4097), (3, 16384), (3, 16388), (3, 40003),
+@pytest.mark.parametrize("steps,n", [(7, 1), (5, 3), (9, 100), (19, 64), (9, 128), (5, 256), (4, 1000), (3, 1024), (3, 1025),
+                                     (4, 4097), (3, 16384), (3, 16388), (3, 40003),
                                      (2, 128256), (2, 151936), (1, 300000)])
 @pytest.mark.parametrize("noise", ["benign", "quantised", "substituted"])
 def test_tv_kl_matches_oracle(imm, ldd, synth, steps, n, noise):
@@ -86,6 +87,20 @@ def test_tv_kl_unaligned_rows_take_the_element_path(imm, ldd, synth):
     check_tv_kl(imm, ldd, odd(dep, n + 7, 0), odd(ref, n + 7, 0))      # aligned base, unaligned pitch
 
 
+def test_short_rows_with_a_row_pitch(imm, ldd, synth):
+    """Expert-routing shapes (one warp per row), rows not contiguous in memory."""
+    steps, n, k = 37, 128, 8
+    ref = synth.reference_logits(11, steps, n, device="cuda")
+    dep = synth.deployed_logits(ref, 11, synth.NOISE_QUANTISED)
+    buf_r = torch.zeros((steps, n + 5), dtype=torch.float32, device="cuda")
+    buf_d = torch.zeros((steps, n + 5), dtype=torch.float32, device="cuda")
+    buf_r[:, :n] = ref
+    buf_d[:, :n] = dep
+    check_tv_kl(imm, ldd, buf_d[:, :n], buf_r[:, :n])
+    top = torch.topk(dep, k, dim=1).indices.to(torch.int32).contiguous()
+    check_topk(imm, ldd, buf_r[:, :n], top)
+
+
 def check_topk(imm, ldd, ref, topk, rel=1e-9):
     dist, status = imm.ldd_topk_distance(ref, topk)
     dist, status = dist.cpu().numpy(), status.cpu().numpy()
@@ -97,7 +112,8 @@ def check_topk(imm, ldd, ref, topk, rel=1e-9):
     return dist
 
 
-@pytest.mark.parametrize("steps,n,k", [(6, 5, 2), (6, 64, 6), (5, 128, 8), (4, 1000, 20), (3, 16384, 20),
+@pytest.mark.parametrize("steps,n,k", [(6, 5, 2), (21, 64, 6), (5, 128, 8), (4, 256, 8), (4, 1000, 20), (3, 1024, 64), (3, 1025, 8),
+                                        (3, 16384, 20),
                                         (3, 40003, 20), (3, 128256, 20), (2, 151936, 20), (2, 128256, 64),
                                         (2, 300000, 1)])
 def test_topk_distance_matches_oracle(imm, ldd, synth, steps, n, k):

@@ -1,6 +1,7 @@
 /*
  * imm.h -- C ABI of the B200 (sm_100a) prover for sumcheck proofs of int8 matrix products
- * over the Goldilocks field p = 2^64 - 2^32 + 1.
+ * over the Goldilocks field p = 2^64 - 2^32 + 1, and (last section) of the logit distance
+ * statistics the same audit reports.
  *
  * Background.  The audited-inference protocol this library serves has the server prove, for an
  * audited request, that the "continuous transformations" of the reference model -- its
@@ -174,16 +175,19 @@ size_t imm_sumcheck_matmul_workspace(const imm_matmul_desc* descs_host, int npro
  *   d_status      : DEVICE array of nproofs int32, set to IMM_OK per proof (reserved for
  *                   device-detected conditions)
  *   d_ws          : DEVICE workspace, >= imm_sumcheck_matmul_workspace(...) bytes
- * The whole batch is a fixed sequence of kernel launches on `stream`; results are valid once
- * the stream has been synchronised.
+ * The whole batch is a fixed sequence of five kernel launches ordered after the work already on
+ * `stream`; results are valid once the stream has been synchronised.  For a batch of less than
+ * 2 GiB of matrices the three contractions run side by side on two library-owned streams (created
+ * on the first such call per device) that fork from and join back into `stream`.
  * Errors: IMM_ERR_ARG, IMM_ERR_SHAPE, IMM_ERR_ALIGN, IMM_ERR_WORKSPACE, IMM_ERR_CUDA. */
 int imm_sumcheck_matmul_prove(const imm_matmul_desc* descs_host, int nproofs, uint64_t seed,
                               imm_fe* d_transcripts, int64_t stride, int32_t* d_status,
                               void* d_ws, size_t ws_bytes, void* stream);
 
 /* Phase timing of imm_sumcheck_matmul_prove, for measurement.  While enabled, every prove call
- * records CUDA events on its stream around each of its five launches, into the next of
- * `capacity` event sets (a ring), without synchronising.  Phases:
+ * records a pair of CUDA events around each of its five launches (on the stream the launch runs
+ * on), into the next of `capacity` event sets (a ring), without synchronising.  When the three
+ * contractions run side by side (small batches) their times overlap.  Phases:
  *   [0] eq tables, [1] claim C~ (int32 point contraction), [2] A~ row binding,
  *   [3] B~ column binding, [4] sumcheck rounds.
  * The event ring is per process; profiled calls must not overlap on different host threads.

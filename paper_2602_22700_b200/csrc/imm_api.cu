@@ -7,6 +7,7 @@
 #include <string.h>
 
 #include <algorithm>
+#include <mutex>
 #include <string>
 #include <vector>
 
@@ -337,9 +338,39 @@ Plan make_plan(const imm_matmul_desc* descs, int nproofs)
 }
 
 // phase-timing events (see imm_profile_enable)
-constexpr int PROF_EV = IMM_PROFILE_PHASES + 1;
+constexpr int PROF_EV = 2 * IMM_PROFILE_PHASES;    // a (start, end) pair per phase
 std::vector<cudaEvent_t> g_prof_ev;        // capacity * PROF_EV events, empty when profiling is off
 int64_t g_prof_calls = 0;
+
+// Small batches do not fill the GPU with one contraction at a time: their three contractions (claim,
+// row binding, column binding) are independent and run on three streams.  Two side streams and the
+// fork / join events per device, created on first use.
+constexpr int MAX_DEVICES = 64;
+constexpr int64_t FORK_BELOW_BYTES = (int64_t)2 << 30;       // batches under 2 GiB of matrices fork
+struct SideStreams {
+    bool ready = false;
+    cudaStream_t s[2] = {nullptr, nullptr};
+    cudaEvent_t fork = nullptr, join[2] = {nullptr, nullptr};
+};
+SideStreams g_side[MAX_DEVICES];
+std::mutex g_side_mutex;
+
+SideStreams* side_streams()
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return nullptr;
+    std::lock_guard<std::mutex> lock(g_side_mutex);
+    SideStreams& ss = g_side[dev];
+    if (!ss.ready) {
+        for (int i = 0; i < 2; i++) {
+            if (cudaStreamCreateWithFlags(&ss.s[i], cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+            if (cudaEventCreateWithFlags(&ss.join[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        }
+        if (cudaEventCreateWithFlags(&ss.fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
+        ss.ready = true;
+    }
+    return &ss;
+}
 
 int check_stride(const imm_matmul_desc* descs, int nproofs, int64_t stride)
 {
@@ -568,8 +599,8 @@ int imm_profile_read(int64_t call, float* ms_host, int count)
     const int64_t cap = (int64_t)(g_prof_ev.size() / PROF_EV);
     if (call < 0 || call >= g_prof_calls || call < g_prof_calls - cap) return IMM_ERR_ARG;
     cudaEvent_t* ev = &g_prof_ev[(size_t)(call % cap) * PROF_EV];
-    CU(cudaEventSynchronize(ev[IMM_PROFILE_PHASES]));
-    for (int i = 0; i < IMM_PROFILE_PHASES; i++) CU(cudaEventElapsedTime(&ms_host[i], ev[i], ev[i + 1]));
+    CU(cudaEventSynchronize(ev[PROF_EV - 1]));                  // the end of the last phase: everything before it is done
+    for (int i = 0; i < IMM_PROFILE_PHASES; i++) CU(cudaEventElapsedTime(&ms_host[i], ev[2 * i], ev[2 * i + 1]));
     return IMM_OK;
 }
 
@@ -649,28 +680,46 @@ int imm_sumcheck_matmul_prove(const imm_matmul_desc* descs_host, int nproofs, ui
     const bool prof = !g_prof_ev.empty();
     cudaEvent_t* pev = prof ? &g_prof_ev[(size_t)(g_prof_calls % (int64_t)(g_prof_ev.size() / PROF_EV)) * PROF_EV]
                             : nullptr;
-#define PROF_MARK(i) do { if (prof) CU(cudaEventRecord(pev[i], st)); } while (0)
-    CU(cudaMemcpyAsync(base, hdr.data(), hdr.size(), cudaMemcpyHostToDevice, st));
-    PROF_MARK(0);
-    CU(launch_eq_batch((const EqTask*)(base + p.off_eq), 2 * nproofs, p.max_cover, st));
-    PROF_MARK(1);
-    if (p.mma) {
-        CU(launch_bytedot(true, true, p.mt_c, (const MatJob*)(base + p.off_jobs_c), nproofs, p.tiles_c, st));
-        PROF_MARK(2);
-        CU(launch_rowmma((const MatJob*)(base + p.off_jobs_a), nproofs, p.tiles_a, p.cols_a / 128, st));
-        PROF_MARK(3);
-        CU(launch_bytedot(false, false, p.mt_b, (const MatJob*)(base + p.off_jobs_b), nproofs, p.tiles_b, st));
-    } else {
-        CU(launch_rowbind(IMM_I32, true, (const MatJob*)(base + p.off_jobs_c), nproofs, p.tiles_c, st));
-        PROF_MARK(2);
-        CU(launch_rowbind(IMM_I8, false, (const MatJob*)(base + p.off_jobs_a), nproofs, p.tiles_a, st));
-        PROF_MARK(3);
-        CU(launch_colbind(IMM_I8, (const MatJob*)(base + p.off_jobs_b), nproofs, p.tiles_b, st));
+    // phase i is timed by events 2i (start) and 2i+1 (end), each on the stream its kernel runs on
+#define PROF_MARK(i, stream_) do { if (prof) CU(cudaEventRecord(pev[i], stream_)); } while (0)
+    int64_t batch_bytes = 0;
+    for (int i = 0; i < nproofs; i++) {
+        const imm_matmul_desc& d = descs_host[i];
+        batch_bytes += d.m * d.k + d.k * d.n + 4 * d.m * d.n;
     }
-    PROF_MARK(4);
+    SideStreams* ss = (batch_bytes < FORK_BELOW_BYTES && !getenv("IMM_NO_FORK")) ? side_streams() : nullptr;
+    cudaStream_t st_a = ss ? ss->s[0] : st, st_b = ss ? ss->s[1] : st;
+    CU(cudaMemcpyAsync(base, hdr.data(), hdr.size(), cudaMemcpyHostToDevice, st));
+    PROF_MARK(0, st);
+    CU(launch_eq_batch((const EqTask*)(base + p.off_eq), 2 * nproofs, p.max_cover, st));
+    PROF_MARK(1, st);
+    if (ss) {                                                 // fork: the side streams wait for the eq tables
+        CU(cudaEventRecord(ss->fork, st));
+        CU(cudaStreamWaitEvent(st_a, ss->fork, 0));
+        CU(cudaStreamWaitEvent(st_b, ss->fork, 0));
+    }
+    PROF_MARK(2, st);
+    if (p.mma) CU(launch_bytedot(true, true, p.mt_c, (const MatJob*)(base + p.off_jobs_c), nproofs, p.tiles_c, st));
+    else CU(launch_rowbind(IMM_I32, true, (const MatJob*)(base + p.off_jobs_c), nproofs, p.tiles_c, st));
+    PROF_MARK(3, st);
+    PROF_MARK(4, st_a);
+    if (p.mma) CU(launch_rowmma((const MatJob*)(base + p.off_jobs_a), nproofs, p.tiles_a, p.cols_a / 128, st_a));
+    else CU(launch_rowbind(IMM_I8, false, (const MatJob*)(base + p.off_jobs_a), nproofs, p.tiles_a, st_a));
+    PROF_MARK(5, st_a);
+    PROF_MARK(6, st_b);
+    if (p.mma) CU(launch_bytedot(false, false, p.mt_b, (const MatJob*)(base + p.off_jobs_b), nproofs, p.tiles_b, st_b));
+    else CU(launch_colbind(IMM_I8, (const MatJob*)(base + p.off_jobs_b), nproofs, p.tiles_b, st_b));
+    PROF_MARK(7, st_b);
+    if (ss) {                                                 // join
+        CU(cudaEventRecord(ss->join[0], st_a));
+        CU(cudaEventRecord(ss->join[1], st_b));
+        CU(cudaStreamWaitEvent(st, ss->join[0], 0));
+        CU(cudaStreamWaitEvent(st, ss->join[1], 0));
+    }
+    PROF_MARK(8, st);
     CU(launch_sumcheck((const ProofDev*)(base + p.off_proofs), nproofs, seed, d_transcripts, stride,
                        d_status, p.max_b, env_int("IMM_SC_CLUSTER", 0), st));
-    PROF_MARK(5);
+    PROF_MARK(9, st);
 #undef PROF_MARK
     if (prof) g_prof_calls++;
     return IMM_OK;

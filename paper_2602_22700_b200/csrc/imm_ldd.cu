@@ -477,7 +477,6 @@ topk_merge_kernel(const float* __restrict__ ref, int64_t n, int64_t ld, const in
 // costs), so the same tolerances hold.
 
 constexpr int SMALL_N = 1024;
-constexpr int SMALL_SLOTS = SMALL_N / 32;
 constexpr int SMALL_WARPS = 8;                // rows per block
 
 __device__ __forceinline__ float warp_max(float v)

@@ -195,6 +195,21 @@ def test_audit_statistic_end_to_end(imm, ldd, synth):
     assert 0 < want_p.max() and want_p.min() < 1
 
 
+def test_topk_workspace_is_checked_and_reusable(imm, ldd, synth):
+    steps, n, k = 6, 40000, 20
+    ref = synth.reference_logits(12, steps, n, device="cuda")
+    top = torch.topk(ref, k, dim=1).indices.to(torch.int32).contiguous()
+    need = imm.lib().imm_ldd_topk_workspace(steps, n, k)
+    assert need > 0 and imm.lib().imm_ldd_topk_workspace(steps, n, 65) == 0
+    with pytest.raises(imm.ImmError) as err:
+        imm.ldd_topk_distance(ref, top, workspace=torch.empty(need - 256, dtype=torch.uint8, device="cuda"))
+    assert err.value.code == imm.ERR_WORKSPACE
+    ws = torch.full((need,), 0xAB, dtype=torch.uint8, device="cuda")          # stale contents must not matter
+    d1, s1 = imm.ldd_topk_distance(ref, top, workspace=ws)
+    d2, s2 = imm.ldd_topk_distance(ref, top, workspace=ws)
+    assert (d1 == 0).all() and (d2 == 0).all() and int(s1.abs().max()) == 0 and int(s2.abs().max()) == 0
+
+
 def test_ldd_calls_refuse_bad_arguments(imm, synth):
     ref = synth.reference_logits(1, 2, 64, device="cuda")
     with pytest.raises(ValueError):

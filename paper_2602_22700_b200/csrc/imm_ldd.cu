@@ -222,7 +222,6 @@ tv_kl_kernel(const float* __restrict__ logits, const float* __restrict__ ref, in
 #define IMM_LDD_TK_THREADS 256
 #endif
 constexpr int TK_THREADS = IMM_LDD_TK_THREADS;   // threads per block of the Top-K kernel
-constexpr int TK_WARPS = TK_THREADS / 32;
 constexpr int TK_SLICE = 32 * TK_THREADS;         // entries of a row per block: 32 per thread, in registers
 constexpr int MAX_CAND = 128;                 // group maxima per block (>= 2 * MAX_K)
 constexpr int MERGE_CAP = (IMM_LDD_MAX_N / TK_SLICE) * MAX_K;   // a row's lists, held at once by the merging block
@@ -319,9 +318,10 @@ topk_slice_kernel(const float* __restrict__ ref, int64_t n, int64_t ld, const in
     for (int j = 0; j < PER; j++) best = fmaxf(best, vals[j]);
     const float thread_best = best;                    // (before the group reduction below)
 
-    // group maxima: ncand = the smallest power of two >= 2K (at least one group per warp)
-    int ncand = TK_WARPS;
-    while (ncand < 2 * K) ncand <<= 1;
+    // group maxima: ncand groups, the smallest power of two (32 at least) above K + m, so that the
+    // bound's rank K + m - 1 exists; fewer groups make the ranking below cheaper
+    int ncand = 32;
+    while (ncand <= K + members) ncand <<= 1;          // <= MAX_CAND
     static_assert(MAX_CAND >= 2 * MAX_K && MAX_CAND <= TK_THREADS, "group maxima must fit the block");
     const int G = TK_THREADS / ncand;
     for (int o = 1; o < G; o <<= 1) best = fmaxf(best, __shfl_xor_sync(0xFFFFFFFFu, best, o));

@@ -269,8 +269,14 @@ Plan make_plan(const imm_matmul_desc* descs, int nproofs)
         // tiles per SM aimed at, from sweeps over 1024...16384 tokens: the row-binding kernel (a
         // warp streams its own 128 columns) needs fewer, larger tiles than the byte-dot kernels
         const Geom ga = pick_geom(sa, rows_a, 6, widths_a, 4, 12, "IMM_TILE_ROWS_A", "IMM_TILE_COLS_A");
-        const Geom gb = pick_geom(sb, rows_b, 1, chunks, 5, 24, "IMM_TILE_ROWS_B", "IMM_CHUNK_B");
-        const Geom gc = pick_geom(scb, rows_c, 4, chunks, 5, 24, "IMM_TILE_ROWS_C", "IMM_CHUNK_C");
+        // ... and a short launch (a few hundred MB) runs best on few, larger tiles: 4 per SM below
+        // 256 MB, one more per 64 MB, 24 from 1.5 GB on
+        int64_t bytes_b = 0, bytes_c = 0;
+        for (const Shape& s : sb) bytes_b += s.rows * s.cols;
+        for (const Shape& s : scb) bytes_c += s.rows * s.cols;
+        auto per_sm = [](int64_t bytes) { int64_t t = bytes >> 26; return (int)(t < 4 ? 4 : t > 24 ? 24 : t); };
+        const Geom gb = pick_geom(sb, rows_b, 1, chunks, 5, per_sm(bytes_b), "IMM_TILE_ROWS_B", "IMM_CHUNK_B");
+        const Geom gc = pick_geom(scb, rows_c, 4, chunks, 5, per_sm(bytes_c), "IMM_TILE_ROWS_C", "IMM_CHUNK_C");
         p.rows_a = ga.rows; p.cols_a = ga.width;
         p.rows_b = gb.rows; p.cols_b = gb.width;
         p.rows_c = gc.rows; p.cols_c = gc.width / 4;

@@ -359,7 +359,8 @@ struct SideStreams {
     cudaEvent_t fork = nullptr, join[2] = {nullptr, nullptr};
 };
 SideStreams g_side[MAX_DEVICES];
-std::mutex g_side_mutex;
+std::mutex g_side_mutex;        // guards the creation of the side streams
+std::mutex g_fork_mutex;        // held while one call enqueues its fork ... join: the events are shared
 
 SideStreams* side_streams()
 {
@@ -695,6 +696,11 @@ int imm_sumcheck_matmul_prove(const imm_matmul_desc* descs_host, int nproofs, ui
     }
     SideStreams* ss = (batch_bytes < FORK_BELOW_BYTES && !getenv("IMM_NO_FORK")) ? side_streams() : nullptr;
     cudaStream_t st_a = ss ? ss->s[0] : st, st_b = ss ? ss->s[1] : st;
+    // Host threads proving on different streams share the side streams and their events: one call
+    // at a time enqueues its fork ... join (a wait refers to the record that precedes it, so a later
+    // call's records do not disturb the waits already enqueued).
+    std::unique_lock<std::mutex> fork_lock;
+    if (ss) fork_lock = std::unique_lock<std::mutex>(g_fork_mutex);
     CU(cudaMemcpyAsync(base, hdr.data(), hdr.size(), cudaMemcpyHostToDevice, st));
     PROF_MARK(0, st);
     CU(launch_eq_batch((const EqTask*)(base + p.off_eq), 2 * nproofs, p.max_cover, st));

@@ -403,6 +403,7 @@ topk_merge_kernel(const float* __restrict__ ref, int64_t n, int64_t ld, const in
     __shared__ float all[MERGE_CAP + MAX_K];
     __shared__ float heads[2 * MAX_K + IMM_LDD_MAX_N / TK_SLICE];
     __shared__ float top[MAX_K], inside[MAX_K];
+    __shared__ double top_d[MAX_K], inside_d[MAX_K];       // converted once: float -> double conversions are slow
     __shared__ double cost[2 * MAX_K];
     __shared__ float bound;
     __shared__ int bad, count;
@@ -441,14 +442,16 @@ topk_merge_kernel(const float* __restrict__ ref, int64_t n, int64_t ld, const in
         if (r < K) top[r] = all[i];
     }
     __syncthreads();
+    if (tid < K) { top_d[tid] = (double)top[tid]; inside_d[tid] = (double)inside[tid]; }
+    __syncthreads();
     if (tid < 2 * K) {
-        const double t = tid < K ? (double)top[tid] : (double)inside[tid - K];
+        const double t = tid < K ? top_d[tid] : inside_d[tid - K];
         double c = INFINITY;
         if (t > -INFINITY) {                               // a row with fewer than K entries outside I pads with -inf
             c = 0.0;
             for (int k = 0; k < K; k++) {
-                c += fmax((double)top[k] - t, 0.0);
-                c += fmax(t - (double)inside[k], 0.0);
+                c += fmax(top_d[k] - t, 0.0);
+                c += fmax(t - inside_d[k], 0.0);
             }
         }
         cost[tid] = c;
@@ -547,7 +550,7 @@ __global__ void __launch_bounds__(SMALL_WARPS * 32)
 topk_small_kernel(const float* __restrict__ ref, int64_t steps, int n, int64_t ld, const int32_t* __restrict__ topk, int K,
                   double* __restrict__ dist_out, int32_t* __restrict__ status)
 {
-    __shared__ float outside[SMALL_WARPS][MAX_K], inside[SMALL_WARPS][MAX_K];
+    __shared__ double outside[SMALL_WARPS][MAX_K], inside[SMALL_WARPS][MAX_K];   // as doubles: converted once
     const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
     const int64_t step = (int64_t)blockIdx.x * SMALL_WARPS + w;
     if (step >= steps) return;                         // (whole warp)
@@ -574,7 +577,7 @@ topk_small_kernel(const float* __restrict__ ref, int64_t steps, int n, int64_t l
     bad = __any_sync(0xFFFFFFFFu, bad);
     for (int k = lane; k < K; k += 32) {
         const int idx = I[k];
-        inside[w][k] = (idx >= 0 && idx < n) ? y[idx] : 0.f;
+        inside[w][k] = (idx >= 0 && idx < n) ? (double)y[idx] : 0.0;
     }
 #pragma unroll
     for (int j = 0; j < SLOTS; j++) if ((mine >> j) & 1u) v[j] = NEG_INF;
@@ -587,7 +590,7 @@ topk_small_kernel(const float* __restrict__ ref, int64_t steps, int n, int64_t l
         const unsigned holders = __ballot_sync(0xFFFFFFFFu, best == top);
         const int winner = __ffs(holders) - 1;         // lowest lane holding the maximum
         if (lane == winner) {
-            outside[w][r] = top;                       // (-inf once fewer than K entries are left outside I)
+            outside[w][r] = (double)top;               // (-inf once fewer than K entries are left outside I)
 #pragma unroll
             for (int j = 0; j < SLOTS; j++) if (j == slot) v[j] = NEG_INF;
         }
@@ -595,12 +598,12 @@ topk_small_kernel(const float* __restrict__ ref, int64_t steps, int n, int64_t l
     __syncwarp();
     double best_cost = INFINITY;
     for (int cnd = lane; cnd < 2 * K; cnd += 32) {
-        const double t = cnd < K ? (double)outside[w][cnd] : (double)inside[w][cnd - K];
+        const double t = cnd < K ? outside[w][cnd] : inside[w][cnd - K];
         if (t > -INFINITY) {
             double c = 0.0;
             for (int k = 0; k < K; k++) {
-                c += fmax((double)outside[w][k] - t, 0.0);
-                c += fmax(t - (double)inside[w][k], 0.0);
+                c += fmax(outside[w][k] - t, 0.0);
+                c += fmax(t - inside[w][k], 0.0);
             }
             best_cost = fmin(best_cost, c);
         }

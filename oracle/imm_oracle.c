@@ -28,7 +28,9 @@
  * (2^64 = 2^32-1, 2^96 = -1, the published 2^32-th root of unity), Python big-integer
  * arithmetic, MLE values at Boolean points, exhaustive hypercube sums for every round
  * polynomial on tiny shapes, closed forms (identity / all-ones matrices, extra padding
- * variable), g(0)+g(1) = running claim, accept honest / reject tampered.
+ * variable), g(0)+g(1) = running claim, accept honest / reject tampered; for the batched
+ * proof: the exhaustive big-integer definition of the combined round polynomials, the
+ * single-proof transcript at P = 1, linearity in the per-proof transcripts, soundness cases.
  */
 #include <stdint.h>
 #include <stdlib.h>
@@ -305,4 +307,137 @@ void orc_matmul_i8_i32(const int8_t* A, const int8_t* B, int32_t* C,
             int32_t aiy = A[i * k + y];
             for (int64_t j = 0; j < n; j++) C[i * n + j] += aiy * (int32_t)B[y * n + j];
         }
+}
+
+/* ---------------------------------------------------------------------------------------
+ * Batched proof: P product claims C_p = A_p * B_p with the same number of rounds b are proved
+ * by ONE sumcheck of their random linear combination (the standard batching of sumcheck claims
+ * over a common hypercube; the paper lists the products to prove -- attention and MLPs,
+ * Section 4.1 -- and leaves the proof system and any batching open).
+ *
+ *   rho_p      = challenge(seed, batch_id, 4, p)             combination coefficients
+ *   r_j        = challenge(seed, batch_id, 3, j)             round challenges, shared by all p
+ *   r_row, r_col of proof p come from its own proof_id (domains 1 and 2), as in the single proof.
+ *
+ * Combined claim   c0^B = sum_p rho_p c0_p,  c0_p = C~_p(r_row_p, r_col_p).
+ * Round j          g_j^B(X) = sum_p rho_p g_j^(p)(X), g_j^(p) the single-proof round polynomial
+ *                  of proof p under the shared challenges r_0..r_{j-1}.
+ * After b rounds   a_fin_p = A~_p(r_row_p, r),  b_fin_p = B~_p(r, r_col_p).
+ *
+ * transcript (1 + 3b + 3P words):
+ *   [c0^B, g_0^B(0..2), ..., g_{b-1}^B(0..2), (c0_0, a_fin_0, b_fin_0), ..., (c0_{P-1}, ...)].
+ * Every proof keeps its own vectors; there is no sharing of work between proofs beyond the
+ * challenges.  Returns ORC_ERR_ARG for a bad shape or proofs whose round counts differ.   */
+int orc_sumcheck_matmul_prove_batched(int P, const int8_t* const* A, const int8_t* const* B,
+                                      const int32_t* const* C, const int64_t* m, const int64_t* k,
+                                      const int64_t* n, const int64_t* lda, const int64_t* ldb,
+                                      const int64_t* ldc, uint64_t seed, uint64_t batch_id,
+                                      const uint64_t* proof_ids, uint64_t* transcript)
+{
+    if (P <= 0 || !A || !B || !C || !m || !k || !n || !lda || !ldb || !ldc || !proof_ids || !transcript)
+        return ORC_ERR_ARG;
+    for (int p = 0; p < P; p++)
+        if (m[p] <= 0 || k[p] <= 0 || n[p] <= 0 || lda[p] < k[p] || ldb[p] < n[p] || ldc[p] < n[p])
+            return ORC_ERR_ARG;
+    int b = orc_ceil_log2(k[0]);
+    for (int p = 1; p < P; p++)
+        if (orc_ceil_log2(k[p]) != b) return ORC_ERR_ARG;
+    int64_t kp = (int64_t)1 << b;
+
+    uint64_t** av = (uint64_t**)calloc((size_t)P, sizeof(uint64_t*));
+    uint64_t** bv = (uint64_t**)calloc((size_t)P, sizeof(uint64_t*));
+    uint64_t* rho = (uint64_t*)malloc(sizeof(uint64_t) * (size_t)P);
+    if (!av || !bv || !rho) { free(av); free(bv); free(rho); return ORC_ERR_ARG; }
+    uint64_t* tail = transcript + 1 + 3 * b;
+    uint64_t c0_batch = 0;
+    int rc = ORC_OK;
+    for (int p = 0; p < P && rc == ORC_OK; p++) {
+        int a = orc_ceil_log2(m[p]), c = orc_ceil_log2(n[p]);
+        uint64_t* r_row = (uint64_t*)malloc(sizeof(uint64_t) * (size_t)(a + 1));
+        uint64_t* r_col = (uint64_t*)malloc(sizeof(uint64_t) * (size_t)(c + 1));
+        uint64_t* e_row = (uint64_t*)malloc(sizeof(uint64_t) << a);
+        uint64_t* e_col = (uint64_t*)malloc(sizeof(uint64_t) << c);
+        av[p] = (uint64_t*)calloc((size_t)kp, sizeof(uint64_t));
+        bv[p] = (uint64_t*)calloc((size_t)kp, sizeof(uint64_t));
+        if (!r_row || !r_col || !e_row || !e_col || !av[p] || !bv[p]) rc = ORC_ERR_ARG;
+        else {
+            for (int t = 0; t < a; t++) r_row[t] = orc_challenge(seed, proof_ids[p], 1, (uint32_t)t);
+            for (int t = 0; t < c; t++) r_col[t] = orc_challenge(seed, proof_ids[p], 2, (uint32_t)t);
+            orc_eq_table(r_row, a, e_row);
+            orc_eq_table(r_col, c, e_col);
+            orc_mle_partial_eval(A[p], ORC_I8, m[p], k[p], lda[p], ORC_BIND_ROWS, e_row, av[p]);
+            orc_mle_partial_eval(B[p], ORC_I8, k[p], n[p], ldb[p], ORC_BIND_COLS, e_col, bv[p]);
+            rho[p] = orc_challenge(seed, batch_id, 4, (uint32_t)p);
+            tail[3 * p] = orc_mle_eval_point(C[p], ORC_I32, m[p], n[p], ldc[p], e_row, e_col);
+            c0_batch = orc_add(c0_batch, orc_mul(rho[p], tail[3 * p]));
+        }
+        free(r_row); free(r_col); free(e_row); free(e_col);
+    }
+    if (rc == ORC_OK) {
+        uint64_t* w = transcript;
+        *w++ = c0_batch;
+        for (int j = 0; j < b; j++) {
+            int64_t half = (int64_t)1 << (b - 1 - j);
+            uint64_t r = orc_challenge(seed, batch_id, 3, (uint32_t)j);
+            uint64_t g0 = 0, g1 = 0, g2 = 0;
+            for (int p = 0; p < P; p++) {
+                uint64_t s0 = 0, s1 = 0, s2 = 0;
+                for (int64_t y = 0; y < half; y++) {
+                    uint64_t a0 = av[p][y], a1 = av[p][y + half], b0 = bv[p][y], b1 = bv[p][y + half];
+                    uint64_t a2 = orc_sub(orc_add(a1, a1), a0);
+                    uint64_t b2 = orc_sub(orc_add(b1, b1), b0);
+                    s0 = orc_add(s0, orc_mul(a0, b0));
+                    s1 = orc_add(s1, orc_mul(a1, b1));
+                    s2 = orc_add(s2, orc_mul(a2, b2));
+                }
+                g0 = orc_add(g0, orc_mul(rho[p], s0));
+                g1 = orc_add(g1, orc_mul(rho[p], s1));
+                g2 = orc_add(g2, orc_mul(rho[p], s2));
+                for (int64_t y = 0; y < half; y++) {
+                    av[p][y] = orc_add(av[p][y], orc_mul(r, orc_sub(av[p][y + half], av[p][y])));
+                    bv[p][y] = orc_add(bv[p][y], orc_mul(r, orc_sub(bv[p][y + half], bv[p][y])));
+                }
+            }
+            *w++ = g0; *w++ = g1; *w++ = g2;
+        }
+        for (int p = 0; p < P; p++) { tail[3 * p + 1] = av[p][0]; tail[3 * p + 2] = bv[p][0]; }
+    }
+    for (int p = 0; p < P; p++) { free(av[p]); free(bv[p]); }
+    free(av); free(bv); free(rho);
+    return rc;
+}
+
+/* Verifier of a batched transcript.  claim <- c0^B, which must equal sum_p rho_p c0_p; per round
+ * g(0)+g(1) = claim, claim <- g(r_j); finally claim = sum_p rho_p a_fin_p b_fin_p.  expect, when
+ * non-NULL, holds the verifier's own 3P values (c0_p, a_fin_p, b_fin_p) and is compared word
+ * for word.
+ * *fail_at: -1 accept; j = round j; nrounds = the final check; nrounds+1 = c0^B is not the
+ * combination of the listed c0_p; nrounds+2+t = word t of the per-proof tail differs from
+ * expect.                                                                                 */
+int orc_sumcheck_verify_batched(const uint64_t* transcript, int nrounds, int P, uint64_t seed,
+                                uint64_t batch_id, const uint64_t* expect, int* fail_at)
+{
+    if (!transcript || nrounds < 0 || P <= 0 || !fail_at) return ORC_ERR_ARG;
+    for (int t = 0; t < 1 + 3 * nrounds + 3 * P; t++)
+        if (transcript[t] >= ORC_P) return ORC_ERR_ARG;
+    const uint64_t* tail = transcript + 1 + 3 * nrounds;
+    uint64_t combo = 0, fin = 0;
+    for (int p = 0; p < P; p++) {
+        uint64_t rho = orc_challenge(seed, batch_id, 4, (uint32_t)p);
+        combo = orc_add(combo, orc_mul(rho, tail[3 * p]));
+        fin = orc_add(fin, orc_mul(rho, orc_mul(tail[3 * p + 1], tail[3 * p + 2])));
+    }
+    uint64_t claim = transcript[0];
+    if (claim != combo) { *fail_at = nrounds + 1; return ORC_REJECT; }
+    for (int j = 0; j < nrounds; j++) {
+        uint64_t g0 = transcript[1 + 3 * j], g1 = transcript[2 + 3 * j], g2 = transcript[3 + 3 * j];
+        if (orc_add(g0, g1) != claim) { *fail_at = j; return ORC_REJECT; }
+        claim = orc_interp_deg2(g0, g1, g2, orc_challenge(seed, batch_id, 3, (uint32_t)j));
+    }
+    if (fin != claim) { *fail_at = nrounds; return ORC_REJECT; }
+    if (expect)
+        for (int t = 0; t < 3 * P; t++)
+            if (expect[t] != tail[t]) { *fail_at = nrounds + 2 + t; return ORC_REJECT; }
+    *fail_at = -1;
+    return ORC_OK;
 }

@@ -72,6 +72,10 @@ def lib() -> ctypes.CDLL:
         L.orc_interp_deg2.argtypes = [_u64, _u64, _u64, _u64]
         L.orc_sumcheck_verify.restype = ctypes.c_int
         L.orc_sumcheck_verify.argtypes = [_vp, ctypes.c_int, _u64, _u64, _vp, _vp, _vp, _vp]
+        L.orc_sumcheck_matmul_prove_batched.restype = ctypes.c_int
+        L.orc_sumcheck_matmul_prove_batched.argtypes = [ctypes.c_int] + [_vp] * 9 + [_u64, _u64, _vp, _vp]
+        L.orc_sumcheck_verify_batched.restype = ctypes.c_int
+        L.orc_sumcheck_verify_batched.argtypes = [_vp, ctypes.c_int, ctypes.c_int, _u64, _u64, _vp, _vp]
         L.orc_matmul_i8_i32.restype = None
         L.orc_matmul_i8_i32.argtypes = [_vp, _vp, _vp, _i64, _i64, _i64]
         _lib = L
@@ -245,4 +249,46 @@ def sumcheck_verify(transcript, nrounds: int, seed: int, proof_id: int, expect_c
     fail = ctypes.c_int(-2)
     rc = lib().orc_sumcheck_verify(_ptr(t), nrounds, seed, proof_id, opt(expect_c0),
                                    opt(expect_a_fin), opt(expect_b_fin), ctypes.addressof(fail))
+    return rc, fail.value
+
+
+def batched_transcript_len(k: int, nproofs: int) -> int:
+    return 1 + 3 * ceil_log2(k) + 3 * nproofs
+
+
+def sumcheck_matmul_prove_batched(problems, seed: int, batch_id: int) -> np.ndarray:
+    """``problems`` is a sequence of (A, B, C, proof_id) whose k pad to the same power of two."""
+    mats, dims, ptrs = [], [], [[], [], []]
+    for A, B, C, _ in problems:
+        A, ca, m, k, lda = _mat(A)
+        B, cb, k2, n, ldb = _mat(B)
+        C, cc, m2, n2, ldc = _mat(C)
+        assert ca == I8 and cb == I8 and cc == I32 and k == k2 and m == m2 and n == n2
+        mats.append((A, B, C))
+        dims.append((m, k, n, lda, ldb, ldc))
+        for lst, M in zip(ptrs, (A, B, C)):
+            lst.append(_ptr(M))
+    count = len(problems)
+    parr = [np.array(lst, dtype=np.uint64) for lst in ptrs]
+    darr = [np.array([d[i] for d in dims], dtype=np.int64) for i in range(6)]
+    ids = np.array([int(p[3]) for p in problems], dtype=np.uint64)
+    out = np.empty(batched_transcript_len(dims[0][1], count) if count else 0, dtype=np.uint64)
+    rc = lib().orc_sumcheck_matmul_prove_batched(count, *[_ptr(a) for a in parr],
+                                                 *[_ptr(a) for a in darr], seed, batch_id,
+                                                 _ptr(ids), _ptr(out))
+    if rc != OK:
+        raise ValueError(f"orc_sumcheck_matmul_prove_batched returned {rc}")
+    return out
+
+
+def sumcheck_verify_batched(transcript, nrounds: int, nproofs: int, seed: int, batch_id: int,
+                            expect=None):
+    """Return (status, fail_at); ``expect`` is the verifier's own 3*nproofs tail words."""
+    t = _fe_array(transcript)
+    assert len(t) >= 1 + 3 * nrounds + 3 * nproofs
+    e = None if expect is None else _fe_array(expect)
+    assert e is None or len(e) == 3 * nproofs
+    fail = ctypes.c_int(-2)
+    rc = lib().orc_sumcheck_verify_batched(_ptr(t), nrounds, nproofs, seed, batch_id,
+                                           None if e is None else _ptr(e), ctypes.addressof(fail))
     return rc, fail.value

@@ -35,6 +35,7 @@ import torch  # noqa: E402
 METRIC = "proved field-MACs/sec"
 UNIT = "field-MAC/s"
 SEED = 1
+BATCH_ID0 = 1 << 40            # ids of the batched proofs (--batched), clear of the proof ids
 
 
 def parse_args():
@@ -49,6 +50,9 @@ def parse_args():
     ap.add_argument("--tokens", type=int, default=None, help="token count (default: the configuration's own)")
     ap.add_argument("--vocab", type=int, default=128256, help="ldd: entries per logit row")
     ap.add_argument("--topk", type=int, default=20, help="ldd: size of the committed index sets")
+    ap.add_argument("--batched", action="store_true",
+                    help="prove the products of equal round count as one random-linear-combination proof each "
+                         "(device-resident timing only)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=2)
@@ -222,13 +226,28 @@ def run_ours(args):
     macs = synth.prover_field_macs(problems)
     algo_bytes = synth.problem_bytes(problems)
     claim_bytes = sum(4 * m * n for (m, k, n) in shapes)
-    prover = imm.Prover([(p.A, p.B, p.C, p.proof_id) for p in problems], device=dev)
-    imm.profile_enable(min(4096, warmup + steps + 4))
+    groups = {}
+    if args.batched:
+        for p in problems:
+            groups.setdefault(imm.ceil_log2(p.mkn[1]), []).append(p)
+        provers = [imm.BatchedProver([(p.A, p.B, p.C, p.proof_id) for p in g], device=dev) for g in groups.values()]
+
+        def prove_step():
+            for gi, bp in enumerate(provers):
+                bp.prove(SEED, BATCH_ID0 + gi)
+    else:
+        prover = imm.Prover([(p.A, p.B, p.C, p.proof_id) for p in problems], device=dev)
+        provers = [prover]
+
+        def prove_step():
+            prover.prove(SEED)
+    calls_per_step = len(provers)
+    imm.profile_enable(min(4096, (warmup + steps + 4) * calls_per_step))
 
     barrier = rep.barrier
 
     for _ in range(warmup):
-        prover.prove(SEED)
+        prove_step()
     barrier()
     sampler = ClockSampler(local_rank if "CUDA_VISIBLE_DEVICES" not in os.environ else
                            int(os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local_rank]))
@@ -245,7 +264,7 @@ def run_ours(args):
         for a, b in pairs:
             scrub.fill_(1)
             a.record()
-            prover.prove(SEED)
+            prove_step()
             b.record()
         barrier()
         elapsed_ms = sum(a.elapsed_time(b) for a, b in pairs)
@@ -253,7 +272,7 @@ def run_ours(args):
         ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         ev0.record()
         for _ in range(steps):
-            prover.prove(SEED)
+            prove_step()
         ev1.record()
         barrier()
         elapsed_ms = ev0.elapsed_time(ev1)
@@ -261,20 +280,28 @@ def run_ours(args):
     clocks = sampler.stop(t0, t1)
     elapsed_ms = rep.max_over_ranks(elapsed_ms)
     phase_ms = [0.0] * len(imm.PROFILE_PHASES)
-    for c in range(first_call, first_call + steps):
+    for c in range(first_call, first_call + steps * calls_per_step):
         for i, v in enumerate(imm.profile_read(c)):
             phase_ms[i] += v / steps
     imm.profile_enable(0)
 
     # every proof of the timed batch must be accepted by the verifier
-    host_t = prover.transcripts.cpu()
-    assert int(prover.status.abs().max()) == 0
     accepted = 0
-    for i, p in enumerate(problems):
-        b = imm.ceil_log2(p.A.shape[1])
-        words = [int(v) & 0xFFFFFFFFFFFFFFFF for v in host_t[i, :3 * b + 3]]
-        if imm.sumcheck_verify(words, b, SEED, p.proof_id) == (imm.OK, -1):
-            accepted += 1
+    if args.batched:
+        host_t = None
+        for gi, (b, g) in enumerate(groups.items()):
+            assert int(provers[gi].status.abs().max()) == 0
+            words = [int(v) & 0xFFFFFFFFFFFFFFFF for v in provers[gi].transcript.cpu()]
+            if imm.sumcheck_verify_batched(words, b, len(g), SEED, BATCH_ID0 + gi) == (imm.OK, -1):
+                accepted += len(g)
+    else:
+        host_t = prover.transcripts.cpu()
+        assert int(prover.status.abs().max()) == 0
+        for i, p in enumerate(problems):
+            b = imm.ceil_log2(p.A.shape[1])
+            words = [int(v) & 0xFFFFFFFFFFFFFFFF for v in host_t[i, :3 * b + 3]]
+            if imm.sumcheck_verify(words, b, SEED, p.proof_id) == (imm.OK, -1):
+                accepted += 1
     if accepted != len(problems):
         raise SystemExit(f"only {accepted}/{len(problems)} proofs verified")
 
@@ -287,7 +314,8 @@ def run_ours(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "u64", "data": "synthetic",
-        "config": {"workload": workload_name(args.config, args.layers, args.tokens),
+        "config": {"workload": workload_name(args.config, args.layers, args.tokens) +
+                               (f", as {calls_per_step} batched proofs (one per round count)" if args.batched else ""),
                    "layers": args.layers if args.config == "decoder" else min(args.layers, 8) if args.config == "attn" else None,
                    "tokens": args.tokens, "proofs_per_gpu": len(problems), "field": "Goldilocks 2^64-2^32+1",
                    "input_bytes_per_gpu": algo_bytes,
@@ -307,13 +335,17 @@ def run_ours(args):
                      "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": claim_gbs / peak,
                      "frac_of_8tbs": claim_gbs / 8000.0,
                      "traffic": (CLAIM_KERNEL_TRAFFIC_RATIO * claim_bytes) if CLAIM_KERNEL_TRAFFIC_RATIO else None},
-        "gpu_launches": 5 * steps,
+        "gpu_launches": (6 if args.batched else 5) * calls_per_step * steps,
+        "transcript_words_per_step": (sum(int(bp.length) for bp in provers) if args.batched else
+                                      sum(3 * imm.ceil_log2(k) + 3 for (m, k, n) in shapes)),
         "clocks": clocks,
     }
 
     # ---- end to end: pinned host inputs -> device arena -> proofs -> host transcripts
     e2e = None
-    if not args.no_e2e:
+    if args.batched:
+        e2e = {"value": None, "unit": UNIT, "skipped": "the host-buffer entry point proves proof by proof"}
+    elif not args.no_e2e:
         need = algo_bytes
         if mem_available_bytes() < int(1.25 * need * (world if world > 1 else 1)):
             e2e = {"value": None, "unit": UNIT, "skipped": "not enough host memory for pinned inputs"}
@@ -340,7 +372,7 @@ def run_ours(args):
     out["e2e"] = e2e
 
     # ---- the oracle beside it (rank 0, single GPU): first two layers' proofs, one per thread
-    if not args.no_cpu_baseline and world == 1:
+    if not args.no_cpu_baseline and world == 1 and not args.batched:
         nsample = min(len(problems), 8)
         sample = sample_to_host(problems[:nsample])
         threads = min(os.cpu_count() or 1, nsample)
@@ -557,7 +589,8 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world,
         "steps": steps, "warmup": warmup, "ms_per_step": per * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "u64", "data": "synthetic",
-        "config": {"workload": workload_name(args.config, args.layers, args.tokens),
+        "config": {"workload": workload_name(args.config, args.layers, args.tokens) +
+                               (f", as {calls_per_step} batched proofs (one per round count)" if args.batched else ""),
                    "layers": args.layers if args.config == "decoder" else None,
                    "tokens": args.tokens, "sampled": desc,
                    "note": None if tokens == args.tokens else "no CUDA device for input generation: token count reduced"},

@@ -21,7 +21,8 @@
  *   - A dimension d is zero-padded (implicitly) at the high end to 2^ceil(log2 d).
  *   - Challenges are public coins of an interactive verifier, drawn from a counter-based
  *     generator (SplitMix64 mixer) keyed by (seed, proof_id); they do not depend on the
- *     prover's messages.  domain 1 = r_row, 2 = r_col, 3 = sumcheck rounds.
+ *     prover's messages.  domain 1 = r_row, 2 = r_col, 3 = sumcheck rounds, 4 = the
+ *     coefficients of a batched proof (keyed by the batch's id).
  *   - Transcript of one proof: [c0, g_0(0), g_0(1), g_0(2), ..., g_{b-1}(0), g_{b-1}(1),
  *     g_{b-1}(2), a_fin, b_fin], b = ceil(log2 k), 3b+3 words.
  *
@@ -78,7 +79,7 @@ int imm_version(void);
  * The pointer stays valid until the thread's next failing call. */
 const char* imm_last_cuda_error(void);
 
-/* HOST.  Challenge `index` of `domain` (1 = r_row, 2 = r_col, 3 = sumcheck round) for
+/* HOST.  Challenge `index` of `domain` (1 = r_row, 2 = r_col, 3 = sumcheck round, 4 = batching coefficient) for
  * (seed, proof_id): canon(mix64(key + G*(ctr+1))) with key = mix64(mix64(seed+G) + G*(proof_id+1)),
  * ctr = domain<<32 | index, G = 0x9E3779B97F4A7C15, canon(x) = x >= p ? x-p : x.  These are the
  * verifier's public coins (Section 2.2's Vrfy side). */
@@ -230,6 +231,55 @@ int imm_sumcheck_matmul_prove_host(const imm_matmul_desc* descs_host, int nproof
 int imm_sumcheck_verify(const imm_fe* transcript_host, int nrounds, uint64_t seed,
                         uint64_t proof_id, const imm_fe* expect_c0, const imm_fe* expect_a_fin,
                         const imm_fe* expect_b_fin, int* fail_at);
+
+/* ---------------------------------------------------------------------------------------------
+ * Batched proof: one sumcheck for a random linear combination of product claims
+ * ---------------------------------------------------------------------------------------------
+ * The products a proof of the reference execution must cover are many (the attention and MLP
+ * products of every layer, Section 4.1).  Claims whose k pad to the same 2^b can share one
+ * sumcheck: with public coins rho_p = imm_challenge(seed, batch_id, 4, p) the prover shows
+ *   sum_p rho_p * sum_y A_p~(r_row_p, y) B_p~(y, r_col_p) = sum_p rho_p C_p~(r_row_p, r_col_p),
+ * all proofs folding with the same round challenges r_j = imm_challenge(seed, batch_id, 3, j);
+ * r_row_p and r_col_p stay each proof's own (domains 1, 2 under its proof_id).  The verifier then
+ * reads 1 + 3b + 3P words instead of P * (3b + 3).
+ *
+ * Batched transcript, imm_sumcheck_batched_transcript_len(b, P) = 1 + 3b + 3P words:
+ *   [c0B, g_0(0), g_0(1), g_0(2), ..., g_{b-1}(0..2), (c0_0, a_fin_0, b_fin_0), ..., (c0_{P-1}, ..)]
+ *   c0B = sum_p rho_p c0_p;  g_j = sum_p rho_p g_j^(p);  a_fin_p = A_p~(r_row_p, r),
+ *   b_fin_p = B_p~(r, r_col_p) at the shared point r = (r_0..r_{b-1}).                          */
+#define IMM_BATCH_MAX_PROOFS (1 << 24)
+
+/* Transcript words of a batched proof (0 on invalid arguments). */
+int64_t imm_sumcheck_batched_transcript_len(int nrounds, int nproofs);
+
+/* Workspace bytes imm_sumcheck_matmul_prove_batched needs (0 on invalid input, which includes
+ * proofs whose ceil(log2 k) differ). */
+size_t imm_sumcheck_matmul_batched_workspace(const imm_matmul_desc* descs_host, int nproofs);
+
+/* Batched prover.  Runs the launch sequence of imm_sumcheck_matmul_prove with the shared round
+ * challenges (per-proof transcripts go to the workspace), then one more launch forms the
+ * batched transcript.
+ *   descs_host   : HOST array of nproofs descriptors with DEVICE matrix pointers; every
+ *                  ceil(log2 k) must be the same, else IMM_ERR_SHAPE
+ *   d_transcript : DEVICE array of imm_sumcheck_batched_transcript_len(b, nproofs) words
+ *   d_status     : DEVICE array of nproofs int32 (as imm_sumcheck_matmul_prove)
+ *   d_ws         : DEVICE workspace, 256-byte aligned, >= imm_sumcheck_matmul_batched_workspace(...)
+ * Errors: IMM_ERR_ARG, IMM_ERR_SHAPE, IMM_ERR_ALIGN, IMM_ERR_WORKSPACE, IMM_ERR_LIMIT (more than
+ * IMM_BATCH_MAX_PROOFS proofs), IMM_ERR_CUDA. */
+int imm_sumcheck_matmul_prove_batched(const imm_matmul_desc* descs_host, int nproofs, uint64_t seed,
+                                      uint64_t batch_id, imm_fe* d_transcript, int32_t* d_status,
+                                      void* d_ws, size_t ws_bytes, void* stream);
+
+/* HOST verifier of a batched transcript.  Requires c0B = sum_p rho_p c0_p; then, with
+ * claim <- c0B, per round g_j(0) + g_j(1) = claim and claim <- g_j(r_j); finally
+ * claim = sum_p rho_p a_fin_p b_fin_p.  expect_host, when non-NULL, holds the verifier's own
+ * 3*nproofs values (c0_p, a_fin_p, b_fin_p in transcript order) and is compared word for word.
+ *   fail_at : HOST out.  -1 accepted; j in [0,nrounds) = round j; nrounds = the final check;
+ *             nrounds+1 = c0B is not the combination of the listed c0_p; nrounds+2+t = word t of
+ *             the per-proof part differs from expect_host
+ * Returns IMM_OK, IMM_REJECT, IMM_ERR_ARG or IMM_ERR_NONCANONICAL. */
+int imm_sumcheck_verify_batched(const imm_fe* transcript_host, int nrounds, int nproofs, uint64_t seed,
+                                uint64_t batch_id, const imm_fe* expect_host, int* fail_at);
 
 /* ---------------------------------------------------------------------------------------------
  * Logit distance distribution (LDD)

@@ -617,9 +617,11 @@ size_t imm_sumcheck_matmul_workspace(const imm_matmul_desc* descs_host, int npro
     return p.status == IMM_OK ? p.total_bytes : 0;
 }
 
-int imm_sumcheck_matmul_prove(const imm_matmul_desc* descs_host, int nproofs, uint64_t seed,
-                              imm_fe* d_transcripts, int64_t stride, int32_t* d_status,
-                              void* d_ws, size_t ws_bytes, void* stream)
+// The launch sequence of a batch.  shared_round_id: null = every proof draws its round challenges
+// under its own proof_id; else all proofs draw them under that one id (a batched proof).
+static int prove_batch(const imm_matmul_desc* descs_host, int nproofs, uint64_t seed,
+                       const uint64_t* shared_round_id, imm_fe* d_transcripts, int64_t stride,
+                       int32_t* d_status, void* d_ws, size_t ws_bytes, void* stream)
 {
     if (!d_transcripts || !d_status || !d_ws) return IMM_ERR_ARG;
     Plan p = make_plan(descs_host, nproofs);
@@ -650,7 +652,7 @@ int imm_sumcheck_matmul_prove(const imm_matmul_desc* descs_host, int nproofs, ui
         P.part_a = (imm_fe*)(base + q.part_a);
         P.part_b = (imm_fe*)(base + q.part_b);
         P.part_c = (imm_fe*)(base + q.part_c);
-        P.proof_id = d.proof_id;
+        P.round_id = shared_round_id ? *shared_round_id : d.proof_id;
         P.m = (int32_t)d.m; P.k = (int32_t)d.k; P.n = (int32_t)d.n;
         P.a = q.a; P.b = q.b; P.c = q.c;
         P.n_part_a = q.n_part_a; P.n_part_b = q.n_part_b; P.n_part_c = q.n_part_c;
@@ -734,6 +736,61 @@ int imm_sumcheck_matmul_prove(const imm_matmul_desc* descs_host, int nproofs, ui
     PROF_MARK(9, st);
 #undef PROF_MARK
     if (prof) g_prof_calls++;
+    return IMM_OK;
+}
+
+int imm_sumcheck_matmul_prove(const imm_matmul_desc* descs_host, int nproofs, uint64_t seed,
+                              imm_fe* d_transcripts, int64_t stride, int32_t* d_status,
+                              void* d_ws, size_t ws_bytes, void* stream)
+{
+    return prove_batch(descs_host, nproofs, seed, nullptr, d_transcripts, stride, d_status, d_ws, ws_bytes, stream);
+}
+
+// Batched proof: the per-proof transcripts (shared round challenges) go to the head of the
+// workspace, the prover's own workspace follows, and one more launch combines them.
+static int batched_layout(const imm_matmul_desc* descs_host, int nproofs, int* b, size_t* rows_bytes, size_t* total)
+{
+    Plan p = make_plan(descs_host, nproofs);
+    if (p.status != IMM_OK) return p.status;
+    if (nproofs > IMM_BATCH_MAX_PROOFS) return IMM_ERR_LIMIT;
+    *b = ceil_log2(descs_host[0].k);
+    for (int i = 1; i < nproofs; i++)
+        if (ceil_log2(descs_host[i].k) != *b) return IMM_ERR_SHAPE;
+    *rows_bytes = align_up((size_t)nproofs * (size_t)(3 * *b + 3) * sizeof(imm_fe));
+    *total = *rows_bytes + p.total_bytes;
+    return IMM_OK;
+}
+
+size_t imm_sumcheck_matmul_batched_workspace(const imm_matmul_desc* descs_host, int nproofs)
+{
+    int b;
+    size_t rows, total;
+    return batched_layout(descs_host, nproofs, &b, &rows, &total) == IMM_OK ? total : 0;
+}
+
+int64_t imm_sumcheck_batched_transcript_len(int nrounds, int nproofs)
+{
+    if (nrounds < 0 || nrounds > 64 || nproofs <= 0 || nproofs > IMM_BATCH_MAX_PROOFS) return 0;
+    return 1 + 3 * (int64_t)nrounds + 3 * (int64_t)nproofs;
+}
+
+int imm_sumcheck_matmul_prove_batched(const imm_matmul_desc* descs_host, int nproofs, uint64_t seed,
+                                      uint64_t batch_id, imm_fe* d_transcript, int32_t* d_status,
+                                      void* d_ws, size_t ws_bytes, void* stream)
+{
+    if (!d_transcript || !d_status || !d_ws) return IMM_ERR_ARG;
+    int b;
+    size_t rows, total;
+    int rc = batched_layout(descs_host, nproofs, &b, &rows, &total);
+    if (rc != IMM_OK) return rc;
+    if ((uintptr_t)d_ws % ALIGN != 0 || (uintptr_t)d_transcript % 8 != 0) return IMM_ERR_ALIGN;
+    if (ws_bytes < total) return IMM_ERR_WORKSPACE;
+    imm_fe* d_rows = (imm_fe*)d_ws;
+    const int64_t stride = 3 * b + 3;
+    rc = prove_batch(descs_host, nproofs, seed, &batch_id, d_rows, stride, d_status, (char*)d_ws + rows,
+                     ws_bytes - rows, stream);
+    if (rc != IMM_OK) return rc;
+    CU(launch_combine(d_rows, stride, nproofs, b, seed, batch_id, d_transcript, (cudaStream_t)stream));
     return IMM_OK;
 }
 
@@ -879,6 +936,49 @@ int imm_sumcheck_verify(const imm_fe* transcript_host, int nrounds, uint64_t see
     if (expect_c0 && *expect_c0 != t[0]) { *fail_at = nrounds + 1; return IMM_REJECT; }
     if (expect_a_fin && *expect_a_fin != a_fin) { *fail_at = nrounds + 2; return IMM_REJECT; }
     if (expect_b_fin && *expect_b_fin != b_fin) { *fail_at = nrounds + 3; return IMM_REJECT; }
+    *fail_at = -1;
+    return IMM_OK;
+}
+
+int imm_sumcheck_verify_batched(const imm_fe* transcript_host, int nrounds, int nproofs, uint64_t seed,
+                                uint64_t batch_id, const imm_fe* expect_host, int* fail_at)
+{
+    if (!transcript_host || !fail_at || nrounds < 0 || nrounds > 64 || nproofs <= 0 ||
+        nproofs > IMM_BATCH_MAX_PROOFS)
+        return IMM_ERR_ARG;
+    const imm_fe* t = transcript_host;
+    const int64_t len = 1 + 3 * (int64_t)nrounds + 3 * (int64_t)nproofs;
+    for (int64_t i = 0; i < len; i++)
+        if (t[i] >= IMM_P) return IMM_ERR_NONCANONICAL;
+    if (expect_host)
+        for (int64_t i = 0; i < 3 * (int64_t)nproofs; i++)
+            if (expect_host[i] >= IMM_P) return IMM_ERR_NONCANONICAL;
+    const imm_fe* tail = t + 1 + 3 * nrounds;
+    uint64_t combo = 0, fin = 0;
+    for (int p = 0; p < nproofs; p++) {
+        const uint64_t rho = gl::challenge(seed, batch_id, 4, (uint32_t)p);
+        combo = gl::add(combo, gl::mul(rho, tail[3 * (int64_t)p]));
+        fin = gl::add(fin, gl::mul(rho, gl::mul(tail[3 * (int64_t)p + 1], tail[3 * (int64_t)p + 2])));
+    }
+    uint64_t claim = t[0];
+    if (claim != combo) { *fail_at = nrounds + 1; return IMM_REJECT; }
+    const uint64_t inv2 = 0x7FFFFFFF80000001ULL;
+    for (int j = 0; j < nrounds; j++) {
+        const uint64_t g0 = t[1 + 3 * j], g1 = t[2 + 3 * j], g2 = t[3 + 3 * j];
+        if (gl::add(g0, g1) != claim) { *fail_at = j; return IMM_REJECT; }
+        const uint64_t r = gl::challenge(seed, batch_id, 3, (uint32_t)j);
+        const uint64_t d1 = gl::sub(g1, g0);
+        const uint64_t d2 = gl::sub(gl::sub(g2, g1), d1);
+        const uint64_t c2 = gl::mul(gl::mul(r, gl::sub(r, 1)), inv2);
+        claim = gl::add(g0, gl::add(gl::mul(r, d1), gl::mul(c2, d2)));
+    }
+    if (fin != claim) { *fail_at = nrounds; return IMM_REJECT; }
+    if (expect_host)
+        for (int64_t i = 0; i < 3 * (int64_t)nproofs; i++)
+            if (expect_host[i] != tail[i]) {
+                *fail_at = nrounds + 2 + (int)i;
+                return IMM_REJECT;
+            }
     *fail_at = -1;
     return IMM_OK;
 }

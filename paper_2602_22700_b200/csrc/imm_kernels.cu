@@ -649,7 +649,7 @@ sumcheck_kernel(const ProofDev* proofs, uint64_t seed, imm_fe* transcripts, int6
     const int J = dist ? b - SC_FINAL_VARS : b;            // rounds run on the local tables
     const int L = (int)(((int64_t)1 << b) / (dist ? nc : 1));
 
-    if (tid < b) sh.r[tid] = gl::challenge(seed, pr.proof_id, 3, (uint32_t)tid);
+    if (tid < b) sh.r[tid] = gl::challenge(seed, pr.round_id, 3, (uint32_t)tid);
     for (int i = tid; i < MAX_K_VARS * SC_WARPS * 3; i += SUMCHECK_THREADS) (&sh.warp_sums[0][0][0])[i] = 0;
     for (int i = tid; i < MAX_K_VARS * 32 * 3; i += SUMCHECK_THREADS) (&sh.lane_sums[0][0][0])[i] = 0;
     if (c == 0) {
@@ -820,6 +820,40 @@ cudaError_t launch_point_finish(const imm_fe* parts, int64_t count, const imm_fe
                                 const imm_fe* sum_col, int nsc, imm_fe* out, cudaStream_t st)
 {
     point_finish_kernel<<<1, 1024, 0, st>>>(parts, count, sum_row, nsr, sum_col, nsc, out);
+    return cudaGetLastError();
+}
+
+// Batched transcript of `nproofs` proofs that ran under shared round challenges (rows of
+// `stride` words in `tr`, each 3b+3 long): word w < 1+3b of `out` is sum_p rho_p tr[p][w] with
+// rho_p = challenge(seed, batch_id, 4, p) -- one block per word -- and the remaining blocks copy
+// every proof's (c0, a_fin, b_fin) behind them.
+__global__ void __launch_bounds__(COMBINE_THREADS)
+combine_kernel(const imm_fe* tr, int64_t stride, int nproofs, int b, uint64_t seed, uint64_t batch_id, imm_fe* out)
+{
+    __shared__ uint64_t red[33];
+    const int nw = 1 + 3 * b;
+    if ((int)blockIdx.x < nw) {
+        uint64_t s = 0;
+        for (int p = threadIdx.x; p < nproofs; p += COMBINE_THREADS)
+            s = gl::add(s, gl::mul(gl::challenge(seed, batch_id, 4, (uint32_t)p), tr[(int64_t)p * stride + blockIdx.x]));
+        s = block_sum_fe(s, red);
+        if (threadIdx.x == 0) out[blockIdx.x] = s;
+        return;
+    }
+    const int p = ((int)blockIdx.x - nw) * COMBINE_THREADS + threadIdx.x;
+    if (p >= nproofs) return;
+    const imm_fe* row = tr + (int64_t)p * stride;
+    imm_fe* o = out + nw + 3 * (int64_t)p;
+    o[0] = row[0];
+    o[1] = row[3 * b + 1];
+    o[2] = row[3 * b + 2];
+}
+
+cudaError_t launch_combine(const imm_fe* tr, int64_t stride, int nproofs, int b, uint64_t seed, uint64_t batch_id,
+                           imm_fe* out, cudaStream_t st)
+{
+    const unsigned blocks = (unsigned)(1 + 3 * b + (nproofs + COMBINE_THREADS - 1) / COMBINE_THREADS);
+    combine_kernel<<<blocks, COMBINE_THREADS, 0, st>>>(tr, stride, nproofs, b, seed, batch_id, out);
     return cudaGetLastError();
 }
 

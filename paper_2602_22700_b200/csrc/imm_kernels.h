@@ -29,5 +29,8 @@ cudaError_t launch_point_finish(const imm_fe* parts, int64_t count, const imm_fe
 // cluster: blocks per proof (1, 2, 4 or 8), or 0 to let the launch choose from the batch size
 cudaError_t launch_sumcheck(const ProofDev* d_proofs, int nproofs, uint64_t seed, imm_fe* transcripts,
                             int64_t stride, int32_t* status, int max_b, int cluster, cudaStream_t st);
+// batched transcript (1 + 3b + 3*nproofs words) from per-proof transcripts proved under shared round challenges
+cudaError_t launch_combine(const imm_fe* tr, int64_t stride, int nproofs, int b, uint64_t seed, uint64_t batch_id,
+                           imm_fe* out, cudaStream_t st);
 
 }  // namespace imm

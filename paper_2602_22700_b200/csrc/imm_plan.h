@@ -35,6 +35,7 @@ constexpr int ROWLDM_STAGE_BYTES = 32 * ROWLDM_PITCH;
 constexpr int EQ_BATCH_THREADS = 256;
 constexpr int EQ_SLICE_QUADS = 512;           // groups of four table entries per block of eq_batch_kernel
 constexpr int SUMCHECK_THREADS = 512;
+constexpr int COMBINE_THREADS = 128;        // threads of a block of the batched-transcript kernel
 constexpr int SUMCHECK_MAX_CLUSTER = 16;    // most blocks per proof (a power of two dividing 256)
 constexpr int MAX_EQ_VARS = 20;
 constexpr int MAX_K_VARS = 17;
@@ -67,7 +68,7 @@ struct ProofDev {
     const imm_fe* sum_row;     // [n_sum_row] slice sums of E_row over the real rows    } only when the claim
     const imm_fe* sum_col;     // [n_sum_col] slice sums of E_col over the real columns } kernel leaves the
                                //             2^31 offset of its unsigned bytes in part_c (c_offset != 0)
-    uint64_t proof_id;
+    uint64_t round_id;         // id the round challenges are drawn under: the proof's own, or its batch's
     int32_t m, k, n;
     int32_t a, b, c;           // ceil(log2 m), ceil(log2 k), ceil(log2 n)
     int32_t n_part_a, n_part_b, n_part_c;

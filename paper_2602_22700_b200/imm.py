@@ -30,7 +30,9 @@ EXPORTS = ("imm_version", "imm_last_cuda_error", "imm_challenge", "imm_field_bin
            "imm_sumcheck_matmul_workspace", "imm_sumcheck_matmul_prove",
            "imm_sumcheck_matmul_host_arena", "imm_sumcheck_matmul_prove_host", "imm_sumcheck_verify",
            "imm_profile_enable", "imm_profile_calls", "imm_profile_read", "imm_mle_eval_point_noalloc",
-           "imm_ldd_tv_kl", "imm_ldd_topk_workspace", "imm_ldd_topk_distance", "imm_ldd_tail_fraction")
+           "imm_ldd_tv_kl", "imm_ldd_topk_workspace", "imm_ldd_topk_distance", "imm_ldd_tail_fraction",
+           "imm_sumcheck_batched_transcript_len", "imm_sumcheck_matmul_batched_workspace",
+           "imm_sumcheck_matmul_prove_batched", "imm_sumcheck_verify_batched")
 NOALLOC_MAX_TILES = 8192
 PROFILE_PHASES = ("eq_tables", "claim_C", "bind_rows_A", "bind_cols_B", "sumcheck_rounds")
 
@@ -101,6 +103,14 @@ def lib() -> ctypes.CDLL:
     L.imm_ldd_tail_fraction.argtypes = [vp, vp, i64, ctypes.c_double, ctypes.c_double, vp, vp, vp]
     L.imm_sumcheck_verify.restype = ci
     L.imm_sumcheck_verify.argtypes = [vp, ci, u64, u64, vp, vp, vp, vp]
+    L.imm_sumcheck_batched_transcript_len.restype = i64
+    L.imm_sumcheck_batched_transcript_len.argtypes = [ci, ci]
+    L.imm_sumcheck_matmul_batched_workspace.restype = sz
+    L.imm_sumcheck_matmul_batched_workspace.argtypes = [vp, ci]
+    L.imm_sumcheck_matmul_prove_batched.restype = ci
+    L.imm_sumcheck_matmul_prove_batched.argtypes = [vp, ci, u64, u64, vp, vp, vp, sz, vp]
+    L.imm_sumcheck_verify_batched.restype = ci
+    L.imm_sumcheck_verify_batched.argtypes = [vp, ci, ci, u64, u64, vp, vp]
     _lib = L
     return L
 
@@ -338,6 +348,71 @@ def sumcheck_verify(transcript: Sequence[int], nrounds: int, seed: int, proof_id
     rc = lib().imm_sumcheck_verify(ctypes.addressof(arr), nrounds, seed, proof_id, opt(expect_c0),
                                    opt(expect_a_fin), opt(expect_b_fin), ctypes.addressof(fail))
     _check(rc, "imm_sumcheck_verify")
+    return rc, fail.value
+
+
+# ------------------------------------------------------------------ batched proof
+
+
+def batched_transcript_len(nrounds: int, nproofs: int) -> int:
+    return lib().imm_sumcheck_batched_transcript_len(nrounds, nproofs)
+
+
+class BatchedProver:
+    """One sumcheck for a random linear combination of product claims whose k pad to the same
+    power of two.  Holds descriptors, workspace and outputs; ``prove`` allocates nothing."""
+
+    def __init__(self, problems, device="cuda"):
+        self.problems = list(problems)
+        self.descs = make_descs(self.problems)
+        self.nproofs = len(self.problems)
+        self.nrounds = ceil_log2(self.problems[0][0].shape[1])
+        need = lib().imm_sumcheck_matmul_batched_workspace(ctypes.addressof(self.descs), self.nproofs)
+        if need == 0:
+            raise ImmError(ERR_SHAPE, "imm_sumcheck_matmul_batched_workspace")
+        self.ws = torch.empty(need, dtype=torch.uint8, device=device)
+        self.length = batched_transcript_len(self.nrounds, self.nproofs)
+        self.transcript = torch.zeros((self.length,), dtype=torch.int64, device=device)
+        self.status = torch.full((self.nproofs,), -99, dtype=torch.int32, device=device)
+
+    def prove(self, seed: int, batch_id: int) -> torch.Tensor:
+        """Enqueue one batched proving pass on the current stream; returns the device transcript."""
+        _check(lib().imm_sumcheck_matmul_prove_batched(ctypes.addressof(self.descs), self.nproofs, seed,
+                                                       batch_id, self.transcript.data_ptr(),
+                                                       self.status.data_ptr(), self.ws.data_ptr(),
+                                                       self.ws.numel(), _stream()),
+               "imm_sumcheck_matmul_prove_batched")
+        return self.transcript
+
+
+def sumcheck_matmul_prove_batched(problems, seed: int, batch_id: int) -> List[int]:
+    """Convenience: one batched proof as Python ints (synchronises)."""
+    pr = BatchedProver(problems)
+    t = pr.prove(seed, batch_id)
+    torch.cuda.synchronize()
+    if int(pr.status.abs().max()) != 0:
+        raise ImmError(int(pr.status.min()), "device status")
+    return [int(v) & 0xFFFFFFFFFFFFFFFF for v in t.cpu()]
+
+
+def sumcheck_verify_batched(transcript: Sequence[int], nrounds: int, nproofs: int, seed: int,
+                            batch_id: int, expect: Optional[Sequence[int]] = None) -> Tuple[int, int]:
+    """Host verifier of a batched transcript; returns (status, fail_at)."""
+    n = 1 + 3 * nrounds + 3 * nproofs
+    words = [int(v) & 0xFFFFFFFFFFFFFFFF for v in list(transcript)[:n]]
+    if len(words) != n:
+        raise ValueError("transcript too short")
+    arr = (ctypes.c_uint64 * n)(*words)
+    exp = None
+    if expect is not None:
+        if len(expect) != 3 * nproofs:
+            raise ValueError("expect must hold 3 words per proof")
+        exp = (ctypes.c_uint64 * (3 * nproofs))(*[int(v) & 0xFFFFFFFFFFFFFFFF for v in expect])
+    fail = ctypes.c_int(-2)
+    rc = lib().imm_sumcheck_verify_batched(ctypes.addressof(arr), nrounds, nproofs, seed, batch_id,
+                                           None if exp is None else ctypes.addressof(exp),
+                                           ctypes.addressof(fail))
+    _check(rc, "imm_sumcheck_verify_batched")
     return rc, fail.value
 
 

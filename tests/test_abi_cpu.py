@@ -34,7 +34,7 @@ def test_challenges_match_oracle(imm, oracle):
     rng = random.Random(1)
     for _ in range(200):
         seed, pid = rng.getrandbits(64), rng.getrandbits(64)
-        dom, idx = rng.choice((1, 2, 3)), rng.randrange(0, 40)
+        dom, idx = rng.choice((1, 2, 3, 4)), rng.randrange(0, 40)
         assert imm.challenge(seed, pid, dom, idx) == oracle.challenge(seed, pid, dom, idx)
     assert imm.challenge(1, 0, 1, 0) == 0x0F583436CC1AB29E
 
@@ -65,6 +65,36 @@ def test_host_verifier_matches_oracle_verifier(imm, oracle):
         imm.sumcheck_verify([oracle.P, 0, 0], 0, 1, 0)
 
 
+def test_batched_host_verifier_matches_oracle_verifier(imm, oracle):
+    rng = random.Random(3)
+    for shapes in ([(3, 8, 2), (2, 5, 4), (1, 7, 1)], [(2, 1, 2), (1, 1, 3)], [(4, 16, 4)]):
+        probs = []
+        for i, (m, k, n) in enumerate(shapes):
+            A = np.array([[rng.randint(-128, 127) for _ in range(k)] for _ in range(m)], dtype=np.int8)
+            B = np.array([[rng.randint(-128, 127) for _ in range(n)] for _ in range(k)], dtype=np.int8)
+            probs.append((A, B, (A.astype(np.int64) @ B.astype(np.int64)).astype(np.int32), 100 + i))
+        seed, bid, b, count = rng.getrandbits(64), rng.getrandbits(30), oracle.ceil_log2(shapes[0][1]), len(shapes)
+        t = [int(w) for w in oracle.sumcheck_matmul_prove_batched(probs, seed, bid)]
+        assert len(t) == imm.batched_transcript_len(b, count)
+        assert imm.sumcheck_verify_batched(t, b, count, seed, bid) == (imm.OK, -1)
+        assert imm.sumcheck_verify_batched(t, b, count, seed, bid, t[-3 * count:]) == (imm.OK, -1)
+        for pos in range(len(t)):
+            bad = list(t)
+            bad[pos] = (bad[pos] + 1 + rng.randrange(oracle.P - 1)) % oracle.P
+            got = imm.sumcheck_verify_batched(bad, b, count, seed, bid)
+            assert got == oracle.sumcheck_verify_batched(bad, b, count, seed, bid) and got[0] == imm.REJECT
+        for pos in range(3 * count):
+            exp = t[-3 * count:]
+            exp[pos] = (exp[pos] + 1) % oracle.P
+            got = imm.sumcheck_verify_batched(t, b, count, seed, bid, exp)
+            assert got == oracle.sumcheck_verify_batched(t, b, count, seed, bid, exp) == (imm.REJECT, b + 2 + pos)
+        assert imm.sumcheck_verify_batched(t, b, count, seed, bid + 1) == (imm.REJECT, b + 1)
+    with pytest.raises(imm.ImmError):
+        imm.sumcheck_verify_batched([oracle.P, 0, 0, 0], 0, 1, 1, 0)
+    assert imm.batched_transcript_len(12, 96) == 1 + 36 + 288
+    assert imm.batched_transcript_len(-1, 4) == 0 and imm.batched_transcript_len(3, 0) == 0
+
+
 def _desc_array(imm, shapes, base=0x10000):
     arr = (imm.MatmulDesc * len(shapes))()
     for i, (m, k, n) in enumerate(shapes):
@@ -89,6 +119,22 @@ def test_workspace_planner(imm):
     assert L.imm_sumcheck_matmul_host_arena(ctypes.addressof(d2), 2) > w2 + 512 * 4096 + 4096 * 4096
     assert L.imm_mle_workspace(0, 100, 100, 0) > 0 and L.imm_mle_workspace(2, 100, 100, 0) == 0
     assert L.imm_mle_workspace(1, 0, 100, 1) == 0
+
+
+def test_batched_workspace_and_validation(imm):
+    L = imm.lib()
+    d = _desc_array(imm, [(64, 4096, 64), (512, 3000, 4096)])         # both k pad to 2^12
+    plain = L.imm_sumcheck_matmul_workspace(ctypes.addressof(d), 2)
+    need = L.imm_sumcheck_matmul_batched_workspace(ctypes.addressof(d), 2)
+    assert need >= plain + 2 * 39 * 8 and need % 256 == 0
+    mixed = _desc_array(imm, [(64, 4096, 64), (64, 2048, 64)])
+    assert L.imm_sumcheck_matmul_batched_workspace(ctypes.addressof(mixed), 2) == 0
+    prove = L.imm_sumcheck_matmul_prove_batched
+    assert prove(ctypes.addressof(mixed), 2, 1, 1, 0x1000, 0x1000, 0x1000, 1 << 30, None) == imm.ERR_SHAPE
+    assert prove(ctypes.addressof(d), 2, 1, 1, 0x1000, 0x1000, 0x1000, need - 1, None) == imm.ERR_WORKSPACE
+    assert prove(ctypes.addressof(d), 2, 1, 1, 0x1000, 0x1000, 0x1010, need, None) == imm.ERR_ALIGN
+    assert prove(ctypes.addressof(d), 2, 1, 1, None, 0x1000, 0x1000, need, None) == imm.ERR_ARG
+    assert prove(ctypes.addressof(d), 0, 1, 1, 0x1000, 0x1000, 0x1000, need, None) == imm.ERR_ARG
 
 
 def test_argument_validation_happens_before_any_device_work(imm):

@@ -6,7 +6,9 @@ shares no code with the CUDA library.
 * the Goldilocks sumcheck matmul proof: ``imm_oracle.c`` (plain C, ``% p`` on 128-bit integers)
   wrapped through ctypes and re-exported here; its header lists the conventions and the pins;
 * the logit distance distribution (TV / KL distances, Top-K distance, the per-request tail
-  statistic): ``oracle.ldd`` (plain numpy in float64); its header lists the readings and the pins.
+  statistic): ``oracle.ldd`` (plain numpy in float64); its header lists the readings and the pins;
+* the hash commitment (SHA-256 Merkle tree, ``hashlib`` as the library step): ``oracle.commitment``.
 """
+from . import commit_oracle as commitment  # noqa: F401
 from . import ldd_oracle as ldd  # noqa: F401
 from .imm_oracle import *  # noqa: F401,F403

@@ -282,6 +282,49 @@ int imm_sumcheck_verify_batched(const imm_fe* transcript_host, int nrounds, int 
                                 uint64_t batch_id, const imm_fe* expect_host, int* fail_at);
 
 /* ---------------------------------------------------------------------------------------------
+ * Hash commitments
+ * ---------------------------------------------------------------------------------------------
+ * c = Hash(m || r) (Section 2.1, cryptographic commitment): the server's commitment to the model
+ * and, under fresh randomness r, to the logits of a response (Algorithm 1); the auditor recomputes
+ * both (first check of the auditing algorithm).  The paper names no hash; here
+ *   Hash  = SHA-256 (FIPS 180-4) in a tree mode, so that a message of gigabytes hashes in parallel:
+ *   root  = Merkle tree hash of RFC 6962, Section 2.1, over the message cut into
+ *           IMM_COMMIT_LEAF-byte pieces (the last may be shorter; an empty message is one empty
+ *           piece): leaf = SHA-256(0x00 || piece), node = SHA-256(0x01 || left || right), the split
+ *           of n pieces at the largest power of two below n;
+ *   c     = SHA-256(0x02 || root || le64(nbytes) || r), r = 32 bytes, or none for a commitment
+ *           that hides nothing (the model's).
+ * Digests are the usual 32-byte big-endian serialisation. */
+#define IMM_COMMIT_LEAF 4096
+#define IMM_COMMIT_MAX_MESSAGES (1 << 20)
+#define IMM_COMMIT_MAX_BYTES (1ull << 40)
+
+typedef struct {
+    const void* msg;        /* DEVICE pointer to nbytes contiguous bytes (may be NULL when nbytes = 0) */
+    uint64_t nbytes;
+    uint8_t r[32];          /* the commitment's randomness (read when r_len = 32) */
+    int32_t r_len;          /* 0 or 32 */
+    int32_t reserved;       /* set to 0 */
+} imm_commit_desc;
+
+/* Workspace bytes imm_commit needs for this batch (0 on invalid input). */
+size_t imm_commit_workspace(const imm_commit_desc* descs_host, int n);
+
+/* Commits to every message of the batch.
+ *   descs_host : HOST array of n descriptors (at most IMM_COMMIT_MAX_MESSAGES, each message at
+ *                most IMM_COMMIT_MAX_BYTES)
+ *   d_digests  : DEVICE array of n x 32 bytes: the commitments c
+ *   d_roots    : DEVICE array of n x 32 bytes for the tree roots, or NULL
+ *   d_ws       : DEVICE workspace, 256-byte aligned, >= imm_commit_workspace(...) bytes
+ * Messages whose pointer is 16-byte aligned are read with 128-bit loads, others byte by byte
+ * (slow).  The batch is one leaf launch (one thread per leaf; the 128 leaves of a block fold to a
+ * subtree root on chip), one launch per further factor of 1024 in the largest leaf count, and a
+ * final launch; all are enqueued on `stream`, nothing is synchronised or allocated.
+ * Errors: IMM_ERR_ARG, IMM_ERR_LIMIT, IMM_ERR_ALIGN, IMM_ERR_WORKSPACE, IMM_ERR_CUDA. */
+int imm_commit(const imm_commit_desc* descs_host, int n, uint8_t* d_digests, uint8_t* d_roots,
+               void* d_ws, size_t ws_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
  * Logit distance distribution (LDD)
  * ---------------------------------------------------------------------------------------------
  * The auditing footprint of the paper: for every discrete decision of an audited request, the

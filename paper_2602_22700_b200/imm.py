@@ -32,7 +32,9 @@ EXPORTS = ("imm_version", "imm_last_cuda_error", "imm_challenge", "imm_field_bin
            "imm_profile_enable", "imm_profile_calls", "imm_profile_read", "imm_mle_eval_point_noalloc",
            "imm_ldd_tv_kl", "imm_ldd_topk_workspace", "imm_ldd_topk_distance", "imm_ldd_tail_fraction",
            "imm_sumcheck_batched_transcript_len", "imm_sumcheck_matmul_batched_workspace",
-           "imm_sumcheck_matmul_prove_batched", "imm_sumcheck_verify_batched")
+           "imm_sumcheck_matmul_prove_batched", "imm_sumcheck_verify_batched",
+           "imm_commit_workspace", "imm_commit")
+COMMIT_LEAF = 4096
 NOALLOC_MAX_TILES = 8192
 PROFILE_PHASES = ("eq_tables", "claim_C", "bind_rows_A", "bind_cols_B", "sumcheck_rounds")
 
@@ -41,6 +43,11 @@ class ImmError(RuntimeError):
     def __init__(self, code: int, where: str, detail: str = ""):
         self.code = code
         super().__init__(f"{where}: {ERRORS.get(code, code)}" + (f" ({detail})" if detail else ""))
+
+
+class CommitDesc(ctypes.Structure):
+    _fields_ = [("msg", ctypes.c_void_p), ("nbytes", ctypes.c_uint64), ("r", ctypes.c_uint8 * 32),
+                ("r_len", ctypes.c_int32), ("reserved", ctypes.c_int32)]
 
 
 class MatmulDesc(ctypes.Structure):
@@ -109,6 +116,10 @@ def lib() -> ctypes.CDLL:
     L.imm_sumcheck_matmul_batched_workspace.argtypes = [vp, ci]
     L.imm_sumcheck_matmul_prove_batched.restype = ci
     L.imm_sumcheck_matmul_prove_batched.argtypes = [vp, ci, u64, u64, vp, vp, vp, sz, vp]
+    L.imm_commit_workspace.restype = sz
+    L.imm_commit_workspace.argtypes = [vp, ci]
+    L.imm_commit.restype = ci
+    L.imm_commit.argtypes = [vp, ci, vp, vp, vp, sz, vp]
     L.imm_sumcheck_verify_batched.restype = ci
     L.imm_sumcheck_verify_batched.argtypes = [vp, ci, ci, u64, u64, vp, vp]
     _lib = L
@@ -414,6 +425,60 @@ def sumcheck_verify_batched(transcript: Sequence[int], nrounds: int, nproofs: in
                                            ctypes.addressof(fail))
     _check(rc, "imm_sumcheck_verify_batched")
     return rc, fail.value
+
+
+# ------------------------------------------------------------------ hash commitments
+
+
+class Committer:
+    """Commitments c = Hash(m || r) to a batch of CUDA tensors (each tensor's bytes, which must be
+    contiguous, are one message).  Holds descriptors, workspace and outputs; ``commit`` allocates
+    nothing.  ``randomness``: None (no r for any message) or one 32-byte string (or None) per message."""
+
+    def __init__(self, messages, randomness=None, device="cuda"):
+        self.messages = list(messages)
+        n = len(self.messages)
+        if randomness is None:
+            randomness = [None] * n
+        if len(randomness) != n:
+            raise ValueError("one randomness entry per message")
+        self.descs = (CommitDesc * max(n, 1))()
+        self.nbytes = 0
+        for i, (t, r) in enumerate(zip(self.messages, randomness)):
+            if not isinstance(t, torch.Tensor) or t.device.type != "cuda":
+                raise ValueError("messages must be CUDA tensors (no CPU path exists)")
+            if not t.is_contiguous():
+                raise ValueError("a message must be contiguous")
+            size = t.numel() * t.element_size()
+            self.descs[i].msg = t.data_ptr() if size else None
+            self.descs[i].nbytes = size
+            self.nbytes += size
+            if r is not None:
+                if len(r) != 32:
+                    raise ValueError("randomness must be 32 bytes")
+                self.descs[i].r = (ctypes.c_uint8 * 32)(*bytes(r))
+                self.descs[i].r_len = 32
+        self.n = n
+        need = lib().imm_commit_workspace(ctypes.addressof(self.descs), n)
+        if need == 0:
+            raise ImmError(ERR_ARG, "imm_commit_workspace")
+        self.ws = torch.empty(need, dtype=torch.uint8, device=device)
+        self.digests = torch.zeros((n, 32), dtype=torch.uint8, device=device)
+        self.roots = torch.zeros((n, 32), dtype=torch.uint8, device=device)
+
+    def commit(self) -> torch.Tensor:
+        """Enqueue the commitments on the current stream; returns the (n, 32) device tensor of digests."""
+        _check(lib().imm_commit(ctypes.addressof(self.descs), self.n, self.digests.data_ptr(),
+                                self.roots.data_ptr(), self.ws.data_ptr(), self.ws.numel(), _stream()),
+               "imm_commit")
+        return self.digests
+
+
+def commit(messages, randomness=None) -> List[bytes]:
+    """Convenience: commitments as bytes objects (synchronises)."""
+    c = Committer(messages, randomness)
+    d = c.commit().cpu().numpy()
+    return [bytes(row) for row in d]
 
 
 # ------------------------------------------------------------------ logit distance distribution

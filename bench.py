@@ -70,6 +70,8 @@ WORKLOADS = {
     "ffn": (2048, "dense FFN up/down pair: {tokens}x4096 times 4096x14336, requantised hidden times 14336x4096, two proofs"),
     "moe": (4096, "MoE expert batch: 8 experts 4096x14336, top-2 routing of {tokens} tokens, one proof per expert"),
     "attn": (2048, "attention products: {layers} layers x 32 heads x (Q K^T with k = 128, P V with k = {tokens}), {tokens} tokens, one proof per product"),
+    "commit": (8192, "response commitments: {tokens} decision steps x vocabulary {vocab} (float32 logits) cut into "
+                     "{tokens}/128 requests of uneven length, one SHA-256 tree commitment per request"),
     "ldd": (8192, "logit distance distribution: {tokens} decision steps x vocabulary {vocab} (float32), TV + KL + Top-{topk} distance + tail statistic"),
 }
 L2_BYTES = 126 << 20
@@ -202,6 +204,12 @@ def measured_peaks():
 # profiles/ (dram__bytes_read.sum + dram__bytes_write.sum over 4*m*n); None until a capture of the
 # current kernel exists.
 LDD_TVKL_TRAFFIC_RATIO = 1.0721 / 1.050673   # tv_kl_kernel<aligned, 512 threads>: (dram read + write) / (8 bytes per entry pair)
+COMMIT_TRAFFIC_RATIO = (1.070806 + 0.018732) / 1.050673152                   # commit_leaf_kernel: (dram read + write) / message bytes
+# SHA-256 leaf hashing against the integer ALU pipe (rotates, three-input logic, byte permutes): the
+# pipe retires 64 thread instructions per cycle per SM; the kernel issues 17.55 of them per hashed
+# byte (ncu: 576.3 M warp instructions on that pipe for 1.0507 GB), so at 1965 MHz the pipe allows
+# 148 x 64 x 1.965e9 / 17.55 = 1060 GB/s.
+COMMIT_ALU_PEAK_GBS_AT_1965 = 1060.0
 CLAIM_KERNEL_TRAFFIC_RATIO = 239.64 / 234.881024  # bytedot_kernel<1,1,1>: (dram read + write) / (4 bytes per entry), small-case capture
 
 
@@ -534,6 +542,132 @@ def run_ldd(args):
     rep.close()
 
 
+# ------------------------------------------------------------------------ hash commitments
+
+
+def commit_workload(imm, synth, seed, T, n, dev):
+    """Deployed logits of T decision steps cut into requests; one message and one 32-byte r per request."""
+    ref = synth.reference_logits(seed, T, n, device=dev)
+    dep = synth.deployed_logits(ref, seed, synth.NOISE_BENIGN)
+    del ref
+    requests = max(1, T // 128)
+    off = synth.request_offsets(seed, T, requests, device="cpu").tolist()
+    msgs = [dep[off[i]:off[i + 1]] for i in range(requests)]
+    rs = [bytes((7 * i + j) & 255 for j in range(32)) for i in range(requests)]
+    return dep, off, msgs, rs
+
+
+def run_commit(args):
+    """One step = the commitment psi = Hash(r, logits) of every request of the batch."""
+    from paper_2602_22700_b200 import imm, synth
+    from paper_2602_22700_b200.replicas import Replicas
+    rank, local_rank, world = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    rep = Replicas("nccl", dev)
+    imm.lib()
+    warmup, steps = max(args.warmup, 3), max(args.steps, 1)
+    T, n = args.tokens, args.vocab
+    dep, off, msgs, rs = commit_workload(imm, synth, rep.seed(SEED), T, n, dev)
+    nbytes = dep.numel() * 4
+    com = imm.Committer(msgs, rs, device=dev)
+    barrier = rep.barrier
+    for _ in range(warmup):
+        com.commit()
+    barrier()
+    sampler = ClockSampler(local_rank if "CUDA_VISIBLE_DEVICES" not in os.environ else
+                           int(os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local_rank]))
+    sampler.start()
+    time.sleep(0.25)
+    flush = nbytes < 2 * L2_BYTES
+    scrub = torch.empty(512 << 20, dtype=torch.uint8, device=dev) if flush else None
+    pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    t0 = time.time()
+    for a, b in pairs:
+        if flush:
+            scrub.fill_(1)
+        a.record()
+        com.commit()
+        b.record()
+    barrier()
+    t1w = time.time()
+    clocks = sampler.stop(t0, t1w)
+    elapsed_ms = rep.max_over_ranks(sum(a.elapsed_time(b) for a, b in pairs))
+    ms_per_step = elapsed_ms / steps
+    digests = com.digests.cpu().numpy()
+    gbs = nbytes / (ms_per_step * 1e-3) / 1e9
+    sm_mhz = clocks.get("sm_mhz") or 1965.0
+    alu_peak = COMMIT_ALU_PEAK_GBS_AT_1965 * sm_mhz / 1965.0
+    res = {
+        "metric": "committed bytes/sec", "value": nbytes * world / (ms_per_step * 1e-3), "unit": "B/s",
+        "n_gpus": world, "steps": steps, "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "u32", "data": "synthetic",
+        "config": {"workload": workload_name("commit", 0, T, n), "tokens": T, "vocab": n, "requests": len(msgs),
+                   "hash": "SHA-256, RFC 6962 tree over 4096-byte leaves, length-bound final hash with 32-byte r",
+                   "input_bytes_per_gpu": nbytes,
+                   "l2": ("L2 flushed between steps (512 MB overwritten outside the timed event pairs)" if flush else
+                          f"inputs ({nbytes / 2**30:.2f} GiB) exceed the 126 MB L2 many times over; no flush"),
+                   "parallelism": "1 GPU" if world == 1 else f"{world} independent replicas, no collective"},
+        "hbm_gbs_whole_step": gbs,
+        "roofline": {"kernel": "commit_leaf_kernel (SHA-256 of 4096-byte leaves, one per thread); timed as the whole imm_commit "
+                               "call, of which the leaf kernel is 96 % in the launch list", "bound": "alu",
+                     "achieved": gbs, "peak": alu_peak, "unit": "GB/s", "frac": gbs / alu_peak,
+                     "peak_kind": "integer ALU pipe: 148 SMs x 64 lanes x sampled SM clock / 17.55 ALU instructions per hashed byte",
+                     "traffic": (COMMIT_TRAFFIC_RATIO * nbytes) if COMMIT_TRAFFIC_RATIO else None},
+        "gpu_launches": com.launches * steps,
+        "clocks": clocks,
+    }
+    e2e = None
+    if not args.no_e2e:
+        host = torch.empty(dep.shape, dtype=dep.dtype, pin_memory=True).copy_(dep)
+        stage = torch.empty_like(dep)
+        smsgs = [stage[off[i]:off[i + 1]] for i in range(len(msgs))]
+        com2 = imm.Committer(smsgs, rs, device=dev)
+        out = torch.empty((len(msgs), 32), dtype=torch.uint8, pin_memory=True)
+        torch.cuda.synchronize()
+
+        def e2e_pass():
+            stage.copy_(host, non_blocking=True)
+            out.copy_(com2.commit(), non_blocking=True)
+            torch.cuda.synchronize()
+
+        e2e_pass()
+        barrier()
+        k2 = max(1, args.e2e_steps)
+        w0 = time.perf_counter()
+        for _ in range(k2):
+            e2e_pass()
+        e2e_s = rep.max_over_ranks((time.perf_counter() - w0) / k2)
+        e2e = {"value": nbytes * world / e2e_s, "unit": "B/s", "ms_per_step": e2e_s * 1e3, "steps": k2,
+               "h2d_bytes_per_step": nbytes, "d2h_bytes_per_step": out.numel(),
+               "matches_device_path": bool((out.numpy() == digests).all())}
+        del host, stage, com2
+    res["e2e"] = e2e
+    if not args.no_cpu_baseline and world == 1:
+        from oracle import commitment
+        pick, total = [], 0
+        for i in sorted(range(len(msgs)), key=lambda i: msgs[i].numel()):
+            if total + msgs[i].numel() * 4 > (6 << 30) and pick:
+                break
+            pick.append(i)
+            total += msgs[i].numel() * 4
+        data = {i: msgs[i].cpu().numpy().tobytes() for i in pick}
+        w0 = time.perf_counter()
+        want = {i: commitment.commit(data[i], rs[i]) for i in pick}
+        secs = time.perf_counter() - w0
+        ok = all(bytes(digests[i]) == want[i] for i in pick)
+        res["cpu_baseline"] = {"value": total / secs, "unit": "B/s", "cores": 1, "kind": "oracle", "seconds": secs,
+                               "sample": f"{len(pick)} of the {len(msgs)} requests ({total} bytes), same inputs as the GPU run",
+                               "gpu_matches_oracle": ok}
+        if not ok:
+            raise SystemExit("GPU commitments differ from the oracle")
+    if rank == 0:
+        print(json.dumps(res))
+    rep.close()
+
+
 # ------------------------------------------------------------------------ reference arm (CPU oracle)
 
 
@@ -567,6 +701,30 @@ def run_reference(args):
             "e2e": {"value": rows / per, "unit": "steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         }))
         return
+    if args.config == "commit":
+        from oracle import commitment
+        rows = 256
+        ref = synth.reference_logits(SEED, rows, args.vocab, device=device)
+        data = synth.deployed_logits(ref, SEED, synth.NOISE_BENIGN).cpu().numpy().tobytes()
+        r = bytes(range(32))
+        warmup, steps = max(args.warmup, 1), max(args.steps, 1)
+        for _ in range(warmup):
+            commitment.commit(data[:1 << 20], r)
+        w0 = time.perf_counter()
+        for _ in range(steps):
+            commitment.commit(data, r)
+        per = (time.perf_counter() - w0) / steps
+        desc = f"one request of {rows} decision steps ({len(data)} bytes) per step, one thread"
+        print(json.dumps({
+            "impl": "reference", "metric": "committed bytes/sec", "value": len(data) / per, "unit": "B/s",
+            "n_gpus": world, "steps": steps, "warmup": warmup, "ms_per_step": per * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "u32", "data": "synthetic",
+            "config": {"workload": workload_name("commit", 0, args.tokens, args.vocab), "tokens": args.tokens,
+                       "vocab": args.vocab, "sampled": desc},
+            "cpu_baseline": {"value": len(data) / per, "unit": "B/s", "cores": 1, "kind": "oracle", "sample": desc},
+            "e2e": {"value": len(data) / per, "unit": "B/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        }))
+        return
     layers = min(args.layers, 2)
     tokens = args.tokens if device == "cuda" else min(args.tokens, 256)
     problems = make_problems(args.config, SEED, layers, tokens, device)[:8]
@@ -589,8 +747,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world,
         "steps": steps, "warmup": warmup, "ms_per_step": per * 1e3, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "u64", "data": "synthetic",
-        "config": {"workload": workload_name(args.config, args.layers, args.tokens) +
-                               (f", as {calls_per_step} batched proofs (one per round count)" if args.batched else ""),
+        "config": {"workload": workload_name(args.config, args.layers, args.tokens),
                    "layers": args.layers if args.config == "decoder" else None,
                    "tokens": args.tokens, "sampled": desc,
                    "note": None if tokens == args.tokens else "no CUDA device for input generation: token count reduced"},
@@ -607,6 +764,8 @@ def main():
         run_reference(args)
     elif args.config == "ldd":
         run_ldd(args)
+    elif args.config == "commit":
+        run_commit(args)
     else:
         run_ours(args)
 

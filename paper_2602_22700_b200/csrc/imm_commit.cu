@@ -9,7 +9,9 @@
 // c = H(0x02 || root || le64(length) || r).
 //
 // SHA-256 is a serial chain of 32-bit adds, rotates and three-input logic per 64-byte block, so
-// the work is bound by integer-pipe instruction issue, not by HBM.  One thread hashes one leaf
+// the work is bound by integer-pipe instruction issue, not by HBM: the rotates and the logic fill
+// the integer ALU pipe (one warp instruction per two cycles per SM sub-partition); the adds are
+// written as multiply-adds so that they issue on the other pipe.  One thread hashes one leaf
 // (65 compressions); the 128 leaves of a block are then folded to one subtree root in shared
 // memory, so the leaf digests never go to global memory.  Later passes fold 1024 digests per block
 // until every message has one root, and a last launch forms the commitments.
@@ -49,32 +51,55 @@ __device__ __forceinline__ void iv(uint32_t (&h)[8])    // FIPS 180-4, 5.3.3: sq
     h[4] = 0x510e527fu; h[5] = 0x9b05688cu; h[6] = 0x1f83d9abu; h[7] = 0x5be0cd19u;
 }
 
+// a + b on the multiply-add pipe: a * one + b with `one` a register the compiler cannot see through
+// (it holds 1).  The rotates and three-input logic of SHA-256 fill the integer ALU pipe, which
+// issues at half rate; the adds, written as multiply-adds, run beside them on the other pipe.
+__device__ __forceinline__ uint32_t add_m(uint32_t a, uint32_t b, uint32_t one)
+{
+    uint32_t d;
+    asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(one), "r"(b));
+    return d;
+}
+
+// One round (FIPS 180-4, 6.2.2, step 3) on the working variables, with w + K already added.
+#define IMM_SHA_ROUND(kw)                                                          \
+    do {                                                                           \
+        const uint32_t S1 = rotr(e, 6) ^ rotr(e, 11) ^ rotr(e, 25);                \
+        const uint32_t ch = (e & f) ^ (~e & g);                                    \
+        const uint32_t t1 = add_m(add_m(add_m(hh, (kw), one), ch, one), S1, one);  \
+        const uint32_t S0 = rotr(a, 2) ^ rotr(a, 13) ^ rotr(a, 22);                \
+        const uint32_t maj = (a & b) ^ (a & c) ^ (b & c);                          \
+        hh = g; g = f; f = e; e = add_m(d, t1, one);                               \
+        d = c; c = b; b = a; a = add_m(add_m(S0, maj, one), t1, one);              \
+    } while (0)
+
 // One compression (FIPS 180-4, 6.2.2).  w holds the sixteen message words and is overwritten by
-// the rolling message schedule.
-__device__ __forceinline__ void compress(uint32_t (&h)[8], uint32_t (&w)[16])
+// the rolling message schedule.  `one` must hold 1 (see add_m).  Rounds 0..15 are straight-line
+// code; rounds 16..63 are three trips through one sixteen-round body, so that the whole function
+// stays small enough for the instruction caches close to the schedulers (fully unrolled, the
+// warps of an SM stream 24 KB of code per compression and stall on instruction fetch).
+__device__ __forceinline__ void compress(uint32_t (&h)[8], uint32_t (&w)[16], uint32_t one)
 {
     uint32_t a = h[0], b = h[1], c = h[2], d = h[3], e = h[4], f = h[5], g = h[6], hh = h[7];
 #pragma unroll
-    for (int t = 0; t < 64; t++) {
-        if (t >= 16) {
-            const uint32_t w15 = w[(t - 15) & 15], w2 = w[(t - 2) & 15];
+    for (int t = 0; t < 16; t++) IMM_SHA_ROUND(add_m(w[t], K[t], one));
+#pragma unroll 1
+    for (int base = 16; base < 64; base += 16) {
+#pragma unroll
+        for (int j = 0; j < 16; j++) {
+            const uint32_t w15 = w[(j + 1) & 15], w2 = w[(j + 14) & 15];
             const uint32_t s0 = rotr(w15, 7) ^ rotr(w15, 18) ^ (w15 >> 3);
             const uint32_t s1 = rotr(w2, 17) ^ rotr(w2, 19) ^ (w2 >> 10);
-            w[t & 15] = w[t & 15] + s0 + w[(t - 7) & 15] + s1;
+            w[j] = add_m(add_m(w[j], s0, one), add_m(w[(j + 9) & 15], s1, one), one);
+            IMM_SHA_ROUND(add_m(w[j], K[base + j], one));
         }
-        const uint32_t S1 = rotr(e, 6) ^ rotr(e, 11) ^ rotr(e, 25);
-        const uint32_t ch = (e & f) ^ (~e & g);
-        const uint32_t t1 = hh + S1 + ch + K[t] + w[t & 15];
-        const uint32_t S0 = rotr(a, 2) ^ rotr(a, 13) ^ rotr(a, 22);
-        const uint32_t maj = (a & b) ^ (a & c) ^ (b & c);
-        hh = g; g = f; f = e; e = d + t1;
-        d = c; c = b; b = a; a = t1 + S0 + maj;
     }
     h[0] += a; h[1] += b; h[2] += c; h[3] += d; h[4] += e; h[5] += f; h[6] += g; h[7] += hh;
 }
 
 // node = SHA-256(0x01 || left || right): 65 bytes, two compressions
-__device__ __forceinline__ void node_hash(const uint32_t (&l)[8], const uint32_t (&r)[8], uint32_t (&out)[8])
+__device__ __forceinline__ void node_hash(const uint32_t (&l)[8], const uint32_t (&r)[8], uint32_t (&out)[8],
+                                          uint32_t one)
 {
     uint32_t w[16];
     w[0] = 0x01000000u | (l[0] >> 8);
@@ -84,18 +109,18 @@ __device__ __forceinline__ void node_hash(const uint32_t (&l)[8], const uint32_t
 #pragma unroll
     for (int i = 1; i < 8; i++) w[8 + i] = (r[i - 1] << 24) | (r[i] >> 8);
     iv(out);
-    compress(out, w);
+    compress(out, w, one);
     w[0] = (r[7] << 24) | 0x00800000u;
 #pragma unroll
     for (int i = 1; i < 15; i++) w[i] = 0;
     w[15] = 65 * 8;
-    compress(out, w);
+    compress(out, w, one);
 }
 
 // A full leaf whose data is 16-byte aligned: SHA-256(0x00 || 4096 bytes), 65 compressions.  Message
 // word t of a block is the last byte of little-endian data word t-1 followed by the first three
 // bytes of data word t (the tag byte shifts everything by one).
-__device__ __forceinline__ void leaf_hash_full(const uint4* __restrict__ src, uint32_t (&h)[8])
+__device__ __forceinline__ void leaf_hash_full(const uint4* __restrict__ src, uint32_t (&h)[8], uint32_t one)
 {
     iv(h);
     uint32_t prev = 0;                         // the tag 0x00 in the top byte
@@ -110,19 +135,20 @@ __device__ __forceinline__ void leaf_hash_full(const uint4* __restrict__ src, ui
 #pragma unroll
         for (int t = 1; t < 16; t++) w[t] = __byte_perm(x[t - 1], x[t], 0x3456);
         prev = x[15];
-        compress(h, w);
+        compress(h, w, one);
     }
     uint32_t w[16];
     w[0] = (prev & 0xFF000000u) | 0x00800000u;
 #pragma unroll
     for (int i = 1; i < 15; i++) w[i] = 0;
     w[15] = (LEAF + 1) * 8;
-    compress(h, w);
+    compress(h, w, one);
 }
 
 // Any leaf, byte by byte: SHA-256(0x00 || len bytes), len in [0, LEAF].  Used for the short last
 // leaf of a message and for messages that are not 16-byte aligned.
-__device__ __noinline__ void leaf_hash_bytes(const uint8_t* __restrict__ p, uint32_t len, uint32_t (&h)[8])
+__device__ __noinline__ void leaf_hash_bytes(const uint8_t* __restrict__ p, uint32_t len, uint32_t (&h)[8],
+                                             uint32_t one)
 {
     iv(h);
     const uint32_t total = len + 1;                        // tag + data
@@ -143,20 +169,20 @@ __device__ __noinline__ void leaf_hash_bytes(const uint8_t* __restrict__ p, uint
             w[t] = v;
         }
         if (blk == nblocks - 1) w[15] = total * 8;         // (w[14], the high length word, is already 0)
-        compress(h, w);
+        compress(h, w, one);
     }
 }
 
 // Folds the `count` digests in sd (count <= blockDim.x) to one in sd[0]: neighbours pair level by
 // level, an unpaired last digest moves up unchanged.
-__device__ __forceinline__ void fold(Digest* sd, int count)
+__device__ __forceinline__ void fold(Digest* sd, int count, uint32_t one)
 {
     const int t = threadIdx.x;
     while (count > 1) {
         const int half = count >> 1;
         uint32_t out[8];
         const bool pair = t < half, lift = (count & 1) && t == half;
-        if (pair) node_hash(sd[2 * t].h, sd[2 * t + 1].h, out);
+        if (pair) node_hash(sd[2 * t].h, sd[2 * t + 1].h, out, one);
         else if (lift) {
 #pragma unroll
             for (int i = 0; i < 8; i++) out[i] = sd[count - 1].h[i];
@@ -180,7 +206,7 @@ struct PassJob {
     uint64_t nbytes;           // leaf pass
     uint64_t count;            // leaves / input digests
     uint32_t group0;
-    uint32_t pad_;
+    uint32_t one;              // 1: the multiplier of the multiply-add form of the adds (see add_m)
 };
 
 struct FinalJob {
@@ -188,7 +214,7 @@ struct FinalJob {
     uint64_t nbytes;
     uint8_t r[32];
     int32_t r_len;
-    int32_t pad_;
+    uint32_t one;              // 1 (see add_m)
 };
 
 __device__ __forceinline__ int find_pass_job(const PassJob* jobs, int njobs, uint32_t block)
@@ -217,13 +243,13 @@ __global__ void __launch_bounds__(LEAF_THREADS) commit_leaf_kernel(const PassJob
         const uint64_t off = leaf * LEAF;
         const uint64_t left = jb.nbytes - off;             // (an empty message: one leaf of length 0)
         uint32_t h[8];
-        if (left >= LEAF && ((uintptr_t)jb.msg & 15) == 0) leaf_hash_full((const uint4*)(jb.msg + off), h);
-        else leaf_hash_bytes(jb.msg + off, left < LEAF ? (uint32_t)left : LEAF, h);
+        if (left >= LEAF && ((uintptr_t)jb.msg & 15) == 0) leaf_hash_full((const uint4*)(jb.msg + off), h, jb.one);
+        else leaf_hash_bytes(jb.msg + off, left < LEAF ? (uint32_t)left : LEAF, h, jb.one);
 #pragma unroll
         for (int i = 0; i < 8; i++) sd[threadIdx.x].h[i] = h[i];
     }
     __syncthreads();
-    fold(sd, count);
+    fold(sd, count, jb.one);
     if (threadIdx.x < 8) jb.out[blockIdx.x - jb.group0].h[threadIdx.x] = sd[0].h[threadIdx.x];
 }
 
@@ -239,7 +265,7 @@ __global__ void __launch_bounds__(NODE_THREADS) commit_node_kernel(const PassJob
     const int count = remaining < NODE_THREADS ? (int)remaining : NODE_THREADS;
     if ((int)threadIdx.x < count) sd[threadIdx.x] = jb.in[first + threadIdx.x];
     __syncthreads();
-    fold(sd, count);
+    fold(sd, count, jb.one);
     if (threadIdx.x < 8) jb.out[blockIdx.x - jb.group0].h[threadIdx.x] = sd[0].h[threadIdx.x];
 }
 
@@ -264,6 +290,7 @@ __global__ void commit_final_kernel(const FinalJob* jobs, int njobs, uint8_t* di
     m[total] = 0x80;
     m[64 * nblocks - 2] = (uint8_t)((total * 8) >> 8);
     m[64 * nblocks - 1] = (uint8_t)(total * 8);
+    const uint32_t one = jb.one;
     uint32_t h[8];
     iv(h);
     for (int blk = 0; blk < nblocks; blk++) {
@@ -272,7 +299,7 @@ __global__ void commit_final_kernel(const FinalJob* jobs, int njobs, uint8_t* di
             const uint8_t* p = m + 64 * blk + 4 * t;
             w[t] = ((uint32_t)p[0] << 24) | ((uint32_t)p[1] << 16) | ((uint32_t)p[2] << 8) | p[3];
         }
-        compress(h, w);
+        compress(h, w, one);
     }
     for (int wd = 0; wd < 8; wd++)
         for (int q = 0; q < 4; q++) {
@@ -383,6 +410,7 @@ int imm_commit(const imm_commit_desc* descs_host, int n, uint8_t* d_digests, uin
             jb.nbytes = descs_host[e.msg].nbytes;
             jb.count = e.count;
             jb.group0 = g;
+            jb.one = 1;
             g += (uint32_t)e.groups;
         }
         blocks[ps] = g;
@@ -392,6 +420,7 @@ int imm_commit(const imm_commit_desc* descs_host, int n, uint8_t* d_digests, uin
         fj[i].root = (const Digest*)(digs + p.root_off[i]);
         fj[i].nbytes = descs_host[i].nbytes;
         fj[i].r_len = descs_host[i].r_len;
+        fj[i].one = 1;
         memcpy(fj[i].r, descs_host[i].r, 32);
     }
     if (cudaMemcpyAsync(base, hdr.data(), hdr.size(), cudaMemcpyHostToDevice, st) != cudaSuccess) return IMM_ERR_CUDA;

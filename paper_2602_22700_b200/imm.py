@@ -459,6 +459,13 @@ class Committer:
                 self.descs[i].r = (ctypes.c_uint8 * 32)(*bytes(r))
                 self.descs[i].r_len = 32
         self.n = n
+        # launches per call: the leaf pass, one node pass per factor of 1024 left in the largest count, the final hash
+        most = max([max(1, -(-int(d.nbytes) // COMMIT_LEAF)) for d in self.descs[:n]] + [1])
+        most = -(-most // 128)
+        self.launches = 2
+        while most > 1:
+            most = -(-most // 1024)
+            self.launches += 1
         need = lib().imm_commit_workspace(ctypes.addressof(self.descs), n)
         if need == 0:
             raise ImmError(ERR_ARG, "imm_commit_workspace")

@@ -1,0 +1,139 @@
+"""CPU oracle of the non-interactive (Fiat-Shamir) matmul proof -- TEST INFRASTRUCTURE ONLY (nothing
+on the product path may import this file; it shares no code or table with the CUDA library).
+
+What it instantiates.  Algorithm 1 of the paper has the server send a proof pi with its response:
+no verifier is on line to draw coins, so the public coins of the interactive sumcheck
+(``imm_oracle.c``) are replaced by hashes of everything sent so far -- the Fiat-Shamir transform.
+The paper fixes none of this; the readings below are this build's.
+
+  H           SHA-256 (``hashlib``, a library step).  Integers are little-endian; a field element is
+              the le64 of its canonical value.
+  fe(d)       the first 8 bytes of a digest as a big-endian integer v, minus p if v >= p.
+  s_0         H(0x10 || com_A || com_B || com_C || le64(m) || le64(k) || le64(n) || le64(proof_id)):
+              the statement -- the three 32-byte commitments (``commit_oracle``) and the shape.
+  points      r_row[t] = fe(H(0x11 || s_0 || le32(1) || le32(t))), r_col[t] likewise with le32(2).
+  claim       c0 = C~(r_row, r_col);  s_1 = H(0x12 || s_0 || le64(c0)).
+  round j     the prover sends g_j(0), g_j(1), g_j(2);
+              s_{j+2} = H(0x13 || s_{j+1} || le64(g_j(0)) || le64(g_j(1)) || le64(g_j(2)));
+              r_j = fe(s_{j+2}); both tables fold with r_j.
+  transcript  [c0, g_0(0..2), ..., g_{b-1}(0..2), a_fin, b_fin], as in the interactive proof.
+
+The field arithmetic of the steps (eq tables, the two partial evaluations, the claim) is the C
+oracle's, called through its binding; the rounds are written out here in Python integers.
+
+Pins (tests/test_oracle_fs.py): every challenge re-derived with a SHA-256 written from the standard;
+every round polynomial against exhaustive hypercube sums in big integers at those challenges;
+g_j(0)+g_j(1) = running claim and the final product; each challenge depends on everything before it
+(commitments, shape, proof id, c0, earlier rounds); the verifier accepts the honest transcript and
+rejects every single-word change.
+"""
+from __future__ import annotations
+
+import hashlib
+
+import numpy as np
+
+from . import imm_oracle as orc
+
+P = orc.P
+
+
+def _h(data: bytes) -> bytes:
+    return hashlib.sha256(data).digest()
+
+
+def _le64(v: int) -> bytes:
+    return int(v).to_bytes(8, "little")
+
+
+def _le32(v: int) -> bytes:
+    return int(v).to_bytes(4, "little")
+
+
+def fe(digest: bytes) -> int:
+    v = int.from_bytes(digest[:8], "big")
+    return v - P if v >= P else v
+
+
+def statement(coms, m: int, k: int, n: int, proof_id: int) -> bytes:
+    """s_0 from the three 32-byte commitments (com_A, com_B, com_C) and the shape."""
+    com_a, com_b, com_c = (bytes(c) for c in coms)
+    assert len(com_a) == len(com_b) == len(com_c) == 32
+    return _h(b"\x10" + com_a + com_b + com_c + _le64(m) + _le64(k) + _le64(n) + _le64(proof_id))
+
+
+def point(s0: bytes, domain: int, count: int):
+    return [fe(_h(b"\x11" + s0 + _le32(domain) + _le32(t))) for t in range(count)]
+
+
+def absorb_claim(s0: bytes, c0: int) -> bytes:
+    return _h(b"\x12" + s0 + _le64(c0))
+
+
+def absorb_round(s: bytes, g0: int, g1: int, g2: int) -> bytes:
+    return _h(b"\x13" + s + _le64(g0) + _le64(g1) + _le64(g2))
+
+
+def prove(A: np.ndarray, B: np.ndarray, C: np.ndarray, coms, proof_id: int):
+    """Transcript (list of ints) of the non-interactive proof of the claim C = A*B (C used as given)."""
+    m, k = A.shape
+    n = B.shape[1]
+    a, b, c = orc.ceil_log2(m), orc.ceil_log2(k), orc.ceil_log2(n)
+    s0 = statement(coms, m, k, n, proof_id)
+    e_row = orc.eq_table(point(s0, 1, a))
+    e_col = orc.eq_table(point(s0, 2, c))
+    av = [int(v) for v in orc.mle_partial_eval(A, orc.BIND_ROWS, e_row)] + [0] * ((1 << b) - k)
+    bv = [int(v) for v in orc.mle_partial_eval(B, orc.BIND_COLS, e_col)] + [0] * ((1 << b) - k)
+    c0 = orc.mle_eval_point(C, e_row, e_col)
+    out = [c0]
+    s = absorb_claim(s0, c0)
+    for j in range(b):
+        half = 1 << (b - 1 - j)
+        g0 = g1 = g2 = 0
+        for y in range(half):
+            a0, a1, b0, b1 = av[y], av[y + half], bv[y], bv[y + half]
+            g0 += a0 * b0
+            g1 += a1 * b1
+            g2 += (2 * a1 - a0) * (2 * b1 - b0)
+        g0, g1, g2 = g0 % P, g1 % P, g2 % P
+        out += [g0, g1, g2]
+        s = absorb_round(s, g0, g1, g2)
+        r = fe(s)
+        av = [(av[y] + r * (av[y + half] - av[y])) % P for y in range(half)]
+        bv = [(bv[y] + r * (bv[y + half] - bv[y])) % P for y in range(half)]
+    return out + [av[0], bv[0]]
+
+
+def challenges(transcript, nrounds: int, coms, m: int, k: int, n: int, proof_id: int):
+    """(r_row, r_col, r_k) as the verifier derives them from the statement and the transcript."""
+    s0 = statement(coms, m, k, n, proof_id)
+    r_row, r_col = point(s0, 1, orc.ceil_log2(m)), point(s0, 2, orc.ceil_log2(n))
+    s = absorb_claim(s0, transcript[0])
+    r_k = []
+    for j in range(nrounds):
+        s = absorb_round(s, *transcript[1 + 3 * j:4 + 3 * j])
+        r_k.append(fe(s))
+    return r_row, r_col, r_k
+
+
+def verify(transcript, nrounds: int, coms, m: int, k: int, n: int, proof_id: int, expect=None):
+    """(status, fail_at) with the interactive verifier's meaning of fail_at; ``expect`` is the
+    verifier's own (c0, a_fin, b_fin) or None."""
+    t = [int(w) for w in transcript]
+    if len(t) < 3 * nrounds + 3 or any(w >= P or w < 0 for w in t[:3 * nrounds + 3]):
+        return -5, -2
+    _, _, r_k = challenges(t, nrounds, coms, m, k, n, proof_id)
+    claim = t[0]
+    for j in range(nrounds):
+        g0, g1, g2 = t[1 + 3 * j:4 + 3 * j]
+        if (g0 + g1) % P != claim:
+            return orc.REJECT, j
+        claim = orc.interp_deg2(g0, g1, g2, r_k[j])
+    a_fin, b_fin = t[3 * nrounds + 1], t[3 * nrounds + 2]
+    if a_fin * b_fin % P != claim:
+        return orc.REJECT, nrounds
+    if expect is not None:
+        for i, (want, got) in enumerate(zip(expect, (t[0], a_fin, b_fin))):
+            if want is not None and want != got:
+                return orc.REJECT, nrounds + 1 + i
+    return orc.OK, -1

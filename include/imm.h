@@ -325,6 +325,50 @@ int imm_commit(const imm_commit_desc* descs_host, int n, uint8_t* d_digests, uin
                void* d_ws, size_t ws_bytes, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * Non-interactive proof (Fiat-Shamir)
+ * ---------------------------------------------------------------------------------------------
+ * Algorithm 1 has the server attach a proof pi to its response: no verifier is on line to draw
+ * coins, so the public coins of the proof above are replaced by hashes of everything sent so far.
+ * H = SHA-256; integers are little-endian; a field element is the le64 of its canonical value;
+ * fe(d) = the first 8 bytes of a digest as a big-endian integer, minus p if not below p.
+ *   s_0      = H(0x10 || com_A || com_B || com_C || le64(m) || le64(k) || le64(n) || le64(proof_id)),
+ *              com_X the 32-byte commitments to the three matrices (imm_commit);
+ *   r_row[t] = fe(H(0x11 || s_0 || le32(1) || le32(t))),  r_col[t] the same with le32(2);
+ *   s_1      = H(0x12 || s_0 || le64(c0));
+ *   round j:   s_{j+2} = H(0x13 || s_{j+1} || le64(g_j(0)) || le64(g_j(1)) || le64(g_j(2))),
+ *              r_j = fe(s_{j+2}).
+ * The transcript has the layout of the interactive proof (3b+3 words). */
+
+/* Workspace bytes imm_sumcheck_matmul_prove_fs needs (0 on invalid input). */
+size_t imm_sumcheck_matmul_fs_workspace(const imm_matmul_desc* descs_host, int nproofs);
+
+/* Non-interactive prover.  As imm_sumcheck_matmul_prove, but every challenge is hashed: one launch
+ * hashes the statements and derives r_row, r_col, and the round kernel (one block per proof) hashes
+ * each round's three values before it folds with the challenge they give.
+ *   d_commitments : DEVICE array, nproofs x 96 bytes: com_A || com_B || com_C of each proof
+ *   d_ws          : DEVICE workspace, 256-byte aligned, >= imm_sumcheck_matmul_fs_workspace(...)
+ * Other arguments and errors as imm_sumcheck_matmul_prove. */
+int imm_sumcheck_matmul_prove_fs(const imm_matmul_desc* descs_host, int nproofs, const uint8_t* d_commitments,
+                                 imm_fe* d_transcripts, int64_t stride, int32_t* d_status,
+                                 void* d_ws, size_t ws_bytes, void* stream);
+
+/* HOST.  The challenges of a non-interactive proof, as the verifier derives them: r_row
+ * (ceil(log2 m) values), r_col (ceil(log2 n)) from the statement, r_k (nrounds) from the statement
+ * and the transcript's first 3*nrounds+1 words.  Any output pointer may be NULL (transcript_host
+ * may be NULL when r_k_host is).  nrounds must equal ceil(log2 k).
+ * Returns IMM_OK, IMM_ERR_ARG, IMM_ERR_SHAPE or IMM_ERR_NONCANONICAL. */
+int imm_fs_challenges(const imm_fe* transcript_host, int nrounds, const uint8_t* commitments_host,
+                      int64_t m, int64_t k, int64_t n, uint64_t proof_id,
+                      imm_fe* r_row_host, imm_fe* r_col_host, imm_fe* r_k_host);
+
+/* HOST verifier of a non-interactive proof: the checks of imm_sumcheck_verify with the hashed round
+ * challenges; fail_at has the same meaning.  commitments_host: the 96 bytes of the statement.
+ * Returns IMM_OK, IMM_REJECT, IMM_ERR_ARG, IMM_ERR_SHAPE or IMM_ERR_NONCANONICAL. */
+int imm_sumcheck_verify_fs(const imm_fe* transcript_host, int nrounds, const uint8_t* commitments_host,
+                           int64_t m, int64_t k, int64_t n, uint64_t proof_id, const imm_fe* expect_c0,
+                           const imm_fe* expect_a_fin, const imm_fe* expect_b_fin, int* fail_at);
+
+/* ---------------------------------------------------------------------------------------------
  * Logit distance distribution (LDD)
  * ---------------------------------------------------------------------------------------------
  * The auditing footprint of the paper: for every discrete decision of an audited request, the

@@ -15,6 +15,7 @@
 #include "gl64.cuh"
 #include "imm_kernels.h"
 #include "imm_plan.h"
+#include "sha256.cuh"
 
 namespace {
 
@@ -619,8 +620,35 @@ size_t imm_sumcheck_matmul_workspace(const imm_matmul_desc* descs_host, int npro
 
 // The launch sequence of a batch.  shared_round_id: null = every proof draws its round challenges
 // under its own proof_id; else all proofs draw them under that one id (a batched proof).
+// fs: null = public coins from the generator; else the challenges are hashed from the commitments
+// and the transcript (non-interactive proof) and fs describes the extra device arrays.
+struct FsArgs {
+    const uint8_t* d_com;      // nproofs x 96 bytes
+    char* ext;                 // device region laid out by fs_layout
+};
+
+struct FsLayout {
+    size_t off_fs = 0, off_points = 0, off_state = 0, bytes = 0;
+    std::vector<size_t> off_tabs;
+};
+
+static FsLayout fs_layout(const imm_matmul_desc* descs, int nproofs)
+{
+    FsLayout L;
+    size_t off = align_up((size_t)nproofs * sizeof(FsProof));
+    L.off_points = off; off = align_up(off + (size_t)nproofs * 2 * FS_POINT_SLOTS * sizeof(imm_fe));
+    L.off_state = off;  off = align_up(off + (size_t)nproofs * 8 * sizeof(uint32_t));
+    L.off_tabs.resize(nproofs);
+    for (int i = 0; i < nproofs; i++) {
+        L.off_tabs[i] = off;
+        off = align_up(off + 2 * (sizeof(imm_fe) << ceil_log2(descs[i].k)));
+    }
+    L.bytes = off;
+    return L;
+}
+
 static int prove_batch(const imm_matmul_desc* descs_host, int nproofs, uint64_t seed,
-                       const uint64_t* shared_round_id, imm_fe* d_transcripts, int64_t stride,
+                       const uint64_t* shared_round_id, const FsArgs* fs, imm_fe* d_transcripts, int64_t stride,
                        int32_t* d_status, void* d_ws, size_t ws_bytes, void* stream)
 {
     if (!d_transcripts || !d_status || !d_ws) return IMM_ERR_ARG;
@@ -642,6 +670,12 @@ static int prove_batch(const imm_matmul_desc* descs_host, int nproofs, uint64_t 
     MatJob* jc = (MatJob*)(hdr.data() + p.off_jobs_c);
     EqTask* eq = (EqTask*)(hdr.data() + p.off_eq);
     const int acols = p.cols_a, bcols = p.cols_b, ccols = p.cols_c;
+    FsLayout fsl;
+    std::vector<FsProof> fsp;
+    if (fs) {
+        fsl = fs_layout(descs_host, nproofs);
+        fsp.assign(nproofs, FsProof{});
+    }
     uint32_t ta = 0, tb = 0, tc = 0;
     for (int i = 0; i < nproofs; i++) {
         const imm_matmul_desc& d = descs_host[i];
@@ -676,6 +710,7 @@ static int prove_batch(const imm_matmul_desc* descs_host, int nproofs, uint64_t 
             jb[i].wtab = (const uint32_t*)(base + q.w_cols_b);
             jc[i].wtab = (const uint32_t*)(base + q.w_cols_c);
         }
+        const imm_fe* pts = fs ? (const imm_fe*)(fs->ext + fsl.off_points) + (size_t)i * 2 * FS_POINT_SLOTS : nullptr;
         eq[2 * i] = EqTask{P.e_row, seed, d.proof_id, 1u, q.a,
                            p.mma ? (uint32_t*)(base + q.w_rows) : nullptr, nullptr, nullptr, (int32_t)d.m, 0,
                            p.mma ? (imm_fe*)(base + q.sum_row) : nullptr};
@@ -683,6 +718,18 @@ static int prove_batch(const imm_matmul_desc* descs_host, int nproofs, uint64_t 
                                p.mma ? (uint32_t*)(base + q.w_cols_b) : nullptr,
                                p.mma ? (uint32_t*)(base + q.w_cols_c) : nullptr, (int32_t)d.n, 0,
                                p.mma ? (imm_fe*)(base + q.sum_col) : nullptr};
+        if (fs) {
+            eq[2 * i].point = pts;
+            eq[2 * i + 1].point = pts + FS_POINT_SLOTS;
+            FsProof& F = fsp[i];
+            F.com = fs->d_com + (size_t)i * 96;
+            F.points = (imm_fe*)pts;
+            F.state = (uint32_t*)(fs->ext + fsl.off_state) + (size_t)i * 8;
+            F.ta = (imm_fe*)(fs->ext + fsl.off_tabs[i]);
+            F.tb = F.ta + ((size_t)1 << q.b);
+            F.proof_id = d.proof_id;
+            F.one = 1;
+        }
     }
     if (ta != p.tiles_a || tb != p.tiles_b || tc != p.tiles_c) return IMM_ERR_ARG;   // planner invariant
 
@@ -704,6 +751,10 @@ static int prove_batch(const imm_matmul_desc* descs_host, int nproofs, uint64_t 
     std::unique_lock<std::mutex> fork_lock;
     if (ss) fork_lock = std::unique_lock<std::mutex>(g_fork_mutex);
     CU(cudaMemcpyAsync(base, hdr.data(), hdr.size(), cudaMemcpyHostToDevice, st));
+    if (fs) {
+        CU(cudaMemcpyAsync(fs->ext + fsl.off_fs, fsp.data(), fsp.size() * sizeof(FsProof), cudaMemcpyHostToDevice, st));
+        CU(launch_fs_points((const ProofDev*)(base + p.off_proofs), (const FsProof*)(fs->ext + fsl.off_fs), nproofs, st));
+    }
     PROF_MARK(0, st);
     CU(launch_eq_batch((const EqTask*)(base + p.off_eq), 2 * nproofs, p.max_cover, st));
     PROF_MARK(1, st);
@@ -731,8 +782,12 @@ static int prove_batch(const imm_matmul_desc* descs_host, int nproofs, uint64_t 
         CU(cudaStreamWaitEvent(st, ss->join[1], 0));
     }
     PROF_MARK(8, st);
-    CU(launch_sumcheck((const ProofDev*)(base + p.off_proofs), nproofs, seed, d_transcripts, stride,
-                       d_status, p.max_b, env_int("IMM_SC_CLUSTER", 0), st));
+    if (fs)
+        CU(launch_sumcheck_fs((const ProofDev*)(base + p.off_proofs), (const FsProof*)(fs->ext + fsl.off_fs), nproofs,
+                              d_transcripts, stride, d_status, st));
+    else
+        CU(launch_sumcheck((const ProofDev*)(base + p.off_proofs), nproofs, seed, d_transcripts, stride,
+                           d_status, p.max_b, env_int("IMM_SC_CLUSTER", 0), st));
     PROF_MARK(9, st);
 #undef PROF_MARK
     if (prof) g_prof_calls++;
@@ -743,7 +798,8 @@ int imm_sumcheck_matmul_prove(const imm_matmul_desc* descs_host, int nproofs, ui
                               imm_fe* d_transcripts, int64_t stride, int32_t* d_status,
                               void* d_ws, size_t ws_bytes, void* stream)
 {
-    return prove_batch(descs_host, nproofs, seed, nullptr, d_transcripts, stride, d_status, d_ws, ws_bytes, stream);
+    return prove_batch(descs_host, nproofs, seed, nullptr, nullptr, d_transcripts, stride, d_status, d_ws, ws_bytes,
+                       stream);
 }
 
 // Batched proof: the per-proof transcripts (shared round challenges) go to the head of the
@@ -787,10 +843,160 @@ int imm_sumcheck_matmul_prove_batched(const imm_matmul_desc* descs_host, int npr
     if (ws_bytes < total) return IMM_ERR_WORKSPACE;
     imm_fe* d_rows = (imm_fe*)d_ws;
     const int64_t stride = 3 * b + 3;
-    rc = prove_batch(descs_host, nproofs, seed, &batch_id, d_rows, stride, d_status, (char*)d_ws + rows,
+    rc = prove_batch(descs_host, nproofs, seed, &batch_id, nullptr, d_rows, stride, d_status, (char*)d_ws + rows,
                      ws_bytes - rows, stream);
     if (rc != IMM_OK) return rc;
     CU(launch_combine(d_rows, stride, nproofs, b, seed, batch_id, d_transcript, (cudaStream_t)stream));
+    return IMM_OK;
+}
+
+}  // extern "C"
+
+// ------------------------------------------------------------------ non-interactive proof ---
+
+extern "C" {
+
+size_t imm_sumcheck_matmul_fs_workspace(const imm_matmul_desc* descs_host, int nproofs)
+{
+    Plan p = make_plan(descs_host, nproofs);
+    if (p.status != IMM_OK) return 0;
+    return fs_layout(descs_host, nproofs).bytes + p.total_bytes;
+}
+
+int imm_sumcheck_matmul_prove_fs(const imm_matmul_desc* descs_host, int nproofs, const uint8_t* d_commitments,
+                                 imm_fe* d_transcripts, int64_t stride, int32_t* d_status,
+                                 void* d_ws, size_t ws_bytes, void* stream)
+{
+    if (!d_commitments || !d_ws) return IMM_ERR_ARG;
+    Plan p = make_plan(descs_host, nproofs);
+    if (p.status != IMM_OK) return p.status;
+    if ((uintptr_t)d_ws % ALIGN != 0) return IMM_ERR_ALIGN;
+    const size_t ext = fs_layout(descs_host, nproofs).bytes;
+    if (ws_bytes < ext + p.total_bytes) return IMM_ERR_WORKSPACE;
+    FsArgs fs{d_commitments, (char*)d_ws};
+    return prove_batch(descs_host, nproofs, 0, nullptr, &fs, d_transcripts, stride, d_status, (char*)d_ws + ext,
+                       ws_bytes - ext, stream);
+}
+
+}  // extern "C"
+
+namespace {
+
+// host side of the transcript hashing (the same byte strings as the kernels')
+uint64_t fs_fe_host(const uint32_t (&h)[8])
+{
+    const uint64_t v = ((uint64_t)h[0] << 32) | h[1];
+    return v >= IMM_P ? v - IMM_P : v;
+}
+
+void put_le(uint8_t* dst, uint64_t v, int nbytes)
+{
+    for (int q = 0; q < nbytes; q++) dst[q] = (uint8_t)(v >> (8 * q));
+}
+
+void fs_absorb_host(uint32_t (&s)[8], uint8_t tag, const uint64_t* vals, int nvals)
+{
+    uint8_t m[64];
+    m[0] = tag;
+    imm_sha::digest_bytes(s, m + 1);
+    for (int i = 0; i < nvals; i++) put_le(m + 33 + 8 * i, vals[i], 8);
+    imm_sha::sha256_short(m, 33 + 8 * (uint32_t)nvals, s, 1);
+}
+
+void fs_statement_host(const uint8_t* com, int64_t m_, int64_t k, int64_t n, uint64_t proof_id, uint32_t (&s0)[8])
+{
+    uint8_t m[136];
+    m[0] = 0x10;
+    memcpy(m + 1, com, 96);
+    put_le(m + 97, (uint64_t)m_, 8);
+    put_le(m + 105, (uint64_t)k, 8);
+    put_le(m + 113, (uint64_t)n, 8);
+    put_le(m + 121, proof_id, 8);
+    imm_sha::sha256_short(m, 129, s0, 1);
+}
+
+uint64_t fs_point_host(const uint32_t (&s0)[8], uint32_t domain, uint32_t t)
+{
+    uint8_t m[48];
+    uint32_t h[8];
+    m[0] = 0x11;
+    imm_sha::digest_bytes(s0, m + 1);
+    put_le(m + 33, domain, 4);
+    put_le(m + 37, t, 4);
+    imm_sha::sha256_short(m, 41, h, 1);
+    return fs_fe_host(h);
+}
+
+int fs_check_shape(int64_t m, int64_t k, int64_t n, int nrounds)
+{
+    if (m <= 0 || k <= 0 || n <= 0 || m > MAX_EXTENT || n > MAX_EXTENT || k > MAX_K) return IMM_ERR_SHAPE;
+    if (nrounds != ceil_log2(k)) return IMM_ERR_SHAPE;
+    return IMM_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int imm_fs_challenges(const imm_fe* transcript_host, int nrounds, const uint8_t* commitments_host,
+                      int64_t m, int64_t k, int64_t n, uint64_t proof_id,
+                      imm_fe* r_row_host, imm_fe* r_col_host, imm_fe* r_k_host)
+{
+    if (!commitments_host) return IMM_ERR_ARG;
+    int rc = fs_check_shape(m, k, n, nrounds);
+    if (rc != IMM_OK) return rc;
+    uint32_t s[8];
+    fs_statement_host(commitments_host, m, k, n, proof_id, s);
+    if (r_row_host)
+        for (int t = 0; t < ceil_log2(m); t++) r_row_host[t] = fs_point_host(s, 1, (uint32_t)t);
+    if (r_col_host)
+        for (int t = 0; t < ceil_log2(n); t++) r_col_host[t] = fs_point_host(s, 2, (uint32_t)t);
+    if (r_k_host) {
+        if (!transcript_host) return IMM_ERR_ARG;
+        for (int i = 0; i < 3 * nrounds + 1; i++)
+            if (transcript_host[i] >= IMM_P) return IMM_ERR_NONCANONICAL;
+        fs_absorb_host(s, 0x12, transcript_host, 1);
+        for (int j = 0; j < nrounds; j++) {
+            fs_absorb_host(s, 0x13, transcript_host + 1 + 3 * j, 3);
+            r_k_host[j] = fs_fe_host(s);
+        }
+    }
+    return IMM_OK;
+}
+
+int imm_sumcheck_verify_fs(const imm_fe* transcript_host, int nrounds, const uint8_t* commitments_host,
+                           int64_t m, int64_t k, int64_t n, uint64_t proof_id, const imm_fe* expect_c0,
+                           const imm_fe* expect_a_fin, const imm_fe* expect_b_fin, int* fail_at)
+{
+    if (!transcript_host || !commitments_host || !fail_at) return IMM_ERR_ARG;
+    int rc = fs_check_shape(m, k, n, nrounds);
+    if (rc != IMM_OK) return rc;
+    const imm_fe* t = transcript_host;
+    for (int i = 0; i < 3 * nrounds + 3; i++)
+        if (t[i] >= IMM_P) return IMM_ERR_NONCANONICAL;
+    if ((expect_c0 && *expect_c0 >= IMM_P) || (expect_a_fin && *expect_a_fin >= IMM_P) ||
+        (expect_b_fin && *expect_b_fin >= IMM_P))
+        return IMM_ERR_NONCANONICAL;
+    uint64_t r_k[64];
+    rc = imm_fs_challenges(t, nrounds, commitments_host, m, k, n, proof_id, nullptr, nullptr, r_k);
+    if (rc != IMM_OK) return rc;
+    const uint64_t inv2 = 0x7FFFFFFF80000001ULL;
+    uint64_t claim = t[0];
+    for (int j = 0; j < nrounds; j++) {
+        const uint64_t g0 = t[1 + 3 * j], g1 = t[2 + 3 * j], g2 = t[3 + 3 * j];
+        if (gl::add(g0, g1) != claim) { *fail_at = j; return IMM_REJECT; }
+        const uint64_t r = r_k[j];
+        const uint64_t d1 = gl::sub(g1, g0);
+        const uint64_t d2 = gl::sub(gl::sub(g2, g1), d1);
+        const uint64_t c2 = gl::mul(gl::mul(r, gl::sub(r, 1)), inv2);
+        claim = gl::add(g0, gl::add(gl::mul(r, d1), gl::mul(c2, d2)));
+    }
+    const uint64_t a_fin = t[3 * nrounds + 1], b_fin = t[3 * nrounds + 2];
+    if (gl::mul(a_fin, b_fin) != claim) { *fail_at = nrounds; return IMM_REJECT; }
+    if (expect_c0 && *expect_c0 != t[0]) { *fail_at = nrounds + 1; return IMM_REJECT; }
+    if (expect_a_fin && *expect_a_fin != a_fin) { *fail_at = nrounds + 2; return IMM_REJECT; }
+    if (expect_b_fin && *expect_b_fin != b_fin) { *fail_at = nrounds + 3; return IMM_REJECT; }
+    *fail_at = -1;
     return IMM_OK;
 }
 

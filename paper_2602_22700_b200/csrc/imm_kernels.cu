@@ -11,6 +11,7 @@
 #include "gl64.cuh"
 #include "imm_kernels.h"
 #include "imm_plan.h"
+#include "sha256.cuh"
 
 namespace imm {
 
@@ -725,8 +726,154 @@ sumcheck_kernel(const ProofDev* proofs, uint64_t seed, imm_fe* transcripts, int6
 }
 
 // ------------------------------------------------------------------------------------------
+// non-interactive (Fiat-Shamir) proof: challenges hashed from the statement and the transcript
+// ------------------------------------------------------------------------------------------
+// H = SHA-256; integers little-endian; a field element is the le64 of its canonical value;
+// fe(d) = the first 8 bytes of a digest as a big-endian integer, minus p if not below p.
+//   s_0     = H(0x10 || com_A || com_B || com_C || le64(m) || le64(k) || le64(n) || le64(proof_id))
+//   r_row[t] = fe(H(0x11 || s_0 || le32(1) || le32(t))),  r_col[t] with le32(2)
+//   s_1     = H(0x12 || s_0 || le64(c0))
+//   s_{j+2} = H(0x13 || s_{j+1} || le64(g_j(0)) || le64(g_j(1)) || le64(g_j(2))),  r_j = fe(s_{j+2})
+
+__device__ __forceinline__ uint64_t fs_fe(const uint32_t (&h)[8])
+{
+    const uint64_t v = ((uint64_t)h[0] << 32) | h[1];
+    return v >= gl::P ? v - gl::P : v;
+}
+
+__device__ __forceinline__ void fs_put_le(uint8_t* dst, uint64_t v, int nbytes)
+{
+    for (int q = 0; q < nbytes; q++) dst[q] = (uint8_t)(v >> (8 * q));
+}
+
+// s <- H(tag || s || le64(vals[0..nvals)))
+__device__ __noinline__ void fs_absorb(uint32_t (&s)[8], uint8_t tag, const uint64_t* vals, int nvals, uint32_t one)
+{
+    uint8_t m[64];
+    m[0] = tag;
+    imm_sha::digest_bytes(s, m + 1);
+    for (int i = 0; i < nvals; i++) fs_put_le(m + 33 + 8 * i, vals[i], 8);
+    imm_sha::sha256_short(m, 33 + 8 * (uint32_t)nvals, s, one);
+}
+
+// Statement hash and the two evaluation points of every proof (one block per proof).
+__global__ void __launch_bounds__(2 * FS_POINT_SLOTS) fs_points_kernel(const ProofDev* proofs, const FsProof* fs)
+{
+    __shared__ uint32_t s0[8];
+    const ProofDev& pr = proofs[blockIdx.x];
+    const FsProof& f = fs[blockIdx.x];
+    if (threadIdx.x == 0) {
+        uint8_t m[136];
+        m[0] = 0x10;
+        for (int i = 0; i < 96; i++) m[1 + i] = f.com[i];
+        fs_put_le(m + 97, (uint64_t)pr.m, 8);
+        fs_put_le(m + 105, (uint64_t)pr.k, 8);
+        fs_put_le(m + 113, (uint64_t)pr.n, 8);
+        fs_put_le(m + 121, f.proof_id, 8);
+        uint32_t h[8];
+        imm_sha::sha256_short(m, 129, h, f.one);
+        for (int i = 0; i < 8; i++) { s0[i] = h[i]; f.state[i] = h[i]; }
+    }
+    __syncthreads();
+    const int which = threadIdx.x / FS_POINT_SLOTS, t = threadIdx.x % FS_POINT_SLOTS;     // 0: r_row, 1: r_col
+    if (t < (which == 0 ? pr.a : pr.c)) {
+        uint8_t m[48];
+        uint32_t h[8];
+        for (int i = 0; i < 8; i++) h[i] = s0[i];
+        m[0] = 0x11;
+        imm_sha::digest_bytes(h, m + 1);
+        fs_put_le(m + 33, (uint64_t)(which + 1), 4);
+        fs_put_le(m + 37, (uint64_t)t, 4);
+        imm_sha::sha256_short(m, 41, h, f.one);
+        f.points[which * FS_POINT_SLOTS + t] = fs_fe(h);
+    }
+}
+
+// The rounds of one proof by one block: every round's three sums are reduced over the block, hashed
+// into the transcript state by thread 0, and only then is the round's challenge known and the fold
+// can run.  The two tables live in global memory (they stay in L2).
+__global__ void __launch_bounds__(FS_THREADS)
+sumcheck_fs_kernel(const ProofDev* proofs, const FsProof* fs, imm_fe* transcripts, int64_t stride, int32_t* status)
+{
+    __shared__ uint64_t red[33];
+    __shared__ uint64_t r_sh;
+    const ProofDev pr = proofs[blockIdx.x];
+    const FsProof f = fs[blockIdx.x];
+    imm_fe* tr = transcripts + (int64_t)blockIdx.x * stride;
+    const int tid = threadIdx.x, b = pr.b;
+    imm_fe* ta = f.ta;
+    imm_fe* tb = f.tb;
+
+    // claim c0 = sum of the partial sums of C (minus the 2^31 offset of the byte-wise kernel)
+    uint64_t s = 0;
+    for (int i = tid; i < pr.n_part_c; i += FS_THREADS) s = gl::add(s, pr.part_c[i]);
+    s = block_sum_fe(s, red);
+    if (pr.c_offset) {
+        uint64_t sr = 0, sc = 0;
+        for (int i = tid; i < pr.n_sum_row; i += FS_THREADS) sr = gl::add(sr, pr.sum_row[i]);
+        for (int i = tid; i < pr.n_sum_col; i += FS_THREADS) sc = gl::add(sc, pr.sum_col[i]);
+        sr = block_sum_fe(sr, red);
+        sc = block_sum_fe(sc, red);
+        s = gl::sub(s, gl::shl(gl::mul(sr, sc), 31));
+    }
+    uint32_t st[8];                                        // the transcript state (thread 0)
+    if (tid == 0) {
+        tr[0] = s;
+        status[blockIdx.x] = 0;
+        for (int i = 0; i < 8; i++) st[i] = f.state[i];
+        fs_absorb(st, 0x12, &s, 1, f.one);
+    }
+    for (int64_t i = 3 * b + 3 + tid; i < stride; i += FS_THREADS) tr[i] = 0;
+
+    // both tables from the partial vectors; entries past k are the zero padding
+    const int n0 = 1 << b;
+    for (int y = tid; y < n0; y += FS_THREADS) {
+        const bool live = y < pr.k;
+        ta[y] = live ? sum_parts_at(pr.part_a, pr.n_part_a, pr.k, y) : 0;
+        tb[y] = live ? sum_parts_at(pr.part_b, pr.n_part_b, pr.k, y) : 0;
+    }
+    __syncthreads();
+
+    for (int j = 0, n = n0; j < b; j++, n >>= 1) {
+        const int h = n >> 1;
+        Sums3 acc = {0, 0, 0};
+        for (int e = tid; e < h; e += FS_THREADS) sums_add(acc, ta[e], ta[e + h], tb[e], tb[e + h]);
+        uint64_t g[3];
+        g[0] = block_sum_fe(acc.g0, red);
+        g[1] = block_sum_fe(acc.g1, red);
+        g[2] = block_sum_fe(acc.g2, red);
+        if (tid == 0) {
+            tr[1 + 3 * j] = g[0]; tr[2 + 3 * j] = g[1]; tr[3 + 3 * j] = g[2];
+            fs_absorb(st, 0x13, g, 3, f.one);
+            r_sh = fs_fe(st);
+        }
+        __syncthreads();
+        const uint64_t r = r_sh;
+        for (int e = tid; e < h; e += FS_THREADS) {        // in place: writes go below h, second operands sit above
+            ta[e] = fold1(ta[e], ta[e + h], r);
+            tb[e] = fold1(tb[e], tb[e + h], r);
+        }
+        __syncthreads();
+    }
+    if (tid == 0) { tr[3 * b + 1] = ta[0]; tr[3 * b + 2] = tb[0]; }
+}
+
+// ------------------------------------------------------------------------------------------
 // launch wrappers
 // ------------------------------------------------------------------------------------------
+
+cudaError_t launch_fs_points(const ProofDev* d_proofs, const FsProof* d_fs, int nproofs, cudaStream_t st)
+{
+    fs_points_kernel<<<nproofs, 2 * FS_POINT_SLOTS, 0, st>>>(d_proofs, d_fs);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_sumcheck_fs(const ProofDev* d_proofs, const FsProof* d_fs, int nproofs, imm_fe* transcripts,
+                               int64_t stride, int32_t* status, cudaStream_t st)
+{
+    sumcheck_fs_kernel<<<nproofs, FS_THREADS, 0, st>>>(d_proofs, d_fs, transcripts, stride, status);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_field_binop(int op, const imm_fe* x, const imm_fe* y, imm_fe* out, int64_t n,
                                cudaStream_t st)

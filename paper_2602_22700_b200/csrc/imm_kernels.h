@@ -32,5 +32,9 @@ cudaError_t launch_sumcheck(const ProofDev* d_proofs, int nproofs, uint64_t seed
 // batched transcript (1 + 3b + 3*nproofs words) from per-proof transcripts proved under shared round challenges
 cudaError_t launch_combine(const imm_fe* tr, int64_t stride, int nproofs, int b, uint64_t seed, uint64_t batch_id,
                            imm_fe* out, cudaStream_t st);
+// non-interactive proof: statement hash and hashed evaluation points; rounds with hashed challenges
+cudaError_t launch_fs_points(const ProofDev* d_proofs, const FsProof* d_fs, int nproofs, cudaStream_t st);
+cudaError_t launch_sumcheck_fs(const ProofDev* d_proofs, const FsProof* d_fs, int nproofs, imm_fe* transcripts,
+                               int64_t stride, int32_t* status, cudaStream_t st);
 
 }  // namespace imm

@@ -107,7 +107,8 @@ __global__ void __launch_bounds__(EQ_BATCH_THREADS) eq_batch_kernel(const EqTask
     const int nlo = (tk.nvars + 1) / 2, nhi = tk.nvars - nlo;
     if (!from_table) {                                 // (uniform over the block)
         if ((int)threadIdx.x < tk.nvars) {
-            const uint64_t r = gl::challenge(tk.seed, tk.proof_id, tk.domain, threadIdx.x);
+            const uint64_t r = tk.point ? tk.point[threadIdx.x]
+                                        : gl::challenge(tk.seed, tk.proof_id, tk.domain, threadIdx.x);
             r_sh[threadIdx.x] = r;
             omr_sh[threadIdx.x] = gl::sub(1, r);
         }

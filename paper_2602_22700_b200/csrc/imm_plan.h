@@ -92,6 +92,21 @@ struct EqTask {
     imm_fe* slice_sums;        // one entry per block of the task: sum of its entries below `extent` (or null)
     const imm_fe* given;       // non-null: the table exists already (`extent` entries are read from here, nothing
                                // is derived or written to `out`); only the limb tables and slice sums are produced
+    const imm_fe* point;       // non-null: r is read from here (nvars entries) instead of the generator
+};
+
+// Per proof of a non-interactive (Fiat-Shamir) batch: where its statement and hashed challenges live.
+constexpr int FS_POINT_SLOTS = 32;          // slots per point: r_row at [0, a), r_col at [FS_POINT_SLOTS, FS_POINT_SLOTS + c)
+constexpr int FS_THREADS = 1024;            // threads of the round kernel's block (one block per proof)
+struct FsProof {
+    const uint8_t* com;        // 96 bytes: the commitments to A, B, C
+    imm_fe* points;            // [2 * FS_POINT_SLOTS]
+    uint32_t* state;           // [8]: s_0, the hash of the statement
+    imm_fe* ta;                // [2^b] the round kernel's tables
+    imm_fe* tb;
+    uint64_t proof_id;
+    uint32_t one;              // 1 (the multiplier of the multiply-add form of SHA-256's adds)
+    uint32_t pad_;
 };
 
 // A single eq table with r supplied by the caller (passed by value to the kernel).

@@ -33,7 +33,9 @@ EXPORTS = ("imm_version", "imm_last_cuda_error", "imm_challenge", "imm_field_bin
            "imm_ldd_tv_kl", "imm_ldd_topk_workspace", "imm_ldd_topk_distance", "imm_ldd_tail_fraction",
            "imm_sumcheck_batched_transcript_len", "imm_sumcheck_matmul_batched_workspace",
            "imm_sumcheck_matmul_prove_batched", "imm_sumcheck_verify_batched",
-           "imm_commit_workspace", "imm_commit")
+           "imm_commit_workspace", "imm_commit",
+           "imm_sumcheck_matmul_fs_workspace", "imm_sumcheck_matmul_prove_fs", "imm_fs_challenges",
+           "imm_sumcheck_verify_fs")
 COMMIT_LEAF = 4096
 NOALLOC_MAX_TILES = 8192
 PROFILE_PHASES = ("eq_tables", "claim_C", "bind_rows_A", "bind_cols_B", "sumcheck_rounds")
@@ -116,6 +118,14 @@ def lib() -> ctypes.CDLL:
     L.imm_sumcheck_matmul_batched_workspace.argtypes = [vp, ci]
     L.imm_sumcheck_matmul_prove_batched.restype = ci
     L.imm_sumcheck_matmul_prove_batched.argtypes = [vp, ci, u64, u64, vp, vp, vp, sz, vp]
+    L.imm_sumcheck_matmul_fs_workspace.restype = sz
+    L.imm_sumcheck_matmul_fs_workspace.argtypes = [vp, ci]
+    L.imm_sumcheck_matmul_prove_fs.restype = ci
+    L.imm_sumcheck_matmul_prove_fs.argtypes = [vp, ci, vp, vp, i64, vp, vp, sz, vp]
+    L.imm_fs_challenges.restype = ci
+    L.imm_fs_challenges.argtypes = [vp, ci, vp, i64, i64, i64, u64, vp, vp, vp]
+    L.imm_sumcheck_verify_fs.restype = ci
+    L.imm_sumcheck_verify_fs.argtypes = [vp, ci, vp, i64, i64, i64, u64, vp, vp, vp, vp]
     L.imm_commit_workspace.restype = sz
     L.imm_commit_workspace.argtypes = [vp, ci]
     L.imm_commit.restype = ci
@@ -486,6 +496,104 @@ def commit(messages, randomness=None) -> List[bytes]:
     c = Committer(messages, randomness)
     d = c.commit().cpu().numpy()
     return [bytes(row) for row in d]
+
+
+# ------------------------------------------------------------------ non-interactive proof
+
+
+def commit_matrices(problems, randomness=None) -> torch.Tensor:
+    """(nproofs, 96) uint8 CUDA tensor: the commitments to A, B and C of every problem, in that order
+    (the statement of a non-interactive proof).  ``randomness``: None or one 32-byte string per matrix."""
+    msgs = [t for (A, B, C, _) in problems for t in (A, B, C)]
+    c = Committer(msgs, randomness)
+    return c.commit().view(len(problems), 96)
+
+
+class FsProver:
+    """Non-interactive prover: challenges hashed from the commitments and the transcript."""
+
+    def __init__(self, problems, commitments: torch.Tensor, device="cuda"):
+        self.problems = list(problems)
+        self.descs = make_descs(self.problems)
+        self.nproofs = len(self.problems)
+        self.commitments = _cuda(commitments, torch.uint8, "commitments").contiguous()
+        if self.commitments.numel() != 96 * self.nproofs:
+            raise ValueError("commitments must hold 96 bytes per proof")
+        self.stride = max(transcript_len(A.shape[1]) for (A, _, _, _) in self.problems)
+        need = lib().imm_sumcheck_matmul_fs_workspace(ctypes.addressof(self.descs), self.nproofs)
+        if need == 0:
+            raise ImmError(ERR_SHAPE, "imm_sumcheck_matmul_fs_workspace")
+        self.ws = torch.empty(need, dtype=torch.uint8, device=device)
+        self.transcripts = torch.zeros((self.nproofs, self.stride), dtype=torch.int64, device=device)
+        self.status = torch.full((self.nproofs,), -99, dtype=torch.int32, device=device)
+
+    def prove(self) -> torch.Tensor:
+        _check(lib().imm_sumcheck_matmul_prove_fs(ctypes.addressof(self.descs), self.nproofs,
+                                                  self.commitments.data_ptr(), self.transcripts.data_ptr(),
+                                                  self.stride, self.status.data_ptr(), self.ws.data_ptr(),
+                                                  self.ws.numel(), _stream()), "imm_sumcheck_matmul_prove_fs")
+        return self.transcripts
+
+    def lengths(self) -> List[int]:
+        return [transcript_len(A.shape[1]) for (A, _, _, _) in self.problems]
+
+
+def sumcheck_matmul_prove_fs(problems, commitments: torch.Tensor) -> List[List[int]]:
+    """Convenience: non-interactive transcripts as Python ints (synchronises)."""
+    pr = FsProver(problems, commitments)
+    t = pr.prove()
+    torch.cuda.synchronize()
+    if int(pr.status.abs().max()) != 0:
+        raise ImmError(int(pr.status.min()), "device status")
+    host = t.cpu()
+    return [[int(v) & 0xFFFFFFFFFFFFFFFF for v in host[i, :n]] for i, n in enumerate(pr.lengths())]
+
+
+def _com96(commitments) -> "ctypes.Array":
+    data = bytes(commitments)
+    if len(data) != 96:
+        raise ValueError("the statement's commitments are 96 bytes")
+    return (ctypes.c_uint8 * 96)(*data)
+
+
+def fs_challenges(transcript: Optional[Sequence[int]], nrounds: int, commitments, m: int, k: int, n: int,
+                  proof_id: int) -> Tuple[List[int], List[int], List[int]]:
+    """(r_row, r_col, r_k) as the verifier of a non-interactive proof derives them (r_k empty when no
+    transcript is given)."""
+    com = _com96(commitments)
+    a, c = ceil_log2(m), ceil_log2(n)
+    rr, rc_, rk = (ctypes.c_uint64 * max(a, 1))(), (ctypes.c_uint64 * max(c, 1))(), (ctypes.c_uint64 * max(nrounds, 1))()
+    arr = None
+    if transcript is not None:
+        words = [int(v) & 0xFFFFFFFFFFFFFFFF for v in list(transcript)[:3 * nrounds + 1]]
+        arr = (ctypes.c_uint64 * len(words))(*words)
+    _check(lib().imm_fs_challenges(None if arr is None else ctypes.addressof(arr), nrounds, ctypes.addressof(com),
+                                   m, k, n, proof_id, ctypes.addressof(rr), ctypes.addressof(rc_),
+                                   None if arr is None else ctypes.addressof(rk)), "imm_fs_challenges")
+    return list(rr)[:a], list(rc_)[:c], (list(rk)[:nrounds] if arr is not None else [])
+
+
+def sumcheck_verify_fs(transcript: Sequence[int], nrounds: int, commitments, m: int, k: int, n: int, proof_id: int,
+                       expect_c0: Optional[int] = None, expect_a_fin: Optional[int] = None,
+                       expect_b_fin: Optional[int] = None) -> Tuple[int, int]:
+    """Host verifier of a non-interactive proof; returns (status, fail_at)."""
+    cnt = 3 * nrounds + 3
+    arr = (ctypes.c_uint64 * cnt)(*[int(v) & 0xFFFFFFFFFFFFFFFF for v in list(transcript)[:cnt]])
+    com = _com96(commitments)
+    keep = []
+
+    def opt(v):
+        if v is None:
+            return None
+        box = ctypes.c_uint64(int(v))
+        keep.append(box)
+        return ctypes.addressof(box)
+
+    fail = ctypes.c_int(-2)
+    rc = lib().imm_sumcheck_verify_fs(ctypes.addressof(arr), nrounds, ctypes.addressof(com), m, k, n, proof_id,
+                                      opt(expect_c0), opt(expect_a_fin), opt(expect_b_fin), ctypes.addressof(fail))
+    _check(rc, "imm_sumcheck_verify_fs")
+    return rc, fail.value
 
 
 # ------------------------------------------------------------------ logit distance distribution

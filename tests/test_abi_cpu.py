@@ -95,6 +95,35 @@ def test_batched_host_verifier_matches_oracle_verifier(imm, oracle):
     assert imm.batched_transcript_len(-1, 4) == 0 and imm.batched_transcript_len(3, 0) == 0
 
 
+def test_fs_host_challenges_and_verifier_match_oracle(imm, oracle):
+    rng = random.Random(4)
+    for (m, k, n) in ((3, 8, 2), (2, 5, 4), (4, 1, 4), (1, 16, 1), (5, 33, 7)):
+        A = np.array([[rng.randint(-128, 127) for _ in range(k)] for _ in range(m)], dtype=np.int8)
+        B = np.array([[rng.randint(-128, 127) for _ in range(n)] for _ in range(k)], dtype=np.int8)
+        C = (A.astype(np.int64) @ B.astype(np.int64)).astype(np.int32)
+        coms, pid = [rng.randbytes(32) for _ in range(3)], rng.getrandbits(64)
+        com96 = b"".join(coms)
+        t = oracle.fs.prove(A, B, C, coms, pid)
+        b = oracle.ceil_log2(k)
+        want = oracle.fs.challenges(t, b, coms, m, k, n, pid)
+        assert imm.fs_challenges(t, b, com96, m, k, n, pid) == tuple(want)
+        assert imm.fs_challenges(None, b, com96, m, k, n, pid)[:2] == (want[0], want[1])
+        assert imm.sumcheck_verify_fs(t, b, com96, m, k, n, pid) == (imm.OK, -1)
+        assert imm.sumcheck_verify_fs(t, b, com96, m, k, n, pid, t[0], t[-2], t[-1]) == (imm.OK, -1)
+        for pos in range(len(t)):
+            bad = list(t)
+            bad[pos] = (bad[pos] + 1 + rng.randrange(oracle.P - 1)) % oracle.P
+            got = imm.sumcheck_verify_fs(bad, b, com96, m, k, n, pid)
+            assert got == oracle.fs.verify(bad, b, coms, m, k, n, pid) and got[0] == imm.REJECT
+        flipped = bytes([com96[40] ^ 4]) .join([com96[:40], com96[41:]])
+        assert imm.sumcheck_verify_fs(t, b, flipped, m, k, n, pid)[0] == (imm.REJECT if b > 0 else imm.OK)
+        assert imm.sumcheck_verify_fs(t, b, com96, m, k, n, pid, None, (t[-2] + 1) % oracle.P) == (imm.REJECT, b + 2)
+        with pytest.raises(imm.ImmError):
+            imm.sumcheck_verify_fs(t, b + 1, com96, m, k, n, pid)            # nrounds must be ceil(log2 k)
+    with pytest.raises(imm.ImmError):
+        imm.sumcheck_verify_fs([oracle.P, 0, 0], 0, bytes(96), 1, 1, 1, 0)
+
+
 def _desc_array(imm, shapes, base=0x10000):
     arr = (imm.MatmulDesc * len(shapes))()
     for i, (m, k, n) in enumerate(shapes):
@@ -135,6 +164,33 @@ def test_batched_workspace_and_validation(imm):
     assert prove(ctypes.addressof(d), 2, 1, 1, 0x1000, 0x1000, 0x1010, need, None) == imm.ERR_ALIGN
     assert prove(ctypes.addressof(d), 2, 1, 1, None, 0x1000, 0x1000, need, None) == imm.ERR_ARG
     assert prove(ctypes.addressof(d), 0, 1, 1, 0x1000, 0x1000, 0x1000, need, None) == imm.ERR_ARG
+
+
+def test_fs_and_commit_workspace_and_validation(imm):
+    L = imm.lib()
+    d = _desc_array(imm, [(64, 4096, 64), (512, 3000, 4096)])
+    plain = L.imm_sumcheck_matmul_workspace(ctypes.addressof(d), 2)
+    need = L.imm_sumcheck_matmul_fs_workspace(ctypes.addressof(d), 2)
+    assert need >= plain + 2 * 2 * 4096 * 8 and need % 256 == 0             # two tables of 2^12 entries per proof
+    prove = L.imm_sumcheck_matmul_prove_fs
+    assert prove(ctypes.addressof(d), 2, None, 0x1000, 39, 0x1000, 0x1000, need, None) == imm.ERR_ARG
+    assert prove(ctypes.addressof(d), 2, 0x1000, 0x1000, 39, 0x1000, 0x1000, need - 1, None) == imm.ERR_WORKSPACE
+    assert prove(ctypes.addressof(d), 2, 0x1000, 0x1000, 38, 0x1000, 0x1000, need, None) == imm.ERR_SHAPE
+    assert prove(ctypes.addressof(d), 2, 0x1000, 0x1000, 39, 0x1000, 0x1010, need, None) == imm.ERR_ALIGN
+    c = (imm.CommitDesc * 2)()
+    c[0].msg, c[0].nbytes = 0x1000, 5 << 20
+    c[1].msg, c[1].nbytes, c[1].r_len = None, 0, 32
+    w = L.imm_commit_workspace(ctypes.addressof(c), 2)
+    assert w > 0 and w % 256 == 0 and w >= (10 + 1 + 1 + 1) * 32             # subtree roots of both, then the big one's root
+    assert L.imm_commit(ctypes.addressof(c), 2, 0x1000, None, 0x1000, w - 1, None) == imm.ERR_WORKSPACE
+    assert L.imm_commit(ctypes.addressof(c), 2, None, None, 0x1000, w, None) == imm.ERR_ARG
+    assert L.imm_commit(ctypes.addressof(c), 2, 0x1000, None, 0x1010, w, None) == imm.ERR_ALIGN
+    c[1].r_len = 16
+    assert L.imm_commit_workspace(ctypes.addressof(c), 2) == 0
+    c[1].r_len, c[1].nbytes = 0, 100                                         # bytes without a pointer
+    assert L.imm_commit_workspace(ctypes.addressof(c), 2) == 0
+    c[1].nbytes, c[0].nbytes = 0, (1 << 40) + 1
+    assert L.imm_commit(ctypes.addressof(c), 2, 0x1000, None, 0x1000, 1 << 30, None) == imm.ERR_LIMIT
 
 
 def test_argument_validation_happens_before_any_device_work(imm):

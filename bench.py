@@ -53,6 +53,9 @@ def parse_args():
     ap.add_argument("--batched", action="store_true",
                     help="prove the products of equal round count as one random-linear-combination proof each "
                          "(device-resident timing only)")
+    ap.add_argument("--fs", action="store_true",
+                    help="non-interactive proofs: a step commits to every matrix (SHA-256 trees) and proves with "
+                         "challenges hashed from the commitments and the transcript (device-resident timing only)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=2)
@@ -243,6 +246,21 @@ def run_ours(args):
         def prove_step():
             for gi, bp in enumerate(provers):
                 bp.prove(SEED, BATCH_ID0 + gi)
+    elif args.fs:
+        triples = [(p.A, p.B, p.C, p.proof_id) for p in problems]
+        com = imm.Committer([t for (A, B, C, _) in triples for t in (A, B, C)], device=dev)
+        fsp = imm.FsProver(triples, com.digests.view(len(triples), 96), device=dev)
+        provers = [fsp]
+        fs_ev = []
+
+        def prove_step():
+            e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+            e[0].record()
+            com.commit()
+            e[1].record()
+            fsp.prove()
+            e[2].record()
+            fs_ev.append(e)
     else:
         prover = imm.Prover([(p.A, p.B, p.C, p.proof_id) for p in problems], device=dev)
         provers = [prover]
@@ -295,7 +313,17 @@ def run_ours(args):
 
     # every proof of the timed batch must be accepted by the verifier
     accepted = 0
-    if args.batched:
+    if args.fs:
+        host_t = fsp.transcripts.cpu()
+        assert int(fsp.status.abs().max()) == 0
+        host_c = com.digests.view(len(problems), 96).cpu().numpy()
+        for i, p in enumerate(problems):
+            m_, k_, n_ = p.mkn
+            b = imm.ceil_log2(k_)
+            words = [int(v) & 0xFFFFFFFFFFFFFFFF for v in host_t[i, :3 * b + 3]]
+            if imm.sumcheck_verify_fs(words, b, bytes(host_c[i]), m_, k_, n_, p.proof_id) == (imm.OK, -1):
+                accepted += 1
+    elif args.batched:
         host_t = None
         for gi, (b, g) in enumerate(groups.items()):
             assert int(provers[gi].status.abs().max()) == 0
@@ -323,7 +351,9 @@ def run_ours(args):
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "u64", "data": "synthetic",
         "config": {"workload": workload_name(args.config, args.layers, args.tokens) +
-                               (f", as {calls_per_step} batched proofs (one per round count)" if args.batched else ""),
+                               (f", as {calls_per_step} batched proofs (one per round count)" if args.batched else "") +
+                               (", non-interactive: SHA-256 tree commitments to every matrix, then proofs with hashed "
+                                "challenges" if args.fs else ""),
                    "layers": args.layers if args.config == "decoder" else min(args.layers, 8) if args.config == "attn" else None,
                    "tokens": args.tokens, "proofs_per_gpu": len(problems), "field": "Goldilocks 2^64-2^32+1",
                    "input_bytes_per_gpu": algo_bytes,
@@ -343,7 +373,7 @@ def run_ours(args):
                      "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": claim_gbs / peak,
                      "frac_of_8tbs": claim_gbs / 8000.0,
                      "traffic": (CLAIM_KERNEL_TRAFFIC_RATIO * claim_bytes) if CLAIM_KERNEL_TRAFFIC_RATIO else None},
-        "gpu_launches": (6 if args.batched else 5) * calls_per_step * steps,
+        "gpu_launches": ((6 + com.launches) if args.fs else 6 if args.batched else 5) * calls_per_step * steps,
         "transcript_words_per_step": (sum(int(bp.length) for bp in provers) if args.batched else
                                       sum(3 * imm.ceil_log2(k) + 3 for (m, k, n) in shapes)),
         "clocks": clocks,
@@ -351,8 +381,13 @@ def run_ours(args):
 
     # ---- end to end: pinned host inputs -> device arena -> proofs -> host transcripts
     e2e = None
-    if args.batched:
-        e2e = {"value": None, "unit": UNIT, "skipped": "the host-buffer entry point proves proof by proof"}
+    if args.fs:
+        tail = fs_ev[-steps:]
+        out["fs_phases"] = {"commit_ms": sum(e[0].elapsed_time(e[1]) for e in tail) / steps,
+                            "prove_ms": sum(e[1].elapsed_time(e[2]) for e in tail) / steps,
+                            "committed_bytes": algo_bytes}
+    if args.batched or args.fs:
+        e2e = {"value": None, "unit": UNIT, "skipped": "the host-buffer entry point proves interactively, proof by proof"}
     elif not args.no_e2e:
         need = algo_bytes
         if mem_available_bytes() < int(1.25 * need * (world if world > 1 else 1)):
@@ -380,7 +415,7 @@ def run_ours(args):
     out["e2e"] = e2e
 
     # ---- the oracle beside it (rank 0, single GPU): first two layers' proofs, one per thread
-    if not args.no_cpu_baseline and world == 1 and not args.batched:
+    if not args.no_cpu_baseline and world == 1 and not args.batched and not args.fs:
         nsample = min(len(problems), 8)
         sample = sample_to_host(problems[:nsample])
         threads = min(os.cpu_count() or 1, nsample)

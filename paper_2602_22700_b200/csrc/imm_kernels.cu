@@ -746,14 +746,61 @@ __device__ __forceinline__ void fs_put_le(uint8_t* dst, uint64_t v, int nbytes)
     for (int q = 0; q < nbytes; q++) dst[q] = (uint8_t)(v >> (8 * q));
 }
 
-// s <- H(tag || s || le64(vals[0..nvals)))
-__device__ __noinline__ void fs_absorb(uint32_t (&s)[8], uint8_t tag, const uint64_t* vals, int nvals, uint32_t one)
+// s <- H(tag || s || le64(vals[0..NV))), NV = 1 or 3.  The message is the word stream
+// [s_0..s_7, byte-swapped halves of the values] moved one byte to the right behind the tag, so its
+// words are built with shifts instead of byte by byte (the hash sits on the rounds' critical path:
+// one thread, nothing to overlap it with).
+template <int NV>
+__device__ __forceinline__ void fs_absorb(uint32_t (&s)[8], uint32_t tag, const uint64_t (&vals)[NV], uint32_t one)
 {
-    uint8_t m[64];
-    m[0] = tag;
-    imm_sha::digest_bytes(s, m + 1);
-    for (int i = 0; i < nvals; i++) fs_put_le(m + 33 + 8 * i, vals[i], 8);
-    imm_sha::sha256_short(m, 33 + 8 * (uint32_t)nvals, s, one);
+    constexpr int L = 8 + 2 * NV;                          // stream words; the message has 1 + 4 L bytes
+    uint32_t st[L];
+#pragma unroll
+    for (int i = 0; i < 8; i++) st[i] = s[i];
+#pragma unroll
+    for (int i = 0; i < NV; i++) {
+        st[8 + 2 * i] = __byte_perm((uint32_t)vals[i], 0, 0x0123);            // little-endian bytes in stream order
+        st[9 + 2 * i] = __byte_perm((uint32_t)(vals[i] >> 32), 0, 0x0123);
+    }
+    uint32_t w[16];
+    w[0] = (tag << 24) | (st[0] >> 8);
+#pragma unroll
+    for (int i = 1; i < 16; i++) {
+        if (i < L) w[i] = (st[i - 1] << 24) | (st[i] >> 8);
+        else if (i == L) w[i] = (st[L - 1] << 24) | 0x00800000u;
+        else w[i] = 0;
+    }
+    const uint32_t bits = (1 + 4 * L) * 8;
+    constexpr int NBLOCKS = L < 14 ? 1 : 2;                // one block if 0x80 and the length fit behind the words
+    if (NBLOCKS == 1) w[15] = bits;
+    imm_sha::iv(s);
+#pragma unroll 1
+    for (int blk = 0; blk < NBLOCKS; blk++) {              // (one copy of the compression in the code)
+        if (blk == 1) {
+#pragma unroll
+            for (int i = 0; i < 15; i++) w[i] = 0;
+            w[15] = bits;
+        }
+        imm_sha::compress_compact(s, w, one);
+    }
+}
+
+// Sums of three values per thread over the block at once; results valid in thread 0.
+__device__ __forceinline__ void block_sum3_fe(uint64_t (&v)[3], uint64_t (*scratch)[32])
+{
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = (blockDim.x + 31) >> 5;
+#pragma unroll
+    for (int i = 0; i < 3; i++) v[i] = warp_sum_fe(v[i]);
+    __syncthreads();                       // scratch may still be read from the previous round
+    if (lane == 0) {
+#pragma unroll
+        for (int i = 0; i < 3; i++) scratch[i][warp] = v[i];
+    }
+    __syncthreads();
+    if (warp == 0) {
+#pragma unroll
+        for (int i = 0; i < 3; i++) v[i] = warp_sum_fe(lane < nwarp ? scratch[i][lane] : 0);
+    }
 }
 
 // Statement hash and the two evaluation points of every proof (one block per proof).
@@ -796,6 +843,7 @@ __global__ void __launch_bounds__(FS_THREADS)
 sumcheck_fs_kernel(const ProofDev* proofs, const FsProof* fs, imm_fe* transcripts, int64_t stride, int32_t* status)
 {
     __shared__ uint64_t red[33];
+    __shared__ uint64_t red3[3][32];
     __shared__ uint64_t r_sh;
     const ProofDev pr = proofs[blockIdx.x];
     const FsProof f = fs[blockIdx.x];
@@ -820,8 +868,10 @@ sumcheck_fs_kernel(const ProofDev* proofs, const FsProof* fs, imm_fe* transcript
     if (tid == 0) {
         tr[0] = s;
         status[blockIdx.x] = 0;
+#pragma unroll
         for (int i = 0; i < 8; i++) st[i] = f.state[i];
-        fs_absorb(st, 0x12, &s, 1, f.one);
+        const uint64_t c0[1] = {s};
+        fs_absorb<1>(st, 0x12, c0, f.one);
     }
     for (int64_t i = 3 * b + 3 + tid; i < stride; i += FS_THREADS) tr[i] = 0;
 
@@ -834,27 +884,34 @@ sumcheck_fs_kernel(const ProofDev* proofs, const FsProof* fs, imm_fe* transcript
     }
     __syncthreads();
 
+    // round 0's sums come from the tables; every later round's sums are taken from the folded
+    // values as the fold of the round before produces them (one pass over the tables per round)
+    Sums3 acc = {0, 0, 0};
+    for (int e = tid; e < (n0 >> 1); e += FS_THREADS) sums_add(acc, ta[e], ta[e + (n0 >> 1)], tb[e], tb[e + (n0 >> 1)]);
     for (int j = 0, n = n0; j < b; j++, n >>= 1) {
-        const int h = n >> 1;
-        Sums3 acc = {0, 0, 0};
-        for (int e = tid; e < h; e += FS_THREADS) sums_add(acc, ta[e], ta[e + h], tb[e], tb[e + h]);
-        uint64_t g[3];
-        g[0] = block_sum_fe(acc.g0, red);
-        g[1] = block_sum_fe(acc.g1, red);
-        g[2] = block_sum_fe(acc.g2, red);
+        const int h = n >> 1, q = n >> 2;
+        uint64_t g[3] = {acc.g0, acc.g1, acc.g2};
+        block_sum3_fe(g, red3);                            // (its barriers also order the fold's writes before the next reads)
         if (tid == 0) {
             tr[1 + 3 * j] = g[0]; tr[2 + 3 * j] = g[1]; tr[3 + 3 * j] = g[2];
-            fs_absorb(st, 0x13, g, 3, f.one);
+            fs_absorb<3>(st, 0x13, g, f.one);
             r_sh = fs_fe(st);
         }
         __syncthreads();
         const uint64_t r = r_sh;
-        for (int e = tid; e < h; e += FS_THREADS) {        // in place: writes go below h, second operands sit above
-            ta[e] = fold1(ta[e], ta[e + h], r);
-            tb[e] = fold1(tb[e], tb[e + h], r);
+        acc = Sums3{0, 0, 0};
+        if (h == 1) {
+            if (tid == 0) { ta[0] = fold1(ta[0], ta[1], r); tb[0] = fold1(tb[0], tb[1], r); }
+        } else {
+            for (int e = tid; e < q; e += FS_THREADS) {    // in place: each thread rewrites only what it alone read
+                const uint64_t fa0 = fold1(ta[e], ta[e + h], r), fa1 = fold1(ta[e + q], ta[e + q + h], r);
+                const uint64_t fb0 = fold1(tb[e], tb[e + h], r), fb1 = fold1(tb[e + q], tb[e + q + h], r);
+                ta[e] = fa0; ta[e + q] = fa1; tb[e] = fb0; tb[e + q] = fb1;
+                sums_add(acc, fa0, fa1, fb0, fb1);
+            }
         }
-        __syncthreads();
     }
+    __syncthreads();
     if (tid == 0) { tr[3 * b + 1] = ta[0]; tr[3 * b + 2] = tb[0]; }
 }
 

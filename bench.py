@@ -2,13 +2,18 @@
 """Throughput of the sumcheck matmul prover on synthetic transformer-shaped layers.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--config decoder|qkv|ffn|moe|attn|ldd] [--layers L] [--tokens T] [--no-e2e] [--no-cpu-baseline]
+                    [--config decoder|qkv|ffn|moe|attn|ldd|commit] [--batched | --fs]
+                    [--layers L] [--tokens T] [--no-e2e] [--no-cpu-baseline]
 
 One step = one proving pass over the whole batch: eq tables, A~ / B~ partial evaluations, the
 claim C~, every sumcheck round, transcripts written.  The default workload is the audited decoder
 block: 32 layers x (QKV 4096x6144, O 4096x4096, FFN up 4096x14336, FFN down 14336x4096) at 8192
 tokens, 128 proofs, 39.25 GiB of int8/int32 inputs resident in HBM (far larger than L2, so no
 flush is needed between steps).  Rank 0 prints ONE JSON line.
+
+--batched proves the products of equal round count as one random-linear-combination proof each;
+--fs makes a step commit to every matrix (SHA-256 trees) and prove non-interactively; --config ldd
+and --config commit time the logit distances and the response commitments (their own metrics).
 
 --impl reference times the plain CPU oracle on the host cores, on a bounded sample of the same
 workload.  With N > 1 (launched by torch.distributed.run) every rank proves an independent

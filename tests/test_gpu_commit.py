@@ -121,3 +121,15 @@ def test_response_logits_of_the_benchmark_workload(imm, oracle):
     for i in range(requests):
         assert got[i] == C.commit(host[off[i]:off[i + 1]].tobytes(), rs[i])
     assert len(set(got)) == requests
+
+
+def test_message_beyond_four_gibibytes(imm, oracle):
+    """Byte offsets above 2^32 and three levels of launches (1.18 M leaves -> 9217 -> 10 -> 1)."""
+    n = (9 << 29) + 4096 * 3 + 5                       # 4.5 GiB and a bit
+    g = torch.Generator(device="cuda").manual_seed(7)
+    m = torch.randint(0, 256, (n,), dtype=torch.uint8, device="cuda", generator=g)
+    r = bytes(range(64, 96))
+    c = imm.Committer([m], [r])
+    assert c.launches == 4
+    got = bytes(c.commit().cpu().numpy()[0])
+    assert got == oracle.commitment.commit(m.cpu().numpy().tobytes(), r)

@@ -335,8 +335,9 @@ int imm_commit(const imm_commit_desc* descs_host, int n, uint8_t* d_digests, uin
  *              com_X the 32-byte commitments to the three matrices (imm_commit);
  *   r_row[t] = fe(H(0x11 || s_0 || le32(1) || le32(t))),  r_col[t] the same with le32(2);
  *   s_1      = H(0x12 || s_0 || le64(c0));
- *   round j:   s_{j+2} = H(0x13 || s_{j+1} || le64(g_j(0)) || le64(g_j(1)) || le64(g_j(2))),
- *              r_j = fe(s_{j+2}).
+ *   round j:   s_{j+2} = H(0x13 || s_{j+1} || le64(g_j(0)) || le64(g_j(2))),  r_j = fe(s_{j+2});
+ *              g_j(1) is in the transcript but not in the hash: the verifier's check
+ *              g_j(0) + g_j(1) = claim pins it, and the message stays one SHA-256 block.
  * The transcript has the layout of the interactive proof (3b+3 words). */
 
 /* Workspace bytes imm_sumcheck_matmul_prove_fs needs (0 on invalid input). */

@@ -14,8 +14,12 @@ The paper fixes none of this; the readings below are this build's.
   points      r_row[t] = fe(H(0x11 || s_0 || le32(1) || le32(t))), r_col[t] likewise with le32(2).
   claim       c0 = C~(r_row, r_col);  s_1 = H(0x12 || s_0 || le64(c0)).
   round j     the prover sends g_j(0), g_j(1), g_j(2);
-              s_{j+2} = H(0x13 || s_{j+1} || le64(g_j(0)) || le64(g_j(1)) || le64(g_j(2)));
+              s_{j+2} = H(0x13 || s_{j+1} || le64(g_j(0)) || le64(g_j(2)));
               r_j = fe(s_{j+2}); both tables fold with r_j.
+              g_j(1) is not hashed: the verifier requires g_j(0) + g_j(1) = claim, and the claim is
+              a function of what the state already binds, so g_j(1) carries nothing new -- and
+              without it the message is 49 bytes, one SHA-256 block instead of two, on the one
+              step of the proof that nothing can overlap.
   transcript  [c0, g_0(0..2), ..., g_{b-1}(0..2), a_fin, b_fin], as in the interactive proof.
 
 The field arithmetic of the steps (eq tables, the two partial evaluations, the claim) is the C
@@ -24,7 +28,7 @@ oracle's, called through its binding; the rounds are written out here in Python 
 Pins (tests/test_oracle_fs.py): every challenge re-derived with a SHA-256 written from the standard;
 every round polynomial against exhaustive hypercube sums in big integers at those challenges;
 g_j(0)+g_j(1) = running claim and the final product; each challenge depends on everything before it
-(commitments, shape, proof id, c0, earlier rounds); the verifier accepts the honest transcript and
+(commitments, shape, proof id, c0, g(0) and g(2) of earlier rounds); the verifier accepts the honest transcript and
 rejects every single-word change.
 """
 from __future__ import annotations
@@ -71,7 +75,8 @@ def absorb_claim(s0: bytes, c0: int) -> bytes:
 
 
 def absorb_round(s: bytes, g0: int, g1: int, g2: int) -> bytes:
-    return _h(b"\x13" + s + _le64(g0) + _le64(g1) + _le64(g2))
+    """g1 is part of the round's message but not of the hash (see the header)."""
+    return _h(b"\x13" + s + _le64(g0) + _le64(g2))
 
 
 def prove(A: np.ndarray, B: np.ndarray, C: np.ndarray, coms, proof_id: int):

@@ -957,7 +957,8 @@ int imm_fs_challenges(const imm_fe* transcript_host, int nrounds, const uint8_t*
             if (transcript_host[i] >= IMM_P) return IMM_ERR_NONCANONICAL;
         fs_absorb_host(s, 0x12, transcript_host, 1);
         for (int j = 0; j < nrounds; j++) {
-            fs_absorb_host(s, 0x13, transcript_host + 1 + 3 * j, 3);
+            const uint64_t hashed[2] = {transcript_host[1 + 3 * j], transcript_host[3 + 3 * j]};     // g_j(0), g_j(2)
+            fs_absorb_host(s, 0x13, hashed, 2);
             r_k_host[j] = fs_fe_host(s);
         }
     }

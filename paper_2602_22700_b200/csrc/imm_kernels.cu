@@ -733,7 +733,9 @@ sumcheck_kernel(const ProofDev* proofs, uint64_t seed, imm_fe* transcripts, int6
 //   s_0     = H(0x10 || com_A || com_B || com_C || le64(m) || le64(k) || le64(n) || le64(proof_id))
 //   r_row[t] = fe(H(0x11 || s_0 || le32(1) || le32(t))),  r_col[t] with le32(2)
 //   s_1     = H(0x12 || s_0 || le64(c0))
-//   s_{j+2} = H(0x13 || s_{j+1} || le64(g_j(0)) || le64(g_j(1)) || le64(g_j(2))),  r_j = fe(s_{j+2})
+//   s_{j+2} = H(0x13 || s_{j+1} || le64(g_j(0)) || le64(g_j(2))),  r_j = fe(s_{j+2})
+// (g_j(1) is sent but not hashed: the verifier's sum check pins it to the claim; without it the
+// message is one SHA-256 block)
 
 __device__ __forceinline__ uint64_t fs_fe(const uint32_t (&h)[8])
 {
@@ -746,7 +748,7 @@ __device__ __forceinline__ void fs_put_le(uint8_t* dst, uint64_t v, int nbytes)
     for (int q = 0; q < nbytes; q++) dst[q] = (uint8_t)(v >> (8 * q));
 }
 
-// s <- H(tag || s || le64(vals[0..NV))), NV = 1 or 3.  The message is the word stream
+// s <- H(tag || s || le64(vals[0..NV))), NV = 1 or 2.  The message is the word stream
 // [s_0..s_7, byte-swapped halves of the values] moved one byte to the right behind the tag, so its
 // words are built with shifts instead of byte by byte (the hash sits on the rounds' critical path:
 // one thread, nothing to overlap it with).
@@ -781,7 +783,7 @@ __device__ __forceinline__ void fs_absorb(uint32_t (&s)[8], uint32_t tag, const 
             for (int i = 0; i < 15; i++) w[i] = 0;
             w[15] = bits;
         }
-        imm_sha::compress_compact(s, w, one);
+        imm_sha::compress(s, w, one);
     }
 }
 
@@ -894,7 +896,8 @@ sumcheck_fs_kernel(const ProofDev* proofs, const FsProof* fs, imm_fe* transcript
         block_sum3_fe(g, red3);                            // (its barriers also order the fold's writes before the next reads)
         if (tid == 0) {
             tr[1 + 3 * j] = g[0]; tr[2 + 3 * j] = g[1]; tr[3 + 3 * j] = g[2];
-            fs_absorb<3>(st, 0x13, g, f.one);
+            const uint64_t hashed[2] = {g[0], g[2]};
+            fs_absorb<2>(st, 0x13, hashed, f.one);
             r_sh = fs_fe(st);
         }
         __syncthreads();

@@ -95,28 +95,6 @@ __host__ __device__ __forceinline__ void compress(uint32_t (&h)[8], uint32_t (&w
     h[0] += a; h[1] += b; h[2] += c; h[3] += d; h[4] += e; h[5] += f; h[6] += g; h[7] += hh;
 }
 
-// The same function in a quarter of the code: four trips through one sixteen-round body, the
-// message schedule skipped on the first.  For a lone thread hashing on a critical path (transcript
-// hashing), where straight-line code is fetched once per use and the fetch is what the warp waits for.
-__host__ __device__ __forceinline__ void compress_compact(uint32_t (&h)[8], uint32_t (&w)[16], uint32_t one)
-{
-    uint32_t a = h[0], b = h[1], c = h[2], d = h[3], e = h[4], f = h[5], g = h[6], hh = h[7];
-#pragma unroll 1
-    for (int base = 0; base < 64; base += 16) {
-#pragma unroll
-        for (int j = 0; j < 16; j++) {
-            if (base != 0) {
-                const uint32_t w15 = w[(j + 1) & 15], w2 = w[(j + 14) & 15];
-                const uint32_t s0 = rotr(w15, 7) ^ rotr(w15, 18) ^ (w15 >> 3);
-                const uint32_t s1 = rotr(w2, 17) ^ rotr(w2, 19) ^ (w2 >> 10);
-                w[j] = add_m(add_m(w[j], s0, one), add_m(w[(j + 9) & 15], s1, one), one);
-            }
-            IMM_SHA_ROUND(add_m(w[j], kc(base + j), one));
-        }
-    }
-    h[0] += a; h[1] += b; h[2] += c; h[3] += d; h[4] += e; h[5] += f; h[6] += g; h[7] += hh;
-}
-
 #undef IMM_SHA_ROUND
 
 // SHA-256 of a short message held in addressable memory (a few blocks: statement and transcript

@@ -35,7 +35,7 @@ def derive_independently(t, b, coms, m, k, n, pid):
     s = sha256_py(b"\x12" + s0 + le(t[0], 8))
     r_k = []
     for j in range(b):
-        s = sha256_py(b"\x13" + s + b"".join(le(w, 8) for w in t[1 + 3 * j:4 + 3 * j]))
+        s = sha256_py(b"\x13" + s + le(t[1 + 3 * j], 8) + le(t[3 + 3 * j], 8))      # g_j(0), g_j(2); not g_j(1)
         r_k.append(to_fe(s))
     return r_row, r_col, r_k
 
@@ -90,12 +90,17 @@ def test_every_challenge_depends_on_everything_before_it(oracle):
         other = oracle.fs.challenges(t, 3, coms, *dims, pid)
         assert all(x != y for x, y in zip(flat(base), flat(other)))
     assert all(x != y for x, y in zip(flat(base), flat(oracle.fs.challenges(t, 3, coms, m, k, n, pid + 1))))
-    # transcript: word i moves every round challenge drawn after it and none before
+    # transcript: c0, g_j(0) and g_j(2) move every round challenge drawn after them and none before;
+    # g_j(1) is not hashed (the sum check pins it to the claim)
     for pos in range(1 + 3 * 3):
         u = list(t)
         u[pos] = (u[pos] + 1) % P
         other = oracle.fs.challenges(u, 3, coms, m, k, n, pid)
         assert other[0] == base[0] and other[1] == base[1]
+        if pos > 0 and (pos - 1) % 3 == 1:
+            assert other == base
+            assert oracle.fs.verify(u, 3, coms, m, k, n, pid) == (oracle.REJECT, (pos - 1) // 3)
+            continue
         first = 0 if pos == 0 else (pos - 1) // 3
         assert other[2][:first] == base[2][:first]
         assert all(x != y for x, y in zip(other[2][first:], base[2][first:]))

@@ -310,8 +310,9 @@ void orc_matmul_i8_i32(const int8_t* A, const int8_t* B, int32_t* C,
 }
 
 /* ---------------------------------------------------------------------------------------
- * Batched proof: P product claims C_p = A_p * B_p with the same number of rounds b are proved
- * by ONE sumcheck of their random linear combination (the standard batching of sumcheck claims
+ * Batched proof: P product claims C_p = A_p * B_p are proved by ONE sumcheck of their random
+ * linear combination over b = max_p ceil(log2 k_p) variables (a member with a smaller k is
+ * zero-padded to 2^b like any other: padding k changes neither its product nor its claim) (the standard batching of sumcheck claims
  * over a common hypercube; the paper lists the products to prove -- attention and MLPs,
  * Section 4.1 -- and leaves the proof system and any batching open).
  *
@@ -327,7 +328,7 @@ void orc_matmul_i8_i32(const int8_t* A, const int8_t* B, int32_t* C,
  * transcript (1 + 3b + 3P words):
  *   [c0^B, g_0^B(0..2), ..., g_{b-1}^B(0..2), (c0_0, a_fin_0, b_fin_0), ..., (c0_{P-1}, ...)].
  * Every proof keeps its own vectors; there is no sharing of work between proofs beyond the
- * challenges.  Returns ORC_ERR_ARG for a bad shape or proofs whose round counts differ.   */
+ * challenges.  Returns ORC_ERR_ARG for a bad shape.                                       */
 int orc_sumcheck_matmul_prove_batched(int P, const int8_t* const* A, const int8_t* const* B,
                                       const int32_t* const* C, const int64_t* m, const int64_t* k,
                                       const int64_t* n, const int64_t* lda, const int64_t* ldb,
@@ -339,9 +340,9 @@ int orc_sumcheck_matmul_prove_batched(int P, const int8_t* const* A, const int8_
     for (int p = 0; p < P; p++)
         if (m[p] <= 0 || k[p] <= 0 || n[p] <= 0 || lda[p] < k[p] || ldb[p] < n[p] || ldc[p] < n[p])
             return ORC_ERR_ARG;
-    int b = orc_ceil_log2(k[0]);
-    for (int p = 1; p < P; p++)
-        if (orc_ceil_log2(k[p]) != b) return ORC_ERR_ARG;
+    int b = 0;
+    for (int p = 0; p < P; p++)
+        if (orc_ceil_log2(k[p]) > b) b = orc_ceil_log2(k[p]);
     int64_t kp = (int64_t)1 << b;
 
     uint64_t** av = (uint64_t**)calloc((size_t)P, sizeof(uint64_t*));

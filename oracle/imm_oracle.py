@@ -253,11 +253,12 @@ def sumcheck_verify(transcript, nrounds: int, seed: int, proof_id: int, expect_c
 
 
 def batched_transcript_len(k: int, nproofs: int) -> int:
+    """k: the largest inner dimension of the batch."""
     return 1 + 3 * ceil_log2(k) + 3 * nproofs
 
 
 def sumcheck_matmul_prove_batched(problems, seed: int, batch_id: int) -> np.ndarray:
-    """``problems`` is a sequence of (A, B, C, proof_id) whose k pad to the same power of two."""
+    """``problems`` is a sequence of (A, B, C, proof_id); every k is padded to the largest 2^b."""
     mats, dims, ptrs = [], [], [[], [], []]
     for A, B, C, _ in problems:
         A, ca, m, k, lda = _mat(A)
@@ -272,7 +273,7 @@ def sumcheck_matmul_prove_batched(problems, seed: int, batch_id: int) -> np.ndar
     parr = [np.array(lst, dtype=np.uint64) for lst in ptrs]
     darr = [np.array([d[i] for d in dims], dtype=np.int64) for i in range(6)]
     ids = np.array([int(p[3]) for p in problems], dtype=np.uint64)
-    out = np.empty(batched_transcript_len(dims[0][1], count) if count else 0, dtype=np.uint64)
+    out = np.empty(batched_transcript_len(max(d[1] for d in dims), count) if count else 0, dtype=np.uint64)
     rc = lib().orc_sumcheck_matmul_prove_batched(count, *[_ptr(a) for a in parr],
                                                  *[_ptr(a) for a in darr], seed, batch_id,
                                                  _ptr(ids), _ptr(out))

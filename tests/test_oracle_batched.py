@@ -148,11 +148,40 @@ def test_one_wrong_member_sinks_the_batch(oracle, which):
     assert oracle.sumcheck_verify_batched(bad, b, 3, seed, bid) == (oracle.REJECT, 0)
 
 
-def test_members_must_share_the_round_count(oracle):
-    rng = random.Random(1)
-    probs = group(rng, [(2, 4, 2), (2, 5, 2)])
-    with pytest.raises(ValueError):
-        oracle.sumcheck_matmul_prove_batched(probs, 1, 1)
+def zero_padded(A, B, kp):
+    """The same product with the inner dimension padded to kp by zero columns of A and zero rows of B."""
+    m, k = A.shape
+    Ap = np.zeros((m, kp), dtype=A.dtype)
+    Ap[:, :k] = A
+    Bp = np.zeros((kp, B.shape[1]), dtype=B.dtype)
+    Bp[:k] = B
+    return Ap, Bp
+
+
+def test_members_of_different_inner_size_are_padded_to_the_largest(oracle):
+    """k = 3, 16, 1, 6 in one batch: four rounds for everybody.  Against the exhaustive definition on
+    explicitly padded matrices, and against the batch of those padded matrices itself."""
+    rng = random.Random(31)
+    shapes = [(2, 3, 3), (1, 16, 2), (3, 1, 1), (2, 6, 4)]
+    probs = group(rng, shapes)
+    seed, bid, b = 8, 15, 4
+    t = oracle.sumcheck_matmul_prove_batched(probs, seed, bid)
+    c0B, rounds, tail = split(t, b, 4)
+    padded = [zero_padded(A, B, 16) + (C, pid) for A, B, C, pid in probs]
+    assert [int(w) for w in oracle.sumcheck_matmul_prove_batched(padded, seed, bid)] == [int(w) for w in t]
+    rho, r_k = chal(oracle, seed, bid, 4, 4), chal(oracle, seed, bid, 3, b)
+    claim = c0B
+    for j in range(b):
+        g = [0, 0, 0]
+        for r, (Ap, Bp, C, pid) in zip(rho, padded):
+            rr = chal(oracle, seed, pid, 1, clog2(Ap.shape[0]))
+            rc = chal(oracle, seed, pid, 2, clog2(Bp.shape[1]))
+            for X in (0, 1, 2):
+                g[X] = (g[X] + r * round_poly_by_definition(Ap.tolist(), Bp.tolist(), rr, rc, r_k[:j], X)) % P
+        assert rounds[j] == g and (g[0] + g[1]) % P == claim
+        claim = interp_deg2(g[0], g[1], g[2], r_k[j])
+    assert claim == sum(r * x[1] * x[2] for r, x in zip(rho, tail)) % P
+    assert oracle.sumcheck_verify_batched(t, b, 4, seed, bid) == (oracle.OK, -1)
 
 
 def test_zero_round_batch(oracle):

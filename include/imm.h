@@ -236,8 +236,9 @@ int imm_sumcheck_verify(const imm_fe* transcript_host, int nrounds, uint64_t see
  * Batched proof: one sumcheck for a random linear combination of product claims
  * ---------------------------------------------------------------------------------------------
  * The products a proof of the reference execution must cover are many (the attention and MLP
- * products of every layer, Section 4.1).  Claims whose k pad to the same 2^b can share one
- * sumcheck: with public coins rho_p = imm_challenge(seed, batch_id, 4, p) the prover shows
+ * products of every layer, Section 4.1).  They can share one sumcheck over b = max_p ceil(log2 k_p)
+ * variables (a smaller k is zero-padded to 2^b like any other, which changes neither the product
+ * nor the claim): with public coins rho_p = imm_challenge(seed, batch_id, 4, p) the prover shows
  *   sum_p rho_p * sum_y A_p~(r_row_p, y) B_p~(y, r_col_p) = sum_p rho_p C_p~(r_row_p, r_col_p),
  * all proofs folding with the same round challenges r_j = imm_challenge(seed, batch_id, 3, j);
  * r_row_p and r_col_p stay each proof's own (domains 1, 2 under its proof_id).  The verifier then
@@ -252,16 +253,15 @@ int imm_sumcheck_verify(const imm_fe* transcript_host, int nrounds, uint64_t see
 /* Transcript words of a batched proof (0 on invalid arguments). */
 int64_t imm_sumcheck_batched_transcript_len(int nrounds, int nproofs);
 
-/* Workspace bytes imm_sumcheck_matmul_prove_batched needs (0 on invalid input, which includes
- * proofs whose ceil(log2 k) differ). */
+/* Workspace bytes imm_sumcheck_matmul_prove_batched needs (0 on invalid input). */
 size_t imm_sumcheck_matmul_batched_workspace(const imm_matmul_desc* descs_host, int nproofs);
 
 /* Batched prover.  Runs the launch sequence of imm_sumcheck_matmul_prove with the shared round
  * challenges (per-proof transcripts go to the workspace), then one more launch forms the
  * batched transcript.
- *   descs_host   : HOST array of nproofs descriptors with DEVICE matrix pointers; every
- *                  ceil(log2 k) must be the same, else IMM_ERR_SHAPE
- *   d_transcript : DEVICE array of imm_sumcheck_batched_transcript_len(b, nproofs) words
+ *   descs_host   : HOST array of nproofs descriptors with DEVICE matrix pointers
+ *   d_transcript : DEVICE array of imm_sumcheck_batched_transcript_len(b, nproofs) words,
+ *                  b = ceil(log2 of the largest k)
  *   d_status     : DEVICE array of nproofs int32 (as imm_sumcheck_matmul_prove)
  *   d_ws         : DEVICE workspace, 256-byte aligned, >= imm_sumcheck_matmul_batched_workspace(...)
  * Errors: IMM_ERR_ARG, IMM_ERR_SHAPE, IMM_ERR_ALIGN, IMM_ERR_WORKSPACE, IMM_ERR_LIMIT (more than

@@ -619,7 +619,8 @@ size_t imm_sumcheck_matmul_workspace(const imm_matmul_desc* descs_host, int npro
 }
 
 // The launch sequence of a batch.  shared_round_id: null = every proof draws its round challenges
-// under its own proof_id; else all proofs draw them under that one id (a batched proof).
+// under its own proof_id and runs its own ceil(log2 k) rounds; else all proofs draw them under that
+// one id and run the rounds of the largest k (a batched proof).
 // fs: null = public coins from the generator; else the challenges are hashed from the commitments
 // and the transcript (non-interactive proof) and fs describes the extra device arrays.
 struct FsArgs {
@@ -688,7 +689,7 @@ static int prove_batch(const imm_matmul_desc* descs_host, int nproofs, uint64_t 
         P.part_c = (imm_fe*)(base + q.part_c);
         P.round_id = shared_round_id ? *shared_round_id : d.proof_id;
         P.m = (int32_t)d.m; P.k = (int32_t)d.k; P.n = (int32_t)d.n;
-        P.a = q.a; P.b = q.b; P.c = q.c;
+        P.a = q.a; P.b = shared_round_id ? p.max_b : q.b; P.c = q.c;   // a batched proof pads every k to the largest 2^b
         P.n_part_a = q.n_part_a; P.n_part_b = q.n_part_b; P.n_part_c = q.n_part_c;
         P.sum_row = (imm_fe*)(base + q.sum_row); P.sum_col = (imm_fe*)(base + q.sum_col);
         P.n_sum_row = q.n_sum_row; P.n_sum_col = q.n_sum_col;
@@ -809,9 +810,7 @@ static int batched_layout(const imm_matmul_desc* descs_host, int nproofs, int* b
     Plan p = make_plan(descs_host, nproofs);
     if (p.status != IMM_OK) return p.status;
     if (nproofs > IMM_BATCH_MAX_PROOFS) return IMM_ERR_LIMIT;
-    *b = ceil_log2(descs_host[0].k);
-    for (int i = 1; i < nproofs; i++)
-        if (ceil_log2(descs_host[i].k) != *b) return IMM_ERR_SHAPE;
+    *b = p.max_b;
     *rows_bytes = align_up((size_t)nproofs * (size_t)(3 * *b + 3) * sizeof(imm_fe));
     *total = *rows_bytes + p.total_bytes;
     return IMM_OK;

@@ -380,14 +380,14 @@ def batched_transcript_len(nrounds: int, nproofs: int) -> int:
 
 
 class BatchedProver:
-    """One sumcheck for a random linear combination of product claims whose k pad to the same
-    power of two.  Holds descriptors, workspace and outputs; ``prove`` allocates nothing."""
+    """One sumcheck for a random linear combination of product claims (every k padded to the largest
+    2^b).  Holds descriptors, workspace and outputs; ``prove`` allocates nothing."""
 
     def __init__(self, problems, device="cuda"):
         self.problems = list(problems)
         self.descs = make_descs(self.problems)
         self.nproofs = len(self.problems)
-        self.nrounds = ceil_log2(self.problems[0][0].shape[1])
+        self.nrounds = max(ceil_log2(A.shape[1]) for (A, _, _, _) in self.problems)
         need = lib().imm_sumcheck_matmul_batched_workspace(ctypes.addressof(self.descs), self.nproofs)
         if need == 0:
             raise ImmError(ERR_SHAPE, "imm_sumcheck_matmul_batched_workspace")

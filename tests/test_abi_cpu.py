@@ -67,13 +67,14 @@ def test_host_verifier_matches_oracle_verifier(imm, oracle):
 
 def test_batched_host_verifier_matches_oracle_verifier(imm, oracle):
     rng = random.Random(3)
-    for shapes in ([(3, 8, 2), (2, 5, 4), (1, 7, 1)], [(2, 1, 2), (1, 1, 3)], [(4, 16, 4)]):
+    for shapes in ([(3, 8, 2), (2, 5, 4), (1, 7, 1)], [(2, 1, 2), (1, 1, 3)], [(4, 16, 4)], [(2, 3, 2), (1, 9, 1)]):
         probs = []
         for i, (m, k, n) in enumerate(shapes):
             A = np.array([[rng.randint(-128, 127) for _ in range(k)] for _ in range(m)], dtype=np.int8)
             B = np.array([[rng.randint(-128, 127) for _ in range(n)] for _ in range(k)], dtype=np.int8)
             probs.append((A, B, (A.astype(np.int64) @ B.astype(np.int64)).astype(np.int32), 100 + i))
-        seed, bid, b, count = rng.getrandbits(64), rng.getrandbits(30), oracle.ceil_log2(shapes[0][1]), len(shapes)
+        seed, bid, count = rng.getrandbits(64), rng.getrandbits(30), len(shapes)
+        b = max(oracle.ceil_log2(k) for (_, k, _) in shapes)
         t = [int(w) for w in oracle.sumcheck_matmul_prove_batched(probs, seed, bid)]
         assert len(t) == imm.batched_transcript_len(b, count)
         assert imm.sumcheck_verify_batched(t, b, count, seed, bid) == (imm.OK, -1)
@@ -156,10 +157,9 @@ def test_batched_workspace_and_validation(imm):
     plain = L.imm_sumcheck_matmul_workspace(ctypes.addressof(d), 2)
     need = L.imm_sumcheck_matmul_batched_workspace(ctypes.addressof(d), 2)
     assert need >= plain + 2 * 39 * 8 and need % 256 == 0
-    mixed = _desc_array(imm, [(64, 4096, 64), (64, 2048, 64)])
-    assert L.imm_sumcheck_matmul_batched_workspace(ctypes.addressof(mixed), 2) == 0
+    mixed = _desc_array(imm, [(64, 4096, 64), (64, 2048, 64)])                  # padded to twelve rounds each
+    assert L.imm_sumcheck_matmul_batched_workspace(ctypes.addressof(mixed), 2) >= 2 * 39 * 8
     prove = L.imm_sumcheck_matmul_prove_batched
-    assert prove(ctypes.addressof(mixed), 2, 1, 1, 0x1000, 0x1000, 0x1000, 1 << 30, None) == imm.ERR_SHAPE
     assert prove(ctypes.addressof(d), 2, 1, 1, 0x1000, 0x1000, 0x1000, need - 1, None) == imm.ERR_WORKSPACE
     assert prove(ctypes.addressof(d), 2, 1, 1, 0x1000, 0x1000, 0x1010, need, None) == imm.ERR_ALIGN
     assert prove(ctypes.addressof(d), 2, 1, 1, None, 0x1000, 0x1000, need, None) == imm.ERR_ARG

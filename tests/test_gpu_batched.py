@@ -57,7 +57,7 @@ def test_batched_transcript_equals_oracle(imm, oracle, backend, shapes):
     want = [int(w) for w in oracle.sumcheck_matmul_prove_batched(group, seed, bid)]
     got = imm.sumcheck_matmul_prove_batched(on_gpu(group), seed, bid)
     assert got == want
-    b = oracle.ceil_log2(shapes[0][1])
+    b = max(oracle.ceil_log2(k) for (_, k, _) in shapes)
     assert imm.sumcheck_verify_batched(got, b, len(shapes), seed, bid) == (imm.OK, -1)
 
 
@@ -144,9 +144,12 @@ def test_repeated_and_interleaved_calls_reuse_buffers(imm, oracle):
         assert t == [int(w) for w in oracle.sumcheck_matmul_prove(A, B, C, 5, pid)]
 
 
-def test_members_with_different_round_counts_are_refused(imm):
+def test_members_of_different_inner_size_share_the_longest_round_count(imm, oracle, backend):
+    """k from 1 to 5000 in one batch: thirteen rounds for every member (tables zero beyond each k)."""
     rng = np.random.default_rng(1)
-    dev = on_gpu(make_group(rng, [(4, 64, 4), (4, 65, 4)]))
-    with pytest.raises(imm.ImmError) as e:
-        imm.BatchedProver(dev)
-    assert e.value.code == imm.ERR_SHAPE
+    shapes = [(4, 64, 4), (4, 65, 4), (9, 1, 3), (2, 5000, 7), (130, 300, 2), (1, 4096, 1)]
+    group = make_group(rng, shapes, first_id=40)
+    got = imm.sumcheck_matmul_prove_batched(on_gpu(group), 6, 7)
+    assert got == [int(w) for w in oracle.sumcheck_matmul_prove_batched(group, 6, 7)]
+    assert len(got) == 1 + 39 + 18
+    assert imm.sumcheck_verify_batched(got, 13, 6, 6, 7) == (imm.OK, -1)

@@ -161,25 +161,24 @@ def test_decoder_block_in_bench_geometry(imm, oracle, synth, tokens):
         assert got[i][-1] == two_sided(oracle, B, r_k, r_col)
         check_sampled_entries_of_C(p, rng, 8)
 
-    # The same products as two batched proofs (96 members of twelve rounds, 32 of fourteen): the
-    # verifier accepts each; every member's c0 is the one of its own proof above; for sampled
-    # members a_fin and b_fin are the oracle's evaluations at the batch's shared point.
+    # The same products as ONE batched proof (every k padded to 2^14): the verifier accepts it; every
+    # member's c0 is the one of its own proof above; for sampled members a_fin and b_fin are the
+    # oracle's evaluations at the batch's shared point.
     del prover
-    for b, count, bid in ((12, 96, 4242), (14, 32, 4243)):
-        idx = [i for i, p in enumerate(probs) if imm.ceil_log2(p.mkn[1]) == b]
-        assert len(idx) == count
-        bt = imm.sumcheck_matmul_prove_batched([(probs[i].A, probs[i].B, probs[i].C, probs[i].proof_id)
-                                                for i in idx], SEED, bid)
-        assert len(bt) == 1 + 3 * b + 3 * count
-        assert imm.sumcheck_verify_batched(bt, b, count, SEED, bid) == (imm.OK, -1)
-        tail = bt[1 + 3 * b:]
-        assert [tail[3 * j] for j in range(count)] == [got[i][0] for i in idx]
-        r_k = oracle.challenges(SEED, bid, 3, b)
-        for j in sorted(int(v) for v in rng.choice(count, size=2, replace=False)):
-            p = probs[idx[j]]
-            m, k, n = p.mkn
-            r_row = oracle.challenges(SEED, p.proof_id, 1, oracle.ceil_log2(m))
-            r_col = oracle.challenges(SEED, p.proof_id, 2, oracle.ceil_log2(n))
-            A, B, _ = host(p)
-            assert tail[3 * j + 1] == two_sided(oracle, A, r_row, r_k)
-            assert tail[3 * j + 2] == two_sided(oracle, B, r_k, r_col)
+    b, count, bid = 14, 128, 4242
+    bt = imm.sumcheck_matmul_prove_batched([(p.A, p.B, p.C, p.proof_id) for p in probs], SEED, bid)
+    assert len(bt) == 1 + 3 * b + 3 * count
+    assert imm.sumcheck_verify_batched(bt, b, count, SEED, bid) == (imm.OK, -1)
+    tail = bt[1 + 3 * b:]
+    assert [tail[3 * j] for j in range(count)] == [got[i][0] for i in range(count)]
+    r_k = oracle.challenges(SEED, bid, 3, b)
+    e_k = oracle.eq_table(r_k)
+    for j in sorted(int(v) for v in rng.choice(count, size=3, replace=False)):
+        p = probs[j]
+        m, k, n = p.mkn
+        e_row = oracle.eq_table(oracle.challenges(SEED, p.proof_id, 1, oracle.ceil_log2(m)))
+        e_col = oracle.eq_table(oracle.challenges(SEED, p.proof_id, 2, oracle.ceil_log2(n)))
+        A, B, _ = host(p)
+        # (the first k entries of the 2^14-entry table weigh the real inner indices; the rest meet zero padding)
+        assert tail[3 * j + 1] == oracle.mle_eval_point(A, e_row, e_k)
+        assert tail[3 * j + 2] == oracle.mle_eval_point(B, e_k, e_col)

@@ -212,12 +212,12 @@ def measured_peaks():
 # profiles/ (dram__bytes_read.sum + dram__bytes_write.sum over 4*m*n); None until a capture of the
 # current kernel exists.
 LDD_TVKL_TRAFFIC_RATIO = 1.0721 / 1.050673   # tv_kl_kernel<aligned, 512 threads>: (dram read + write) / (8 bytes per entry pair)
-COMMIT_TRAFFIC_RATIO = (1.070806 + 0.018732) / 1.050673152                   # commit_leaf_kernel: (dram read + write) / message bytes
+COMMIT_TRAFFIC_RATIO = (1.077891 + 0.018910) / 1.050673152                   # commit_leaf_kernel: (dram read + write) / message bytes
 # SHA-256 leaf hashing against the integer ALU pipe (rotates, three-input logic, byte permutes): the
-# pipe retires 64 thread instructions per cycle per SM; the kernel issues 17.55 of them per hashed
-# byte (ncu: 576.3 M warp instructions on that pipe for 1.0507 GB), so at 1965 MHz the pipe allows
-# 148 x 64 x 1.965e9 / 17.55 = 1060 GB/s.
-COMMIT_ALU_PEAK_GBS_AT_1965 = 1060.0
+# pipe retires 64 thread instructions per cycle per SM; the kernel issues 17.18 of them per hashed
+# byte (ncu: 564.2 M warp instructions on that pipe for 1.0507 GB), so at 1965 MHz the pipe allows
+# 148 x 64 x 1.965e9 / 17.18 = 1083 GB/s.
+COMMIT_ALU_PEAK_GBS_AT_1965 = 1083.0
 CLAIM_KERNEL_TRAFFIC_RATIO = 239.64 / 234.881024  # bytedot_kernel<1,1,1>: (dram read + write) / (4 bytes per entry), small-case capture
 
 
@@ -651,9 +651,9 @@ def run_commit(args):
                    "parallelism": "1 GPU" if world == 1 else f"{world} independent replicas, no collective"},
         "hbm_gbs_whole_step": gbs,
         "roofline": {"kernel": "commit_leaf_kernel (SHA-256 of 4096-byte leaves, one per thread); timed as the whole imm_commit "
-                               "call, of which the leaf kernel is 96 % in the launch list", "bound": "alu",
+                               "call, of which the leaf kernel is 97 % in the launch list", "bound": "alu",
                      "achieved": gbs, "peak": alu_peak, "unit": "GB/s", "frac": gbs / alu_peak,
-                     "peak_kind": "integer ALU pipe: 148 SMs x 64 lanes x sampled SM clock / 17.55 ALU instructions per hashed byte",
+                     "peak_kind": "integer ALU pipe: 148 SMs x 64 lanes x sampled SM clock / 17.18 ALU instructions per hashed byte",
                      "traffic": (COMMIT_TRAFFIC_RATIO * nbytes) if COMMIT_TRAFFIC_RATIO else None},
         "gpu_launches": com.launches * steps,
         "clocks": clocks,

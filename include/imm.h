@@ -310,6 +310,9 @@ typedef struct {
 /* Workspace bytes imm_commit needs for this batch (0 on invalid input). */
 size_t imm_commit_workspace(const imm_commit_desc* descs_host, int n);
 
+/* Kernel launches imm_commit enqueues for this batch (0 on invalid input). */
+int imm_commit_launches(const imm_commit_desc* descs_host, int n);
+
 /* Commits to every message of the batch.
  *   descs_host : HOST array of n descriptors (at most IMM_COMMIT_MAX_MESSAGES, each message at
  *                most IMM_COMMIT_MAX_BYTES)
@@ -317,9 +320,9 @@ size_t imm_commit_workspace(const imm_commit_desc* descs_host, int n);
  *   d_roots    : DEVICE array of n x 32 bytes for the tree roots, or NULL
  *   d_ws       : DEVICE workspace, 256-byte aligned, >= imm_commit_workspace(...) bytes
  * Messages whose pointer is 16-byte aligned are read with 128-bit loads, others byte by byte
- * (slow).  The batch is one leaf launch (one thread per leaf; the 128 leaves of a block fold to a
- * subtree root on chip), one launch per further factor of 1024 in the largest leaf count, and a
- * final launch; all are enqueued on `stream`, nothing is synchronised or allocated.
+ * (slow).  The batch is one leaf launch (one thread per leaf; the 128 to 512 leaves of a block fold
+ * to a subtree root on chip), one launch per further factor of 1024 in the largest count of subtree
+ * roots, and a final launch; all are enqueued on `stream`, nothing is synchronised or allocated.
  * Errors: IMM_ERR_ARG, IMM_ERR_LIMIT, IMM_ERR_ALIGN, IMM_ERR_WORKSPACE, IMM_ERR_CUDA. */
 int imm_commit(const imm_commit_desc* descs_host, int n, uint8_t* d_digests, uint8_t* d_roots,
                void* d_ws, size_t ws_bytes, void* stream);

@@ -12,7 +12,7 @@
 // the work is bound by integer-pipe instruction issue, not by HBM: the rotates and the logic fill
 // the integer ALU pipe (one warp instruction per two cycles per SM sub-partition); the adds are
 // written as multiply-adds so that they issue on the other pipe.  One thread hashes one leaf
-// (65 compressions); the 128 leaves of a block are then folded to one subtree root in shared
+// (65 compressions); the 128 to 512 leaves of a block are then folded to one subtree root in shared
 // memory, so the leaf digests never go to global memory.  Later passes fold 1024 digests per block
 // until every message has one root, and a last launch forms the commitments.
 #include <cuda_runtime.h>
@@ -27,7 +27,14 @@
 namespace imm_hash {
 
 constexpr int LEAF = IMM_COMMIT_LEAF;         // bytes per leaf
-constexpr int LEAF_THREADS = 128;             // leaves per block of the leaf pass
+// Leaves per block of the leaf pass: large blocks for large batches (measured on 4 GiB: 128 threads
+// 852 GB/s, 256 881, 512 900, 1024 853), small ones when the batch has few leaves to spread over the SMs.
+inline int pick_leaf_threads(uint64_t total_leaves)
+{
+    if (total_leaves >= 200000) return 512;
+    if (total_leaves >= 16384) return 256;
+    return 128;
+}
 constexpr int NODE_THREADS = 1024;            // digests per block of a node pass
 constexpr size_t ALIGN = 256;
 
@@ -167,6 +174,7 @@ __device__ __forceinline__ int find_pass_job(const PassJob* jobs, int njobs, uin
     return lo;
 }
 
+template <int LEAF_THREADS>
 __global__ void __launch_bounds__(LEAF_THREADS) commit_leaf_kernel(const PassJob* jobs, int njobs)
 {
     __shared__ Digest sd[LEAF_THREADS];
@@ -242,6 +250,7 @@ struct Plan {
     std::vector<std::vector<Entry>> passes;
     std::vector<size_t> root_off;              // where each message's root ends up
     std::vector<size_t> pass_hdr_off;          // PassJob arrays in the header
+    int leaf_threads = 128;
     size_t final_hdr_off = 0, header_bytes = 0, total_bytes = 0;
 };
 
@@ -257,11 +266,14 @@ Plan make_plan(const imm_commit_desc* descs, int n)
         if (descs[i].nbytes > IMM_COMMIT_MAX_BYTES) { p.status = IMM_ERR_LIMIT; return p; }
         count[i] = descs[i].nbytes == 0 ? 1 : (descs[i].nbytes + LEAF - 1) / LEAF;
     }
+    uint64_t total_leaves = 0;
+    for (int i = 0; i < n; i++) total_leaves += count[i];
+    p.leaf_threads = pick_leaf_threads(total_leaves);
     // digest arrays after the header; sizes first, offsets are rebased once the header size is known
     size_t dig = 0;
     p.root_off.assign(n, 0);
     for (int pass = 0;; pass++) {
-        const uint64_t per = pass == 0 ? LEAF_THREADS : NODE_THREADS;
+        const uint64_t per = pass == 0 ? (uint64_t)p.leaf_threads : NODE_THREADS;
         std::vector<Plan::Entry> es;
         uint64_t groups_total = 0;
         for (int i = 0; i < n; i++) {
@@ -307,6 +319,12 @@ size_t imm_commit_workspace(const imm_commit_desc* descs_host, int n)
     return p.status == IMM_OK ? p.total_bytes : 0;
 }
 
+int imm_commit_launches(const imm_commit_desc* descs_host, int n)
+{
+    Plan p = make_plan(descs_host, n);
+    return p.status == IMM_OK ? (int)p.passes.size() + 1 : 0;
+}
+
 int imm_commit(const imm_commit_desc* descs_host, int n, uint8_t* d_digests, uint8_t* d_roots,
                void* d_ws, size_t ws_bytes, void* stream)
 {
@@ -350,7 +368,11 @@ int imm_commit(const imm_commit_desc* descs_host, int n, uint8_t* d_digests, uin
     for (size_t ps = 0; ps < p.passes.size(); ps++) {
         const PassJob* d_jobs = (const PassJob*)(base + p.pass_hdr_off[ps]);
         const int njobs = (int)p.passes[ps].size();
-        if (ps == 0) commit_leaf_kernel<<<blocks[ps], LEAF_THREADS, 0, st>>>(d_jobs, njobs);
+        if (ps == 0) {
+            if (p.leaf_threads == 512) commit_leaf_kernel<512><<<blocks[ps], 512, 0, st>>>(d_jobs, njobs);
+            else if (p.leaf_threads == 256) commit_leaf_kernel<256><<<blocks[ps], 256, 0, st>>>(d_jobs, njobs);
+            else commit_leaf_kernel<128><<<blocks[ps], 128, 0, st>>>(d_jobs, njobs);
+        }
         else commit_node_kernel<<<blocks[ps], NODE_THREADS, 0, st>>>(d_jobs, njobs);
         if (cudaGetLastError() != cudaSuccess) return IMM_ERR_CUDA;
     }

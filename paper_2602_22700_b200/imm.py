@@ -33,7 +33,7 @@ EXPORTS = ("imm_version", "imm_last_cuda_error", "imm_challenge", "imm_field_bin
            "imm_ldd_tv_kl", "imm_ldd_topk_workspace", "imm_ldd_topk_distance", "imm_ldd_tail_fraction",
            "imm_sumcheck_batched_transcript_len", "imm_sumcheck_matmul_batched_workspace",
            "imm_sumcheck_matmul_prove_batched", "imm_sumcheck_verify_batched",
-           "imm_commit_workspace", "imm_commit",
+           "imm_commit_workspace", "imm_commit", "imm_commit_launches",
            "imm_sumcheck_matmul_fs_workspace", "imm_sumcheck_matmul_prove_fs", "imm_fs_challenges",
            "imm_sumcheck_verify_fs")
 COMMIT_LEAF = 4096
@@ -126,6 +126,8 @@ def lib() -> ctypes.CDLL:
     L.imm_fs_challenges.argtypes = [vp, ci, vp, i64, i64, i64, u64, vp, vp, vp]
     L.imm_sumcheck_verify_fs.restype = ci
     L.imm_sumcheck_verify_fs.argtypes = [vp, ci, vp, i64, i64, i64, u64, vp, vp, vp, vp]
+    L.imm_commit_launches.restype = ci
+    L.imm_commit_launches.argtypes = [vp, ci]
     L.imm_commit_workspace.restype = sz
     L.imm_commit_workspace.argtypes = [vp, ci]
     L.imm_commit.restype = ci
@@ -469,13 +471,7 @@ class Committer:
                 self.descs[i].r = (ctypes.c_uint8 * 32)(*bytes(r))
                 self.descs[i].r_len = 32
         self.n = n
-        # launches per call: the leaf pass, one node pass per factor of 1024 left in the largest count, the final hash
-        most = max([max(1, -(-int(d.nbytes) // COMMIT_LEAF)) for d in self.descs[:n]] + [1])
-        most = -(-most // 128)
-        self.launches = 2
-        while most > 1:
-            most = -(-most // 1024)
-            self.launches += 1
+        self.launches = lib().imm_commit_launches(ctypes.addressof(self.descs), n)
         need = lib().imm_commit_workspace(ctypes.addressof(self.descs), n)
         if need == 0:
             raise ImmError(ERR_ARG, "imm_commit_workspace")

@@ -182,6 +182,7 @@ def test_fs_and_commit_workspace_and_validation(imm):
     c[1].msg, c[1].nbytes, c[1].r_len = None, 0, 32
     w = L.imm_commit_workspace(ctypes.addressof(c), 2)
     assert w > 0 and w % 256 == 0 and w >= (10 + 1 + 1 + 1) * 32             # subtree roots of both, then the big one's root
+    assert L.imm_commit_launches(ctypes.addressof(c), 2) == 3                # leaves, one node pass, final hashes
     assert L.imm_commit(ctypes.addressof(c), 2, 0x1000, None, 0x1000, w - 1, None) == imm.ERR_WORKSPACE
     assert L.imm_commit(ctypes.addressof(c), 2, None, None, 0x1000, w, None) == imm.ERR_ARG
     assert L.imm_commit(ctypes.addressof(c), 2, 0x1000, None, 0x1010, w, None) == imm.ERR_ALIGN

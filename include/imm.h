@@ -328,6 +328,36 @@ int imm_commit(const imm_commit_desc* descs_host, int n, uint8_t* d_digests, uin
                void* d_ws, size_t ws_bytes, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * The verifier's pass
+ * ---------------------------------------------------------------------------------------------
+ * Vrfy of Section 2.2 accepts a transcript only if its c0, a_fin, b_fin are the verifier's OWN
+ * evaluations C~(r_row, r_col), A~(r_row, r_k), B~(r_k, r_col) of the opened matrices (the expect_*
+ * arguments of the host verifiers).  That is one pass over every matrix, like proving: the three
+ * contractions are the prover's, and where the prover runs the rounds the verifier takes the
+ * inner products of A~(r_row, .) and B~(., r_col) with E_k = eq(r_k, .). */
+
+/* Workspace bytes imm_sumcheck_expected needs (0 on invalid input).  batched != 0: for the members
+ * of a batched proof (every k padded to the largest 2^b). */
+size_t imm_sumcheck_expected_workspace(const imm_matmul_desc* descs_host, int nproofs, int batched);
+
+/* The verifier's own (c0, a_fin, b_fin) of every proof of a batch.
+ *   descs_host  : HOST descriptors with DEVICE matrix pointers (the opened A, B and claimed C)
+ *   seed        : the verifier's coins (interactive and batched proofs; ignored with points_host)
+ *   batch_id    : HOST, NULL for proofs proved one by one (r_k under each proof_id, ceil(log2 k)
+ *                 rounds); else the id of the batched proof (shared r_k, the batch's round count)
+ *   points_host : HOST, NULL to draw r_row, r_col, r_k from the generator; else nproofs x 96 given
+ *                 canonical values, per proof r_row at [0, 32), r_col at [32, 64), r_k at [64, 96)
+ *                 (a non-interactive proof: imm_fs_challenges)
+ *   d_expected  : DEVICE array of nproofs x 3 words: c0, a_fin, b_fin per proof
+ *   d_status    : DEVICE array of nproofs int32, set to IMM_OK per proof
+ *   d_ws        : DEVICE workspace, 256-byte aligned, >= imm_sumcheck_expected_workspace(...)
+ * Launch sequence and errors as imm_sumcheck_matmul_prove (IMM_ERR_NONCANONICAL for a given point
+ * not below p). */
+int imm_sumcheck_expected(const imm_matmul_desc* descs_host, int nproofs, uint64_t seed, const uint64_t* batch_id,
+                          const imm_fe* points_host, imm_fe* d_expected, int32_t* d_status,
+                          void* d_ws, size_t ws_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
  * Non-interactive proof (Fiat-Shamir)
  * ---------------------------------------------------------------------------------------------
  * Algorithm 1 has the server attach a proof pi to its response: no verifier is on line to draw

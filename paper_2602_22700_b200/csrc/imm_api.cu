@@ -648,14 +648,42 @@ static FsLayout fs_layout(const imm_matmul_desc* descs, int nproofs)
     return L;
 }
 
+// vf: non-null = the verifier's pass: the rounds are replaced by the inner products with E_k and
+// d_transcripts receives three words per proof (stride 3): its own c0, a_fin, b_fin.
+struct VerifyArgs {
+    char* ext;                 // device region laid out by verify_layout
+    const imm_fe* points_host; // null: challenges from the generator; else nproofs x VERIFY_POINT_SLOTS given values
+};
+
+struct VerifyLayout {
+    size_t off_ex = 0, off_tasks = 0, off_points = 0, bytes = 0;
+    std::vector<size_t> off_ek;
+};
+
+static VerifyLayout verify_layout(const imm_matmul_desc* descs, int nproofs, int shared_b /* 0: per proof */)
+{
+    VerifyLayout L;
+    size_t off = align_up((size_t)nproofs * sizeof(ExpectDev));
+    L.off_tasks = off;  off = align_up(off + (size_t)nproofs * sizeof(EqTask));
+    L.off_points = off; off = align_up(off + (size_t)nproofs * VERIFY_POINT_SLOTS * sizeof(imm_fe));
+    L.off_ek.resize(nproofs);
+    for (int i = 0; i < nproofs; i++) {
+        L.off_ek[i] = off;
+        off = align_up(off + (sizeof(imm_fe) << (shared_b ? shared_b : ceil_log2(descs[i].k))));
+    }
+    L.bytes = off;
+    return L;
+}
+
 static int prove_batch(const imm_matmul_desc* descs_host, int nproofs, uint64_t seed,
-                       const uint64_t* shared_round_id, const FsArgs* fs, imm_fe* d_transcripts, int64_t stride,
+                       const uint64_t* shared_round_id, const FsArgs* fs, const VerifyArgs* vf,
+                       imm_fe* d_transcripts, int64_t stride,
                        int32_t* d_status, void* d_ws, size_t ws_bytes, void* stream)
 {
     if (!d_transcripts || !d_status || !d_ws) return IMM_ERR_ARG;
     Plan p = make_plan(descs_host, nproofs);
     if (p.status != IMM_OK) return p.status;
-    int rc = check_stride(descs_host, nproofs, stride);
+    int rc = vf ? IMM_OK : check_stride(descs_host, nproofs, stride);
     if (rc != IMM_OK) return rc;
     if ((uintptr_t)d_ws % 16 != 0 || (uintptr_t)d_transcripts % 8 != 0 || (uintptr_t)d_status % 4 != 0)
         return IMM_ERR_ALIGN;
@@ -676,6 +704,14 @@ static int prove_batch(const imm_matmul_desc* descs_host, int nproofs, uint64_t 
     if (fs) {
         fsl = fs_layout(descs_host, nproofs);
         fsp.assign(nproofs, FsProof{});
+    }
+    VerifyLayout vl;
+    std::vector<ExpectDev> exd;
+    std::vector<EqTask> ekt;
+    if (vf) {
+        vl = verify_layout(descs_host, nproofs, shared_round_id ? p.max_b : 0);
+        exd.assign(nproofs, ExpectDev{});
+        ekt.assign(nproofs, EqTask{});
     }
     uint32_t ta = 0, tb = 0, tc = 0;
     for (int i = 0; i < nproofs; i++) {
@@ -719,6 +755,18 @@ static int prove_batch(const imm_matmul_desc* descs_host, int nproofs, uint64_t 
                                p.mma ? (uint32_t*)(base + q.w_cols_b) : nullptr,
                                p.mma ? (uint32_t*)(base + q.w_cols_c) : nullptr, (int32_t)d.n, 0,
                                p.mma ? (imm_fe*)(base + q.sum_col) : nullptr};
+        if (vf) {
+            const imm_fe* given = vf->points_host
+                ? (const imm_fe*)(vf->ext + vl.off_points) + (size_t)i * VERIFY_POINT_SLOTS : nullptr;
+            if (given) {
+                eq[2 * i].point = given;
+                eq[2 * i + 1].point = given + FS_POINT_SLOTS;
+            }
+            imm_fe* e_k = (imm_fe*)(vf->ext + vl.off_ek[i]);
+            ekt[i] = EqTask{e_k, seed, P.round_id, 3u, P.b, nullptr, nullptr, nullptr, (int32_t)d.k, 0, nullptr};
+            if (given) ekt[i].point = given + 2 * FS_POINT_SLOTS;
+            exd[i].e_k = e_k;
+        }
         if (fs) {
             eq[2 * i].point = pts;
             eq[2 * i + 1].point = pts + FS_POINT_SLOTS;
@@ -756,8 +804,16 @@ static int prove_batch(const imm_matmul_desc* descs_host, int nproofs, uint64_t 
         CU(cudaMemcpyAsync(fs->ext + fsl.off_fs, fsp.data(), fsp.size() * sizeof(FsProof), cudaMemcpyHostToDevice, st));
         CU(launch_fs_points((const ProofDev*)(base + p.off_proofs), (const FsProof*)(fs->ext + fsl.off_fs), nproofs, st));
     }
+    if (vf) {
+        CU(cudaMemcpyAsync(vf->ext + vl.off_ex, exd.data(), exd.size() * sizeof(ExpectDev), cudaMemcpyHostToDevice, st));
+        CU(cudaMemcpyAsync(vf->ext + vl.off_tasks, ekt.data(), ekt.size() * sizeof(EqTask), cudaMemcpyHostToDevice, st));
+        if (vf->points_host)
+            CU(cudaMemcpyAsync(vf->ext + vl.off_points, vf->points_host,
+                               (size_t)nproofs * VERIFY_POINT_SLOTS * sizeof(imm_fe), cudaMemcpyHostToDevice, st));
+    }
     PROF_MARK(0, st);
     CU(launch_eq_batch((const EqTask*)(base + p.off_eq), 2 * nproofs, p.max_cover, st));
+    if (vf) CU(launch_eq_batch((const EqTask*)(vf->ext + vl.off_tasks), nproofs, (int64_t)1 << p.max_b, st));
     PROF_MARK(1, st);
     if (ss) {                                                 // fork: the side streams wait for the eq tables
         CU(cudaEventRecord(ss->fork, st));
@@ -783,7 +839,10 @@ static int prove_batch(const imm_matmul_desc* descs_host, int nproofs, uint64_t 
         CU(cudaStreamWaitEvent(st, ss->join[1], 0));
     }
     PROF_MARK(8, st);
-    if (fs)
+    if (vf)
+        CU(launch_expected((const ProofDev*)(base + p.off_proofs), (const ExpectDev*)(vf->ext + vl.off_ex), nproofs,
+                           d_transcripts, d_status, st));
+    else if (fs)
         CU(launch_sumcheck_fs((const ProofDev*)(base + p.off_proofs), (const FsProof*)(fs->ext + fsl.off_fs), nproofs,
                               d_transcripts, stride, d_status, st));
     else
@@ -799,8 +858,8 @@ int imm_sumcheck_matmul_prove(const imm_matmul_desc* descs_host, int nproofs, ui
                               imm_fe* d_transcripts, int64_t stride, int32_t* d_status,
                               void* d_ws, size_t ws_bytes, void* stream)
 {
-    return prove_batch(descs_host, nproofs, seed, nullptr, nullptr, d_transcripts, stride, d_status, d_ws, ws_bytes,
-                       stream);
+    return prove_batch(descs_host, nproofs, seed, nullptr, nullptr, nullptr, d_transcripts, stride, d_status, d_ws,
+                       ws_bytes, stream);
 }
 
 // Batched proof: the per-proof transcripts (shared round challenges) go to the head of the
@@ -842,11 +901,45 @@ int imm_sumcheck_matmul_prove_batched(const imm_matmul_desc* descs_host, int npr
     if (ws_bytes < total) return IMM_ERR_WORKSPACE;
     imm_fe* d_rows = (imm_fe*)d_ws;
     const int64_t stride = 3 * b + 3;
-    rc = prove_batch(descs_host, nproofs, seed, &batch_id, nullptr, d_rows, stride, d_status, (char*)d_ws + rows,
-                     ws_bytes - rows, stream);
+    rc = prove_batch(descs_host, nproofs, seed, &batch_id, nullptr, nullptr, d_rows, stride, d_status,
+                     (char*)d_ws + rows, ws_bytes - rows, stream);
     if (rc != IMM_OK) return rc;
     CU(launch_combine(d_rows, stride, nproofs, b, seed, batch_id, d_transcript, (cudaStream_t)stream));
     return IMM_OK;
+}
+
+}  // extern "C"
+
+// ------------------------------------------------------------------ the verifier's pass -----
+
+extern "C" {
+
+size_t imm_sumcheck_expected_workspace(const imm_matmul_desc* descs_host, int nproofs, int batched)
+{
+    Plan p = make_plan(descs_host, nproofs);
+    if (p.status != IMM_OK) return 0;
+    return verify_layout(descs_host, nproofs, batched ? p.max_b : 0).bytes + p.total_bytes;
+}
+
+int imm_sumcheck_expected(const imm_matmul_desc* descs_host, int nproofs, uint64_t seed, const uint64_t* batch_id,
+                          const imm_fe* points_host, imm_fe* d_expected, int32_t* d_status,
+                          void* d_ws, size_t ws_bytes, void* stream)
+{
+    if (!d_expected || !d_status || !d_ws) return IMM_ERR_ARG;
+    Plan p = make_plan(descs_host, nproofs);
+    if (p.status != IMM_OK) return p.status;
+    if ((uintptr_t)d_ws % ALIGN != 0 || (uintptr_t)d_expected % 8 != 0) return IMM_ERR_ALIGN;
+    if (points_host)
+        for (int64_t i = 0; i < (int64_t)nproofs * VERIFY_POINT_SLOTS; i++)
+            if (points_host[i] >= IMM_P) return IMM_ERR_NONCANONICAL;
+    const size_t ext = verify_layout(descs_host, nproofs, batch_id ? p.max_b : 0).bytes;
+    if (ws_bytes < ext + p.total_bytes) return IMM_ERR_WORKSPACE;
+    // a pageable copy: its upload is staged before the call returns, whatever memory the caller's array is in
+    std::vector<imm_fe> points;
+    if (points_host) points.assign(points_host, points_host + (size_t)nproofs * VERIFY_POINT_SLOTS);
+    VerifyArgs vf{(char*)d_ws, points_host ? points.data() : nullptr};
+    return prove_batch(descs_host, nproofs, seed, batch_id, nullptr, &vf, d_expected, 3, d_status,
+                       (char*)d_ws + ext, ws_bytes - ext, stream);
 }
 
 }  // extern "C"
@@ -873,8 +966,8 @@ int imm_sumcheck_matmul_prove_fs(const imm_matmul_desc* descs_host, int nproofs,
     const size_t ext = fs_layout(descs_host, nproofs).bytes;
     if (ws_bytes < ext + p.total_bytes) return IMM_ERR_WORKSPACE;
     FsArgs fs{d_commitments, (char*)d_ws};
-    return prove_batch(descs_host, nproofs, 0, nullptr, &fs, d_transcripts, stride, d_status, (char*)d_ws + ext,
-                       ws_bytes - ext, stream);
+    return prove_batch(descs_host, nproofs, 0, nullptr, &fs, nullptr, d_transcripts, stride, d_status,
+                       (char*)d_ws + ext, ws_bytes - ext, stream);
 }
 
 }  // extern "C"

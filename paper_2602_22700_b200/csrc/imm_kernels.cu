@@ -919,8 +919,54 @@ sumcheck_fs_kernel(const ProofDev* proofs, const FsProof* fs, imm_fe* transcript
 }
 
 // ------------------------------------------------------------------------------------------
+// the verifier's own evaluations: c0 = C~(r_row, r_col), a_fin = A~(r_row, r_k), b_fin = B~(r_k, r_col)
+// ------------------------------------------------------------------------------------------
+// The three contractions are the prover's (partial sums of C, partial vectors of A and B); where the
+// prover runs the rounds, the verifier only needs the two inner products with E_k.  One block per proof.
+__global__ void __launch_bounds__(SUMCHECK_THREADS)
+expected_kernel(const ProofDev* proofs, const ExpectDev* ex, imm_fe* expected, int32_t* status)
+{
+    __shared__ uint64_t red[33];
+    const ProofDev pr = proofs[blockIdx.x];
+    const imm_fe* e_k = ex[blockIdx.x].e_k;
+    const int tid = threadIdx.x;
+    uint64_t s = 0;
+    for (int i = tid; i < pr.n_part_c; i += SUMCHECK_THREADS) s = gl::add(s, pr.part_c[i]);
+    s = block_sum_fe(s, red);
+    if (pr.c_offset) {                                     // the byte-wise claim kernel read every entry 2^31 too high
+        uint64_t sr = 0, sc = 0;
+        for (int i = tid; i < pr.n_sum_row; i += SUMCHECK_THREADS) sr = gl::add(sr, pr.sum_row[i]);
+        for (int i = tid; i < pr.n_sum_col; i += SUMCHECK_THREADS) sc = gl::add(sc, pr.sum_col[i]);
+        sr = block_sum_fe(sr, red);
+        sc = block_sum_fe(sc, red);
+        s = gl::sub(s, gl::shl(gl::mul(sr, sc), 31));
+    }
+    uint64_t a = 0, b = 0;
+    for (int y = tid; y < pr.k; y += SUMCHECK_THREADS) {   // entries past k meet the zero padding
+        const uint64_t w = e_k[y];
+        a = gl::add(a, gl::mul(w, sum_parts_at(pr.part_a, pr.n_part_a, pr.k, y)));
+        b = gl::add(b, gl::mul(w, sum_parts_at(pr.part_b, pr.n_part_b, pr.k, y)));
+    }
+    a = block_sum_fe(a, red);
+    b = block_sum_fe(b, red);
+    if (tid == 0) {
+        expected[3 * (int64_t)blockIdx.x] = s;
+        expected[3 * (int64_t)blockIdx.x + 1] = a;
+        expected[3 * (int64_t)blockIdx.x + 2] = b;
+        status[blockIdx.x] = 0;
+    }
+}
+
+// ------------------------------------------------------------------------------------------
 // launch wrappers
 // ------------------------------------------------------------------------------------------
+
+cudaError_t launch_expected(const ProofDev* d_proofs, const ExpectDev* d_ex, int nproofs, imm_fe* expected,
+                            int32_t* status, cudaStream_t st)
+{
+    expected_kernel<<<nproofs, SUMCHECK_THREADS, 0, st>>>(d_proofs, d_ex, expected, status);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_fs_points(const ProofDev* d_proofs, const FsProof* d_fs, int nproofs, cudaStream_t st)
 {

@@ -36,5 +36,8 @@ cudaError_t launch_combine(const imm_fe* tr, int64_t stride, int nproofs, int b,
 cudaError_t launch_fs_points(const ProofDev* d_proofs, const FsProof* d_fs, int nproofs, cudaStream_t st);
 cudaError_t launch_sumcheck_fs(const ProofDev* d_proofs, const FsProof* d_fs, int nproofs, imm_fe* transcripts,
                                int64_t stride, int32_t* status, cudaStream_t st);
+// the verifier's own (c0, a_fin, b_fin) per proof from the contractions' partial results and E_k
+cudaError_t launch_expected(const ProofDev* d_proofs, const ExpectDev* d_ex, int nproofs, imm_fe* expected,
+                            int32_t* status, cudaStream_t st);
 
 }  // namespace imm

@@ -109,6 +109,12 @@ struct FsProof {
     uint32_t pad_;
 };
 
+// Per proof of a verifier's pass: the eq table of the round challenges, E_k[y] = eq(r_k, y).
+constexpr int VERIFY_POINT_SLOTS = 3 * FS_POINT_SLOTS;      // caller-given points per proof: r_row, r_col, r_k
+struct ExpectDev {
+    const imm_fe* e_k;         // 2^b entries, b the proof's round count (the batch's for a batched proof)
+};
+
 // A single eq table with r supplied by the caller (passed by value to the kernel).
 struct EqDirect {
     imm_fe r[MAX_EQ_VARS];

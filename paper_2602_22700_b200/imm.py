@@ -35,7 +35,7 @@ EXPORTS = ("imm_version", "imm_last_cuda_error", "imm_challenge", "imm_field_bin
            "imm_sumcheck_matmul_prove_batched", "imm_sumcheck_verify_batched",
            "imm_commit_workspace", "imm_commit", "imm_commit_launches",
            "imm_sumcheck_matmul_fs_workspace", "imm_sumcheck_matmul_prove_fs", "imm_fs_challenges",
-           "imm_sumcheck_verify_fs")
+           "imm_sumcheck_verify_fs", "imm_sumcheck_expected_workspace", "imm_sumcheck_expected")
 COMMIT_LEAF = 4096
 NOALLOC_MAX_TILES = 8192
 PROFILE_PHASES = ("eq_tables", "claim_C", "bind_rows_A", "bind_cols_B", "sumcheck_rounds")
@@ -126,6 +126,10 @@ def lib() -> ctypes.CDLL:
     L.imm_fs_challenges.argtypes = [vp, ci, vp, i64, i64, i64, u64, vp, vp, vp]
     L.imm_sumcheck_verify_fs.restype = ci
     L.imm_sumcheck_verify_fs.argtypes = [vp, ci, vp, i64, i64, i64, u64, vp, vp, vp, vp]
+    L.imm_sumcheck_expected_workspace.restype = sz
+    L.imm_sumcheck_expected_workspace.argtypes = [vp, ci, ci]
+    L.imm_sumcheck_expected.restype = ci
+    L.imm_sumcheck_expected.argtypes = [vp, ci, u64, vp, vp, vp, vp, vp, sz, vp]
     L.imm_commit_launches.restype = ci
     L.imm_commit_launches.argtypes = [vp, ci]
     L.imm_commit_workspace.restype = sz
@@ -590,6 +594,60 @@ def sumcheck_verify_fs(transcript: Sequence[int], nrounds: int, commitments, m: 
                                       opt(expect_c0), opt(expect_a_fin), opt(expect_b_fin), ctypes.addressof(fail))
     _check(rc, "imm_sumcheck_verify_fs")
     return rc, fail.value
+
+
+# ------------------------------------------------------------------ the verifier's pass
+
+
+class Verifier:
+    """The verifier's own (c0, a_fin, b_fin) of every proof: one pass over the opened matrices.
+    ``batched``: the problems are the members of one batched proof."""
+
+    def __init__(self, problems, batched: bool = False, device="cuda"):
+        self.problems = list(problems)
+        self.descs = make_descs(self.problems)
+        self.nproofs = len(self.problems)
+        self.batched = bool(batched)
+        need = lib().imm_sumcheck_expected_workspace(ctypes.addressof(self.descs), self.nproofs, int(self.batched))
+        if need == 0:
+            raise ImmError(ERR_SHAPE, "imm_sumcheck_expected_workspace")
+        self.ws = torch.empty(need, dtype=torch.uint8, device=device)
+        self.values = torch.zeros((self.nproofs, 3), dtype=torch.int64, device=device)
+        self.status = torch.full((self.nproofs,), -99, dtype=torch.int32, device=device)
+
+    def expected(self, seed: int = 0, batch_id: Optional[int] = None, points=None) -> torch.Tensor:
+        """Enqueue the pass on the current stream; returns the (nproofs, 3) device tensor.  ``points``:
+        per proof (r_row, r_col, r_k) for hashed challenges, else they come from the generator."""
+        if self.batched != (batch_id is not None):
+            raise ValueError("batch_id goes with batched=True")
+        bid = ctypes.c_uint64(int(batch_id)) if batch_id is not None else None
+        arr = None
+        if points is not None:
+            if len(points) != self.nproofs:
+                raise ValueError("one (r_row, r_col, r_k) per proof")
+            arr = (ctypes.c_uint64 * (96 * self.nproofs))()
+            for i, triple in enumerate(points):
+                for j, vals in enumerate(triple):
+                    if len(vals) > 32:
+                        raise ValueError("at most 32 challenges per point")
+                    for t, v in enumerate(vals):
+                        arr[96 * i + 32 * j + t] = int(v)
+        _check(lib().imm_sumcheck_expected(ctypes.addressof(self.descs), self.nproofs, seed,
+                                           None if bid is None else ctypes.addressof(bid),
+                                           None if arr is None else ctypes.addressof(arr),
+                                           self.values.data_ptr(), self.status.data_ptr(), self.ws.data_ptr(),
+                                           self.ws.numel(), _stream()), "imm_sumcheck_expected")
+        return self.values
+
+
+def sumcheck_expected(problems, seed: int = 0, batch_id: Optional[int] = None, points=None) -> List[Tuple[int, int, int]]:
+    """Convenience: the verifier's (c0, a_fin, b_fin) per proof as Python ints (synchronises)."""
+    v = Verifier(problems, batched=batch_id is not None)
+    t = v.expected(seed, batch_id, points)
+    torch.cuda.synchronize()
+    if int(v.status.abs().max()) != 0:
+        raise ImmError(int(v.status.min()), "device status")
+    return [tuple(int(x) & 0xFFFFFFFFFFFFFFFF for x in row) for row in t.cpu()]
 
 
 # ------------------------------------------------------------------ logit distance distribution

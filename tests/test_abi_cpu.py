@@ -194,6 +194,26 @@ def test_fs_and_commit_workspace_and_validation(imm):
     assert L.imm_commit(ctypes.addressof(c), 2, 0x1000, None, 0x1000, 1 << 30, None) == imm.ERR_LIMIT
 
 
+def test_verifier_pass_workspace_and_validation(imm):
+    L = imm.lib()
+    d = _desc_array(imm, [(64, 4096, 64), (512, 3000, 4096), (8, 100, 8)])
+    plain = L.imm_sumcheck_matmul_workspace(ctypes.addressof(d), 3)
+    each = L.imm_sumcheck_expected_workspace(ctypes.addressof(d), 3, 0)
+    shared = L.imm_sumcheck_expected_workspace(ctypes.addressof(d), 3, 1)
+    assert each >= plain + 8 * (4096 + 4096 + 128) and each % 256 == 0      # one E_k table per proof
+    assert shared >= plain + 8 * 3 * 4096 and shared > each                     # every table at the largest size
+    assert L.imm_sumcheck_expected_workspace(None, 3, 0) == 0
+    call = L.imm_sumcheck_expected
+    assert call(ctypes.addressof(d), 3, 1, None, None, None, 0x1000, 0x1000, each, None) == imm.ERR_ARG
+    assert call(ctypes.addressof(d), 3, 1, None, None, 0x1000, 0x1000, 0x1000, each - 1, None) == imm.ERR_WORKSPACE
+    assert call(ctypes.addressof(d), 3, 1, None, None, 0x1000, 0x1000, 0x1010, each, None) == imm.ERR_ALIGN
+    pts = (ctypes.c_uint64 * (96 * 3))()
+    pts[100] = imm.P
+    assert call(ctypes.addressof(d), 3, 1, None, ctypes.addressof(pts), 0x1000, 0x1000, 0x1000, each, None) == imm.ERR_NONCANONICAL
+    bid = ctypes.c_uint64(5)
+    assert call(ctypes.addressof(d), 3, 1, ctypes.addressof(bid), None, 0x1000, 0x1000, 0x1000, each, None) == imm.ERR_WORKSPACE
+
+
 def test_argument_validation_happens_before_any_device_work(imm):
     L = imm.lib()
     r = (ctypes.c_uint64 * 4)(1, 2, 3, imm.P)

@@ -2,7 +2,7 @@
 """Throughput of the sumcheck matmul prover on synthetic transformer-shaped layers.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--config decoder|qkv|ffn|moe|attn|ldd|commit] [--batched | --fs]
+                    [--config decoder|qkv|ffn|moe|attn|ldd|commit] [--batched | --fs | --verify]
                     [--layers L] [--tokens T] [--no-e2e] [--no-cpu-baseline]
 
 One step = one proving pass over the whole batch: eq tables, A~ / B~ partial evaluations, the
@@ -12,7 +12,8 @@ tokens, 128 proofs, 39.25 GiB of int8/int32 inputs resident in HBM (far larger t
 flush is needed between steps).  Rank 0 prints ONE JSON line.
 
 --batched proves all products of the workload as one random-linear-combination proof;
---fs makes a step commit to every matrix (SHA-256 trees) and prove non-interactively; --config ldd
+--fs makes a step commit to every matrix (SHA-256 trees) and prove non-interactively; --verify times
+the verifier's pass over the same matrices; --config ldd
 and --config commit time the logit distances and the response commitments (their own metrics).
 
 --impl reference times the plain CPU oracle on the host cores, on a bounded sample of the same
@@ -35,6 +36,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+import numpy as np  # noqa: E402
 import torch  # noqa: E402
 
 METRIC = "proved field-MACs/sec"
@@ -61,6 +63,9 @@ def parse_args():
     ap.add_argument("--fs", action="store_true",
                     help="non-interactive proofs: a step commits to every matrix (SHA-256 trees) and proves with "
                          "challenges hashed from the commitments and the transcript (device-resident timing only)")
+    ap.add_argument("--verify", action="store_true",
+                    help="time the verifier's pass instead: its own (c0, a_fin, b_fin) of every proof "
+                         "(device-resident timing only)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--e2e-steps", type=int, default=2)
@@ -250,6 +255,12 @@ def run_ours(args):
         def prove_step():
             for gi, bp in enumerate(provers):
                 bp.prove(SEED, BATCH_ID0 + gi)
+    elif args.verify:
+        ver = imm.Verifier([(p.A, p.B, p.C, p.proof_id) for p in problems], device=dev)
+        provers = [ver]
+
+        def prove_step():
+            ver.expected(SEED)
     elif args.fs:
         triples = [(p.A, p.B, p.C, p.proof_id) for p in problems]
         com = imm.Committer([t for (A, B, C, _) in triples for t in (A, B, C)], device=dev)
@@ -317,7 +328,20 @@ def run_ours(args):
 
     # every proof of the timed batch must be accepted by the verifier
     accepted = 0
-    if args.fs:
+    if args.verify:
+        # the timed pass's values must accept an honest prover's transcripts
+        host_t = None
+        vals = ver.values.cpu().numpy().view(np.uint64)
+        assert int(ver.status.abs().max()) == 0
+        pr2 = imm.Prover([(p.A, p.B, p.C, p.proof_id) for p in problems], device=dev)
+        tr2 = pr2.prove(SEED).cpu().numpy().view(np.uint64)
+        for i, p in enumerate(problems):
+            b = imm.ceil_log2(p.A.shape[1])
+            words = [int(v) for v in tr2[i, :3 * b + 3]]
+            if imm.sumcheck_verify(words, b, SEED, p.proof_id, *[int(v) for v in vals[i]]) == (imm.OK, -1):
+                accepted += 1
+        del pr2
+    elif args.fs:
         host_t = fsp.transcripts.cpu()
         assert int(fsp.status.abs().max()) == 0
         host_c = com.digests.view(len(problems), 96).cpu().numpy()
@@ -356,6 +380,7 @@ def run_ours(args):
         "dtype": "u64", "data": "synthetic",
         "config": {"workload": workload_name(args.config, args.layers, args.tokens) +
                                (", as one batched proof (every k padded to the largest 2^b)" if args.batched else "") +
+                               (", the verifier's pass (its own c0, a_fin, b_fin per proof)" if args.verify else "") +
                                (", non-interactive: SHA-256 tree commitments to every matrix, then proofs with hashed "
                                 "challenges" if args.fs else ""),
                    "layers": args.layers if args.config == "decoder" else min(args.layers, 8) if args.config == "attn" else None,
@@ -377,7 +402,7 @@ def run_ours(args):
                      "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": claim_gbs / peak,
                      "frac_of_8tbs": claim_gbs / 8000.0,
                      "traffic": (CLAIM_KERNEL_TRAFFIC_RATIO * claim_bytes) if CLAIM_KERNEL_TRAFFIC_RATIO else None},
-        "gpu_launches": ((6 + com.launches) if args.fs else 6 if args.batched else 5) * calls_per_step * steps,
+        "gpu_launches": ((6 + com.launches) if args.fs else 6 if (args.batched or args.verify) else 5) * calls_per_step * steps,
         "transcript_words_per_step": (sum(int(bp.length) for bp in provers) if args.batched else
                                       sum(3 * imm.ceil_log2(k) + 3 for (m, k, n) in shapes)),
         "clocks": clocks,
@@ -390,7 +415,7 @@ def run_ours(args):
         out["fs_phases"] = {"commit_ms": sum(e[0].elapsed_time(e[1]) for e in tail) / steps,
                             "prove_ms": sum(e[1].elapsed_time(e[2]) for e in tail) / steps,
                             "committed_bytes": algo_bytes}
-    if args.batched or args.fs:
+    if args.batched or args.fs or args.verify:
         e2e = {"value": None, "unit": UNIT, "skipped": "the host-buffer entry point proves interactively, proof by proof"}
     elif not args.no_e2e:
         need = algo_bytes
@@ -419,7 +444,7 @@ def run_ours(args):
     out["e2e"] = e2e
 
     # ---- the oracle beside it (rank 0, single GPU): first two layers' proofs, one per thread
-    if not args.no_cpu_baseline and world == 1 and not args.batched and not args.fs:
+    if not args.no_cpu_baseline and world == 1 and not (args.batched or args.fs or args.verify):
         nsample = min(len(problems), 8)
         sample = sample_to_host(problems[:nsample])
         threads = min(os.cpu_count() or 1, nsample)

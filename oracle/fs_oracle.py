@@ -25,6 +25,18 @@ The paper fixes none of this; the readings below are this build's.
 The field arithmetic of the steps (eq tables, the two partial evaluations, the claim) is the C
 oracle's, called through its binding; the rounds are written out here in Python integers.
 
+Batched form (one non-interactive proof for P products, ``prove_batched``): the batched proof of
+``imm_oracle.c`` (random linear combination, every k padded to the largest 2^b) with hashed coins:
+  root        the Merkle tree hash of RFC 6962 (``commit_oracle.merkle_tree_hash``) over the list of
+              member statements s_0^(0), ..., s_0^(P-1) (32-byte leaves)
+  T           H(0x14 || root || le64(batch_id) || le32(P)): binds every member before any coin
+  rho_p       fe(H(0x15 || T || le32(p)))
+  claim       c0B = sum_p rho_p c0_p;  s_1 = H(0x12 || T || le64(c0B))
+  round j     as above on the combined values G_j = sum_p rho_p g_j^(p)
+  transcript  [c0B, G_0(0..2), ..., G_{b-1}(0..2), (c0_p, a_fin_p, b_fin_p) for every p].
+The c0_p are not hashed: with binding commitments they are functions of the statements, and the
+verifier compares them (and a_fin_p, b_fin_p) with its own evaluations.
+
 Pins (tests/test_oracle_fs.py): every challenge re-derived with a SHA-256 written from the standard;
 every round polynomial against exhaustive hypercube sums in big integers at those challenges;
 g_j(0)+g_j(1) = running claim and the final product; each challenge depends on everything before it
@@ -141,4 +153,101 @@ def verify(transcript, nrounds: int, coms, m: int, k: int, n: int, proof_id: int
         for i, (want, got) in enumerate(zip(expect, (t[0], a_fin, b_fin))):
             if want is not None and want != got:
                 return orc.REJECT, nrounds + 1 + i
+    return orc.OK, -1
+
+
+# ------------------------------------------------------------------ batched form
+
+
+def batch_seed(statements, batch_id: int) -> bytes:
+    """T from the member statements (list of 32-byte s_0) and the batch id."""
+    from .commit_oracle import merkle_tree_hash
+    root = merkle_tree_hash([bytes(x) for x in statements])
+    return _h(b"\x14" + root + _le64(batch_id) + _le32(len(statements)))
+
+
+def rho(T: bytes, count: int):
+    return [fe(_h(b"\x15" + T + _le32(p))) for p in range(count)]
+
+
+def prove_batched(problems, batch_id: int):
+    """``problems``: list of (A, B, C, coms, proof_id).  Returns the batched transcript (list of ints)."""
+    count = len(problems)
+    b = max(orc.ceil_log2(A.shape[1]) for (A, _, _, _, _) in problems)
+    stmts, tabs, c0s = [], [], []
+    for A, B, C, coms, pid in problems:
+        m, k = A.shape
+        n = B.shape[1]
+        s0 = statement(coms, m, k, n, pid)
+        e_row = orc.eq_table(point(s0, 1, orc.ceil_log2(m)))
+        e_col = orc.eq_table(point(s0, 2, orc.ceil_log2(n)))
+        av = [int(v) for v in orc.mle_partial_eval(A, orc.BIND_ROWS, e_row)] + [0] * ((1 << b) - k)
+        bv = [int(v) for v in orc.mle_partial_eval(B, orc.BIND_COLS, e_col)] + [0] * ((1 << b) - k)
+        stmts.append(s0)
+        tabs.append([av, bv])
+        c0s.append(orc.mle_eval_point(C, e_row, e_col))
+    T = batch_seed(stmts, batch_id)
+    rh = rho(T, count)
+    c0B = sum(r * c for r, c in zip(rh, c0s)) % P
+    out = [c0B]
+    s = absorb_claim(T, c0B)
+    for j in range(b):
+        half = 1 << (b - 1 - j)
+        G = [0, 0, 0]
+        for r, (av, bv) in zip(rh, tabs):
+            g0 = g1 = g2 = 0
+            for y in range(half):
+                a0, a1, b0, b1 = av[y], av[y + half], bv[y], bv[y + half]
+                g0 += a0 * b0
+                g1 += a1 * b1
+                g2 += (2 * a1 - a0) * (2 * b1 - b0)
+            G[0] += r * (g0 % P)
+            G[1] += r * (g1 % P)
+            G[2] += r * (g2 % P)
+        G = [g % P for g in G]
+        out += G
+        s = absorb_round(s, *G)
+        rj = fe(s)
+        for t in tabs:
+            t[0] = [(t[0][y] + rj * (t[0][y + half] - t[0][y])) % P for y in range(half)]
+            t[1] = [(t[1][y] + rj * (t[1][y + half] - t[1][y])) % P for y in range(half)]
+    for c0, (av, bv) in zip(c0s, tabs):
+        out += [c0, av[0], bv[0]]
+    return out
+
+
+def challenges_batched(transcript, nrounds: int, statements, batch_id: int):
+    """(rho, r_k) as the verifier derives them from the member statements and the transcript."""
+    T = batch_seed(statements, batch_id)
+    s = absorb_claim(T, transcript[0])
+    r_k = []
+    for j in range(nrounds):
+        s = absorb_round(s, *transcript[1 + 3 * j:4 + 3 * j])
+        r_k.append(fe(s))
+    return rho(T, len(statements)), r_k
+
+
+def verify_batched(transcript, nrounds: int, statements, batch_id: int, expect=None):
+    """(status, fail_at) with the meaning of ``orc_sumcheck_verify_batched``."""
+    count = len(statements)
+    t = [int(w) for w in transcript]
+    total = 1 + 3 * nrounds + 3 * count
+    if len(t) < total or any(w >= P or w < 0 for w in t[:total]):
+        return -5, -2
+    rh, r_k = challenges_batched(t, nrounds, statements, batch_id)
+    tail = t[1 + 3 * nrounds:total]
+    if t[0] != sum(r * tail[3 * p] for p, r in enumerate(rh)) % P:
+        return orc.REJECT, nrounds + 1
+    claim = t[0]
+    for j in range(nrounds):
+        g0, g1, g2 = t[1 + 3 * j:4 + 3 * j]
+        if (g0 + g1) % P != claim:
+            return orc.REJECT, j
+        claim = orc.interp_deg2(g0, g1, g2, r_k[j])
+    if claim != sum(r * tail[3 * p + 1] * tail[3 * p + 2] for p, r in enumerate(rh)) % P:
+        return orc.REJECT, nrounds
+    if expect is not None:
+        for i, (want, got) in enumerate(zip(expect, tail)):
+            if want != got:
+                return orc.REJECT, nrounds + 2 + i
     return orc.OK, -1

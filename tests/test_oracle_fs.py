@@ -147,3 +147,115 @@ def test_wrong_product_is_rejected(oracle):
     coms = coms_for(rng)
     t = oracle.fs.prove(A, B, C, coms, 0)
     assert oracle.fs.verify(t, 3, coms, 4, 8, 4, 0) == (oracle.REJECT, 0)
+
+
+# ------------------------------------------------------------------ batched form
+
+def levelwise_root_of(leaves, H):
+    level = [H(b"\x00" + d) for d in leaves]
+    while len(level) > 1:
+        nxt = [H(b"\x01" + level[i] + level[i + 1]) for i in range(0, len(level) - 1, 2)]
+        if len(level) % 2:
+            nxt.append(level[-1])
+        level = nxt
+    return level[0]
+
+
+def batch_problems(rng, shapes, first_id=50):
+    out = []
+    for i, (m, k, n) in enumerate(shapes):
+        A, B, C = rand_problem(rng, m, k, n)
+        out.append((A, B, C, coms_for(rng), first_id + 2 * i))
+    return out
+
+
+def padded_lists(A, B, kp):
+    m, k = A.shape
+    Ap = np.zeros((m, kp), dtype=np.int64)
+    Ap[:, :k] = A
+    Bp = np.zeros((kp, B.shape[1]), dtype=np.int64)
+    Bp[:k] = B
+    return Ap.tolist(), Bp.tolist()
+
+
+@pytest.mark.parametrize("shapes", [[(2, 4, 2), (3, 4, 1)], [(1, 8, 3), (2, 3, 2), (3, 1, 1)], [(2, 2, 2)],
+                                    [(1, 2, 1), (2, 2, 1), (1, 1, 2), (2, 2, 2), (1, 2, 2)]])
+def test_batched_transcript_matches_definitions_at_hashed_coins(oracle, shapes):
+    rng = random.Random(7 + sum(sum(x) for x in shapes))
+    probs = batch_problems(rng, shapes)
+    bid = rng.getrandbits(50)
+    t = oracle.fs.prove_batched(probs, bid)
+    count, b = len(probs), max(clog2(k) for (_, k, _) in shapes)
+    assert len(t) == 1 + 3 * b + 3 * count
+    # every coin re-derived without hashlib: statements, tree over them, T, rho, the chain
+    stmts, pts = [], []
+    for A, B, C, coms, pid in probs:
+        m, k = A.shape
+        n = B.shape[1]
+        s0 = sha256_py(b"\x10" + coms[0] + coms[1] + coms[2] + le(m, 8) + le(k, 8) + le(n, 8) + le(pid, 8))
+        stmts.append(s0)
+        pts.append(([to_fe(sha256_py(b"\x11" + s0 + le(1, 4) + le(i, 4))) for i in range(clog2(m))],
+                    [to_fe(sha256_py(b"\x11" + s0 + le(2, 4) + le(i, 4))) for i in range(clog2(n))]))
+    T = sha256_py(b"\x14" + levelwise_root_of(stmts, sha256_py) + le(bid, 8) + le(count, 4))
+    rho = [to_fe(sha256_py(b"\x15" + T + le(p, 4))) for p in range(count)]
+    s = sha256_py(b"\x12" + T + le(t[0], 8))
+    r_k = []
+    for j in range(b):
+        s = sha256_py(b"\x13" + s + le(t[1 + 3 * j], 8) + le(t[3 + 3 * j], 8))
+        r_k.append(to_fe(s))
+    assert (rho, r_k) == tuple(oracle.fs.challenges_batched(t, b, stmts, bid))
+    assert stmts == [oracle.fs.statement(c, A.shape[0], A.shape[1], B.shape[1], pid) for A, B, C, c, pid in probs]
+    # the words against exhaustive sums on explicitly padded matrices
+    tail = [t[1 + 3 * b + 3 * p:4 + 3 * b + 3 * p] for p in range(count)]
+    lists = [padded_lists(A, B, 1 << b) for A, B, _, _, _ in probs]
+    for (A, B, C, _, _), (rr, rc), (Al, Bl), (c0, af, bf) in zip(probs, pts, lists, tail):
+        assert c0 == mle(C.tolist(), rr, rc)
+        assert af == mle(Al, rr, r_k) and bf == mle(Bl, r_k, rc)
+    assert t[0] == sum(r * x[0] for r, x in zip(rho, tail)) % P
+    claim = t[0]
+    for j in range(b):
+        g = [sum(r * round_poly_by_definition(Al, Bl, rr, rc, r_k[:j], X)
+                 for r, (Al, Bl), (rr, rc) in zip(rho, lists, pts)) % P for X in (0, 1, 2)]
+        assert t[1 + 3 * j:4 + 3 * j] == g and (g[0] + g[1]) % P == claim
+        claim = interp_deg2(g[0], g[1], g[2], r_k[j])
+    assert claim == sum(r * x[1] * x[2] for r, x in zip(rho, tail)) % P
+    assert oracle.fs.verify_batched(t, b, stmts, bid) == (oracle.OK, -1)
+    assert oracle.fs.verify_batched(t, b, stmts, bid, expect=[w for x in tail for w in x]) == (oracle.OK, -1)
+
+
+def test_batched_coins_bind_every_member_and_the_verifier_locates_changes(oracle):
+    rng = random.Random(77)
+    shapes = [(2, 8, 2), (3, 5, 1), (1, 8, 4)]
+    probs = batch_problems(rng, shapes)
+    bid, b, count = 9, 3, 3
+    t = oracle.fs.prove_batched(probs, bid)
+    stmts = [oracle.fs.statement(c, A.shape[0], A.shape[1], B.shape[1], pid) for A, B, C, c, pid in probs]
+    rho, r_k = oracle.fs.challenges_batched(t, b, stmts, bid)
+    # any member's statement, the order of members, the batch id and the member count move every coin
+    for alt in ([stmts[0], stmts[2], stmts[1]], [bytes([stmts[0][0] ^ 1]) + stmts[0][1:]] + stmts[1:], stmts[:2]):
+        r2, k2 = oracle.fs.challenges_batched(t, b, alt, bid)
+        assert all(x != y for x, y in zip(rho, r2)) and all(x != y for x, y in zip(r_k, k2))
+    r2, k2 = oracle.fs.challenges_batched(t, b, stmts, bid + 1)
+    assert all(x != y for x, y in zip(rho, r2)) and all(x != y for x, y in zip(r_k, k2))
+    assert oracle.fs.verify_batched(t, b, stmts, bid) == (oracle.OK, -1)
+    for pos in range(len(t)):
+        u = list(t)
+        u[pos] = (u[pos] + 1 + rng.randrange(P - 1)) % P
+        status, where = oracle.fs.verify_batched(u, b, stmts, bid)
+        assert status == oracle.REJECT
+        if pos == 0:
+            assert where == b + 1
+        elif pos <= 3 * b:
+            j, part = (pos - 1) // 3, (pos - 1) % 3
+            assert where == (j if part < 2 else j + 1)
+        else:
+            assert where == (b + 1 if (pos - 1 - 3 * b) % 3 == 0 else b)
+    exp = t[1 + 3 * b:]
+    exp[4] = (exp[4] + 1) % P
+    assert oracle.fs.verify_batched(t, b, stmts, bid, expect=exp) == (oracle.REJECT, b + 2 + 4)
+    # one wrong member sinks the batch at round 0
+    A, B, C, coms, pid = probs[1]
+    C2 = C.copy()
+    C2[0, 0] += 1
+    bad = oracle.fs.prove_batched([probs[0], (A, B, C2, coms, pid), probs[2]], bid)
+    assert oracle.fs.verify_batched(bad, b, stmts, bid) == (oracle.REJECT, 0)

@@ -395,6 +395,41 @@ int imm_fs_challenges(const imm_fe* transcript_host, int nrounds, const uint8_t*
                       int64_t m, int64_t k, int64_t n, uint64_t proof_id,
                       imm_fe* r_row_host, imm_fe* r_col_host, imm_fe* r_k_host);
 
+/* Batched non-interactive proof: ONE proof for all products of a batch, every coin hashed.  The
+ * batched proof above with
+ *   root  = Merkle tree hash (RFC 6962: leaf = H(0x00 || d), node = H(0x01 || l || r)) over the member
+ *           statements s_0^(0), ..., s_0^(P-1) as 32-byte leaves,
+ *   T     = H(0x14 || root || le64(batch_id) || le32(P)),   rho_p = fe(H(0x15 || T || le32(p))),
+ *   s_1   = H(0x12 || T || le64(c0B)),  rounds as for the single proof on the combined values;
+ * r_row, r_col of a member come from its own statement.  The member values c0_p are not hashed: with
+ * binding commitments they are functions of the statements, and the verifier compares them with
+ * its own.  At most IMM_FS_BATCH_MAX members.  Transcript layout: that of the batched proof. */
+#define IMM_FS_BATCH_MAX 1024
+
+size_t imm_sumcheck_matmul_fs_batched_workspace(const imm_matmul_desc* descs_host, int nproofs);
+
+/* Prover.  Arguments as imm_sumcheck_matmul_prove_fs; d_transcript holds
+ * imm_sumcheck_batched_transcript_len(b, nproofs) words, b = ceil(log2 of the largest k).  After the
+ * contractions the rounds are a chain of 3 + 2b small launches (every round needs the sum over all
+ * members before its challenge exists).  IMM_ERR_LIMIT for more than IMM_FS_BATCH_MAX members. */
+int imm_sumcheck_matmul_prove_fs_batched(const imm_matmul_desc* descs_host, int nproofs, const uint8_t* d_commitments,
+                                         uint64_t batch_id, imm_fe* d_transcript, int32_t* d_status,
+                                         void* d_ws, size_t ws_bytes, void* stream);
+
+/* HOST.  The coins of a batched non-interactive proof: rho (nproofs values) and r_k (nrounds values,
+ * from the transcript's first 3*nrounds+1 words).  descs_host gives every member's m, k, n and
+ * proof_id (matrix pointers are not read); commitments_host holds nproofs x 96 bytes.  Either
+ * output may be NULL.  The members' r_row, r_col: imm_fs_challenges with a NULL transcript. */
+int imm_fs_batched_challenges(const imm_fe* transcript_host, int nrounds, const imm_matmul_desc* descs_host,
+                              int nproofs, const uint8_t* commitments_host, uint64_t batch_id,
+                              imm_fe* rho_host, imm_fe* r_k_host);
+
+/* HOST verifier of a batched non-interactive proof: the checks and fail_at of
+ * imm_sumcheck_verify_batched with the hashed coins. */
+int imm_sumcheck_verify_fs_batched(const imm_fe* transcript_host, int nrounds, const imm_matmul_desc* descs_host,
+                                   int nproofs, const uint8_t* commitments_host, uint64_t batch_id,
+                                   const imm_fe* expect_host, int* fail_at);
+
 /* HOST verifier of a non-interactive proof: the checks of imm_sumcheck_verify with the hashed round
  * challenges; fail_at has the same meaning.  commitments_host: the 96 bytes of the statement.
  * Returns IMM_OK, IMM_REJECT, IMM_ERR_ARG, IMM_ERR_SHAPE or IMM_ERR_NONCANONICAL. */

@@ -33,6 +33,7 @@ int cuda_fail(cudaError_t e)
 constexpr int64_t MAX_EXTENT = (int64_t)1 << 20;
 constexpr int64_t MAX_K = (int64_t)1 << MAX_K_VARS;
 constexpr size_t ALIGN = 256;
+static_assert(FS_BATCH_MAX == IMM_FS_BATCH_MAX, "the header's limit is the kernels'");
 
 size_t align_up(size_t x) { return (x + ALIGN - 1) / ALIGN * ALIGN; }
 
@@ -626,14 +627,16 @@ size_t imm_sumcheck_matmul_workspace(const imm_matmul_desc* descs_host, int npro
 struct FsArgs {
     const uint8_t* d_com;      // nproofs x 96 bytes
     char* ext;                 // device region laid out by fs_layout
+    bool batched;              // one proof for all members (shared_round_id carries the batch id)
 };
 
 struct FsLayout {
     size_t off_fs = 0, off_points = 0, off_state = 0, bytes = 0;
     std::vector<size_t> off_tabs;
+    size_t off_T = 0, off_bstate = 0, off_rho = 0, off_c0 = 0, off_partial = 0, off_r = 0;   // batched proof only
 };
 
-static FsLayout fs_layout(const imm_matmul_desc* descs, int nproofs)
+static FsLayout fs_layout(const imm_matmul_desc* descs, int nproofs, int shared_b /* 0: per proof */)
 {
     FsLayout L;
     size_t off = align_up((size_t)nproofs * sizeof(FsProof));
@@ -642,8 +645,14 @@ static FsLayout fs_layout(const imm_matmul_desc* descs, int nproofs)
     L.off_tabs.resize(nproofs);
     for (int i = 0; i < nproofs; i++) {
         L.off_tabs[i] = off;
-        off = align_up(off + 2 * (sizeof(imm_fe) << ceil_log2(descs[i].k)));
+        off = align_up(off + 2 * (sizeof(imm_fe) << (shared_b ? shared_b : ceil_log2(descs[i].k))));
     }
+    L.off_T = off;       off = align_up(off + 8 * sizeof(uint32_t));
+    L.off_bstate = off;  off = align_up(off + 8 * sizeof(uint32_t));
+    L.off_rho = off;     off = align_up(off + (size_t)nproofs * sizeof(imm_fe));
+    L.off_c0 = off;      off = align_up(off + (size_t)nproofs * sizeof(imm_fe));
+    L.off_partial = off; off = align_up(off + (size_t)nproofs * 3 * sizeof(imm_fe));
+    L.off_r = off;       off = align_up(off + MAX_K_VARS * sizeof(imm_fe));
     L.bytes = off;
     return L;
 }
@@ -702,7 +711,7 @@ static int prove_batch(const imm_matmul_desc* descs_host, int nproofs, uint64_t 
     FsLayout fsl;
     std::vector<FsProof> fsp;
     if (fs) {
-        fsl = fs_layout(descs_host, nproofs);
+        fsl = fs_layout(descs_host, nproofs, fs->batched ? p.max_b : 0);
         fsp.assign(nproofs, FsProof{});
     }
     VerifyLayout vl;
@@ -775,7 +784,7 @@ static int prove_batch(const imm_matmul_desc* descs_host, int nproofs, uint64_t 
             F.points = (imm_fe*)pts;
             F.state = (uint32_t*)(fs->ext + fsl.off_state) + (size_t)i * 8;
             F.ta = (imm_fe*)(fs->ext + fsl.off_tabs[i]);
-            F.tb = F.ta + ((size_t)1 << q.b);
+            F.tb = F.ta + ((size_t)1 << P.b);
             F.proof_id = d.proof_id;
             F.one = 1;
         }
@@ -842,7 +851,21 @@ static int prove_batch(const imm_matmul_desc* descs_host, int nproofs, uint64_t 
     if (vf)
         CU(launch_expected((const ProofDev*)(base + p.off_proofs), (const ExpectDev*)(vf->ext + vl.off_ex), nproofs,
                            d_transcripts, d_status, st));
-    else if (fs)
+    else if (fs && fs->batched) {
+        FsBatch fb{};
+        fb.T = (uint32_t*)(fs->ext + fsl.off_T);
+        fb.state = (uint32_t*)(fs->ext + fsl.off_bstate);
+        fb.rho = (imm_fe*)(fs->ext + fsl.off_rho);
+        fb.c0 = (imm_fe*)(fs->ext + fsl.off_c0);
+        fb.partial = (imm_fe*)(fs->ext + fsl.off_partial);
+        fb.r = (imm_fe*)(fs->ext + fsl.off_r);
+        fb.batch_id = *shared_round_id;
+        fb.nproofs = nproofs;
+        fb.b = p.max_b;
+        fb.one = 1;
+        CU(launch_fs_batched_rounds((const ProofDev*)(base + p.off_proofs), (const FsProof*)(fs->ext + fsl.off_fs), fb,
+                                    d_transcripts, d_status, st));
+    } else if (fs)
         CU(launch_sumcheck_fs((const ProofDev*)(base + p.off_proofs), (const FsProof*)(fs->ext + fsl.off_fs), nproofs,
                               d_transcripts, stride, d_status, st));
     else
@@ -952,7 +975,7 @@ size_t imm_sumcheck_matmul_fs_workspace(const imm_matmul_desc* descs_host, int n
 {
     Plan p = make_plan(descs_host, nproofs);
     if (p.status != IMM_OK) return 0;
-    return fs_layout(descs_host, nproofs).bytes + p.total_bytes;
+    return fs_layout(descs_host, nproofs, 0).bytes + p.total_bytes;
 }
 
 int imm_sumcheck_matmul_prove_fs(const imm_matmul_desc* descs_host, int nproofs, const uint8_t* d_commitments,
@@ -963,10 +986,33 @@ int imm_sumcheck_matmul_prove_fs(const imm_matmul_desc* descs_host, int nproofs,
     Plan p = make_plan(descs_host, nproofs);
     if (p.status != IMM_OK) return p.status;
     if ((uintptr_t)d_ws % ALIGN != 0) return IMM_ERR_ALIGN;
-    const size_t ext = fs_layout(descs_host, nproofs).bytes;
+    const size_t ext = fs_layout(descs_host, nproofs, 0).bytes;
     if (ws_bytes < ext + p.total_bytes) return IMM_ERR_WORKSPACE;
-    FsArgs fs{d_commitments, (char*)d_ws};
+    FsArgs fs{d_commitments, (char*)d_ws, false};
     return prove_batch(descs_host, nproofs, 0, nullptr, &fs, nullptr, d_transcripts, stride, d_status,
+                       (char*)d_ws + ext, ws_bytes - ext, stream);
+}
+
+size_t imm_sumcheck_matmul_fs_batched_workspace(const imm_matmul_desc* descs_host, int nproofs)
+{
+    Plan p = make_plan(descs_host, nproofs);
+    if (p.status != IMM_OK || nproofs > FS_BATCH_MAX) return 0;
+    return fs_layout(descs_host, nproofs, p.max_b).bytes + p.total_bytes;
+}
+
+int imm_sumcheck_matmul_prove_fs_batched(const imm_matmul_desc* descs_host, int nproofs, const uint8_t* d_commitments,
+                                         uint64_t batch_id, imm_fe* d_transcript, int32_t* d_status,
+                                         void* d_ws, size_t ws_bytes, void* stream)
+{
+    if (!d_commitments || !d_ws) return IMM_ERR_ARG;
+    Plan p = make_plan(descs_host, nproofs);
+    if (p.status != IMM_OK) return p.status;
+    if (nproofs > FS_BATCH_MAX) return IMM_ERR_LIMIT;
+    if ((uintptr_t)d_ws % ALIGN != 0) return IMM_ERR_ALIGN;
+    const size_t ext = fs_layout(descs_host, nproofs, p.max_b).bytes;
+    if (ws_bytes < ext + p.total_bytes) return IMM_ERR_WORKSPACE;
+    FsArgs fs{d_commitments, (char*)d_ws, true};
+    return prove_batch(descs_host, nproofs, 0, &batch_id, &fs, nullptr, d_transcript, 3 * p.max_b + 3, d_status,
                        (char*)d_ws + ext, ws_bytes - ext, stream);
 }
 
@@ -1019,6 +1065,33 @@ uint64_t fs_point_host(const uint32_t (&s0)[8], uint32_t domain, uint32_t t)
     return fs_fe_host(h);
 }
 
+// Merkle tree hash (RFC 6962) over 32-byte leaves given as state words; neighbours pair level by level,
+// an unpaired last node moves up unchanged.
+void merkle_root_host(std::vector<imm_sha::Digest> level, uint32_t (&root)[8])
+{
+    for (imm_sha::Digest& d : level) {
+        uint8_t m[40];
+        m[0] = 0x00;
+        imm_sha::digest_bytes(d.h, m + 1);
+        imm_sha::sha256_short(m, 33, d.h, 1);
+    }
+    while (level.size() > 1) {
+        std::vector<imm_sha::Digest> next;
+        for (size_t i = 0; i + 1 < level.size(); i += 2) {
+            uint8_t m[72];
+            m[0] = 0x01;
+            imm_sha::digest_bytes(level[i].h, m + 1);
+            imm_sha::digest_bytes(level[i + 1].h, m + 33);
+            imm_sha::Digest d;
+            imm_sha::sha256_short(m, 65, d.h, 1);
+            next.push_back(d);
+        }
+        if (level.size() % 2) next.push_back(level.back());
+        level.swap(next);
+    }
+    for (int i = 0; i < 8; i++) root[i] = level[0].h[i];
+}
+
 int fs_check_shape(int64_t m, int64_t k, int64_t n, int nrounds)
 {
     if (m <= 0 || k <= 0 || n <= 0 || m > MAX_EXTENT || n > MAX_EXTENT || k > MAX_K) return IMM_ERR_SHAPE;
@@ -1054,6 +1127,100 @@ int imm_fs_challenges(const imm_fe* transcript_host, int nrounds, const uint8_t*
             r_k_host[j] = fs_fe_host(s);
         }
     }
+    return IMM_OK;
+}
+
+int imm_fs_batched_challenges(const imm_fe* transcript_host, int nrounds, const imm_matmul_desc* descs_host,
+                              int nproofs, const uint8_t* commitments_host, uint64_t batch_id,
+                              imm_fe* rho_host, imm_fe* r_k_host)
+{
+    if (!descs_host || !commitments_host || nproofs <= 0 || nproofs > FS_BATCH_MAX || nrounds < 0 ||
+        nrounds > MAX_K_VARS)
+        return IMM_ERR_ARG;
+    int b = 0;
+    std::vector<imm_sha::Digest> stmts(nproofs);
+    for (int i = 0; i < nproofs; i++) {
+        const imm_matmul_desc& d = descs_host[i];
+        int rc = fs_check_shape(d.m, d.k, d.n, ceil_log2(d.k));
+        if (rc != IMM_OK) return rc;
+        if (ceil_log2(d.k) > b) b = ceil_log2(d.k);
+        fs_statement_host(commitments_host + (size_t)i * 96, d.m, d.k, d.n, d.proof_id, stmts[i].h);
+    }
+    if (nrounds != b) return IMM_ERR_SHAPE;
+    uint32_t T[8];
+    merkle_root_host(stmts, T);
+    {
+        uint8_t m[48];
+        m[0] = 0x14;
+        imm_sha::digest_bytes(T, m + 1);
+        put_le(m + 33, batch_id, 8);
+        put_le(m + 41, (uint64_t)nproofs, 4);
+        imm_sha::sha256_short(m, 45, T, 1);
+    }
+    if (rho_host)
+        for (int p = 0; p < nproofs; p++) {
+            uint8_t m[40];
+            uint32_t h[8];
+            m[0] = 0x15;
+            imm_sha::digest_bytes(T, m + 1);
+            put_le(m + 33, (uint64_t)p, 4);
+            imm_sha::sha256_short(m, 37, h, 1);
+            rho_host[p] = fs_fe_host(h);
+        }
+    if (r_k_host) {
+        if (!transcript_host) return IMM_ERR_ARG;
+        for (int i = 0; i < 3 * nrounds + 1; i++)
+            if (transcript_host[i] >= IMM_P) return IMM_ERR_NONCANONICAL;
+        fs_absorb_host(T, 0x12, transcript_host, 1);
+        for (int j = 0; j < nrounds; j++) {
+            const uint64_t hashed[2] = {transcript_host[1 + 3 * j], transcript_host[3 + 3 * j]};
+            fs_absorb_host(T, 0x13, hashed, 2);
+            r_k_host[j] = fs_fe_host(T);
+        }
+    }
+    return IMM_OK;
+}
+
+int imm_sumcheck_verify_fs_batched(const imm_fe* transcript_host, int nrounds, const imm_matmul_desc* descs_host,
+                                   int nproofs, const uint8_t* commitments_host, uint64_t batch_id,
+                                   const imm_fe* expect_host, int* fail_at)
+{
+    if (!transcript_host || !fail_at) return IMM_ERR_ARG;
+    std::vector<uint64_t> rho((size_t)(nproofs > 0 ? nproofs : 1));
+    uint64_t r_k[64];
+    int rc = imm_fs_batched_challenges(transcript_host, nrounds, descs_host, nproofs, commitments_host, batch_id,
+                                       rho.data(), r_k);
+    if (rc != IMM_OK) return rc;
+    const imm_fe* t = transcript_host;
+    const int64_t len = 1 + 3 * (int64_t)nrounds + 3 * (int64_t)nproofs;
+    for (int64_t i = 0; i < len; i++)
+        if (t[i] >= IMM_P) return IMM_ERR_NONCANONICAL;
+    if (expect_host)
+        for (int64_t i = 0; i < 3 * (int64_t)nproofs; i++)
+            if (expect_host[i] >= IMM_P) return IMM_ERR_NONCANONICAL;
+    const imm_fe* tail = t + 1 + 3 * nrounds;
+    uint64_t combo = 0, fin = 0;
+    for (int p = 0; p < nproofs; p++) {
+        combo = gl::add(combo, gl::mul(rho[p], tail[3 * (int64_t)p]));
+        fin = gl::add(fin, gl::mul(rho[p], gl::mul(tail[3 * (int64_t)p + 1], tail[3 * (int64_t)p + 2])));
+    }
+    uint64_t claim = t[0];
+    if (claim != combo) { *fail_at = nrounds + 1; return IMM_REJECT; }
+    const uint64_t inv2 = 0x7FFFFFFF80000001ULL;
+    for (int j = 0; j < nrounds; j++) {
+        const uint64_t g0 = t[1 + 3 * j], g1 = t[2 + 3 * j], g2 = t[3 + 3 * j];
+        if (gl::add(g0, g1) != claim) { *fail_at = j; return IMM_REJECT; }
+        const uint64_t r = r_k[j];
+        const uint64_t d1 = gl::sub(g1, g0);
+        const uint64_t d2 = gl::sub(gl::sub(g2, g1), d1);
+        const uint64_t c2 = gl::mul(gl::mul(r, gl::sub(r, 1)), inv2);
+        claim = gl::add(g0, gl::add(gl::mul(r, d1), gl::mul(c2, d2)));
+    }
+    if (fin != claim) { *fail_at = nrounds; return IMM_REJECT; }
+    if (expect_host)
+        for (int64_t i = 0; i < 3 * (int64_t)nproofs; i++)
+            if (expect_host[i] != tail[i]) { *fail_at = nrounds + 2 + (int)i; return IMM_REJECT; }
+    *fail_at = -1;
     return IMM_OK;
 }
 

@@ -58,27 +58,8 @@ constexpr size_t ALIGN = 256;
 using imm_sha::compress;
 using imm_sha::iv;
 
-struct Digest { uint32_t h[8]; };             // the eight state words (big-endian when serialised)
-
-// node = SHA-256(0x01 || left || right): 65 bytes, two compressions
-__device__ __forceinline__ void node_hash(const uint32_t (&l)[8], const uint32_t (&r)[8], uint32_t (&out)[8],
-                                          uint32_t one)
-{
-    uint32_t w[16];
-    w[0] = 0x01000000u | (l[0] >> 8);
-#pragma unroll
-    for (int i = 1; i < 8; i++) w[i] = (l[i - 1] << 24) | (l[i] >> 8);
-    w[8] = (l[7] << 24) | (r[0] >> 8);
-#pragma unroll
-    for (int i = 1; i < 8; i++) w[8 + i] = (r[i - 1] << 24) | (r[i] >> 8);
-    iv(out);
-    compress(out, w, one);
-    w[0] = (r[7] << 24) | 0x00800000u;
-#pragma unroll
-    for (int i = 1; i < 15; i++) w[i] = 0;
-    w[15] = 65 * 8;
-    compress(out, w, one);
-}
+using imm_sha::Digest;
+using imm_sha::fold;
 
 // A full leaf whose data is 16-byte aligned: SHA-256(0x00 || 4096 bytes), 65 compressions.  Message
 // word t of a block is the last byte of little-endian data word t-1 followed by the first three
@@ -133,30 +114,6 @@ __device__ __noinline__ void leaf_hash_bytes(const uint8_t* __restrict__ p, uint
         }
         if (blk == nblocks - 1) w[15] = total * 8;         // (w[14], the high length word, is already 0)
         compress(h, w, one);
-    }
-}
-
-// Folds the `count` digests in sd (count <= blockDim.x) to one in sd[0]: neighbours pair level by
-// level, an unpaired last digest moves up unchanged.
-__device__ __forceinline__ void fold(Digest* sd, int count, uint32_t one)
-{
-    const int t = threadIdx.x;
-    while (count > 1) {
-        const int half = count >> 1;
-        uint32_t out[8];
-        const bool pair = t < half, lift = (count & 1) && t == half;
-        if (pair) node_hash(sd[2 * t].h, sd[2 * t + 1].h, out, one);
-        else if (lift) {
-#pragma unroll
-            for (int i = 0; i < 8; i++) out[i] = sd[count - 1].h[i];
-        }
-        __syncthreads();
-        if (pair || lift) {
-#pragma unroll
-            for (int i = 0; i < 8; i++) sd[t].h[i] = out[i];
-        }
-        __syncthreads();
-        count = (count + 1) >> 1;
     }
 }
 

@@ -919,6 +919,176 @@ sumcheck_fs_kernel(const ProofDev* proofs, const FsProof* fs, imm_fe* transcript
 }
 
 // ------------------------------------------------------------------------------------------
+// batched non-interactive proof: one sumcheck for all members, every coin hashed
+// ------------------------------------------------------------------------------------------
+//   root  = Merkle tree hash (RFC 6962) over the member statements s_0^(p) (32-byte leaves)
+//   T     = H(0x14 || root || le64(batch_id) || le32(P)),   rho_p = fe(H(0x15 || T || le32(p)))
+//   s_1   = H(0x12 || T || le64(c0B)), c0B = sum_p rho_p c0_p;  rounds as above on the combined sums.
+// Every round needs the sum over ALL members before its challenge exists, so the rounds are a chain
+// of small launches (members fold side by side, one block combines and hashes) instead of blocks
+// that wait for one another.
+
+__global__ void __launch_bounds__(FS_BATCH_MAX) fsb_seed_kernel(const FsProof* fs, FsBatch fb)
+{
+    __shared__ imm_sha::Digest sd[FS_BATCH_MAX];
+    __shared__ uint32_t T_sh[8];
+    const int p = threadIdx.x;
+    if (p < fb.nproofs) {                                  // leaf = H(0x00 || s_0^(p))
+        uint8_t m[40];
+        uint32_t h[8];
+        for (int i = 0; i < 8; i++) h[i] = fs[p].state[i];
+        m[0] = 0x00;
+        imm_sha::digest_bytes(h, m + 1);
+        imm_sha::sha256_short(m, 33, h, fb.one);
+        for (int i = 0; i < 8; i++) sd[p].h[i] = h[i];
+    }
+    __syncthreads();
+    imm_sha::fold(sd, fb.nproofs, fb.one);
+    if (p == 0) {
+        uint8_t m[48];
+        uint32_t h[8];
+        for (int i = 0; i < 8; i++) h[i] = sd[0].h[i];
+        m[0] = 0x14;
+        imm_sha::digest_bytes(h, m + 1);
+        fs_put_le(m + 33, fb.batch_id, 8);
+        fs_put_le(m + 41, (uint64_t)fb.nproofs, 4);
+        imm_sha::sha256_short(m, 45, h, fb.one);
+        for (int i = 0; i < 8; i++) { T_sh[i] = h[i]; fb.T[i] = h[i]; }
+    }
+    __syncthreads();
+    if (p < fb.nproofs) {
+        uint8_t m[40];
+        uint32_t h[8];
+        for (int i = 0; i < 8; i++) h[i] = T_sh[i];
+        m[0] = 0x15;
+        imm_sha::digest_bytes(h, m + 1);
+        fs_put_le(m + 33, (uint64_t)p, 4);
+        imm_sha::sha256_short(m, 37, h, fb.one);
+        fb.rho[p] = fs_fe(h);
+    }
+}
+
+// Member p: its claim, its two tables, and rho_p times the sums of round 0.  With no rounds at all
+// (every k = 1) the member's three transcript words are complete here.
+__global__ void __launch_bounds__(FS_THREADS)
+fsb_build_kernel(const ProofDev* proofs, const FsProof* fs, FsBatch fb, imm_fe* tr, int32_t* status)
+{
+    __shared__ uint64_t red[33];
+    __shared__ uint64_t red3[3][32];
+    const int p = blockIdx.x, tid = threadIdx.x, b = fb.b;
+    const ProofDev pr = proofs[p];
+    imm_fe* ta = fs[p].ta;
+    imm_fe* tb = fs[p].tb;
+    uint64_t s = 0;
+    for (int i = tid; i < pr.n_part_c; i += FS_THREADS) s = gl::add(s, pr.part_c[i]);
+    s = block_sum_fe(s, red);
+    if (pr.c_offset) {
+        uint64_t sr = 0, sc = 0;
+        for (int i = tid; i < pr.n_sum_row; i += FS_THREADS) sr = gl::add(sr, pr.sum_row[i]);
+        for (int i = tid; i < pr.n_sum_col; i += FS_THREADS) sc = gl::add(sc, pr.sum_col[i]);
+        sr = block_sum_fe(sr, red);
+        sc = block_sum_fe(sc, red);
+        s = gl::sub(s, gl::shl(gl::mul(sr, sc), 31));
+    }
+    const int n0 = 1 << b;
+    for (int y = tid; y < n0; y += FS_THREADS) {
+        const bool live = y < pr.k;
+        ta[y] = live ? sum_parts_at(pr.part_a, pr.n_part_a, pr.k, y) : 0;
+        tb[y] = live ? sum_parts_at(pr.part_b, pr.n_part_b, pr.k, y) : 0;
+    }
+    __syncthreads();
+    Sums3 acc = {0, 0, 0};
+    for (int e = tid; e < (n0 >> 1); e += FS_THREADS) sums_add(acc, ta[e], ta[e + (n0 >> 1)], tb[e], tb[e + (n0 >> 1)]);
+    uint64_t g[3] = {acc.g0, acc.g1, acc.g2};
+    block_sum3_fe(g, red3);
+    if (tid == 0) {
+        const uint64_t rho = fb.rho[p];
+        fb.c0[p] = s;
+        status[p] = 0;
+        for (int i = 0; i < 3; i++) fb.partial[3 * p + i] = gl::mul(rho, g[i]);
+        imm_fe* tail = tr + 1 + 3 * b + 3 * (int64_t)p;
+        tail[0] = s;
+        if (b == 0) { tail[1] = ta[0]; tail[2] = tb[0]; }
+    }
+}
+
+// Round j of the whole batch (one block): the combined sums, the transcript words, the hash, r_j.
+// j = 0 also forms the combined claim and starts the transcript state; with b = 0 that is all.
+__global__ void __launch_bounds__(FS_BATCH_MAX) fsb_combine_kernel(FsBatch fb, int j, imm_fe* tr)
+{
+    __shared__ uint64_t red[33];
+    __shared__ uint64_t red3[3][32];
+    const int tid = threadIdx.x;
+    uint32_t st[8];
+    if (j == 0) {
+        uint64_t c = 0;
+        for (int p = tid; p < fb.nproofs; p += FS_BATCH_MAX) c = gl::add(c, gl::mul(fb.rho[p], fb.c0[p]));
+        c = block_sum_fe(c, red);
+        if (tid == 0) {
+            tr[0] = c;
+#pragma unroll
+            for (int i = 0; i < 8; i++) st[i] = fb.T[i];
+            const uint64_t c0[1] = {c};
+            fs_absorb<1>(st, 0x12, c0, fb.one);
+            if (fb.b == 0) {
+#pragma unroll
+                for (int i = 0; i < 8; i++) fb.state[i] = st[i];
+            }
+        }
+        if (fb.b == 0) return;
+    } else if (tid == 0) {
+#pragma unroll
+        for (int i = 0; i < 8; i++) st[i] = fb.state[i];
+    }
+    uint64_t g[3] = {0, 0, 0};
+    for (int p = tid; p < fb.nproofs; p += FS_BATCH_MAX)
+        for (int i = 0; i < 3; i++) g[i] = gl::add(g[i], fb.partial[3 * p + i]);
+    block_sum3_fe(g, red3);
+    if (tid == 0) {
+        tr[1 + 3 * j] = g[0]; tr[2 + 3 * j] = g[1]; tr[3 + 3 * j] = g[2];
+        const uint64_t hashed[2] = {g[0], g[2]};
+        fs_absorb<2>(st, 0x13, hashed, fb.one);
+        fb.r[j] = fs_fe(st);
+#pragma unroll
+        for (int i = 0; i < 8; i++) fb.state[i] = st[i];
+    }
+}
+
+// Member p folds with r_j and takes rho_p times the sums of round j + 1 from the folded values; after
+// the last round its a_fin, b_fin complete its three transcript words.
+__global__ void __launch_bounds__(FS_THREADS)
+fsb_fold_kernel(const FsProof* fs, FsBatch fb, int j, imm_fe* tr)
+{
+    __shared__ uint64_t red3[3][32];
+    const int p = blockIdx.x, tid = threadIdx.x, b = fb.b;
+    imm_fe* ta = fs[p].ta;
+    imm_fe* tb = fs[p].tb;
+    const uint64_t r = fb.r[j];
+    const int n = 1 << (b - j), h = n >> 1, q = n >> 2;
+    if (h == 1) {
+        if (tid == 0) {
+            imm_fe* tail = tr + 1 + 3 * b + 3 * (int64_t)p;
+            tail[1] = fold1(ta[0], ta[1], r);
+            tail[2] = fold1(tb[0], tb[1], r);
+        }
+        return;
+    }
+    Sums3 acc = {0, 0, 0};
+    for (int e = tid; e < q; e += FS_THREADS) {            // in place: each thread rewrites only what it alone read
+        const uint64_t fa0 = fold1(ta[e], ta[e + h], r), fa1 = fold1(ta[e + q], ta[e + q + h], r);
+        const uint64_t fb0 = fold1(tb[e], tb[e + h], r), fb1 = fold1(tb[e + q], tb[e + q + h], r);
+        ta[e] = fa0; ta[e + q] = fa1; tb[e] = fb0; tb[e + q] = fb1;
+        sums_add(acc, fa0, fa1, fb0, fb1);
+    }
+    uint64_t g[3] = {acc.g0, acc.g1, acc.g2};
+    block_sum3_fe(g, red3);
+    if (tid == 0) {
+        const uint64_t rho = fb.rho[p];
+        for (int i = 0; i < 3; i++) fb.partial[3 * p + i] = gl::mul(rho, g[i]);
+    }
+}
+
+// ------------------------------------------------------------------------------------------
 // the verifier's own evaluations: c0 = C~(r_row, r_col), a_fin = A~(r_row, r_k), b_fin = B~(r_k, r_col)
 // ------------------------------------------------------------------------------------------
 // The three contractions are the prover's (partial sums of C, partial vectors of A and B); where the
@@ -960,6 +1130,19 @@ expected_kernel(const ProofDev* proofs, const ExpectDev* ex, imm_fe* expected, i
 // ------------------------------------------------------------------------------------------
 // launch wrappers
 // ------------------------------------------------------------------------------------------
+
+cudaError_t launch_fs_batched_rounds(const ProofDev* d_proofs, const FsProof* d_fs, const FsBatch& fb, imm_fe* transcript,
+                                     int32_t* status, cudaStream_t st)
+{
+    fsb_seed_kernel<<<1, FS_BATCH_MAX, 0, st>>>(d_fs, fb);
+    fsb_build_kernel<<<fb.nproofs, FS_THREADS, 0, st>>>(d_proofs, d_fs, fb, transcript, status);
+    fsb_combine_kernel<<<1, FS_BATCH_MAX, 0, st>>>(fb, 0, transcript);
+    for (int j = 0; j < fb.b; j++) {
+        if (j > 0) fsb_combine_kernel<<<1, FS_BATCH_MAX, 0, st>>>(fb, j, transcript);
+        fsb_fold_kernel<<<fb.nproofs, FS_THREADS, 0, st>>>(d_fs, fb, j, transcript);
+    }
+    return cudaGetLastError();
+}
 
 cudaError_t launch_expected(const ProofDev* d_proofs, const ExpectDev* d_ex, int nproofs, imm_fe* expected,
                             int32_t* status, cudaStream_t st)

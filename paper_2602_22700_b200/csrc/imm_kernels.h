@@ -39,5 +39,9 @@ cudaError_t launch_sumcheck_fs(const ProofDev* d_proofs, const FsProof* d_fs, in
 // the verifier's own (c0, a_fin, b_fin) per proof from the contractions' partial results and E_k
 cudaError_t launch_expected(const ProofDev* d_proofs, const ExpectDev* d_ex, int nproofs, imm_fe* expected,
                             int32_t* status, cudaStream_t st);
+// batched non-interactive proof: seed and coefficients, members' tables, then per round a combining launch and a
+// folding launch (3 + 2b launches in all)
+cudaError_t launch_fs_batched_rounds(const ProofDev* d_proofs, const FsProof* d_fs, const FsBatch& fb, imm_fe* transcript,
+                                     int32_t* status, cudaStream_t st);
 
 }  // namespace imm

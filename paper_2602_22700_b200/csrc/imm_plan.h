@@ -109,6 +109,20 @@ struct FsProof {
     uint32_t pad_;
 };
 
+// One batched non-interactive proof: where its coins and per-round exchange live (device pointers).
+constexpr int FS_BATCH_MAX = 1024;          // members of one batched non-interactive proof (one block folds their statements)
+struct FsBatch {
+    uint32_t* T;               // [8]  the batch seed: hash of the tree over the member statements, the id, the count
+    uint32_t* state;           // [8]  the transcript state
+    imm_fe* rho;               // [P]  combination coefficients
+    imm_fe* c0;                // [P]  the members' claims
+    imm_fe* partial;           // [P][3] rho_p times the current round's three sums of member p
+    imm_fe* r;                 // [MAX_K_VARS] round challenges as they become known
+    uint64_t batch_id;
+    int32_t nproofs, b;
+    uint32_t one, pad_;
+};
+
 // Per proof of a verifier's pass: the eq table of the round challenges, E_k[y] = eq(r_k, y).
 constexpr int VERIFY_POINT_SLOTS = 3 * FS_POINT_SLOTS;      // caller-given points per proof: r_row, r_col, r_k
 struct ExpectDev {

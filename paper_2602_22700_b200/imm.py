@@ -35,7 +35,10 @@ EXPORTS = ("imm_version", "imm_last_cuda_error", "imm_challenge", "imm_field_bin
            "imm_sumcheck_matmul_prove_batched", "imm_sumcheck_verify_batched",
            "imm_commit_workspace", "imm_commit", "imm_commit_launches",
            "imm_sumcheck_matmul_fs_workspace", "imm_sumcheck_matmul_prove_fs", "imm_fs_challenges",
-           "imm_sumcheck_verify_fs", "imm_sumcheck_expected_workspace", "imm_sumcheck_expected")
+           "imm_sumcheck_verify_fs", "imm_sumcheck_expected_workspace", "imm_sumcheck_expected",
+           "imm_sumcheck_matmul_fs_batched_workspace", "imm_sumcheck_matmul_prove_fs_batched",
+           "imm_fs_batched_challenges", "imm_sumcheck_verify_fs_batched")
+FS_BATCH_MAX = 1024
 COMMIT_LEAF = 4096
 NOALLOC_MAX_TILES = 8192
 PROFILE_PHASES = ("eq_tables", "claim_C", "bind_rows_A", "bind_cols_B", "sumcheck_rounds")
@@ -126,6 +129,14 @@ def lib() -> ctypes.CDLL:
     L.imm_fs_challenges.argtypes = [vp, ci, vp, i64, i64, i64, u64, vp, vp, vp]
     L.imm_sumcheck_verify_fs.restype = ci
     L.imm_sumcheck_verify_fs.argtypes = [vp, ci, vp, i64, i64, i64, u64, vp, vp, vp, vp]
+    L.imm_sumcheck_matmul_fs_batched_workspace.restype = sz
+    L.imm_sumcheck_matmul_fs_batched_workspace.argtypes = [vp, ci]
+    L.imm_sumcheck_matmul_prove_fs_batched.restype = ci
+    L.imm_sumcheck_matmul_prove_fs_batched.argtypes = [vp, ci, vp, u64, vp, vp, vp, sz, vp]
+    L.imm_fs_batched_challenges.restype = ci
+    L.imm_fs_batched_challenges.argtypes = [vp, ci, vp, ci, vp, u64, vp, vp]
+    L.imm_sumcheck_verify_fs_batched.restype = ci
+    L.imm_sumcheck_verify_fs_batched.argtypes = [vp, ci, vp, ci, vp, u64, vp, vp]
     L.imm_sumcheck_expected_workspace.restype = sz
     L.imm_sumcheck_expected_workspace.argtypes = [vp, ci, ci]
     L.imm_sumcheck_expected.restype = ci
@@ -593,6 +604,103 @@ def sumcheck_verify_fs(transcript: Sequence[int], nrounds: int, commitments, m: 
     rc = lib().imm_sumcheck_verify_fs(ctypes.addressof(arr), nrounds, ctypes.addressof(com), m, k, n, proof_id,
                                       opt(expect_c0), opt(expect_a_fin), opt(expect_b_fin), ctypes.addressof(fail))
     _check(rc, "imm_sumcheck_verify_fs")
+    return rc, fail.value
+
+
+class FsBatchedProver:
+    """One non-interactive proof for all products of a batch (at most FS_BATCH_MAX members)."""
+
+    def __init__(self, problems, commitments: torch.Tensor, device="cuda"):
+        self.problems = list(problems)
+        self.descs = make_descs(self.problems)
+        self.nproofs = len(self.problems)
+        self.commitments = _cuda(commitments, torch.uint8, "commitments").contiguous()
+        if self.commitments.numel() != 96 * self.nproofs:
+            raise ValueError("commitments must hold 96 bytes per proof")
+        self.nrounds = max(ceil_log2(A.shape[1]) for (A, _, _, _) in self.problems)
+        need = lib().imm_sumcheck_matmul_fs_batched_workspace(ctypes.addressof(self.descs), self.nproofs)
+        if need == 0:
+            raise ImmError(ERR_LIMIT if self.nproofs > FS_BATCH_MAX else ERR_SHAPE,
+                           "imm_sumcheck_matmul_fs_batched_workspace")
+        self.ws = torch.empty(need, dtype=torch.uint8, device=device)
+        self.length = batched_transcript_len(self.nrounds, self.nproofs)
+        self.transcript = torch.zeros((self.length,), dtype=torch.int64, device=device)
+        self.status = torch.full((self.nproofs,), -99, dtype=torch.int32, device=device)
+        self.launches = 6 + 3 + 2 * self.nrounds            # statements, eq, three contractions ... and the round chain
+
+    def prove(self, batch_id: int) -> torch.Tensor:
+        _check(lib().imm_sumcheck_matmul_prove_fs_batched(ctypes.addressof(self.descs), self.nproofs,
+                                                          self.commitments.data_ptr(), batch_id,
+                                                          self.transcript.data_ptr(), self.status.data_ptr(),
+                                                          self.ws.data_ptr(), self.ws.numel(), _stream()),
+               "imm_sumcheck_matmul_prove_fs_batched")
+        return self.transcript
+
+
+def sumcheck_matmul_prove_fs_batched(problems, commitments: torch.Tensor, batch_id: int) -> List[int]:
+    """Convenience: the batched non-interactive transcript as Python ints (synchronises)."""
+    pr = FsBatchedProver(problems, commitments)
+    t = pr.prove(batch_id)
+    torch.cuda.synchronize()
+    if int(pr.status.abs().max()) != 0:
+        raise ImmError(int(pr.status.min()), "device status")
+    return [int(v) & 0xFFFFFFFFFFFFFFFF for v in t.cpu()]
+
+
+def _shape_descs(shapes_and_ids):
+    """Descriptor array that carries only m, k, n and proof_id (for the host functions)."""
+    arr = (MatmulDesc * len(shapes_and_ids))()
+    for i, (m, k, n, pid) in enumerate(shapes_and_ids):
+        arr[i] = MatmulDesc(None, None, None, m, k, n, k, n, n, pid)
+    return arr
+
+
+def fs_batched_challenges(transcript: Optional[Sequence[int]], nrounds: int, shapes_and_ids, commitments,
+                          batch_id: int) -> Tuple[List[int], List[int]]:
+    """(rho, r_k) of a batched non-interactive proof; ``shapes_and_ids``: (m, k, n, proof_id) per member,
+    ``commitments``: 96 bytes per member."""
+    n = len(shapes_and_ids)
+    descs = _shape_descs(shapes_and_ids)
+    data = bytes(commitments)
+    if len(data) != 96 * n:
+        raise ValueError("96 commitment bytes per member")
+    com = (ctypes.c_uint8 * len(data))(*data)
+    rho, rk = (ctypes.c_uint64 * n)(), (ctypes.c_uint64 * max(nrounds, 1))()
+    arr = None
+    if transcript is not None:
+        words = [int(v) & 0xFFFFFFFFFFFFFFFF for v in list(transcript)[:3 * nrounds + 1]]
+        arr = (ctypes.c_uint64 * len(words))(*words)
+    _check(lib().imm_fs_batched_challenges(None if arr is None else ctypes.addressof(arr), nrounds,
+                                           ctypes.addressof(descs), n, ctypes.addressof(com), batch_id,
+                                           ctypes.addressof(rho), None if arr is None else ctypes.addressof(rk)),
+           "imm_fs_batched_challenges")
+    return list(rho), (list(rk)[:nrounds] if arr is not None else [])
+
+
+def sumcheck_verify_fs_batched(transcript: Sequence[int], nrounds: int, shapes_and_ids, commitments, batch_id: int,
+                               expect: Optional[Sequence[int]] = None) -> Tuple[int, int]:
+    """Host verifier of a batched non-interactive proof; returns (status, fail_at)."""
+    n = len(shapes_and_ids)
+    total = 1 + 3 * nrounds + 3 * n
+    words = [int(v) & 0xFFFFFFFFFFFFFFFF for v in list(transcript)[:total]]
+    if len(words) != total:
+        raise ValueError("transcript too short")
+    arr = (ctypes.c_uint64 * total)(*words)
+    descs = _shape_descs(shapes_and_ids)
+    data = bytes(commitments)
+    if len(data) != 96 * n:
+        raise ValueError("96 commitment bytes per member")
+    com = (ctypes.c_uint8 * len(data))(*data)
+    exp = None
+    if expect is not None:
+        if len(expect) != 3 * n:
+            raise ValueError("expect must hold 3 words per member")
+        exp = (ctypes.c_uint64 * (3 * n))(*[int(v) & 0xFFFFFFFFFFFFFFFF for v in expect])
+    fail = ctypes.c_int(-2)
+    rc = lib().imm_sumcheck_verify_fs_batched(ctypes.addressof(arr), nrounds, ctypes.addressof(descs), n,
+                                              ctypes.addressof(com), batch_id,
+                                              None if exp is None else ctypes.addressof(exp), ctypes.addressof(fail))
+    _check(rc, "imm_sumcheck_verify_fs_batched")
     return rc, fail.value
 
 

@@ -125,6 +125,49 @@ def test_fs_host_challenges_and_verifier_match_oracle(imm, oracle):
         imm.sumcheck_verify_fs([oracle.P, 0, 0], 0, bytes(96), 1, 1, 1, 0)
 
 
+def test_fs_batched_host_coins_and_verifier_match_oracle(imm, oracle):
+    rng = random.Random(5)
+    for shapes in ([(3, 8, 2), (2, 5, 4), (1, 7, 1)], [(2, 1, 2), (1, 1, 3)], [(4, 16, 4)],
+                   [(2, 3, 2), (1, 9, 1), (3, 2, 2), (2, 2, 2), (1, 1, 1)]):
+        probs, meta = [], []
+        for i, (m, k, n) in enumerate(shapes):
+            A = np.array([[rng.randint(-128, 127) for _ in range(k)] for _ in range(m)], dtype=np.int8)
+            B = np.array([[rng.randint(-128, 127) for _ in range(n)] for _ in range(k)], dtype=np.int8)
+            C = (A.astype(np.int64) @ B.astype(np.int64)).astype(np.int32)
+            coms, pid = [rng.randbytes(32) for _ in range(3)], rng.getrandbits(40)
+            probs.append((A, B, C, coms, pid))
+            meta.append((m, k, n, pid))
+        bid, count = rng.getrandbits(64), len(shapes)
+        b = max(oracle.ceil_log2(k) for (_, k, _) in shapes)
+        t = oracle.fs.prove_batched(probs, bid)
+        com = b"".join(b"".join(c) for (_, _, _, c, _) in probs)
+        stmts = [oracle.fs.statement(c, m, k, n, pid) for (_, _, _, c, _), (m, k, n, pid) in zip(probs, meta)]
+        want = oracle.fs.challenges_batched(t, b, stmts, bid)
+        assert imm.fs_batched_challenges(t, b, meta, com, bid) == tuple(want)
+        assert imm.sumcheck_verify_fs_batched(t, b, meta, com, bid) == (imm.OK, -1)
+        assert imm.sumcheck_verify_fs_batched(t, b, meta, com, bid, t[-3 * count:]) == (imm.OK, -1)
+        for pos in range(len(t)):
+            bad = list(t)
+            bad[pos] = (bad[pos] + 1 + rng.randrange(oracle.P - 1)) % oracle.P
+            got = imm.sumcheck_verify_fs_batched(bad, b, meta, com, bid)
+            assert got == oracle.fs.verify_batched(bad, b, stmts, bid)
+            if got[0] != imm.REJECT:
+                # only a factor whose partner is zero can change unnoticed by the rounds (the verifier's
+                # own evaluations catch it): a_fin_p next to b_fin_p = 0, or the other way round
+                off = pos - (1 + 3 * b)
+                assert off >= 0 and off % 3 in (1, 2) and t[pos + (1 if off % 3 == 1 else -1)] == 0
+        assert imm.sumcheck_verify_fs_batched(t, b, meta, com, bid + 1)[0] == imm.REJECT
+        swapped = bytes([com[5] ^ 1]).join([com[:5], com[6:]])
+        assert imm.sumcheck_verify_fs_batched(t, b, meta, swapped, bid)[0] == imm.REJECT
+        with pytest.raises(imm.ImmError):
+            imm.sumcheck_verify_fs_batched(t + [0] * 3, b + 1, meta, com, bid)       # nrounds is the largest ceil(log2 k)
+    L = imm.lib()
+    big = _desc_array(imm, [(2, 4, 2)] * 1025)
+    assert L.imm_sumcheck_matmul_fs_batched_workspace(ctypes.addressof(big), 1025) == 0
+    assert L.imm_sumcheck_matmul_prove_fs_batched(ctypes.addressof(big), 1025, 0x1000, 1, 0x1000, 0x1000, 0x1000,
+                                                  1 << 30, None) == imm.ERR_LIMIT
+
+
 def _desc_array(imm, shapes, base=0x10000):
     arr = (imm.MatmulDesc * len(shapes))()
     for i, (m, k, n) in enumerate(shapes):

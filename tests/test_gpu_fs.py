@@ -138,3 +138,84 @@ def test_repeated_calls_and_interleaving_with_the_interactive_prover(imm, oracle
     assert torch.equal(first, again) and int(fp.status.abs().max()) == 0
     for (A, B, C, pid), t in zip(group, plain):
         assert t == [int(w) for w in oracle.sumcheck_matmul_prove(A, B, C, 5, pid)]
+
+
+# ------------------------------------------------------------------ batched non-interactive proof
+
+def batched_case(imm, oracle, group, bid, rs=None):
+    dev = on_gpu(group)
+    coms = imm.commit_matrices(dev, rs)
+    want_coms = oracle_coms(oracle, group, rs)
+    got = imm.sumcheck_matmul_prove_fs_batched(dev, coms, bid)
+    want = oracle.fs.prove_batched([(A, B, C, cm, pid) for (A, B, C, pid), cm in zip(group, want_coms)], bid)
+    assert got == want
+    meta = [(A.shape[0], A.shape[1], B.shape[1], pid) for A, B, C, pid in group]
+    com = b"".join(b"".join(c) for c in want_coms)
+    b = max(oracle.ceil_log2(k) for (_, k, _, _) in meta)
+    assert imm.sumcheck_verify_fs_batched(got, b, meta, com, bid) == (imm.OK, -1)
+    return dev, got, meta, com, b
+
+
+@pytest.mark.parametrize("shapes", [
+    [(3, 8, 2), (2, 5, 4), (1, 7, 1)],
+    [(2, 1, 2), (1, 1, 3)],                                          # no rounds
+    [(5, 2, 5)],                                                     # one member, one round
+    [(33, 300, 17), (64, 512, 64), (1, 257, 129), (130, 511, 3), (9, 1, 3)],
+    [(4, 100 + 37 * i, 3 + i % 4) for i in range(37)],               # 37 members: odd tree levels over the statements
+])
+def test_batched_transcripts_equal_oracle(imm, oracle, backend, shapes):
+    rng = np.random.default_rng(sum(sum(s) for s in shapes) + 1)
+    group = make(rng, shapes, first_id=8)
+    batched_case(imm, oracle, group, bid=2**63 + 11)
+
+
+def test_batched_full_loop_with_the_verifiers_pass(imm, oracle):
+    """Prove, derive the coins on the host, evaluate the opened matrices on the GPU, verify."""
+    rng = np.random.default_rng(21)
+    group = make(rng, [(40, 700, 9), (3, 513, 200), (64, 64, 64), (7, 5000, 2)], first_id=1)
+    dev, got, meta, com, b = batched_case(imm, oracle, group, bid=5)
+    _, r_k = imm.fs_batched_challenges(got, b, meta, com, 5)
+    points = []
+    for i, (m, k, n, pid) in enumerate(meta):
+        r_row, r_col, _ = imm.fs_challenges(None, oracle.ceil_log2(k), com[96 * i:96 * i + 96], m, k, n, pid)
+        points.append((r_row, r_col, r_k))
+    own = imm.sumcheck_expected(dev, batch_id=5, points=points)
+    flat = [w for vals in own for w in vals]
+    assert got[1 + 3 * b:] == flat
+    assert imm.sumcheck_verify_fs_batched(got, b, meta, com, 5, expect=flat) == (imm.OK, -1)
+    # an opened matrix that differs from the committed one: other statement, other coins, rejected
+    A, B, C, pid = group[2]
+    C2 = C.copy()
+    C2[1, 1] += 1
+    bad = [group[0], group[1], (A, B, C2, pid), group[3]]
+    com2 = imm.commit_matrices(on_gpu(bad)).cpu().numpy().tobytes()
+    assert imm.sumcheck_verify_fs_batched(got, b, meta, com2, 5)[0] == imm.REJECT
+
+
+def test_batched_many_members_and_limit(imm, oracle):
+    rng = np.random.default_rng(22)
+    shapes = [(1 + i % 3, 40 + i % 50, 1 + i % 4) for i in range(1024)]
+    group = make(rng, shapes, first_id=0)
+    batched_case(imm, oracle, group, bid=1)
+    dev = on_gpu(make(rng, [(2, 4, 2)] * 1025))
+    coms = torch.zeros((1025, 96), dtype=torch.uint8, device="cuda")
+    with pytest.raises(imm.ImmError) as e:
+        imm.FsBatchedProver(dev, coms)
+    assert e.value.code == imm.ERR_LIMIT
+
+
+def test_batched_decoder_layers_full_size(imm, oracle):
+    """Four layers of the decoder block at 8192 tokens (16 products, k = 4096 and 14336) as one
+    non-interactive proof of fourteen rounds, against the oracle."""
+    from paper_2602_22700_b200 import synth
+    probs = synth.decoder_block(1, 4, 8192, device="cuda")
+    dev = [(p.A, p.B, p.C, p.proof_id) for p in probs]
+    coms = imm.commit_matrices(dev)
+    got = imm.sumcheck_matmul_prove_fs_batched(dev, coms, 99)
+    host_coms = coms.cpu().numpy()
+    members = []
+    for p, c in zip(probs, host_coms):
+        members.append((p.A.cpu().numpy(), p.B.cpu().numpy(), p.C.cpu().numpy(),
+                        [bytes(c[0:32]), bytes(c[32:64]), bytes(c[64:96])], p.proof_id))
+    assert got == oracle.fs.prove_batched(members, 99)
+    assert len(got) == 1 + 42 + 48

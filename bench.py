@@ -2,7 +2,7 @@
 """Throughput of the sumcheck matmul prover on synthetic transformer-shaped layers.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--config decoder|qkv|ffn|moe|attn|ldd|commit] [--batched | --fs | --verify]
+                    [--config decoder|qkv|ffn|moe|attn|ldd|commit] [--batched] [--fs] [--verify]
                     [--layers L] [--tokens T] [--no-e2e] [--no-cpu-baseline]
 
 One step = one proving pass over the whole batch: eq tables, A~ / B~ partial evaluations, the
@@ -12,7 +12,8 @@ tokens, 128 proofs, 39.25 GiB of int8/int32 inputs resident in HBM (far larger t
 flush is needed between steps).  Rank 0 prints ONE JSON line.
 
 --batched proves all products of the workload as one random-linear-combination proof;
---fs makes a step commit to every matrix (SHA-256 trees) and prove non-interactively; --verify times
+--fs makes a step commit to every matrix (SHA-256 trees) and prove non-interactively (with --batched: one
+non-interactive proof for the whole workload); --verify times
 the verifier's pass over the same matrices; --config ldd
 and --config commit time the logit distances and the response commitments (their own metrics).
 
@@ -248,7 +249,7 @@ def run_ours(args):
     algo_bytes = synth.problem_bytes(problems)
     claim_bytes = sum(4 * m * n for (m, k, n) in shapes)
     groups = {}
-    if args.batched:
+    if args.batched and not args.fs:
         groups[max(imm.ceil_log2(p.mkn[1]) for p in problems)] = list(problems)
         provers = [imm.BatchedProver([(p.A, p.B, p.C, p.proof_id) for p in g], device=dev) for g in groups.values()]
 
@@ -264,7 +265,12 @@ def run_ours(args):
     elif args.fs:
         triples = [(p.A, p.B, p.C, p.proof_id) for p in problems]
         com = imm.Committer([t for (A, B, C, _) in triples for t in (A, B, C)], device=dev)
-        fsp = imm.FsProver(triples, com.digests.view(len(triples), 96), device=dev)
+        if args.batched:
+            fsp = imm.FsBatchedProver(triples, com.digests.view(len(triples), 96), device=dev)
+            fsp_prove = lambda: fsp.prove(BATCH_ID0)
+        else:
+            fsp = imm.FsProver(triples, com.digests.view(len(triples), 96), device=dev)
+            fsp_prove = fsp.prove
         provers = [fsp]
         fs_ev = []
 
@@ -273,7 +279,7 @@ def run_ours(args):
             e[0].record()
             com.commit()
             e[1].record()
-            fsp.prove()
+            fsp_prove()
             e[2].record()
             fs_ev.append(e)
     else:
@@ -341,6 +347,14 @@ def run_ours(args):
             if imm.sumcheck_verify(words, b, SEED, p.proof_id, *[int(v) for v in vals[i]]) == (imm.OK, -1):
                 accepted += 1
         del pr2
+    elif args.fs and args.batched:
+        host_t = None
+        assert int(fsp.status.abs().max()) == 0
+        words = [int(v) & 0xFFFFFFFFFFFFFFFF for v in fsp.transcript.cpu()]
+        meta = [tuple(p.mkn) + (p.proof_id,) for p in problems]
+        host_c = com.digests.cpu().numpy().tobytes()
+        if imm.sumcheck_verify_fs_batched(words, fsp.nrounds, meta, host_c, BATCH_ID0) == (imm.OK, -1):
+            accepted = len(problems)
     elif args.fs:
         host_t = fsp.transcripts.cpu()
         assert int(fsp.status.abs().max()) == 0
@@ -402,8 +416,10 @@ def run_ours(args):
                      "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": claim_gbs / peak,
                      "frac_of_8tbs": claim_gbs / 8000.0,
                      "traffic": (CLAIM_KERNEL_TRAFFIC_RATIO * claim_bytes) if CLAIM_KERNEL_TRAFFIC_RATIO else None},
-        "gpu_launches": ((6 + com.launches) if args.fs else 6 if (args.batched or args.verify) else 5) * calls_per_step * steps,
-        "transcript_words_per_step": (sum(int(bp.length) for bp in provers) if args.batched else
+        "gpu_launches": ((fsp.launches + com.launches) if (args.fs and args.batched) else (6 + com.launches) if args.fs
+                         else 6 if (args.batched or args.verify) else 5) * calls_per_step * steps,
+        "transcript_words_per_step": (int(fsp.length) if (args.fs and args.batched) else
+                                      sum(int(bp.length) for bp in provers) if args.batched else
                                       sum(3 * imm.ceil_log2(k) + 3 for (m, k, n) in shapes)),
         "clocks": clocks,
     }

@@ -4,7 +4,7 @@ on the product path may import this file; it shares no code or table with the CU
 What it instantiates.  Algorithm 1 of the paper has the server send a proof pi with its response:
 no verifier is on line to draw coins, so the public coins of the interactive sumcheck
 (``imm_oracle.c``) are replaced by hashes of everything sent so far -- the Fiat-Shamir transform.
-The paper fixes none of this; the readings below are this build's.
+The paper fixes none of this; the readings below are this implementation's.
 
   H           SHA-256 (``hashlib``, a library step).  Integers are little-endian; a field element is
               the le64 of its canonical value.

@@ -14,7 +14,7 @@
  * itself (reduction with the % operator on 128-bit integers, plain loops, no blocking, no
  * fusion, no reordering).
  *
- * Conventions (fixed by this build; the paper is silent on all of them):
+ * Conventions (fixed by this implementation; the paper is silent on all of them):
  *   field       p = 2^64 - 2^32 + 1; elements are canonical uint64 in [0, p).
  *   lift        signed integer v -> v mod p (negative v -> p - |v|).
  *   variables   an index of n bits has variables z_0..z_{n-1}, z_0 the MOST significant bit.

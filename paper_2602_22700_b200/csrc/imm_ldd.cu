@@ -43,7 +43,7 @@ __device__ __forceinline__ float ex2(float x)
 // Slice of block c: [s0, s1), s0 a multiple of 4 so that 16-byte loads stay aligned.
 __device__ __forceinline__ void slice_bounds(int64_t n, int nc, int c, int64_t& s0, int64_t& s1)
 {
-    const int64_t per = ((n + nc - 1) / nc + 3) / 4 * 4;
+    const int64_t per = (((uint32_t)n + (uint32_t)nc - 1) / (uint32_t)nc + 3) / 4 * 4;     // (n <= 2^20: a 32-bit division)
     s0 = min(n, (int64_t)c * per);
     s1 = min(n, s0 + per);
 }
@@ -65,21 +65,17 @@ __device__ __forceinline__ void ms_add1(MaxSum& a, float x)
     a.s += ex2((x - a.m) * LOG2E);
 }
 
-__device__ __forceinline__ MaxSum ms_merge(MaxSum a, MaxSum b)
-{
-    const float m = fmaxf(a.m, b.m);
-    if (m == NEG_INF) return MaxSum{NEG_INF, 0.f};                    // both empty
-    return MaxSum{m, a.s * ex2((a.m - m) * LOG2E) + b.s * ex2((b.m - m) * LOG2E)};
-}
-
+// Merge over a warp: the maximum first, then every lane rescales its own sum once and the sums are
+// added (one exponential per lane instead of two per merge step).
 __device__ __forceinline__ MaxSum ms_warp(MaxSum a)
 {
+    float m = a.m;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        MaxSum b{__shfl_xor_sync(0xFFFFFFFFu, a.m, o), __shfl_xor_sync(0xFFFFFFFFu, a.s, o)};
-        a = ms_merge(a, b);
-    }
-    return a;
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+    float s = a.m == NEG_INF ? 0.f : a.s * ex2((a.m - m) * LOG2E);          // (an empty lane contributes nothing)
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
+    return MaxSum{m, s};
 }
 
 __device__ __forceinline__ float4 ld4(const float* p)
@@ -101,7 +97,7 @@ struct TvKlShared {
     MaxSum pub_p, pub_q;                  // this block's slice; read by the other blocks
     float max_p, max_q, l2s_p, l2s_q;     // the rows' maxima and log2 of their sums of exp(x - max)
     float warp_tv[NW], warp_kl[NW];
-    double pub_tv, pub_kl;                // this block's share; read by block 0
+    double share_tv[MAX_CLUSTER], share_kl[MAX_CLUSTER];   // block 0: every block's share, stored here by its owner
 };
 
 template <bool VEC, int NT>
@@ -180,22 +176,19 @@ tv_kl_kernel(const float* __restrict__ logits, const float* __restrict__ ref, in
     }
     if (lane == 0) { sh.warp_tv[warp] = tv; sh.warp_kl[warp] = kl; }
     __syncthreads();
-    if (tid == 0) {
-        double a = 0.0, b = 0.0;
+    if (tid == 0) {                                        // this block's share goes into block 0's shared memory
+        double a = 0.0, b = 0.0;                           // (every block is running: the barrier above was passed)
         for (int w = 0; w < NW; w++) { a += (double)sh.warp_tv[w]; b += (double)sh.warp_kl[w]; }
-        sh.pub_tv = a; sh.pub_kl = b;
+        *cluster.map_shared_rank(&sh.share_tv[c], 0) = a;
+        *cluster.map_shared_rank(&sh.share_kl[c], 0) = b;
     }
-    cluster.sync();                                        // every block's share is published
+    cluster.sync();                                        // the shares have arrived; nobody reads another block any more
     if (c == 0 && tid == 0) {
         double a = 0.0, b = 0.0;
-        for (int cc = 0; cc < nc; cc++) {
-            a += *cluster.map_shared_rank(&sh.pub_tv, cc);
-            b += *cluster.map_shared_rank(&sh.pub_kl, cc);
-        }
+        for (int cc = 0; cc < nc; cc++) { a += sh.share_tv[cc]; b += sh.share_kl[cc]; }
         tv_out[step] = 0.5 * a;
         kl_out[step] = b;
     }
-    cluster.sync();                                        // block 0 has read the shares: the others may leave
 }
 
 // ------------------------------------------------------------------------------------------

@@ -217,7 +217,7 @@ def measured_peaks():
 # DRAM traffic of the claim kernel per algorithmic byte, from the ncu capture summarised under
 # profiles/ (dram__bytes_read.sum + dram__bytes_write.sum over 4*m*n); None until a capture of the
 # current kernel exists.
-LDD_TVKL_TRAFFIC_RATIO = (1.074211 + 0.004344) / 1.050673   # tv_kl_kernel<aligned, 512 threads>: (dram read + write) / (8 bytes per entry pair)
+LDD_TVKL_TRAFFIC_RATIO = (1.078953 + 0.004193) / 1.050673   # tv_kl_kernel<aligned, 512 threads>: (dram read + write) / (8 bytes per entry pair)
 COMMIT_TRAFFIC_RATIO = (1.077891 + 0.018910) / 1.050673152                   # commit_leaf_kernel: (dram read + write) / message bytes
 # SHA-256 leaf hashing against the integer ALU pipe (rotates, three-input logic, byte permutes): the
 # pipe retires 64 thread instructions per cycle per SM; the kernel issues 17.18 of them per hashed

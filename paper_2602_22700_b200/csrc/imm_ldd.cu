@@ -165,7 +165,7 @@ tv_kl_kernel(const float* __restrict__ logits, const float* __restrict__ ref, in
                 const float xr = xs[e] - mp, yr = ys[e] - mq;
                 const float p = ex2(fmaf(xr, LOG2E, -lp)), q = ex2(fmaf(yr, LOG2E, -lq));
                 tv += fabsf(p - q);
-                kl = fmaf(q, (yr - xr) - dl, kl);            // log q_v - log p_v
+                kl = fmaf(q, yr - xr, kl);                   // q_v (log q_v - log p_v) without its constant part: below
             }
         }
     }
@@ -187,7 +187,7 @@ tv_kl_kernel(const float* __restrict__ logits, const float* __restrict__ ref, in
         double a = 0.0, b = 0.0;
         for (int cc = 0; cc < nc; cc++) { a += sh.share_tv[cc]; b += sh.share_kl[cc]; }
         tv_out[step] = 0.5 * a;
-        kl_out[step] = b;
+        kl_out[step] = b - (double)dl;                     // sum_v q_v (log S_q - log S_p) = log S_q - log S_p: q sums to 1
     }
 }
 

@@ -535,6 +535,66 @@ tv_kl_small_kernel(const float* __restrict__ logits, const float* __restrict__ r
     if (lane == 0) { tv_out[step] = 0.5 * dtv; kl_out[step] = dkl; }
 }
 
+// Rows of at most 256 entries: a group of LPR lanes per row (8 or 16 lanes, sixteen entries per
+// lane), 32 / LPR rows per warp: the shuffle steps are fewer and serve every row of the warp.
+template <int LPR>
+__global__ void __launch_bounds__(SMALL_WARPS * 32)
+tv_kl_sub_kernel(const float* __restrict__ logits, const float* __restrict__ ref, int64_t steps, int n, int64_t ld,
+                 double* __restrict__ tv_out, double* __restrict__ kl_out)
+{
+    constexpr int RPW = 32 / LPR, SLOTS = 16;
+    const int lane = threadIdx.x & 31, g = lane / LPR, gl = lane % LPR;
+    const int64_t step = ((int64_t)blockIdx.x * SMALL_WARPS + (threadIdx.x >> 5)) * RPW + g;
+    const bool live = step < steps;                    // (lanes of a row past the end idle along)
+    const float* x = logits + (live ? step : 0) * ld;
+    const float* y = ref + (live ? step : 0) * ld;
+    float xs[SLOTS], ys[SLOTS];
+    float mx = NEG_INF, my = NEG_INF;
+#pragma unroll
+    for (int j = 0; j < SLOTS; j++) {
+        const int e = gl + LPR * j;
+        xs[j] = (live && e < n) ? x[e] : NEG_INF;
+        ys[j] = (live && e < n) ? y[e] : NEG_INF;
+        mx = fmaxf(mx, xs[j]); my = fmaxf(my, ys[j]);
+    }
+#pragma unroll
+    for (int o = LPR / 2; o > 0; o >>= 1) {
+        mx = fmaxf(mx, __shfl_xor_sync(0xFFFFFFFFu, mx, o));
+        my = fmaxf(my, __shfl_xor_sync(0xFFFFFFFFu, my, o));
+    }
+    if (!live) { mx = 0.f; my = 0.f; }                 // (keeps the idle lanes' arithmetic finite)
+    float sx = 0.f, sy = 0.f;
+#pragma unroll
+    for (int j = 0; j < SLOTS; j++) {                  // slots past the end hold -inf: they add 0
+        sx += ex2((xs[j] - mx) * LOG2E);
+        sy += ex2((ys[j] - my) * LOG2E);
+    }
+#pragma unroll
+    for (int o = LPR / 2; o > 0; o >>= 1) {
+        sx += __shfl_xor_sync(0xFFFFFFFFu, sx, o);
+        sy += __shfl_xor_sync(0xFFFFFFFFu, sy, o);
+    }
+    const float lp = log2f(sx), lq = log2f(sy);
+    const float dl = (lq - lp) * (1.0f / LOG2E);
+    float tv = 0.f, kl = 0.f;
+#pragma unroll
+    for (int j = 0; j < SLOTS; j++) {
+        if (live && gl + LPR * j < n) {
+            const float xr = xs[j] - mx, yr = ys[j] - my;
+            const float p = ex2(fmaf(xr, LOG2E, -lp)), q = ex2(fmaf(yr, LOG2E, -lq));
+            tv += fabsf(p - q);
+            kl = fmaf(q, (yr - xr) - dl, kl);
+        }
+    }
+    double dtv = (double)tv, dkl = (double)kl;
+#pragma unroll
+    for (int o = LPR / 2; o > 0; o >>= 1) {
+        dtv += __shfl_xor_sync(0xFFFFFFFFu, dtv, o);
+        dkl += __shfl_xor_sync(0xFFFFFFFFu, dkl, o);
+    }
+    if (live && gl == 0) { tv_out[step] = 0.5 * dtv; kl_out[step] = dkl; }
+}
+
 // Top-K distance of a short row.  The K largest entries outside I are pulled out one at a time
 // (K warp-wide arg-max rounds over the registers); the cost is then evaluated at the 2K
 // breakpoints in float64, as in the long-row kernel.
@@ -612,6 +672,89 @@ topk_small_kernel(const float* __restrict__ ref, int64_t steps, int n, int64_t l
 // slots per lane a row of n entries needs, rounded to the instantiated sizes
 inline int small_slots(int64_t n) { return n <= 128 ? 4 : n <= 256 ? 8 : n <= 512 ? 16 : 32; }
 
+// Rows of at most 256 entries with a small K: a group of LPR lanes per row (LPR = 8 or 16, sixteen
+// entries per lane), so a warp works on 32 / LPR rows at once and every shuffle, ballot and compare
+// instruction serves all of them.  Same selection as topk_small_kernel: K rounds of a group-wide
+// arg-max over the entries outside I, then the cost at the 2K breakpoints in float64.
+constexpr int SUB_SLOTS = 16;
+constexpr int SUB_MAX_K = 16;
+
+template <int LPR>
+__global__ void __launch_bounds__(SMALL_WARPS * 32)
+topk_sub_kernel(const float* __restrict__ ref, int64_t steps, int n, int64_t ld, const int32_t* __restrict__ topk, int K,
+                double* __restrict__ dist_out, int32_t* __restrict__ status)
+{
+    constexpr int RPW = 32 / LPR;                          // rows per warp
+    __shared__ double outside[SMALL_WARPS][RPW][SUB_MAX_K], inside[SMALL_WARPS][RPW][SUB_MAX_K];
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+    const int g = lane / LPR, gl = lane % LPR;             // the row of this lane within the warp, its lane within the row
+    const unsigned gmask = (LPR == 32 ? 0xFFFFFFFFu : ((1u << LPR) - 1u)) << (g * LPR);
+    const int64_t step = ((int64_t)blockIdx.x * SMALL_WARPS + w) * RPW + g;
+    const bool live = step < steps;                        // (lanes of a row past the end idle along: the shuffles are warp-wide)
+    const float* y = ref + (live ? step : 0) * ld;
+    const int32_t* I = topk + (live ? step : 0) * K;
+    float v[SUB_SLOTS];
+#pragma unroll
+    for (int j = 0; j < SUB_SLOTS; j++) {
+        const int e = gl + LPR * j;
+        v[j] = (live && e < n) ? y[e] : NEG_INF;
+    }
+    bool bad = false;
+    uint32_t mine = 0;                                     // bit j: this lane's slot j belongs to I
+    for (int k = 0; k < K; k++) {
+        const int idx = live ? I[k] : 0;
+        if (idx < 0 || idx >= n) { bad = true; continue; }
+        if (idx % LPR == gl) {
+            const uint32_t bit = 1u << (idx / LPR);
+            if (mine & bit) bad = true;                    // the same index twice
+            mine |= bit;
+        }
+    }
+    bad = (__ballot_sync(0xFFFFFFFFu, bad) & gmask) != 0;
+    if (live)
+        for (int k = gl; k < K; k += LPR) {
+            const int idx = I[k];
+            inside[w][g][k] = (idx >= 0 && idx < n) ? (double)y[idx] : 0.0;
+        }
+#pragma unroll
+    for (int j = 0; j < SUB_SLOTS; j++) if ((mine >> j) & 1u) v[j] = NEG_INF;
+    for (int r = 0; r < K; r++) {
+        float best = NEG_INF;
+        int slot = 0;
+#pragma unroll
+        for (int j = 0; j < SUB_SLOTS; j++) if (v[j] > best) { best = v[j]; slot = j; }
+        float top = best;
+#pragma unroll
+        for (int o = LPR / 2; o > 0; o >>= 1) top = fmaxf(top, __shfl_xor_sync(0xFFFFFFFFu, top, o));
+        const unsigned holders = __ballot_sync(0xFFFFFFFFu, best == top) & gmask;
+        const int winner = __ffs(holders) - 1;             // lowest lane of the row holding its maximum
+        if (lane == winner) {
+            outside[w][g][r] = (double)top;                // (-inf once fewer than K entries are left outside I)
+#pragma unroll
+            for (int j = 0; j < SUB_SLOTS; j++) if (j == slot) v[j] = NEG_INF;
+        }
+    }
+    __syncwarp();
+    double best_cost = INFINITY;
+    for (int cnd = gl; cnd < 2 * K; cnd += LPR) {
+        const double t = cnd < K ? outside[w][g][cnd] : inside[w][g][cnd - K];
+        if (t > -INFINITY) {
+            double c = 0.0;
+            for (int k = 0; k < K; k++) {
+                c += fmax(outside[w][g][k] - t, 0.0);
+                c += fmax(t - inside[w][g][k], 0.0);
+            }
+            best_cost = fmin(best_cost, c);
+        }
+    }
+#pragma unroll
+    for (int o = LPR / 2; o > 0; o >>= 1) best_cost = fmin(best_cost, __shfl_xor_sync(0xFFFFFFFFu, best_cost, o));
+    if (live && gl == 0) {
+        dist_out[step] = bad ? NAN : best_cost;
+        status[step] = bad ? IMM_ERR_ARG : IMM_OK;
+    }
+}
+
 // ------------------------------------------------------------------------------------------
 // per-request tail statistic
 // ------------------------------------------------------------------------------------------
@@ -681,6 +824,16 @@ int imm_ldd_tv_kl(const float* d_logits, const float* d_ref_logits, int64_t step
     if ((uintptr_t)d_logits % 4 || (uintptr_t)d_ref_logits % 4 || (uintptr_t)d_tv % 8 || (uintptr_t)d_kl % 8) return IMM_ERR_ALIGN;
     if (steps == 0) return IMM_OK;
     cudaStream_t st = (cudaStream_t)stream;
+    if (n <= 256) {                                    // very short rows: several rows per warp
+        if (n <= 128) {
+            const unsigned g2 = (unsigned)((steps + SMALL_WARPS * 4 - 1) / (SMALL_WARPS * 4));
+            tv_kl_sub_kernel<8><<<g2, SMALL_WARPS * 32, 0, st>>>(d_logits, d_ref_logits, steps, (int)n, ld, d_tv, d_kl);
+        } else {
+            const unsigned g2 = (unsigned)((steps + SMALL_WARPS * 2 - 1) / (SMALL_WARPS * 2));
+            tv_kl_sub_kernel<16><<<g2, SMALL_WARPS * 32, 0, st>>>(d_logits, d_ref_logits, steps, (int)n, ld, d_tv, d_kl);
+        }
+        return cudaGetLastError() == cudaSuccess ? IMM_OK : IMM_ERR_CUDA;
+    }
     if (n <= SMALL_N) {                                // short rows: one warp per row
         const unsigned grid = (unsigned)((steps + SMALL_WARPS - 1) / SMALL_WARPS);
         switch (small_slots(n)) {
@@ -724,6 +877,16 @@ int imm_ldd_topk_distance(const float* d_ref_logits, int64_t steps, int64_t n, i
     if (n <= SMALL_N) {                                // short rows: one warp per row, no workspace traffic
         const unsigned grid = (unsigned)((steps + SMALL_WARPS - 1) / SMALL_WARPS);
         cudaStream_t sst = (cudaStream_t)stream;
+        if (n <= 16 * SUB_SLOTS && k <= SUB_MAX_K) {       // very short rows: several rows per warp
+            if (n <= 8 * SUB_SLOTS) {
+                const unsigned g2 = (unsigned)((steps + SMALL_WARPS * 4 - 1) / (SMALL_WARPS * 4));
+                topk_sub_kernel<8><<<g2, SMALL_WARPS * 32, 0, sst>>>(d_ref_logits, steps, (int)n, ld, d_topk, k, d_dist, d_status);
+            } else {
+                const unsigned g2 = (unsigned)((steps + SMALL_WARPS * 2 - 1) / (SMALL_WARPS * 2));
+                topk_sub_kernel<16><<<g2, SMALL_WARPS * 32, 0, sst>>>(d_ref_logits, steps, (int)n, ld, d_topk, k, d_dist, d_status);
+            }
+            return cudaGetLastError() == cudaSuccess ? IMM_OK : IMM_ERR_CUDA;
+        }
         switch (small_slots(n)) {
         case 4: topk_small_kernel<4><<<grid, SMALL_WARPS * 32, 0, sst>>>(d_ref_logits, steps, (int)n, ld, d_topk, k, d_dist, d_status); break;
         case 8: topk_small_kernel<8><<<grid, SMALL_WARPS * 32, 0, sst>>>(d_ref_logits, steps, (int)n, ld, d_topk, k, d_dist, d_status); break;

@@ -50,6 +50,7 @@ def check_tv_kl(imm, ldd, x, y):
 
 
 @pytest.mark.parametrize("steps,n", [(7, 1), (5, 3), (9, 100), (19, 64), (9, 128), (5, 256), (4, 1000), (3, 1024), (3, 1025),
+                                     (1003, 100), (515, 200), (66, 257),
                                      (4, 4097), (3, 16384), (3, 16388), (3, 40003),
                                      (2, 128256), (2, 151936), (1, 300000)])
 @pytest.mark.parametrize("noise", ["benign", "quantised", "substituted"])
@@ -113,6 +114,8 @@ def check_topk(imm, ldd, ref, topk, rel=1e-9):
 
 
 @pytest.mark.parametrize("steps,n,k", [(6, 5, 2), (21, 64, 6), (5, 128, 8), (4, 256, 8), (4, 1000, 20), (3, 1024, 64), (3, 1025, 8),
+                                        (1003, 100, 5), (515, 200, 16), (67, 129, 2), (9, 256, 17),      # several rows per warp; K past that path
+
                                         (3, 16384, 20),
                                         (3, 40003, 20), (3, 128256, 20), (2, 151936, 20), (2, 128256, 64),
                                         (2, 300000, 1)])

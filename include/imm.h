@@ -1,7 +1,10 @@
 /*
  * imm.h -- C ABI of the B200 (sm_100a) prover for sumcheck proofs of int8 matrix products
- * over the Goldilocks field p = 2^64 - 2^32 + 1, and (last section) of the logit distance
- * statistics the same audit reports.
+ * over the Goldilocks field p = 2^64 - 2^32 + 1, and of what the same audit needs around it.
+ * Sections, in this order: field and eq-table helpers; multilinear evaluations; the interactive
+ * proof (prover, phase timing, host-buffer variant, host verifier); the batched proof; hash
+ * commitments; the verifier's pass over the opened matrices; the non-interactive (Fiat-Shamir)
+ * proof, per product and per batch; the logit distance statistics.
  *
  * Background.  The audited-inference protocol this library serves has the server prove, for an
  * audited request, that the "continuous transformations" of the reference model -- its
@@ -22,7 +25,8 @@
  *   - Challenges are public coins of an interactive verifier, drawn from a counter-based
  *     generator (SplitMix64 mixer) keyed by (seed, proof_id); they do not depend on the
  *     prover's messages.  domain 1 = r_row, 2 = r_col, 3 = sumcheck rounds, 4 = the
- *     coefficients of a batched proof (keyed by the batch's id).
+ *     coefficients of a batched proof (keyed by the batch's id).  The non-interactive proofs
+ *     hash their challenges from the commitments and the transcript instead (their section).
  *   - Transcript of one proof: [c0, g_0(0), g_0(1), g_0(2), ..., g_{b-1}(0), g_{b-1}(1),
  *     g_{b-1}(2), a_fin, b_fin], b = ceil(log2 k), 3b+3 words.
  *

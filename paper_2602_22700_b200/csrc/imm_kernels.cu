@@ -1022,7 +1022,7 @@ __global__ void __launch_bounds__(FS_BATCH_MAX) fsb_combine_kernel(FsBatch fb, i
     uint32_t st[8];
     if (j == 0) {
         uint64_t c = 0;
-        for (int p = tid; p < fb.nproofs; p += FS_BATCH_MAX) c = gl::add(c, gl::mul(fb.rho[p], fb.c0[p]));
+        for (int p = tid; p < fb.nproofs; p += (int)blockDim.x) c = gl::add(c, gl::mul(fb.rho[p], fb.c0[p]));
         c = block_sum_fe(c, red);
         if (tid == 0) {
             tr[0] = c;
@@ -1041,7 +1041,7 @@ __global__ void __launch_bounds__(FS_BATCH_MAX) fsb_combine_kernel(FsBatch fb, i
         for (int i = 0; i < 8; i++) st[i] = fb.state[i];
     }
     uint64_t g[3] = {0, 0, 0};
-    for (int p = tid; p < fb.nproofs; p += FS_BATCH_MAX)
+    for (int p = tid; p < fb.nproofs; p += (int)blockDim.x)
         for (int i = 0; i < 3; i++) g[i] = gl::add(g[i], fb.partial[3 * p + i]);
     block_sum3_fe(g, red3);
     if (tid == 0) {
@@ -1134,11 +1134,13 @@ expected_kernel(const ProofDev* proofs, const ExpectDev* ex, imm_fe* expected, i
 cudaError_t launch_fs_batched_rounds(const ProofDev* d_proofs, const FsProof* d_fs, const FsBatch& fb, imm_fe* transcript,
                                      int32_t* status, cudaStream_t st)
 {
+    int ct = (fb.nproofs + 31) / 32 * 32;                  // threads of the combining block: one per member, whole warps
+    if (ct > FS_BATCH_MAX) ct = FS_BATCH_MAX;
     fsb_seed_kernel<<<1, FS_BATCH_MAX, 0, st>>>(d_fs, fb);
     fsb_build_kernel<<<fb.nproofs, FS_THREADS, 0, st>>>(d_proofs, d_fs, fb, transcript, status);
-    fsb_combine_kernel<<<1, FS_BATCH_MAX, 0, st>>>(fb, 0, transcript);
+    fsb_combine_kernel<<<1, ct, 0, st>>>(fb, 0, transcript);
     for (int j = 0; j < fb.b; j++) {
-        if (j > 0) fsb_combine_kernel<<<1, FS_BATCH_MAX, 0, st>>>(fb, j, transcript);
+        if (j > 0) fsb_combine_kernel<<<1, ct, 0, st>>>(fb, j, transcript);
         fsb_fold_kernel<<<fb.nproofs, FS_THREADS, 0, st>>>(d_fs, fb, j, transcript);
     }
     return cudaGetLastError();

@@ -23,13 +23,25 @@ Readings (the paper leaves these open)
   * The comparison in p(t1) is strict (">"), as printed.
   * I is a set of K distinct indices; ties in the logits need no rule because entries equal to the
     threshold cost nothing on either side.
+  * Masked entries.  A logit of -inf (a vocabulary entry the sampler has masked out) is a legal
+    input: its softmax probability is exactly 0.  The KL sum uses the usual convention
+    0 * log(0 / x) = 0, so an entry the reference gives no mass adds nothing, and KL = +inf when
+    the reference gives mass to an entry the deployed row masks.  The Top-K cost is minimised over
+    finite thresholds; raising a masked member of I to a finite threshold costs +inf, lowering a
+    masked outside entry costs nothing.  A row with no finite entry has no softmax: TV and KL are
+    NaN (its Top-K distance is +inf, like that of any row whose I has a masked member).
+  * A distance that is not a number (such a row, or a malformed committed index set) must not
+    help the server: p(t1) counts a step unless its distance is known to be <= t1, so NaN counts
+    as exceeding the threshold.  For ordinary numbers this is the printed strict comparison.
 
 Pins (tests/test_oracle_ldd.py): closed forms for two-entry vectors; TV of a vector with itself,
 of disjoint peaks, bounds, symmetry, shift invariance; Pinsker's inequality; scipy's softmax /
 entropy routines as a second opinion; Top-K distance zero iff I is a valid top-K set, the
 swap-one-neighbour closed form, 1-Lipschitz in l, the O(n^2) evaluation of every threshold
 straight from the cost definition, and the minimisation solved as a linear programme by scipy on
-small cases.  No function here is "parity unpinned".
+small cases; masked (-inf) entries against the same functions on the row with those entries
+removed, scipy's entropy on distributions with zeros, and the every-threshold evaluation; NaN
+distances in the tail count.  No function here is "parity unpinned".
 """
 from __future__ import annotations
 
@@ -37,8 +49,11 @@ import numpy as np
 
 
 def log_softmax(logits) -> np.ndarray:
-    """log softmax(l) in float64: l - max - log(sum exp(l - max))."""
+    """log softmax(l) in float64: l - max - log(sum exp(l - max)); -inf entries stay -inf
+    (probability 0); a row without a finite entry gives NaN throughout."""
     x = np.asarray(logits, dtype=np.float64)
+    if not np.isfinite(x).any():
+        return np.full(x.shape, np.nan)
     z = x - x.max()
     return z - np.log(np.exp(z).sum())
 
@@ -56,14 +71,19 @@ def tv_distance(logits, ref_logits) -> float:
 def kl_divergence(logits, ref_logits) -> float:
     """KL(softmax(l*) || softmax(l)): the reference distribution first (a reading, see the header)."""
     lp, lq = log_softmax(logits), log_softmax(ref_logits)
+    if np.isnan(lp).any() or np.isnan(lq).any():
+        return float("nan")
     q = np.exp(lq)
-    return float((q * (lq - lp)).sum())
+    live = q > 0.0                                             # 0 * log(0 / x) = 0
+    with np.errstate(invalid="ignore"):
+        return float((q[live] * (lq[live] - lp[live])).sum())
 
 
 def tail_fraction(distances, t1: float) -> float:
-    """p(t1) of Section 5.3 for one request: the share of its steps whose distance exceeds t1."""
+    """p(t1) of Section 5.3 for one request: the share of its steps whose distance exceeds t1.
+    A step counts unless its distance is known to be <= t1 (NaN counts: see the header)."""
     d = np.asarray(distances, dtype=np.float64)
-    return float((d > t1).sum()) / float(d.size)
+    return float((~(d <= t1)).sum()) / float(d.size)
 
 
 def request_tail_fractions(distances, offsets, t1: float) -> np.ndarray:
@@ -87,9 +107,12 @@ def topk_cost(logits, index_set, t: float) -> float:
 
 
 def topk_distance_all_thresholds(logits, index_set) -> float:
-    """Delta(l, I) by trying every entry of l as the threshold: O(n^2), small inputs only."""
+    """Delta(l, I) by trying every finite entry of l as the threshold: O(n^2), small inputs only."""
     x = np.asarray(logits, dtype=np.float64)
-    return min(topk_cost(x, index_set, float(t)) for t in x)
+    finite = x[np.isfinite(x)]
+    if finite.size == 0:
+        return float("inf")
+    return min(topk_cost(x, index_set, float(t)) for t in finite)
 
 
 def topk_distance(logits, index_set) -> float:
@@ -103,6 +126,10 @@ def topk_distance(logits, index_set) -> float:
     inside[idx] = True
     order = np.argsort(-x, kind="stable")
     xs, ins = x[order], inside[order]
+    nfin = int(np.isfinite(xs).sum())                          # masked (-inf) entries sort last
+    if ins[nfin:].any():                                       # a masked member of I cannot be raised
+        return float("inf")
+    xs, ins = xs[:nfin], ins[:nfin]                            # masked outside entries cost nothing
     out_cnt = np.cumsum(~ins)                                  # entries outside I among the first u
     out_sum = np.cumsum(np.where(ins, 0.0, xs))
     in_cnt_after = ins.sum() - np.cumsum(ins)                  # entries of I after the u-th

@@ -76,6 +76,37 @@ def test_large_logits_do_not_overflow():
     assert ldd.tv_distance(l, ls) == pytest.approx(abs(sigmoid(1.0) - sigmoid(-1.0)), abs=1e-12)
 
 
+def test_masked_entries_have_probability_zero():
+    """-inf logits: the distances are those of the rows with the masked entries removed, where both
+    rows mask the same entries; scipy's entropy (which treats 0 log 0 as 0 and q > 0 = p as inf) as a
+    second opinion where they differ."""
+    from scipy.stats import entropy
+    rng = np.random.default_rng(11)
+    n = 40
+    l, ls = rng.normal(0, 3, n), rng.normal(0, 3, n)
+    mask = rng.random(n) < 0.3
+    lm, lsm = np.where(mask, -np.inf, l), np.where(mask, -np.inf, ls)
+    assert ldd.softmax(lm)[mask].tolist() == [0.0] * int(mask.sum())
+    assert ldd.softmax(lm).sum() == pytest.approx(1.0, abs=1e-15)
+    assert ldd.tv_distance(lm, lsm) == pytest.approx(ldd.tv_distance(l[~mask], ls[~mask]), abs=1e-15)
+    assert ldd.kl_divergence(lm, lsm) == pytest.approx(ldd.kl_divergence(l[~mask], ls[~mask]), abs=1e-14)
+    # only the reference masks: those entries add nothing to KL(q || p); TV sees p's mass there
+    p, q = ldd.softmax(l), ldd.softmax(lsm)
+    assert ldd.kl_divergence(l, lsm) == pytest.approx(entropy(q, p), rel=1e-12)
+    assert ldd.tv_distance(l, lsm) == pytest.approx(0.5 * np.abs(p - q).sum(), abs=1e-15)
+    assert math.isfinite(ldd.kl_divergence(l, lsm))
+    # only the deployed row masks an entry the reference gives mass: infinite divergence, finite TV
+    assert ldd.kl_divergence(lm, ls) == math.inf and entropy(ldd.softmax(ls), ldd.softmax(lm)) == math.inf
+    assert 0.0 < ldd.tv_distance(lm, ls) <= 1.0
+    # two-entry closed form with a third, masked entry
+    a, b = 1.5, -0.25
+    assert ldd.tv_distance([a, 0.0, -np.inf], [b, 0.0, -np.inf]) == pytest.approx(abs(sigmoid(a) - sigmoid(b)), abs=1e-15)
+    assert ldd.kl_divergence([a, -np.inf, 0.0], [b, -np.inf, 0.0]) == pytest.approx(bernoulli_kl(sigmoid(b), sigmoid(a)), abs=1e-14)
+    # no finite entry: no distribution
+    dead = np.full(5, -np.inf)
+    assert math.isnan(ldd.tv_distance(dead, l[:5])) and math.isnan(ldd.kl_divergence(l[:5], dead))
+
+
 # ------------------------------------------------------------------ tail statistic
 
 
@@ -87,6 +118,18 @@ def test_tail_fraction_and_flags():
     assert p.tolist() == [1 / 3, 3 / 5]
     assert ldd.flag_requests(d, offsets, 0.1, 0.5).tolist() == [False, True]
     assert ldd.flag_requests(d, offsets, 0.1, 0.6).tolist() == [False, False]   # strict in t2 as well
+
+
+def test_tail_fraction_counts_what_is_not_known_to_be_below():
+    """NaN (a malformed index set, a row without a distribution) and +inf count as exceeding t1; for
+    ordinary numbers the rule is the strict comparison."""
+    d = np.array([0.05, np.nan, 0.1, np.inf, 0.2, np.nan])
+    assert ldd.tail_fraction(d, 0.1) == 4 / 6
+    assert ldd.tail_fraction(np.array([np.nan]), 1e9) == 1.0
+    assert ldd.flag_requests(d, [0, 3, 6], 0.1, 0.5).tolist() == [False, True]
+    rng = np.random.default_rng(12)
+    x = rng.uniform(0, 1, 1000)
+    assert ldd.tail_fraction(x, 0.4) == float((x > 0.4).sum()) / 1000
 
 
 # ------------------------------------------------------------------ Top-K distance
@@ -129,6 +172,30 @@ def test_topk_distance_matches_every_threshold_evaluation():
         l = np.round(rng.normal(0, 2, n), 1 if trial % 2 else 6)   # rounded values give ties
         I = rng.choice(n, size=k, replace=False)
         assert ldd.topk_distance(l, I) == pytest.approx(ldd.topk_distance_all_thresholds(l, I), abs=1e-12)
+
+
+def test_topk_distance_with_masked_entries():
+    """-inf entries outside I cost nothing (the distance is that of the row without them); a masked
+    member of I cannot be raised to any finite threshold."""
+    rng = np.random.default_rng(13)
+    for trial in range(30):
+        n = int(rng.integers(6, 50))
+        k = int(rng.integers(1, 5))
+        l = np.round(rng.normal(0, 2, n), 1 if trial % 2 else 6)
+        I = rng.choice(n, size=k, replace=False)
+        inside = np.zeros(n, dtype=bool); inside[I] = True
+        mask = (rng.random(n) < 0.4) & ~inside
+        lm = np.where(mask, -np.inf, l)
+        keep = np.flatnonzero(~mask)
+        I_kept = [int(np.flatnonzero(keep == i)[0]) for i in I]
+        want = ldd.topk_distance(l[keep], I_kept)
+        assert ldd.topk_distance(lm, I) == pytest.approx(want, abs=1e-12)
+        assert ldd.topk_distance_all_thresholds(lm, I) == pytest.approx(want, abs=1e-12)
+        lm2 = lm.copy(); lm2[I[0]] = -np.inf
+        assert ldd.topk_distance(lm2, I) == math.inf and ldd.topk_distance_all_thresholds(lm2, I) == math.inf
+    assert ldd.topk_distance(np.full(4, -np.inf), [1]) == math.inf
+    # a masked entry is a valid non-member: the true top-K of the finite part still costs nothing
+    assert ldd.topk_distance([3.0, -np.inf, 2.0, 1.0], [0, 2]) == 0.0
 
 
 def test_topk_distance_is_the_l1_minimum_linear_programme():

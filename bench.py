@@ -49,7 +49,9 @@ BATCH_ID0 = 1 << 40            # ids of the batched proofs (--batched), clear of
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=30)
+    ap.add_argument("--steps", type=int, default=100,
+                    help="timed steps (default 100: a step takes milliseconds, and the clock sampler needs a region "
+                         "of a good fraction of a second)")
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="decoder", choices=sorted(WORKLOADS),
@@ -114,17 +116,58 @@ def make_problems(config, seed, layers, tokens, device):
 
 
 class ClockSampler:
-    """Samples SM clock and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+    """Samples SM clock and throttle reasons of one GPU while the timed region runs: through NVML
+    every 5 ms where the bindings load (read-only queries), else with nvidia-smi every 100 ms."""
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
               "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+    # NVML's clocks-event-reason bits
+    REASON_BITS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown", 0x4: "sw_power_cap"}
 
     def __init__(self, index: int):
         self.index = index
         self.proc = None
         self.lines = []
+        self.nvml = None
+        self.samples = []            # (time, sm MHz, max MHz, watts, reason bits)
+        self.stop_flag = False
+
+    def _nvml_loop(self):
+        n, h = self.nvml
+        while not self.stop_flag:
+            try:
+                sm = n.nvmlDeviceGetClockInfo(h, n.NVML_CLOCK_SM)
+                try:
+                    bits = n.nvmlDeviceGetCurrentClocksEventReasons(h)
+                except AttributeError:
+                    bits = n.nvmlDeviceGetCurrentClocksThrottleReasons(h)
+                watts = n.nvmlDeviceGetPowerUsage(h) / 1000.0
+                self.samples.append((time.time(), float(sm), self.nvml_max, watts, int(bits)))
+            except Exception:
+                pass
+            time.sleep(0.005)
 
     def start(self):
+        try:
+            import pynvml as n
+            n.nvmlInit()
+            uuid = torch.cuda.get_device_properties(torch.cuda.current_device()).uuid
+            h = None
+            for i in range(n.nvmlDeviceGetCount()):
+                hi = n.nvmlDeviceGetHandleByIndex(i)
+                u = n.nvmlDeviceGetUUID(hi)
+                u = u.decode() if isinstance(u, bytes) else u
+                if str(uuid) in u:
+                    h = hi
+            if h is None:
+                h = n.nvmlDeviceGetHandleByIndex(self.index)
+            self.nvml_max = float(n.nvmlDeviceGetMaxClockInfo(h, n.NVML_CLOCK_SM))
+            self.nvml = (n, h)
+            self.thread = threading.Thread(target=self._nvml_loop, daemon=True)
+            self.thread.start()
+            return
+        except Exception:
+            self.nvml = None
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
@@ -139,6 +182,20 @@ class ClockSampler:
             self.lines.append((time.time(), line.strip()))
 
     def stop(self, t0: float, t1: float):
+        if self.nvml is not None:
+            self.stop_flag = True
+            self.thread.join(timeout=1)
+            rows = [r for r in self.samples if t0 <= r[0] <= t1] or self.samples[-3:]
+            if not rows:
+                return None
+            sm = sorted(r[1] for r in rows)
+            reasons = set()
+            for r in rows:
+                for bit, name in self.REASON_BITS.items():
+                    if r[4] & bit:
+                        reasons.add(name)
+            return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": rows[0][2], "power_w_max": max(r[3] for r in rows),
+                    "samples": len(rows), "reasons": sorted(reasons), "source": "nvml, 5 ms period"}
         if self.proc is None:
             return None
         time.sleep(0.15)
@@ -165,7 +222,7 @@ class ClockSampler:
             return None
         sm.sort()
         return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": max(smax), "power_w_max": max(power),
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "samples": len(sm), "reasons": sorted(reasons), "source": "nvidia-smi, 100 ms period"}
 
 
 # ------------------------------------------------------------------------ oracle timing
@@ -184,6 +241,11 @@ def oracle_time_sample(sample, threads):
     with ThreadPoolExecutor(max_workers=threads) as ex:
         out = list(ex.map(one, sample))
     return time.perf_counter() - t0, out
+
+
+def oracle_build_line():
+    from oracle import imm_oracle
+    return "gcc " + " ".join(imm_oracle.BUILD_FLAGS) + " (plain C, single-threaded per proof, % on unsigned __int128)"
 
 
 def field_macs(shapes):
@@ -415,6 +477,8 @@ def run_ours(args):
         "roofline": {"kernel": "bytedot_kernel<int32 as bytes, POINT> (claim C~)", "bound": "hbm", "achieved": claim_gbs,
                      "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": claim_gbs / peak,
                      "frac_of_8tbs": claim_gbs / 8000.0,
+                     # achieved GB/s per sampled SM MHz: comparable across pods whose clocks differ
+                     "gbs_per_sm_mhz": (claim_gbs / clocks["sm_mhz"]) if clocks and clocks.get("sm_mhz") else None,
                      "traffic": (CLAIM_KERNEL_TRAFFIC_RATIO * claim_bytes) if CLAIM_KERNEL_TRAFFIC_RATIO else None},
         "gpu_launches": ((fsp.launches + com.launches) if (args.fs and args.batched) else (6 + com.launches) if args.fs
                          else 6 if (args.batched or args.verify) else 5) * calls_per_step * steps,
@@ -468,6 +532,7 @@ def run_ours(args):
         ok = all([int(v) & 0xFFFFFFFFFFFFFFFF for v in host_t[i, :len(w)]] == [int(x) for x in w]
                  for i, w in enumerate(want))
         out["cpu_baseline"] = {"value": field_macs(shapes[:nsample]) / secs, "unit": UNIT, "cores": threads,
+                               "nproc": os.cpu_count(), "compiler": oracle_build_line(),
                                "kind": "oracle", "seconds": secs,
                                "sample": f"the first {nsample} of the {len(problems)} proofs, "
                                          f"one proof per thread, same inputs as the GPU run",
@@ -567,6 +632,7 @@ def run_ldd(args):
         "roofline": {"kernel": "tv_kl_kernel (two logit rows read once from HBM, second pass from L2)", "bound": "hbm",
                      "achieved": tvkl_gbs, "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": tvkl_gbs / peak,
                      "frac_of_8tbs": tvkl_gbs / 8000.0,
+                     "gbs_per_sm_mhz": (tvkl_gbs / clocks["sm_mhz"]) if clocks and clocks.get("sm_mhz") else None,
                      "traffic": (LDD_TVKL_TRAFFIC_RATIO * bytes_tvkl) if LDD_TVKL_TRAFFIC_RATIO else None},
         "gpu_launches": 3 * steps,
         "clocks": clocks,
@@ -612,7 +678,8 @@ def run_ldd(args):
         ok = (max(abs(a - b) for a, b in zip(gtv, otv)) <= 2e-5 and
               all(abs(a - b) <= 2e-5 + 2e-4 * abs(b) for a, b in zip(gkl, okl)) and
               all(abs(a - b) <= 1e-9 * max(1.0, abs(b)) for a, b in zip(gd, odist)))
-        res["cpu_baseline"] = {"value": len(rows) / secs, "unit": "steps/s", "cores": 1, "kind": "oracle", "seconds": secs,
+        res["cpu_baseline"] = {"value": len(rows) / secs, "unit": "steps/s", "cores": 1, "nproc": os.cpu_count(),
+                               "kind": "oracle", "seconds": secs,
                                "sample": f"{len(rows)} of the {T} decision steps, evenly spaced, same inputs as the GPU run",
                                "gpu_matches_oracle_within_tolerance": ok}
         if not ok:
@@ -738,7 +805,8 @@ def run_commit(args):
         want = {i: commitment.commit(data[i], rs[i]) for i in pick}
         secs = time.perf_counter() - w0
         ok = all(bytes(digests[i]) == want[i] for i in pick)
-        res["cpu_baseline"] = {"value": total / secs, "unit": "B/s", "cores": 1, "kind": "oracle", "seconds": secs,
+        res["cpu_baseline"] = {"value": total / secs, "unit": "B/s", "cores": 1, "nproc": os.cpu_count(),
+                               "kind": "oracle", "seconds": secs,
                                "sample": f"{len(pick)} of the {len(msgs)} requests ({total} bytes), same inputs as the GPU run",
                                "gpu_matches_oracle": ok}
         if not ok:
@@ -831,7 +899,8 @@ def run_reference(args):
                    "layers": args.layers if args.config == "decoder" else None,
                    "tokens": args.tokens, "sampled": desc,
                    "note": None if tokens == args.tokens else "no CUDA device for input generation: token count reduced"},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": desc},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "nproc": os.cpu_count(),
+                         "compiler": oracle_build_line(), "kind": "oracle", "sample": desc},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
 

@@ -35,7 +35,14 @@
  *     also return IMM_REJECT).  Nothing throws or aborts across this boundary.
  *   - The caller owns every buffer.  The library allocates no device memory: scratch comes from
  *     a caller-provided device workspace whose size a query call returns.  Workspace and output
- *     pointers must be 16-byte aligned.
+ *     pointers must be 16-byte aligned.  What the library does keep, per process: two
+ *     non-blocking CUDA streams and three events per device, created by the first prove call on
+ *     that device whose batch is small enough to run its contractions side by side (see
+ *     imm_sumcheck_matmul_prove), the event ring of imm_profile_enable, and the 64 KiB device array
+ *     of imm_mle_eval_point_noalloc.
+ *   - One environment variable is read, on every prove / evaluation call: IMM_CONTRACT=alu selects
+ *     the integer-pipe contraction kernels instead of the tensor-core ones (same results; meant for
+ *     A/B measurements).  Anything else, or unset, is the default.
  *   - Pointers named d_* are DEVICE pointers, *_host are HOST pointers.
  *   - Device calls enqueue work on the given CUDA stream (a cudaStream_t passed as void*; NULL =
  *     the legacy default stream) and return without synchronising, unless stated otherwise.
@@ -70,7 +77,9 @@ enum {
     IMM_ERR_WORKSPACE = -4,      /* workspace smaller than the query call asks for         */
     IMM_ERR_NONCANONICAL = -5,   /* a field element >= p on input                          */
     IMM_ERR_CUDA = -6,           /* a CUDA runtime call failed (see imm_last_cuda_error)   */
-    IMM_ERR_LIMIT = -7           /* larger than the fixed capacity of a no-allocation call */
+    IMM_ERR_TIMEOUT = -7,        /* reserved: a bounded device-side wait ran out.  No kernel
+                                    of this library waits on a flag, so nothing returns it */
+    IMM_ERR_LIMIT = -8           /* beyond a fixed capacity stated with the call           */
 };
 enum { IMM_I8 = 0, IMM_I32 = 1 };
 enum { IMM_BIND_ROWS = 0, IMM_BIND_COLS = 1 };
@@ -451,8 +460,9 @@ int imm_sumcheck_verify_fs(const imm_fe* transcript_host, int nrounds, const uin
  * instead of a whole logit vector (appendix on the verification of Top-K).
  *
  * Logit rows are float32, row-major: step i occupies entries [i*ld, i*ld + n) of its matrix
- * (ld >= n).  Entries must be finite.  Rows that are 16-byte aligned (base pointer and ld*4) are
- * read with 128-bit loads, others element by element.  All pointers are DEVICE pointers; calls
+ * (ld >= n).  An entry may be -inf (a masked vocabulary entry: probability exactly 0); NaN and
+ * +inf entries are not inputs (the row's results are then NaN, unchecked).  Rows that are 16-byte
+ * aligned (base pointer and ld*4) are read with 128-bit loads, others element by element.  All pointers are DEVICE pointers; calls
  * enqueue on `stream` and do not synchronise; nothing is allocated.  The arithmetic is float32
  * per entry (exp2-based softmax) with the cross-thread sums in float64; the Top-K distance is
  * selected exactly and evaluated in float64.
@@ -464,7 +474,10 @@ int imm_sumcheck_verify_fs(const imm_fe* transcript_host, int nrounds, const uin
 /* tv[i] = 1/2 * sum_v |p_v - q_v| and kl[i] = sum_v q_v (log q_v - log p_v), where
  * p = softmax(logits row i) (the deployed execution) and q = softmax(ref_logits row i) (the
  * reference), temperature 1.  The paper names "KL divergence or TV distance" without fixing the
- * KL direction: the reference distribution comes first here.
+ * KL direction: the reference distribution comes first here.  Masked entries: 0 log 0 = 0, so an
+ * entry without reference mass adds nothing to kl; kl[i] = +inf when the reference gives mass to an
+ * entry the deployed row masks; a row with no finite entry has no distribution and gives
+ * tv[i] = kl[i] = NaN (which imm_ldd_tail_fraction counts as exceeding any threshold).
  * Errors: IMM_ERR_ARG (null pointer), IMM_ERR_SHAPE (n <= 0, ld < n, n or steps beyond the limits
  * above), IMM_ERR_ALIGN (pointers not aligned to their element size), IMM_ERR_CUDA. */
 int imm_ldd_tv_kl(const float* d_logits, const float* d_ref_logits, int64_t steps, int64_t n, int64_t ld,
@@ -473,7 +486,8 @@ int imm_ldd_tv_kl(const float* d_logits, const float* d_ref_logits, int64_t step
 /* dist[i] = min over rows l' whose K largest entries are exactly the index set I_i of
  * ||l' - l_i||_1, with l_i = ref_logits row i and I_i = d_topk[i*k .. i*k + k) (k distinct
  * indices in [0, n)).  It is 0 iff I_i is a valid top-K set of the row.  Computed as the minimum
- * over thresholds t of  sum_{j not in I} max(l_j - t, 0) + sum_{i in I} max(t - l_i, 0).
+ * over finite thresholds t of  sum_{j not in I} max(l_j - t, 0) + sum_{i in I} max(t - l_i, 0):
+ * a masked (-inf) entry outside I costs nothing, a masked member of I makes dist[i] = +inf.
  * status[i] = IMM_OK, IMM_ERR_ARG (an index out of range or repeated; dist[i] = NaN), or
  * IMM_ERR_LIMIT (after six refinements more than 256 entries of one 8192-entry slice still lie
  * above the bound on its K-th largest entry; dist[i] = NaN).
@@ -489,7 +503,10 @@ int imm_ldd_topk_distance(const float* d_ref_logits, int64_t steps, int64_t n, i
 /* Per-request tail statistic: request r owns the steps offsets[r] .. offsets[r+1]-1 of `dist`
  * (offsets: nrequests + 1 non-decreasing int64 values).  p[r] = (number of its steps with
  * dist > t1) / (number of its steps), 0 for an empty request; flag[r] = 1 if p[r] > t2 else 0
- * (d_flag may be null).  Both comparisons are strict, as the paper prints them. */
+ * (d_flag may be null).  Both comparisons are strict, as the paper prints them.  A step whose
+ * distance is NaN -- imm_ldd_topk_distance writes NaN for a malformed index set, imm_ldd_tv_kl for
+ * a row without a finite logit -- counts as exceeding t1: what is not known to be within the
+ * threshold never lowers p[r], so a server cannot escape the flag by committing garbage. */
 int imm_ldd_tail_fraction(const double* d_dist, const int64_t* d_offsets, int64_t nrequests, double t1, double t2,
                           double* d_p, int32_t* d_flag, void* stream);
 

@@ -21,6 +21,8 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "imm_oracle.c")
 _LIB = os.path.join(_HERE, "liboracle.so")
 
+BUILD_FLAGS = ["-O2", "-Wall", "-shared", "-fPIC"]        # how the oracle is compiled (reported beside its timings)
+
 _u64 = ctypes.c_uint64
 _i64 = ctypes.c_int64
 _vp = ctypes.c_void_p
@@ -30,7 +32,7 @@ def build(force: bool = False) -> str:
     """Compile ``imm_oracle.c`` with gcc into ``liboracle.so`` beside it (plain -O2)."""
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
         tmp = _LIB + f".tmp{os.getpid()}"
-        subprocess.check_call(["gcc", "-O2", "-Wall", "-shared", "-fPIC", "-o", tmp, _SRC])
+        subprocess.check_call(["gcc"] + BUILD_FLAGS + ["-o", tmp, _SRC])
         os.replace(tmp, _LIB)
     return _LIB
 

@@ -38,7 +38,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
            "-shared", "-Xcompiler", "-fPIC", "-cudart", "shared"]
     if verbose:
         cmd += ["-Xptxas", "-v"]
-    cmd += os.environ.get("IMM_NVCC_FLAGS", "").split()      # e.g. -DIMM_BYTEDOT_CHUNK_BYTES=8192
+    cmd += os.environ.get("IMM_NVCC_FLAGS", "").split()      # e.g. -DIMM_TUNING (tile-geometry overrides for sweeps)
     cmd += [os.path.join(CSRC, s) for s in SOURCES] + ["-o", tmp]
     subprocess.check_call(cmd)
     os.replace(tmp, LIB)

@@ -51,6 +51,9 @@ bool rows_vectorisable(const void* p, int64_t ld, int dtype)
     return ((uintptr_t)p % 16 == 0) && ((ld * (int64_t)elem_size(dtype)) % 16 == 0);
 }
 
+// Tile-geometry overrides for sweeps exist only in a library built with -DIMM_TUNING; the shipped
+// library reads one environment variable, IMM_CONTRACT (documented in imm.h).
+#ifdef IMM_TUNING
 int env_int(const char* name, int dflt)
 {
     const char* s = getenv(name);
@@ -58,6 +61,11 @@ int env_int(const char* name, int dflt)
     int v = atoi(s);
     return v > 0 ? v : dflt;
 }
+bool env_set(const char* name) { return getenv(name) != nullptr; }
+#else
+int env_int(const char*, int dflt) { return dflt; }
+bool env_set(const char*) { return false; }
+#endif
 
 // Columns per tile of each kernel family.
 int rowbind_cols(int dtype) { return ROWBIND_THREADS * (dtype == IMM_I8 ? 16 : 4); }
@@ -82,7 +90,7 @@ int pick_tile_rows(const std::vector<Shape>& mats, int cols_per_tile, const char
         int v = forced < 32 ? 32 : forced > MAX_TILE_ROWS ? MAX_TILE_ROWS : forced;
         return v / 32 * 32;
     }
-    const int64_t target = (int64_t)148 * env_int("IMM_TILES_PER_SM", 24);
+    const int64_t target = (int64_t)sm_count() * env_int("IMM_TILES_PER_SM", 24);
     const int cand[] = {1024, 512, 256, 128, 64, 32};
     for (int c : cand) {
         if (c > max_rows) continue;
@@ -112,7 +120,7 @@ int64_t count_tiles(const std::vector<Shape>& mats, int rows, int width)
 Geom pick_geom(const std::vector<Shape>& mats, const int* rows, int nrows, const int* widths, int nwidths,
                int tiles_per_sm, const char* env_rows, const char* env_width)
 {
-    const int64_t target = (int64_t)148 * env_int("IMM_TILES_PER_SM", tiles_per_sm);
+    const int64_t target = (int64_t)sm_count() * env_int("IMM_TILES_PER_SM", tiles_per_sm);
     Geom best{rows[nrows - 1], widths[nwidths - 1]};          // candidates are listed largest first
     int64_t best_area = -1;
     for (int i = 0; i < nrows; i++)
@@ -801,7 +809,7 @@ static int prove_batch(const imm_matmul_desc* descs_host, int nproofs, uint64_t 
         const imm_matmul_desc& d = descs_host[i];
         batch_bytes += d.m * d.k + d.k * d.n + 4 * d.m * d.n;
     }
-    SideStreams* ss = (batch_bytes < FORK_BELOW_BYTES && !getenv("IMM_NO_FORK")) ? side_streams() : nullptr;
+    SideStreams* ss = (batch_bytes < FORK_BELOW_BYTES && !env_set("IMM_NO_FORK")) ? side_streams() : nullptr;
     cudaStream_t st_a = ss ? ss->s[0] : st, st_b = ss ? ss->s[1] : st;
     // Host threads proving on different streams share the side streams and their events: one call
     // at a time enqueues its fork ... join (a wait refers to the record that precedes it, so a later

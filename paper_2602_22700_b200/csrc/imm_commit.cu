@@ -22,6 +22,7 @@
 #include <vector>
 
 #include "../../include/imm.h"
+#include "imm_kernels.h"
 #include "sha256.cuh"
 
 namespace imm_hash {
@@ -32,12 +33,12 @@ constexpr int LEAF = IMM_COMMIT_LEAF;         // bytes per leaf
 // fullest SM in the last, partial wave) units; larger blocks run a few per cent faster per warp
 // (measured on 4 GiB: 128 threads 852 GB/s, 256 881, 512 900) but leave a coarser tail.  The
 // candidate with the lowest estimate is taken.
-constexpr int SM_COUNT = 148;
 struct LeafChoice { int threads, blocks_per_sm; double cost; };    // blocks per SM as the registers allow
 constexpr LeafChoice LEAF_CHOICES[3] = {{128, 9, 1.055}, {256, 4, 1.023}, {512, 2, 1.0}};
 
 inline int pick_leaf_threads(const std::vector<uint64_t>& leaves)
 {
+    const int SM_COUNT = imm::sm_count();
     int best = LEAF_CHOICES[0].threads;
     double best_t = -1;
     for (const LeafChoice& c : LEAF_CHOICES) {

@@ -1131,6 +1131,24 @@ expected_kernel(const ProofDev* proofs, const ExpectDev* ex, imm_fe* expected, i
 // launch wrappers
 // ------------------------------------------------------------------------------------------
 
+// Streaming multiprocessors of the current device, looked up once per device; 148 (a B200) where no
+// device answers, so that the host-side planning calls still work without one.
+int sm_count()
+{
+    static int cached[64];
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { (void)cudaGetLastError(); return 148; }
+    if (cached[dev] == 0) {
+        int v = 0;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) {
+            (void)cudaGetLastError();
+            return 148;
+        }
+        cached[dev] = v;
+    }
+    return cached[dev];
+}
+
 cudaError_t launch_fs_batched_rounds(const ProofDev* d_proofs, const FsProof* d_fs, const FsBatch& fb, imm_fe* transcript,
                                      int32_t* status, cudaStream_t st)
 {
@@ -1171,7 +1189,7 @@ cudaError_t launch_field_binop(int op, const imm_fe* x, const imm_fe* y, imm_fe*
 {
     if (n <= 0) return cudaSuccess;
     int64_t blocks = (n + 255) / 256;
-    if (blocks > 148 * 16) blocks = 148 * 16;
+    if (blocks > sm_count() * 16) blocks = sm_count() * 16;
     field_binop_kernel<<<(unsigned)blocks, 256, 0, st>>>(op, x, y, out, n);
     return cudaGetLastError();
 }
@@ -1304,7 +1322,7 @@ cudaError_t launch_sumcheck(const ProofDev* d_proofs, int nproofs, uint64_t seed
     // of the 2^b entries of both tables).
     int nc = 1;
     if (max_b > SC_SOLO_VARS) {
-        while (2 * nc <= SC_PORTABLE_CLUSTER && (int64_t)2 * nc * nproofs <= 2 * 148) nc *= 2;
+        while (2 * nc <= SC_PORTABLE_CLUSTER && (int64_t)2 * nc * nproofs <= 2 * sm_count()) nc *= 2;
         if (cluster == 1 || cluster == 2 || cluster == 4 || cluster == 8) nc = cluster;     // caller's choice
         while (nc < SUMCHECK_MAX_CLUSTER && (((int64_t)1 << max_b) / nc) > SC_MAX_CAP) nc *= 2;
     }

@@ -7,6 +7,9 @@
 
 namespace imm {
 
+// streaming multiprocessors of the current device (cached per device; 148 when no device answers)
+int sm_count();
+
 cudaError_t launch_field_binop(int op, const imm_fe* x, const imm_fe* y, imm_fe* out, int64_t n,
                                cudaStream_t st);
 cudaError_t launch_eq_direct(const EqDirect& r, int nvars, imm_fe* out, cudaStream_t st);

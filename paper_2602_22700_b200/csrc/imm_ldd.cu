@@ -32,6 +32,10 @@ constexpr int COLLECT_CAP = 256;              // entries above the bound a block
 constexpr int MAX_REFINE = 6;
 constexpr float LOG2E = 1.4426950408889634f;
 constexpr float NEG_INF = -INFINITY;
+// Running maxima start at the lowest finite float, not at -inf: a masked logit (-inf, probability
+// 0) then always meets a finite maximum, so (x - max) is -inf and its exponential 0, never the
+// NaN of (-inf) - (-inf).
+constexpr float EMPTY_MAX = -3.402823466e+38f;
 
 __device__ __forceinline__ float ex2(float x)
 {
@@ -72,7 +76,7 @@ __device__ __forceinline__ MaxSum ms_warp(MaxSum a)
     float m = a.m;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
-    float s = a.m == NEG_INF ? 0.f : a.s * ex2((a.m - m) * LOG2E);          // (an empty lane contributes nothing)
+    float s = a.s * ex2((a.m - m) * LOG2E);                // (an empty lane holds sum 0 and contributes nothing)
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
     return MaxSum{m, s};
@@ -116,7 +120,7 @@ tv_kl_kernel(const float* __restrict__ logits, const float* __restrict__ ref, in
     int64_t s0, s1;
     slice_bounds(n, nc, c, s0, s1);
 
-    MaxSum ap{NEG_INF, 0.f}, aq{NEG_INF, 0.f};
+    MaxSum ap{EMPTY_MAX, 0.f}, aq{EMPTY_MAX, 0.f};
     for (int64_t i = s0 + 4 * tid; i < s1; i += 4 * NT) {
         if (VEC && i + 4 <= s1) {
             const float4 a = ld4(x + i), b = ld4(y + i);
@@ -130,15 +134,15 @@ tv_kl_kernel(const float* __restrict__ logits, const float* __restrict__ ref, in
     if (lane == 0) { sh.warp_p[warp] = ap; sh.warp_q[warp] = aq; }
     __syncthreads();
     if (warp == 0) {
-        MaxSum p = lane < NW ? sh.warp_p[lane] : MaxSum{NEG_INF, 0.f};
-        MaxSum q = lane < NW ? sh.warp_q[lane] : MaxSum{NEG_INF, 0.f};
+        MaxSum p = lane < NW ? sh.warp_p[lane] : MaxSum{EMPTY_MAX, 0.f};
+        MaxSum q = lane < NW ? sh.warp_q[lane] : MaxSum{EMPTY_MAX, 0.f};
         p = ms_warp(p); q = ms_warp(q);
         if (lane == 0) { sh.pub_p = p; sh.pub_q = q; }
     }
     cluster.sync();                                        // every block's slice result is published
     if (warp == 0) {
-        MaxSum p = lane < nc ? *cluster.map_shared_rank(&sh.pub_p, lane) : MaxSum{NEG_INF, 0.f};
-        MaxSum q = lane < nc ? *cluster.map_shared_rank(&sh.pub_q, lane) : MaxSum{NEG_INF, 0.f};
+        MaxSum p = lane < nc ? *cluster.map_shared_rank(&sh.pub_p, lane) : MaxSum{EMPTY_MAX, 0.f};
+        MaxSum q = lane < nc ? *cluster.map_shared_rank(&sh.pub_q, lane) : MaxSum{EMPTY_MAX, 0.f};
         p = ms_warp(p); q = ms_warp(q);
         if (lane == 0) { sh.max_p = p.m; sh.max_q = q.m; sh.l2s_p = log2f(p.s); sh.l2s_q = log2f(q.s); }
     }
@@ -165,7 +169,9 @@ tv_kl_kernel(const float* __restrict__ logits, const float* __restrict__ ref, in
                 const float xr = xs[e] - mp, yr = ys[e] - mq;
                 const float p = ex2(fmaf(xr, LOG2E, -lp)), q = ex2(fmaf(yr, LOG2E, -lq));
                 tv += fabsf(p - q);
-                kl = fmaf(q, yr - xr, kl);                   // q_v (log q_v - log p_v) without its constant part: below
+                // q_v (log q_v - log p_v) without its constant part (below); 0 log 0 = 0, so an entry
+                // without reference mass is skipped (its yr - xr may be -inf or NaN)
+                if (q > 0.f) kl = fmaf(q, yr - xr, kl);
             }
         }
     }
@@ -186,8 +192,10 @@ tv_kl_kernel(const float* __restrict__ logits, const float* __restrict__ ref, in
     if (c == 0 && tid == 0) {
         double a = 0.0, b = 0.0;
         for (int cc = 0; cc < nc; cc++) { a += sh.share_tv[cc]; b += sh.share_kl[cc]; }
-        tv_out[step] = 0.5 * a;
-        kl_out[step] = b - (double)dl;                     // sum_v q_v (log S_q - log S_p) = log S_q - log S_p: q sums to 1
+        // a row without a finite entry has sum 0 (log2 = -inf) and no distribution: both distances are NaN
+        const bool dead = !(lp > NEG_INF) || !(lq > NEG_INF);
+        tv_out[step] = dead ? (double)NAN : 0.5 * a;
+        kl_out[step] = dead ? (double)NAN : b - (double)dl;   // sum_v q_v (log S_q - log S_p) = log S_q - log S_p: q sums to 1
     }
 }
 
@@ -523,7 +531,7 @@ tv_kl_small_kernel(const float* __restrict__ logits, const float* __restrict__ r
             const float xr = xs[j] - mx, yr = ys[j] - my;
             const float p = ex2(fmaf(xr, LOG2E, -lp)), q = ex2(fmaf(yr, LOG2E, -lq));
             tv += fabsf(p - q);
-            kl = fmaf(q, (yr - xr) - dl, kl);
+            if (q > 0.f) kl = fmaf(q, (yr - xr) - dl, kl);       // 0 log 0 = 0
         }
     }
     double dtv = (double)tv, dkl = (double)kl;
@@ -532,7 +540,8 @@ tv_kl_small_kernel(const float* __restrict__ logits, const float* __restrict__ r
         dtv += __shfl_xor_sync(0xFFFFFFFFu, dtv, o);
         dkl += __shfl_xor_sync(0xFFFFFFFFu, dkl, o);
     }
-    if (lane == 0) { tv_out[step] = 0.5 * dtv; kl_out[step] = dkl; }
+    const bool dead = !(lp > NEG_INF) || !(lq > NEG_INF);      // a row without a finite entry: NaN
+    if (lane == 0) { tv_out[step] = dead ? (double)NAN : 0.5 * dtv; kl_out[step] = dead ? (double)NAN : dkl; }
 }
 
 // Rows of at most 256 entries: a group of LPR lanes per row (8 or 16 lanes, sixteen entries per
@@ -583,7 +592,7 @@ tv_kl_sub_kernel(const float* __restrict__ logits, const float* __restrict__ ref
             const float xr = xs[j] - mx, yr = ys[j] - my;
             const float p = ex2(fmaf(xr, LOG2E, -lp)), q = ex2(fmaf(yr, LOG2E, -lq));
             tv += fabsf(p - q);
-            kl = fmaf(q, (yr - xr) - dl, kl);
+            if (q > 0.f) kl = fmaf(q, (yr - xr) - dl, kl);       // 0 log 0 = 0
         }
     }
     double dtv = (double)tv, dkl = (double)kl;
@@ -592,7 +601,8 @@ tv_kl_sub_kernel(const float* __restrict__ logits, const float* __restrict__ ref
         dtv += __shfl_xor_sync(0xFFFFFFFFu, dtv, o);
         dkl += __shfl_xor_sync(0xFFFFFFFFu, dkl, o);
     }
-    if (live && gl == 0) { tv_out[step] = 0.5 * dtv; kl_out[step] = dkl; }
+    const bool dead = !(lp > NEG_INF) || !(lq > NEG_INF);      // a row without a finite entry: NaN
+    if (live && gl == 0) { tv_out[step] = dead ? (double)NAN : 0.5 * dtv; kl_out[step] = dead ? (double)NAN : dkl; }
 }
 
 // Top-K distance of a short row.  The K largest entries outside I are pulled out one at a time
@@ -759,6 +769,8 @@ topk_sub_kernel(const float* __restrict__ ref, int64_t steps, int n, int64_t ld,
 // per-request tail statistic
 // ------------------------------------------------------------------------------------------
 // p[r] = |{ steps of request r with distance > t1 }| / (steps of request r);  flag[r] = p[r] > t2.
+// A step counts unless its distance is known to be <= t1: a NaN distance (a malformed index set, a
+// row without a finite logit) counts as exceeding the threshold, so it can never lower p.
 
 __global__ void __launch_bounds__(256)
 tail_fraction_kernel(const double* __restrict__ dist, const int64_t* __restrict__ offsets, double t1, double t2,
@@ -768,7 +780,7 @@ tail_fraction_kernel(const double* __restrict__ dist, const int64_t* __restrict_
     const int64_t r = blockIdx.x;
     const int64_t b = offsets[r], e = offsets[r + 1];
     int cnt = 0;
-    for (int64_t i = b + threadIdx.x; i < e; i += blockDim.x) cnt += dist[i] > t1 ? 1 : 0;
+    for (int64_t i = b + threadIdx.x; i < e; i += blockDim.x) cnt += !(dist[i] <= t1) ? 1 : 0;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) cnt += __shfl_xor_sync(0xFFFFFFFFu, cnt, o);
     if ((threadIdx.x & 31) == 0) warp_cnt[threadIdx.x >> 5] = cnt;

@@ -15,11 +15,11 @@ import torch
 
 P = 0xFFFFFFFF00000001
 OK, REJECT = 0, 1
-ERR_ARG, ERR_SHAPE, ERR_ALIGN, ERR_WORKSPACE, ERR_NONCANONICAL, ERR_CUDA, ERR_LIMIT = -1, -2, -3, -4, -5, -6, -7
+ERR_ARG, ERR_SHAPE, ERR_ALIGN, ERR_WORKSPACE, ERR_NONCANONICAL, ERR_CUDA, ERR_TIMEOUT, ERR_LIMIT = -1, -2, -3, -4, -5, -6, -7, -8
 I8, I32 = 0, 1
 BIND_ROWS, BIND_COLS = 0, 1
 FIELD_ADD, FIELD_SUB, FIELD_MUL = 0, 1, 2
-ERRORS = {-7: "IMM_ERR_LIMIT", -1: "IMM_ERR_ARG", -2: "IMM_ERR_SHAPE", -3: "IMM_ERR_ALIGN", -4: "IMM_ERR_WORKSPACE",
+ERRORS = {-8: "IMM_ERR_LIMIT", -7: "IMM_ERR_TIMEOUT", -1: "IMM_ERR_ARG", -2: "IMM_ERR_SHAPE", -3: "IMM_ERR_ALIGN", -4: "IMM_ERR_WORKSPACE",
           -5: "IMM_ERR_NONCANONICAL", -6: "IMM_ERR_CUDA"}
 
 _HERE = os.path.dirname(os.path.abspath(__file__))

@@ -45,8 +45,14 @@ def check_tv_kl(imm, ldd, x, y):
     xs, ys = x.cpu().numpy(), y.cpu().numpy()
     for i in range(xs.shape[0]):
         want_tv, want_kl = ldd.tv_distance(xs[i], ys[i]), ldd.kl_divergence(xs[i], ys[i])
+        if math.isnan(want_tv):                               # a row without a finite entry
+            assert math.isnan(tv[i]) and math.isnan(kl[i]) and math.isnan(want_kl), (i, tv[i], kl[i])
+            continue
         assert abs(tv[i] - want_tv) <= TV_TOL, (i, tv[i], want_tv)
-        assert abs(kl[i] - want_kl) <= KL_ABS + KL_REL * abs(want_kl), (i, kl[i], want_kl)
+        if math.isinf(want_kl):                               # reference mass on an entry the deployed row masks
+            assert kl[i] == want_kl, (i, kl[i], want_kl)
+        else:
+            assert abs(kl[i] - want_kl) <= KL_ABS + KL_REL * abs(want_kl), (i, kl[i], want_kl)
 
 
 @pytest.mark.parametrize("steps,n", [(7, 1), (5, 3), (9, 100), (19, 64), (9, 128), (5, 256), (4, 1000), (3, 1024), (3, 1025),
@@ -71,6 +77,34 @@ def test_tv_kl_identical_rows_and_far_rows(imm, ldd, synth):
     far[:, 123] += 60.0                                   # all mass on one entry
     check_tv_kl(imm, ldd, far, ref)
     check_tv_kl(imm, ldd, ref + 1000.0, ref - 500.0)      # shifts cancel: large magnitudes must not overflow
+
+
+@pytest.mark.parametrize("n", [40, 200, 700, 5000, 40003, 128256])
+def test_tv_kl_masked_logits(imm, ldd, synth, n):
+    """-inf entries (masked vocabulary): one, many, a whole slice, all but one, and all of a row; in
+    both rows, in the reference only (those entries add nothing to KL) and in the deployed row only
+    (KL = +inf when the reference keeps mass there).  Every kernel family by row length."""
+    steps = 8
+    ref = synth.reference_logits(21, steps, n, device="cuda")
+    dep = synth.deployed_logits(ref, 21, synth.NOISE_QUANTISED)
+    g = torch.Generator().manual_seed(n)
+    many = (torch.rand(n, generator=g) < 0.5).cuda()
+    one = torch.zeros(n, dtype=torch.bool, device="cuda"); one[n // 3] = True
+    head = torch.zeros(n, dtype=torch.bool, device="cuda"); head[:min(n - 1, 20000)] = True     # whole slices of a long row
+    but_one = torch.ones(n, dtype=torch.bool, device="cuda"); but_one[n - 2] = False
+    everything = torch.ones(n, dtype=torch.bool, device="cuda")
+    masks = [one, many, head, but_one, everything, many, many, one]
+    both_r, both_d = ref.clone(), dep.clone()
+    for i in range(5):
+        both_r[i, masks[i]] = -math.inf
+        both_d[i, masks[i]] = -math.inf
+    both_r[5, masks[5]] = -math.inf                        # reference only
+    both_d[6, masks[6]] = -math.inf                        # deployed only: infinite divergence
+    both_d[7, :] = -math.inf                               # deployed row dead, reference alive
+    check_tv_kl(imm, ldd, both_d, both_r)
+    tv, kl = imm.ldd_tv_kl(both_d, both_r)
+    assert math.isnan(float(tv[4])) and math.isnan(float(kl[7])) and float(kl[6]) == math.inf
+    assert float(tv[3]) <= TV_TOL                           # one live entry on both sides: identical distributions
 
 
 def test_tv_kl_unaligned_rows_take_the_element_path(imm, ldd, synth):
@@ -160,6 +194,64 @@ def test_topk_distance_whole_row_inside_and_bad_indices(imm, ldd):
     good_and_bad = torch.tensor([[3, 0], [2, -1]], dtype=torch.int32, device="cuda")
     dist, status = imm.ldd_topk_distance(ref, good_and_bad)
     assert status.cpu().tolist() == [0, imm.ERR_ARG] and float(dist[0]) == 0.0
+
+
+@pytest.mark.parametrize("n,k", [(100, 4), (256, 8), (1000, 20), (40003, 20), (128256, 20)])
+def test_topk_distance_masked_logits(imm, ldd, synth, n, k):
+    """Masked entries outside I cost nothing; a masked member of I makes the distance +inf; a row
+    with no finite entry likewise.  Checked against the oracle on every kernel family."""
+    steps = 6
+    ref = synth.reference_logits(22, steps, n, device="cuda")
+    dep = synth.deployed_logits(ref, 22, synth.NOISE_QUANTISED)
+    top = torch.topk(dep, k, dim=1).indices.to(torch.int32).contiguous()
+    g = torch.Generator().manual_seed(n + k)
+    for i in range(steps):
+        mask = (torch.rand(n, generator=g) < (0.5 if i < 3 else 0.95)).cuda()
+        mask[top[i].long()] = False
+        ref[i, mask] = -math.inf
+    ref[2, :min(n, 9000)] = -math.inf                      # a whole slice of a long row, members of I included or not
+    ref[4, int(top[4, 1])] = -math.inf                     # a masked member of I
+    ref[5, :] = -math.inf                                  # nothing finite
+    dist, status = imm.ldd_topk_distance(ref, top)
+    dist, status = dist.cpu().numpy(), status.cpu().numpy()
+    ys, idx = ref.cpu().numpy(), top.cpu().numpy()
+    assert (status == 0).all()
+    for i in range(steps):
+        want = ldd.topk_distance(ys[i], idx[i])
+        if math.isinf(want):
+            assert dist[i] == want, (i, dist[i])
+        else:
+            assert abs(dist[i] - want) <= 1e-9 * max(1.0, abs(want)), (i, dist[i], want)
+    assert dist[4] == math.inf and dist[5] == math.inf
+
+
+def test_malformed_index_sets_cannot_lower_the_tail_statistic(imm, ldd):
+    """A committed index set that is repeated or out of range gives a NaN distance, and the tail
+    statistic counts NaN as exceeding t1 -- the oracle's rule -- so garbage never lowers p(t1)."""
+    rng = np.random.default_rng(23)
+    steps, n, k = 40, 300, 5
+    ref = torch.from_numpy(rng.normal(0, 2, (steps, n)).astype(np.float32)).cuda()
+    top = torch.topk(ref, k, dim=1).indices.to(torch.int32).contiguous()           # valid sets: distance 0
+    top[3, 1] = top[3, 0]                                                            # repeated
+    top[17, 2] = n + 5                                                               # out of range
+    top[18, 0] = -1
+    top[30] = torch.topk(-ref[30], k).indices.to(torch.int32)                        # a wrong but well-formed set
+    dist, status = imm.ldd_topk_distance(ref, top)
+    assert status.cpu().tolist().count(imm.ERR_ARG) == 3
+    d = dist.cpu().numpy()
+    assert np.isnan(d[[3, 17, 18]]).all() and d[30] > 0 and np.nansum(d) == d[30]
+    offsets = np.array([0, 10, 20, 40], dtype=np.int64)
+    t1, t2 = 0.5, 0.09
+    p, flag = imm.ldd_tail_fraction(dist, torch.from_numpy(offsets).cuda(), t1, t2)
+    want = ldd.request_tail_fractions(d, offsets, t1)
+    assert want.tolist() == [1 / 10, 2 / 10, 1 / 20]
+    assert (p.cpu().numpy() == want).all()
+    assert flag.cpu().tolist() == [1, 1, 0] and ldd.flag_requests(d, offsets, t1, t2).tolist() == [True, True, False]
+    # a NaN from the TV/KL call (a dead row) counts the same way
+    x = ref.clone(); x[7, :] = -math.inf
+    tv, _ = imm.ldd_tv_kl(x, ref)
+    p2, _ = imm.ldd_tail_fraction(tv, torch.from_numpy(offsets).cuda(), 0.9, 0.0)
+    assert p2.cpu().tolist() == [1 / 10, 0.0, 0.0]
 
 
 def test_tail_fraction_is_exact(imm, ldd, synth):

@@ -8,9 +8,11 @@ shares no code with the CUDA library.
 * the logit distance distribution (TV / KL distances, Top-K distance, the per-request tail
   statistic): ``oracle.ldd`` (plain numpy in float64); its header lists the readings and the pins;
 * the hash commitment (SHA-256 Merkle tree, ``hashlib`` as the library step): ``oracle.commitment``;
-* the non-interactive (Fiat-Shamir) form of the matmul proof: ``oracle.fs``.
+* the non-interactive (Fiat-Shamir) form of the matmul proof: ``oracle.fs``;
+* the element-wise links between proved products (requantisation): ``oracle.glue``.
 """
 from . import commit_oracle as commitment  # noqa: F401
 from . import fs_oracle as fs  # noqa: F401
+from . import glue_oracle as glue  # noqa: F401
 from . import ldd_oracle as ldd  # noqa: F401
 from .imm_oracle import *  # noqa: F401,F403

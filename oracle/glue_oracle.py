@@ -1,0 +1,48 @@
+"""CPU oracle for the element-wise links between proved matrix products -- TEST INFRASTRUCTURE ONLY.
+
+Plain numpy on 64-bit integers, one definition per function, no blocking.  Only the tests, the smoke
+check and the benchmark's CPU-baseline leg may import it; it shares no code with the CUDA library.
+
+What it follows.  The reference execution F_theta* is a chain of attention, MLP and normalisation
+steps (Section 4.1), and the proof must establish that these continuous transformations were
+computed with the committed model (Section 5.2, item 2).  The sumcheck proofs cover the matrix
+products one by one; what ties one product's output to the next product's input is an element-wise
+map.  In an int8-quantised execution that map is the requantisation of the int32 accumulators
+
+    H[i, j] = clamp( floor( (C[i, j] + rnd) / 2^shift ), lo, hi )
+
+(round-half-up division by a power of two when rnd = 2^(shift-1), then saturation), and a verifier
+that holds the opened tensors checks it by recomputing it: the link holds iff no entry of H differs.
+
+Readings (the paper names the parts of F_theta* and nothing about their arithmetic): the division
+rounds toward minus infinity (floor), which is what an arithmetic right shift of a two's-complement
+integer computes; 0 <= rnd < 2^shift; the check reports how many entries differ and the row-major
+position i*cols + j of the first one (-1 if none), so that a failing audit can name the entry.
+
+Pins (tests/test_oracle_glue.py): Python big-integer floor division and exact fractions
+(round-half-up of C / 2^shift) on hand-written values at the rounding boundaries, both signs, the
+clamp edges and the int32 extremes; shift = 0; idempotence under the clamp; monotonicity; the input
+generator's own hidden activations; counts and first positions of planted differences.  No function
+here is "parity unpinned".
+"""
+from __future__ import annotations
+
+import numpy as np
+
+
+def requantize(C, shift: int, rnd: int, lo: int, hi: int) -> np.ndarray:
+    """H = clamp(floor((C + rnd) / 2^shift), lo, hi) as int8; C holds int32 values."""
+    assert 0 <= shift <= 30 and 0 <= rnd < (1 << shift) or (shift == 0 and rnd == 0)
+    assert -128 <= lo <= hi <= 127
+    t = np.asarray(C, dtype=np.int64) + int(rnd)
+    q = np.floor_divide(t, np.int64(1) << np.int64(shift))
+    return np.clip(q, lo, hi).astype(np.int8)
+
+
+def requant_check(C, H, shift: int, rnd: int, lo: int, hi: int):
+    """(number of entries where H differs from requantize(C), row-major index of the first or -1)."""
+    C = np.asarray(C)
+    H = np.asarray(H)
+    assert C.shape == H.shape
+    bad = np.flatnonzero((requantize(C, shift, rnd, lo, hi) != H.astype(np.int8)).reshape(-1))
+    return int(bad.size), (int(bad[0]) if bad.size else -1)

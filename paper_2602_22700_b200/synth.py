@@ -143,8 +143,9 @@ def exact_matmul_i32(A: torch.Tensor, B: torch.Tensor, row_chunk: int = 4096) ->
 
 
 def requantize_i8(C: torch.Tensor) -> torch.Tensor:
-    """int32 FFN hidden -> int8 input of the down projection: clamp((C + 256) >> 9, -127, 127)."""
-    return torch.clamp((C + 256) >> 9, -127, 127).to(torch.int8)
+    """int32 FFN hidden -> int8 input of the down projection: clamp((C + 256) >> 9, -127, 127), with the
+    sum taken without 32-bit wrap-around: (C >> 9) + (((C & 511) + 256) >> 9)."""
+    return torch.clamp((C >> 9) + (((C & 511) + 256) >> 9), -127, 127).to(torch.int8)
 
 
 # ---------------------------------------------------------------------------- workloads

@@ -2,7 +2,7 @@
 """Throughput of the sumcheck matmul prover on synthetic transformer-shaped layers.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
-                    [--config decoder|qkv|ffn|moe|attn|ldd|commit] [--batched] [--fs] [--verify]
+                    [--config decoder|qkv|ffn|moe|attn|ldd|commit|glue] [--batched] [--fs] [--verify]
                     [--layers L] [--tokens T] [--no-e2e] [--no-cpu-baseline]
 
 One step = one proving pass over the whole batch: eq tables, A~ / B~ partial evaluations, the
@@ -15,7 +15,8 @@ flush is needed between steps).  Rank 0 prints ONE JSON line.
 --fs makes a step commit to every matrix (SHA-256 trees) and prove non-interactively (with --batched: one
 non-interactive proof for the whole workload); --verify times
 the verifier's pass over the same matrices; --config ldd
-and --config commit time the logit distances and the response commitments (their own metrics).
+and --config commit time the logit distances and the response commitments, --config glue the
+requantisation link between the FFN products (their own metrics).
 
 --impl reference times the plain CPU oracle on the host cores, on a bounded sample of the same
 workload.  With N > 1 (launched by torch.distributed.run) every rank proves an independent
@@ -89,6 +90,8 @@ WORKLOADS = {
     "commit": (8192, "response commitments: {tokens} decision steps x vocabulary {vocab} (float32 logits) cut into "
                      "{tokens}/128 requests of uneven length, one SHA-256 tree commitment per request"),
     "ldd": (8192, "logit distance distribution: {tokens} decision steps x vocabulary {vocab} (float32), TV + KL + Top-{topk} distance + tail statistic"),
+    "glue": (8192, "requantisation link of the FFN pair: hidden activations {tokens} x 14336, int32 accumulators of the up "
+                   "projection against the int8 input of the down projection"),
 }
 L2_BYTES = 126 << 20
 
@@ -286,6 +289,7 @@ COMMIT_TRAFFIC_RATIO = (1.077891 + 0.018910) / 1.050673152                   # c
 # byte (ncu: 564.2 M warp instructions on that pipe for 1.0507 GB), so at 1965 MHz the pipe allows
 # 148 x 64 x 1.965e9 / 17.18 = 1083 GB/s.
 COMMIT_ALU_PEAK_GBS_AT_1965 = 1083.0
+GLUE_TRAFFIC_RATIO = None        # requant_check_kernel: (dram read + write) / (5 bytes per entry); None until captured
 CLAIM_KERNEL_TRAFFIC_RATIO = 239.64 / 234.881024  # bytedot_kernel<1,1,1>: (dram read + write) / (4 bytes per entry), small-case capture
 
 
@@ -689,6 +693,124 @@ def run_ldd(args):
     rep.close()
 
 
+# ------------------------------------------------------------------------ links between products
+
+
+def run_glue(args):
+    """One step = the element-wise check that the down projection's int8 input is the requantised int32
+    output of the up projection (every entry of a tokens x 14336 hidden matrix)."""
+    from paper_2602_22700_b200 import imm, synth
+    from paper_2602_22700_b200.replicas import Replicas
+    rank, local_rank, world = dist_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: there is no CPU path")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    rep = Replicas("nccl", dev)
+    imm.lib()
+    warmup, steps = max(args.warmup, 3), max(args.steps, 1)
+    T, d_model, d_ff = args.tokens, 4096, 14336
+    seed = rep.seed(SEED)
+    A = synth.gauss_i8(seed, synth.tid(0, synth.ROLE_ACT), T, d_model, synth.Q_SIGMA20, dev)
+    W = synth.gauss_i8(seed, synth.tid(0, synth.ROLE_W), d_model, d_ff, synth.Q_SIGMA8, dev)
+    C = synth.exact_matmul_i32(A, W)
+    H = synth.requantize_i8(C)
+    del A, W
+    nbytes = 5 * T * d_ff
+    out = torch.empty(2, dtype=torch.int64, device=dev)
+    barrier = rep.barrier
+    for _ in range(warmup):
+        imm.requant_check(C, H, out=out)
+    barrier()
+    sampler = ClockSampler(local_rank if "CUDA_VISIBLE_DEVICES" not in os.environ else
+                           int(os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local_rank]))
+    sampler.start()
+    time.sleep(0.25)
+    flush = nbytes < 2 * L2_BYTES
+    scrub = torch.empty(512 << 20, dtype=torch.uint8, device=dev) if flush else None
+    pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    t0 = time.time()
+    for a, b in pairs:
+        if flush:
+            scrub.fill_(1)
+        a.record()
+        imm.requant_check(C, H, out=out)
+        b.record()
+    barrier()
+    t1w = time.time()
+    clocks = sampler.stop(t0, t1w)
+    elapsed_ms = rep.max_over_ranks(sum(a.elapsed_time(b) for a, b in pairs))
+    ms_per_step = elapsed_ms / steps
+    got = [int(v) for v in out.cpu()]
+    if got != [0, -1]:
+        raise SystemExit(f"the honest link does not hold: {got}")
+    peak, peak_kind = measured_peaks()
+    gbs = nbytes / (ms_per_step * 1e-3) / 1e9
+    res = {
+        "metric": "checked entries/sec", "value": T * d_ff * world / (ms_per_step * 1e-3), "unit": "entries/s",
+        "n_gpus": world, "steps": steps, "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "i32", "data": "synthetic",
+        "config": {"workload": workload_name("glue", 0, T), "tokens": T, "input_bytes_per_gpu": nbytes,
+                   "map": "clamp((C + 256) >> 9, -127, 127)",
+                   "l2": ("L2 flushed between steps (512 MB overwritten outside the timed event pairs)" if flush else
+                          f"inputs ({nbytes / 2**30:.2f} GiB) exceed the 126 MB L2 several times over; no flush"),
+                   "parallelism": "1 GPU" if world == 1 else f"{world} independent replicas, no collective"},
+        "hbm_gbs_whole_step": gbs,
+        "roofline": {"kernel": "requant_check_kernel (4 bytes of C + 1 byte of H per entry, read once); timed as the whole "
+                               "imm_requant_check call (two 8-byte memsets + the kernel)", "bound": "hbm", "achieved": gbs,
+                     "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": gbs / peak, "frac_of_8tbs": gbs / 8000.0,
+                     "gbs_per_sm_mhz": (gbs / clocks["sm_mhz"]) if clocks and clocks.get("sm_mhz") else None,
+                     "traffic": (GLUE_TRAFFIC_RATIO * nbytes) if GLUE_TRAFFIC_RATIO else None},
+        "gpu_launches": steps,
+        "clocks": clocks,
+    }
+    e2e = None
+    if not args.no_e2e:
+        hC = torch.empty(C.shape, dtype=C.dtype, pin_memory=True).copy_(C)
+        hH = torch.empty(H.shape, dtype=H.dtype, pin_memory=True).copy_(H)
+        dC, dH = torch.empty_like(C), torch.empty_like(H)
+        hout = torch.empty(2, dtype=torch.int64, pin_memory=True)
+        torch.cuda.synchronize()
+
+        def e2e_pass():
+            dC.copy_(hC, non_blocking=True); dH.copy_(hH, non_blocking=True)
+            hout.copy_(imm.requant_check(dC, dH, out=out), non_blocking=True)
+            torch.cuda.synchronize()
+
+        e2e_pass()
+        barrier()
+        k2 = max(1, args.e2e_steps)
+        w0 = time.perf_counter()
+        for _ in range(k2):
+            e2e_pass()
+        e2e_s = rep.max_over_ranks((time.perf_counter() - w0) / k2)
+        e2e = {"value": T * d_ff * world / e2e_s, "unit": "entries/s", "ms_per_step": e2e_s * 1e3, "steps": k2,
+               "h2d_bytes_per_step": nbytes, "d2h_bytes_per_step": 16,
+               "matches_device_path": [int(v) for v in hout] == got}
+        del hC, hH, dC, dH
+    res["e2e"] = e2e
+    if not args.no_cpu_baseline and world == 1:
+        from oracle import glue
+        rows = min(T, 512)
+        Ch, Hh = C[:rows].cpu().numpy(), H[:rows].cpu().numpy()
+        Hh[rows // 2, 77] ^= 1                               # one planted difference, found by both sides
+        Hd = H[:rows].clone()
+        Hd[rows // 2, 77] ^= 1
+        w0 = time.perf_counter()
+        want = glue.requant_check(Ch, Hh, 9, 256, -127, 127)
+        secs = time.perf_counter() - w0
+        ok = [int(v) for v in imm.requant_check(C[:rows], Hd).cpu()] == list(want) and want[0] == 1
+        res["cpu_baseline"] = {"value": rows * d_ff / secs, "unit": "entries/s", "cores": 1, "nproc": os.cpu_count(),
+                               "kind": "oracle", "seconds": secs,
+                               "sample": f"the first {rows} of the {T} rows, one planted difference, same inputs as the GPU run",
+                               "gpu_matches_oracle": ok}
+        if not ok:
+            raise SystemExit("GPU link check differs from the oracle")
+    if rank == 0:
+        print(json.dumps(res))
+    rep.close()
+
+
 # ------------------------------------------------------------------------ hash commitments
 
 
@@ -873,6 +995,30 @@ def run_reference(args):
             "e2e": {"value": len(data) / per, "unit": "B/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         }))
         return
+    if args.config == "glue":
+        from oracle import glue
+        rows = 512
+        rng = np.random.default_rng(SEED)
+        Ch = rng.integers(-70000, 70000, size=(rows, 14336)).astype(np.int32)
+        Hh = glue.requantize(Ch, 9, 256, -127, 127)
+        warmup, steps = max(args.warmup, 1), max(args.steps, 1)
+        for _ in range(warmup):
+            glue.requant_check(Ch[:32], Hh[:32], 9, 256, -127, 127)
+        w0 = time.perf_counter()
+        for _ in range(steps):
+            glue.requant_check(Ch, Hh, 9, 256, -127, 127)
+        per = (time.perf_counter() - w0) / steps
+        desc = f"{rows} rows of 14336 entries per step, one thread"
+        print(json.dumps({
+            "impl": "reference", "metric": "checked entries/sec", "value": rows * 14336 / per, "unit": "entries/s",
+            "n_gpus": world, "steps": steps, "warmup": warmup, "ms_per_step": per * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "i64", "data": "synthetic",
+            "config": {"workload": workload_name("glue", 0, args.tokens), "tokens": args.tokens, "sampled": desc},
+            "cpu_baseline": {"value": rows * 14336 / per, "unit": "entries/s", "cores": 1, "nproc": os.cpu_count(),
+                             "kind": "oracle", "sample": desc},
+            "e2e": {"value": rows * 14336 / per, "unit": "entries/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        }))
+        return
     layers = min(args.layers, 2)
     tokens = args.tokens if device == "cuda" else min(args.tokens, 256)
     problems = make_problems(args.config, SEED, layers, tokens, device)[:8]
@@ -915,6 +1061,8 @@ def main():
         run_ldd(args)
     elif args.config == "commit":
         run_commit(args)
+    elif args.config == "glue":
+        run_glue(args)
     else:
         run_ours(args)
 

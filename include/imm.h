@@ -3,8 +3,9 @@
  * over the Goldilocks field p = 2^64 - 2^32 + 1, and of what the same audit needs around it.
  * Sections, in this order: field and eq-table helpers; multilinear evaluations; the interactive
  * proof (prover, phase timing, host-buffer variant, host verifier); the batched proof; hash
- * commitments; the verifier's pass over the opened matrices; the non-interactive (Fiat-Shamir)
- * proof, per product and per batch; the logit distance statistics.
+ * commitments; the verifier's pass over the opened matrices; the element-wise links between
+ * products; the non-interactive (Fiat-Shamir) proof, per product and per batch; the logit
+ * distance statistics.
  *
  * Background.  The audited-inference protocol this library serves has the server prove, for an
  * audited request, that the "continuous transformations" of the reference model -- its
@@ -369,6 +370,36 @@ size_t imm_sumcheck_expected_workspace(const imm_matmul_desc* descs_host, int np
 int imm_sumcheck_expected(const imm_matmul_desc* descs_host, int nproofs, uint64_t seed, const uint64_t* batch_id,
                           const imm_fe* points_host, imm_fe* d_expected, int32_t* d_status,
                           void* d_ws, size_t ws_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Links between products
+ * ---------------------------------------------------------------------------------------------
+ * The reference execution is a chain of attention, MLP and normalisation steps (Section 4.1), and
+ * the proof must cover the whole chain (Section 5.2, item 2).  The sumcheck proofs above cover its
+ * matrix products one at a time; nothing in them says that the int8 input of one product is the
+ * output of the one before.  In an int8-quantised execution the map between the two is the
+ * requantisation of the int32 accumulators,
+ *     H[i,j] = clamp( floor( (C[i,j] + rnd) / 2^shift ), lo, hi )
+ * (round-half-up division by 2^shift when rnd = 2^(shift-1), then saturation; e.g. the FFN hidden
+ * activations between the up and the down projection).  A verifier that holds the opened tensors
+ * checks such a link by recomputing it: one streaming pass, 4 bytes of C and 1 byte of H per entry. */
+
+/* d_result[0] = number of entries where H differs from the requantised C, d_result[1] = the row-major
+ * position i*cols + j of the first such entry (UINT64_MAX if there is none).  The link holds iff
+ * d_result[0] == 0.
+ *   d_C      : DEVICE int32 matrix, rows x cols, leading dimension ldc (elements)
+ *   d_H      : DEVICE int8 matrix, rows x cols, leading dimension ldh
+ *   shift    : 0..30;  rnd : 0 <= rnd < 2^shift;  -128 <= lo <= hi <= 127
+ *   d_result : DEVICE array of two uint64, 8-byte aligned; overwritten
+ * Rows of C that are 32-byte (or 16-byte) aligned with rows of H 16-byte aligned are read with
+ * 256-bit (128-bit) loads, anything else element by element.  Two memsets and one kernel are
+ * enqueued on `stream`; nothing is allocated or synchronised.  A differing entry is an audit
+ * finding, not an error: the call still returns IMM_OK.
+ * Errors: IMM_ERR_ARG (null pointer, parameters out of range), IMM_ERR_SHAPE (zero or > 2^20
+ * extent, ld < cols), IMM_ERR_ALIGN, IMM_ERR_CUDA. */
+int imm_requant_check(const int32_t* d_C, const int8_t* d_H, int64_t rows, int64_t cols, int64_t ldc,
+                      int64_t ldh, int shift, int32_t rnd, int32_t lo, int32_t hi, uint64_t* d_result,
+                      void* stream);
 
 /* ---------------------------------------------------------------------------------------------
  * Non-interactive proof (Fiat-Shamir)

@@ -37,7 +37,7 @@ EXPORTS = ("imm_version", "imm_last_cuda_error", "imm_challenge", "imm_field_bin
            "imm_sumcheck_matmul_fs_workspace", "imm_sumcheck_matmul_prove_fs", "imm_fs_challenges",
            "imm_sumcheck_verify_fs", "imm_sumcheck_expected_workspace", "imm_sumcheck_expected",
            "imm_sumcheck_matmul_fs_batched_workspace", "imm_sumcheck_matmul_prove_fs_batched",
-           "imm_fs_batched_challenges", "imm_sumcheck_verify_fs_batched")
+           "imm_fs_batched_challenges", "imm_sumcheck_verify_fs_batched", "imm_requant_check")
 FS_BATCH_MAX = 1024
 COMMIT_LEAF = 4096
 NOALLOC_MAX_TILES = 8192
@@ -149,6 +149,8 @@ def lib() -> ctypes.CDLL:
     L.imm_commit.argtypes = [vp, ci, vp, vp, vp, sz, vp]
     L.imm_sumcheck_verify_batched.restype = ci
     L.imm_sumcheck_verify_batched.argtypes = [vp, ci, ci, u64, u64, vp, vp]
+    L.imm_requant_check.restype = ci
+    L.imm_requant_check.argtypes = [vp, vp, i64, i64, i64, i64, ci, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp, vp]
     _lib = L
     return L
 
@@ -756,6 +758,26 @@ def sumcheck_expected(problems, seed: int = 0, batch_id: Optional[int] = None, p
     if int(v.status.abs().max()) != 0:
         raise ImmError(int(v.status.min()), "device status")
     return [tuple(int(x) & 0xFFFFFFFFFFFFFFFF for x in row) for row in t.cpu()]
+
+
+# ------------------------------------------------------------------ links between products
+
+
+def requant_check(C: torch.Tensor, H: torch.Tensor, shift: int = 9, rnd: int = 256, lo: int = -127, hi: int = 127,
+                  out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Checks H == clamp(floor((C + rnd) / 2^shift), lo, hi) entry by entry (C int32, H int8, same
+    shape).  Returns a 2-element int64 CUDA tensor: the number of differing entries and the row-major
+    position of the first (-1 if none).  Enqueued on the current stream; ``out`` to reuse a buffer."""
+    pc, cc, rows, cols, ldc = _matrix(C, "C")
+    ph, ch, rows2, cols2, ldh = _matrix(H, "H")
+    if cc != I32 or ch != I8 or (rows, cols) != (rows2, cols2):
+        raise ValueError("need C int32 and H int8 of the same shape")
+    if out is None:
+        out = torch.empty(2, dtype=torch.int64, device=C.device)
+    _cuda(out, torch.int64, "out")
+    _check(lib().imm_requant_check(pc, ph, rows, cols, ldc, ldh, int(shift), int(rnd), int(lo), int(hi),
+                                   out.data_ptr(), _stream()), "imm_requant_check")
+    return out
 
 
 # ------------------------------------------------------------------ logit distance distribution

@@ -36,11 +36,9 @@
  *     also return IMM_REJECT).  Nothing throws or aborts across this boundary.
  *   - The caller owns every buffer.  The library allocates no device memory: scratch comes from
  *     a caller-provided device workspace whose size a query call returns.  Workspace and output
- *     pointers must be 16-byte aligned.  What the library does keep, per process: two
- *     non-blocking CUDA streams and three events per device, created by the first prove call on
- *     that device whose batch is small enough to run its contractions side by side (see
- *     imm_sumcheck_matmul_prove), the event ring of imm_profile_enable, and the 64 KiB device array
- *     of imm_mle_eval_point_noalloc.
+ *     pointers must be 16-byte aligned.  What the library does keep, per process: the event
+ *     ring of imm_profile_enable (while enabled) and the 64 KiB device array of
+ *     imm_mle_eval_point_noalloc.  It creates no streams and launches only on the caller's.
  *   - One environment variable is read, on every prove / evaluation call: IMM_CONTRACT=alu selects
  *     the integer-pipe contraction kernels instead of the tensor-core ones (same results; meant for
  *     A/B measurements).  Anything else, or unset, is the default.
@@ -190,21 +188,32 @@ size_t imm_sumcheck_matmul_workspace(const imm_matmul_desc* descs_host, int npro
  *   d_status      : DEVICE array of nproofs int32, set to IMM_OK per proof (reserved for
  *                   device-detected conditions)
  *   d_ws          : DEVICE workspace, >= imm_sumcheck_matmul_workspace(...) bytes
- * The whole batch is a fixed sequence of five kernel launches ordered after the work already on
- * `stream`; results are valid once the stream has been synchronised.  For a batch of less than
- * 2 GiB of matrices the three contractions run side by side on two library-owned streams (created
- * on the first such call per device) that fork from and join back into `stream`.
+ * The whole batch is one small host-to-device copy (the job lists) and a fixed sequence of kernel
+ * launches on `stream`, ordered after the work already there; results are valid once the stream has
+ * been synchronised.  A batch of 2 GiB of matrices or more takes five launches: eq tables and
+ * weight limb tables, the claim, the row binding, the column binding, the rounds.  A smaller batch
+ * is bound by launch latency rather than bandwidth and takes three, chained by programmatic
+ * dependent launch: one contraction launch for all three matrix kinds, whose tiles build their own
+ * slice of the eq tables from the challenges (no table reaches memory); a reduction of the partial
+ * vectors into the round tables; the rounds.  Same transcripts either way.
  * Errors: IMM_ERR_ARG, IMM_ERR_SHAPE, IMM_ERR_ALIGN, IMM_ERR_WORKSPACE, IMM_ERR_CUDA. */
 int imm_sumcheck_matmul_prove(const imm_matmul_desc* descs_host, int nproofs, uint64_t seed,
                               imm_fe* d_transcripts, int64_t stride, int32_t* d_status,
                               void* d_ws, size_t ws_bytes, void* stream);
 
+/* Kernel launches imm_sumcheck_matmul_prove enqueues for this batch: 5, or 3 for a batch small
+ * enough for the fused contraction launch (0 on invalid input). */
+int imm_sumcheck_matmul_launches(const imm_matmul_desc* descs_host, int nproofs);
+
 /* Phase timing of imm_sumcheck_matmul_prove, for measurement.  While enabled, every prove call
- * records a pair of CUDA events around each of its five launches (on the stream the launch runs
- * on), into the next of `capacity` event sets (a ring), without synchronising.  When the three
- * contractions run side by side (small batches) their times overlap.  Phases:
+ * records a pair of CUDA events around each of its launches, into the next of `capacity` event sets
+ * (a ring), without synchronising.  Phases:
  *   [0] eq tables, [1] claim C~ (int32 point contraction), [2] A~ row binding,
  *   [3] B~ column binding, [4] sumcheck rounds.
+ * A batch that takes the fused contraction launch (see imm_sumcheck_matmul_prove) reports that launch
+ * as phase [1], phases [0], [2], [3] as (almost) zero, and the reduction plus the rounds as [4]; the
+ * events between its launches undo their programmatic overlap, so whole steps are best timed with
+ * phase timing off.
  * The event ring is per process; profiled calls must not overlap on different host threads.
  * imm_profile_enable(capacity): capacity in 1..4096 creates the ring and resets the call count
  *   (needs a CUDA device); capacity 0 destroys it.

@@ -117,10 +117,19 @@ int64_t count_tiles(const std::vector<Shape>& mats, int rows, int width)
 // several times over (the last wave is then a small fraction of the launch); for a batch too small
 // for that, the smallest tile, i.e. the most parallelism there is.  Large tiles amortise the
 // per-tile set-up (weight limbs staged in shared memory) and keep DRAM pages open longer.
+Geom pick_geom_for(const std::vector<Shape>& mats, const int* rows, int nrows, const int* widths, int nwidths,
+                   int64_t target, const char* env_rows, const char* env_width);
+
 Geom pick_geom(const std::vector<Shape>& mats, const int* rows, int nrows, const int* widths, int nwidths,
                int tiles_per_sm, const char* env_rows, const char* env_width)
 {
-    const int64_t target = (int64_t)sm_count() * env_int("IMM_TILES_PER_SM", tiles_per_sm);
+    return pick_geom_for(mats, rows, nrows, widths, nwidths,
+                         (int64_t)sm_count() * env_int("IMM_TILES_PER_SM", tiles_per_sm), env_rows, env_width);
+}
+
+Geom pick_geom_for(const std::vector<Shape>& mats, const int* rows, int nrows, const int* widths, int nwidths,
+                   int64_t target, const char* env_rows, const char* env_width)
+{
     Geom best{rows[nrows - 1], widths[nwidths - 1]};          // candidates are listed largest first
     int64_t best_area = -1;
     for (int i = 0; i < nrows; i++)
@@ -142,6 +151,14 @@ Geom pick_geom(const std::vector<Shape>& mats, const int* rows, int nrows, const
 const int rows_a[] = {1024, 512, 256, 128, 64, 32}, widths_a[] = {1024, 512, 256, 128};
 const int rows_b[] = {256}, rows_c[] = {1024, 512, 256, 128};
 const int chunks[] = {4096, 2048, 1024, 512, 256};
+// fused launch (small batches): one persistent grid, a run of equal bytes per block
+constexpr int64_t FUSE_BELOW_BYTES = (int64_t)2 << 30;       // batches under 2 GiB of matrices take the fused launch
+constexpr int FUSED_A_TILE_COLS = 1024;                      // 8 warps x 128 columns
+constexpr int64_t FUSED_MIN_RUN_BYTES = 32 << 10;            // below this a run is all set-up
+constexpr int FUSED_COST_A = 250, FUSED_COST_C = 180;        // time per byte of A and of C relative to B, per cent (measured)
+// rows one pass of a block's eight warps covers: row ranges are cut at multiples of it, so that no pass runs
+// on a few warps only (16 rows per warp and pass)
+constexpr int FUSED_PASS_ROWS_C = 128, FUSED_PASS_ROWS_B = 128;
 
 void fill_job(MatJob& j, const void* mat, int dtype, int64_t rows, int64_t cols, int64_t ld,
               int tile_rows, int cols_per_tile)
@@ -226,15 +243,16 @@ struct Plan {
     int nproofs = 0;
     int max_b = 0;
     bool mma = true;
+    bool fused = false;                        // one contraction launch with the eq weights built in the tiles
     int64_t max_cover = 0;                     // most entries an eq task covers (table or padded limb tables)
     int rows_a = 0, rows_b = 0, rows_c = 0;
     int cols_a = 0, cols_b = 0, cols_c = 0;    // columns (elements) per tile of the three contractions
     int mt_b = 2, mt_c = 1;                    // MMA row tiles per warp pass of the byte-dot kernels
     uint32_t tiles_a = 0, tiles_b = 0, tiles_c = 0;
     // byte offsets from the workspace base
-    size_t off_proofs = 0, off_jobs_a = 0, off_jobs_b = 0, off_jobs_c = 0, off_eq = 0, header_bytes = 0;
+    size_t off_proofs = 0, off_jobs_a = 0, off_jobs_b = 0, off_jobs_c = 0, off_eq = 0, off_fjobs = 0, header_bytes = 0;
     struct PerProof {
-        size_t e_row, e_col, part_a, part_b, part_c, sum_row, sum_col;
+        size_t e_row, e_col, part_a, part_b, part_c, sum_row, sum_col, tab, c0_ready;
         int n_sum_row, n_sum_col;
         size_t w_rows, w_cols_b, w_cols_c;          // limb tables (tensor-core back end)
         int nw_rows, nw_cols_b, nw_cols_c;          // their sizes in 32-bit words
@@ -242,7 +260,113 @@ struct Plan {
     };
     std::vector<PerProof> pp;
     size_t total_bytes = 0;
+    // fused launch: per-proof geometry, the segment list and each block's first segment
+    struct FusedGeom { int rows_a, nrb_a, ncc_a, chunk_b, ncc_b, chunk_c, ncc_c, seg0_c, nseg_c; };
+    std::vector<FusedGeom> fg;
+    std::vector<FusedSeg> segs;
+    std::vector<uint32_t> block_first;          // blocks + 1 entries
+    size_t off_segs = 0, off_block_first = 0;
 };
+
+int pow2_ceil_clamped(int64_t v, int lo, int hi)
+{
+    int c = lo;
+    while (c < hi && c < v) c *= 2;
+    return c;
+}
+
+int pow2_floor_clamped(int64_t v, int lo, int hi)
+{
+    int c = lo;
+    while (2 * c <= hi && 2 * c <= v) c *= 2;
+    return c;
+}
+
+// The fused launch's partition: every block of the persistent grid gets one contiguous run of the
+// sequence [tiles of every A][row ranges of every column chunk of every C][the same for every B],
+// cut so that all runs hold (almost) the same number of matrix bytes.
+void plan_fused(Plan& p, const imm_matmul_desc* descs, int nproofs)
+{
+    const int64_t blocks = (int64_t)sm_count() * FUSED_BLOCKS_PER_SM;
+    // cost of a byte of each kind relative to B, in per cent (measured: see FUSED_COST_*)
+    const int64_t cost_a = env_int("IMM_FUSED_COST_A", FUSED_COST_A), cost_c = env_int("IMM_FUSED_COST_C", FUSED_COST_C);
+    int64_t total = 0;
+    for (int i = 0; i < nproofs; i++)
+        total += descs[i].m * descs[i].k * cost_a / 100 + descs[i].k * descs[i].n + 4 * descs[i].m * descs[i].n * cost_c / 100;
+    const int64_t run = std::max<int64_t>((total + blocks - 1) / blocks, FUSED_MIN_RUN_BYTES);
+    // widest column chunk that still cuts a run into several passes of all eight warps (the cuts fall on pass
+    // boundaries, so the passes per run set how evenly the runs can be sized)
+    const int passes = env_int("IMM_FUSED_PASSES", 4);
+    const int pass_c = env_int("IMM_FUSED_PASS_C", FUSED_PASS_ROWS_C), pass_b = env_int("IMM_FUSED_PASS_B", FUSED_PASS_ROWS_B);
+    const int cap = env_int("IMM_FUSED_CHUNK", BYTEDOT_MAX_CHUNK_BYTES);
+    p.fg.resize(nproofs);
+    std::vector<int32_t> seg_block;
+    int64_t cum = 0;
+    auto block_of = [&](int64_t pos) { return (int32_t)std::min<int64_t>(blocks - 1, pos / run); };
+    // A: whole tiles of about half a run
+    for (int i = 0; i < nproofs; i++) {
+        const imm_matmul_desc& d = descs[i];
+        Plan::FusedGeom& g = p.fg[i];
+        const int64_t width = std::min<int64_t>(FUSED_A_TILE_COLS, d.k);
+        int64_t rows = (run * 100 / cost_a / 2 / width) / 32 * 32;
+        rows = rows < 32 ? 32 : rows > MAX_TILE_ROWS ? MAX_TILE_ROWS : rows;
+        g.nrb_a = (int)((d.m + rows - 1) / rows);
+        rows = ((d.m + g.nrb_a - 1) / g.nrb_a + 31) / 32 * 32;                // even row blocks
+        g.rows_a = (int)rows;
+        g.nrb_a = (int)((d.m + rows - 1) / rows);
+        g.ncc_a = (int)((d.k + FUSED_A_TILE_COLS - 1) / FUSED_A_TILE_COLS);
+        for (int rb = 0; rb < g.nrb_a; rb++)
+            for (int cc = 0; cc < g.ncc_a; cc++) {
+                const int64_t tr = std::min<int64_t>(rows, d.m - (int64_t)rb * rows);
+                const int64_t tc = std::min<int64_t>(FUSED_A_TILE_COLS, d.k - (int64_t)cc * FUSED_A_TILE_COLS);
+                p.segs.push_back(FusedSeg{i, rb * g.ncc_a + cc, 0, 0});
+                seg_block.push_back(block_of(cum));
+                cum += tr * tc * cost_a / 100;
+            }
+    }
+    // C then B: row ranges of column chunks
+    for (int kind = 1; kind < 3; kind++)
+        for (int i = 0; i < nproofs; i++) {
+            const imm_matmul_desc& d = descs[i];
+            Plan::FusedGeom& g = p.fg[i];
+            const int64_t rows = kind == 1 ? d.m : d.k;
+            const int64_t row_bytes = kind == 1 ? 4 * d.n : d.n;
+            const int64_t cost = kind == 1 ? cost_c : 100;
+            const int64_t step = kind == 1 ? pass_c : pass_b;
+            const int chunk = pow2_ceil_clamped(row_bytes, 256, pow2_floor_clamped(run * 100 / cost / (passes * step), 256, cap));
+            const int ncc = (int)((row_bytes + chunk - 1) / chunk);
+            if (kind == 1) { g.chunk_c = chunk; g.ncc_c = ncc; g.seg0_c = (int)p.segs.size(); }
+            else { g.chunk_b = chunk; g.ncc_b = ncc; }
+            for (int cc = 0; cc < ncc; cc++) {
+                if (kind == 1 && cc == 0) g.nseg_c = 0;
+                const int64_t w = std::max<int64_t>(1, std::min<int64_t>(chunk, row_bytes - (int64_t)cc * chunk) * cost / 100);
+                int64_t r = 0;
+                while (r < rows) {
+                    const int32_t b = block_of(cum);
+                    int64_t nr = rows - r;
+                    if (b < blocks - 1) {
+                        const int64_t room = (int64_t)(b + 1) * run - cum;
+                        int64_t want = ((room + w / 2) / w + step / 2) / step * step;           // to the nearest pass boundary
+                        if (want < step) want = step;
+                        if (r + want + step <= rows) nr = want;                  // (a remainder under one pass joins this range)
+                    }
+                    p.segs.push_back(FusedSeg{kind * nproofs + i, cc, (int32_t)r, (int32_t)(r + nr)});
+                    seg_block.push_back(b);
+                    if (kind == 1) g.nseg_c++;
+                    cum += nr * w;
+                    r += nr;
+                }
+            }
+        }
+    const int used = seg_block.empty() ? 0 : seg_block.back() + 1;
+    p.block_first.assign(used + 1, 0);
+    size_t si = 0;
+    for (int b = 0; b <= used; b++) {
+        while (si < seg_block.size() && seg_block[si] < b) si++;
+        p.block_first[b] = (uint32_t)si;
+    }
+}
+
 
 int check_desc(const imm_matmul_desc& d)
 {
@@ -267,7 +391,13 @@ Plan make_plan(const imm_matmul_desc* descs, int nproofs)
         sc.push_back({descs[i].m, descs[i].n});
     }
     p.mma = use_mma();
-    if (p.mma) {
+    int64_t batch_bytes = 0;
+    for (int i = 0; i < nproofs; i++)
+        batch_bytes += descs[i].m * descs[i].k + descs[i].k * descs[i].n + 4 * descs[i].m * descs[i].n;
+    p.fused = p.mma && batch_bytes < FUSE_BELOW_BYTES && !env_set("IMM_NO_FUSE");
+    if (p.fused) {
+        plan_fused(p, descs, nproofs);
+    } else if (p.mma) {
         // A: rows x (128 columns per warp).  B, C: rows x byte-columns; a block pass covers
         // 128 rows per MMA row tile, so shorter tiles would leave warps idle.  Measured on the
         // decoder-block workload: B (two row tiles per warp) is best at 256 rows per tile, C (one) at
@@ -304,6 +434,9 @@ Plan make_plan(const imm_matmul_desc* descs, int nproofs)
     p.off_jobs_b = off; off = align_up(off + sizeof(MatJob) * nproofs);
     p.off_jobs_c = off; off = align_up(off + sizeof(MatJob) * nproofs);
     p.off_eq = off;     off = align_up(off + sizeof(EqTask) * 2 * nproofs);
+    p.off_fjobs = off;  off = align_up(off + (p.fused ? sizeof(FusedJob) * 3 * (size_t)nproofs : 0));
+    p.off_segs = off;   off = align_up(off + sizeof(FusedSeg) * p.segs.size());
+    p.off_block_first = off; off = align_up(off + sizeof(uint32_t) * p.block_first.size());
     p.header_bytes = off;
 
     uint64_t ta = 0, tb = 0, tc = 0;
@@ -313,18 +446,29 @@ Plan make_plan(const imm_matmul_desc* descs, int nproofs)
         Plan::PerProof& q = p.pp[i];
         q.a = ceil_log2(d.m); q.b = ceil_log2(d.k); q.c = ceil_log2(d.n);
         if (q.b > p.max_b) p.max_b = q.b;
-        q.n_part_a = (int)((d.m + p.rows_a - 1) / p.rows_a);
-        q.n_part_b = (int)((d.n + bcols - 1) / bcols);
-        const int64_t c_nrb = (d.m + p.rows_c - 1) / p.rows_c;
-        const int64_t c_ncc = (d.n + ccols - 1) / ccols;
-        q.n_part_c = (int)(c_nrb * c_ncc) * (p.mma ? BYTEDOT_THREADS / 32 : 1);   // tensor-core kernel: one per warp
+        int64_t c_nrb = 0, c_ncc = 0;
+        if (p.fused) {
+            // one partial avec per row block of A, one partial bvec per column chunk of B, eight warp
+            // partials per segment of C
+            const Plan::FusedGeom& g = p.fg[i];
+            q.n_part_a = g.nrb_a;
+            q.n_part_b = g.ncc_b;
+            q.n_part_c = g.nseg_c * (BYTEDOT_THREADS / 32);
+        } else {
+            q.n_part_a = (int)((d.m + p.rows_a - 1) / p.rows_a);
+            q.n_part_b = (int)((d.n + bcols - 1) / bcols);
+            c_nrb = (d.m + p.rows_c - 1) / p.rows_c;
+            c_ncc = (d.n + ccols - 1) / ccols;
+            q.n_part_c = (int)(c_nrb * c_ncc) * (p.mma ? BYTEDOT_THREADS / 32 : 1);   // tensor-core kernel: one per warp
+        }
         const int64_t slice = 4 * (int64_t)EQ_SLICE_QUADS;                  // entries per block of the eq kernel
         q.n_sum_row = (int)((std::max<int64_t>((int64_t)1 << q.a, (d.m + 31) / 32 * 32) + slice - 1) / slice);
         q.n_sum_col = (int)((std::max<int64_t>((int64_t)1 << q.c, (d.n + 255) / 256 * 256) + slice - 1) / slice);
         if (((int64_t)1 << q.a) > p.max_cover) p.max_cover = (int64_t)1 << q.a;
         if (((int64_t)1 << q.c) > p.max_cover) p.max_cover = (int64_t)1 << q.c;
-        q.e_row = off;  off = align_up(off + sizeof(imm_fe) * ((size_t)1 << q.a));
-        q.e_col = off;  off = align_up(off + sizeof(imm_fe) * ((size_t)1 << q.c));
+        if (p.fused) { q.n_sum_row = q.n_sum_col = 0; }
+        q.e_row = off;  off = align_up(off + (p.fused ? 0 : sizeof(imm_fe) * ((size_t)1 << q.a)));
+        q.e_col = off;  off = align_up(off + (p.fused ? 0 : sizeof(imm_fe) * ((size_t)1 << q.c)));
         q.part_a = off; off = align_up(off + sizeof(imm_fe) * (size_t)q.n_part_a * d.k);
         q.part_b = off; off = align_up(off + sizeof(imm_fe) * (size_t)q.n_part_b * d.k);
         q.part_c = off; off = align_up(off + sizeof(imm_fe) * (size_t)q.n_part_c);
@@ -332,7 +476,7 @@ Plan make_plan(const imm_matmul_desc* descs, int nproofs)
         q.sum_col = off; off = align_up(off + sizeof(imm_fe) * (size_t)q.n_sum_col);
         q.nw_rows = q.nw_cols_b = q.nw_cols_c = 0;
         q.w_rows = q.w_cols_b = q.w_cols_c = 0;
-        if (p.mma) {
+        if (p.mma && !p.fused) {
             q.nw_rows = (int)((d.m + 31) / 32) * 64;
             q.nw_cols_b = (int)((d.n + 255) / 256) * 512;
             q.nw_cols_c = (int)((4 * d.n + 255) / 256) * 512;
@@ -343,12 +487,19 @@ Plan make_plan(const imm_matmul_desc* descs, int nproofs)
             if (cover_rows > p.max_cover) p.max_cover = cover_rows;
             if (cover_cols > p.max_cover) p.max_cover = cover_cols;
         }
-        ta += (uint64_t)q.n_part_a * ((d.k + acols - 1) / acols);
-        tb += (uint64_t)((d.k + p.rows_b - 1) / p.rows_b) * q.n_part_b;
-        tc += (uint64_t)(c_nrb * c_ncc);
+        if (!p.fused) {
+            ta += (uint64_t)q.n_part_a * ((d.k + acols - 1) / acols);
+            tb += (uint64_t)((d.k + p.rows_b - 1) / p.rows_b) * q.n_part_b;
+            tc += (uint64_t)(c_nrb * c_ncc);
+        }
     }
-    if (ta > 0x7FFFFFFFu || tb > 0x7FFFFFFFu || tc > 0x7FFFFFFFu) { p.status = IMM_ERR_SHAPE; return p; }
+    if (ta > 0x7FFFFFFFu || tb > 0x7FFFFFFFu || tc > 0x7FFFFFFFu || ta + tb + tc > 0x7FFFFFFFu) { p.status = IMM_ERR_SHAPE; return p; }
     p.tiles_a = (uint32_t)ta; p.tiles_b = (uint32_t)tb; p.tiles_c = (uint32_t)tc;
+    if (p.fused)                                 // both round tables (2^max_b entries each: a batched proof pads every k) and the claim
+        for (int i = 0; i < nproofs; i++) {
+            p.pp[i].tab = off;      off = align_up(off + 2 * (sizeof(imm_fe) << p.max_b));
+            p.pp[i].c0_ready = off; off = align_up(off + sizeof(imm_fe));
+        }
     p.total_bytes = off;
     return p;
 }
@@ -357,37 +508,6 @@ Plan make_plan(const imm_matmul_desc* descs, int nproofs)
 constexpr int PROF_EV = 2 * IMM_PROFILE_PHASES;    // a (start, end) pair per phase
 std::vector<cudaEvent_t> g_prof_ev;        // capacity * PROF_EV events, empty when profiling is off
 int64_t g_prof_calls = 0;
-
-// Small batches do not fill the GPU with one contraction at a time: their three contractions (claim,
-// row binding, column binding) are independent and run on three streams.  Two side streams and the
-// fork / join events per device, created on first use.
-constexpr int MAX_DEVICES = 64;
-constexpr int64_t FORK_BELOW_BYTES = (int64_t)2 << 30;       // batches under 2 GiB of matrices fork
-struct SideStreams {
-    bool ready = false;
-    cudaStream_t s[2] = {nullptr, nullptr};
-    cudaEvent_t fork = nullptr, join[2] = {nullptr, nullptr};
-};
-SideStreams g_side[MAX_DEVICES];
-std::mutex g_side_mutex;        // guards the creation of the side streams
-std::mutex g_fork_mutex;        // held while one call enqueues its fork ... join: the events are shared
-
-SideStreams* side_streams()
-{
-    int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return nullptr;
-    std::lock_guard<std::mutex> lock(g_side_mutex);
-    SideStreams& ss = g_side[dev];
-    if (!ss.ready) {
-        for (int i = 0; i < 2; i++) {
-            if (cudaStreamCreateWithFlags(&ss.s[i], cudaStreamNonBlocking) != cudaSuccess) return nullptr;
-            if (cudaEventCreateWithFlags(&ss.join[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
-        }
-        if (cudaEventCreateWithFlags(&ss.fork, cudaEventDisableTiming) != cudaSuccess) return nullptr;
-        ss.ready = true;
-    }
-    return &ss;
-}
 
 int check_stride(const imm_matmul_desc* descs, int nproofs, int64_t stride)
 {
@@ -627,6 +747,13 @@ size_t imm_sumcheck_matmul_workspace(const imm_matmul_desc* descs_host, int npro
     return p.status == IMM_OK ? p.total_bytes : 0;
 }
 
+int imm_sumcheck_matmul_launches(const imm_matmul_desc* descs_host, int nproofs)
+{
+    Plan p = make_plan(descs_host, nproofs);
+    if (p.status != IMM_OK) return 0;
+    return p.fused ? 3 : 5;
+}
+
 // The launch sequence of a batch.  shared_round_id: null = every proof draws its round challenges
 // under its own proof_id and runs its own ceil(log2 k) rounds; else all proofs draw them under that
 // one id and run the rounds of the largest k (a batched proof).
@@ -715,6 +842,8 @@ static int prove_batch(const imm_matmul_desc* descs_host, int nproofs, uint64_t 
     MatJob* jb = (MatJob*)(hdr.data() + p.off_jobs_b);
     MatJob* jc = (MatJob*)(hdr.data() + p.off_jobs_c);
     EqTask* eq = (EqTask*)(hdr.data() + p.off_eq);
+    FusedJob* fj = p.fused ? (FusedJob*)(hdr.data() + p.off_fjobs) : nullptr;
+    const bool tables_ready = p.fused && !fs && !vf;            // reduce_parts_kernel finishes the round tables
     const int acols = p.cols_a, bcols = p.cols_b, ccols = p.cols_c;
     FsLayout fsl;
     std::vector<FsProof> fsp;
@@ -744,22 +873,29 @@ static int prove_batch(const imm_matmul_desc* descs_host, int nproofs, uint64_t 
         P.m = (int32_t)d.m; P.k = (int32_t)d.k; P.n = (int32_t)d.n;
         P.a = q.a; P.b = shared_round_id ? p.max_b : q.b; P.c = q.c;   // a batched proof pads every k to the largest 2^b
         P.n_part_a = q.n_part_a; P.n_part_b = q.n_part_b; P.n_part_c = q.n_part_c;
-        P.sum_row = (imm_fe*)(base + q.sum_row); P.sum_col = (imm_fe*)(base + q.sum_col);
+        P.sum_row = p.fused ? nullptr : (imm_fe*)(base + q.sum_row);
+        P.sum_col = p.fused ? nullptr : (imm_fe*)(base + q.sum_col);
         P.n_sum_row = q.n_sum_row; P.n_sum_col = q.n_sum_col;
         P.c_offset = p.mma ? 1 : 0;
+        P.seed = seed; P.proof_id = d.proof_id;
+        P.pt_row = P.pt_col = nullptr;
+        P.tab = tables_ready ? (imm_fe*)(base + q.tab) : nullptr;
+        P.c0_ready = tables_ready ? (imm_fe*)(base + q.c0_ready) : nullptr;
 
-        fill_job(ja[i], d.A, IMM_I8, d.m, d.k, d.lda, p.rows_a, acols);
-        ja[i].eq_row = P.e_row; ja[i].out = (imm_fe*)P.part_a; ja[i].tile0 = ta;
-        ta += (uint32_t)(ja[i].nrb * ja[i].ncc);
-        fill_job(jb[i], d.B, IMM_I8, d.k, d.n, d.ldb, p.rows_b, bcols);
-        jb[i].eq_col = P.e_col; jb[i].out = (imm_fe*)P.part_b; jb[i].tile0 = tb; jb[i].chunk = bcols;
-        tb += (uint32_t)(jb[i].nrb * jb[i].ncc);
-        fill_job(jc[i], d.C, IMM_I32, d.m, d.n, d.ldc, p.rows_c, ccols);
-        jc[i].eq_row = P.e_row; jc[i].eq_col = P.e_col; jc[i].out = (imm_fe*)P.part_c; jc[i].tile0 = tc;
-        jc[i].chunk = 4 * ccols;
-        tc += (uint32_t)(jc[i].nrb * jc[i].ncc);
+        if (!p.fused) {
+            fill_job(ja[i], d.A, IMM_I8, d.m, d.k, d.lda, p.rows_a, acols);
+            ja[i].eq_row = P.e_row; ja[i].out = (imm_fe*)P.part_a; ja[i].tile0 = ta;
+            ta += (uint32_t)(ja[i].nrb * ja[i].ncc);
+            fill_job(jb[i], d.B, IMM_I8, d.k, d.n, d.ldb, p.rows_b, bcols);
+            jb[i].eq_col = P.e_col; jb[i].out = (imm_fe*)P.part_b; jb[i].tile0 = tb; jb[i].chunk = bcols;
+            tb += (uint32_t)(jb[i].nrb * jb[i].ncc);
+            fill_job(jc[i], d.C, IMM_I32, d.m, d.n, d.ldc, p.rows_c, ccols);
+            jc[i].eq_row = P.e_row; jc[i].eq_col = P.e_col; jc[i].out = (imm_fe*)P.part_c; jc[i].tile0 = tc;
+            jc[i].chunk = 4 * ccols;
+            tc += (uint32_t)(jc[i].nrb * jc[i].ncc);
+        }
 
-        if (p.mma) {
+        if (p.mma && !p.fused) {
             ja[i].wtab = (const uint32_t*)(base + q.w_rows);
             jb[i].wtab = (const uint32_t*)(base + q.w_cols_b);
             jc[i].wtab = (const uint32_t*)(base + q.w_cols_c);
@@ -778,6 +914,7 @@ static int prove_batch(const imm_matmul_desc* descs_host, int nproofs, uint64_t 
             if (given) {
                 eq[2 * i].point = given;
                 eq[2 * i + 1].point = given + FS_POINT_SLOTS;
+                P.pt_row = given; P.pt_col = given + FS_POINT_SLOTS;
             }
             imm_fe* e_k = (imm_fe*)(vf->ext + vl.off_ek[i]);
             ekt[i] = EqTask{e_k, seed, P.round_id, 3u, P.b, nullptr, nullptr, nullptr, (int32_t)d.k, 0, nullptr};
@@ -787,6 +924,7 @@ static int prove_batch(const imm_matmul_desc* descs_host, int nproofs, uint64_t 
         if (fs) {
             eq[2 * i].point = pts;
             eq[2 * i + 1].point = pts + FS_POINT_SLOTS;
+            P.pt_row = pts; P.pt_col = pts + FS_POINT_SLOTS;
             FsProof& F = fsp[i];
             F.com = fs->d_com + (size_t)i * 96;
             F.points = (imm_fe*)pts;
@@ -797,25 +935,44 @@ static int prove_batch(const imm_matmul_desc* descs_host, int nproofs, uint64_t 
             F.one = 1;
         }
     }
-    if (ta != p.tiles_a || tb != p.tiles_b || tc != p.tiles_c) return IMM_ERR_ARG;   // planner invariant
+    if (!p.fused && (ta != p.tiles_a || tb != p.tiles_b || tc != p.tiles_c)) return IMM_ERR_ARG;   // planner invariant
+    if (p.fused) {
+        // the fused launch's job list, kind-major: every A, every C, every B (the order of the segments)
+        for (int kind = 0; kind < 3; kind++)
+            for (int i = 0; i < nproofs; i++) {
+                const imm_matmul_desc& d = descs_host[i];
+                const Plan::FusedGeom& g = p.fg[i];
+                FusedJob& F = fj[kind * nproofs + i];
+                memset(&F, 0, sizeof(F));
+                if (kind == 0) {
+                    fill_job(F.mj, d.A, IMM_I8, d.m, d.k, d.lda, g.rows_a, FUSED_A_TILE_COLS);
+                    F.mj.out = (imm_fe*)pd[i].part_a;
+                    F.kind = JOB_ROWBIND;
+                } else if (kind == 1) {
+                    fill_job(F.mj, d.C, IMM_I32, d.m, d.n, d.ldc, MAX_TILE_ROWS, g.chunk_c / 4);
+                    F.mj.chunk = g.chunk_c;
+                    F.mj.out = (imm_fe*)pd[i].part_c;
+                    F.kind = JOB_POINT;
+                    F.seg0 = g.seg0_c;
+                } else {
+                    fill_job(F.mj, d.B, IMM_I8, d.k, d.n, d.ldb, MAX_TILE_ROWS, g.chunk_b);
+                    F.mj.chunk = g.chunk_b;
+                    F.mj.out = (imm_fe*)pd[i].part_b;
+                    F.kind = JOB_COLBIND;
+                }
+                F.seed = seed; F.proof_id = d.proof_id;
+                F.pt_row = pd[i].pt_row; F.pt_col = pd[i].pt_col;
+                F.a = p.pp[i].a; F.c = p.pp[i].c;
+            }
+        memcpy(hdr.data() + p.off_segs, p.segs.data(), sizeof(FusedSeg) * p.segs.size());
+        memcpy(hdr.data() + p.off_block_first, p.block_first.data(), sizeof(uint32_t) * p.block_first.size());
+    }
 
     const bool prof = !g_prof_ev.empty();
     cudaEvent_t* pev = prof ? &g_prof_ev[(size_t)(g_prof_calls % (int64_t)(g_prof_ev.size() / PROF_EV)) * PROF_EV]
                             : nullptr;
     // phase i is timed by events 2i (start) and 2i+1 (end), each on the stream its kernel runs on
 #define PROF_MARK(i, stream_) do { if (prof) CU(cudaEventRecord(pev[i], stream_)); } while (0)
-    int64_t batch_bytes = 0;
-    for (int i = 0; i < nproofs; i++) {
-        const imm_matmul_desc& d = descs_host[i];
-        batch_bytes += d.m * d.k + d.k * d.n + 4 * d.m * d.n;
-    }
-    SideStreams* ss = (batch_bytes < FORK_BELOW_BYTES && !env_set("IMM_NO_FORK")) ? side_streams() : nullptr;
-    cudaStream_t st_a = ss ? ss->s[0] : st, st_b = ss ? ss->s[1] : st;
-    // Host threads proving on different streams share the side streams and their events: one call
-    // at a time enqueues its fork ... join (a wait refers to the record that precedes it, so a later
-    // call's records do not disturb the waits already enqueued).
-    std::unique_lock<std::mutex> fork_lock;
-    if (ss) fork_lock = std::unique_lock<std::mutex>(g_fork_mutex);
     CU(cudaMemcpyAsync(base, hdr.data(), hdr.size(), cudaMemcpyHostToDevice, st));
     if (fs) {
         CU(cudaMemcpyAsync(fs->ext + fsl.off_fs, fsp.data(), fsp.size() * sizeof(FsProof), cudaMemcpyHostToDevice, st));
@@ -828,33 +985,29 @@ static int prove_batch(const imm_matmul_desc* descs_host, int nproofs, uint64_t 
             CU(cudaMemcpyAsync(vf->ext + vl.off_points, vf->points_host,
                                (size_t)nproofs * VERIFY_POINT_SLOTS * sizeof(imm_fe), cudaMemcpyHostToDevice, st));
     }
+    // (While phase timing is on, the events recorded between the launches of a fused batch undo their
+    // programmatic overlap: whole steps are timed with it off.)
     PROF_MARK(0, st);
-    CU(launch_eq_batch((const EqTask*)(base + p.off_eq), 2 * nproofs, p.max_cover, st));
+    if (!p.fused) CU(launch_eq_batch((const EqTask*)(base + p.off_eq), 2 * nproofs, p.max_cover, st));
     if (vf) CU(launch_eq_batch((const EqTask*)(vf->ext + vl.off_tasks), nproofs, (int64_t)1 << p.max_b, st));
     PROF_MARK(1, st);
-    if (ss) {                                                 // fork: the side streams wait for the eq tables
-        CU(cudaEventRecord(ss->fork, st));
-        CU(cudaStreamWaitEvent(st_a, ss->fork, 0));
-        CU(cudaStreamWaitEvent(st_b, ss->fork, 0));
-    }
     PROF_MARK(2, st);
-    if (p.mma) CU(launch_bytedot(true, true, p.mt_c, (const MatJob*)(base + p.off_jobs_c), nproofs, p.tiles_c, st));
+    if (p.fused)
+        CU(launch_fused_contract((const FusedJob*)(base + p.off_fjobs), (const FusedSeg*)(base + p.off_segs),
+                                 (const uint32_t*)(base + p.off_block_first), (uint32_t)p.block_first.size() - 1, st));
+    else if (p.mma) CU(launch_bytedot(true, true, p.mt_c, (const MatJob*)(base + p.off_jobs_c), nproofs, p.tiles_c, st));
     else CU(launch_rowbind(IMM_I32, true, (const MatJob*)(base + p.off_jobs_c), nproofs, p.tiles_c, st));
     PROF_MARK(3, st);
-    PROF_MARK(4, st_a);
-    if (p.mma) CU(launch_rowmma((const MatJob*)(base + p.off_jobs_a), nproofs, p.tiles_a, p.cols_a / 128, st_a));
-    else CU(launch_rowbind(IMM_I8, false, (const MatJob*)(base + p.off_jobs_a), nproofs, p.tiles_a, st_a));
-    PROF_MARK(5, st_a);
-    PROF_MARK(6, st_b);
-    if (p.mma) CU(launch_bytedot(false, false, p.mt_b, (const MatJob*)(base + p.off_jobs_b), nproofs, p.tiles_b, st_b));
-    else CU(launch_colbind(IMM_I8, (const MatJob*)(base + p.off_jobs_b), nproofs, p.tiles_b, st_b));
-    PROF_MARK(7, st_b);
-    if (ss) {                                                 // join
-        CU(cudaEventRecord(ss->join[0], st_a));
-        CU(cudaEventRecord(ss->join[1], st_b));
-        CU(cudaStreamWaitEvent(st, ss->join[0], 0));
-        CU(cudaStreamWaitEvent(st, ss->join[1], 0));
-    }
+    PROF_MARK(4, st);
+    if (p.fused) {}
+    else if (p.mma) CU(launch_rowmma((const MatJob*)(base + p.off_jobs_a), nproofs, p.tiles_a, p.cols_a / 128, st));
+    else CU(launch_rowbind(IMM_I8, false, (const MatJob*)(base + p.off_jobs_a), nproofs, p.tiles_a, st));
+    PROF_MARK(5, st);
+    PROF_MARK(6, st);
+    if (p.fused) {}
+    else if (p.mma) CU(launch_bytedot(false, false, p.mt_b, (const MatJob*)(base + p.off_jobs_b), nproofs, p.tiles_b, st));
+    else CU(launch_colbind(IMM_I8, (const MatJob*)(base + p.off_jobs_b), nproofs, p.tiles_b, st));
+    PROF_MARK(7, st);
     PROF_MARK(8, st);
     if (vf)
         CU(launch_expected((const ProofDev*)(base + p.off_proofs), (const ExpectDev*)(vf->ext + vl.off_ex), nproofs,
@@ -876,9 +1029,11 @@ static int prove_batch(const imm_matmul_desc* descs_host, int nproofs, uint64_t 
     } else if (fs)
         CU(launch_sumcheck_fs((const ProofDev*)(base + p.off_proofs), (const FsProof*)(fs->ext + fsl.off_fs), nproofs,
                               d_transcripts, stride, d_status, st));
-    else
+    else {
+        if (tables_ready) CU(launch_reduce_parts((const ProofDev*)(base + p.off_proofs), nproofs, p.max_b, st));
         CU(launch_sumcheck((const ProofDev*)(base + p.off_proofs), nproofs, seed, d_transcripts, stride,
-                           d_status, p.max_b, env_int("IMM_SC_CLUSTER", 0), st));
+                           d_status, p.max_b, env_int("IMM_SC_CLUSTER", 0), tables_ready, st));
+    }
     PROF_MARK(9, st);
 #undef PROF_MARK
     if (prof) g_prof_calls++;

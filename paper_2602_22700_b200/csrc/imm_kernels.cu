@@ -529,7 +529,9 @@ __device__ __forceinline__ uint64_t fold1(uint64_t lo, uint64_t hi, uint64_t r)
 
 // sum_p parts[p][y]: the loads of eight partial vectors are issued together (the chain is bound by
 // memory latency, not by the additions).
-__device__ __forceinline__ uint64_t sum_parts_at(const imm_fe* __restrict__ parts, int nparts, int len, int y)
+// (Loads go to L2, not through the read-only path: the kernel that wrote the partials may still have
+// been running when this one was launched, see imm_fused.cuh.)
+__device__ __forceinline__ uint64_t sum_parts_at(const imm_fe* parts, int nparts, int len, int y)
 {
     const imm_fe* src = parts + y;
     uint64_t s = 0;
@@ -537,18 +539,40 @@ __device__ __forceinline__ uint64_t sum_parts_at(const imm_fe* __restrict__ part
     for (; p + 8 <= nparts; p += 8) {
         uint64_t v[8];
 #pragma unroll
-        for (int pp = 0; pp < 8; pp++) v[pp] = __ldg(src + (int64_t)(p + pp) * len);
+        for (int pp = 0; pp < 8; pp++) v[pp] = __ldcg(src + (int64_t)(p + pp) * len);
 #pragma unroll
         for (int pp = 0; pp < 8; pp++) s = gl::add(s, v[pp]);
     }
     if (p < nparts) {
         uint64_t v[8];
 #pragma unroll
-        for (int pp = 0; pp < 8; pp++) v[pp] = p + pp < nparts ? __ldg(src + (int64_t)(p + pp) * len) : 0;
+        for (int pp = 0; pp < 8; pp++) v[pp] = p + pp < nparts ? __ldcg(src + (int64_t)(p + pp) * len) : 0;
 #pragma unroll
         for (int pp = 0; pp < 8; pp++) s = gl::add(s, v[pp]);
     }
     return s;
+}
+
+}  // namespace imm
+
+#include "imm_fused.cuh"
+
+namespace imm {
+
+// 2^31 * (sum of E_row over the real rows) * (sum of E_col over the real columns): what the claim
+// kernel's unsigned view of the int32 entries adds to the sum of its partial results.  The two sums
+// come from the eq kernel's slice sums where those exist, else from the challenges in closed form.
+// Block-wide call; `red` holds 33 words plus two; valid in every thread.
+__device__ __forceinline__ uint64_t claim_offset_block(const ProofDev& pr, uint64_t* red)
+{
+    if (!pr.c_offset) return 0;
+    if (pr.sum_row == nullptr) return gl::shl(offset_sums_closed_form(pr, red + 33), 31);
+    uint64_t sr = 0, sc = 0;
+    for (int i = threadIdx.x; i < pr.n_sum_row; i += blockDim.x) sr = gl::add(sr, pr.sum_row[i]);
+    for (int i = threadIdx.x; i < pr.n_sum_col; i += blockDim.x) sc = gl::add(sc, pr.sum_col[i]);
+    sr = block_sum_fe(sr, red);
+    sc = block_sum_fe(sc, red);
+    return gl::shl(gl::mul(sr, sc), 31);
 }
 
 struct ScShared {
@@ -630,6 +654,7 @@ __global__ void __launch_bounds__(SUMCHECK_THREADS, 2)
 sumcheck_kernel(const ProofDev* proofs, uint64_t seed, imm_fe* transcripts, int64_t stride,
                 int32_t* status, int cap /* entries per shared-memory table */)
 {
+    pdl_launch_dependents();
     namespace cg = cooperative_groups;
     extern __shared__ __align__(16) uint64_t tabs[];       // [2][cap]
     __shared__ ScShared sh;
@@ -653,35 +678,51 @@ sumcheck_kernel(const ProofDev* proofs, uint64_t seed, imm_fe* transcripts, int6
     if (tid < b) sh.r[tid] = gl::challenge(seed, pr.round_id, 3, (uint32_t)tid);
     for (int i = tid; i < MAX_K_VARS * SC_WARPS * 3; i += SUMCHECK_THREADS) (&sh.warp_sums[0][0][0])[i] = 0;
     for (int i = tid; i < MAX_K_VARS * 32 * 3; i += SUMCHECK_THREADS) (&sh.lane_sums[0][0][0])[i] = 0;
-    if (c == 0) {
-        // claim c0 = sum of the partial sums of C
-        uint64_t s = 0;
-        for (int i = tid; i < pr.n_part_c; i += SUMCHECK_THREADS) s = gl::add(s, pr.part_c[i]);
-        s = warp_sum_fe(s);
-        if ((tid & 31) == 0) sh.red[tid >> 5] = s;
-        __syncthreads();
-        if (tid < 32) s = warp_sum_fe(tid < SC_WARPS ? sh.red[tid] : 0);
-        if (tid < 32 && pr.c_offset) {
-            // the claim kernel summed unsigned bytes: every entry reads 2^31 too high
-            uint64_t sr = 0, sc = 0;
-            for (int i = tid; i < pr.n_sum_row; i += 32) sr = gl::add(sr, pr.sum_row[i]);
-            for (int i = tid; i < pr.n_sum_col; i += 32) sc = gl::add(sc, pr.sum_col[i]);
-            sr = warp_sum_fe(sr); sc = warp_sum_fe(sc);
-            s = gl::sub(s, gl::shl(gl::mul(sr, sc), 31));
+    pdl_wait();                                            // from here on: results of the launches before
+    if (pr.tab) {
+        // the tables and the claim were finished by reduce_parts_kernel
+        if (c == 0) {
+            if (tid == 0) { tr[0] = __ldcg(pr.c0_ready); status[proof] = 0; }
+            for (int64_t i = 3 * b + 3 + tid; i < stride; i += SUMCHECK_THREADS) tr[i] = 0;
         }
-        if (tid == 0) { tr[0] = s; status[proof] = 0; }
-        for (int64_t i = 3 * b + 3 + tid; i < stride; i += SUMCHECK_THREADS) tr[i] = 0;
-    }
-    __syncthreads();
+        const int n0 = 1 << b;
+#pragma unroll 4
+        for (int e = tid; e < L; e += SUMCHECK_THREADS) {
+            const int y = (e / W) * F + c * W + (e % W);
+            ta[e] = __ldcg(pr.tab + y);
+            tb[e] = __ldcg(pr.tab + n0 + y);
+        }
+    } else {
+        if (c == 0) {
+            // claim c0 = sum of the partial sums of C
+            uint64_t s = 0;
+            for (int i = tid; i < pr.n_part_c; i += SUMCHECK_THREADS) s = gl::add(s, pr.part_c[i]);
+            s = warp_sum_fe(s);
+            if ((tid & 31) == 0) sh.red[tid >> 5] = s;
+            __syncthreads();
+            if (tid < 32) s = warp_sum_fe(tid < SC_WARPS ? sh.red[tid] : 0);
+            if (tid < 32 && pr.c_offset) {
+                // the claim kernel summed unsigned bytes: every entry reads 2^31 too high
+                uint64_t sr = 0, sc = 0;
+                for (int i = tid; i < pr.n_sum_row; i += 32) sr = gl::add(sr, pr.sum_row[i]);
+                for (int i = tid; i < pr.n_sum_col; i += 32) sc = gl::add(sc, pr.sum_col[i]);
+                sr = warp_sum_fe(sr); sc = warp_sum_fe(sc);
+                s = gl::sub(s, gl::shl(gl::mul(sr, sc), 31));
+            }
+            if (tid == 0) { tr[0] = s; status[proof] = 0; }
+            for (int64_t i = 3 * b + 3 + tid; i < stride; i += SUMCHECK_THREADS) tr[i] = 0;
+        }
+        __syncthreads();
 
-    // build this block's entries from the partial vectors (all threads, one entry of each table
-    // at a time), then the local rounds
+        // build this block's entries from the partial vectors (all threads, one entry of each table
+        // at a time), then the local rounds
 #pragma unroll 1
-    for (int e = tid; e < L; e += SUMCHECK_THREADS) {
-        const int y = (e / W) * F + c * W + (e % W);
-        const bool live = y < pr.k;                        // entries past k are the zero padding
-        ta[e] = live ? sum_parts_at(pr.part_a, pr.n_part_a, pr.k, y) : 0;
-        tb[e] = live ? sum_parts_at(pr.part_b, pr.n_part_b, pr.k, y) : 0;
+        for (int e = tid; e < L; e += SUMCHECK_THREADS) {
+            const int y = (e / W) * F + c * W + (e % W);
+            const bool live = y < pr.k;                    // entries past k are the zero padding
+            ta[e] = live ? sum_parts_at(pr.part_a, pr.n_part_a, pr.k, y) : 0;
+            tb[e] = live ? sum_parts_at(pr.part_b, pr.n_part_b, pr.k, y) : 0;
+        }
     }
     __syncthreads();
     run_rounds(sh, ta, tb, L, 0, J);
@@ -844,7 +885,7 @@ __global__ void __launch_bounds__(2 * FS_POINT_SLOTS) fs_points_kernel(const Pro
 __global__ void __launch_bounds__(FS_THREADS)
 sumcheck_fs_kernel(const ProofDev* proofs, const FsProof* fs, imm_fe* transcripts, int64_t stride, int32_t* status)
 {
-    __shared__ uint64_t red[33];
+    __shared__ uint64_t red[35];
     __shared__ uint64_t red3[3][32];
     __shared__ uint64_t r_sh;
     const ProofDev pr = proofs[blockIdx.x];
@@ -858,14 +899,7 @@ sumcheck_fs_kernel(const ProofDev* proofs, const FsProof* fs, imm_fe* transcript
     uint64_t s = 0;
     for (int i = tid; i < pr.n_part_c; i += FS_THREADS) s = gl::add(s, pr.part_c[i]);
     s = block_sum_fe(s, red);
-    if (pr.c_offset) {
-        uint64_t sr = 0, sc = 0;
-        for (int i = tid; i < pr.n_sum_row; i += FS_THREADS) sr = gl::add(sr, pr.sum_row[i]);
-        for (int i = tid; i < pr.n_sum_col; i += FS_THREADS) sc = gl::add(sc, pr.sum_col[i]);
-        sr = block_sum_fe(sr, red);
-        sc = block_sum_fe(sc, red);
-        s = gl::sub(s, gl::shl(gl::mul(sr, sc), 31));
-    }
+    s = gl::sub(s, claim_offset_block(pr, red));
     uint32_t st[8];                                        // the transcript state (thread 0)
     if (tid == 0) {
         tr[0] = s;
@@ -973,7 +1007,7 @@ __global__ void __launch_bounds__(FS_BATCH_MAX) fsb_seed_kernel(const FsProof* f
 __global__ void __launch_bounds__(FS_THREADS)
 fsb_build_kernel(const ProofDev* proofs, const FsProof* fs, FsBatch fb, imm_fe* tr, int32_t* status)
 {
-    __shared__ uint64_t red[33];
+    __shared__ uint64_t red[35];
     __shared__ uint64_t red3[3][32];
     const int p = blockIdx.x, tid = threadIdx.x, b = fb.b;
     const ProofDev pr = proofs[p];
@@ -982,14 +1016,7 @@ fsb_build_kernel(const ProofDev* proofs, const FsProof* fs, FsBatch fb, imm_fe* 
     uint64_t s = 0;
     for (int i = tid; i < pr.n_part_c; i += FS_THREADS) s = gl::add(s, pr.part_c[i]);
     s = block_sum_fe(s, red);
-    if (pr.c_offset) {
-        uint64_t sr = 0, sc = 0;
-        for (int i = tid; i < pr.n_sum_row; i += FS_THREADS) sr = gl::add(sr, pr.sum_row[i]);
-        for (int i = tid; i < pr.n_sum_col; i += FS_THREADS) sc = gl::add(sc, pr.sum_col[i]);
-        sr = block_sum_fe(sr, red);
-        sc = block_sum_fe(sc, red);
-        s = gl::sub(s, gl::shl(gl::mul(sr, sc), 31));
-    }
+    s = gl::sub(s, claim_offset_block(pr, red));
     const int n0 = 1 << b;
     for (int y = tid; y < n0; y += FS_THREADS) {
         const bool live = y < pr.k;
@@ -1096,21 +1123,14 @@ fsb_fold_kernel(const FsProof* fs, FsBatch fb, int j, imm_fe* tr)
 __global__ void __launch_bounds__(SUMCHECK_THREADS)
 expected_kernel(const ProofDev* proofs, const ExpectDev* ex, imm_fe* expected, int32_t* status)
 {
-    __shared__ uint64_t red[33];
+    __shared__ uint64_t red[35];
     const ProofDev pr = proofs[blockIdx.x];
     const imm_fe* e_k = ex[blockIdx.x].e_k;
     const int tid = threadIdx.x;
     uint64_t s = 0;
     for (int i = tid; i < pr.n_part_c; i += SUMCHECK_THREADS) s = gl::add(s, pr.part_c[i]);
     s = block_sum_fe(s, red);
-    if (pr.c_offset) {                                     // the byte-wise claim kernel read every entry 2^31 too high
-        uint64_t sr = 0, sc = 0;
-        for (int i = tid; i < pr.n_sum_row; i += SUMCHECK_THREADS) sr = gl::add(sr, pr.sum_row[i]);
-        for (int i = tid; i < pr.n_sum_col; i += SUMCHECK_THREADS) sc = gl::add(sc, pr.sum_col[i]);
-        sr = block_sum_fe(sr, red);
-        sc = block_sum_fe(sc, red);
-        s = gl::sub(s, gl::shl(gl::mul(sr, sc), 31));
-    }
+    s = gl::sub(s, claim_offset_block(pr, red));           // the byte-wise claim kernel read every entry 2^31 too high
     uint64_t a = 0, b = 0;
     for (int y = tid; y < pr.k; y += SUMCHECK_THREADS) {   // entries past k meet the zero padding
         const uint64_t w = e_k[y];
@@ -1313,8 +1333,36 @@ cudaError_t launch_combine(const imm_fe* tr, int64_t stride, int nproofs, int b,
     return cudaGetLastError();
 }
 
+cudaError_t launch_fused_contract(const FusedJob* d_jobs, const FusedSeg* d_segs, const uint32_t* d_block_first,
+                                  uint32_t nblocks, cudaStream_t st)
+{
+    if (nblocks == 0) return cudaSuccess;
+    fused_contract_kernel<<<nblocks, BYTEDOT_THREADS, 0, st>>>(d_jobs, d_segs, d_block_first);
+    return cudaGetLastError();
+}
+
+// Launched as a programmatic dependent of the kernel before it in the stream: it may start while that
+// one drains and waits (griddepcontrol.wait) before it reads its results.
+cudaError_t launch_reduce_parts(const ProofDev* d_proofs, int nproofs, int max_b, cudaStream_t st)
+{
+    if (nproofs <= 0) return cudaSuccess;
+    const int n0 = 1 << (max_b > 0 ? max_b : 0);
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3((unsigned)((n0 + REDUCE_THREADS - 1) / REDUCE_THREADS + 1), (unsigned)nproofs);
+    cfg.blockDim = dim3(REDUCE_THREADS);
+    cfg.stream = st;
+    cudaLaunchAttribute attr;
+    memset(&attr, 0, sizeof(attr));
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, reduce_parts_kernel, d_proofs);
+}
+
 cudaError_t launch_sumcheck(const ProofDev* d_proofs, int nproofs, uint64_t seed, imm_fe* transcripts,
-                            int64_t stride, int32_t* status, int max_b, int cluster, cudaStream_t st)
+                            int64_t stride, int32_t* status, int max_b, int cluster, bool dependent, cudaStream_t st)
 {
     if (nproofs <= 0) return cudaSuccess;
     // Blocks per proof: as many as keep every proof of the batch resident at once (two blocks fit
@@ -1343,14 +1391,16 @@ cudaError_t launch_sumcheck(const ProofDev* d_proofs, int nproofs, uint64_t seed
     cfg.blockDim = dim3(SUMCHECK_THREADS);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
-    cudaLaunchAttribute attr;
-    memset(&attr, 0, sizeof(attr));
-    attr.id = cudaLaunchAttributeClusterDimension;
-    attr.val.clusterDim.x = (unsigned)nc;
-    attr.val.clusterDim.y = 1;
-    attr.val.clusterDim.z = 1;
-    cfg.attrs = &attr;
-    cfg.numAttrs = 1;
+    cudaLaunchAttribute attr[2];
+    memset(attr, 0, sizeof(attr));
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)nc;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;       // see launch_reduce_parts
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = dependent ? 2 : 1;
     return cudaLaunchKernelEx(&cfg, sumcheck_kernel, d_proofs, seed, transcripts, stride, status, (int)cap);
 }
 

@@ -29,9 +29,16 @@ cudaError_t launch_sum_all(const imm_fe* parts, int64_t count, imm_fe* out, cuda
 // sum of the partial sums of a tensor-core point evaluation, minus the 2^31 offset of an int32 matrix (nsr > 0)
 cudaError_t launch_point_finish(const imm_fe* parts, int64_t count, const imm_fe* sum_row, int nsr,
                                 const imm_fe* sum_col, int nsc, imm_fe* out, cudaStream_t st);
-// cluster: blocks per proof (1, 2, 4 or 8), or 0 to let the launch choose from the batch size
+// cluster: blocks per proof (1, 2, 4 or 8), or 0 to let the launch choose from the batch size;
+// dependent: launched as a programmatic dependent of the kernel before it (reduce_parts_kernel)
 cudaError_t launch_sumcheck(const ProofDev* d_proofs, int nproofs, uint64_t seed, imm_fe* transcripts,
-                            int64_t stride, int32_t* status, int max_b, int cluster, cudaStream_t st);
+                            int64_t stride, int32_t* status, int max_b, int cluster, bool dependent, cudaStream_t st);
+// small batches: all three contractions in one persistent launch (a run of segments per block), the eq
+// weights built inside the blocks
+cudaError_t launch_fused_contract(const FusedJob* d_jobs, const FusedSeg* d_segs, const uint32_t* d_block_first,
+                                  uint32_t nblocks, cudaStream_t st);
+// the round tables and the claim of every proof from the contractions' partial results
+cudaError_t launch_reduce_parts(const ProofDev* d_proofs, int nproofs, int max_b, cudaStream_t st);
 // batched transcript (1 + 3b + 3*nproofs words) from per-proof transcripts proved under shared round challenges
 cudaError_t launch_combine(const imm_fe* tr, int64_t stride, int nproofs, int b, uint64_t seed, uint64_t batch_id,
                            imm_fe* out, cudaStream_t st);

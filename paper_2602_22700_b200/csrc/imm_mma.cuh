@@ -224,27 +224,22 @@ __device__ __forceinline__ void load64(const char* p, int64_t left, uint32_t (&d
     }
 }
 
-template <bool I32, bool POINT, int VL, int MT>
-__device__ __forceinline__ void bytedot_tile(const MatJob& job, uint32_t local, uint4* sW)
+// Rows [r0, r1) of column chunk cci of one matrix, by one block: every warp takes 16*MT rows at a
+// time across the chunk's slabs; sW holds the chunk's weight limbs.  POINT: returns this thread's
+// share of sum_row row_weight(row) * u[row] (to be summed over the warp by the caller);
+// otherwise writes u[row] to job.out[cci][row] and returns 0.
+template <bool I32, bool POINT, int VL, int MT, int UNROLL = BYTEDOT_UNROLL, class RowWeight>
+__device__ __forceinline__ uint64_t bytedot_rows(const MatJob& job, int cci, int r0, int r1, const uint4* sW, RowWeight row_weight)
 {
     static_assert(POINT || !I32, "the int32 byte view is offset by 2^31 per entry: point evaluation only");
     using T = typename std::conditional<I32, int32_t, int8_t>::type;
     constexpr int ESZ = (int)sizeof(T);
     constexpr int NWARP = BYTEDOT_THREADS / 32;
-    const int rbi = local / job.ncc, cci = local % job.ncc;
-    const int r0 = rbi * job.tile_rows;
-    const int r1 = min(r0 + job.tile_rows, job.rows);
     const int64_t row_bytes = (int64_t)job.cols * ESZ;
     const int64_t cb0 = (int64_t)cci * job.chunk;
     const int nslab = (int)min((int64_t)(job.chunk / 256), (row_bytes - cb0 + 255) / 256);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int g = lane >> 2, t = lane & 3;
-
-    const uint4* wsrc = reinterpret_cast<const uint4*>(job.wtab) + (cb0 / 256) * 128;
-    for (int i = threadIdx.x; i < nslab * 128; i += BYTEDOT_THREADS) sW[i] = wsrc[i];
-
-    __syncthreads();
-
     const int64_t pitch = job.ld * (int64_t)ESZ;
     uint64_t part = 0;
     for (int rg = r0 + warp * (16 * MT); rg < r1; rg += NWARP * (16 * MT)) {
@@ -260,7 +255,7 @@ __device__ __forceinline__ void bytedot_tile(const MatJob& job, uint32_t local, 
                 p[mt][h] = (const char*)job.mat + (int64_t)row * pitch + cb0 + 64 * t;
             }
         }
-#pragma unroll BYTEDOT_UNROLL
+#pragma unroll UNROLL
         for (int s = 0; s < nslab; s++) {
             const int64_t left = row_bytes - (cb0 + 256 * s + 64 * t);    // bytes of the row from this thread's piece on
             uint32_t d[MT][2][16];
@@ -286,21 +281,43 @@ __device__ __forceinline__ void bytedot_tile(const MatJob& job, uint32_t local, 
                 }
             }
         }
+        // every lane of a group of four holds u; the rows' products (or stores) are shared out over the four
 #pragma unroll
         for (int mt = 0; mt < MT; mt++)
 #pragma unroll
             for (int h = 0; h < 2; h++) {
                 const int row = rg + 16 * mt + g + 8 * h;
                 uint64_t u = combine_limbs(acc[mt][2 * h], acc[mt][2 * h + 1], t);
-                if (t == 0 && row < r1) {
-                    if (POINT) part = gl::add(part, gl::mul(job.eq_row[row], u));
+                if (t == ((2 * mt + h) & 3) && row < r1) {
+                    if (POINT) part = gl::add(part, gl::mul(row_weight(row), u));
                     else job.out[(int64_t)cci * job.rows + row] = u;
                 }
             }
     }
+    return part;
+}
+
+// One tile = rows [rbi * tile_rows, ...) of chunk cci: stages the chunk's weight limbs from job.wtab
+// and takes the row weights from job.eq_row.
+template <bool I32, bool POINT, int VL, int MT>
+__device__ __forceinline__ void bytedot_tile(const MatJob& job, uint32_t local, uint4* sW)
+{
+    constexpr int ESZ = I32 ? 4 : 1;
+    constexpr int NWARP = BYTEDOT_THREADS / 32;
+    const int rbi = local / job.ncc, cci = local % job.ncc;
+    const int r0 = rbi * job.tile_rows;
+    const int r1 = min(r0 + job.tile_rows, job.rows);
+    const int64_t row_bytes = (int64_t)job.cols * ESZ;
+    const int64_t cb0 = (int64_t)cci * job.chunk;
+    const int nslab = (int)min((int64_t)(job.chunk / 256), (row_bytes - cb0 + 255) / 256);
+    const uint4* wsrc = reinterpret_cast<const uint4*>(job.wtab) + (cb0 / 256) * 128;
+    for (int i = threadIdx.x; i < nslab * 128; i += BYTEDOT_THREADS) sW[i] = wsrc[i];
+    __syncthreads();
+    const imm_fe* erow = job.eq_row;
+    uint64_t part = bytedot_rows<I32, POINT, VL, MT, BYTEDOT_UNROLL>(job, cci, r0, r1, sW, [erow](int row) { return erow[row]; });
     if (POINT) {                               // one partial per warp: no block barrier at the end of a tile
         part = warp_sum_fe(part);
-        if (lane == 0) job.out[(int64_t)local * NWARP + warp] = part;
+        if ((threadIdx.x & 31) == 0) job.out[(int64_t)local * NWARP + (threadIdx.x >> 5)] = part;
     }
 }
 
@@ -327,7 +344,9 @@ __global__ void __launch_bounds__(BYTEDOT_THREADS, MT == 1 ? 3 : 2) bytedot_kern
 // rows.  One tile = tile_rows rows x (128 columns per warp of the block); the block size is chosen
 // per batch (8 warps for large inputs, fewer so that small ones still spread over all SMs).
 
-template <bool VEC>
+// STAGE: copy the tile's weight limbs from job.wtab into sR; otherwise the caller has filled sR
+// (and synchronised).
+template <bool VEC, bool STAGE = true>
 __device__ __forceinline__ void rowmma_tile(const MatJob& job, uint32_t local, uint2* sR)
 {
     const int rbi = local / job.ncc, cci = local % job.ncc;
@@ -337,9 +356,11 @@ __device__ __forceinline__ void rowmma_tile(const MatJob& job, uint32_t local, u
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int g = lane >> 2, t = lane & 3;
 
-    const uint2* wsrc = reinterpret_cast<const uint2*>(job.wtab) + (int64_t)(r0 / 32) * 32;
-    for (int i = threadIdx.x; i < ngroups * 32; i += blockDim.x) sR[i] = wsrc[i];
-    __syncthreads();
+    if (STAGE) {
+        const uint2* wsrc = reinterpret_cast<const uint2*>(job.wtab) + (int64_t)(r0 / 32) * 32;
+        for (int i = threadIdx.x; i < ngroups * 32; i += blockDim.x) sR[i] = wsrc[i];
+        __syncthreads();
+    }
 
     const int tile_cols = (int)blockDim.x * 4;                    // 128 columns per warp
     const int col = cci * tile_cols + warp * 128 + 16 * g;        // this thread's 16 columns

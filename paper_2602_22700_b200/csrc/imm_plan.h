@@ -32,6 +32,10 @@ constexpr int ROWMMA_MAX_WARPS = 8;            // a block of w warps covers w x 
 constexpr int ROWLDM_STAGES = 4;               // shared-memory stages per warp of the row-binding kernel
 constexpr int ROWLDM_PITCH = 144;              // bytes per staged row: 128 of data, 16 of padding
 constexpr int ROWLDM_STAGE_BYTES = 32 * ROWLDM_PITCH;
+#ifndef IMM_FUSED_BLOCKS
+#define IMM_FUSED_BLOCKS 3
+#endif
+constexpr int FUSED_BLOCKS_PER_SM = IMM_FUSED_BLOCKS;         // resident blocks per SM of the fused contraction launch
 constexpr int EQ_BATCH_THREADS = 256;
 constexpr int EQ_SLICE_QUADS = 512;           // groups of four table entries per block of eq_batch_kernel
 constexpr int SUMCHECK_THREADS = 512;
@@ -58,6 +62,27 @@ struct MatJob {
     int32_t chunk;             // byte-dot kernel: byte-columns per tile (multiple of 256)
 };
 
+// Fused launch (small batches): one persistent grid over all three matrix kinds.  The work is a
+// sequence of segments -- a tile of A, or rows [r0, r1) of one column chunk of B or C -- cut on the
+// host into one contiguous run per block with equal bytes, so that all blocks finish together.  The
+// blocks build the eq weights they need from the challenges: no eq table or limb table is in memory.
+struct FusedJob {
+    MatJob mj;                 // matrix, geometry, output (wtab / eq_row / eq_col unused).  A: tile_rows x 1024-column
+                               // tiles, out[nrb][cols]; B: chunk, ncc, out[ncc][rows]; C: chunk, ncc, out[segments * 8]
+    uint64_t seed, proof_id;   // r_row = challenge(seed, proof_id, 1, .), r_col = challenge(seed, proof_id, 2, .)
+    const imm_fe* pt_row;      // non-null: r_row is read from here (a variables) instead of the generator
+    const imm_fe* pt_col;      // non-null: r_col likewise (c variables)
+    int32_t kind;              // JobKind: ROWBIND = A (int8), COLBIND = B (int8), POINT = C (int32)
+    int32_t a, c;              // variables of this matrix's row / column index
+    int32_t seg0;              // C: its first segment (a segment's eight warp partials go to out[(seg - seg0) * 8 ..])
+};
+
+struct FusedSeg {
+    int32_t job;               // index into the FusedJob list
+    int32_t cci;               // B, C: column chunk;  A: tile index within the job (row block * ncc + column block)
+    int32_t r0, r1;            // B, C: rows [r0, r1)
+};
+
 // Per-proof state of the round kernel.
 struct ProofDev {
     imm_fe* e_row;             // 2^a entries
@@ -72,8 +97,16 @@ struct ProofDev {
     int32_t m, k, n;
     int32_t a, b, c;           // ceil(log2 m), ceil(log2 k), ceil(log2 n)
     int32_t n_part_a, n_part_b, n_part_c;
-    int32_t c_offset;          // 1: c0 = sum(part_c) - 2^31 * sum(sum_row) * sum(sum_col)
+    int32_t c_offset;          // 1: c0 = sum(part_c) - 2^31 * (sum of E_row over the real rows) * (sum of E_col over the
+                               //    real columns); the two sums come from sum_row / sum_col, or, where those are
+                               //    null, from the challenges in closed form
     int32_t n_sum_row, n_sum_col;
+    uint64_t seed, proof_id;   // the proof's own coins (r_row, r_col), for the closed form
+    const imm_fe* pt_row;      // non-null: r_row / r_col are read from here instead of the generator
+    const imm_fe* pt_col;
+    imm_fe* tab;               // non-null: [2][2^b] both round tables, summed over the partial vectors and zero-padded
+                               //           by reduce_parts_kernel, which also leaves the claim in c0_ready
+    imm_fe* c0_ready;
 };
 
 // One eq table of a batch: r is derived in-kernel from (seed, proof_id, domain).  The same pass

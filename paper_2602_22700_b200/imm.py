@@ -37,7 +37,7 @@ EXPORTS = ("imm_version", "imm_last_cuda_error", "imm_challenge", "imm_field_bin
            "imm_sumcheck_matmul_fs_workspace", "imm_sumcheck_matmul_prove_fs", "imm_fs_challenges",
            "imm_sumcheck_verify_fs", "imm_sumcheck_expected_workspace", "imm_sumcheck_expected",
            "imm_sumcheck_matmul_fs_batched_workspace", "imm_sumcheck_matmul_prove_fs_batched",
-           "imm_fs_batched_challenges", "imm_sumcheck_verify_fs_batched", "imm_requant_check")
+           "imm_fs_batched_challenges", "imm_sumcheck_verify_fs_batched", "imm_requant_check", "imm_sumcheck_matmul_launches")
 FS_BATCH_MAX = 1024
 COMMIT_LEAF = 4096
 NOALLOC_MAX_TILES = 8192
@@ -149,6 +149,8 @@ def lib() -> ctypes.CDLL:
     L.imm_commit.argtypes = [vp, ci, vp, vp, vp, sz, vp]
     L.imm_sumcheck_verify_batched.restype = ci
     L.imm_sumcheck_verify_batched.argtypes = [vp, ci, ci, u64, u64, vp, vp]
+    L.imm_sumcheck_matmul_launches.restype = ci
+    L.imm_sumcheck_matmul_launches.argtypes = [vp, ci]
     L.imm_requant_check.restype = ci
     L.imm_requant_check.argtypes = [vp, vp, i64, i64, i64, i64, ci, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp, vp]
     _lib = L
@@ -302,6 +304,7 @@ class Prover:
         self.ws = torch.empty(need, dtype=torch.uint8, device=device)
         self.transcripts = torch.zeros((self.nproofs, self.stride), dtype=torch.int64, device=device)
         self.status = torch.full((self.nproofs,), -99, dtype=torch.int32, device=device)
+        self.launches = lib().imm_sumcheck_matmul_launches(ctypes.addressof(self.descs), self.nproofs)
 
     def prove(self, seed: int) -> torch.Tensor:
         """Enqueue one proving pass on the current stream; returns the device transcript tensor."""

@@ -289,7 +289,8 @@ COMMIT_TRAFFIC_RATIO = (1.077891 + 0.018910) / 1.050673152                   # c
 # byte (ncu: 564.2 M warp instructions on that pipe for 1.0507 GB), so at 1965 MHz the pipe allows
 # 148 x 64 x 1.965e9 / 17.18 = 1083 GB/s.
 COMMIT_ALU_PEAK_GBS_AT_1965 = 1083.0
-GLUE_TRAFFIC_RATIO = None        # requant_check_kernel: (dram read + write) / (5 bytes per entry); None until captured
+GLUE_TRAFFIC_RATIO = (146.819072 + 3.869952) / 146.80064    # requant_check_kernel: (dram read + write) / (5 bytes per entry), 2048-token capture
+FUSED_TRAFFIC_RATIO = (308.909568 + 12.264448) / 306.184192   # fused_contract_kernel: (dram read + write) / algorithmic bytes, FFN-pair capture
 CLAIM_KERNEL_TRAFFIC_RATIO = 239.64 / 234.881024  # bytedot_kernel<1,1,1>: (dram read + write) / (4 bytes per entry), small-case capture
 
 
@@ -495,10 +496,9 @@ def run_ours(args):
                      "frac_of_8tbs": claim_gbs / 8000.0,
                      # achieved GB/s per sampled SM MHz: comparable across pods whose clocks differ
                      "gbs_per_sm_mhz": (claim_gbs / clocks["sm_mhz"]) if clocks and clocks.get("sm_mhz") else None,
-                     "traffic": (CLAIM_KERNEL_TRAFFIC_RATIO * claim_bytes) if (CLAIM_KERNEL_TRAFFIC_RATIO and not fused) else None},
+                     "traffic": (FUSED_TRAFFIC_RATIO if fused else CLAIM_KERNEL_TRAFFIC_RATIO) * claim_bytes},
         "phase_steps": psteps,
-        "gpu_launches": ((fsp.launches + com.launches) if (args.fs and args.batched) else (6 + com.launches) if args.fs
-                         else 6 if (args.batched or args.verify) else prover.launches) * calls_per_step * steps,
+        "gpu_launches": ((fsp.launches + com.launches) if args.fs else sum(pv.launches for pv in provers)) * steps,
         "transcript_words_per_step": (int(fsp.length) if (args.fs and args.batched) else
                                       sum(int(bp.length) for bp in provers) if args.batched else
                                       sum(3 * imm.ceil_log2(k) + 3 for (m, k, n) in shapes)),

@@ -289,6 +289,13 @@ def sumcheck_matmul_workspace(descs) -> int:
     return lib().imm_sumcheck_matmul_workspace(ctypes.addressof(descs), len(descs))
 
 
+def _launch_counts(descs) -> Tuple[int, int]:
+    """(launches of a plain proving pass, launches of its contraction side alone) for this batch: 3 and 1
+    when it takes the fused contraction launch, else 5 and 4 (eq tables + three contractions)."""
+    plain = lib().imm_sumcheck_matmul_launches(ctypes.addressof(descs), len(descs))
+    return plain, (1 if plain == 3 else 4)
+
+
 class Prover:
     """Holds the descriptor array, workspace and output buffers of one batch so that repeated
     ``prove`` calls do no allocation.  ``problems``: list of (A, B, C, proof_id) CUDA tensors."""
@@ -304,7 +311,7 @@ class Prover:
         self.ws = torch.empty(need, dtype=torch.uint8, device=device)
         self.transcripts = torch.zeros((self.nproofs, self.stride), dtype=torch.int64, device=device)
         self.status = torch.full((self.nproofs,), -99, dtype=torch.int32, device=device)
-        self.launches = lib().imm_sumcheck_matmul_launches(ctypes.addressof(self.descs), self.nproofs)
+        self.launches = _launch_counts(self.descs)[0]
 
     def prove(self, seed: int) -> torch.Tensor:
         """Enqueue one proving pass on the current stream; returns the device transcript tensor."""
@@ -417,6 +424,7 @@ class BatchedProver:
         self.length = batched_transcript_len(self.nrounds, self.nproofs)
         self.transcript = torch.zeros((self.length,), dtype=torch.int64, device=device)
         self.status = torch.full((self.nproofs,), -99, dtype=torch.int32, device=device)
+        self.launches = _launch_counts(self.descs)[0] + 1        # ... and the combining launch
 
     def prove(self, seed: int, batch_id: int) -> torch.Tensor:
         """Enqueue one batched proving pass on the current stream; returns the device transcript."""
@@ -542,6 +550,7 @@ class FsProver:
         self.ws = torch.empty(need, dtype=torch.uint8, device=device)
         self.transcripts = torch.zeros((self.nproofs, self.stride), dtype=torch.int64, device=device)
         self.status = torch.full((self.nproofs,), -99, dtype=torch.int32, device=device)
+        self.launches = _launch_counts(self.descs)[1] + 2        # statements, contractions, hashed rounds
 
     def prove(self) -> torch.Tensor:
         _check(lib().imm_sumcheck_matmul_prove_fs(ctypes.addressof(self.descs), self.nproofs,
@@ -631,7 +640,7 @@ class FsBatchedProver:
         self.length = batched_transcript_len(self.nrounds, self.nproofs)
         self.transcript = torch.zeros((self.length,), dtype=torch.int64, device=device)
         self.status = torch.full((self.nproofs,), -99, dtype=torch.int32, device=device)
-        self.launches = 6 + 3 + 2 * self.nrounds            # statements, eq, three contractions ... and the round chain
+        self.launches = _launch_counts(self.descs)[1] + 1 + 3 + 2 * self.nrounds     # statements, contractions, the round chain
 
     def prove(self, batch_id: int) -> torch.Tensor:
         _check(lib().imm_sumcheck_matmul_prove_fs_batched(ctypes.addressof(self.descs), self.nproofs,
@@ -727,6 +736,7 @@ class Verifier:
         self.ws = torch.empty(need, dtype=torch.uint8, device=device)
         self.values = torch.zeros((self.nproofs, 3), dtype=torch.int64, device=device)
         self.status = torch.full((self.nproofs,), -99, dtype=torch.int32, device=device)
+        self.launches = _launch_counts(self.descs)[1] + 2        # E_k tables, contractions, the inner products
 
     def expected(self, seed: int = 0, batch_id: Optional[int] = None, points=None) -> torch.Tensor:
         """Enqueue the pass on the current stream; returns the (nproofs, 3) device tensor.  ``points``:

@@ -12,7 +12,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libimm.so")
 SOURCES = ["imm_kernels.cu", "imm_api.cu", "imm_ldd.cu", "imm_commit.cu", "imm_glue.cu"]
-DEPS = SOURCES + ["sha256.cuh", "gl64.cuh", "imm_plan.h", "imm_kernels.h", "imm_mma.cuh", os.path.join("..", "..", "include", "imm.h")]
+DEPS = SOURCES + ["sha256.cuh", "gl64.cuh", "imm_plan.h", "imm_kernels.h", "imm_mma.cuh", "imm_fused.cuh", os.path.join("..", "..", "include", "imm.h")]
 
 
 def _nvcc() -> str:

@@ -24,6 +24,11 @@ __device__ __forceinline__ uint64_t shfl_xor_u64(uint64_t v, int mask)
     return __shfl_xor_sync(0xFFFFFFFFu, v, mask);
 }
 
+__device__ __forceinline__ uint64_t shfl_idx_u64(uint64_t v, int src_lane)
+{
+    return __shfl_sync(0xFFFFFFFFu, v, src_lane);
+}
+
 __device__ __forceinline__ uint64_t warp_sum_fe(uint64_t v)
 {
 #pragma unroll
@@ -493,14 +498,14 @@ point_finish_kernel(const imm_fe* parts, int64_t count, const imm_fe* sum_row, i
 //
 // Three facts shape the kernel.  (1) Challenges are public coins, so nothing waits for a round
 // polynomial: a pass folds with r_j AND accumulates round j+1's three sums from the values it
-// has just produced (a thread folds the two pairs that form one pair of the next round), and the
-// partial sums of every round are reduced once, after the last round, not once per round:
-// a round costs one barrier.  (2) Rounds bind the index from its top bit down, so the first
+// has just produced (four lanes fold the two pairs that form one pair of the next round, one value
+// each, and share them by shuffle), and the partial sums of every round are reduced once, after
+// the last round, not once per round: a round costs one barrier.  (2) Rounds bind the index from its top bit down, so the first
 // J = b - 8 rounds never mix entries whose low 8 index bits differ: block c of the cluster owns
 // the entries whose low bits fall in its slice of 256 / (cluster size) values, runs those J
-// rounds on its own shared-memory tables, and hands its slice of the 256-entry folded tables
-// plus its partial sums to block 0 over distributed shared memory; block 0 runs the last 8
-// rounds.  (3) Field addition is exact, so the order of these reductions does not change a word.
+// rounds on its own shared-memory tables, and stores its slice of the 256-entry folded tables
+// plus its partial sums into block 0's shared memory (one cluster barrier); block 0 runs the last
+// 8 rounds.  (3) Field addition is exact, so the order of these reductions does not change a word.
 // The cluster size is chosen per launch: small batches spread each proof over 8 SMs, large ones
 // keep one or two blocks per proof so that all proofs run at once.  Proofs of at most
 // SC_SOLO_VARS rounds are done by block 0 alone.
@@ -579,27 +584,17 @@ struct ScShared {
     uint64_t r[MAX_K_VARS];                    // round challenges
     uint64_t warp_sums[MAX_K_VARS][SC_WARPS][3];   // sums of a round whose pass ran on several warps
     uint64_t lane_sums[MAX_K_VARS][32][3];     // sums of a round whose pass ran on warp 0 alone (not yet reduced)
-    uint64_t block_sums[MAX_K_VARS][3];        // this block's share of g_j(0..2); read by block 0
-    uint64_t fin[2][SC_FINAL];                 // block 0: the gathered 256-entry tables
+    uint64_t block_sums[MAX_K_VARS][3];        // sums of the rounds a block ran alone
+    uint64_t gather[SUMCHECK_MAX_CLUSTER][MAX_K_VARS * 3];   // block 0: every block's share of the local rounds' sums
+    uint64_t fin[2][SC_FINAL];                 // block 0: the 256-entry tables, written by their owners
     uint64_t red[SC_WARPS];
 };
 
-// Keep a pass's sums of round j: `q` is the number of threads the pass used.  Both arrays start
-// at zero and every slot is written at most once.
-__device__ __forceinline__ void stash_sums(ScShared& sh, int j, const Sums3& acc, int q)
-{
-    const int tid = threadIdx.x;
-    if (q <= 32) {
-        if (tid < 32) { uint64_t* w = sh.lane_sums[j][tid]; w[0] = acc.g0; w[1] = acc.g1; w[2] = acc.g2; }
-    } else if ((tid & ~31) < q) {
-        const uint64_t g0 = warp_sum_fe(acc.g0), g1 = warp_sum_fe(acc.g1), g2 = warp_sum_fe(acc.g2);
-        if ((tid & 31) == 0) { uint64_t* w = sh.warp_sums[j][tid >> 5]; w[0] = g0; w[1] = g1; w[2] = g2; }
-    }
-}
-
-// block_sums[j] = all stashed sums of round j, for j in [j0, j1); one warp per round.  Callers
-// put a block barrier before (stashes visible) and after (results visible).
-__device__ __forceinline__ void reduce_round_sums(ScShared& sh, int j0, int j1)
+// dst[3 j + comp] = all stashed sums of round j, for j in [j0, j1); one warp per round.  Callers
+// put a block barrier before (stashes visible) and a barrier after (results visible); dst may lie in
+// another block of the cluster.  (Not inlined, like run_rounds: the kernel is short enough for cold
+// instruction fetches to show, so both stages of a proof share one copy of the code.)
+__device__ __noinline__ void reduce_round_sums(ScShared& sh, int j0, int j1, uint64_t* dst)
 {
     const int lane = threadIdx.x & 31;
     for (int j = j0 + (threadIdx.x >> 5); j < j1; j += SC_WARPS) {
@@ -608,45 +603,85 @@ __device__ __forceinline__ void reduce_round_sums(ScShared& sh, int j0, int j1)
             uint64_t v = sh.lane_sums[j][lane][comp];
             if (lane < SC_WARPS) v = gl::add(v, sh.warp_sums[j][lane][comp]);
             v = warp_sum_fe(v);
-            if (lane == 0) sh.block_sums[j][comp] = v;
+            if (lane == 0) dst[3 * j + comp] = v;
         }
     }
+}
+
+// A pass is bound by the latency of a thread's chain of field multiplications (the carry flag
+// serialises them), not by issue slots, and the kernel is short enough for the size of its code to
+// show as cold instruction fetches.  So there is ONE form of pass, spread over four lanes per pair
+// of entry pairs: lane role 0..3 folds one of a0, a1, b0, b1, the four exchange their results by
+// shuffle, and roles 0..2 form one product each -- two multiplications deep.  A lane keeps ONE sum
+// (component `role` of the round's sums).
+constexpr int SC_QUADS = SUMCHECK_THREADS / 4;             // quads (or pairs, in the first pass) per sweep of the block
+
+// Keep a pass's sums of round j; `nthreads` (a multiple of 4, at most the block) threads took part.
+// Both arrays start at zero and every slot is written at most once per walk over the rounds.
+__device__ __forceinline__ void stash_sums(ScShared& sh, int j, uint64_t acc, int nthreads)
+{
+    const int tid = threadIdx.x, lane = tid & 31, role = tid & 3;
+    if (nthreads <= 32) {
+        if (tid < 32 && role < 3) sh.lane_sums[j][lane][role] = acc;
+    } else if ((tid & ~31) < nthreads) {
+#pragma unroll
+        for (int o = 4; o < 32; o <<= 1) acc = gl::add(acc, shfl_xor_u64(acc, o));
+        if (lane < 3) sh.warp_sums[j][tid >> 5][lane] = acc;
+    }
+}
+
+// the product a lane owes: g(0) = a0 b0, g(1) = a1 b1, g(2) = (2 a1 - a0)(2 b1 - b0)
+__device__ __forceinline__ uint64_t role_product(int role, uint64_t a0, uint64_t a1, uint64_t b0, uint64_t b1)
+{
+    const uint64_t x = role == 0 ? a0 : role == 1 ? a1 : gl::sub(gl::add(a1, a1), a0);
+    const uint64_t y = role == 0 ? b0 : role == 1 ? b1 : gl::sub(gl::add(b1, b1), b0);
+    return gl::mul(x, y);
 }
 
 // Rounds j0..j1-1 on shared-memory tables of n entries each: one pass for round j0's sums, then
 // pass j folds with r_j and accumulates round j+1's sums while j+1 < j1.  Every thread of the
 // block calls this, after a block barrier that made the tables visible.  A pass whose writers
 // all sit in warp 0 is followed by a warp barrier only (its readers sit in warp 0 too).
-__device__ __forceinline__ void run_rounds(ScShared& sh, uint64_t* ta, uint64_t* tb, int n, int j0, int j1)
+// (Not inlined: both stages of a proof share one copy of the code.)
+__device__ __noinline__ void run_rounds(ScShared& sh, uint64_t* ta, uint64_t* tb, int n, int j0, int j1)
 {
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, role = tid & 3;
     if (j0 >= j1) return;
     {
         const int h = n >> 1;
-        Sums3 acc = {0, 0, 0};
-#pragma unroll 1
-        for (int e = tid; e < h; e += SUMCHECK_THREADS) sums_add(acc, ta[e], ta[e + h], tb[e], tb[e + h]);
-        stash_sums(sh, j0, acc, h);
+        uint64_t acc = 0;
+        if (role < 3)
+            for (int e = tid >> 2; e < h; e += SC_QUADS) acc = gl::add(acc, role_product(role, ta[e], ta[e + h], tb[e], tb[e + h]));
+        stash_sums(sh, j0, acc, min(4 * h, SUMCHECK_THREADS));
     }
 #pragma unroll 1
     for (int j = j0; j < j1; j++, n >>= 1) {
         const uint64_t r = sh.r[j];
         const int h = n >> 1, q = n >> 2;
+        const bool next = j + 1 < j1;
+        const int writers = min(4 * q, SUMCHECK_THREADS);  // threads that write table entries in this pass
         if (n == 2) {
-            if (tid == 0) { ta[0] = fold1(ta[0], ta[1], r); tb[0] = fold1(tb[0], tb[1], r); }
-        } else {
-            const bool next = j + 1 < j1;
-            Sums3 acc = {0, 0, 0};
+            if (tid < 2) { uint64_t* t = tid ? tb : ta; t[0] = fold1(t[0], t[1], r); }
+        } else if ((tid & ~31) < writers) {                // whole warps: the shuffles below need every lane
+            uint64_t* t = role < 2 ? ta : tb;
+            const int shift = (role & 1) * q;              // roles 0, 2: entry e; roles 1, 3: entry e + q
+            const int base = tid & 28;                     // the quad's first lane
+            uint64_t acc = 0;
 #pragma unroll 1
-            for (int e = tid; e < q; e += SUMCHECK_THREADS) {
-                const uint64_t fa0 = fold1(ta[e], ta[e + h], r), fa1 = fold1(ta[e + q], ta[e + q + h], r);
-                const uint64_t fb0 = fold1(tb[e], tb[e + h], r), fb1 = fold1(tb[e + q], tb[e + q + h], r);
-                ta[e] = fa0; ta[e + q] = fa1; tb[e] = fb0; tb[e + q] = fb1;      // in place: only this thread reads them
-                if (next) sums_add(acc, fa0, fa1, fb0, fb1);
+            for (int e0 = 0; e0 < q; e0 += SC_QUADS) {
+                const bool live = e0 + (tid >> 2) < q;     // (q < 8 leaves lanes of warp 0 without a quad)
+                const int at = (live ? e0 + (tid >> 2) : q - 1) + shift;
+                const uint64_t f = fold1(t[at], t[at + h], r);
+                if (live) t[at] = f;                       // in place: only this lane reads it
+                if (next) {
+                    const uint64_t fa0 = shfl_idx_u64(f, base), fa1 = shfl_idx_u64(f, base + 1);
+                    const uint64_t fb0 = shfl_idx_u64(f, base + 2), fb1 = shfl_idx_u64(f, base + 3);
+                    if (live && role < 3) acc = gl::add(acc, role_product(role, fa0, fa1, fb0, fb1));
+                }
             }
-            if (next) stash_sums(sh, j + 1, acc, q);
+            if (next) stash_sums(sh, j + 1, acc, writers);
         }
-        if (q > 32) __syncthreads(); else __syncwarp();
+        if (writers > 32) __syncthreads(); else __syncwarp();
     }
 }
 
@@ -678,6 +713,7 @@ sumcheck_kernel(const ProofDev* proofs, uint64_t seed, imm_fe* transcripts, int6
     if (tid < b) sh.r[tid] = gl::challenge(seed, pr.round_id, 3, (uint32_t)tid);
     for (int i = tid; i < MAX_K_VARS * SC_WARPS * 3; i += SUMCHECK_THREADS) (&sh.warp_sums[0][0][0])[i] = 0;
     for (int i = tid; i < MAX_K_VARS * 32 * 3; i += SUMCHECK_THREADS) (&sh.lane_sums[0][0][0])[i] = 0;
+    if (dist) cluster.barrier_arrive();                    // waited for before the first store into block 0's memory
     pdl_wait();                                            // from here on: results of the launches before
     if (pr.tab) {
         // the tables and the claim were finished by reduce_parts_kernel
@@ -727,40 +763,37 @@ sumcheck_kernel(const ProofDev* proofs, uint64_t seed, imm_fe* transcripts, int6
     __syncthreads();
     run_rounds(sh, ta, tb, L, 0, J);
     __syncthreads();
-    reduce_round_sums(sh, 0, J);                           // this block's share of the local rounds' sums
     if (!dist) {
+        reduce_round_sums(sh, 0, J, &sh.block_sums[0][0]);
         __syncthreads();
         if (tid < 3 * b) tr[1 + tid] = (&sh.block_sums[0][0])[tid];
         if (tid == 0) { tr[3 * b + 1] = ta[0]; tr[3 * b + 2] = tb[0]; }
         return;
     }
 
-    cluster.sync();                                        // every block's slice and sums are in place
-    if (c == 0) {
-        for (int i = tid; i < SC_FINAL; i += SUMCHECK_THREADS) {
-            const int cc = i / W, w = i % W;
-            sh.fin[0][i] = cluster.map_shared_rank(ta, cc)[w];
-            sh.fin[1][i] = cluster.map_shared_rank(tb, cc)[w];
+    // every block hands its slice of the folded tables and its share of the sums to block 0 (stores
+    // into block 0's shared memory), then one cluster barrier: block 0 goes on, the others leave
+    cluster.barrier_wait();                                // (arrived at the top) block 0 is running: its memory may be written
+    {
+        ScShared* sh0 = cluster.map_shared_rank(&sh, 0);
+        if (tid < 2 * W) {
+            const int which = tid >= W, w = tid - which * W;
+            sh0->fin[which][c * W + w] = (which ? tb : ta)[w];
         }
-        if (tid < 3 * J) {
-            uint64_t v[SUMCHECK_MAX_CLUSTER];
-#pragma unroll
-            for (int cc = 0; cc < SUMCHECK_MAX_CLUSTER; cc++)
-                v[cc] = cc < nc ? cluster.map_shared_rank(&sh.block_sums[0][0], cc)[tid] : 0;
-            uint64_t s = 0;
-#pragma unroll
-            for (int cc = 0; cc < SUMCHECK_MAX_CLUSTER; cc++) s = gl::add(s, v[cc]);
-            tr[1 + tid] = s;
-        }
+        reduce_round_sums(sh, 0, J, &sh0->gather[c][0]);
     }
-    cluster.sync();                                        // remote reads are done: the other blocks may leave
+    cluster.sync();                                        // release / acquire: the stores above are visible to block 0
     if (c != 0) return;
 
-    // block 0: the remaining rounds on the gathered tables
-    __syncthreads();
+    // block 0: the local rounds' sums, then the remaining rounds on the gathered tables
+    if (tid < 3 * J) {
+        uint64_t v = 0;
+        for (int cc = 0; cc < nc; cc++) v = gl::add(v, sh.gather[cc][tid]);
+        tr[1 + tid] = v;
+    }
     run_rounds(sh, sh.fin[0], sh.fin[1], SC_FINAL, J, b);
     __syncthreads();
-    reduce_round_sums(sh, J, b);
+    reduce_round_sums(sh, J, b, &sh.block_sums[0][0]);
     __syncthreads();
     if (tid < 3 * (b - J)) tr[1 + 3 * J + tid] = (&sh.block_sums[J][0])[tid];
     if (tid == 0) { tr[3 * b + 1] = sh.fin[0][0]; tr[3 * b + 2] = sh.fin[1][0]; }

@@ -219,3 +219,39 @@ def test_batched_decoder_layers_full_size(imm, oracle):
                         [bytes(c[0:32]), bytes(c[32:64]), bytes(c[64:96])], p.proof_id))
     assert got == oracle.fs.prove_batched(members, 99)
     assert len(got) == 1 + 42 + 48
+
+
+def test_weight_commitments_computed_once_serve_every_request(imm, oracle):
+    """The weights belong to the model commitment: hashed once, their digests are reused while the
+    activations and outputs of each audited request are hashed afresh.  Statement and proof must equal
+    the oracle's (which hashes all three matrices of every request), request after request."""
+    rng = np.random.default_rng(41)
+    shapes = [(33, 300, 17), (64, 512, 64), (5, 129, 130)]
+    weights = [rng.integers(-128, 127, size=(k, n), endpoint=True).astype(np.int8) for (_, k, n) in shapes]
+    dev_w = [torch.from_numpy(B).cuda() for B in weights]
+    com_w = imm.Committer(dev_w)
+    com_w.commit()                                             # once
+    cached = com_w.digests.view(len(shapes), 32).clone()
+    n = len(shapes)
+    for request in range(3):
+        group = []
+        for i, (m, k, _) in enumerate(shapes):
+            A = rng.integers(-128, 127, size=(m, k), endpoint=True).astype(np.int8)
+            C = (A.astype(np.int64) @ weights[i].astype(np.int64)).astype(np.int32)
+            group.append((A, weights[i], C, 100 * request + i))
+        dev = [(torch.from_numpy(A).cuda(), dev_w[i], torch.from_numpy(C).cuda(), pid) for i, (A, _, C, pid) in enumerate(group)]
+        fresh = imm.Committer([t for (A, _, C, _) in dev for t in (A, C)])
+        fresh.commit()
+        stmt = torch.empty((n, 96), dtype=torch.uint8, device="cuda")
+        stmt.view(n, 3, 32)[:, 0].copy_(fresh.digests.view(n, 2, 32)[:, 0])
+        stmt.view(n, 3, 32)[:, 1].copy_(cached)
+        stmt.view(n, 3, 32)[:, 2].copy_(fresh.digests.view(n, 2, 32)[:, 1])
+        want = oracle_coms(oracle, group)
+        host = stmt.cpu().numpy()
+        for i in range(n):
+            assert bytes(host[i]) == b"".join(want[i])
+        assert bytes(imm.commit_matrices(dev).cpu().numpy().tobytes()) == host.tobytes()
+        got = imm.sumcheck_matmul_prove_fs(dev, stmt)
+        for (A, B, C, pid), t, cm in zip(group, got, want):
+            assert t == oracle.fs.prove(A, B, C, cm, pid)
+            assert imm.sumcheck_verify_fs(t, oracle.ceil_log2(A.shape[1]), b"".join(cm), A.shape[0], A.shape[1], B.shape[1], pid) == (imm.OK, -1)

@@ -285,3 +285,17 @@ def test_binding_refuses_cpu_tensors(imm):
         imm.make_descs([(A, A, A.to(torch.int32), 0)])
     with pytest.raises(ValueError):
         imm.mle_partial_eval(A, imm.BIND_ROWS, torch.zeros(4, dtype=torch.int64))
+
+
+def test_launch_count_of_a_proving_pass(imm, monkeypatch):
+    """Three launches while the batch is small enough for the fused contraction launch (under 2 GiB),
+    five from there on; the integer-pipe back end always takes five; 0 on invalid input."""
+    L = imm.lib()
+    small = _desc_array(imm, [(512, 4096, 4096)])
+    assert L.imm_sumcheck_matmul_launches(ctypes.addressof(small), 1) == 3
+    big = _desc_array(imm, [(8192, 4096, 14336)] * 8)                         # 4.7 GB of matrices
+    assert L.imm_sumcheck_matmul_launches(ctypes.addressof(big), 8) == 5
+    assert L.imm_sumcheck_matmul_launches(ctypes.addressof(big), 0) == 0
+    assert L.imm_sumcheck_matmul_launches(None, 1) == 0
+    monkeypatch.setenv("IMM_CONTRACT", "alu")
+    assert L.imm_sumcheck_matmul_launches(ctypes.addressof(small), 1) == 5

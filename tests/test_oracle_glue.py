@@ -98,3 +98,85 @@ def test_the_input_generators_hidden_activations_satisfy_the_link():
     assert glue.requant_check(up.C.numpy(), down.A.numpy(), 9, 256, -127, 127) == (0, -1)
     x = torch.tensor(EDGES_9, dtype=torch.int32)
     assert synth.requantize_i8(x).tolist() == glue.requantize(np.array(EDGES_9, dtype=np.int32), 9, 256, -127, 127).tolist()
+
+
+# ---------------------------------------------------------------- activation and gating link
+
+def relu_table():
+    return np.array([max(0, v) for v in range(-128, 128)], dtype=np.int8)
+
+
+def silu_like_table():
+    """An arbitrary odd-looking int8 table (round(x * sigmoid(x / 16))): any table is valid input."""
+    return np.array([int(round(v / (1.0 + math.exp(-v / 16.0)))) for v in range(-128, 128)], dtype=np.int8)
+
+
+def gated_by_hand(g: int, u, act, shift, rnd, shift2, rnd2, lo, hi) -> int:
+    """The definition entry by entry in Python integers."""
+    q = max(-128, min(127, (g + rnd) // (1 << shift)))
+    a = int(act[q + 128])
+    if u is None:
+        return a
+    w = max(-128, min(127, (u + rnd) // (1 << shift)))
+    return max(lo, min(hi, (a * w + rnd2) // (1 << shift2)))
+
+
+def test_activation_alone_reduces_to_known_maps():
+    rng = np.random.default_rng(11)
+    G = np.concatenate([rng.integers(-90000, 90000, 3000), np.array(EDGES_9)]).astype(np.int32)
+    ident = np.arange(-128, 128, dtype=np.int8)
+    # identity table: the plain requantisation to the full int8 range
+    assert (glue.gated_link(G, None, ident, 9, 256, 0, 0, -128, 127) == glue.requantize(G, 9, 256, -128, 127)).all()
+    # ReLU table: the requantisation clamped at zero
+    assert (glue.gated_link(G, None, relu_table(), 9, 256, 0, 0, -128, 127) == glue.requantize(G, 9, 256, 0, 127)).all()
+    # a constant table ignores its input; a reversed table negates (except at -128, which has no negative)
+    assert (glue.activation(G, np.full(256, 7, dtype=np.int8), 9, 256) == 7).all()
+    rev = np.array([max(-128, min(127, -v)) for v in range(-128, 128)], dtype=np.int8)
+    q = glue.requantize(G, 9, 256, -128, 127).astype(np.int64)
+    assert (glue.activation(G, rev, 9, 256).astype(np.int64) == np.clip(-q, -128, 127)).all()
+    # the table is indexed by value + 128: entry 0 answers -128, entry 255 answers 127
+    probe = np.zeros(256, dtype=np.int8); probe[0] = 11; probe[255] = 22; probe[128] = 33
+    assert glue.activation(np.array([-2**31, 2**31 - 1, 0, 255, 256]), probe, 9, 256).tolist() == [11, 22, 33, 33, 0]
+
+
+@pytest.mark.parametrize("shift2,rnd2", [(0, 0), (6, 32), (7, 64), (7, 0), (7, 127), (14, 1 << 13)])
+def test_gated_link_matches_python_integers(shift2, rnd2):
+    rng = np.random.default_rng(100 + shift2 + rnd2)
+    n = 3000
+    G = np.concatenate([rng.integers(-70000, 70000, n), np.array(EDGES_9)]).astype(np.int32)
+    U = np.concatenate([rng.integers(-70000, 70000, n), np.array(EDGES_9[::-1])]).astype(np.int32)
+    for act in (silu_like_table(), relu_table(), np.arange(-128, 128, dtype=np.int8)):
+        for lo, hi in ((-127, 127), (-128, 127), (0, 100)):
+            got = glue.gated_link(G, U, act, 9, 256, shift2, rnd2, lo, hi)
+            want = [gated_by_hand(int(g), int(u), act, 9, 256, shift2, rnd2, lo, hi) for g, u in zip(G, U)]
+            assert got.tolist() == want
+
+
+def test_gated_link_rounding_boundaries_of_the_product():
+    """g * u = 64 (2 t + 1) sits exactly between t and t + 1 at shift2 = 7: ties go up, for both signs;
+    the extreme products (-128 * -128 = 16384, -128 * 127) saturate."""
+    ident = np.arange(-128, 128, dtype=np.int8)
+    pairs = [(8, 8), (8, -8), (-8, -8), (24, 8), (-24, 8), (1, 63), (1, 64), (1, 65), (-1, 64), (-1, 65), (-128, -128), (-128, 127), (127, 127)]
+    G = np.array([g for g, _ in pairs], dtype=np.int32)          # shift 0: the accumulators are the int8 values
+    U = np.array([u for _, u in pairs], dtype=np.int32)
+    got = glue.gated_link(G, U, ident, 0, 0, 7, 64, -127, 127).tolist()
+    exact = [max(-127, min(127, math.floor(Fraction(g * u, 128) + Fraction(1, 2)))) for g, u in pairs]
+    assert got == exact == [1, 0, 1, 2, -1, 0, 1, 1, 0, -1, 127, -127, 126]
+
+
+def test_gated_link_check_counts_and_locates():
+    rng = np.random.default_rng(12)
+    G = rng.integers(-60000, 60000, (19, 23)).astype(np.int32)
+    U = rng.integers(-60000, 60000, (19, 23)).astype(np.int32)
+    act = silu_like_table()
+    H = glue.gated_link(G, U, act, 9, 256, 7, 64, -127, 127)
+    args = (act, 9, 256, 7, 64, -127, 127)
+    assert glue.gated_link_check(G, U, H, *args) == (0, -1)
+    H2 = H.copy(); H2[3, 4] += 1; H2[18, 22] -= 1
+    assert glue.gated_link_check(G, U, H2, *args) == (2, 3 * 23 + 4)
+    # another table, or the gate and up operands swapped, is another map
+    assert glue.gated_link_check(G, U, H, relu_table(), 9, 256, 7, 64, -127, 127)[0] > 0
+    assert glue.gated_link_check(U, G, H, *args)[0] > 0
+    # without U the check is of the activation alone
+    A = glue.gated_link(G, None, act, 9, 256, 0, 0, -128, 127)
+    assert glue.gated_link_check(G, None, A, act, 9, 256, 0, 0, -128, 127) == (0, -1)

@@ -27,6 +27,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import subprocess
 import sys
@@ -70,6 +71,9 @@ def parse_args():
     ap.add_argument("--cached-weights", action="store_true",
                     help="with --fs: the weight matrices (B of every product) are committed once, outside the "
                          "timed steps, as part of the model commitment; a step re-hashes only A and C")
+    ap.add_argument("--gated", action="store_true",
+                    help="with --config glue: the gated link instead (activation table of the gate projection times the "
+                         "up projection, 9 bytes per entry)")
     ap.add_argument("--verify", action="store_true",
                     help="time the verifier's pass instead: its own (c0, a_fin, b_fin) of every proof "
                          "(device-resident timing only)")
@@ -759,13 +763,35 @@ def run_glue(args):
     A = synth.gauss_i8(seed, synth.tid(0, synth.ROLE_ACT), T, d_model, synth.Q_SIGMA20, dev)
     W = synth.gauss_i8(seed, synth.tid(0, synth.ROLE_W), d_model, d_ff, synth.Q_SIGMA8, dev)
     C = synth.exact_matmul_i32(A, W)
-    H = synth.requantize_i8(C)
+    gated = bool(args.gated)
+    if gated:
+        # gate = C; up = a second product of the same activations; H manufactured with torch integer ops
+        W2 = synth.gauss_i8(seed, synth.tid(1, synth.ROLE_W), d_model, d_ff, synth.Q_SIGMA8, dev)
+        U = synth.exact_matmul_i32(A, W2)
+        del W2
+        act_host = [int(round(v / (1.0 + math.exp(-v / 16.0)))) for v in range(-128, 128)]
+        act_dev = torch.tensor(act_host, dtype=torch.int32, device=dev)
+        H = torch.empty((T, d_ff), dtype=torch.int8, device=dev)
+        for r0 in range(0, T, 1024):                           # in slabs: the intermediates are 64-bit
+            q = lambda X: torch.clamp((X >> 9) + (((X & 511) + 256) >> 9), -128, 127)
+            pr = act_dev[(q(C[r0:r0 + 1024]) + 128).long()] * q(U[r0:r0 + 1024])
+            H[r0:r0 + 1024] = torch.clamp((pr >> 7) + (((pr & 127) + 64) >> 7), -127, 127).to(torch.int8)
+        del pr, act_dev
+
+        def check(G_, U_, H_, out_):
+            return imm.gated_link_check(G_, U_, H_, act_host, 9, 256, 7, 64, -127, 127, out=out_)
+    else:
+        U = None
+        H = synth.requantize_i8(C)
+
+        def check(G_, U_, H_, out_):
+            return imm.requant_check(G_, H_, out=out_)
     del A, W
-    nbytes = 5 * T * d_ff
+    nbytes = (9 if gated else 5) * T * d_ff
     out = torch.empty(2, dtype=torch.int64, device=dev)
     barrier = rep.barrier
     for _ in range(warmup):
-        imm.requant_check(C, H, out=out)
+        check(C, U, H, out)
     barrier()
     sampler = ClockSampler(local_rank if "CUDA_VISIBLE_DEVICES" not in os.environ else
                            int(os.environ["CUDA_VISIBLE_DEVICES"].split(",")[local_rank]))
@@ -779,7 +805,7 @@ def run_glue(args):
         if flush:
             scrub.fill_(1)
         a.record()
-        imm.requant_check(C, H, out=out)
+        check(C, U, H, out)
         b.record()
     barrier()
     t1w = time.time()
@@ -795,17 +821,22 @@ def run_glue(args):
         "metric": "checked entries/sec", "value": T * d_ff * world / (ms_per_step * 1e-3), "unit": "entries/s",
         "n_gpus": world, "steps": steps, "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "i32", "data": "synthetic",
-        "config": {"workload": workload_name("glue", 0, T), "tokens": T, "input_bytes_per_gpu": nbytes,
-                   "map": "clamp((C + 256) >> 9, -127, 127)",
+        "config": {"workload": workload_name("glue", 0, T) + (" -- gated: activation table of the gate times the up "
+                                                                  "projection" if gated else ""),
+                   "tokens": T, "input_bytes_per_gpu": nbytes,
+                   "map": ("clamp((act[q(G)] * q(U) + 64) >> 7, -127, 127), q(X) = clamp((X + 256) >> 9, -128, 127), act = "
+                           "round(x * sigmoid(x / 16))" if gated else "clamp((C + 256) >> 9, -127, 127)"),
                    "l2": ("L2 flushed between steps (512 MB overwritten outside the timed event pairs)" if flush else
                           f"inputs ({nbytes / 2**30:.2f} GiB) exceed the 126 MB L2 several times over; no flush"),
                    "parallelism": "1 GPU" if world == 1 else f"{world} independent replicas, no collective"},
         "hbm_gbs_whole_step": gbs,
-        "roofline": {"kernel": "requant_check_kernel (4 bytes of C + 1 byte of H per entry, read once); timed as the whole "
-                               "imm_requant_check call (two 8-byte memsets + the kernel)", "bound": "hbm", "achieved": gbs,
+        "roofline": {"kernel": ("gated_link_kernel (4 bytes of G + 4 of U + 1 of H per entry, read once); timed as the whole "
+                                "imm_gated_link_check call (two 8-byte memsets + the kernel)" if gated else
+                                "requant_check_kernel (4 bytes of C + 1 byte of H per entry, read once); timed as the whole "
+                                "imm_requant_check call (two 8-byte memsets + the kernel)"), "bound": "hbm", "achieved": gbs,
                      "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": gbs / peak, "frac_of_8tbs": gbs / 8000.0,
                      "gbs_per_sm_mhz": (gbs / clocks["sm_mhz"]) if clocks and clocks.get("sm_mhz") else None,
-                     "traffic": (GLUE_TRAFFIC_RATIO * nbytes) if GLUE_TRAFFIC_RATIO else None},
+                     "traffic": (GLUE_TRAFFIC_RATIO * nbytes) if GLUE_TRAFFIC_RATIO and not gated else None},
         "gpu_launches": steps,
         "clocks": clocks,
     }
@@ -814,12 +845,16 @@ def run_glue(args):
         hC = torch.empty(C.shape, dtype=C.dtype, pin_memory=True).copy_(C)
         hH = torch.empty(H.shape, dtype=H.dtype, pin_memory=True).copy_(H)
         dC, dH = torch.empty_like(C), torch.empty_like(H)
+        hU = torch.empty(U.shape, dtype=U.dtype, pin_memory=True).copy_(U) if gated else None
+        dU = torch.empty_like(U) if gated else None
         hout = torch.empty(2, dtype=torch.int64, pin_memory=True)
         torch.cuda.synchronize()
 
         def e2e_pass():
             dC.copy_(hC, non_blocking=True); dH.copy_(hH, non_blocking=True)
-            hout.copy_(imm.requant_check(dC, dH, out=out), non_blocking=True)
+            if gated:
+                dU.copy_(hU, non_blocking=True)
+            hout.copy_(check(dC, dU, dH, out), non_blocking=True)
             torch.cuda.synchronize()
 
         e2e_pass()
@@ -832,7 +867,7 @@ def run_glue(args):
         e2e = {"value": T * d_ff * world / e2e_s, "unit": "entries/s", "ms_per_step": e2e_s * 1e3, "steps": k2,
                "h2d_bytes_per_step": nbytes, "d2h_bytes_per_step": 16,
                "matches_device_path": [int(v) for v in hout] == got}
-        del hC, hH, dC, dH
+        del hC, hH, dC, dH, hU, dU
     res["e2e"] = e2e
     if not args.no_cpu_baseline and world == 1:
         from oracle import glue
@@ -841,10 +876,14 @@ def run_glue(args):
         Hh[rows // 2, 77] ^= 1                               # one planted difference, found by both sides
         Hd = H[:rows].clone()
         Hd[rows // 2, 77] ^= 1
+        Uh = U[:rows].cpu().numpy() if gated else None
         w0 = time.perf_counter()
-        want = glue.requant_check(Ch, Hh, 9, 256, -127, 127)
+        if gated:
+            want = glue.gated_link_check(Ch, Uh, Hh, np.array(act_host, dtype=np.int8), 9, 256, 7, 64, -127, 127)
+        else:
+            want = glue.requant_check(Ch, Hh, 9, 256, -127, 127)
         secs = time.perf_counter() - w0
-        ok = [int(v) for v in imm.requant_check(C[:rows], Hd).cpu()] == list(want) and want[0] == 1
+        ok = [int(v) for v in check(C[:rows], U[:rows] if gated else None, Hd, out).cpu()] == list(want) and want[0] == 1
         res["cpu_baseline"] = {"value": rows * d_ff / secs, "unit": "entries/s", "cores": 1, "nproc": os.cpu_count(),
                                "kind": "oracle", "seconds": secs,
                                "sample": f"the first {rows} of the {T} rows, one planted difference, same inputs as the GPU run",

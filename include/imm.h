@@ -410,6 +410,28 @@ int imm_requant_check(const int32_t* d_C, const int8_t* d_H, int64_t rows, int64
                       int64_t ldh, int shift, int32_t rnd, int32_t lo, int32_t hi, uint64_t* d_result,
                       void* stream);
 
+/* The element-wise step of a gated feed-forward block (the MLP of the decoder models of Section 6.1;
+ * one of the parts of the reference execution in Section 4.1): an activation of the gate projection
+ * and its product with the up projection give the int8 input of the down projection,
+ *     g[i,j] = act[ clamp(floor((G[i,j] + rnd) / 2^shift), -128, 127) + 128 ]
+ *     u[i,j] =      clamp(floor((U[i,j] + rnd) / 2^shift), -128, 127)
+ *     H[i,j] = clamp( floor( (g[i,j] * u[i,j] + rnd2) / 2^shift2 ), lo, hi )
+ * with G, U the int32 outputs of the two products.  The activation is the committed model's own
+ * int8 -> int8 table (the paper fixes no integer arithmetic).  d_U == NULL: the activation alone,
+ * H = g (shift2, rnd2, lo, hi are then ignored).  Results as for imm_requant_check: d_result[0] the
+ * number of entries of H that differ, d_result[1] the position of the first (UINT64_MAX if none).
+ *   d_G, d_U : DEVICE int32 matrices, rows x cols, leading dimensions ldg, ldu (elements)
+ *   d_H      : DEVICE int8 matrix, rows x cols, leading dimension ldh
+ *   act_host : HOST array of 256 int8: act_host[v + 128] answers the value v; copied into the launch
+ *   shift    : 0..30, 0 <= rnd < 2^shift;  shift2 : 0..14, 0 <= rnd2 < 2^shift2;  -128 <= lo <= hi <= 127
+ * One streaming pass: 4 (+4) bytes of G (and U) and 1 byte of H per entry, each read once; 16-byte
+ * aligned rows are read with 128-bit loads, anything else element by element.  Two memsets and one
+ * kernel on `stream`; nothing allocated or synchronised; a differing entry is a finding, not an error.
+ * Errors: IMM_ERR_ARG, IMM_ERR_SHAPE (zero or > 2^20 extent, ld < cols), IMM_ERR_ALIGN, IMM_ERR_CUDA. */
+int imm_gated_link_check(const int32_t* d_G, const int32_t* d_U, const int8_t* d_H, int64_t rows, int64_t cols,
+                         int64_t ldg, int64_t ldu, int64_t ldh, const int8_t* act_host, int shift, int32_t rnd,
+                         int shift2, int32_t rnd2, int32_t lo, int32_t hi, uint64_t* d_result, void* stream);
+
 /* ---------------------------------------------------------------------------------------------
  * Non-interactive proof (Fiat-Shamir)
  * ---------------------------------------------------------------------------------------------

@@ -37,7 +37,8 @@ EXPORTS = ("imm_version", "imm_last_cuda_error", "imm_challenge", "imm_field_bin
            "imm_sumcheck_matmul_fs_workspace", "imm_sumcheck_matmul_prove_fs", "imm_fs_challenges",
            "imm_sumcheck_verify_fs", "imm_sumcheck_expected_workspace", "imm_sumcheck_expected",
            "imm_sumcheck_matmul_fs_batched_workspace", "imm_sumcheck_matmul_prove_fs_batched",
-           "imm_fs_batched_challenges", "imm_sumcheck_verify_fs_batched", "imm_requant_check", "imm_sumcheck_matmul_launches")
+           "imm_fs_batched_challenges", "imm_sumcheck_verify_fs_batched", "imm_requant_check", "imm_sumcheck_matmul_launches",
+           "imm_gated_link_check")
 FS_BATCH_MAX = 1024
 COMMIT_LEAF = 4096
 NOALLOC_MAX_TILES = 8192
@@ -153,6 +154,9 @@ def lib() -> ctypes.CDLL:
     L.imm_sumcheck_matmul_launches.argtypes = [vp, ci]
     L.imm_requant_check.restype = ci
     L.imm_requant_check.argtypes = [vp, vp, i64, i64, i64, i64, ci, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, vp, vp]
+    L.imm_gated_link_check.restype = ci
+    L.imm_gated_link_check.argtypes = [vp, vp, vp, i64, i64, i64, i64, i64, vp, ci, ctypes.c_int32, ci, ctypes.c_int32,
+                                       ctypes.c_int32, ctypes.c_int32, vp, vp]
     _lib = L
     return L
 
@@ -790,6 +794,32 @@ def requant_check(C: torch.Tensor, H: torch.Tensor, shift: int = 9, rnd: int = 2
     _cuda(out, torch.int64, "out")
     _check(lib().imm_requant_check(pc, ph, rows, cols, ldc, ldh, int(shift), int(rnd), int(lo), int(hi),
                                    out.data_ptr(), _stream()), "imm_requant_check")
+    return out
+
+
+def gated_link_check(G: torch.Tensor, U: Optional[torch.Tensor], H: torch.Tensor, act, shift: int = 9, rnd: int = 256,
+                     shift2: int = 7, rnd2: int = 64, lo: int = -127, hi: int = 127,
+                     out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Checks H == clamp(floor((act[q(G)] * q(U) + rnd2) / 2^shift2), lo, hi) entry by entry, q(X) =
+    clamp(floor((X + rnd) / 2^shift), -128, 127); U None: H == act[q(G)].  G, U int32 and H int8 CUDA
+    matrices of one shape; ``act``: 256 int8 values (bytes, list or CPU tensor), act[v + 128] answers v.
+    Returns a 2-element int64 CUDA tensor: differing entries and the position of the first (-1 if none)."""
+    pg, cg, rows, cols, ldg = _matrix(G, "G")
+    ph, ch, rows2, cols2, ldh = _matrix(H, "H")
+    if cg != I32 or ch != I8 or (rows, cols) != (rows2, cols2):
+        raise ValueError("need G int32 and H int8 of the same shape")
+    pu, ldu = None, ldg
+    if U is not None:
+        pu, cu, rows3, cols3, ldu = _matrix(U, "U")
+        if cu != I32 or (rows3, cols3) != (rows, cols):
+            raise ValueError("need U int32 of the shape of G")
+    table = (ctypes.c_int8 * 256)(*[int(v) for v in (act.tolist() if hasattr(act, "tolist") else act)])
+    if out is None:
+        out = torch.empty(2, dtype=torch.int64, device=G.device)
+    _cuda(out, torch.int64, "out")
+    _check(lib().imm_gated_link_check(pg, pu, ph, rows, cols, ldg, ldu, ldh, ctypes.addressof(table), int(shift), int(rnd),
+                                      int(shift2), int(rnd2), int(lo), int(hi), out.data_ptr(), _stream()),
+           "imm_gated_link_check")
     return out
 
 

@@ -297,6 +297,7 @@ COMMIT_TRAFFIC_RATIO = (1.077891 + 0.018910) / 1.050673152                   # c
 # 148 x 64 x 1.965e9 / 17.18 = 1083 GB/s.
 COMMIT_ALU_PEAK_GBS_AT_1965 = 1083.0
 GLUE_TRAFFIC_RATIO = (146.819072 + 3.869952) / 146.80064    # requant_check_kernel: (dram read + write) / (5 bytes per entry), 2048-token capture
+GATED_TRAFFIC_RATIO = (264.269312 + 3.397632) / 264.241152   # gated_link_kernel: (dram read + write) / (9 bytes per entry), 2048-token capture
 FUSED_TRAFFIC_RATIO = (308.909568 + 12.264448) / 306.184192   # fused_contract_kernel: (dram read + write) / algorithmic bytes, FFN-pair capture
 CLAIM_KERNEL_TRAFFIC_RATIO = 239.64 / 234.881024  # bytedot_kernel<1,1,1>: (dram read + write) / (4 bytes per entry), small-case capture
 
@@ -836,7 +837,7 @@ def run_glue(args):
                                 "imm_requant_check call (two 8-byte memsets + the kernel)"), "bound": "hbm", "achieved": gbs,
                      "peak": peak, "peak_kind": peak_kind, "unit": "GB/s", "frac": gbs / peak, "frac_of_8tbs": gbs / 8000.0,
                      "gbs_per_sm_mhz": (gbs / clocks["sm_mhz"]) if clocks and clocks.get("sm_mhz") else None,
-                     "traffic": (GLUE_TRAFFIC_RATIO * nbytes) if GLUE_TRAFFIC_RATIO and not gated else None},
+                     "traffic": (GATED_TRAFFIC_RATIO if gated else GLUE_TRAFFIC_RATIO) * nbytes},
         "gpu_launches": steps,
         "clocks": clocks,
     }

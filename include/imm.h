@@ -190,19 +190,20 @@ size_t imm_sumcheck_matmul_workspace(const imm_matmul_desc* descs_host, int npro
  *   d_ws          : DEVICE workspace, >= imm_sumcheck_matmul_workspace(...) bytes
  * The whole batch is one small host-to-device copy (the job lists) and a fixed sequence of kernel
  * launches on `stream`, ordered after the work already there; results are valid once the stream has
- * been synchronised.  A batch of 2 GiB of matrices or more takes five launches: eq tables and
- * weight limb tables, the claim, the row binding, the column binding, the rounds.  A smaller batch
- * is bound by launch latency rather than bandwidth and takes three, chained by programmatic
- * dependent launch: one contraction launch for all three matrix kinds, whose tiles build their own
- * slice of the eq tables from the challenges (no table reaches memory); a reduction of the partial
- * vectors into the round tables; the rounds.  Same transcripts either way.
+ * been synchronised.  A large batch takes five launches: eq tables and weight limb tables, the
+ * claim, the row binding, the column binding, the rounds.  A batch under 512 MiB of matrices, or
+ * under 16 GiB whose proofs average 32 MiB or more, is held back by launch latency and the gaps
+ * between kernels more than by bandwidth and takes three, chained by programmatic dependent
+ * launch: one contraction launch for all three matrix kinds, whose tiles build their own slice of
+ * the eq tables from the challenges (no table reaches memory); a reduction of the partial vectors
+ * into the round tables; the rounds.  Same transcripts either way.
  * Errors: IMM_ERR_ARG, IMM_ERR_SHAPE, IMM_ERR_ALIGN, IMM_ERR_WORKSPACE, IMM_ERR_CUDA. */
 int imm_sumcheck_matmul_prove(const imm_matmul_desc* descs_host, int nproofs, uint64_t seed,
                               imm_fe* d_transcripts, int64_t stride, int32_t* d_status,
                               void* d_ws, size_t ws_bytes, void* stream);
 
-/* Kernel launches imm_sumcheck_matmul_prove enqueues for this batch: 5, or 3 for a batch small
- * enough for the fused contraction launch (0 on invalid input). */
+/* Kernel launches imm_sumcheck_matmul_prove enqueues for this batch: 5, or 3 for a batch that takes
+ * the fused contraction launch (0 on invalid input). */
 int imm_sumcheck_matmul_launches(const imm_matmul_desc* descs_host, int nproofs);
 
 /* Phase timing of imm_sumcheck_matmul_prove, for measurement.  While enabled, every prove call

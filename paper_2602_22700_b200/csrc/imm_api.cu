@@ -152,7 +152,14 @@ const int rows_a[] = {1024, 512, 256, 128, 64, 32}, widths_a[] = {1024, 512, 256
 const int rows_b[] = {256}, rows_c[] = {1024, 512, 256, 128};
 const int chunks[] = {4096, 2048, 1024, 512, 256};
 // fused launch (small batches): one persistent grid, a run of equal bytes per block
-constexpr int64_t FUSE_BELOW_BYTES = (int64_t)2 << 30;       // batches under 2 GiB of matrices take the fused launch
+// Which batches take the fused contraction launch (measured on expert, decoder-block and attention batches):
+// it saves about 40 us of launches and dependencies but streams a little slower than the three tuned
+// kernels, and its per-job set-up weighs on batches of many small proofs.  Fused: every batch under 512 MiB;
+// up to 16 GiB when a proof averages 32 MiB or more (decoder projections, experts), where it wins by 15 % at
+// 2 GiB and 1 % at 13 GiB; attention-sized proofs (11 MiB each) from 512 MiB on run the five launches.
+constexpr int64_t FUSE_ALWAYS_BELOW_BYTES = (int64_t)512 << 20;
+constexpr int64_t FUSE_BELOW_BYTES = (int64_t)16 << 30;
+constexpr int64_t FUSE_MIN_BYTES_PER_PROOF = (int64_t)32 << 20;
 constexpr int FUSED_A_TILE_COLS = 1024;                      // 8 warps x 128 columns
 constexpr int64_t FUSED_MIN_RUN_BYTES = 32 << 10;            // below this a run is all set-up
 constexpr int FUSED_COST_A = 250, FUSED_COST_C = 180;        // time per byte of A and of C relative to B, per cent (measured)
@@ -394,7 +401,10 @@ Plan make_plan(const imm_matmul_desc* descs, int nproofs)
     int64_t batch_bytes = 0;
     for (int i = 0; i < nproofs; i++)
         batch_bytes += descs[i].m * descs[i].k + descs[i].k * descs[i].n + 4 * descs[i].m * descs[i].n;
-    p.fused = p.mma && batch_bytes < FUSE_BELOW_BYTES && !env_set("IMM_NO_FUSE");
+    const int64_t fuse_below = (int64_t)env_int("IMM_FUSE_BELOW_MB", (int)(FUSE_BELOW_BYTES >> 20)) << 20;
+    p.fused = p.mma && !env_set("IMM_NO_FUSE") &&
+              (batch_bytes < std::min(fuse_below, FUSE_ALWAYS_BELOW_BYTES) ||
+               (batch_bytes < fuse_below && batch_bytes / nproofs >= FUSE_MIN_BYTES_PER_PROOF));
     if (p.fused) {
         plan_fused(p, descs, nproofs);
     } else if (p.mma) {

@@ -288,13 +288,19 @@ def test_binding_refuses_cpu_tensors(imm):
 
 
 def test_launch_count_of_a_proving_pass(imm, monkeypatch):
-    """Three launches while the batch is small enough for the fused contraction launch (under 2 GiB),
-    five from there on; the integer-pipe back end always takes five; 0 on invalid input."""
+    """Three launches where the batch takes the fused contraction launch (under 512 MiB, or under 16 GiB
+    with proofs of 32 MiB or more on average), five otherwise; the integer-pipe back end always takes
+    five; 0 on invalid input."""
     L = imm.lib()
     small = _desc_array(imm, [(512, 4096, 4096)])
     assert L.imm_sumcheck_matmul_launches(ctypes.addressof(small), 1) == 3
-    big = _desc_array(imm, [(8192, 4096, 14336)] * 8)                         # 4.7 GB of matrices
-    assert L.imm_sumcheck_matmul_launches(ctypes.addressof(big), 8) == 5
+    experts = _desc_array(imm, [(8192, 4096, 14336)] * 8)                     # 4.5 GB, 562 MB per proof
+    assert L.imm_sumcheck_matmul_launches(ctypes.addressof(experts), 8) == 3
+    big = _desc_array(imm, [(8192, 4096, 14336)] * 40)                        # 22 GB
+    assert L.imm_sumcheck_matmul_launches(ctypes.addressof(big), 40) == 5
+    heads = _desc_array(imm, [(2048, 128, 2048)] * 64)                        # 1.1 GB of 17 MB proofs
+    assert L.imm_sumcheck_matmul_launches(ctypes.addressof(heads), 64) == 5
+    assert L.imm_sumcheck_matmul_launches(ctypes.addressof(heads), 16) == 3   # 277 MB: small enough whatever the proofs
     assert L.imm_sumcheck_matmul_launches(ctypes.addressof(big), 0) == 0
     assert L.imm_sumcheck_matmul_launches(None, 1) == 0
     monkeypatch.setenv("IMM_CONTRACT", "alu")

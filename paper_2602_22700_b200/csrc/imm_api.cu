@@ -162,6 +162,7 @@ constexpr int64_t FUSE_BELOW_BYTES = (int64_t)16 << 30;
 constexpr int64_t FUSE_MIN_BYTES_PER_PROOF = (int64_t)32 << 20;
 constexpr int FUSED_A_TILE_COLS = 1024;                      // 8 warps x 128 columns
 constexpr int64_t FUSED_MIN_RUN_BYTES = 32 << 10;            // below this a run is all set-up
+constexpr int FUSED_JOB_SETUP_KB = 160, FUSED_CHUNK_SETUP_KB = 24;  // a job's and a chunk's set-up in bytes a block streams meanwhile (from sweeps over expert, FFN and attention batches)
 constexpr int FUSED_COST_A = 250, FUSED_COST_C = 180;        // time per byte of A and of C relative to B, per cent (measured)
 // rows one pass of a block's eight warps covers: row ranges are cut at multiples of it, so that no pass runs
 // on a few warps only (16 rows per warp and pass)
@@ -292,15 +293,17 @@ int pow2_floor_clamped(int64_t v, int lo, int hi)
 // The fused launch's partition: every block of the persistent grid gets one contiguous run of the
 // sequence [tiles of every A][row ranges of every column chunk of every C][the same for every B],
 // cut so that all runs hold (almost) the same number of matrix bytes.
-void plan_fused(Plan& p, const imm_matmul_desc* descs, int nproofs)
+// Lays the sequence out for runs of `run` cost units (bytes of B); returns the cost of the whole sequence.
+// A job's set-up (challenges, eq tables: some 6 us) and a chunk's or tile's (weight limbs: 1-2 us) are
+// charged as the bytes a block would stream meanwhile, so that a run of many small matrices is not
+// taken for a short one.
+int64_t plan_fused_runs(Plan& p, const imm_matmul_desc* descs, int nproofs, int64_t blocks, int64_t run)
 {
-    const int64_t blocks = (int64_t)sm_count() * FUSED_BLOCKS_PER_SM;
     // cost of a byte of each kind relative to B, in per cent (measured: see FUSED_COST_*)
     const int64_t cost_a = env_int("IMM_FUSED_COST_A", FUSED_COST_A), cost_c = env_int("IMM_FUSED_COST_C", FUSED_COST_C);
-    int64_t total = 0;
-    for (int i = 0; i < nproofs; i++)
-        total += descs[i].m * descs[i].k * cost_a / 100 + descs[i].k * descs[i].n + 4 * descs[i].m * descs[i].n * cost_c / 100;
-    const int64_t run = std::max<int64_t>((total + blocks - 1) / blocks, FUSED_MIN_RUN_BYTES);
+    const int64_t job_cost = (int64_t)env_int("IMM_FUSED_JOB_KB", FUSED_JOB_SETUP_KB) << 10;
+    const int64_t chunk_cost = (int64_t)env_int("IMM_FUSED_CHUNK_KB", FUSED_CHUNK_SETUP_KB) << 10;
+    p.segs.clear();
     // widest column chunk that still cuts a run into several passes of all eight warps (the cuts fall on pass
     // boundaries, so the passes per run set how evenly the runs can be sized)
     const int passes = env_int("IMM_FUSED_PASSES", 4);
@@ -314,6 +317,7 @@ void plan_fused(Plan& p, const imm_matmul_desc* descs, int nproofs)
     for (int i = 0; i < nproofs; i++) {
         const imm_matmul_desc& d = descs[i];
         Plan::FusedGeom& g = p.fg[i];
+        cum += job_cost;
         const int64_t width = std::min<int64_t>(FUSED_A_TILE_COLS, d.k);
         int64_t rows = (run * 100 / cost_a / 2 / width) / 32 * 32;
         rows = rows < 32 ? 32 : rows > MAX_TILE_ROWS ? MAX_TILE_ROWS : rows;
@@ -328,7 +332,7 @@ void plan_fused(Plan& p, const imm_matmul_desc* descs, int nproofs)
                 const int64_t tc = std::min<int64_t>(FUSED_A_TILE_COLS, d.k - (int64_t)cc * FUSED_A_TILE_COLS);
                 p.segs.push_back(FusedSeg{i, rb * g.ncc_a + cc, 0, 0});
                 seg_block.push_back(block_of(cum));
-                cum += tr * tc * cost_a / 100;
+                cum += tr * tc * cost_a / 100 + chunk_cost / 2;
             }
     }
     // C then B: row ranges of column chunks
@@ -344,8 +348,10 @@ void plan_fused(Plan& p, const imm_matmul_desc* descs, int nproofs)
             const int ncc = (int)((row_bytes + chunk - 1) / chunk);
             if (kind == 1) { g.chunk_c = chunk; g.ncc_c = ncc; g.seg0_c = (int)p.segs.size(); }
             else { g.chunk_b = chunk; g.ncc_b = ncc; }
+            cum += job_cost;
             for (int cc = 0; cc < ncc; cc++) {
                 if (kind == 1 && cc == 0) g.nseg_c = 0;
+                cum += chunk_cost;
                 const int64_t w = std::max<int64_t>(1, std::min<int64_t>(chunk, row_bytes - (int64_t)cc * chunk) * cost / 100);
                 int64_t r = 0;
                 while (r < rows) {
@@ -372,6 +378,22 @@ void plan_fused(Plan& p, const imm_matmul_desc* descs, int nproofs)
         while (si < seg_block.size() && seg_block[si] < b) si++;
         p.block_first[b] = (uint32_t)si;
     }
+    return cum;
+}
+
+void plan_fused(Plan& p, const imm_matmul_desc* descs, int nproofs)
+{
+    const int64_t blocks = (int64_t)sm_count() * FUSED_BLOCKS_PER_SM;
+    const int64_t cost_a = env_int("IMM_FUSED_COST_A", FUSED_COST_A), cost_c = env_int("IMM_FUSED_COST_C", FUSED_COST_C);
+    int64_t total = 0;
+    for (int i = 0; i < nproofs; i++)
+        total += descs[i].m * descs[i].k * cost_a / 100 + descs[i].k * descs[i].n + 4 * descs[i].m * descs[i].n * cost_c / 100;
+    // the set-up charges depend on the chunk widths, which depend on the run: lay out once to learn the
+    // sequence's cost, then again with the run that cost gives
+    int64_t run = std::max<int64_t>((total + blocks - 1) / blocks, FUSED_MIN_RUN_BYTES);
+    const int64_t cost = plan_fused_runs(p, descs, nproofs, blocks, run);
+    run = std::max<int64_t>((cost + blocks - 1) / blocks, FUSED_MIN_RUN_BYTES);
+    plan_fused_runs(p, descs, nproofs, blocks, run);
 }
 
 
@@ -404,7 +426,8 @@ Plan make_plan(const imm_matmul_desc* descs, int nproofs)
     const int64_t fuse_below = (int64_t)env_int("IMM_FUSE_BELOW_MB", (int)(FUSE_BELOW_BYTES >> 20)) << 20;
     p.fused = p.mma && !env_set("IMM_NO_FUSE") &&
               (batch_bytes < std::min(fuse_below, FUSE_ALWAYS_BELOW_BYTES) ||
-               (batch_bytes < fuse_below && batch_bytes / nproofs >= FUSE_MIN_BYTES_PER_PROOF));
+               (batch_bytes < fuse_below &&
+                batch_bytes / nproofs >= (int64_t)env_int("IMM_FUSE_MIN_PROOF_MB", (int)(FUSE_MIN_BYTES_PER_PROOF >> 20)) << 20));
     if (p.fused) {
         plan_fused(p, descs, nproofs);
     } else if (p.mma) {

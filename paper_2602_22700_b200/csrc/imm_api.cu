@@ -154,10 +154,11 @@ const int chunks[] = {4096, 2048, 1024, 512, 256};
 // fused launch (small batches): one persistent grid, a run of equal bytes per block
 // Which batches take the fused contraction launch (measured on expert, decoder-block and attention batches):
 // it saves about 40 us of launches and dependencies but streams a little slower than the three tuned
-// kernels, and its per-job set-up weighs on batches of many small proofs.  Fused: every batch under 512 MiB;
+// kernels, and its per-job set-up weighs on batches of many small proofs.  Fused: every batch under 2 GiB;
 // up to 16 GiB when a proof averages 32 MiB or more (decoder projections, experts), where it wins by 15 % at
-// 2 GiB and 1 % at 13 GiB; attention-sized proofs (11 MiB each) from 512 MiB on run the five launches.
-constexpr int64_t FUSE_ALWAYS_BELOW_BYTES = (int64_t)512 << 20;
+// 2 GiB and 1 % at 13 GiB; attention-sized proofs (11 MiB each) win by 3 % at 0.7 and 2 % at 1.4 GiB and
+// lose by 14 % at 5.4 GiB.
+constexpr int64_t FUSE_ALWAYS_BELOW_BYTES = (int64_t)2 << 30;
 constexpr int64_t FUSE_BELOW_BYTES = (int64_t)16 << 30;
 constexpr int64_t FUSE_MIN_BYTES_PER_PROOF = (int64_t)32 << 20;
 constexpr int FUSED_A_TILE_COLS = 1024;                      // 8 warps x 128 columns

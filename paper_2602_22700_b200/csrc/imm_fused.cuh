@@ -176,8 +176,8 @@ fused_contract_kernel(const FusedJob* jobs, const FusedSeg* segs, const uint32_t
                 for (int g = 0; g < 8; g++) dst[G * 64 + (4 * g + t) * 2 + h] = limb[g];
             }
             __syncthreads();
-            if (job.vec) rowmma_tile<true, false>(job, (uint32_t)seg.cci, sh.sR);
-            else rowmma_tile<false, false>(job, (uint32_t)seg.cci, sh.sR);
+            if (job.vec) rowmma_tile<true, false, true>(job, (uint32_t)seg.cci, sh.sR);
+            else rowmma_tile<false, false, true>(job, (uint32_t)seg.cci, sh.sR);
             cur_cci = -1;
             continue;
         }

@@ -346,7 +346,10 @@ __global__ void __launch_bounds__(BYTEDOT_THREADS, MT == 1 ? 3 : 2) bytedot_kern
 
 // STAGE: copy the tile's weight limbs from job.wtab into sR; otherwise the caller has filled sR
 // (and synchronised).
-template <bool VEC, bool STAGE = true>
+// SPLIT: a tile narrower than the block (k below 128 columns per warp, e.g. an attention head's Q) leaves
+// warps without columns; they then share the rows instead -- warp w takes column group w % ncw and every
+// (8 / ncw)-th group of 32 rows -- and the partial column sums meet in shared memory (sR, once the loop is done).
+template <bool VEC, bool STAGE = true, bool SPLIT = false>
 __device__ __forceinline__ void rowmma_tile(const MatJob& job, uint32_t local, uint2* sR)
 {
     const int rbi = local / job.ncc, cci = local % job.ncc;
@@ -363,7 +366,16 @@ __device__ __forceinline__ void rowmma_tile(const MatJob& job, uint32_t local, u
     }
 
     const int tile_cols = (int)blockDim.x * 4;                    // 128 columns per warp
-    const int col = cci * tile_cols + warp * 128 + 16 * g;        // this thread's 16 columns
+    int cw = warp, rw = 0, rs = 1, ncw = (int)blockDim.x >> 5;
+    if (SPLIT) {
+        const int need = (min(tile_cols, job.cols - cci * tile_cols) + 127) >> 7;     // warps that have columns
+        ncw = 1;
+        while (ncw < need) ncw <<= 1;
+        rs = ((int)blockDim.x >> 5) / ncw;
+        cw = warp % ncw;
+        rw = warp / ncw;
+    }
+    const int col = cci * tile_cols + cw * 128 + 16 * g;          // this thread's 16 columns
     const int nvalid = min(16, job.cols - col);
     const bool full = nvalid == 16;
     int32_t acc[8][4];
@@ -372,8 +384,8 @@ __device__ __forceinline__ void rowmma_tile(const MatJob& job, uint32_t local, u
 #pragma unroll
         for (int c = 0; c < 4; c++) acc[i][c] = 0;
 
-    if (warp * 128 + cci * tile_cols < job.cols) {              // whole warp in or out
-        for (int G = 0; G < ngroups; G++) {
+    if (cw * 128 + cci * tile_cols < job.cols) {                // whole warp in or out
+        for (int G = rw; G < ngroups; G += rs) {
             uint4 d[2][4];
 #pragma unroll
             for (int h = 0; h < 2; h++)
@@ -398,6 +410,32 @@ __device__ __forceinline__ void rowmma_tile(const MatJob& job, uint32_t local, u
         }
     }
     // MMA i: row-slot g is column col + 2i, row-slot g+8 is column col + 2i + 1
+    if (SPLIT && rs > 1) {
+        __syncthreads();                                        // every warp is done with the weights in sR
+        uint64_t* red = reinterpret_cast<uint64_t*>(sR);        // [warp][128 columns]: 8 KiB, the size of sR
+#pragma unroll
+        for (int i = 0; i < 8; i++)
+#pragma unroll
+            for (int h = 0; h < 2; h++) {
+                const uint64_t v = combine_limbs(acc[i][2 * h], acc[i][2 * h + 1], t);
+                if (t == 0) red[warp * 128 + 16 * g + 2 * i + h] = v;
+            }
+        __syncthreads();
+        if (rw == 0 && t == 0) {
+#pragma unroll
+            for (int i = 0; i < 8; i++)
+#pragma unroll
+                for (int h = 0; h < 2; h++) {
+                    const int c = col + 2 * i + h;
+                    if (c < job.cols) {
+                        uint64_t v = 0;
+                        for (int r = 0; r < rs; r++) v = gl::add(v, red[(r * ncw + cw) * 128 + 16 * g + 2 * i + h]);
+                        job.out[(int64_t)rbi * job.cols + c] = v;
+                    }
+                }
+        }
+        return;                                                 // (the caller synchronises before it refills sR)
+    }
 #pragma unroll
     for (int i = 0; i < 8; i++)
 #pragma unroll

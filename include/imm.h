@@ -191,7 +191,7 @@ size_t imm_sumcheck_matmul_workspace(const imm_matmul_desc* descs_host, int npro
  * The whole batch is one small host-to-device copy (the job lists) and a fixed sequence of kernel
  * launches on `stream`, ordered after the work already there; results are valid once the stream has
  * been synchronised.  A large batch takes five launches: eq tables and weight limb tables, the
- * claim, the row binding, the column binding, the rounds.  A batch under 2 GiB of matrices, or
+ * claim, the row binding, the column binding, the rounds.  A batch under 4 GiB of matrices, or
  * under 16 GiB whose proofs average 32 MiB or more, is held back by launch latency and the gaps
  * between kernels more than by bandwidth and takes three, chained by programmatic dependent
  * launch: one contraction launch for all three matrix kinds, whose tiles build their own slice of

@@ -154,11 +154,11 @@ const int chunks[] = {4096, 2048, 1024, 512, 256};
 // fused launch (small batches): one persistent grid, a run of equal bytes per block
 // Which batches take the fused contraction launch (measured on expert, decoder-block and attention batches):
 // it saves about 40 us of launches and dependencies but streams a little slower than the three tuned
-// kernels, and its per-job set-up weighs on batches of many small proofs.  Fused: every batch under 2 GiB;
+// kernels, and its per-job set-up weighs on batches of many small proofs.  Fused: every batch under 4 GiB;
 // up to 16 GiB when a proof averages 32 MiB or more (decoder projections, experts), where it wins by 15 % at
-// 2 GiB and 1 % at 13 GiB; attention-sized proofs (11 MiB each) win by 3 % at 0.7 and 2 % at 1.4 GiB and
-// lose by 14 % at 5.4 GiB.
-constexpr int64_t FUSE_ALWAYS_BELOW_BYTES = (int64_t)2 << 30;
+// 2 GiB and 1 % at 13 GiB; attention-sized proofs (11 MiB each) win by 9 % at 0.7 and 7 % at 2.7 GiB and
+// lose by 3 % at 5.4 GiB.
+constexpr int64_t FUSE_ALWAYS_BELOW_BYTES = (int64_t)4 << 30;
 constexpr int64_t FUSE_BELOW_BYTES = (int64_t)16 << 30;
 constexpr int64_t FUSE_MIN_BYTES_PER_PROOF = (int64_t)32 << 20;
 constexpr int FUSED_A_TILE_COLS = 1024;                      // 8 warps x 128 columns
@@ -353,7 +353,8 @@ int64_t plan_fused_runs(Plan& p, const imm_matmul_desc* descs, int nproofs, int6
             for (int cc = 0; cc < ncc; cc++) {
                 if (kind == 1 && cc == 0) g.nseg_c = 0;
                 cum += chunk_cost;
-                const int64_t w = std::max<int64_t>(1, std::min<int64_t>(chunk, row_bytes - (int64_t)cc * chunk) * cost / 100);
+                // (a row piece costs whole slabs of 256 bytes: a 128-byte row of an attention head's V fills half of one)
+                const int64_t w = std::max<int64_t>(1, (std::min<int64_t>(chunk, row_bytes - (int64_t)cc * chunk) + 255) / 256 * 256 * cost / 100);
                 int64_t r = 0;
                 while (r < rows) {
                     const int32_t b = block_of(cum);

@@ -288,7 +288,7 @@ def test_binding_refuses_cpu_tensors(imm):
 
 
 def test_launch_count_of_a_proving_pass(imm, monkeypatch):
-    """Three launches where the batch takes the fused contraction launch (under 2 GiB, or under 16 GiB
+    """Three launches where the batch takes the fused contraction launch (under 4 GiB, or under 16 GiB
     with proofs of 32 MiB or more on average), five otherwise; the integer-pipe back end always takes
     five; 0 on invalid input."""
     L = imm.lib()
@@ -298,9 +298,9 @@ def test_launch_count_of_a_proving_pass(imm, monkeypatch):
     assert L.imm_sumcheck_matmul_launches(ctypes.addressof(experts), 8) == 3
     big = _desc_array(imm, [(8192, 4096, 14336)] * 40)                        # 22 GB
     assert L.imm_sumcheck_matmul_launches(ctypes.addressof(big), 40) == 5
-    heads = _desc_array(imm, [(2048, 128, 2048)] * 160)                       # 2.8 GB of 17 MB proofs
-    assert L.imm_sumcheck_matmul_launches(ctypes.addressof(heads), 160) == 5
-    assert L.imm_sumcheck_matmul_launches(ctypes.addressof(heads), 64) == 3   # 1.1 GB: small enough whatever the proofs
+    heads = _desc_array(imm, [(2048, 128, 2048)] * 300)                       # 5.2 GB of 17 MB proofs
+    assert L.imm_sumcheck_matmul_launches(ctypes.addressof(heads), 300) == 5
+    assert L.imm_sumcheck_matmul_launches(ctypes.addressof(heads), 160) == 3  # 2.8 GB: small enough whatever the proofs
     assert L.imm_sumcheck_matmul_launches(ctypes.addressof(big), 0) == 0
     assert L.imm_sumcheck_matmul_launches(None, 1) == 0
     monkeypatch.setenv("IMM_CONTRACT", "alu")

@@ -728,20 +728,33 @@ topk_sub_kernel(const float* __restrict__ ref, int64_t steps, int n, int64_t ld,
         }
 #pragma unroll
     for (int j = 0; j < SUB_SLOTS; j++) if ((mine >> j) & 1u) v[j] = NEG_INF;
-    for (int r = 0; r < K; r++) {
-        float best = NEG_INF;
-        int slot = 0;
+    // every lane sorts its sixteen entries once (bitonic network in registers, descending); a round then
+    // compares the lanes' heads only, and the winner moves its list up by one
 #pragma unroll
-        for (int j = 0; j < SUB_SLOTS; j++) if (v[j] > best) { best = v[j]; slot = j; }
-        float top = best;
+    for (int k = 2; k <= SUB_SLOTS; k <<= 1)
+#pragma unroll
+        for (int j = k >> 1; j > 0; j >>= 1)
+#pragma unroll
+            for (int i = 0; i < SUB_SLOTS; i++) {
+                const int l = i ^ j;
+                if (l > i) {
+                    const float hi = fmaxf(v[i], v[l]), lo = fminf(v[i], v[l]);
+                    const bool desc = (i & k) == 0;
+                    v[i] = desc ? hi : lo;
+                    v[l] = desc ? lo : hi;
+                }
+            }
+    for (int r = 0; r < K; r++) {
+        float top = v[0];
 #pragma unroll
         for (int o = LPR / 2; o > 0; o >>= 1) top = fmaxf(top, __shfl_xor_sync(0xFFFFFFFFu, top, o));
-        const unsigned holders = __ballot_sync(0xFFFFFFFFu, best == top) & gmask;
+        const unsigned holders = __ballot_sync(0xFFFFFFFFu, v[0] == top) & gmask;
         const int winner = __ffs(holders) - 1;             // lowest lane of the row holding its maximum
         if (lane == winner) {
             outside[w][g][r] = (double)top;                // (-inf once fewer than K entries are left outside I)
 #pragma unroll
-            for (int j = 0; j < SUB_SLOTS; j++) if (j == slot) v[j] = NEG_INF;
+            for (int j = 0; j + 1 < SUB_SLOTS; j++) v[j] = v[j + 1];
+            v[SUB_SLOTS - 1] = NEG_INF;
         }
     }
     __syncwarp();

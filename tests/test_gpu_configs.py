@@ -120,6 +120,28 @@ def test_attention_products_many_small_proofs(imm, oracle, synth):
         assert imm.sumcheck_verify(t, oracle.ceil_log2(p.mkn[1]), SEED, p.proof_id) == (imm.OK, -1)
 
 
+def test_narrow_left_factors_share_rows_among_warps(imm, oracle):
+    """Left factors with fewer columns than the 1024 a block covers (an attention head's Q has 128): the
+    warps without columns take rows instead and their partial sums are merged.  Widths of one, two,
+    three and five warps, ragged last columns, tiles of several and of one group of 32 rows, rows that
+    do not fill the last group; every transcript against the oracle."""
+    from collections import namedtuple
+    P = namedtuple("P", "A B C proof_id mkn")
+    rng = np.random.default_rng(77)
+    probs = []
+    for pid, (m, k, n) in enumerate([(2048, 128, 2048), (1500, 64, 700), (1100, 200, 300), (3000, 384, 128),
+                                     (2500, 520, 64), (33, 100, 40), (31, 129, 17), (1024, 1, 5)]):
+        A = rng.integers(-128, 128, size=(m, k), dtype=np.int64).astype(np.int8)
+        B = rng.integers(-128, 128, size=(k, n), dtype=np.int64).astype(np.int8)
+        C = (A.astype(np.int64) @ B.astype(np.int64)).astype(np.int32)
+        probs.append(P(torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda(), torch.from_numpy(C).cuda(), 900 + pid, (m, k, n)))
+    got = gpu_transcripts(imm, probs, SEED)
+    assert got == oracle_transcripts(oracle, probs, SEED)
+    # and one at a time (other tile heights: the partition follows the batch)
+    for p in probs[:4]:
+        assert gpu_transcripts(imm, [p], SEED + 1) == oracle_transcripts(oracle, [p], SEED + 1)
+
+
 def two_sided(oracle, M, r_row, r_col):
     return oracle.mle_eval_point(M, oracle.eq_table(r_row), oracle.eq_table(r_col))
 
